@@ -1,0 +1,345 @@
+/*
+ * CPU oracle for the sparse paged decode-attention step.
+ *
+ * THIS IS TEST INFRASTRUCTURE, NOT THE PRODUCT.  It is a plain, slow, readable
+ * restatement of what the decode step computes, used only by the tests, by the
+ * smoke check and by the benchmark's CPU-baseline leg.  It shares no code with
+ * the CUDA library and includes none of its headers.
+ *
+ * What each routine follows (sections / equations of the paper):
+ *   orc_build_summaries  Sec. 7 step 1 "coarse page summaries k_page"; the paper does
+ *                        not define them - here: mean of the page's valid key rows.
+ *   orc_route            Sec. 7 step 1 (page routing: score summaries, select P pages).
+ *   orc_sparse           Sec. 7 steps 2-4 (token routing to K_c candidates, weights on the
+ *                        candidates, gather of values).  The weights are the entropic
+ *                        problem of Eq. (5.1) with its quadratic term linearised, i.e. the
+ *                        softmax at temperature epsilon restricted to the candidates.
+ *                        Diagnostics: Def. 1 (face gap) evaluated with r -> q and
+ *                        I -> candidate set; Sec. 8 gap statistic s(1) - s(2); Cor. 1
+ *                        leakage bound with c = 1; Sec. 10.3 fallback-to-dense policy.
+ *   orc_dense            the plain definition: softmax(<q,k_t>/epsilon) over every token.
+ * (The theory objects on tiny dictionaries - Euclidean projection, exact gap, the full
+ *  entropic minimiser of Eq. (5.1) - live in theory.py next to this file.)
+ *
+ * Precision: everything that decides an integer (which pages, which tokens, which units
+ * fall back) is computed in fp32 in ONE fixed summation order (orc_canon_dot) because the
+ * GPU must reproduce those decisions bit for bit.  Everything else is fp64.
+ *
+ * Parity status: orc_dense, orc_canon_dot, the selections, the candidate softmax, the
+ * leakage identities and the entropic solvers are pinned by the CPU tests.  The choice of
+ * "mean key" as the summary, per-query-head routing and the value of the fallback threshold
+ * are readings of a silent paper: parity unpinned for those three choices.
+ *
+ * Build: gcc -O2 -fopenmp -ffp-contract=off -shared -fPIC (no -ffast-math).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+typedef struct {
+    int32_t batch, n_q_heads, n_kv_heads, head_dim, page_size, max_pages_per_seq;
+    int64_t num_pool_pages;
+    int64_t kv_page_stride, kv_head_stride, kv_token_stride; /* in elements */
+} orc_shape;
+
+enum { ORC_D = 128 };
+
+int orc_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+void orc_set_num_threads(int n)
+{
+#ifdef _OPENMP
+    if (n > 0) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
+/* ---- bf16 <-> fp32 ------------------------------------------------------- */
+
+float orc_bf16_to_f32(uint16_t h)
+{
+    uint32_t u = (uint32_t)h << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+/* round to nearest, ties to even; NaN stays NaN */
+uint16_t orc_f32_to_bf16(float f)
+{
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x0040u);
+    uint32_t lsb = (u >> 16) & 1u;
+    u += 0x7fffu + lsb;
+    return (uint16_t)(u >> 16);
+}
+
+/* ---- the one fp32 summation order every discrete decision depends on ------
+ * 128 products in 16 chunks of 8 consecutive elements.  Chunk partial: left to right.
+ * Then a halving tree over the 16 partials: p[c] += p[c+off], off = 8, 4, 2, 1.
+ * A product of two bf16 numbers is exact in fp32, so it does not matter whether a
+ * machine fuses the multiply into the add. */
+float orc_canon_dot(const uint16_t *x, const uint16_t *y)
+{
+    float p[16];
+    for (int c = 0; c < 16; ++c) {
+        float acc = orc_bf16_to_f32(x[8 * c]) * orc_bf16_to_f32(y[8 * c]);
+        for (int e = 1; e < 8; ++e) {
+            float prod = orc_bf16_to_f32(x[8 * c + e]) * orc_bf16_to_f32(y[8 * c + e]);
+            acc = acc + prod;
+        }
+        p[c] = acc;
+    }
+    for (int off = 8; off >= 1; off >>= 1)
+        for (int c = 0; c < off; ++c) p[c] = p[c] + p[c + off];
+    return p[0];
+}
+
+static double dot64(const uint16_t *x, const uint16_t *y)
+{
+    double s = 0.0;
+    for (int e = 0; e < ORC_D; ++e) s += (double)orc_bf16_to_f32(x[e]) * (double)orc_bf16_to_f32(y[e]);
+    return s;
+}
+
+static int shape_ok(const orc_shape *s)
+{
+    return s && s->head_dim == ORC_D && s->page_size > 0 && s->batch > 0 && s->n_kv_heads > 0 &&
+           s->n_q_heads > 0 && s->n_q_heads % s->n_kv_heads == 0 && s->max_pages_per_seq > 0;
+}
+
+static const uint16_t *kv_row(const orc_shape *s, const uint16_t *pool, int64_t page, int g, int t)
+{
+    return pool + page * s->kv_page_stride + (int64_t)g * s->kv_head_stride + (int64_t)t * s->kv_token_stride;
+}
+
+static int n_pages_of(const orc_shape *s, int T) { return (T + s->page_size - 1) / s->page_size; }
+
+/* ---- step 1a: page summaries ---------------------------------------------
+ * k_page[p, g, :] = bf16( (sum over the page's valid rows, fp32, ascending token) / n ). */
+int orc_build_summaries(const orc_shape *s, const uint16_t *K, const int32_t *bt, const int32_t *seq_lens,
+                        const int32_t *first_page, uint16_t *summaries)
+{
+    if (!shape_ok(s)) return -1;
+    for (int b = 0; b < s->batch; ++b) {
+        int T = seq_lens[b];
+        int nb = n_pages_of(s, T);
+        int l0 = first_page ? first_page[b] : 0;
+        for (int l = l0; l < nb; ++l) {
+            int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
+            int n = T - l * s->page_size;
+            if (n > s->page_size) n = s->page_size;
+            for (int g = 0; g < s->n_kv_heads; ++g) {
+                uint16_t *dst = summaries + (p * s->n_kv_heads + g) * ORC_D;
+                for (int e = 0; e < ORC_D; ++e) {
+                    float acc = 0.0f;
+                    for (int t = 0; t < n; ++t) acc = acc + orc_bf16_to_f32(kv_row(s, K, p, g, t)[e]);
+                    dst[e] = orc_f32_to_bf16(acc / (float)n);
+                }
+            }
+        }
+    }
+    return 0;
+}
+
+/* ---- ordering used by both selections: score descending, index ascending --- */
+typedef struct {
+    float s;
+    int32_t idx;
+} scored;
+
+static int cmp_scored(const void *a, const void *b)
+{
+    const scored *x = (const scored *)a, *y = (const scored *)b;
+    if (x->s > y->s) return -1; /* -0.0f and +0.0f compare equal here */
+    if (x->s < y->s) return 1;
+    return (x->idx > y->idx) - (x->idx < y->idx);
+}
+
+/* ---- step 1b: page routing -------------------------------------------------
+ * c_l = canon_dot(q[b,h], k_page[bt[b][l], g]); routed = first min(P, n_b) pages in the
+ * order above.  routed_pages is [B][Hq][P] padded with -1, listed in that order. */
+int orc_route(const orc_shape *s, const uint16_t *q, const uint16_t *summaries, const int32_t *bt,
+              const int32_t *seq_lens, int P, int32_t *routed_pages, float *routed_scores, float *all_scores)
+{
+    if (!shape_ok(s) || P < 1) return -1;
+    const int G = s->n_q_heads / s->n_kv_heads;
+    const int units = s->batch * s->n_q_heads;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int u = 0; u < units; ++u) {
+        int b = u / s->n_q_heads, h = u % s->n_q_heads, g = h / G;
+        int nb = n_pages_of(s, seq_lens[b]);
+        scored *c = (scored *)malloc(sizeof(scored) * (size_t)(nb > 0 ? nb : 1));
+        const uint16_t *qv = q + (int64_t)u * ORC_D;
+        for (int l = 0; l < nb; ++l) {
+            int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
+            c[l].s = orc_canon_dot(qv, summaries + (p * s->n_kv_heads + g) * ORC_D);
+            c[l].idx = l;
+            if (all_scores) all_scores[(int64_t)u * s->max_pages_per_seq + l] = c[l].s;
+        }
+        qsort(c, (size_t)nb, sizeof(scored), cmp_scored);
+        int keep = nb < P ? nb : P;
+        for (int i = 0; i < P; ++i) {
+            routed_pages[(int64_t)u * P + i] = i < keep ? c[i].idx : -1;
+            if (routed_scores) routed_scores[(int64_t)u * P + i] = i < keep ? c[i].s : -INFINITY;
+        }
+        free(c);
+    }
+    return 0;
+}
+
+/* ---- steps 2-4 + diagnostics ------------------------------------------------ */
+int orc_sparse(const orc_shape *s, const uint16_t *q, const uint16_t *K, const uint16_t *V, const int32_t *bt,
+               const int32_t *seq_lens, const int32_t *routed_pages, int P, int K_c, float epsilon,
+               float gap_threshold, double *out, float *delta, float *delta12, float *s_max, double *lse,
+               double *leak_bound, int32_t *n_candidates, int32_t *fallback, int32_t *cand_pos,
+               double *cand_weight)
+{
+    if (!shape_ok(s) || P < 1 || K_c < 1 || !(epsilon > 0.0f)) return -1;
+    const int G = s->n_q_heads / s->n_kv_heads;
+    const int units = s->batch * s->n_q_heads;
+    const double eps = (double)epsilon;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int u = 0; u < units; ++u) {
+        int b = u / s->n_q_heads, h = u % s->n_q_heads, g = h / G;
+        int T = seq_lens[b];
+        const uint16_t *qv = q + (int64_t)u * ORC_D;
+        scored *c = (scored *)malloc(sizeof(scored) * (size_t)P * (size_t)s->page_size);
+        int nv = 0;
+        /* token routing: exact fp32 score of every valid token of every routed page */
+        for (int i = 0; i < P; ++i) {
+            int l = routed_pages[(int64_t)u * P + i];
+            if (l < 0) continue;
+            int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
+            for (int t = 0; t < s->page_size; ++t) {
+                int pos = l * s->page_size + t;
+                if (pos >= T) break;
+                c[nv].s = orc_canon_dot(qv, kv_row(s, K, p, g, t));
+                c[nv].idx = pos;
+                ++nv;
+            }
+        }
+        qsort(c, (size_t)nv, sizeof(scored), cmp_scored);
+        int ns = nv < K_c ? nv : K_c; /* |S| */
+
+        /* candidate softmax times V, fp64 */
+        double *s64 = (double *)malloc(sizeof(double) * (size_t)(ns > 0 ? ns : 1));
+        double m = -INFINITY;
+        for (int i = 0; i < ns; ++i) {
+            int pos = c[i].idx, l = pos / s->page_size, t = pos % s->page_size;
+            int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
+            s64[i] = dot64(qv, kv_row(s, K, p, g, t));
+            if (s64[i] > m) m = s64[i];
+        }
+        double Z = 0.0, acc[ORC_D];
+        for (int e = 0; e < ORC_D; ++e) acc[e] = 0.0;
+        for (int i = 0; i < ns; ++i) {
+            int pos = c[i].idx, l = pos / s->page_size, t = pos % s->page_size;
+            int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
+            const uint16_t *vr = kv_row(s, V, p, g, t);
+            double w = exp((s64[i] - m) / eps);
+            Z += w;
+            for (int e = 0; e < ORC_D; ++e) acc[e] += w * (double)orc_bf16_to_f32(vr[e]);
+            if (cand_weight) cand_weight[(int64_t)u * K_c + i] = w;
+        }
+        for (int e = 0; e < ORC_D; ++e) out[(int64_t)u * ORC_D + e] = ns > 0 ? acc[e] / Z : 0.0;
+        if (cand_weight)
+            for (int i = 0; i < K_c; ++i)
+                cand_weight[(int64_t)u * K_c + i] = i < ns ? cand_weight[(int64_t)u * K_c + i] / Z : 0.0;
+        if (cand_pos)
+            for (int i = 0; i < K_c; ++i) cand_pos[(int64_t)u * K_c + i] = i < ns ? c[i].idx : -1;
+        lse[u] = ns > 0 ? m / eps + log(Z) : -INFINITY;
+
+        /* diagnostics, fp32 differences of canonical scores */
+        float s1 = ns > 0 ? c[0].s : -INFINITY;
+        float s2 = ns > 1 ? c[1].s : -INFINITY;
+        float d = nv > ns ? s1 - c[ns].s : INFINITY; /* best rejected scored token */
+        float d12 = s1 - s2;
+        s_max[u] = s1;
+        delta[u] = d;
+        delta12[u] = d12;
+        n_candidates[u] = ns;
+        double lb = (double)(T - ns) * exp(-(double)d / eps);
+        leak_bound[u] = lb < 1.0 ? lb : 1.0;
+        fallback[u] = (d < gap_threshold && ns < T) ? 1 : 0;
+        free(s64);
+        free(c);
+    }
+    return 0;
+}
+
+/* ---- the plain definition: dense softmax attention over every token, fp64 ----
+ * Optional extras for one candidate set per unit (cand_pos, -1 padded, K_c wide):
+ *   true_leak  = dense softmax mass outside the candidate set,
+ *   true_gap   = max_t s_t - max_{j not in S} s_j  (fp64 scores),
+ *   y_off      = dense readout renormalised over the complement of S. */
+int orc_dense(const orc_shape *s, const uint16_t *q, const uint16_t *K, const uint16_t *V, const int32_t *bt,
+              const int32_t *seq_lens, float epsilon, const int32_t *unit_mask, double *out, double *lse,
+              const int32_t *cand_pos, int K_c, double *true_leak, double *true_gap, double *y_off)
+{
+    if (!shape_ok(s) || !(epsilon > 0.0f)) return -1;
+    const int G = s->n_q_heads / s->n_kv_heads;
+    const int units = s->batch * s->n_q_heads;
+    const double eps = (double)epsilon;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int u = 0; u < units; ++u) {
+        if (unit_mask && !unit_mask[u]) continue;
+        int b = u / s->n_q_heads, h = u % s->n_q_heads, g = h / G;
+        int T = seq_lens[b];
+        const uint16_t *qv = q + (int64_t)u * ORC_D;
+        double *sc = (double *)malloc(sizeof(double) * (size_t)T);
+        unsigned char *inS = (unsigned char *)calloc((size_t)T, 1);
+        if (cand_pos)
+            for (int i = 0; i < K_c; ++i) {
+                int pos = cand_pos[(int64_t)u * K_c + i];
+                if (pos >= 0 && pos < T) inS[pos] = 1;
+            }
+        double m = -INFINITY, m_off = -INFINITY;
+        for (int pos = 0; pos < T; ++pos) {
+            int l = pos / s->page_size, t = pos % s->page_size;
+            int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
+            sc[pos] = dot64(qv, kv_row(s, K, p, g, t));
+            if (sc[pos] > m) m = sc[pos];
+            if (!inS[pos] && sc[pos] > m_off) m_off = sc[pos];
+        }
+        double Z = 0.0, Zoff = 0.0, acc[ORC_D], accoff[ORC_D];
+        for (int e = 0; e < ORC_D; ++e) acc[e] = accoff[e] = 0.0;
+        for (int pos = 0; pos < T; ++pos) {
+            int l = pos / s->page_size, t = pos % s->page_size;
+            int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
+            const uint16_t *vr = kv_row(s, V, p, g, t);
+            double w = exp((sc[pos] - m) / eps);
+            Z += w;
+            for (int e = 0; e < ORC_D; ++e) acc[e] += w * (double)orc_bf16_to_f32(vr[e]);
+            if (cand_pos && !inS[pos]) {
+                Zoff += w;
+                for (int e = 0; e < ORC_D; ++e) accoff[e] += w * (double)orc_bf16_to_f32(vr[e]);
+            }
+        }
+        for (int e = 0; e < ORC_D; ++e) out[(int64_t)u * ORC_D + e] = acc[e] / Z;
+        lse[u] = m / eps + log(Z);
+        if (cand_pos) {
+            if (true_leak) true_leak[u] = Zoff / Z;
+            if (true_gap) true_gap[u] = m - m_off; /* +inf when nothing lies outside S */
+            if (y_off)
+                for (int e = 0; e < ORC_D; ++e)
+                    y_off[(int64_t)u * ORC_D + e] = Zoff > 0.0 ? accoff[e] / Zoff : 0.0;
+        }
+        free(inS);
+        free(sc);
+    }
+    return 0;
+}
