@@ -1,0 +1,187 @@
+/*
+ * vsa.h - C ABI of the sparse paged decode-attention step for NVIDIA B200 (sm_100a).
+ *
+ * One decode step, per (sequence b, query head h) "unit", over a paged bf16 KV cache
+ * (paper Sec. 7, "Paged KV and routing", steps 1-4, and Sec. 10.3 fallback policy):
+ *
+ *   1. page routing   score one summary vector per page, keep the P best pages
+ *   2. token routing  score every token of those pages, keep the K_c best tokens
+ *   3. weights        entropic (softmax, temperature epsilon) weights on the K_c candidates
+ *   4. fused gather   out = sum_k alpha_k V[page_k, off_k], no candidate list in memory
+ *   +  diagnostic     support-gap proxy Delta and the leakage bound exp(-Delta/epsilon)
+ *   +  fallback       dense attention for every unit whose gap is below a threshold
+ *
+ * Conventions for every entry point
+ *   - "device" pointers are CUDA device memory of the current device; "host" pointers are
+ *     ordinary (preferably pinned) host memory.  The library never allocates, frees or keeps
+ *     any of them.  All buffers are owned by the caller.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls
+ *     only enqueue work on that stream and return; they never synchronise.
+ *   - Return value: 0 on success, a negative VSA_ERR_* code otherwise.  Errors are detected
+ *     on the host before anything is launched, so a failed call leaves all buffers untouched.
+ *   - Data-dependent anomalies (a block-table entry outside the pool, a sequence longer
+ *     than its block-table row, a non-positive length) never trap: the unit's
+ *     diag.status becomes non-zero and its output row is zero-filled.
+ *   - Inputs are assumed finite (no NaN/Inf in q, K, V).
+ *   - v1 shapes: head_dim = 128, page_size = 16, n_q_heads / n_kv_heads in {1, 2, 4, 8},
+ *     1 <= P <= 128, 1 <= K_c <= P * page_size, max_pages_per_seq <= 32768.
+ *
+ * Native layouts (row-major, last dimension contiguous)
+ *   q            bf16 [batch][n_q_heads][head_dim]
+ *   k/v cache    bf16 [num_pool_pages][n_kv_heads][page_size][head_dim]  (strides in shape)
+ *   summaries    bf16 [num_pool_pages][n_kv_heads][head_dim]
+ *   block_table  int32 [batch][max_pages_per_seq]   logical page -> physical page
+ *   seq_lens     int32 [batch]                      tokens in each sequence (T_b)
+ *   out          fp32 [batch][n_q_heads][head_dim]
+ * Query head h reads KV head h / (n_q_heads / n_kv_heads).  A unit id is b * n_q_heads + h.
+ *
+ * Arithmetic contract
+ *   Every score that feeds a selection (page scores, token scores) is an fp32 dot product in
+ *   one fixed order: 16 chunks of 8 consecutive elements summed left to right, then the 16
+ *   partials combined by a halving tree (p[c] += p[c+off], off = 8, 4, 2, 1).  Selections
+ *   order by (score descending, index ascending), -0 and +0 being equal.  Routed pages,
+ *   candidate sets, Delta and the fallback flags are therefore reproducible bit for bit.
+ *   Softmax weights and outputs use fp32 accumulation.
+ */
+#ifndef VSA_H_
+#define VSA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define VSA_OK 0
+#define VSA_ERR_INVALID_ARGUMENT (-1)  /* NULL pointer, size <= 0, bad epsilon/threshold, P/K_c < 1 */
+#define VSA_ERR_UNSUPPORTED_SHAPE (-2) /* outside the v1 shapes listed above                          */
+#define VSA_ERR_WORKSPACE_TOO_SMALL (-3)
+#define VSA_ERR_MISALIGNED (-4)        /* a pointer or stride is not 16-byte aligned                  */
+#define VSA_ERR_CUDA (-5)              /* a launch or copy was rejected by the CUDA runtime           */
+
+typedef struct {
+    int32_t batch, n_q_heads, n_kv_heads, head_dim, page_size;
+    int32_t max_pages_per_seq; /* row stride of block_table                                 */
+    int64_t num_pool_pages;    /* physical pages in the K/V pools and in `summaries`        */
+    int64_t kv_page_stride, kv_head_stride, kv_token_stride; /* elements; 0 = native layout */
+} vsa_shape_t;
+
+/* Per-unit diagnostics (paper Sec. 8 and Cor. 1; Def. 1 evaluated with r -> q, I -> candidates). */
+typedef struct {
+    float delta;          /* s(1) - best rejected scored token; +INF if nothing was rejected */
+    float delta12;        /* s(1) - s(2), the paper's gap statistic; +INF with one candidate  */
+    float s_max;          /* s(1), raw <q, k> of the best candidate                           */
+    float lse;            /* log sum exp(s / epsilon) over the tokens that produced `out`     */
+    float leak_bound;     /* min(1, (T_b - |S|) * exp(-delta / epsilon))                      */
+    int32_t n_candidates; /* |S| = min(K_c, valid tokens in the routed pages)                 */
+    int32_t fallback;     /* 1 if delta < gap_threshold (unit is in the fallback list)        */
+    int32_t status;       /* 0 = ok, else VSA_UNIT_*                                          */
+} vsa_diag_t;
+
+#define VSA_UNIT_BAD_PAGE 1   /* a needed block-table entry is outside [0, num_pool_pages) */
+#define VSA_UNIT_BAD_LENGTH 2 /* seq_len <= 0 or > max_pages_per_seq * page_size           */
+
+/* which_call values of vsa_workspace_bytes */
+#define VSA_WS_ROUTE 1
+#define VSA_WS_SPARSE 2
+#define VSA_WS_DENSE 3
+#define VSA_WS_STEP 4
+
+/*
+ * Page summaries (Sec. 7 step 1: "coarse page summaries k_page"; the paper leaves them
+ * undefined - here the mean of the page's valid key rows, per KV head).
+ * For every sequence b and logical page l in [first_page[b], ceil(T_b / page_size)):
+ *   summaries[block_table[b][l]][g][:] = bf16_rne( (sum_t K[page][g][t][:]) / n ),
+ * fp32 sum over the n valid rows in ascending t.  Pages outside that range are not touched.
+ *   k_cache, block_table, seq_lens, summaries: device.  first_page: device [batch] or NULL (= 0).
+ */
+int vsa_build_page_summaries(const vsa_shape_t* shape, const void* k_cache, const int32_t* block_table,
+                             const int32_t* seq_lens, const int32_t* first_page, void* summaries,
+                             void* stream);
+
+/*
+ * Page routing (Sec. 7 step 1).  For every unit: c_l = <q[b][h], summaries[block_table[b][l]][g]>
+ * for l < n_b = ceil(T_b / page_size); routed_pages[b][h][0..P) = the min(P, n_b) best logical
+ * pages, best first, padded with -1.  routed_scores (optional, may be NULL) receives the scores
+ * in the same order, padded with -INF.
+ *   All pointers device.  ws: device scratch of vsa_workspace_bytes(shape, P, 0, VSA_WS_ROUTE)
+ *   bytes, 16-byte aligned; contents undefined before and after the call.
+ */
+int vsa_route_pages(const vsa_shape_t* shape, const void* q, const void* summaries,
+                    const int32_t* block_table, const int32_t* seq_lens, int32_t P,
+                    int32_t* routed_pages, float* routed_scores, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Token routing + candidate softmax x V + diagnostics (Sec. 7 steps 2-4, Sec. 8, Cor. 1),
+ * one fused pass per unit.  Scores every valid token of the unit's routed pages, keeps
+ * S = the min(K_c, #valid) best, writes
+ *   out[b][h][:] = sum_{i in S} alpha_i V_i,  alpha = softmax over S of <q, k_i> / epsilon,
+ * and diag[b][h].  Units with diag.delta < gap_threshold (strict) are appended to
+ * fallback_list (unit ids, arbitrary order) and counted in *fallback_count, which this call
+ * resets to 0 on the stream first.  gap_threshold = -INF never flags (the "cap-compute"
+ * policy of Sec. 10.3); +INF flags every unit that rejected at least one token.
+ *   routed_pages: device int32 [batch][n_q_heads][P], distinct logical pages or -1.
+ *   fallback_list: device int32 [batch * n_q_heads]; fallback_count: device int32 [1].
+ *   ws may be NULL (this call needs no scratch).  All pointers device.
+ */
+int vsa_sparse_decode(const vsa_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,
+                      const int32_t* block_table, const int32_t* seq_lens, const int32_t* routed_pages,
+                      int32_t P, int32_t K_c, float epsilon, float gap_threshold, float* out,
+                      vsa_diag_t* diag, int32_t* fallback_list, int32_t* fallback_count, void* ws,
+                      size_t ws_bytes, void* stream);
+
+/*
+ * Dense fallback (Sec. 10.3 "fallback-to-dense"): for every unit in fallback_list[0 ..
+ * *fallback_count) recompute out[b][h][:] = softmax(<q, k_t> / epsilon over all T_b tokens) V
+ * with a split-K pass (K and V of a KV head are read once for all listed heads of its
+ * group), overwrite out and diag.lse, and leave every other unit untouched.
+ * fallback_count == NULL (then fallback_list is ignored) means every unit: this is the dense
+ * decode baseline.  The count is read on the device; nothing synchronises with the host.
+ *   diag may be NULL.  ws: device scratch of vsa_workspace_bytes(shape, 0, 0, VSA_WS_DENSE) bytes.
+ */
+int vsa_dense_decode_fallback(const vsa_shape_t* shape, const void* q, const void* k_cache,
+                              const void* v_cache, const int32_t* block_table, const int32_t* seq_lens,
+                              const int32_t* fallback_list, const int32_t* fallback_count, float epsilon,
+                              float* out, vsa_diag_t* diag, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * The whole step on one stream: vsa_route_pages -> vsa_sparse_decode ->
+ * vsa_dense_decode_fallback, same results as the three calls made one after the other.
+ *   routed_pages, diag, fallback_list, fallback_count: device outputs as above.
+ *   ws: device scratch of vsa_workspace_bytes(shape, P, K_c, VSA_WS_STEP) bytes.
+ */
+int vsa_decode_step(const vsa_shape_t* shape, const void* q, const void* summaries, const void* k_cache,
+                    const void* v_cache, const int32_t* block_table, const int32_t* seq_lens, int32_t P,
+                    int32_t K_c, float epsilon, float gap_threshold, float* out, vsa_diag_t* diag,
+                    int32_t* routed_pages, int32_t* fallback_list, int32_t* fallback_count, void* ws,
+                    size_t ws_bytes, void* stream);
+
+/*
+ * The same step for a caller whose per-step tensors live in host memory: copies q_host
+ * (bf16 [batch][n_q_heads][head_dim]) to q_dev, runs vsa_decode_step, and copies the results
+ * back into out_host (fp32 [batch][n_q_heads][head_dim]) and diag_host ([batch][n_q_heads],
+ * may be NULL).  The KV cache, summaries, block table and lengths stay device-resident: they
+ * are the decode state, not per-step inputs.  Copies are asynchronous on `stream`; the host
+ * buffers must stay valid until the stream has been synchronised by the caller.
+ *   q_host, out_host, diag_host: host (pinned for real asynchrony).
+ *   q_dev, out_dev, diag_dev, routed_pages, fallback_list, fallback_count, ws: device staging
+ *   and scratch buffers of the sizes given for vsa_decode_step.
+ */
+int vsa_decode_step_host(const vsa_shape_t* shape, const void* q_host, void* q_dev, const void* summaries,
+                         const void* k_cache, const void* v_cache, const int32_t* block_table,
+                         const int32_t* seq_lens, int32_t P, int32_t K_c, float epsilon,
+                         float gap_threshold, float* out_host, float* out_dev, vsa_diag_t* diag_host,
+                         vsa_diag_t* diag_dev, int32_t* routed_pages, int32_t* fallback_list,
+                         int32_t* fallback_count, void* ws, size_t ws_bytes, void* stream);
+
+/* Scratch bytes needed by one call kind for this shape (0 if the shape is invalid). */
+size_t vsa_workspace_bytes(const vsa_shape_t* shape, int32_t P, int32_t K_c, int which_call);
+
+/* Static, human-readable text for a return code. */
+const char* vsa_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VSA_H_ */

@@ -267,7 +267,7 @@ int orc_sparse(const orc_shape *s, const uint16_t *q, const uint16_t *K, const u
         float s1 = ns > 0 ? c[0].s : -INFINITY;
         float s2 = ns > 1 ? c[1].s : -INFINITY;
         float d = nv > ns ? s1 - c[ns].s : INFINITY; /* best rejected scored token */
-        float d12 = s1 - s2;
+        float d12 = ns > 0 ? s1 - s2 : INFINITY;
         s_max[u] = s1;
         delta[u] = d;
         delta12[u] = d12;

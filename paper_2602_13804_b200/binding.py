@@ -1,0 +1,190 @@
+"""ctypes binding of libvsa.so: argument marshalling only.
+
+Every function has the name and argument order of its C entry point (include/vsa.h) and takes
+torch tensors where C takes pointers.  Tensors are used for their device memory and nothing
+else: no step of the decode path runs in PyTorch.  The library must be present - there is no
+fallback; a missing or unloadable libvsa.so raises at import of this module's ``lib()``.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libvsa.so")
+
+VSA_WS_ROUTE, VSA_WS_SPARSE, VSA_WS_DENSE, VSA_WS_STEP = 1, 2, 3, 4
+DIAG_BYTES = 32
+DIAG_FIELDS = ("delta", "delta12", "s_max", "lse", "leak_bound", "n_candidates", "fallback", "status")
+
+
+class VsaError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where} failed: {lib().vsa_strerror(code).decode()} ({code})")
+
+
+class vsa_shape_t(C.Structure):
+    _fields_ = [
+        ("batch", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+        ("head_dim", C.c_int32), ("page_size", C.c_int32), ("max_pages_per_seq", C.c_int32),
+        ("num_pool_pages", C.c_int64),
+        ("kv_page_stride", C.c_int64), ("kv_head_stride", C.c_int64), ("kv_token_stride", C.c_int64),
+    ]
+
+
+class vsa_diag_t(C.Structure):
+    _fields_ = [
+        ("delta", C.c_float), ("delta12", C.c_float), ("s_max", C.c_float), ("lse", C.c_float),
+        ("leak_bound", C.c_float), ("n_candidates", C.c_int32), ("fallback", C.c_int32), ("status", C.c_int32),
+    ]
+
+
+assert C.sizeof(vsa_diag_t) == DIAG_BYTES
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """The loaded C-ABI library.  Raises if it has not been built (python -m paper_2602_13804_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2602_13804_b200.build`; "
+                               "there is no fallback path")
+        _lib = C.CDLL(LIB_PATH)
+        vp, i32, f32, sz = C.c_void_p, C.c_int32, C.c_float, C.c_size_t
+        shp = C.POINTER(vsa_shape_t)
+        _lib.vsa_strerror.restype = C.c_char_p
+        _lib.vsa_strerror.argtypes = [C.c_int]
+        _lib.vsa_workspace_bytes.restype = sz
+        _lib.vsa_workspace_bytes.argtypes = [shp, i32, i32, C.c_int]
+        _lib.vsa_build_page_summaries.argtypes = [shp, vp, vp, vp, vp, vp, vp]
+        _lib.vsa_route_pages.argtypes = [shp, vp, vp, vp, vp, i32, vp, vp, vp, sz, vp]
+        _lib.vsa_sparse_decode.argtypes = [shp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, vp, vp, vp, vp, vp, sz, vp]
+        _lib.vsa_dense_decode_fallback.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, f32, vp, vp, vp, sz, vp]
+        _lib.vsa_decode_step.argtypes = [shp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, vp, vp, vp, vp, vp, vp, sz, vp]
+        _lib.vsa_decode_step_host.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32,
+                                              vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        for name in ("vsa_build_page_summaries", "vsa_route_pages", "vsa_sparse_decode",
+                     "vsa_dense_decode_fallback", "vsa_decode_step", "vsa_decode_step_host"):
+            getattr(_lib, name).restype = C.c_int
+    return _lib
+
+
+def make_shape(batch: int, n_q_heads: int, n_kv_heads: int, max_pages_per_seq: int, num_pool_pages: int,
+               head_dim: int = 128, page_size: int = 16, kv_page_stride: int = 0, kv_head_stride: int = 0,
+               kv_token_stride: int = 0) -> vsa_shape_t:
+    return vsa_shape_t(batch, n_q_heads, n_kv_heads, head_dim, page_size, max_pages_per_seq, num_pool_pages,
+                       kv_page_stride, kv_head_stride, kv_token_stride)
+
+
+def shape_of(q: torch.Tensor, k_cache: torch.Tensor, block_table: torch.Tensor) -> vsa_shape_t:
+    """Shape struct for q [B, Hq, d], k_cache [pool, Hkv, page, d] (any strides), block_table [B, max_pages]."""
+    assert k_cache.stride(3) == 1, "head dimension must be contiguous"
+    return make_shape(q.shape[0], q.shape[1], k_cache.shape[1], block_table.shape[1], k_cache.shape[0],
+                      head_dim=q.shape[2], page_size=k_cache.shape[2], kv_page_stride=k_cache.stride(0),
+                      kv_head_stride=k_cache.stride(1), kv_token_stride=k_cache.stride(2))
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    if isinstance(stream, int):
+        return stream or None
+    return stream.cuda_stream or None
+
+
+def _check(rc: int, where: str) -> None:
+    if rc != 0:
+        raise VsaError(rc, where)
+
+
+def vsa_strerror(code: int) -> str:
+    return lib().vsa_strerror(code).decode()
+
+
+def vsa_workspace_bytes(shape: vsa_shape_t, P: int, K_c: int, which_call: int) -> int:
+    return int(lib().vsa_workspace_bytes(C.byref(shape), P, K_c, which_call))
+
+
+def vsa_build_page_summaries(shape, k_cache, block_table, seq_lens, first_page, summaries, stream=None) -> None:
+    _check(lib().vsa_build_page_summaries(C.byref(shape), _ptr(k_cache), _ptr(block_table), _ptr(seq_lens),
+                                          _ptr(first_page), _ptr(summaries), _stream(stream)),
+           "vsa_build_page_summaries")
+
+
+def vsa_route_pages(shape, q, summaries, block_table, seq_lens, P, routed_pages, routed_scores, ws,
+                    stream=None) -> None:
+    _check(lib().vsa_route_pages(C.byref(shape), _ptr(q), _ptr(summaries), _ptr(block_table), _ptr(seq_lens), P,
+                                 _ptr(routed_pages), _ptr(routed_scores), _ptr(ws),
+                                 0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
+           "vsa_route_pages")
+
+
+def vsa_sparse_decode(shape, q, k_cache, v_cache, block_table, seq_lens, routed_pages, P, K_c, epsilon,
+                      gap_threshold, out, diag, fallback_list, fallback_count, ws=None, stream=None) -> None:
+    _check(lib().vsa_sparse_decode(C.byref(shape), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(block_table),
+                                   _ptr(seq_lens), _ptr(routed_pages), P, K_c, epsilon, gap_threshold, _ptr(out),
+                                   _ptr(diag), _ptr(fallback_list), _ptr(fallback_count), _ptr(ws),
+                                   0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
+           "vsa_sparse_decode")
+
+
+def vsa_dense_decode_fallback(shape, q, k_cache, v_cache, block_table, seq_lens, fallback_list, fallback_count,
+                              epsilon, out, diag, ws, stream=None) -> None:
+    _check(lib().vsa_dense_decode_fallback(C.byref(shape), _ptr(q), _ptr(k_cache), _ptr(v_cache),
+                                           _ptr(block_table), _ptr(seq_lens), _ptr(fallback_list),
+                                           _ptr(fallback_count), epsilon, _ptr(out), _ptr(diag), _ptr(ws),
+                                           0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
+           "vsa_dense_decode_fallback")
+
+
+def vsa_decode_step(shape, q, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon, gap_threshold,
+                    out, diag, routed_pages, fallback_list, fallback_count, ws, stream=None) -> None:
+    _check(lib().vsa_decode_step(C.byref(shape), _ptr(q), _ptr(summaries), _ptr(k_cache), _ptr(v_cache),
+                                 _ptr(block_table), _ptr(seq_lens), P, K_c, epsilon, gap_threshold, _ptr(out),
+                                 _ptr(diag), _ptr(routed_pages), _ptr(fallback_list), _ptr(fallback_count),
+                                 _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
+           "vsa_decode_step")
+
+
+def vsa_decode_step_host(shape, q_host, q_dev, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c,
+                         epsilon, gap_threshold, out_host, out_dev, diag_host, diag_dev, routed_pages,
+                         fallback_list, fallback_count, ws, stream=None) -> None:
+    _check(lib().vsa_decode_step_host(C.byref(shape), _ptr(q_host), _ptr(q_dev), _ptr(summaries), _ptr(k_cache),
+                                      _ptr(v_cache), _ptr(block_table), _ptr(seq_lens), P, K_c, epsilon,
+                                      gap_threshold, _ptr(out_host), _ptr(out_dev), _ptr(diag_host),
+                                      _ptr(diag_dev), _ptr(routed_pages), _ptr(fallback_list),
+                                      _ptr(fallback_count), _ptr(ws),
+                                      0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
+           "vsa_decode_step_host")
+
+
+# ---- small conveniences for callers (allocation and unpacking only) --------------------------------
+
+def alloc_diag(units: int, device) -> torch.Tensor:
+    """Device buffer for `units` vsa_diag_t records, viewed as int32 [units, 8]."""
+    return torch.zeros((units, DIAG_BYTES // 4), dtype=torch.int32, device=device)
+
+
+def diag_to_dict(diag: torch.Tensor) -> dict:
+    """Unpack a [units, 8] int32 diag buffer into named host tensors."""
+    d = diag.detach().cpu()
+    out = {}
+    for i, name in enumerate(DIAG_FIELDS):
+        col = d[:, i].contiguous()
+        out[name] = col.view(torch.float32).clone() if i < 5 else col.clone()
+    return out
+
+
+def alloc_workspace(shape: vsa_shape_t, P: int, K_c: int, which_call: int, device) -> torch.Tensor:
+    n = vsa_workspace_bytes(shape, P, K_c, which_call)
+    return torch.empty(max(n, 16), dtype=torch.uint8, device=device)

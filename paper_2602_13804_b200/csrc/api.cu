@@ -1,0 +1,241 @@
+// C ABI of libvsa: argument validation (everything is checked on the host before any launch),
+// workspace layout, and the composition of the kernels into the entry points of vsa.h.
+#include <math.h>
+
+#include "vsa_device.cuh"
+#include "vsa_launch.h"
+
+namespace {
+
+using vsa::Geometry;
+
+constexpr int kMaxP = 128;
+constexpr int kMaxPagesPerSeq = 32768;
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// shape checks shared by every entry point; fills the kernel-side geometry
+int make_geometry(const vsa_shape_t* s, Geometry* g)
+{
+    if (!s) return VSA_ERR_INVALID_ARGUMENT;
+    if (s->batch <= 0 || s->n_q_heads <= 0 || s->n_kv_heads <= 0 || s->head_dim <= 0 || s->page_size <= 0 ||
+        s->max_pages_per_seq <= 0 || s->num_pool_pages <= 0)
+        return VSA_ERR_INVALID_ARGUMENT;
+    if (s->n_q_heads % s->n_kv_heads != 0) return VSA_ERR_INVALID_ARGUMENT;
+    if (s->kv_page_stride < 0 || s->kv_head_stride < 0 || s->kv_token_stride < 0) return VSA_ERR_INVALID_ARGUMENT;
+    const int group = s->n_q_heads / s->n_kv_heads;
+    if (s->head_dim != vsa::kHeadDim || s->page_size != vsa::kPageSize) return VSA_ERR_UNSUPPORTED_SHAPE;
+    if (group != 1 && group != 2 && group != 4 && group != 8) return VSA_ERR_UNSUPPORTED_SHAPE;
+    if (s->max_pages_per_seq > kMaxPagesPerSeq) return VSA_ERR_UNSUPPORTED_SHAPE;
+    if (s->num_pool_pages > 0x7fffffffLL) return VSA_ERR_UNSUPPORTED_SHAPE;
+    if ((long long)s->batch * s->n_q_heads > 0x3fffffffLL) return VSA_ERR_UNSUPPORTED_SHAPE;
+    g->batch = s->batch;
+    g->n_q_heads = s->n_q_heads;
+    g->n_kv_heads = s->n_kv_heads;
+    g->group = group;
+    g->max_pages = s->max_pages_per_seq;
+    g->pool_pages = s->num_pool_pages;
+    g->token_stride = s->kv_token_stride ? s->kv_token_stride : s->head_dim;
+    g->head_stride = s->kv_head_stride ? s->kv_head_stride : (long long)s->page_size * g->token_stride;
+    g->page_stride = s->kv_page_stride ? s->kv_page_stride : (long long)s->n_kv_heads * g->head_stride;
+    if (g->token_stride < s->head_dim) return VSA_ERR_INVALID_ARGUMENT;
+    if ((g->token_stride % 8) || (g->head_stride % 8) || (g->page_stride % 8)) return VSA_ERR_MISALIGNED;
+    return VSA_OK;
+}
+
+int check_routing_sizes(const Geometry& g, int P, int K_c, bool need_kc)
+{
+    if (P < 1) return VSA_ERR_INVALID_ARGUMENT;
+    if (P > kMaxP) return VSA_ERR_UNSUPPORTED_SHAPE;
+    if (need_kc) {
+        if (K_c < 1) return VSA_ERR_INVALID_ARGUMENT;
+        if (K_c > P * vsa::kPageSize) return VSA_ERR_UNSUPPORTED_SHAPE;
+    }
+    (void)g;
+    return VSA_OK;
+}
+
+int check_epsilon(float epsilon)
+{
+    if (!(epsilon > 0.0f) || isinf(epsilon)) return VSA_ERR_INVALID_ARGUMENT;
+    return VSA_OK;
+}
+
+// step workspace = [ route scores | dense scratch ], each part 256-byte aligned
+size_t step_route_part(const Geometry& g) { return align_up(vsa::route_workspace_bytes(g), 256); }
+
+int cuda_rc(cudaError_t e) { return e == cudaSuccess ? VSA_OK : VSA_ERR_CUDA; }
+
+}  // namespace
+
+extern "C" {
+
+const char* vsa_strerror(int code)
+{
+    switch (code) {
+        case VSA_OK: return "ok";
+        case VSA_ERR_INVALID_ARGUMENT: return "invalid argument";
+        case VSA_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+        case VSA_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case VSA_ERR_MISALIGNED: return "pointer or stride not 16-byte aligned";
+        case VSA_ERR_CUDA: return "CUDA runtime error";
+        default: return "unknown error code";
+    }
+}
+
+size_t vsa_workspace_bytes(const vsa_shape_t* shape, int32_t P, int32_t K_c, int which_call)
+{
+    Geometry g;
+    if (make_geometry(shape, &g) != VSA_OK) return 0;
+    (void)P;
+    (void)K_c;
+    switch (which_call) {
+        case VSA_WS_ROUTE: return vsa::route_workspace_bytes(g);
+        case VSA_WS_SPARSE: return 0;
+        case VSA_WS_DENSE: return vsa::dense_workspace_bytes(g);
+        case VSA_WS_STEP: return step_route_part(g) + vsa::dense_workspace_bytes(g);
+        default: return 0;
+    }
+}
+
+int vsa_build_page_summaries(const vsa_shape_t* shape, const void* k_cache, const int32_t* block_table,
+                             const int32_t* seq_lens, const int32_t* first_page, void* summaries, void* stream)
+{
+    Geometry g;
+    int rc = make_geometry(shape, &g);
+    if (rc) return rc;
+    if (!k_cache || !block_table || !seq_lens || !summaries) return VSA_ERR_INVALID_ARGUMENT;
+    if (!aligned16(k_cache) || !aligned16(summaries)) return VSA_ERR_MISALIGNED;
+    return cuda_rc(vsa::launch_build_summaries(g, k_cache, block_table, seq_lens, first_page, summaries,
+                                               (cudaStream_t)stream));
+}
+
+int vsa_route_pages(const vsa_shape_t* shape, const void* q, const void* summaries, const int32_t* block_table,
+                    const int32_t* seq_lens, int32_t P, int32_t* routed_pages, float* routed_scores, void* ws,
+                    size_t ws_bytes, void* stream)
+{
+    Geometry g;
+    int rc = make_geometry(shape, &g);
+    if (rc) return rc;
+    if ((rc = check_routing_sizes(g, P, 0, false))) return rc;
+    if (!q || !summaries || !block_table || !seq_lens || !routed_pages || !ws) return VSA_ERR_INVALID_ARGUMENT;
+    if (!aligned16(q) || !aligned16(summaries) || !aligned16(ws)) return VSA_ERR_MISALIGNED;
+    if (ws_bytes < vsa::route_workspace_bytes(g)) return VSA_ERR_WORKSPACE_TOO_SMALL;
+    return cuda_rc(vsa::launch_route(g, q, summaries, block_table, seq_lens, P, routed_pages, routed_scores, ws,
+                                     nullptr, (cudaStream_t)stream));
+}
+
+int vsa_sparse_decode(const vsa_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,
+                      const int32_t* block_table, const int32_t* seq_lens, const int32_t* routed_pages,
+                      int32_t P, int32_t K_c, float epsilon, float gap_threshold, float* out, vsa_diag_t* diag,
+                      int32_t* fallback_list, int32_t* fallback_count, void* ws, size_t ws_bytes, void* stream)
+{
+    (void)ws;
+    (void)ws_bytes;
+    Geometry g;
+    int rc = make_geometry(shape, &g);
+    if (rc) return rc;
+    if ((rc = check_routing_sizes(g, P, K_c, true))) return rc;
+    if ((rc = check_epsilon(epsilon))) return rc;
+    if (isnan(gap_threshold)) return VSA_ERR_INVALID_ARGUMENT;
+    if (!q || !k_cache || !v_cache || !block_table || !seq_lens || !routed_pages || !out || !diag ||
+        !fallback_list || !fallback_count)
+        return VSA_ERR_INVALID_ARGUMENT;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache)) return VSA_ERR_MISALIGNED;
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e = cudaMemsetAsync(fallback_count, 0, sizeof(int32_t), st);
+    if (e != cudaSuccess) return VSA_ERR_CUDA;
+    return cuda_rc(vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, routed_pages, P, K_c,
+                                      epsilon, gap_threshold, out, diag, fallback_list, fallback_count, st));
+}
+
+int vsa_dense_decode_fallback(const vsa_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,
+                              const int32_t* block_table, const int32_t* seq_lens, const int32_t* fallback_list,
+                              const int32_t* fallback_count, float epsilon, float* out, vsa_diag_t* diag,
+                              void* ws, size_t ws_bytes, void* stream)
+{
+    Geometry g;
+    int rc = make_geometry(shape, &g);
+    if (rc) return rc;
+    if ((rc = check_epsilon(epsilon))) return rc;
+    if (!q || !k_cache || !v_cache || !block_table || !seq_lens || !out || !ws) return VSA_ERR_INVALID_ARGUMENT;
+    if (fallback_count && !fallback_list) return VSA_ERR_INVALID_ARGUMENT;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(ws)) return VSA_ERR_MISALIGNED;
+    if (ws_bytes < vsa::dense_workspace_bytes(g)) return VSA_ERR_WORKSPACE_TOO_SMALL;
+    return cuda_rc(vsa::launch_dense(g, q, k_cache, v_cache, block_table, seq_lens, fallback_list, fallback_count,
+                                     epsilon, out, diag, ws, (cudaStream_t)stream));
+}
+
+int vsa_decode_step(const vsa_shape_t* shape, const void* q, const void* summaries, const void* k_cache,
+                    const void* v_cache, const int32_t* block_table, const int32_t* seq_lens, int32_t P,
+                    int32_t K_c, float epsilon, float gap_threshold, float* out, vsa_diag_t* diag,
+                    int32_t* routed_pages, int32_t* fallback_list, int32_t* fallback_count, void* ws,
+                    size_t ws_bytes, void* stream)
+{
+    Geometry g;
+    int rc = make_geometry(shape, &g);
+    if (rc) return rc;
+    if ((rc = check_routing_sizes(g, P, K_c, true))) return rc;
+    if ((rc = check_epsilon(epsilon))) return rc;
+    if (isnan(gap_threshold)) return VSA_ERR_INVALID_ARGUMENT;
+    if (!q || !summaries || !k_cache || !v_cache || !block_table || !seq_lens || !out || !diag ||
+        !routed_pages || !fallback_list || !fallback_count || !ws)
+        return VSA_ERR_INVALID_ARGUMENT;
+    if (!aligned16(q) || !aligned16(summaries) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(ws))
+        return VSA_ERR_MISALIGNED;
+    if (ws_bytes < step_route_part(g) + vsa::dense_workspace_bytes(g)) return VSA_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = (cudaStream_t)stream;
+    void* ws_dense = (char*)ws + step_route_part(g);
+    // the scan kernel clears fallback_count, so the step needs no separate memset for it
+    cudaError_t e = vsa::launch_route(g, q, summaries, block_table, seq_lens, P, routed_pages, nullptr, ws,
+                                      fallback_count, st);
+    if (e != cudaSuccess) return VSA_ERR_CUDA;
+    e = vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, routed_pages, P, K_c, epsilon,
+                           gap_threshold, out, diag, fallback_list, fallback_count, st);
+    if (e != cudaSuccess) return VSA_ERR_CUDA;
+    e = vsa::launch_dense(g, q, k_cache, v_cache, block_table, seq_lens, fallback_list, fallback_count, epsilon,
+                          out, diag, ws_dense, st);
+    return cuda_rc(e);
+}
+
+int vsa_decode_step_host(const vsa_shape_t* shape, const void* q_host, void* q_dev, const void* summaries,
+                         const void* k_cache, const void* v_cache, const int32_t* block_table,
+                         const int32_t* seq_lens, int32_t P, int32_t K_c, float epsilon, float gap_threshold,
+                         float* out_host, float* out_dev, vsa_diag_t* diag_host, vsa_diag_t* diag_dev,
+                         int32_t* routed_pages, int32_t* fallback_list, int32_t* fallback_count, void* ws,
+                         size_t ws_bytes, void* stream)
+{
+    Geometry g;
+    int rc = make_geometry(shape, &g);
+    if (rc) return rc;
+    if (!q_host || !q_dev || !out_host || !out_dev || !diag_dev) return VSA_ERR_INVALID_ARGUMENT;
+    // validate everything else before the first copy is enqueued
+    if ((rc = check_routing_sizes(g, P, K_c, true))) return rc;
+    if ((rc = check_epsilon(epsilon))) return rc;
+    if (isnan(gap_threshold)) return VSA_ERR_INVALID_ARGUMENT;
+    if (!summaries || !k_cache || !v_cache || !block_table || !seq_lens || !routed_pages || !fallback_list ||
+        !fallback_count || !ws)
+        return VSA_ERR_INVALID_ARGUMENT;
+    if (!aligned16(q_dev) || !aligned16(summaries) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(ws))
+        return VSA_ERR_MISALIGNED;
+    if (ws_bytes < step_route_part(g) + vsa::dense_workspace_bytes(g)) return VSA_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t units = (size_t)g.batch * g.n_q_heads;
+    if (cudaMemcpyAsync(q_dev, q_host, units * vsa::kHeadDim * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return VSA_ERR_CUDA;
+    rc = vsa_decode_step(shape, q_dev, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon,
+                         gap_threshold, out_dev, diag_dev, routed_pages, fallback_list, fallback_count, ws,
+                         ws_bytes, stream);
+    if (rc) return rc;
+    if (cudaMemcpyAsync(out_host, out_dev, units * vsa::kHeadDim * sizeof(float), cudaMemcpyDeviceToHost, st) !=
+        cudaSuccess)
+        return VSA_ERR_CUDA;
+    if (diag_host &&
+        cudaMemcpyAsync(diag_host, diag_dev, units * sizeof(vsa_diag_t), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return VSA_ERR_CUDA;
+    return VSA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,334 @@
+// Fused sparse pass for one (sequence, query head) unit per thread block (paper Sec. 7 steps 2-4,
+// Sec. 8 gap statistic, Cor. 1 leakage bound, Sec. 10.3 fallback flag):
+//   score every valid token of the routed pages -> exact top-K_c -> softmax weights at temperature
+//   epsilon -> weighted sum of the candidates' value rows -> diagnostics.
+// The candidate list and the weights live in shared memory and registers only.
+#include <limits.h>
+#include <math.h>
+
+#include "vsa_device.cuh"
+#include "vsa_launch.h"
+
+namespace vsa {
+
+namespace {
+
+constexpr int kSparseThreads = 256;
+constexpr int kSparseWarps = kSparseThreads / 32;
+constexpr int kGroups = 2 * kSparseWarps;   // half-warps per block
+
+struct SparseSmem {
+    int32_t* page_l;      // [P] routed logical pages, ascending, invalid entries last
+    int32_t* page_phys;   // [P]
+    uint32_t* keys;       // [P * 16] token score keys, array index = 16 * slot + token (position order)
+    int32_t* sel;         // [K_c] array indices of the candidates, ascending
+    uint32_t* hist;       // [256]
+    uint32_t* scratch;    // [16]
+    uint32_t* warp_counts;   // [40]
+    float* red;           // [warps][128]
+    float* zred;          // [warps]
+    uint8_t* take;        // [P * 16]
+};
+
+__device__ __forceinline__ SparseSmem carve(uint32_t* base, int P, int K_c)
+{
+    SparseSmem s;
+    const int N = P * kPageSize;
+    s.page_l = (int32_t*)base;
+    s.page_phys = s.page_l + P;
+    s.keys = (uint32_t*)(s.page_phys + P);
+    s.sel = (int32_t*)(s.keys + N);
+    s.hist = (uint32_t*)(s.sel + K_c);
+    s.scratch = s.hist + 256;
+    s.warp_counts = s.scratch + 16;
+    s.red = (float*)(s.warp_counts + 40);
+    s.zred = s.red + kSparseWarps * kHeadDim;
+    s.take = (uint8_t*)(s.zred + kSparseWarps);
+    return s;
+}
+
+__device__ __forceinline__ void write_failed_unit(float* out, vsa_diag_t* diag, long long unit, int status)
+{
+    if (threadIdx.x < kHeadDim) out[unit * kHeadDim + threadIdx.x] = 0.0f;
+    if (threadIdx.x == 0) {
+        vsa_diag_t d;
+        d.delta = d.delta12 = d.s_max = d.lse = d.leak_bound = 0.0f;
+        d.n_candidates = 0;
+        d.fallback = 0;
+        d.status = status;
+        diag[unit] = d;
+    }
+}
+
+__global__ void __launch_bounds__(kSparseThreads)
+sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* __restrict__ k_cache,
+                     const uint16_t* __restrict__ v_cache, const int32_t* __restrict__ block_table,
+                     const int32_t* __restrict__ seq_lens, const int32_t* __restrict__ routed_pages, int P,
+                     int K_c, float epsilon, float gap_threshold, float* __restrict__ out,
+                     vsa_diag_t* __restrict__ diag, int32_t* __restrict__ fallback_list,
+                     int32_t* __restrict__ fallback_count)
+{
+    extern __shared__ uint32_t smem_raw[];
+    const SparseSmem sm = carve(smem_raw, P, K_c);
+    const int N = P * kPageSize;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, c = lane & 15, gi = lane >> 4;
+    const long long unit = blockIdx.x;
+    const int b = (int)(unit / geo.n_q_heads), h = (int)(unit % geo.n_q_heads), g = h / geo.group;
+    const int T = seq_lens[b];
+    if (T <= 0 || T > geo.max_pages * kPageSize) {
+        write_failed_unit(out, diag, unit, VSA_UNIT_BAD_LENGTH);
+        return;
+    }
+    const int nb = (T + kPageSize - 1) / kPageSize;
+
+    // ---- routed pages: validate, sort by logical page so that array order = position order ----
+    int32_t* raw = (int32_t*)sm.keys;   // staging; keys[] (16 P words) is initialised further down
+    for (int t = tid; t < P; t += kSparseThreads) {
+        const int l = routed_pages[unit * P + t];
+        raw[t] = (l >= 0 && l < nb) ? l : INT_MAX;
+    }
+    __syncthreads();
+    for (int t = tid; t < P; t += kSparseThreads) {
+        const int l = raw[t];
+        int rank = 0;
+        for (int j = 0; j < P; ++j) rank += (raw[j] < l) || (raw[j] == l && j < t);
+        sm.page_l[rank] = l;
+    }
+    __syncthreads();
+    int bad = 0;
+    for (int t = tid; t < P; t += kSparseThreads) {
+        const int l = sm.page_l[t];
+        int phys = -1;
+        if (l != INT_MAX) {
+            phys = block_table[(long long)b * geo.max_pages + l];
+            if (phys < 0 || phys >= geo.pool_pages) {
+                phys = -1;
+                bad = 1;
+            }
+        }
+        sm.page_phys[t] = phys;
+    }
+    const int np = __syncthreads_count(tid < P && sm.page_l[tid < P ? tid : 0] != INT_MAX);
+    if (__syncthreads_or(bad)) {
+        write_failed_unit(out, diag, unit, VSA_UNIT_BAD_PAGE);
+        return;
+    }
+    // (P <= 128 < blockDim.x, so the count above saw every slot)
+    for (int i = tid; i < N; i += kSparseThreads) {
+        sm.keys[i] = 0u;
+        sm.take[i] = 0;
+    }
+    __syncthreads();
+
+    // ---- token routing: score all 16 tokens of a page per half-warp ----
+    float qf[8];
+    {
+        const uint4 v = *reinterpret_cast<const uint4*>(q + unit * kHeadDim + c * 8);
+        unpack8(v, qf);
+    }
+    for (int pp = warp; pp * 2 < np; pp += kSparseWarps) {
+        const int slot = pp * 2 + gi;
+        const bool active = slot < np;
+        uint4 rows[kPageSize];
+        if (active) {
+            const uint16_t* src = k_cache + (long long)sm.page_phys[slot] * geo.page_stride +
+                                  (long long)g * geo.head_stride + c * 8;
+#pragma unroll
+            for (int t = 0; t < kPageSize; ++t) rows[t] = ld_nc_16B(src + (long long)t * geo.token_stride);
+        } else {
+#pragma unroll
+            for (int t = 0; t < kPageSize; ++t) rows[t] = make_uint4(0u, 0u, 0u, 0u);
+        }
+        float vals[16];
+#pragma unroll
+        for (int t = 0; t < kPageSize; ++t) {
+            float kf[8];
+            unpack8(rows[t], kf);
+            vals[t] = chunk_partial(qf, kf);
+        }
+        const float s = reduce_scatter16(vals, c);   // lane c: score of token c of the page
+        if (active && sm.page_l[slot] * kPageSize + c < T) sm.keys[slot * kPageSize + c] = float_to_key(s);
+    }
+    // number of valid scored tokens
+    if (warp == 0) {
+        int cnt = 0;
+        for (int t = lane; t < np; t += 32) cnt += min(kPageSize, T - sm.page_l[t] * kPageSize);
+#pragma unroll
+        for (int off = 16; off; off >>= 1) cnt += __shfl_xor_sync(kFullMask, cnt, off);
+        if (lane == 0) sm.scratch[8] = (uint32_t)cnt;
+    }
+    __syncthreads();
+    const int nv = (int)sm.scratch[8];
+    const int ns = min(K_c, nv);
+
+    // ---- exact top-ns; the (ns+1)-th element is the best rejected token ----
+    uint32_t out_key = 0u;
+    bool has_rejected = nv > ns;
+    if (has_rejected) {
+        const SelectResult r = block_select_kth(sm.keys, N, ns + 1, sm.hist, sm.scratch);
+        out_key = r.kth;
+        const int need = ns - r.n_greater;   // how many of the tied-with-cut elements still get in
+        if (need > 0) block_mark_first_equal(sm.keys, N, r.kth, need, sm.take, sm.warp_counts);
+        __syncthreads();
+        for (int i = tid; i < N; i += kSparseThreads)
+            if (sm.keys[i] > out_key) sm.take[i] = 1;
+    } else {
+        for (int i = tid; i < N; i += kSparseThreads)
+            if (sm.keys[i] != 0u) sm.take[i] = 1;
+    }
+
+    // ---- best and second-best key over the scored tokens (multiset order statistics) ----
+    {
+        uint32_t a1 = 0u, a2 = 0u;
+        for (int i = tid; i < N; i += kSparseThreads) {
+            const uint32_t k = sm.keys[i];
+            if (k > a1) {
+                a2 = a1;
+                a1 = k;
+            } else if (k > a2) {
+                a2 = k;
+            }
+        }
+#pragma unroll
+        for (int off = 16; off; off >>= 1) {
+            const uint32_t b1 = __shfl_xor_sync(kFullMask, a1, off), b2 = __shfl_xor_sync(kFullMask, a2, off);
+            const uint32_t n1 = max(a1, b1), n2 = max(min(a1, b1), max(a2, b2));
+            a1 = n1;
+            a2 = n2;
+        }
+        if (lane == 0) {
+            sm.warp_counts[2 * warp] = a1;
+            sm.warp_counts[2 * warp + 1] = a2;
+        }
+    }
+    __syncthreads();
+    uint32_t key1 = 0u, key2 = 0u;
+#pragma unroll
+    for (int w = 0; w < kSparseWarps; ++w) {
+        const uint32_t b1 = sm.warp_counts[2 * w], b2 = sm.warp_counts[2 * w + 1];
+        const uint32_t n1 = max(key1, b1), n2 = max(min(key1, b1), max(key2, b2));
+        key1 = n1;
+        key2 = n2;
+    }
+    __syncthreads();   // warp_counts is reused below
+
+    // ---- ordered compaction of the candidates: sel[] ascending in array (= position) order ----
+    {
+        const int per = (N + kSparseThreads - 1) / kSparseThreads;
+        const int lo = tid * per, hi = min(N, lo + per);
+        int cnt = 0;
+        for (int i = lo; i < hi; ++i) cnt += sm.take[i];
+        int incl = cnt;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int o = __shfl_up_sync(kFullMask, incl, off);
+            if (lane >= off) incl += o;
+        }
+        if (lane == 31) sm.warp_counts[warp] = (uint32_t)incl;
+        __syncthreads();
+        int base = 0;
+        for (int w = 0; w < warp; ++w) base += (int)sm.warp_counts[w];
+        int o = base + incl - cnt;
+        for (int i = lo; i < hi; ++i)
+            if (sm.take[i]) sm.sel[o++] = i;
+    }
+    __syncthreads();
+
+    // ---- softmax weights and value gather ----
+    const float s1 = ns > 0 ? key_to_float(key1) : -INFINITY;
+    const float scale = 1.4426950408889634f / epsilon;   // log2(e) / epsilon
+    float acc[8], z = 0.0f;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] = 0.0f;
+    const int gidx = warp * 2 + gi;
+    constexpr int UNR = 4;
+    for (int j0 = gidx; j0 < ns; j0 += kGroups * UNR) {
+        uint4 rows[UNR];
+        float w[UNR];
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+            const int j = j0 + u * kGroups;
+            rows[u] = make_uint4(0u, 0u, 0u, 0u);
+            w[u] = 0.0f;
+            if (j < ns) {
+                const int i = sm.sel[j];
+                const int slot = i >> 4, t = i & 15;
+                rows[u] = ld_nc_16B(v_cache + (long long)sm.page_phys[slot] * geo.page_stride +
+                                    (long long)g * geo.head_stride + (long long)t * geo.token_stride + c * 8);
+                w[u] = exp2f((key_to_float(sm.keys[i]) - s1) * scale);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+            float vf[8];
+            unpack8(rows[u], vf);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = fmaf(w[u], vf[e], acc[e]);
+            z += w[u];
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] += __shfl_xor_sync(kFullMask, acc[e], 16);
+    z += __shfl_xor_sync(kFullMask, z, 16);
+    if (gi == 0) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) sm.red[warp * kHeadDim + c * 8 + e] = acc[e];
+        if (c == 0) sm.zred[warp] = z;
+    }
+    __syncthreads();
+    float Z = 0.0f;
+#pragma unroll
+    for (int w = 0; w < kSparseWarps; ++w) Z += sm.zred[w];
+    if (tid < kHeadDim) {
+        float a = 0.0f;
+#pragma unroll
+        for (int w = 0; w < kSparseWarps; ++w) a += sm.red[w * kHeadDim + tid];
+        out[unit * kHeadDim + tid] = ns > 0 ? a / Z : 0.0f;
+    }
+
+    // ---- diagnostics and fallback flag ----
+    if (tid == 0) {
+        const float s2 = ns > 1 ? key_to_float(key2) : -INFINITY;
+        const float delta = has_rejected ? s1 - key_to_float(out_key) : INFINITY;
+        vsa_diag_t d;
+        d.delta = delta;
+        d.delta12 = ns > 0 ? s1 - s2 : INFINITY;
+        d.s_max = s1;
+        d.lse = ns > 0 ? s1 / epsilon + logf(Z) : -INFINITY;
+        d.leak_bound = fminf(1.0f, (float)(T - ns) * expf(-delta / epsilon));
+        d.n_candidates = ns;
+        d.fallback = (delta < gap_threshold && ns < T) ? 1 : 0;
+        d.status = 0;
+        diag[unit] = d;
+        if (d.fallback) fallback_list[atomicAdd(fallback_count, 1)] = (int32_t)unit;
+    }
+}
+
+size_t sparse_smem_bytes(int P, int K_c)
+{
+    const size_t N = (size_t)P * kPageSize;
+    return (size_t)P * 8 + N * 4 + (size_t)K_c * 4 + 256 * 4 + 16 * 4 + 40 * 4 +
+           (size_t)kSparseWarps * kHeadDim * 4 + kSparseWarps * 4 + N + 16;
+}
+
+}  // namespace
+
+cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache, const void* v_cache,
+                          const int32_t* block_table, const int32_t* seq_lens, const int32_t* routed_pages,
+                          int P, int K_c, float epsilon, float gap_threshold, float* out, vsa_diag_t* diag,
+                          int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream)
+{
+    const size_t smem = sparse_smem_bytes(P, K_c);
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(sparse_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    const unsigned units = (unsigned)(g.batch * g.n_q_heads);
+    sparse_decode_kernel<<<units, kSparseThreads, smem, stream>>>(
+        g, (const uint16_t*)q, (const uint16_t*)k_cache, (const uint16_t*)v_cache, block_table, seq_lens,
+        routed_pages, P, K_c, epsilon, gap_threshold, out, diag, fallback_list, fallback_count);
+    return cudaGetLastError();
+}
+
+}  // namespace vsa

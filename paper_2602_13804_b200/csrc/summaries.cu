@@ -1,0 +1,71 @@
+// Page summaries: mean of the valid key rows of each page, per KV head (paper Sec. 7 step 1 names
+// "coarse page summaries k_page" without defining them; the mean key is this library's reading).
+#include "vsa_device.cuh"
+#include "vsa_launch.h"
+
+namespace vsa {
+
+// One thread per (logical page, kv head, 16-byte slice of the head dimension): the 16 threads of a
+// (page, head) read one contiguous 256-byte key row per iteration.  fp32 sum in ascending token
+// order, IEEE division by the number of valid rows, round-to-nearest-even to bf16.
+__global__ void __launch_bounds__(256) summaries_kernel(Geometry geo, const uint16_t* __restrict__ k_cache,
+                                                        const int32_t* __restrict__ block_table,
+                                                        const int32_t* __restrict__ seq_lens,
+                                                        const int32_t* __restrict__ first_page,
+                                                        uint16_t* __restrict__ summaries)
+{
+    const int b = blockIdx.y;
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const int c = (int)(idx & 15);
+    const int g = (int)((idx >> 4) % geo.n_kv_heads);
+    const long long l = (idx >> 4) / geo.n_kv_heads;
+    const int T = seq_lens[b];
+    if (T <= 0 || T > geo.max_pages * kPageSize) return;
+    const int nb = (T + kPageSize - 1) / kPageSize;
+    const int l0 = first_page ? first_page[b] : 0;
+    if (l < l0 || l >= nb) return;
+    const long long p = block_table[(long long)b * geo.max_pages + l];
+    if (p < 0 || p >= geo.pool_pages) return;
+    const int n = min(kPageSize, T - (int)l * kPageSize);
+
+    const uint16_t* src = k_cache + p * geo.page_stride + (long long)g * geo.head_stride + c * 8;
+    uint4 rows[kPageSize];
+#pragma unroll
+    for (int t = 0; t < kPageSize; ++t)
+        if (t < n) rows[t] = ld_nc_16B(src + (long long)t * geo.token_stride);
+    float acc[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] = 0.0f;
+#pragma unroll
+    for (int t = 0; t < kPageSize; ++t) {
+        if (t < n) {
+            float f[8];
+            unpack8(rows[t], f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = acc[e] + f[e];
+        }
+    }
+    const float fn = (float)n;
+    uint32_t h[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) h[e] = bf16_bits_rne(__fdiv_rn(acc[e], fn));
+    uint4 o;
+    o.x = h[0] | (h[1] << 16);
+    o.y = h[2] | (h[3] << 16);
+    o.z = h[4] | (h[5] << 16);
+    o.w = h[6] | (h[7] << 16);
+    *reinterpret_cast<uint4*>(summaries + (p * geo.n_kv_heads + g) * kHeadDim + c * 8) = o;
+}
+
+cudaError_t launch_build_summaries(const Geometry& g, const void* k_cache, const int32_t* block_table,
+                                   const int32_t* seq_lens, const int32_t* first_page, void* summaries,
+                                   cudaStream_t stream)
+{
+    const long long threads = (long long)g.max_pages * g.n_kv_heads * 16;
+    dim3 grid((unsigned)((threads + 255) / 256), (unsigned)g.batch);
+    summaries_kernel<<<grid, 256, 0, stream>>>(g, (const uint16_t*)k_cache, block_table, seq_lens, first_page,
+                                               (uint16_t*)summaries);
+    return cudaGetLastError();
+}
+
+}  // namespace vsa

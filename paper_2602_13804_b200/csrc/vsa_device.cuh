@@ -1,0 +1,224 @@
+// Device-side building blocks shared by the kernels of libvsa: bf16 unpacking, the fixed-order
+// fp32 dot product, order-preserving keys and block-wide exact top-k selection.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace vsa {
+
+constexpr int kHeadDim = 128;   // elements per head
+constexpr int kPageSize = 16;   // tokens per page
+constexpr int kRowBytes = kHeadDim * 2;
+constexpr unsigned kFullMask = 0xffffffffu;
+
+// ---- bf16 ------------------------------------------------------------------------------
+// A 16-byte vector holds 8 consecutive bf16 values, element 0 in the low half of .x
+__device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8])
+{
+    f[0] = __uint_as_float(v.x << 16);
+    f[1] = __uint_as_float(v.x & 0xffff0000u);
+    f[2] = __uint_as_float(v.y << 16);
+    f[3] = __uint_as_float(v.y & 0xffff0000u);
+    f[4] = __uint_as_float(v.z << 16);
+    f[5] = __uint_as_float(v.z & 0xffff0000u);
+    f[6] = __uint_as_float(v.w << 16);
+    f[7] = __uint_as_float(v.w & 0xffff0000u);
+}
+
+// round-to-nearest-even fp32 -> bf16 bits (finite inputs)
+__device__ __forceinline__ uint32_t bf16_bits_rne(float f)
+{
+    uint32_t u = __float_as_uint(f);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return (u >> 16) | 0x0040u;
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return u >> 16;
+}
+
+__device__ __forceinline__ uint4 ld_nc_16B(const void* p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+// ---- the fixed-order dot product ---------------------------------------------------------
+// A row of 128 elements is spread over 16 lanes, lane c holding elements 8c .. 8c+7.
+// chunk_partial() is the left-to-right sum of the lane's 8 products (bf16 x bf16 products are
+// exact in fp32, so fusing the multiply into the add changes nothing).
+__device__ __forceinline__ float chunk_partial(const float (&x)[8], const float (&y)[8])
+{
+    float acc = x[0] * y[0];
+#pragma unroll
+    for (int e = 1; e < 8; ++e) acc = fmaf(x[e], y[e], acc);
+    return acc;
+}
+
+// Halving tree over the 16 lanes of a half-warp for 16 independent values at once
+// ("reduce-scatter"): on entry v[i] is this lane's partial of value i, on return lane c
+// (0..15 within its half-warp) holds the complete sum of value c.  For each value the
+// additions are exactly p[c] += p[c+off] for off = 8, 4, 2, 1 (addition is commutative, so
+// which lane of a pair performs it does not change a bit).  15 shuffles for 16 values.
+__device__ __forceinline__ float reduce_scatter16(float (&v)[16], int c)
+{
+    {
+        const bool hi = c & 8;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float send = hi ? v[i] : v[i + 8];
+            const float keep = hi ? v[i + 8] : v[i];
+            v[i] = keep + __shfl_xor_sync(kFullMask, send, 8);
+        }
+    }
+    {
+        const bool hi = c & 4;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float send = hi ? v[i] : v[i + 4];
+            const float keep = hi ? v[i + 4] : v[i];
+            v[i] = keep + __shfl_xor_sync(kFullMask, send, 4);
+        }
+    }
+    {
+        const bool hi = c & 2;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const float send = hi ? v[i] : v[i + 2];
+            const float keep = hi ? v[i + 2] : v[i];
+            v[i] = keep + __shfl_xor_sync(kFullMask, send, 2);
+        }
+    }
+    {
+        const bool hi = c & 1;
+        const float send = hi ? v[0] : v[1];
+        const float keep = hi ? v[1] : v[0];
+        v[0] = keep + __shfl_xor_sync(kFullMask, send, 1);
+    }
+    return v[0];
+}
+
+// ---- order-preserving keys -----------------------------------------------------------------
+// key(a) > key(b)  <=>  a > b for finite floats and infinities; -0 and +0 map to one key.
+// Key 0 is never produced by a non-NaN float and serves as "no element".
+__device__ __forceinline__ uint32_t float_to_key(float f)
+{
+    uint32_t u = __float_as_uint(f);
+    if (u == 0x80000000u) u = 0u;
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__device__ __forceinline__ float key_to_float(uint32_t k)
+{
+    const uint32_t u = (k & 0x80000000u) ? (k & 0x7fffffffu) : ~k;
+    return __uint_as_float(u);
+}
+
+// ---- exact block-wide top-k ------------------------------------------------------------------
+// Elements are keys[0..n) in shared memory (key 0 = absent).  The order is (key descending,
+// array index ascending).  After the call, for k >= 1 and at least k present elements:
+//   *kth       = key of the k-th element in that order,
+//   *n_greater = number of elements with key > *kth  (all of them belong to the top k),
+//   *n_equal   = number of elements with key == *kth; the top k takes the first
+//                k - *n_greater of them in array-index order.
+// MSB-first radix select, 8 bits per pass.  hist: 256 counters in shared memory.
+// All threads of the block must call it; results are valid for all threads on return.
+struct SelectResult {
+    uint32_t kth;
+    int n_greater;
+    int n_equal;
+};
+
+__device__ __forceinline__ SelectResult block_select_kth(const uint32_t* keys, int n, int k, uint32_t* hist,
+                                                         uint32_t* scratch /* >= 4 words */)
+{
+    uint32_t prefix = 0, prefix_mask = 0;
+    int remaining = k;   // rank still to find inside the current prefix bucket
+    int greater = 0;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0;
+        __syncthreads();
+        for (int i = threadIdx.x; i < n; i += blockDim.x) {
+            const uint32_t key = keys[i];
+            if (key != 0u && (key & prefix_mask) == prefix) atomicAdd(&hist[(key >> shift) & 0xffu], 1u);
+        }
+        __syncthreads();
+        if (threadIdx.x < 32) {
+            // lane j owns digits 8j .. 8j+7; find the digit where the count from the top reaches `remaining`
+            const int lane = threadIdx.x;
+            uint32_t c[8], mine = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                c[j] = hist[lane * 8 + j];
+                mine += c[j];
+            }
+            // suffix sum over lanes: above = total count in digits of higher lanes
+            uint32_t incl = mine;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const uint32_t o = __shfl_down_sync(kFullMask, incl, off);
+                if (lane + off < 32) incl += o;
+            }
+            uint32_t above = incl - mine;
+            if (above < (uint32_t)remaining && (uint32_t)remaining <= incl) {
+#pragma unroll
+                for (int j = 7; j >= 0; --j) {
+                    if (above < (uint32_t)remaining && (uint32_t)remaining <= above + c[j]) {
+                        scratch[0] = (uint32_t)(lane * 8 + j);
+                        scratch[1] = above;   // elements of this bucket set that rank strictly higher
+                        scratch[2] = c[j];
+                    }
+                    above += c[j];
+                }
+            }
+        }
+        __syncthreads();
+        const uint32_t digit = scratch[0];
+        greater += (int)scratch[1];
+        remaining -= (int)scratch[1];
+        prefix |= digit << shift;
+        prefix_mask |= 0xffu << shift;
+        const int bucket = (int)scratch[2];
+        __syncthreads();
+        if (shift == 0) {
+            SelectResult r;
+            r.kth = prefix;
+            r.n_greater = greater;
+            r.n_equal = bucket;
+            return r;
+        }
+    }
+    SelectResult r = {0u, 0, 0};
+    return r;
+}
+
+// Rank, in array-index order, of element i among the elements with keys[j] == kth, for every
+// i at once: marks take[i] = 1 for the first `need` of them.  Runs tile by tile; only called when
+// a tie straddles the cut.  warp_counts: >= blockDim.x / 32 + 1 words of shared memory.
+__device__ __forceinline__ void block_mark_first_equal(const uint32_t* keys, int n, uint32_t kth, int need,
+                                                       uint8_t* take, uint32_t* warp_counts)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    int base = 0;
+    for (int start = 0; start < n; start += blockDim.x) {
+        const int i = start + threadIdx.x;
+        const bool eq = i < n && keys[i] == kth;
+        const unsigned b = __ballot_sync(kFullMask, eq);
+        if (lane == 0) warp_counts[warp] = __popc(b);
+        __syncthreads();
+        int before = base;
+        for (int w = 0; w < warp; ++w) before += warp_counts[w];
+        int total = 0;
+        for (int w = 0; w < nwarps; ++w) total += warp_counts[w];
+        if (eq) {
+            const int rank = before + __popc(b & ((1u << lane) - 1u));
+            if (rank < need) take[i] = 1;
+        }
+        base += total;
+        __syncthreads();
+        if (base >= need) break;
+    }
+}
+
+}  // namespace vsa

@@ -1,0 +1,43 @@
+// Host-side launch interface between the C ABI (api.cu) and the kernel files.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/vsa.h"
+
+namespace vsa {
+
+struct Geometry {
+    int batch, n_q_heads, n_kv_heads, group, max_pages;
+    long long pool_pages;
+    long long page_stride, head_stride, token_stride;   // elements
+};
+
+// ---- page summaries -----------------------------------------------------------------------
+cudaError_t launch_build_summaries(const Geometry& g, const void* k_cache, const int32_t* block_table,
+                                   const int32_t* seq_lens, const int32_t* first_page, void* summaries,
+                                   cudaStream_t stream);
+
+// ---- page routing ---------------------------------------------------------------------------
+size_t route_workspace_bytes(const Geometry& g);
+cudaError_t launch_route(const Geometry& g, const void* q, const void* summaries, const int32_t* block_table,
+                         const int32_t* seq_lens, int P, int32_t* routed_pages, float* routed_scores,
+                         void* ws, int32_t* zero_word, cudaStream_t stream);
+
+// ---- fused sparse pass ------------------------------------------------------------------------
+cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache, const void* v_cache,
+                          const int32_t* block_table, const int32_t* seq_lens, const int32_t* routed_pages,
+                          int P, int K_c, float epsilon, float gap_threshold, float* out, vsa_diag_t* diag,
+                          int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream);
+
+// ---- dense split-K pass -------------------------------------------------------------------------
+int dense_pages_per_split(const Geometry& g);
+size_t dense_workspace_bytes(const Geometry& g);
+cudaError_t launch_dense(const Geometry& g, const void* q, const void* k_cache, const void* v_cache,
+                         const int32_t* block_table, const int32_t* seq_lens, const int32_t* fallback_list,
+                         const int32_t* fallback_count, float epsilon, float* out, vsa_diag_t* diag, void* ws,
+                         cudaStream_t stream);
+
+}  // namespace vsa

@@ -1,0 +1,60 @@
+"""Buffer owner around the C-ABI calls: allocates outputs and scratch once, then every call is a
+single library call on the current CUDA stream.  No arithmetic happens here."""
+from __future__ import annotations
+
+from typing import Optional
+
+import torch
+
+from . import binding as B
+
+
+class SparsePagedDecoder:
+    """Device buffers for decode steps of one fixed shape (batch, heads, block-table width, P, K_c)."""
+
+    def __init__(self, shape: B.vsa_shape_t, P: int, K_c: int, epsilon: float, gap_threshold: float,
+                 device="cuda:0", host_io: bool = False):
+        if not torch.cuda.is_available():
+            raise RuntimeError("SparsePagedDecoder needs a CUDA device; there is no CPU path")
+        B.lib()
+        self.shape, self.P, self.K_c = shape, int(P), int(K_c)
+        self.epsilon, self.gap_threshold = float(epsilon), float(gap_threshold)
+        self.device = torch.device(device)
+        units = shape.batch * shape.n_q_heads
+        self.units = units
+        dev = self.device
+        self.out = torch.empty((shape.batch, shape.n_q_heads, shape.head_dim), dtype=torch.float32, device=dev)
+        self.diag = B.alloc_diag(units, dev)
+        self.routed_pages = torch.empty((shape.batch, shape.n_q_heads, self.P), dtype=torch.int32, device=dev)
+        self.fallback_list = torch.empty(units, dtype=torch.int32, device=dev)
+        self.fallback_count = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.ws = B.alloc_workspace(shape, self.P, self.K_c, B.VSA_WS_STEP, dev)
+        self.summaries: Optional[torch.Tensor] = None
+        if host_io:
+            self.q_dev = torch.empty((shape.batch, shape.n_q_heads, shape.head_dim), dtype=torch.bfloat16, device=dev)
+            self.out_host = torch.empty(self.out.shape, dtype=torch.float32).pin_memory()
+            self.diag_host = torch.empty((units, B.DIAG_BYTES // 4), dtype=torch.int32).pin_memory()
+
+    def build_summaries(self, k_cache, block_table, seq_lens, first_page=None, summaries=None) -> torch.Tensor:
+        if summaries is None:
+            summaries = torch.zeros((self.shape.num_pool_pages, self.shape.n_kv_heads, self.shape.head_dim),
+                                    dtype=torch.bfloat16, device=self.device)
+        B.vsa_build_page_summaries(self.shape, k_cache, block_table, seq_lens, first_page, summaries)
+        self.summaries = summaries
+        return summaries
+
+    def step(self, q, summaries, k_cache, v_cache, block_table, seq_lens) -> torch.Tensor:
+        """One decode step with device-resident q; returns the (device) output buffer."""
+        B.vsa_decode_step(self.shape, q, summaries, k_cache, v_cache, block_table, seq_lens, self.P, self.K_c,
+                          self.epsilon, self.gap_threshold, self.out, self.diag, self.routed_pages,
+                          self.fallback_list, self.fallback_count, self.ws)
+        return self.out
+
+    def step_host(self, q_host, summaries, k_cache, v_cache, block_table, seq_lens) -> torch.Tensor:
+        """One decode step with q in (pinned) host memory; results land in self.out_host / self.diag_host
+        once the current stream has been synchronised."""
+        B.vsa_decode_step_host(self.shape, q_host, self.q_dev, summaries, k_cache, v_cache, block_table, seq_lens,
+                               self.P, self.K_c, self.epsilon, self.gap_threshold, self.out_host, self.out,
+                               self.diag_host, self.diag, self.routed_pages, self.fallback_list,
+                               self.fallback_count, self.ws)
+        return self.out_host

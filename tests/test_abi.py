@@ -1,0 +1,136 @@
+"""CPU checks of the C-ABI boundary: the shared library loads, exports every function that
+include/vsa.h declares, and rejects bad arguments on the host with the documented codes.
+No kernel is launched here (every call below fails validation before touching the device)."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2602_13804_b200 import binding as B
+from paper_2602_13804_b200 import build as vsa_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "vsa.h")
+
+
+@pytest.fixture(scope="module")
+def lib():
+    vsa_build.build()
+    return B.lib()
+
+
+def declared_functions():
+    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(vsa_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(lib):
+    names = declared_functions()
+    assert {"vsa_build_page_summaries", "vsa_route_pages", "vsa_sparse_decode", "vsa_dense_decode_fallback",
+            "vsa_decode_step", "vsa_decode_step_host", "vsa_workspace_bytes", "vsa_strerror"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in vsa.h but not exported by libvsa.so"
+
+
+def test_struct_layouts_match_the_header():
+    assert C.sizeof(B.vsa_diag_t) == 32
+    assert C.sizeof(B.vsa_shape_t) == 6 * 4 + 4 * 8
+    assert B.vsa_shape_t.num_pool_pages.offset == 24
+
+
+def test_strerror_covers_all_codes(lib):
+    texts = {c: B.vsa_strerror(c) for c in (0, -1, -2, -3, -4, -5, -99)}
+    assert texts[0] == "ok" and "unknown" in texts[-99]
+    assert len(set(texts.values())) == len(texts)
+
+
+def test_workspace_sizes(lib):
+    s = B.make_shape(8, 32, 8, 2048, 65536)
+    route = B.vsa_workspace_bytes(s, 32, 256, B.VSA_WS_ROUTE)
+    assert route == 8 * 32 * 2048 * 4          # one fp32 score per (unit, logical page)
+    assert B.vsa_workspace_bytes(s, 32, 256, B.VSA_WS_SPARSE) == 0
+    dense = B.vsa_workspace_bytes(s, 32, 256, B.VSA_WS_DENSE)
+    assert dense > 0
+    assert B.vsa_workspace_bytes(s, 32, 256, B.VSA_WS_STEP) >= route + dense
+    bad = B.make_shape(8, 32, 8, 2048, 65536, head_dim=64)
+    assert B.vsa_workspace_bytes(bad, 32, 256, B.VSA_WS_STEP) == 0
+    assert B.vsa_workspace_bytes(s, 32, 256, 77) == 0
+
+
+FAKE = 0x10000   # an aligned non-NULL address that is never dereferenced: validation fails first
+ODD = 0x10008    # not 16-byte aligned
+
+
+def _route(lib, shape, q=FAKE, summ=FAKE, bt=FAKE, sl=FAKE, P=32, routed=FAKE, ws=FAKE, ws_bytes=1 << 40):
+    return lib.vsa_route_pages(C.byref(shape) if shape is not None else None, q, summ, bt, sl, P, routed, None,
+                               ws, ws_bytes, None)
+
+
+def test_route_argument_validation(lib):
+    ok = B.make_shape(2, 8, 2, 64, 256)
+    assert _route(lib, None) == -1
+    assert _route(lib, ok, q=None) == -1
+    assert _route(lib, ok, routed=None) == -1
+    assert _route(lib, ok, ws=None) == -1
+    assert _route(lib, ok, P=0) == -1
+    assert _route(lib, ok, P=129) == -2
+    assert _route(lib, B.make_shape(2, 8, 2, 64, 256, head_dim=64)) == -2
+    assert _route(lib, B.make_shape(2, 8, 2, 64, 256, page_size=32)) == -2
+    assert _route(lib, B.make_shape(2, 6, 2, 64, 256)) == -2          # group of 3
+    assert _route(lib, B.make_shape(2, 7, 2, 64, 256)) == -1          # heads do not divide
+    assert _route(lib, B.make_shape(0, 8, 2, 64, 256)) == -1
+    assert _route(lib, B.make_shape(2, 8, 2, 40000, 256)) == -2       # block-table row too wide
+    assert _route(lib, ok, ws_bytes=16) == -3
+    assert _route(lib, ok, q=ODD) == -4
+    assert _route(lib, B.make_shape(2, 8, 2, 64, 256, kv_token_stride=132)) == -4
+    assert _route(lib, B.make_shape(2, 8, 2, 64, 256, kv_token_stride=64)) == -1
+
+
+def _sparse(lib, shape, P=4, K_c=16, eps=1.0, tau=0.0, out=FAKE, diag=FAKE, fl=FAKE, fc=FAKE, q=FAKE):
+    return lib.vsa_sparse_decode(C.byref(shape), q, FAKE, FAKE, FAKE, FAKE, FAKE, P, K_c, eps, tau, out, diag, fl,
+                                 fc, None, 0, None)
+
+
+def test_sparse_argument_validation(lib):
+    ok = B.make_shape(2, 8, 2, 64, 256)
+    assert _sparse(lib, ok, eps=0.0) == -1
+    assert _sparse(lib, ok, eps=-1.0) == -1
+    assert _sparse(lib, ok, eps=float("inf")) == -1
+    assert _sparse(lib, ok, eps=float("nan")) == -1
+    assert _sparse(lib, ok, tau=float("nan")) == -1
+    assert _sparse(lib, ok, K_c=0) == -1
+    assert _sparse(lib, ok, K_c=4 * 16 + 1) == -2
+    assert _sparse(lib, ok, out=None) == -1
+    assert _sparse(lib, ok, diag=None) == -1
+    assert _sparse(lib, ok, fc=None) == -1
+    assert _sparse(lib, ok, q=ODD) == -4
+
+
+def test_dense_and_step_argument_validation(lib):
+    ok = B.make_shape(2, 8, 2, 64, 256)
+    s = C.byref(ok)
+    f = lib.vsa_dense_decode_fallback
+    assert f(s, FAKE, FAKE, FAKE, FAKE, FAKE, None, FAKE, 1.0, FAKE, None, FAKE, 1 << 40, None) == -1  # count w/o list
+    assert f(s, FAKE, FAKE, FAKE, FAKE, FAKE, None, None, 1.0, FAKE, None, FAKE, 16, None) == -3
+    assert f(s, FAKE, FAKE, FAKE, FAKE, FAKE, None, None, 0.0, FAKE, None, FAKE, 1 << 40, None) == -1
+    assert f(s, FAKE, FAKE, FAKE, FAKE, FAKE, None, None, 1.0, None, None, FAKE, 1 << 40, None) == -1
+    g = lib.vsa_decode_step
+    assert g(s, FAKE, None, FAKE, FAKE, FAKE, FAKE, 4, 16, 1.0, 0.0, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, 1 << 40, None) == -1
+    assert g(s, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, 4, 16, 1.0, 0.0, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, 64, None) == -3
+    h = lib.vsa_decode_step_host
+    assert h(s, None, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, 4, 16, 1.0, 0.0, FAKE, FAKE, None, FAKE, FAKE, FAKE, FAKE,
+             FAKE, 1 << 40, None) == -1
+    assert h(s, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, 4, 16, -2.0, 0.0, FAKE, FAKE, None, FAKE, FAKE, FAKE, FAKE,
+             FAKE, 1 << 40, None) == -1
+    b = lib.vsa_build_page_summaries
+    assert b(s, None, FAKE, FAKE, None, FAKE, None) == -1
+    assert b(s, FAKE, FAKE, FAKE, None, ODD, None) == -4
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(B, "_lib", None)
+    monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "libvsa.so"))
+    with pytest.raises(RuntimeError, match="no fallback"):
+        B.lib()

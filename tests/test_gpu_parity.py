@@ -1,0 +1,220 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same
+seeded bytes.  Discrete results (summaries, routed pages, candidate-derived diagnostics,
+fallback flags and lists) must match bit for bit; floating-point outputs within 1e-2 max-abs
+and 5e-3 relative L2."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2602_13804_b200 import binding as B
+from gpu_runner import check_out, compare, run_gpu
+from util import bits, geometry, host_arrays
+from workloads import WorkloadSpec, config_spec, make_workload
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def spec(**kw):
+    base = dict(name="t", config=9, batch=2, n_q_heads=8, n_kv_heads=2, P=4, K_c=24,
+                seq_lens=(300, 177), needles=3, needle_positions="uniform")
+    base.update(kw)
+    return WorkloadSpec(**base)
+
+
+# ---------------------------------------------------------------- small shapes, every group size
+
+@pytest.mark.parametrize("hq,hkv", [(8, 2), (8, 1), (4, 2), (4, 4), (16, 2)])
+@pytest.mark.parametrize("needles", [3, 0])
+def test_small_ragged(hq, hkv, needles):
+    w = make_workload(spec(n_q_heads=hq, n_kv_heads=hkv, needles=needles), seed=100 + hq * 10 + hkv)
+    stats = compare(w, run_gpu(w))
+    assert 0.0 <= stats["fallback_fraction"] <= 1.0
+
+
+def test_several_tiles_and_ragged_tail():
+    # 5 sequences with lengths around page and 32-page-block boundaries, several scan blocks
+    lens = (16 * 32 * 3 + 5, 16 * 32, 16 * 33 + 15, 1, 16)
+    w = make_workload(spec(batch=5, seq_lens=lens, n_q_heads=8, n_kv_heads=2, P=8, K_c=40, needles=2), seed=201)
+    compare(w, run_gpu(w))
+
+
+def test_routing_fewer_pages_than_P_and_fewer_tokens_than_Kc():
+    w = make_workload(spec(seq_lens=(40, 7), P=8, K_c=128), seed=202)
+    g = run_gpu(w)
+    compare(w, g)
+    assert np.all(g.routed_pages[0, :, 3:] == -1) and np.all(g.routed_pages[1, :, 1:] == -1)
+    assert np.all(np.isposinf(g.diag_sparse["delta"])) and not g.diag_sparse["fallback"].any()
+    assert g.diag_sparse["n_candidates"].reshape(2, 8)[0, 0] == 40
+
+
+def test_engineered_ties_pages_and_tokens():
+    w = make_workload(spec(seq_lens=(160, 96), needles=0, P=3, K_c=20), seed=203)
+    k = w.k_cache.clone()
+    bt = w.block_table
+    for dst in (3, 4, 7):                      # pages 1, 3, 4, 7 of sequence 0 byte-identical
+        k[int(bt[0, dst])] = k[int(bt[0, 1])]
+    k[int(bt[1, 2])] = k[int(bt[1, 0])]        # pages 0 and 2 of sequence 1 identical
+    w.k_cache = k
+    g = run_gpu(w)
+    compare(w, g)
+    # all-equal scores: every page ties, lowest indices win
+    w2 = make_workload(spec(seq_lens=(200, 64), needles=0, P=5, K_c=17), seed=204)
+    w2.k_cache = torch.zeros_like(w2.k_cache)
+    g2 = run_gpu(w2)
+    compare(w2, g2)
+    assert g2.routed_pages[0, 0].tolist() == [0, 1, 2, 3, 4]
+
+
+def test_thresholds_minus_inf_never_and_plus_inf_always():
+    w = make_workload(spec(needles=0), seed=205)
+    g = run_gpu(w, gap_threshold=-math.inf)
+    compare(w, g, gap_threshold=-math.inf)
+    assert len(g.fallback_units) == 0
+    g = run_gpu(w, gap_threshold=math.inf)
+    stats = compare(w, g, gap_threshold=math.inf)
+    assert stats["fallback_fraction"] == 1.0
+
+
+def test_literal_small_epsilon():
+    w = make_workload(spec(seq_lens=(700, 333), needles=4, P=6, K_c=48), seed=206)
+    eps = float(np.float32(1.0 / math.sqrt(128.0)))
+    compare(w, run_gpu(w, epsilon=eps), epsilon=eps)
+
+
+def test_non_native_strides():
+    # cache stored as [pool, page, kv_head, d]: token stride = Hkv * d, head stride = d
+    w = make_workload(spec(), seed=207)
+    wd = w.to(DEV)
+    k_alt = wd.k_cache.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    v_alt = wd.v_cache.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    assert k_alt.stride(2) == 2 * 128 and k_alt.stride(1) == 128
+    wd.k_cache, wd.v_cache = k_alt, v_alt
+    compare(w, run_gpu(wd))
+
+
+def test_dense_baseline_all_units_matches_definition():
+    w = make_workload(spec(seq_lens=(1000, 513), n_q_heads=8, n_kv_heads=2), seed=208).to(DEV)
+    shape = B.shape_of(w.q, w.k_cache, w.block_table)
+    out = torch.full((2, 8, 128), float("nan"), dtype=torch.float32, device=DEV)
+    ws = B.alloc_workspace(shape, 0, 0, B.VSA_WS_DENSE, DEV)
+    B.vsa_dense_decode_fallback(shape, w.q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, None, None, w.epsilon,
+                                out, None, ws)
+    q, K, V, bt, sl = host_arrays(w)
+    dn = oracle.dense(geometry(w), q, K, V, bt, sl, w.epsilon)
+    check_out(out.cpu().numpy(), dn.out, "dense baseline")
+
+
+def test_bad_block_table_entry_and_bad_length_set_status_without_trapping():
+    w = make_workload(spec(seq_lens=(300, 177), needles=0), seed=209).to(DEV)
+    shape = B.shape_of(w.q, w.k_cache, w.block_table)
+    units = 16
+    summ = torch.zeros((shape.num_pool_pages, 2, 128), dtype=torch.bfloat16, device=DEV)
+    B.vsa_build_page_summaries(shape, w.k_cache, w.block_table, w.seq_lens, None, summ)
+    routed = torch.zeros((2, 8, 4), dtype=torch.int32, device=DEV)
+    routed[:, :, :] = torch.tensor([0, 1, 2, 3], dtype=torch.int32, device=DEV)
+    bt = w.block_table.clone()
+    bt[0, 2] = shape.num_pool_pages + 5            # sequence 0 routes through a bad entry
+    sl = w.seq_lens.clone()
+    sl[1] = shape.max_pages_per_seq * 16 + 1       # sequence 1 claims more tokens than its row holds
+    out = torch.full((2, 8, 128), float("nan"), dtype=torch.float32, device=DEV)
+    diag = B.alloc_diag(units, DEV)
+    fl = torch.zeros(units, dtype=torch.int32, device=DEV)
+    fc = torch.zeros(1, dtype=torch.int32, device=DEV)
+    B.vsa_sparse_decode(shape, w.q, w.k_cache, w.v_cache, bt, sl, routed, 4, 24, w.epsilon, w.gap_threshold, out,
+                        diag, fl, fc)
+    torch.cuda.synchronize()
+    d = B.diag_to_dict(diag)
+    assert d["status"].view(2, 8)[0].tolist() == [1] * 8 and d["status"].view(2, 8)[1].tolist() == [2] * 8
+    assert not out.cpu().numpy().any() and int(fc.item()) == 0
+    # routing with the same bad inputs: bad pages score -inf, the over-long sequence routes nothing
+    rp = torch.zeros((2, 8, 4), dtype=torch.int32, device=DEV)
+    ws = B.alloc_workspace(shape, 4, 24, B.VSA_WS_ROUTE, DEV)
+    B.vsa_route_pages(shape, w.q, summ, bt, sl, 4, rp, None, ws)
+    torch.cuda.synchronize()
+    assert 2 not in rp[0].cpu().numpy() and np.all(rp[1].cpu().numpy() == -1)
+
+
+def test_incremental_summary_update_of_the_last_page():
+    w = make_workload(spec(needles=0), seed=210).to(DEV)
+    shape = B.shape_of(w.q, w.k_cache, w.block_table)
+    full = torch.zeros((shape.num_pool_pages, 2, 128), dtype=torch.bfloat16, device=DEV)
+    B.vsa_build_page_summaries(shape, w.k_cache, w.block_table, w.seq_lens, None, full)
+    part = torch.zeros_like(full)
+    first = torch.tensor([(300 - 1) // 16, (177 - 1) // 16], dtype=torch.int32, device=DEV)
+    B.vsa_build_page_summaries(shape, w.k_cache, w.block_table, w.seq_lens, first, part)
+    torch.cuda.synchronize()
+    for b in range(2):
+        last = int(w.block_table[b, int(first[b])])
+        assert torch.equal(part[last], full[last])
+        assert not part[int(w.block_table[b, 0])].any()
+
+
+def test_host_buffer_step_matches_device_step():
+    from paper_2602_13804_b200 import SparsePagedDecoder
+    w = make_workload(spec(seq_lens=(900, 640), needles=2, P=6, K_c=48), seed=211)
+    wd = w.to(DEV)
+    shape = B.shape_of(wd.q, wd.k_cache, wd.block_table)
+    dec = SparsePagedDecoder(shape, 6, 48, w.epsilon, w.gap_threshold, device=DEV, host_io=True)
+    summ = dec.build_summaries(wd.k_cache, wd.block_table, wd.seq_lens)
+    out_dev = dec.step(wd.q, summ, wd.k_cache, wd.v_cache, wd.block_table, wd.seq_lens).clone()
+    q_host = w.q.pin_memory()
+    out_host = dec.step_host(q_host, summ, wd.k_cache, wd.v_cache, wd.block_table, wd.seq_lens)
+    torch.cuda.synchronize()
+    assert torch.equal(out_host, out_dev.cpu())
+    assert torch.equal(dec.diag_host, dec.diag.cpu())
+    q, K, V, bt, sl = host_arrays(w)
+    st = oracle.decode_step(geometry(w), q, K, V, bt, sl, 6, 48, w.epsilon, w.gap_threshold)
+    check_out(out_host.numpy(), st.out, "host step")
+
+
+# ---------------------------------------------------------------- the named configurations
+
+def test_config0_full():
+    w = make_workload(config_spec(0), device=DEV)
+    stats = compare(w, run_gpu(w))
+    assert stats["fallback_fraction"] == 0.0       # planted needles: the support gap is positive
+    eps = float(np.float32(1.0 / math.sqrt(128.0)))  # the literal small temperature, parity only
+    compare(w, run_gpu(w, epsilon=eps), epsilon=eps)
+
+
+def test_config0_round_robin_needles():
+    w = make_workload(config_spec(0, needle_mode="per_qhead_round_robin"), device=DEV)
+    compare(w, run_gpu(w))
+
+
+def test_config1_full_one_layer():
+    w = make_workload(config_spec(1), device=DEV)
+    stats = compare(w, run_gpu(w))
+    assert stats["fallback_fraction"] == 0.0
+
+
+@pytest.mark.parametrize("batch,T", [(1, 131072), (16, 8192), (1, 4096)])
+def test_config2_sweep_points(batch, T):
+    w = make_workload(config_spec(2, batch=batch, T=T), device=DEV, sub=int(math.log2(T)))
+    compare(w, run_gpu(w), dense_sample=16)
+
+
+def test_config3_fallback_regime_reduced():
+    w = make_workload(config_spec(3, batch=4, T=8192, needle_seqs=1), device=DEV)
+    stats = compare(w, run_gpu(w))
+    assert stats["fallback_fraction"] == 0.75
+
+
+def test_config3_full_sampled_dense():
+    w = make_workload(config_spec(3), device=DEV)
+    stats = compare(w, run_gpu(w), dense_sample=24)
+    assert stats["fallback_fraction"] == 0.75      # 12 of 16 sequences have no planted structure
+
+
+def test_config4_ragged_gqa8_reduced():
+    w = make_workload(config_spec(4, batch=6, ragged_T=(300, 5000)), device=DEV)
+    compare(w, run_gpu(w), dense_sample=16)
+
+
+def test_config4_full_sampled_dense():
+    w = make_workload(config_spec(4), device=DEV)
+    compare(w, run_gpu(w), dense_sample=16)
