@@ -158,6 +158,20 @@ int vsa_decode_step(const vsa_shape_t* shape, const void* q, const void* summari
                     size_t ws_bytes, void* stream);
 
 /*
+ * vsa_decode_step with CUDA events recorded on `stream` between its kernels, for per-kernel
+ * timing of exactly the launch sequence the step uses (a measurement aid for the latency
+ * breakdown the paper asks for in Sec. 10.4; results are identical to vsa_decode_step).
+ *   events: host array of 5 cudaEvent_t created by the caller with timing enabled:
+ *   [0] before the page-score scan, [1] after it, [2] after the top-P selection,
+ *   [3] after the fused sparse pass, [4] after the dense fallback pass.
+ */
+int vsa_decode_step_timed(const vsa_shape_t* shape, const void* q, const void* summaries, const void* k_cache,
+                          const void* v_cache, const int32_t* block_table, const int32_t* seq_lens, int32_t P,
+                          int32_t K_c, float epsilon, float gap_threshold, float* out, vsa_diag_t* diag,
+                          int32_t* routed_pages, int32_t* fallback_list, int32_t* fallback_count, void* ws,
+                          size_t ws_bytes, void* stream, void* const* events);
+
+/*
  * The same step for a caller whose per-step tensors live in host memory: copies q_host
  * (bf16 [batch][n_q_heads][head_dim]) to q_dev, runs vsa_decode_step, and copies the results
  * back into out_host (fp32 [batch][n_q_heads][head_dim]) and diag_host ([batch][n_q_heads],

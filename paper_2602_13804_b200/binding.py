@@ -67,10 +67,13 @@ def lib() -> C.CDLL:
         _lib.vsa_sparse_decode.argtypes = [shp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, vp, vp, vp, vp, vp, sz, vp]
         _lib.vsa_dense_decode_fallback.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, f32, vp, vp, vp, sz, vp]
         _lib.vsa_decode_step.argtypes = [shp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, vp, vp, vp, vp, vp, vp, sz, vp]
+        _lib.vsa_decode_step_timed.argtypes = [shp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, vp, vp, vp, vp, vp, vp, sz,
+                                               vp, C.POINTER(C.c_void_p)]
         _lib.vsa_decode_step_host.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32,
                                               vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         for name in ("vsa_build_page_summaries", "vsa_route_pages", "vsa_sparse_decode",
-                     "vsa_dense_decode_fallback", "vsa_decode_step", "vsa_decode_step_host"):
+                     "vsa_dense_decode_fallback", "vsa_decode_step", "vsa_decode_step_timed",
+                     "vsa_decode_step_host"):
             getattr(_lib, name).restype = C.c_int
     return _lib
 
@@ -154,6 +157,21 @@ def vsa_decode_step(shape, q, summaries, k_cache, v_cache, block_table, seq_lens
                                  _ptr(diag), _ptr(routed_pages), _ptr(fallback_list), _ptr(fallback_count),
                                  _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
            "vsa_decode_step")
+
+
+def vsa_decode_step_timed(shape, q, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon,
+                          gap_threshold, out, diag, routed_pages, fallback_list, fallback_count, ws, events,
+                          stream=None) -> None:
+    """`events`: 5 torch.cuda.Event(enable_timing=True) that have been recorded once (so that their
+    CUDA handles exist); they are re-recorded between the kernels of the step."""
+    handles = (C.c_void_p * 5)(*[e.cuda_event for e in events])
+    _check(lib().vsa_decode_step_timed(C.byref(shape), _ptr(q), _ptr(summaries), _ptr(k_cache), _ptr(v_cache),
+                                       _ptr(block_table), _ptr(seq_lens), P, K_c, epsilon, gap_threshold,
+                                       _ptr(out), _ptr(diag), _ptr(routed_pages), _ptr(fallback_list),
+                                       _ptr(fallback_count), _ptr(ws),
+                                       0 if ws is None else ws.numel() * ws.element_size(), _stream(stream),
+                                       handles),
+           "vsa_decode_step_timed")
 
 
 def vsa_decode_step_host(shape, q_host, q_dev, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c,

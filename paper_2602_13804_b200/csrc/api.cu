@@ -168,11 +168,11 @@ int vsa_dense_decode_fallback(const vsa_shape_t* shape, const void* q, const voi
                                      epsilon, out, diag, ws, (cudaStream_t)stream));
 }
 
-int vsa_decode_step(const vsa_shape_t* shape, const void* q, const void* summaries, const void* k_cache,
-                    const void* v_cache, const int32_t* block_table, const int32_t* seq_lens, int32_t P,
-                    int32_t K_c, float epsilon, float gap_threshold, float* out, vsa_diag_t* diag,
-                    int32_t* routed_pages, int32_t* fallback_list, int32_t* fallback_count, void* ws,
-                    size_t ws_bytes, void* stream)
+static int decode_step_impl(const vsa_shape_t* shape, const void* q, const void* summaries, const void* k_cache,
+                            const void* v_cache, const int32_t* block_table, const int32_t* seq_lens, int32_t P,
+                            int32_t K_c, float epsilon, float gap_threshold, float* out, vsa_diag_t* diag,
+                            int32_t* routed_pages, int32_t* fallback_list, int32_t* fallback_count, void* ws,
+                            size_t ws_bytes, void* stream, void* const* events)
 {
     Geometry g;
     int rc = make_geometry(shape, &g);
@@ -187,17 +187,51 @@ int vsa_decode_step(const vsa_shape_t* shape, const void* q, const void* summari
         return VSA_ERR_MISALIGNED;
     if (ws_bytes < step_route_part(g) + vsa::dense_workspace_bytes(g)) return VSA_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t st = (cudaStream_t)stream;
+    cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+    if (events)
+        for (int i = 0; i < 5; ++i) {
+            if (!events[i]) return VSA_ERR_INVALID_ARGUMENT;
+            ev[i] = (cudaEvent_t)events[i];
+        }
     void* ws_dense = (char*)ws + step_route_part(g);
+    if (ev[0] && cudaEventRecord(ev[0], st) != cudaSuccess) return VSA_ERR_CUDA;
     // the scan kernel clears fallback_count, so the step needs no separate memset for it
     cudaError_t e = vsa::launch_route(g, q, summaries, block_table, seq_lens, P, routed_pages, nullptr, ws,
-                                      fallback_count, st);
+                                      fallback_count, st, ev[1]);
     if (e != cudaSuccess) return VSA_ERR_CUDA;
+    if (ev[2] && cudaEventRecord(ev[2], st) != cudaSuccess) return VSA_ERR_CUDA;
     e = vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, routed_pages, P, K_c, epsilon,
                            gap_threshold, out, diag, fallback_list, fallback_count, st);
     if (e != cudaSuccess) return VSA_ERR_CUDA;
+    if (ev[3] && cudaEventRecord(ev[3], st) != cudaSuccess) return VSA_ERR_CUDA;
     e = vsa::launch_dense(g, q, k_cache, v_cache, block_table, seq_lens, fallback_list, fallback_count, epsilon,
                           out, diag, ws_dense, st);
-    return cuda_rc(e);
+    if (e != cudaSuccess) return VSA_ERR_CUDA;
+    if (ev[4] && cudaEventRecord(ev[4], st) != cudaSuccess) return VSA_ERR_CUDA;
+    return VSA_OK;
+}
+
+int vsa_decode_step(const vsa_shape_t* shape, const void* q, const void* summaries, const void* k_cache,
+                    const void* v_cache, const int32_t* block_table, const int32_t* seq_lens, int32_t P,
+                    int32_t K_c, float epsilon, float gap_threshold, float* out, vsa_diag_t* diag,
+                    int32_t* routed_pages, int32_t* fallback_list, int32_t* fallback_count, void* ws,
+                    size_t ws_bytes, void* stream)
+{
+    return decode_step_impl(shape, q, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon,
+                            gap_threshold, out, diag, routed_pages, fallback_list, fallback_count, ws, ws_bytes,
+                            stream, nullptr);
+}
+
+int vsa_decode_step_timed(const vsa_shape_t* shape, const void* q, const void* summaries, const void* k_cache,
+                          const void* v_cache, const int32_t* block_table, const int32_t* seq_lens, int32_t P,
+                          int32_t K_c, float epsilon, float gap_threshold, float* out, vsa_diag_t* diag,
+                          int32_t* routed_pages, int32_t* fallback_list, int32_t* fallback_count, void* ws,
+                          size_t ws_bytes, void* stream, void* const* events)
+{
+    if (!events) return VSA_ERR_INVALID_ARGUMENT;
+    return decode_step_impl(shape, q, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon,
+                            gap_threshold, out, diag, routed_pages, fallback_list, fallback_count, ws, ws_bytes,
+                            stream, events);
 }
 
 int vsa_decode_step_host(const vsa_shape_t* shape, const void* q_host, void* q_dev, const void* summaries,

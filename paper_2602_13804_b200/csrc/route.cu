@@ -197,7 +197,7 @@ size_t route_workspace_bytes(const Geometry& g)
 
 cudaError_t launch_route(const Geometry& g, const void* q, const void* summaries, const int32_t* block_table,
                          const int32_t* seq_lens, int P, int32_t* routed_pages, float* routed_scores,
-                         void* ws, int32_t* zero_word, cudaStream_t stream)
+                         void* ws, int32_t* zero_word, cudaStream_t stream, cudaEvent_t after_scan)
 {
     float* scores = (float*)ws;
     const int bpw = scan_blocks_per_warp(g);
@@ -215,6 +215,7 @@ cudaError_t launch_route(const Geometry& g, const void* q, const void* summaries
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
+    if (after_scan && (e = cudaEventRecord(after_scan, stream)) != cudaSuccess) return e;
 
     const size_t smem = select_smem_bytes(g, P);
     if (smem > 48 * 1024) {

@@ -24,7 +24,7 @@ cudaError_t launch_build_summaries(const Geometry& g, const void* k_cache, const
 size_t route_workspace_bytes(const Geometry& g);
 cudaError_t launch_route(const Geometry& g, const void* q, const void* summaries, const int32_t* block_table,
                          const int32_t* seq_lens, int P, int32_t* routed_pages, float* routed_scores,
-                         void* ws, int32_t* zero_word, cudaStream_t stream);
+                         void* ws, int32_t* zero_word, cudaStream_t stream, cudaEvent_t after_scan = nullptr);
 
 // ---- fused sparse pass ------------------------------------------------------------------------
 cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache, const void* v_cache,
