@@ -313,6 +313,9 @@ def run_ours(args):
             for _ in range(2):
                 step()
             for _ in range(n_rep):
+                # hold the GPU for ~3 ms so that the host enqueues the whole step ahead of it:
+                # the events then bracket kernels that run back to back, not launch gaps
+                torch.cuda._sleep(6_000_000)
                 for i in range(L):
                     w, s = layers[i % distinct], summaries[i % distinct]
                     B.vsa_decode_step_timed(shape, w.q, s, w.k_cache, w.v_cache, w.block_table, w.seq_lens, P, K_c,

@@ -31,6 +31,7 @@ int make_geometry(const vsa_shape_t* s, Geometry* g)
     if (s->max_pages_per_seq > kMaxPagesPerSeq) return VSA_ERR_UNSUPPORTED_SHAPE;
     if (s->num_pool_pages > 0x7fffffffLL) return VSA_ERR_UNSUPPORTED_SHAPE;
     if ((long long)s->batch * s->n_q_heads > 0x3fffffffLL) return VSA_ERR_UNSUPPORTED_SHAPE;
+    if ((long long)s->batch * s->n_kv_heads > 8192) return VSA_ERR_UNSUPPORTED_SHAPE;
     g->batch = s->batch;
     g->n_q_heads = s->n_q_heads;
     g->n_kv_heads = s->n_kv_heads;
@@ -123,8 +124,9 @@ int vsa_route_pages(const vsa_shape_t* shape, const void* q, const void* summari
     if (!q || !summaries || !block_table || !seq_lens || !routed_pages || !ws) return VSA_ERR_INVALID_ARGUMENT;
     if (!aligned16(q) || !aligned16(summaries) || !aligned16(ws)) return VSA_ERR_MISALIGNED;
     if (ws_bytes < vsa::route_workspace_bytes(g)) return VSA_ERR_WORKSPACE_TOO_SMALL;
-    return cuda_rc(vsa::launch_route(g, q, summaries, block_table, seq_lens, P, routed_pages, routed_scores, ws,
-                                     nullptr, (cudaStream_t)stream));
+    cudaError_t e = vsa::launch_route_scan(g, q, summaries, block_table, seq_lens, ws, nullptr, (cudaStream_t)stream);
+    if (e != cudaSuccess) return VSA_ERR_CUDA;
+    return cuda_rc(vsa::launch_route_select(g, ws, seq_lens, P, routed_pages, routed_scores, (cudaStream_t)stream));
 }
 
 int vsa_sparse_decode(const vsa_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,
@@ -147,8 +149,8 @@ int vsa_sparse_decode(const vsa_shape_t* shape, const void* q, const void* k_cac
     cudaStream_t st = (cudaStream_t)stream;
     cudaError_t e = cudaMemsetAsync(fallback_count, 0, sizeof(int32_t), st);
     if (e != cudaSuccess) return VSA_ERR_CUDA;
-    return cuda_rc(vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, routed_pages, P, K_c,
-                                      epsilon, gap_threshold, out, diag, fallback_list, fallback_count, st));
+    return cuda_rc(vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, (int32_t*)routed_pages, nullptr,
+                                      P, K_c, epsilon, gap_threshold, out, diag, fallback_list, fallback_count, st));
 }
 
 int vsa_dense_decode_fallback(const vsa_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,
@@ -196,12 +198,13 @@ static int decode_step_impl(const vsa_shape_t* shape, const void* q, const void*
     void* ws_dense = (char*)ws + step_route_part(g);
     if (ev[0] && cudaEventRecord(ev[0], st) != cudaSuccess) return VSA_ERR_CUDA;
     // the scan kernel clears fallback_count, so the step needs no separate memset for it
-    cudaError_t e = vsa::launch_route(g, q, summaries, block_table, seq_lens, P, routed_pages, nullptr, ws,
-                                      fallback_count, st, ev[1]);
+    cudaError_t e = vsa::launch_route_scan(g, q, summaries, block_table, seq_lens, ws, fallback_count, st);
     if (e != cudaSuccess) return VSA_ERR_CUDA;
+    if (ev[1] && cudaEventRecord(ev[1], st) != cudaSuccess) return VSA_ERR_CUDA;
+    // the top-P selection runs inside the fused kernel, on the scores the scan left in ws
     if (ev[2] && cudaEventRecord(ev[2], st) != cudaSuccess) return VSA_ERR_CUDA;
-    e = vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, routed_pages, P, K_c, epsilon,
-                           gap_threshold, out, diag, fallback_list, fallback_count, st);
+    e = vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, routed_pages, (const float*)ws, P, K_c,
+                           epsilon, gap_threshold, out, diag, fallback_list, fallback_count, st);
     if (e != cudaSuccess) return VSA_ERR_CUDA;
     if (ev[3] && cudaEventRecord(ev[3], st) != cudaSuccess) return VSA_ERR_CUDA;
     e = vsa::launch_dense(g, q, k_cache, v_cache, block_table, seq_lens, fallback_list, fallback_count, epsilon,

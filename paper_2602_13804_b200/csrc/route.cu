@@ -8,6 +8,7 @@
 
 #include "vsa_device.cuh"
 #include "vsa_launch.h"
+#include "vsa_select.cuh"
 
 namespace vsa {
 
@@ -107,76 +108,20 @@ __global__ void route_select_kernel(Geometry geo, const float* __restrict__ scor
                                     int32_t* __restrict__ routed_pages, float* __restrict__ routed_scores)
 {
     extern __shared__ uint32_t smem[];
-    const int max_pages = geo.max_pages;
-    uint32_t* keys = smem;                                  // [max_pages]
-    uint32_t* hist = keys + max_pages;                      // [256]
-    uint32_t* scratch = hist + 256;                         // [8]
-    uint32_t* warp_counts = scratch + 8;                    // [40]
-    uint32_t* win_key = warp_counts + 40;                   // [P]
-    int32_t* win_idx = (int32_t*)(win_key + P);             // [P]
-    uint8_t* take = (uint8_t*)(win_idx + P);                // [max_pages]
-
+    const PageSelectSmem s = carve_page_select(smem, geo.max_pages, P);
     const int h = blockIdx.x, b = blockIdx.y;
     const long long unit = (long long)b * geo.n_q_heads + h;
     const int T = seq_lens[b];
-    const bool ok = T > 0 && T <= max_pages * kPageSize;
+    const bool ok = T > 0 && T <= geo.max_pages * kPageSize;
     const int n = ok ? (T + kPageSize - 1) / kPageSize : 0;
-    const int K = min(P, n);
-    const float* sc = scores + unit * max_pages;
-
-    for (int i = threadIdx.x; i < n; i += blockDim.x) keys[i] = float_to_key(sc[i]);
-    if (threadIdx.x == 0) scratch[4] = 0;   // winner counter
-    __syncthreads();
-
-    if (n > P) {
-        const SelectResult r = block_select_kth(keys, n, K, hist, scratch);
-        const int need = K - r.n_greater;
-        const bool straddle = r.n_equal > need;
-        if (straddle) {
-            for (int i = threadIdx.x; i < n; i += blockDim.x) take[i] = 0;
-            __syncthreads();
-            block_mark_first_equal(keys, n, r.kth, need, take, warp_counts);
-            __syncthreads();
-        }
-        for (int i = threadIdx.x; i < n; i += blockDim.x) {
-            const uint32_t key = keys[i];
-            if (key > r.kth || (key == r.kth && (!straddle || take[i]))) {
-                const int slot = (int)atomicAdd(&scratch[4], 1u);
-                win_key[slot] = key;
-                win_idx[slot] = i;
-            }
-        }
-    } else {
-        for (int i = threadIdx.x; i < n; i += blockDim.x) {
-            win_key[i] = keys[i];
-            win_idx[i] = i;
-        }
-    }
-    __syncthreads();
-
-    // order the K winners (all (key, index) pairs are distinct) and write them best first
+    const int K = select_top_pages(scores + unit * geo.max_pages, n, P, s);
     for (int t = threadIdx.x; t < P; t += blockDim.x) {
-        if (t < K) {
-            const uint32_t key = win_key[t];
-            const int idx = win_idx[t];
-            int rank = 0;
-            for (int j = 0; j < K; ++j) {
-                const uint32_t kj = win_key[j];
-                rank += (kj > key) || (kj == key && win_idx[j] < idx);
-            }
-            routed_pages[unit * P + rank] = idx;
-            if (routed_scores) routed_scores[unit * P + rank] = key_to_float(key);
-        } else {
-            routed_pages[unit * P + t] = -1;
-            if (routed_scores) routed_scores[unit * P + t] = -INFINITY;
-        }
+        routed_pages[unit * P + t] = t < K ? s.win_idx[t] : -1;
+        if (routed_scores) routed_scores[unit * P + t] = t < K ? key_to_float(s.win_key[t]) : -INFINITY;
     }
 }
 
-size_t select_smem_bytes(const Geometry& g, int P)
-{
-    return (size_t)g.max_pages * 4 + 256 * 4 + 8 * 4 + 40 * 4 + (size_t)P * 8 + (size_t)g.max_pages + 16;
-}
+size_t select_smem_bytes(const Geometry& g, int P) { return (size_t)select_pages_words(g.max_pages, P) * 4; }
 
 int scan_blocks_per_warp(const Geometry& g)
 {
@@ -195,9 +140,8 @@ size_t route_workspace_bytes(const Geometry& g)
     return (size_t)g.batch * g.n_q_heads * g.max_pages * sizeof(float);
 }
 
-cudaError_t launch_route(const Geometry& g, const void* q, const void* summaries, const int32_t* block_table,
-                         const int32_t* seq_lens, int P, int32_t* routed_pages, float* routed_scores,
-                         void* ws, int32_t* zero_word, cudaStream_t stream, cudaEvent_t after_scan)
+cudaError_t launch_route_scan(const Geometry& g, const void* q, const void* summaries, const int32_t* block_table,
+                              const int32_t* seq_lens, void* ws, int32_t* zero_word, cudaStream_t stream)
 {
     float* scores = (float*)ws;
     const int bpw = scan_blocks_per_warp(g);
@@ -213,18 +157,20 @@ cudaError_t launch_route(const Geometry& g, const void* q, const void* summaries
         case 8: route_scan_kernel<8><<<grid, kScanThreads, 0, stream>>>(g, qq, ss, block_table, seq_lens, scores, bpw, zero_word); break;
         default: return cudaErrorInvalidValue;
     }
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    if (after_scan && (e = cudaEventRecord(after_scan, stream)) != cudaSuccess) return e;
+    return cudaGetLastError();
+}
 
+cudaError_t launch_route_select(const Geometry& g, const void* ws, const int32_t* seq_lens, int P,
+                                int32_t* routed_pages, float* routed_scores, cudaStream_t stream)
+{
     const size_t smem = select_smem_bytes(g, P);
     if (smem > 48 * 1024) {
-        e = cudaFuncSetAttribute(route_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(route_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    const int threads = g.max_pages <= 1024 ? 256 : 1024;
+    const int threads = g.max_pages <= 4096 ? 256 : 512;
     route_select_kernel<<<dim3((unsigned)g.n_q_heads, (unsigned)g.batch), threads, smem, stream>>>(
-        g, scores, seq_lens, P, routed_pages, routed_scores);
+        g, (const float*)ws, seq_lens, P, routed_pages, routed_scores);
     return cudaGetLastError();
 }
 

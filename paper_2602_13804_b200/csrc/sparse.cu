@@ -1,5 +1,6 @@
 // Fused sparse pass for one (sequence, query head) unit per thread block (paper Sec. 7 steps 2-4,
 // Sec. 8 gap statistic, Cor. 1 leakage bound, Sec. 10.3 fallback flag):
+//   [top-P page selection from the page scores, when fused with routing] ->
 //   score every valid token of the routed pages -> exact top-K_c -> softmax weights at temperature
 //   epsilon -> weighted sum of the candidates' value rows -> diagnostics.
 // The candidate list and the weights live in shared memory and registers only.
@@ -8,6 +9,7 @@
 
 #include "vsa_device.cuh"
 #include "vsa_launch.h"
+#include "vsa_select.cuh"
 
 namespace vsa {
 
@@ -17,33 +19,35 @@ constexpr int kSparseThreads = 256;
 constexpr int kSparseWarps = kSparseThreads / 32;
 constexpr int kGroups = 2 * kSparseWarps;   // half-warps per block
 
-struct SparseSmem {
-    int32_t* page_l;      // [P] routed logical pages, ascending, invalid entries last
-    int32_t* page_phys;   // [P]
-    uint32_t* keys;       // [P * 16] token score keys, array index = 16 * slot + token (position order)
-    int32_t* sel;         // [K_c] array indices of the candidates, ascending
-    uint32_t* hist;       // [256]
-    uint32_t* scratch;    // [16]
-    uint32_t* warp_counts;   // [40]
-    float* red;           // [warps][128]
-    float* zred;          // [warps]
-    uint8_t* take;        // [P * 16]
+// token-phase shared memory, in 4-byte words, after the two page arrays
+__host__ __device__ constexpr int token_phase_words(int P, int K_c)
+{
+    return P * kPageSize /*keys*/ + (P * kPageSize + 3) / 4 /*take*/ + K_c /*sel*/ + 256 + 16 + 72 + kTopkList +
+           kSparseWarps * kHeadDim + kSparseWarps + 4;
+}
+
+struct TokenSmem {
+    uint32_t* keys;   // [P * 16] token score keys, array index = 16 * slot + token (position order)
+    uint8_t* take;    // [P * 16]
+    int32_t* sel;     // [K_c] array indices of the candidates, ascending
+    TopkScratch ts;
+    float* red;       // [warps][128]
+    float* zred;      // [warps]
 };
 
-__device__ __forceinline__ SparseSmem carve(uint32_t* base, int P, int K_c)
+__device__ __forceinline__ TokenSmem carve_tokens(uint32_t* base, int P, int K_c)
 {
-    SparseSmem s;
+    TokenSmem s;
     const int N = P * kPageSize;
-    s.page_l = (int32_t*)base;
-    s.page_phys = s.page_l + P;
-    s.keys = (uint32_t*)(s.page_phys + P);
-    s.sel = (int32_t*)(s.keys + N);
-    s.hist = (uint32_t*)(s.sel + K_c);
-    s.scratch = s.hist + 256;
-    s.warp_counts = s.scratch + 16;
-    s.red = (float*)(s.warp_counts + 40);
+    s.keys = base;
+    s.take = (uint8_t*)(s.keys + N);
+    s.sel = (int32_t*)(s.keys + N + (N + 3) / 4);
+    s.ts.hist = (uint32_t*)(s.sel + K_c);
+    s.ts.misc = s.ts.hist + 256;
+    s.ts.wred = s.ts.misc + 16;
+    s.ts.list = (int32_t*)(s.ts.wred + 72);
+    s.red = (float*)(s.ts.list + kTopkList);
     s.zred = s.red + kSparseWarps * kHeadDim;
-    s.take = (uint8_t*)(s.zred + kSparseWarps);
     return s;
 }
 
@@ -60,16 +64,21 @@ __device__ __forceinline__ void write_failed_unit(float* out, vsa_diag_t* diag, 
     }
 }
 
-__global__ void __launch_bounds__(kSparseThreads)
+// page_scores == nullptr: routed_pages is an input.
+// page_scores != nullptr: the unit's top-P pages are selected here from page_scores[unit][0..n_b)
+//                         and written to routed_pages (best first, -1 padded) as well.
+__global__ void __launch_bounds__(kSparseThreads, 2)
 sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* __restrict__ k_cache,
                      const uint16_t* __restrict__ v_cache, const int32_t* __restrict__ block_table,
-                     const int32_t* __restrict__ seq_lens, const int32_t* __restrict__ routed_pages, int P,
-                     int K_c, float epsilon, float gap_threshold, float* __restrict__ out,
-                     vsa_diag_t* __restrict__ diag, int32_t* __restrict__ fallback_list,
+                     const int32_t* __restrict__ seq_lens, int32_t* __restrict__ routed_pages,
+                     const float* __restrict__ page_scores, int P, int K_c, float epsilon, float gap_threshold,
+                     float* __restrict__ out, vsa_diag_t* __restrict__ diag, int32_t* __restrict__ fallback_list,
                      int32_t* __restrict__ fallback_count)
 {
     extern __shared__ uint32_t smem_raw[];
-    const SparseSmem sm = carve(smem_raw, P, K_c);
+    int32_t* page_l = (int32_t*)smem_raw;   // [P] routed logical pages, ascending, invalid entries last
+    int32_t* page_phys = page_l + P;        // [P]
+    uint32_t* region = smem_raw + 2 * P;    // page-selection scratch first, token-phase arrays afterwards
     const int N = P * kPageSize;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, c = lane & 15, gi = lane >> 4;
     const long long unit = blockIdx.x;
@@ -77,27 +86,33 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     const int T = seq_lens[b];
     if (T <= 0 || T > geo.max_pages * kPageSize) {
         write_failed_unit(out, diag, unit, VSA_UNIT_BAD_LENGTH);
+        if (page_scores)
+            for (int t = tid; t < P; t += kSparseThreads) routed_pages[unit * P + t] = -1;
         return;
     }
     const int nb = (T + kPageSize - 1) / kPageSize;
 
-    // ---- routed pages: validate, sort by logical page so that array order = position order ----
-    int32_t* raw = (int32_t*)sm.keys;   // staging; keys[] (16 P words) is initialised further down
-    for (int t = tid; t < P; t += kSparseThreads) {
-        const int l = routed_pages[unit * P + t];
-        raw[t] = (l >= 0 && l < nb) ? l : INT_MAX;
-    }
-    __syncthreads();
-    for (int t = tid; t < P; t += kSparseThreads) {
-        const int l = raw[t];
-        int rank = 0;
-        for (int j = 0; j < P; ++j) rank += (raw[j] < l) || (raw[j] == l && j < t);
-        sm.page_l[rank] = l;
+    // ---- routed pages -> page_l[] sorted by logical page, so that array order = position order ----
+    int32_t* raw;   // staging of the unsorted page list inside `region` (dead before the token phase)
+    if (page_scores) {
+        const PageSelectSmem ps = carve_page_select(region, geo.max_pages, P);
+        const int K = select_top_pages(page_scores + unit * geo.max_pages, nb, P, ps);
+        for (int t = tid; t < P; t += kSparseThreads) routed_pages[unit * P + t] = t < K ? ps.win_idx[t] : -1;
+        raw = ps.tmp_idx;   // reuse: tmp_idx is dead after select_top_pages
+        for (int t = tid; t < P; t += kSparseThreads) raw[t] = t < K ? ps.win_idx[t] : INT_MAX;
+    } else {
+        raw = (int32_t*)region;
+        for (int t = tid; t < P; t += kSparseThreads) {
+            const int l = routed_pages[unit * P + t];
+            raw[t] = (l >= 0 && l < nb) ? l : INT_MAX;
+        }
     }
     __syncthreads();
     int bad = 0;
     for (int t = tid; t < P; t += kSparseThreads) {
-        const int l = sm.page_l[t];
+        const int l = raw[t];
+        int rank = 0;
+        for (int j = 0; j < P; ++j) rank += (raw[j] < l) || (raw[j] == l && j < t);
         int phys = -1;
         if (l != INT_MAX) {
             phys = block_table[(long long)b * geo.max_pages + l];
@@ -106,14 +121,16 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                 bad = 1;
             }
         }
-        sm.page_phys[t] = phys;
+        page_l[rank] = l;
+        page_phys[rank] = phys;
     }
-    const int np = __syncthreads_count(tid < P && sm.page_l[tid < P ? tid : 0] != INT_MAX);
+    // (P <= 128 < blockDim.x: thread t < P owns slot t in the count below)
+    const int np = __syncthreads_count(tid < P && raw[tid < P ? tid : 0] != INT_MAX);
     if (__syncthreads_or(bad)) {
         write_failed_unit(out, diag, unit, VSA_UNIT_BAD_PAGE);
         return;
     }
-    // (P <= 128 < blockDim.x, so the count above saw every slot)
+    const TokenSmem sm = carve_tokens(region, P, K_c);
     for (int i = tid; i < N; i += kSparseThreads) {
         sm.keys[i] = 0u;
         sm.take[i] = 0;
@@ -131,7 +148,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         const bool active = slot < np;
         uint4 rows[kPageSize];
         if (active) {
-            const uint16_t* src = k_cache + (long long)sm.page_phys[slot] * geo.page_stride +
+            const uint16_t* src = k_cache + (long long)page_phys[slot] * geo.page_stride +
                                   (long long)g * geo.head_stride + c * 8;
 #pragma unroll
             for (int t = 0; t < kPageSize; ++t) rows[t] = ld_nc_16B(src + (long long)t * geo.token_stride);
@@ -147,31 +164,27 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
             vals[t] = chunk_partial(qf, kf);
         }
         const float s = reduce_scatter16(vals, c);   // lane c: score of token c of the page
-        if (active && sm.page_l[slot] * kPageSize + c < T) sm.keys[slot * kPageSize + c] = float_to_key(s);
+        if (active && page_l[slot] * kPageSize + c < T) sm.keys[slot * kPageSize + c] = float_to_key(s);
     }
     // number of valid scored tokens
     if (warp == 0) {
         int cnt = 0;
-        for (int t = lane; t < np; t += 32) cnt += min(kPageSize, T - sm.page_l[t] * kPageSize);
+        for (int t = lane; t < np; t += 32) cnt += min(kPageSize, T - page_l[t] * kPageSize);
 #pragma unroll
         for (int off = 16; off; off >>= 1) cnt += __shfl_xor_sync(kFullMask, cnt, off);
-        if (lane == 0) sm.scratch[8] = (uint32_t)cnt;
+        if (lane == 0) sm.ts.misc[9] = (uint32_t)cnt;
     }
     __syncthreads();
-    const int nv = (int)sm.scratch[8];
+    const int nv = (int)sm.ts.misc[9];
     const int ns = min(K_c, nv);
 
-    // ---- exact top-ns; the (ns+1)-th element is the best rejected token ----
+    // ---- exact top-(ns+1): its last element is the best rejected token, the rest are the candidates ----
     uint32_t out_key = 0u;
-    bool has_rejected = nv > ns;
+    const bool has_rejected = nv > ns;
     if (has_rejected) {
-        const SelectResult r = block_select_kth(sm.keys, N, ns + 1, sm.hist, sm.scratch);
-        out_key = r.kth;
-        const int need = ns - r.n_greater;   // how many of the tied-with-cut elements still get in
-        if (need > 0) block_mark_first_equal(sm.keys, N, r.kth, need, sm.take, sm.warp_counts);
-        __syncthreads();
-        for (int i = tid; i < N; i += kSparseThreads)
-            if (sm.keys[i] > out_key) sm.take[i] = 1;
+        const TopkResult r = block_topk_mark(sm.keys, N, ns + 1, sm.take, sm.ts);
+        out_key = r.kth_key;
+        if (tid == 0) sm.take[r.kth_idx] = 0;
     } else {
         for (int i = tid; i < N; i += kSparseThreads)
             if (sm.keys[i] != 0u) sm.take[i] = 1;
@@ -197,20 +210,20 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
             a2 = n2;
         }
         if (lane == 0) {
-            sm.warp_counts[2 * warp] = a1;
-            sm.warp_counts[2 * warp + 1] = a2;
+            sm.ts.wred[2 * warp] = a1;
+            sm.ts.wred[2 * warp + 1] = a2;
         }
     }
     __syncthreads();
     uint32_t key1 = 0u, key2 = 0u;
 #pragma unroll
     for (int w = 0; w < kSparseWarps; ++w) {
-        const uint32_t b1 = sm.warp_counts[2 * w], b2 = sm.warp_counts[2 * w + 1];
+        const uint32_t b1 = sm.ts.wred[2 * w], b2 = sm.ts.wred[2 * w + 1];
         const uint32_t n1 = max(key1, b1), n2 = max(min(key1, b1), max(key2, b2));
         key1 = n1;
         key2 = n2;
     }
-    __syncthreads();   // warp_counts is reused below
+    __syncthreads();   // wred is reused below
 
     // ---- ordered compaction of the candidates: sel[] ascending in array (= position) order ----
     {
@@ -224,10 +237,10 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
             const int o = __shfl_up_sync(kFullMask, incl, off);
             if (lane >= off) incl += o;
         }
-        if (lane == 31) sm.warp_counts[warp] = (uint32_t)incl;
+        if (lane == 31) sm.ts.wred[warp] = (uint32_t)incl;
         __syncthreads();
         int base = 0;
-        for (int w = 0; w < warp; ++w) base += (int)sm.warp_counts[w];
+        for (int w = 0; w < warp; ++w) base += (int)sm.ts.wred[w];
         int o = base + incl - cnt;
         for (int i = lo; i < hi; ++i)
             if (sm.take[i]) sm.sel[o++] = i;
@@ -241,7 +254,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[e] = 0.0f;
     const int gidx = warp * 2 + gi;
-    constexpr int UNR = 4;
+    constexpr int UNR = 8;
     for (int j0 = gidx; j0 < ns; j0 += kGroups * UNR) {
         uint4 rows[UNR];
         float w[UNR];
@@ -253,7 +266,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
             if (j < ns) {
                 const int i = sm.sel[j];
                 const int slot = i >> 4, t = i & 15;
-                rows[u] = ld_nc_16B(v_cache + (long long)sm.page_phys[slot] * geo.page_stride +
+                rows[u] = ld_nc_16B(v_cache + (long long)page_phys[slot] * geo.page_stride +
                                     (long long)g * geo.head_stride + (long long)t * geo.token_stride + c * 8);
                 w[u] = exp2f((key_to_float(sm.keys[i]) - s1) * scale);
             }
@@ -304,21 +317,21 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     }
 }
 
-size_t sparse_smem_bytes(int P, int K_c)
+size_t sparse_smem_bytes(const Geometry& g, int P, int K_c, bool fused)
 {
-    const size_t N = (size_t)P * kPageSize;
-    return (size_t)P * 8 + N * 4 + (size_t)K_c * 4 + 256 * 4 + 16 * 4 + 40 * 4 +
-           (size_t)kSparseWarps * kHeadDim * 4 + kSparseWarps * 4 + N + 16;
+    int words = token_phase_words(P, K_c);
+    if (fused && select_pages_words(g.max_pages, P) > words) words = select_pages_words(g.max_pages, P);
+    return (size_t)(2 * P + words) * 4 + 16;
 }
 
 }  // namespace
 
 cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache, const void* v_cache,
-                          const int32_t* block_table, const int32_t* seq_lens, const int32_t* routed_pages,
-                          int P, int K_c, float epsilon, float gap_threshold, float* out, vsa_diag_t* diag,
-                          int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream)
+                          const int32_t* block_table, const int32_t* seq_lens, int32_t* routed_pages,
+                          const float* page_scores, int P, int K_c, float epsilon, float gap_threshold, float* out,
+                          vsa_diag_t* diag, int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream)
 {
-    const size_t smem = sparse_smem_bytes(P, K_c);
+    const size_t smem = sparse_smem_bytes(g, P, K_c, page_scores != nullptr);
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(sparse_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)smem);
@@ -327,7 +340,7 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
     const unsigned units = (unsigned)(g.batch * g.n_q_heads);
     sparse_decode_kernel<<<units, kSparseThreads, smem, stream>>>(
         g, (const uint16_t*)q, (const uint16_t*)k_cache, (const uint16_t*)v_cache, block_table, seq_lens,
-        routed_pages, P, K_c, epsilon, gap_threshold, out, diag, fallback_list, fallback_count);
+        routed_pages, page_scores, P, K_c, epsilon, gap_threshold, out, diag, fallback_list, fallback_count);
     return cudaGetLastError();
 }
 

@@ -197,7 +197,8 @@ __device__ __forceinline__ SelectResult block_select_kth(const uint32_t* keys, i
 // i at once: marks take[i] = 1 for the first `need` of them.  Runs tile by tile; only called when
 // a tie straddles the cut.  warp_counts: >= blockDim.x / 32 + 1 words of shared memory.
 __device__ __forceinline__ void block_mark_first_equal(const uint32_t* keys, int n, uint32_t kth, int need,
-                                                       uint8_t* take, uint32_t* warp_counts)
+                                                       uint8_t* take, uint32_t* warp_counts,
+                                                       uint32_t* last_taken = nullptr)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     int base = 0;
@@ -214,11 +215,157 @@ __device__ __forceinline__ void block_mark_first_equal(const uint32_t* keys, int
         if (eq) {
             const int rank = before + __popc(b & ((1u << lane) - 1u));
             if (rank < need) take[i] = 1;
+            if (last_taken && rank == need - 1) *last_taken = (uint32_t)i;
         }
         base += total;
         __syncthreads();
         if (base >= need) break;
     }
+}
+
+// ---- exact block-wide top-K, one histogram pass in the common case --------------------------------
+// Marks take[i] = 1 for exactly the K best of keys[0..n) under (key descending, index ascending);
+// key 0 = absent; take[] must be zero on entry; needs 1 <= K <= number of present keys.  Returns (to
+// every thread) the key and array index of the K-th = worst selected element.
+//
+// Fast path: keys are bucketed LINEARLY in score between the smallest and largest finite score
+// (monotone: a higher score never lands in a lower bucket), so one 256-bin histogram isolates the
+// bucket that contains the cut; buckets above it are taken whole and the few elements of the cut
+// bucket are ranked exactly against each other.  If the cut bucket is crowded (> kTopkList
+// elements) or the score range is degenerate, the MSB radix select above decides instead.
+constexpr int kTopkList = 256;
+
+struct TopkScratch {
+    uint32_t* hist;    // [256]
+    uint32_t* misc;    // [16]
+    uint32_t* wred;    // [72]  per-warp partials (up to 32 warps, two values each) + warp counts
+    int32_t* list;     // [kTopkList]
+};
+
+struct TopkResult {
+    uint32_t kth_key;
+    int kth_idx;
+};
+
+__device__ __forceinline__ TopkResult block_topk_mark(const uint32_t* keys, int n, int K, uint8_t* take,
+                                                      const TopkScratch& s)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+    // ---- range of the finite scores ----
+    float lo = INFINITY, hi = -INFINITY;
+    for (int i = tid; i < n; i += blockDim.x) {
+        const uint32_t key = keys[i];
+        if (key != 0u) {
+            const float f = key_to_float(key);
+            if (f > -INFINITY) lo = fminf(lo, f);
+            hi = fmaxf(hi, f);
+        }
+    }
+#pragma unroll
+    for (int off = 16; off; off >>= 1) {
+        lo = fminf(lo, __shfl_xor_sync(kFullMask, lo, off));
+        hi = fmaxf(hi, __shfl_xor_sync(kFullMask, hi, off));
+    }
+    if (lane == 0) {
+        s.wred[2 * warp] = __float_as_uint(lo);
+        s.wred[2 * warp + 1] = __float_as_uint(hi);
+    }
+    for (int i = tid; i < 256; i += blockDim.x) s.hist[i] = 0u;
+    if (tid == 0) s.misc[4] = 0u;   // list length
+    __syncthreads();
+    lo = INFINITY;
+    hi = -INFINITY;
+    for (int w = 0; w < nwarps; ++w) {
+        lo = fminf(lo, __uint_as_float(s.wred[2 * w]));
+        hi = fmaxf(hi, __uint_as_float(s.wred[2 * w + 1]));
+    }
+    const float scale = 256.0f / (hi - lo);
+    const bool fast = hi > lo && isfinite(scale) && isfinite(hi - lo);
+    int cut = -1, need = K;
+    if (fast) {
+        for (int i = tid; i < n; i += blockDim.x) {
+            const uint32_t key = keys[i];
+            if (key != 0u) {
+                const float f = key_to_float(key);
+                const int b = f > -INFINITY ? min(255, (int)((f - lo) * scale)) : 0;
+                atomicAdd(&s.hist[b], 1u);
+            }
+        }
+        __syncthreads();
+        if (tid < 32) {
+            uint32_t c[8], mine = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                c[j] = s.hist[lane * 8 + j];
+                mine += c[j];
+            }
+            uint32_t incl = mine;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const uint32_t o = __shfl_down_sync(kFullMask, incl, off);
+                if (lane + off < 32) incl += o;
+            }
+            uint32_t above = incl - mine;
+            if (above < (uint32_t)K && (uint32_t)K <= incl) {
+#pragma unroll
+                for (int j = 7; j >= 0; --j) {
+                    if (above < (uint32_t)K && (uint32_t)K <= above + c[j]) {
+                        s.misc[0] = (uint32_t)(lane * 8 + j);
+                        s.misc[1] = above;
+                        s.misc[2] = c[j];
+                    }
+                    above += c[j];
+                }
+            }
+        }
+        __syncthreads();
+        if ((int)s.misc[2] <= kTopkList) {
+            cut = (int)s.misc[0];
+            need = K - (int)s.misc[1];
+        }
+    }
+    if (cut >= 0) {
+        for (int i = tid; i < n; i += blockDim.x) {
+            const uint32_t key = keys[i];
+            if (key != 0u) {
+                const float f = key_to_float(key);
+                const int b = f > -INFINITY ? min(255, (int)((f - lo) * scale)) : 0;
+                if (b > cut) take[i] = 1;
+                if (b == cut) s.list[atomicAdd(&s.misc[4], 1u)] = i;
+            }
+        }
+        __syncthreads();
+        const int m = (int)s.misc[4];
+        for (int t = tid; t < m; t += blockDim.x) {
+            const int idx = s.list[t];
+            const uint32_t key = keys[idx];
+            int rank = 0;
+            for (int j = 0; j < m; ++j) {
+                const int ij = s.list[j];
+                const uint32_t kj = keys[ij];
+                rank += (kj > key) || (kj == key && ij < idx);
+            }
+            if (rank < need) take[idx] = 1;
+            if (rank == need - 1) {
+                s.misc[5] = key;
+                s.misc[6] = (uint32_t)idx;
+            }
+        }
+        __syncthreads();
+    } else {
+        __syncthreads();   // everyone has read misc[] of the fast attempt
+        const SelectResult r = block_select_kth(keys, n, K, s.hist, s.misc);
+        const int need_eq = K - r.n_greater;
+        for (int i = tid; i < n; i += blockDim.x)
+            if (keys[i] > r.kth) take[i] = 1;
+        block_mark_first_equal(keys, n, r.kth, need_eq, take, s.wred, &s.misc[6]);
+        if (tid == 0) s.misc[5] = r.kth;
+        __syncthreads();
+    }
+    TopkResult out;
+    out.kth_key = s.misc[5];
+    out.kth_idx = (int)s.misc[6];
+    return out;
 }
 
 }  // namespace vsa

@@ -22,15 +22,18 @@ cudaError_t launch_build_summaries(const Geometry& g, const void* k_cache, const
 
 // ---- page routing ---------------------------------------------------------------------------
 size_t route_workspace_bytes(const Geometry& g);
-cudaError_t launch_route(const Geometry& g, const void* q, const void* summaries, const int32_t* block_table,
-                         const int32_t* seq_lens, int P, int32_t* routed_pages, float* routed_scores,
-                         void* ws, int32_t* zero_word, cudaStream_t stream, cudaEvent_t after_scan = nullptr);
+cudaError_t launch_route_scan(const Geometry& g, const void* q, const void* summaries, const int32_t* block_table,
+                              const int32_t* seq_lens, void* ws, int32_t* zero_word, cudaStream_t stream);
+cudaError_t launch_route_select(const Geometry& g, const void* ws, const int32_t* seq_lens, int P,
+                                int32_t* routed_pages, float* routed_scores, cudaStream_t stream);
 
 // ---- fused sparse pass ------------------------------------------------------------------------
+// page_scores == nullptr: routed_pages is read; otherwise the top-P selection runs inside the kernel on
+// page_scores (the scan's output) and routed_pages is written.
 cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache, const void* v_cache,
-                          const int32_t* block_table, const int32_t* seq_lens, const int32_t* routed_pages,
-                          int P, int K_c, float epsilon, float gap_threshold, float* out, vsa_diag_t* diag,
-                          int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream);
+                          const int32_t* block_table, const int32_t* seq_lens, int32_t* routed_pages,
+                          const float* page_scores, int P, int K_c, float epsilon, float gap_threshold, float* out,
+                          vsa_diag_t* diag, int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream);
 
 // ---- dense split-K pass -------------------------------------------------------------------------
 int dense_pages_per_split(const Geometry& g);
