@@ -37,8 +37,10 @@
  *
  * Arithmetic contract
  *   Every score that feeds a selection (page scores, token scores) is an fp32 dot product in
- *   one fixed order: 16 chunks of 8 consecutive elements summed left to right, then the 16
- *   partials combined by a halving tree (p[c] += p[c+off], off = 8, 4, 2, 1).  Selections
+ *   one fixed order: 16 chunks of 8 consecutive elements; inside a chunk the even elements'
+ *   products and the odd elements' products are each summed left to right and the two sums
+ *   added; then the 16 chunk sums are combined by a halving tree (p[c] += p[c+off],
+ *   off = 8, 4, 2, 1).  Selections
  *   order by (score descending, index ascending), -0 and +0 being equal.  Routed pages,
  *   candidate sets, Delta and the fallback flags are therefore reproducible bit for bit.
  *   Softmax weights and outputs use fp32 accumulation.

@@ -88,20 +88,27 @@ uint16_t orc_f32_to_bf16(float f)
 }
 
 /* ---- the one fp32 summation order every discrete decision depends on ------
- * 128 products in 16 chunks of 8 consecutive elements.  Chunk partial: left to right.
+ * 128 products in 16 chunks of 8 consecutive elements.  Chunk partial: the products of the
+ * even elements (0, 2, 4, 6) summed left to right, the products of the odd elements
+ * (1, 3, 5, 7) summed left to right, then even sum + odd sum.
  * Then a halving tree over the 16 partials: p[c] += p[c+off], off = 8, 4, 2, 1.
  * A product of two bf16 numbers is exact in fp32, so it does not matter whether a
- * machine fuses the multiply into the add. */
+ * machine fuses the multiply into the add.  (The paper fixes no order; this one is the
+ * library's arithmetic contract.) */
 float orc_canon_dot(const uint16_t *x, const uint16_t *y)
 {
     float p[16];
     for (int c = 0; c < 16; ++c) {
-        float acc = orc_bf16_to_f32(x[8 * c]) * orc_bf16_to_f32(y[8 * c]);
-        for (int e = 1; e < 8; ++e) {
-            float prod = orc_bf16_to_f32(x[8 * c + e]) * orc_bf16_to_f32(y[8 * c + e]);
-            acc = acc + prod;
+        float part[2];
+        for (int par = 0; par < 2; ++par) {
+            float acc = orc_bf16_to_f32(x[8 * c + par]) * orc_bf16_to_f32(y[8 * c + par]);
+            for (int e = 2 + par; e < 8; e += 2) {
+                float prod = orc_bf16_to_f32(x[8 * c + e]) * orc_bf16_to_f32(y[8 * c + e]);
+                acc = acc + prod;
+            }
+            part[par] = acc;
         }
-        p[c] = acc;
+        p[c] = part[0] + part[1];
     }
     for (int off = 8; off >= 1; off >>= 1)
         for (int c = 0; c < off; ++c) p[c] = p[c] + p[c + off];

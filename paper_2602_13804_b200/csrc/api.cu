@@ -124,7 +124,8 @@ int vsa_route_pages(const vsa_shape_t* shape, const void* q, const void* summari
     if (!q || !summaries || !block_table || !seq_lens || !routed_pages || !ws) return VSA_ERR_INVALID_ARGUMENT;
     if (!aligned16(q) || !aligned16(summaries) || !aligned16(ws)) return VSA_ERR_MISALIGNED;
     if (ws_bytes < vsa::route_workspace_bytes(g)) return VSA_ERR_WORKSPACE_TOO_SMALL;
-    cudaError_t e = vsa::launch_route_scan(g, q, summaries, block_table, seq_lens, ws, nullptr, (cudaStream_t)stream);
+    cudaError_t e = vsa::launch_route_scan(g, q, summaries, block_table, seq_lens, ws, nullptr, nullptr, 0,
+                                           (cudaStream_t)stream);
     if (e != cudaSuccess) return VSA_ERR_CUDA;
     return cuda_rc(vsa::launch_route_select(g, ws, seq_lens, P, routed_pages, routed_scores, (cudaStream_t)stream));
 }
@@ -197,8 +198,9 @@ static int decode_step_impl(const vsa_shape_t* shape, const void* q, const void*
         }
     void* ws_dense = (char*)ws + step_route_part(g);
     if (ev[0] && cudaEventRecord(ev[0], st) != cudaSuccess) return VSA_ERR_CUDA;
-    // the scan kernel clears fallback_count, so the step needs no separate memset for it
-    cudaError_t e = vsa::launch_route_scan(g, q, summaries, block_table, seq_lens, ws, fallback_count, st);
+    // the scan kernel clears fallback_count and the dense pass's tickets: the step enqueues no memset
+    cudaError_t e = vsa::launch_route_scan(g, q, summaries, block_table, seq_lens, ws, fallback_count,
+                                           vsa::dense_tickets(ws_dense), vsa::dense_ticket_count(g), st);
     if (e != cudaSuccess) return VSA_ERR_CUDA;
     if (ev[1] && cudaEventRecord(ev[1], st) != cudaSuccess) return VSA_ERR_CUDA;
     // the top-P selection runs inside the fused kernel, on the scores the scan left in ws
@@ -208,7 +210,7 @@ static int decode_step_impl(const vsa_shape_t* shape, const void* q, const void*
     if (e != cudaSuccess) return VSA_ERR_CUDA;
     if (ev[3] && cudaEventRecord(ev[3], st) != cudaSuccess) return VSA_ERR_CUDA;
     e = vsa::launch_dense(g, q, k_cache, v_cache, block_table, seq_lens, fallback_list, fallback_count, epsilon,
-                          out, diag, ws_dense, st);
+                          out, diag, ws_dense, st, /*tickets_cleared=*/true);
     if (e != cudaSuccess) return VSA_ERR_CUDA;
     if (ev[4] && cudaEventRecord(ev[4], st) != cudaSuccess) return VSA_ERR_CUDA;
     return VSA_OK;

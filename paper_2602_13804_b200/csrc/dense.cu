@@ -279,6 +279,10 @@ static size_t dense_counter_bytes(const Geometry& g)
     return (((size_t)g.batch * g.n_kv_heads * sizeof(int32_t)) + 255) / 256 * 256;
 }
 
+int32_t* dense_tickets(void* ws_dense) { return (int32_t*)ws_dense; }
+
+int dense_ticket_count(const Geometry& g) { return g.batch * g.n_kv_heads; }
+
 size_t dense_workspace_bytes(const Geometry& g)
 {
     return dense_counter_bytes(g) +
@@ -288,12 +292,15 @@ size_t dense_workspace_bytes(const Geometry& g)
 cudaError_t launch_dense(const Geometry& g, const void* q, const void* k_cache, const void* v_cache,
                          const int32_t* block_table, const int32_t* seq_lens, const int32_t* fallback_list,
                          const int32_t* fallback_count, float epsilon, float* out, vsa_diag_t* diag, void* ws,
-                         cudaStream_t stream)
+                         cudaStream_t stream, bool tickets_cleared)
 {
     int32_t* counters = (int32_t*)ws;
     float* partials = (float*)((char*)ws + dense_counter_bytes(g));
-    cudaError_t e = cudaMemsetAsync(counters, 0, dense_counter_bytes(g), stream);
-    if (e != cudaSuccess) return e;
+    cudaError_t e = cudaSuccess;
+    if (!tickets_cleared) {
+        e = cudaMemsetAsync(counters, 0, dense_counter_bytes(g), stream);
+        if (e != cudaSuccess) return e;
+    }
     const int pps = dense_pages_per_split(g), ns = dense_n_splits(g);
     const long long n_items = (long long)g.batch * g.n_kv_heads * ns;
     const size_t mask_bytes = ((size_t)g.batch * g.n_kv_heads + 15) / 16 * 16;

@@ -28,7 +28,7 @@ __host__ __device__ constexpr int token_phase_words(int P, int K_c)
 
 struct TokenSmem {
     uint32_t* keys;   // [P * 16] token score keys, array index = 16 * slot + token (position order)
-    uint8_t* take;    // [P * 16]
+    uint8_t* take;    // [P * 16] scratch of the selection's slow path
     int32_t* sel;     // [K_c] array indices of the candidates, ascending
     TopkScratch ts;
     float* red;       // [warps][128]
@@ -64,9 +64,13 @@ __device__ __forceinline__ void write_failed_unit(float* out, vsa_diag_t* diag, 
     }
 }
 
-// page_scores == nullptr: routed_pages is an input.
-// page_scores != nullptr: the unit's top-P pages are selected here from page_scores[unit][0..n_b)
-//                         and written to routed_pages (best first, -1 padded) as well.
+// PAGE_KPT ==  0: routed_pages is an input.
+// PAGE_KPT == -1: fused with routing; page scores staged in shared memory (any block-table width).
+// PAGE_KPT  >  0: fused with routing; each thread keeps PAGE_KPT page scores in registers.
+//   In both fused forms the unit's top-P pages are selected here from page_scores[unit][0..n_b) and
+//   written to routed_pages (best first, -1 padded).
+// TOK_KPT: token scores per thread, P * 16 <= TOK_KPT * 256.
+template <int PAGE_KPT, int TOK_KPT>
 __global__ void __launch_bounds__(kSparseThreads, 2)
 sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* __restrict__ k_cache,
                      const uint16_t* __restrict__ v_cache, const int32_t* __restrict__ block_table,
@@ -86,57 +90,75 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     const int T = seq_lens[b];
     if (T <= 0 || T > geo.max_pages * kPageSize) {
         write_failed_unit(out, diag, unit, VSA_UNIT_BAD_LENGTH);
-        if (page_scores)
+        if (PAGE_KPT != 0)
             for (int t = tid; t < P; t += kSparseThreads) routed_pages[unit * P + t] = -1;
         return;
     }
     const int nb = (T + kPageSize - 1) / kPageSize;
+    const int32_t* bt = block_table + (long long)b * geo.max_pages;
+    VSA_PROBE(0);
 
     // ---- routed pages -> page_l[] sorted by logical page, so that array order = position order ----
-    int32_t* raw;   // staging of the unsorted page list inside `region` (dead before the token phase)
-    if (page_scores) {
+    int np;
+    int bad = 0;
+    if constexpr (PAGE_KPT != 0) {
         const PageSelectSmem ps = carve_page_select(region, geo.max_pages, P);
-        const int K = select_top_pages(page_scores + unit * geo.max_pages, nb, P, ps);
-        for (int t = tid; t < P; t += kSparseThreads) routed_pages[unit * P + t] = t < K ? ps.win_idx[t] : -1;
-        raw = ps.tmp_idx;   // reuse: tmp_idx is dead after select_top_pages
-        for (int t = tid; t < P; t += kSparseThreads) raw[t] = t < K ? ps.win_idx[t] : INT_MAX;
+        if constexpr (PAGE_KPT > 0)
+            np = select_top_pages_reg<PAGE_KPT>(page_scores + unit * geo.max_pages, nb, P, ps);
+        else
+            np = select_top_pages(page_scores + unit * geo.max_pages, nb, P, ps);
+        for (int t = tid; t < P; t += kSparseThreads) {
+            routed_pages[unit * P + t] = t < np ? ps.win_idx[t] : -1;
+            int l = INT_MAX, phys = -1;
+            if (t < np) {
+                l = ps.asc_idx[t];
+                phys = bt[l];
+                if (phys < 0 || phys >= geo.pool_pages) {
+                    phys = -1;
+                    bad = 1;
+                }
+            }
+            page_l[t] = l;
+            page_phys[t] = phys;
+        }
     } else {
-        raw = (int32_t*)region;
+        int32_t* raw = (int32_t*)region;   // staging; dead before the token phase reuses the region
         for (int t = tid; t < P; t += kSparseThreads) {
             const int l = routed_pages[unit * P + t];
             raw[t] = (l >= 0 && l < nb) ? l : INT_MAX;
         }
-    }
-    __syncthreads();
-    int bad = 0;
-    for (int t = tid; t < P; t += kSparseThreads) {
-        const int l = raw[t];
-        int rank = 0;
-        for (int j = 0; j < P; ++j) rank += (raw[j] < l) || (raw[j] == l && j < t);
-        int phys = -1;
-        if (l != INT_MAX) {
-            phys = block_table[(long long)b * geo.max_pages + l];
-            if (phys < 0 || phys >= geo.pool_pages) {
-                phys = -1;
-                bad = 1;
+        __syncthreads();
+        for (int t = tid; t < P; t += kSparseThreads) {
+            const int l = raw[t];
+            int rank = 0;
+#pragma unroll 8
+            for (int j = 0; j < P; ++j) rank += (raw[j] < l) || (raw[j] == l && j < t);
+            int phys = -1;
+            if (l != INT_MAX) {
+                phys = bt[l];
+                if (phys < 0 || phys >= geo.pool_pages) {
+                    phys = -1;
+                    bad = 1;
+                }
             }
+            page_l[rank] = l;
+            page_phys[rank] = phys;
         }
-        page_l[rank] = l;
-        page_phys[rank] = phys;
+        // (P <= 128 < blockDim.x: thread t < P owns slot t in the count)
+        np = __syncthreads_count(tid < P && raw[tid < P ? tid : 0] != INT_MAX);
     }
-    // (P <= 128 < blockDim.x: thread t < P owns slot t in the count below)
-    const int np = __syncthreads_count(tid < P && raw[tid < P ? tid : 0] != INT_MAX);
+    VSA_PROBE(1);
     if (__syncthreads_or(bad)) {
         write_failed_unit(out, diag, unit, VSA_UNIT_BAD_PAGE);
         return;
     }
     const TokenSmem sm = carve_tokens(region, P, K_c);
-    for (int i = tid; i < N; i += kSparseThreads) {
-        sm.keys[i] = 0u;
-        sm.take[i] = 0;
-    }
+#pragma unroll
+    for (int j = 0; j < TOK_KPT; ++j)
+        if (tid + j * kSparseThreads < N) sm.keys[tid + j * kSparseThreads] = 0u;
     __syncthreads();
 
+    VSA_PROBE(2);
     // ---- token routing: score all 16 tokens of a page per half-warp ----
     float qf[8];
     {
@@ -166,87 +188,97 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         const float s = reduce_scatter16(vals, c);   // lane c: score of token c of the page
         if (active && page_l[slot] * kPageSize + c < T) sm.keys[slot * kPageSize + c] = float_to_key(s);
     }
-    // number of valid scored tokens
-    if (warp == 0) {
-        int cnt = 0;
-        for (int t = lane; t < np; t += 32) cnt += min(kPageSize, T - page_l[t] * kPageSize);
-#pragma unroll
-        for (int off = 16; off; off >>= 1) cnt += __shfl_xor_sync(kFullMask, cnt, off);
-        if (lane == 0) sm.ts.misc[9] = (uint32_t)cnt;
-    }
     __syncthreads();
-    const int nv = (int)sm.ts.misc[9];
-    const int ns = min(K_c, nv);
 
-    // ---- exact top-(ns+1): its last element is the best rejected token, the rest are the candidates ----
-    uint32_t out_key = 0u;
-    const bool has_rejected = nv > ns;
-    if (has_rejected) {
-        const TopkResult r = block_topk_mark(sm.keys, N, ns + 1, sm.take, sm.ts);
-        out_key = r.kth_key;
-        if (tid == 0) sm.take[r.kth_idx] = 0;
-    } else {
-        for (int i = tid; i < N; i += kSparseThreads)
-            if (sm.keys[i] != 0u) sm.take[i] = 1;
-    }
-
-    // ---- best and second-best key over the scored tokens (multiset order statistics) ----
-    {
-        uint32_t a1 = 0u, a2 = 0u;
-        for (int i = tid; i < N; i += kSparseThreads) {
-            const uint32_t k = sm.keys[i];
-            if (k > a1) {
-                a2 = a1;
-                a1 = k;
-            } else if (k > a2) {
-                a2 = k;
-            }
-        }
+    VSA_PROBE(3);
+    // ---- every thread takes its TOK_KPT token keys into registers ----
+    uint32_t key[TOK_KPT];
+    int present = 0;
+    uint32_t a1 = 0u, a2 = 0u;   // best and second-best key (multiset order statistics)
 #pragma unroll
-        for (int off = 16; off; off >>= 1) {
-            const uint32_t b1 = __shfl_xor_sync(kFullMask, a1, off), b2 = __shfl_xor_sync(kFullMask, a2, off);
-            const uint32_t n1 = max(a1, b1), n2 = max(min(a1, b1), max(a2, b2));
-            a1 = n1;
-            a2 = n2;
+    for (int j = 0; j < TOK_KPT; ++j) {
+        const int i = tid + j * kSparseThreads;
+        key[j] = i < N ? sm.keys[i] : 0u;
+        present += key[j] != 0u;
+        if (key[j] > a1) {
+            a2 = a1;
+            a1 = key[j];
+        } else if (key[j] > a2) {
+            a2 = key[j];
         }
-        if (lane == 0) {
-            sm.ts.wred[2 * warp] = a1;
-            sm.ts.wred[2 * warp + 1] = a2;
-        }
+    }
+    // number of valid scored tokens, and the two best keys, block-wide
+#pragma unroll
+    for (int off = 16; off; off >>= 1) {
+        present += __shfl_xor_sync(kFullMask, present, off);
+        const uint32_t b1 = __shfl_xor_sync(kFullMask, a1, off), b2 = __shfl_xor_sync(kFullMask, a2, off);
+        const uint32_t n1 = max(a1, b1), n2 = max(min(a1, b1), max(a2, b2));
+        a1 = n1;
+        a2 = n2;
+    }
+    if (lane == 0) {
+        sm.ts.wred[3 * warp] = a1;
+        sm.ts.wred[3 * warp + 1] = a2;
+        sm.ts.wred[3 * warp + 2] = (uint32_t)present;
     }
     __syncthreads();
     uint32_t key1 = 0u, key2 = 0u;
+    int n_valid = 0;
 #pragma unroll
     for (int w = 0; w < kSparseWarps; ++w) {
-        const uint32_t b1 = sm.ts.wred[2 * w], b2 = sm.ts.wred[2 * w + 1];
+        const uint32_t b1 = sm.ts.wred[3 * w], b2 = sm.ts.wred[3 * w + 1];
         const uint32_t n1 = max(key1, b1), n2 = max(min(key1, b1), max(key2, b2));
         key1 = n1;
         key2 = n2;
+        n_valid += (int)sm.ts.wred[3 * w + 2];
     }
-    __syncthreads();   // wred is reused below
+    const int ns = min(K_c, n_valid);
+    __syncthreads();   // wred is reused by the selection
 
+    VSA_PROBE(4);
+    // ---- exact top-(ns+1): its last element is the best rejected token, the rest are the candidates ----
+    uint32_t out_key = 0u, mask = 0u;
+    const bool has_rejected = n_valid > ns;
+    if (has_rejected) {
+        const TopkRegResult r = block_topk_reg<TOK_KPT>(key, N, ns + 1, sm.ts, sm.keys, sm.take);
+        out_key = r.kth_key;
+        mask = r.mask;
+#pragma unroll
+        for (int j = 0; j < TOK_KPT; ++j)
+            if (tid + j * kSparseThreads == r.kth_idx) mask &= ~(1u << j);
+    } else {
+#pragma unroll
+        for (int j = 0; j < TOK_KPT; ++j)
+            if (key[j] != 0u) mask |= 1u << j;
+    }
+
+    VSA_PROBE(5);
     // ---- ordered compaction of the candidates: sel[] ascending in array (= position) order ----
     {
-        const int per = (N + kSparseThreads - 1) / kSparseThreads;
-        const int lo = tid * per, hi = min(N, lo + per);
-        int cnt = 0;
-        for (int i = lo; i < hi; ++i) cnt += sm.take[i];
-        int incl = cnt;
+        int before[TOK_KPT];
 #pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const int o = __shfl_up_sync(kFullMask, incl, off);
-            if (lane >= off) incl += o;
+        for (int j = 0; j < TOK_KPT; ++j) {
+            const unsigned bal = __ballot_sync(kFullMask, (mask >> j) & 1u);
+            before[j] = __popc(bal & ((1u << lane) - 1u));
+            if (lane == 0) sm.ts.wred[j * kSparseWarps + warp] = (uint32_t)__popc(bal);
         }
-        if (lane == 31) sm.ts.wred[warp] = (uint32_t)incl;
         __syncthreads();
         int base = 0;
-        for (int w = 0; w < warp; ++w) base += (int)sm.ts.wred[w];
-        int o = base + incl - cnt;
-        for (int i = lo; i < hi; ++i)
-            if (sm.take[i]) sm.sel[o++] = i;
+#pragma unroll
+        for (int j = 0; j < TOK_KPT; ++j) {
+            // elements of row j (indices j * 256 + tid) come after all of rows < j
+            int mine = base;
+            for (int w = 0; w < kSparseWarps; ++w) {
+                const int cw = (int)sm.ts.wred[j * kSparseWarps + w];
+                if (w < warp) mine += cw;
+                base += cw;
+            }
+            if ((mask >> j) & 1u) sm.sel[mine + before[j]] = tid + j * kSparseThreads;
+        }
     }
     __syncthreads();
 
+    VSA_PROBE(6);
     // ---- softmax weights and value gather ----
     const float s1 = ns > 0 ? key_to_float(key1) : -INFINITY;
     const float scale = 1.4426950408889634f / epsilon;   // log2(e) / epsilon
@@ -280,6 +312,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
             z += w[u];
         }
     }
+    VSA_PROBE(7);
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[e] += __shfl_xor_sync(kFullMask, acc[e], 16);
     z += __shfl_xor_sync(kFullMask, z, 16);
@@ -299,6 +332,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         out[unit * kHeadDim + tid] = ns > 0 ? a / Z : 0.0f;
     }
 
+    VSA_PROBE(8);
     // ---- diagnostics and fallback flag ----
     if (tid == 0) {
         const float s2 = ns > 1 ? key_to_float(key2) : -INFINITY;
@@ -324,7 +358,46 @@ size_t sparse_smem_bytes(const Geometry& g, int P, int K_c, bool fused)
     return (size_t)(2 * P + words) * 4 + 16;
 }
 
+template <int PAGE_KPT, int TOK_KPT>
+cudaError_t launch_one(const Geometry& g, size_t smem, const uint16_t* q, const uint16_t* k, const uint16_t* v,
+                       const int32_t* block_table, const int32_t* seq_lens, int32_t* routed_pages,
+                       const float* page_scores, int P, int K_c, float epsilon, float gap_threshold, float* out,
+                       vsa_diag_t* diag, int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream)
+{
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(sparse_decode_kernel<PAGE_KPT, TOK_KPT>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    const unsigned units = (unsigned)(g.batch * g.n_q_heads);
+    sparse_decode_kernel<PAGE_KPT, TOK_KPT><<<units, kSparseThreads, smem, stream>>>(
+        g, q, k, v, block_table, seq_lens, routed_pages, page_scores, P, K_c, epsilon, gap_threshold, out, diag,
+        fallback_list, fallback_count);
+    return cudaGetLastError();
+}
+
+template <int PAGE_KPT>
+cudaError_t launch_tok(const Geometry& g, size_t smem, const uint16_t* q, const uint16_t* k, const uint16_t* v,
+                       const int32_t* block_table, const int32_t* seq_lens, int32_t* routed_pages,
+                       const float* page_scores, int P, int K_c, float epsilon, float gap_threshold, float* out,
+                       vsa_diag_t* diag, int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream)
+{
+    const int N = P * kPageSize;
+#define VSA_ARGS g, smem, q, k, v, block_table, seq_lens, routed_pages, page_scores, P, K_c, epsilon, gap_threshold, \
+                 out, diag, fallback_list, fallback_count, stream
+    if (N <= 2 * kSparseThreads) return launch_one<PAGE_KPT, 2>(VSA_ARGS);
+    if (N <= 4 * kSparseThreads) return launch_one<PAGE_KPT, 4>(VSA_ARGS);
+    return launch_one<PAGE_KPT, 8>(VSA_ARGS);
+}
+
 }  // namespace
+
+#ifdef VSA_ENABLE_PROBES
+extern "C" int vsa_probe_read(long long* host64)
+{
+    return (int)cudaMemcpyFromSymbol(host64, vsa_probe_buf, sizeof(long long) * 64);
+}
+#endif
 
 cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache, const void* v_cache,
                           const int32_t* block_table, const int32_t* seq_lens, int32_t* routed_pages,
@@ -332,16 +405,17 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
                           vsa_diag_t* diag, int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream)
 {
     const size_t smem = sparse_smem_bytes(g, P, K_c, page_scores != nullptr);
-    if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(sparse_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)smem);
-        if (e != cudaSuccess) return e;
-    }
-    const unsigned units = (unsigned)(g.batch * g.n_q_heads);
-    sparse_decode_kernel<<<units, kSparseThreads, smem, stream>>>(
-        g, (const uint16_t*)q, (const uint16_t*)k_cache, (const uint16_t*)v_cache, block_table, seq_lens,
-        routed_pages, page_scores, P, K_c, epsilon, gap_threshold, out, diag, fallback_list, fallback_count);
-    return cudaGetLastError();
+    const uint16_t *qq = (const uint16_t*)q, *k = (const uint16_t*)k_cache, *v = (const uint16_t*)v_cache;
+    const uint16_t* q_ = qq;
+#undef VSA_ARGS
+#define VSA_ARGS g, smem, q_, k, v, block_table, seq_lens, routed_pages, page_scores, P, K_c, epsilon, gap_threshold, \
+                 out, diag, fallback_list, fallback_count, stream
+    if (!page_scores) return launch_tok<0>(VSA_ARGS);
+    if (g.max_pages <= 8 * kSparseThreads) return launch_tok<8>(VSA_ARGS);
+    if (g.max_pages <= 16 * kSparseThreads) return launch_tok<16>(VSA_ARGS);
+    if (g.max_pages <= 32 * kSparseThreads) return launch_tok<32>(VSA_ARGS);
+    return launch_tok<-1>(VSA_ARGS);
+#undef VSA_ARGS
 }
 
 }  // namespace vsa

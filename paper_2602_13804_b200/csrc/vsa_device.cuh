@@ -5,6 +5,21 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+// Phase-timing probes for development builds (-DVSA_ENABLE_PROBES): one thread of one block records
+// clock64() at marked points.  They compile to nothing otherwise.
+#ifdef VSA_ENABLE_PROBES
+#ifndef VSA_PROBE_BLOCK
+#define VSA_PROBE_BLOCK 0
+#endif
+static __device__ long long vsa_probe_buf[64];
+#define VSA_PROBE(i)                                                                   \
+    do {                                                                               \
+        if (blockIdx.x == VSA_PROBE_BLOCK && blockIdx.y == 0 && threadIdx.x == 0) vsa_probe_buf[i] = clock64(); \
+    } while (0)
+#else
+#define VSA_PROBE(i)
+#endif
+
 namespace vsa {
 
 constexpr int kHeadDim = 128;   // elements per head
@@ -46,14 +61,35 @@ __device__ __forceinline__ uint4 ld_nc_16B(const void* p)
 
 // ---- the fixed-order dot product ---------------------------------------------------------
 // A row of 128 elements is spread over 16 lanes, lane c holding elements 8c .. 8c+7.
-// chunk_partial() is the left-to-right sum of the lane's 8 products (bf16 x bf16 products are
-// exact in fp32, so fusing the multiply into the add changes nothing).
+// chunk_partial() sums the lane's 8 products as two interleaved chains,
+//     (((x0 y0 + x2 y2) + x4 y4) + x6 y6)  +  (((x1 y1 + x3 y3) + x5 y5) + x7 y7),
+// which is exactly what one packed mul.f32x2 followed by three packed fma.rn.f32x2 compute on the
+// (even, odd) element pairs that unpacking a 32-bit word yields (bf16 x bf16 products are exact in
+// fp32, so fusing the multiply into the add changes nothing).
+__device__ __forceinline__ void mul2(float& d0, float& d1, float a0, float a1, float b0, float b1)
+{
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+        "mul.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d0), "=f"(d1)
+        : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+
+__device__ __forceinline__ void fma2(float& d0, float& d1, float a0, float a1, float b0, float b1)
+{
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rd, {%0, %1};\n\t"
+        "fma.rn.f32x2 rd, ra, rb, rd;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+        : "+f"(d0), "+f"(d1)
+        : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+
 __device__ __forceinline__ float chunk_partial(const float (&x)[8], const float (&y)[8])
 {
-    float acc = x[0] * y[0];
-#pragma unroll
-    for (int e = 1; e < 8; ++e) acc = fmaf(x[e], y[e], acc);
-    return acc;
+    float even, odd;
+    mul2(even, odd, x[0], x[1], y[0], y[1]);
+    fma2(even, odd, x[2], x[3], y[2], y[3]);
+    fma2(even, odd, x[4], x[5], y[4], y[5]);
+    fma2(even, odd, x[6], x[7], y[6], y[7]);
+    return even + odd;
 }
 
 // Halving tree over the 16 lanes of a half-warp for 16 independent values at once
@@ -365,6 +401,159 @@ __device__ __forceinline__ TopkResult block_topk_mark(const uint32_t* keys, int 
     TopkResult out;
     out.kth_key = s.misc[5];
     out.kth_idx = (int)s.misc[6];
+    return out;
+}
+
+// ---- the same selection with the keys held in registers -------------------------------------------
+// Thread t owns elements t, t + blockDim, ..., t + (KPT-1) * blockDim (key[j] = 0 where the element is
+// absent or past n).  On return bit j of the result's `mask` is set iff element t + j * blockDim is
+// among the K best, for every thread; kth_key / kth_idx describe the K-th (worst selected) element.
+// No pass re-reads shared memory for the keys, so the per-thread work of a pass is KPT independent
+// register operations.  `spill` ([n] words) and `spill_take` ([n] bytes) are only touched on the slow
+// path (crowded cut bucket or degenerate range), which stores the keys and runs the routine above.
+struct TopkRegResult {
+    uint32_t mask;
+    uint32_t kth_key;
+    int kth_idx;
+};
+
+template <int KPT>
+__device__ __forceinline__ TopkRegResult block_topk_reg(const uint32_t (&key)[KPT], int n, int K,
+                                                        const TopkScratch& s, uint32_t* spill, uint8_t* spill_take)
+{
+    static_assert(KPT <= 32, "one mask bit per owned element");
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+    const int stride = blockDim.x;
+    float f[KPT];
+    float lo = INFINITY, hi = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < KPT; ++j) {
+        f[j] = key_to_float(key[j]);
+        if (key[j] != 0u) {
+            if (f[j] > -INFINITY) lo = fminf(lo, f[j]);
+            hi = fmaxf(hi, f[j]);
+        }
+    }
+#pragma unroll
+    for (int off = 16; off; off >>= 1) {
+        lo = fminf(lo, __shfl_xor_sync(kFullMask, lo, off));
+        hi = fmaxf(hi, __shfl_xor_sync(kFullMask, hi, off));
+    }
+    if (lane == 0) {
+        s.wred[2 * warp] = __float_as_uint(lo);
+        s.wred[2 * warp + 1] = __float_as_uint(hi);
+    }
+    for (int i = tid; i < 256; i += stride) s.hist[i] = 0u;
+    if (tid == 0) s.misc[4] = 0u;   // list length
+    __syncthreads();
+    lo = INFINITY;
+    hi = -INFINITY;
+    for (int w = 0; w < nwarps; ++w) {
+        lo = fminf(lo, __uint_as_float(s.wred[2 * w]));
+        hi = fmaxf(hi, __uint_as_float(s.wred[2 * w + 1]));
+    }
+    const float scale = 256.0f / (hi - lo);
+    const bool fast = hi > lo && isfinite(scale) && isfinite(hi - lo);
+    int cut = -1, need = K;
+    int bucket[KPT];
+    if (fast) {
+#pragma unroll
+        for (int j = 0; j < KPT; ++j) {
+            bucket[j] = f[j] > -INFINITY ? min(255, (int)((f[j] - lo) * scale)) : 0;
+            if (key[j] != 0u) atomicAdd(&s.hist[bucket[j]], 1u);
+        }
+        __syncthreads();
+        if (tid < 32) {
+            uint32_t c[8], mine = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                c[j] = s.hist[lane * 8 + j];
+                mine += c[j];
+            }
+            uint32_t incl = mine;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const uint32_t o = __shfl_down_sync(kFullMask, incl, off);
+                if (lane + off < 32) incl += o;
+            }
+            uint32_t above = incl - mine;
+            if (above < (uint32_t)K && (uint32_t)K <= incl) {
+#pragma unroll
+                for (int j = 7; j >= 0; --j) {
+                    if (above < (uint32_t)K && (uint32_t)K <= above + c[j]) {
+                        s.misc[0] = (uint32_t)(lane * 8 + j);
+                        s.misc[1] = above;
+                        s.misc[2] = c[j];
+                    }
+                    above += c[j];
+                }
+            }
+        }
+        __syncthreads();
+        if ((int)s.misc[2] <= kTopkList) {
+            cut = (int)s.misc[0];
+            need = K - (int)s.misc[1];
+        }
+    }
+    TopkRegResult out;
+    out.mask = 0u;
+    if (cut >= 0) {
+        // list entries: element index in list[], its key in hist[] (the histogram is dead by now)
+        uint32_t in_cut = 0u;
+#pragma unroll
+        for (int j = 0; j < KPT; ++j) {
+            if (key[j] != 0u) {
+                if (bucket[j] > cut) out.mask |= 1u << j;
+                if (bucket[j] == cut) {
+                    // the histogram is dead (warp 0 read it before the last barrier): reuse it for the keys
+                    const int slot = (int)atomicAdd(&s.misc[4], 1u);
+                    s.list[slot] = tid + j * stride;
+                    s.hist[slot] = key[j];
+                    in_cut |= 1u << j;
+                }
+            }
+        }
+        __syncthreads();
+        const int m = (int)s.misc[4];
+        for (int t = tid; t < m; t += stride) {
+            const int idx = s.list[t];
+            const uint32_t kt = s.hist[t];
+            int rank = 0;
+            for (int u = 0; u < m; ++u) {
+                const uint32_t ku = s.hist[u];
+                rank += (ku > kt) || (ku == kt && s.list[u] < idx);
+            }
+            spill_take[idx] = rank < need ? 1 : 0;   // read back by the element's owner below
+            if (rank == need - 1) {
+                s.misc[5] = kt;
+                s.misc[6] = (uint32_t)idx;
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < KPT; ++j)
+            if (((in_cut >> j) & 1u) && spill_take[tid + j * stride]) out.mask |= 1u << j;
+    } else {
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < KPT; ++j) {
+            const int i = tid + j * stride;
+            if (i < n) {
+                spill[i] = key[j];
+                spill_take[i] = 0;
+            }
+        }
+        __syncthreads();
+        block_topk_mark(spill, n, K, spill_take, s);
+#pragma unroll
+        for (int j = 0; j < KPT; ++j) {
+            const int i = tid + j * stride;
+            if (i < n && spill_take[i]) out.mask |= 1u << j;
+        }
+    }
+    out.kth_key = s.misc[5];
+    out.kth_idx = (int)s.misc[6];
+    __syncthreads();   // scratch may be reused by the caller right away
     return out;
 }
 

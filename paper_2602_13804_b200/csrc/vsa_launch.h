@@ -22,8 +22,10 @@ cudaError_t launch_build_summaries(const Geometry& g, const void* k_cache, const
 
 // ---- page routing ---------------------------------------------------------------------------
 size_t route_workspace_bytes(const Geometry& g);
+// zero_word (one int) and zero_words[0..zero_count) are cleared by the scan kernel when not null
 cudaError_t launch_route_scan(const Geometry& g, const void* q, const void* summaries, const int32_t* block_table,
-                              const int32_t* seq_lens, void* ws, int32_t* zero_word, cudaStream_t stream);
+                              const int32_t* seq_lens, void* ws, int32_t* zero_word, int32_t* zero_words,
+                              int zero_count, cudaStream_t stream);
 cudaError_t launch_route_select(const Geometry& g, const void* ws, const int32_t* seq_lens, int P,
                                 int32_t* routed_pages, float* routed_scores, cudaStream_t stream);
 
@@ -41,6 +43,9 @@ size_t dense_workspace_bytes(const Geometry& g);
 cudaError_t launch_dense(const Geometry& g, const void* q, const void* k_cache, const void* v_cache,
                          const int32_t* block_table, const int32_t* seq_lens, const int32_t* fallback_list,
                          const int32_t* fallback_count, float epsilon, float* out, vsa_diag_t* diag, void* ws,
-                         cudaStream_t stream);
+                         cudaStream_t stream, bool tickets_cleared = false);
+// the per-(sequence, KV head) tickets at the start of the dense workspace, and how many there are
+int32_t* dense_tickets(void* ws_dense);
+int dense_ticket_count(const Geometry& g);
 
 }  // namespace vsa

@@ -8,20 +8,21 @@
 
 namespace vsa {
 
-// Shared-memory needs of select_top_pages for n_max scores and P pages, in 4-byte words.
+// Shared-memory needs of the page selection for n_max scores and P pages, in 4-byte words.
 __host__ __device__ constexpr int select_pages_words(int n_max, int P)
 {
-    return n_max /*keys*/ + (n_max + 3) / 4 /*take*/ + 256 + 16 + 72 + kTopkList /*scratch*/ + 4 * P /*tmp + winners*/;
+    return n_max /*keys*/ + (n_max + 3) / 4 /*take*/ + 256 + 16 + 72 + kTopkList /*scratch*/ + 5 * P /*lists*/;
 }
 
 struct PageSelectSmem {
-    uint32_t* keys;      // [n_max]
+    uint32_t* keys;      // [n_max]  (register variant: only the slow path stores keys here)
     uint8_t* take;       // [n_max]
     TopkScratch ts;
     uint32_t* tmp_key;   // [P] winners, unordered
     int32_t* tmp_idx;    // [P]
     uint32_t* win_key;   // [P] winners, best first
     int32_t* win_idx;    // [P]
+    int32_t* asc_idx;    // [P] winners by ascending page index
 };
 
 __device__ __forceinline__ PageSelectSmem carve_page_select(uint32_t* base, int n_max, int P)
@@ -37,12 +38,34 @@ __device__ __forceinline__ PageSelectSmem carve_page_select(uint32_t* base, int 
     s.tmp_idx = (int32_t*)(s.tmp_key + P);
     s.win_key = (uint32_t*)(s.tmp_idx + P);
     s.win_idx = (int32_t*)(s.win_key + P);
+    s.asc_idx = s.win_idx + P;
     return s;
 }
 
-// Exact top-min(P, n) of sc[0..n) under (score descending, page ascending).  On return (after a
-// block barrier) s.win_idx[0..K) / s.win_key[0..K) hold the winners best first; returns K.
-// All threads of the block call it.
+// Orders the K unordered winners in tmp_key/tmp_idx: win_* best first (key descending, index
+// ascending), asc_idx by ascending index.  Ends with a block barrier.
+__device__ __forceinline__ void order_winners(int K, const PageSelectSmem& s)
+{
+    for (int t = threadIdx.x; t < K; t += blockDim.x) {
+        const uint32_t key = s.tmp_key[t];
+        const int idx = s.tmp_idx[t];
+        int rank = 0, rank_asc = 0;
+#pragma unroll 8
+        for (int j = 0; j < K; ++j) {
+            const uint32_t kj = s.tmp_key[j];
+            const int ij = s.tmp_idx[j];
+            rank += (kj > key) || (kj == key && ij < idx);
+            rank_asc += ij < idx;
+        }
+        s.win_key[rank] = key;
+        s.win_idx[rank] = idx;
+        s.asc_idx[rank_asc] = idx;
+    }
+    __syncthreads();
+}
+
+// Exact top-min(P, n) of sc[0..n) under (score descending, page ascending), keys staged in shared
+// memory (any n up to the carve size).  Returns K; winners in s.win_* / s.asc_idx.
 __device__ __forceinline__ int select_top_pages(const float* __restrict__ sc, int n, int P, const PageSelectSmem& s)
 {
     const int K = min(P, n);
@@ -68,18 +91,43 @@ __device__ __forceinline__ int select_top_pages(const float* __restrict__ sc, in
         }
     }
     __syncthreads();
-    for (int t = threadIdx.x; t < K; t += blockDim.x) {
-        const uint32_t key = s.tmp_key[t];
-        const int idx = s.tmp_idx[t];
-        int rank = 0;
-        for (int j = 0; j < K; ++j) {
-            const uint32_t kj = s.tmp_key[j];
-            rank += (kj > key) || (kj == key && s.tmp_idx[j] < idx);
+    order_winners(K, s);
+    return K;
+}
+
+// The same with each thread holding its KPT scores in registers (n <= KPT * blockDim.x).
+template <int KPT>
+__device__ __forceinline__ int select_top_pages_reg(const float* __restrict__ sc, int n, int P,
+                                                    const PageSelectSmem& s)
+{
+    const int K = min(P, n);
+    const int tid = threadIdx.x, stride = blockDim.x;
+    uint32_t key[KPT];
+#pragma unroll
+    for (int j = 0; j < KPT; ++j) {
+        const int i = tid + j * stride;
+        key[j] = i < n ? float_to_key(__ldcg(sc + i)) : 0u;
+    }
+    if (tid == 0) s.ts.misc[8] = 0u;
+    uint32_t mask = 0u;
+    if (n > P) {
+        mask = block_topk_reg<KPT>(key, n, K, s.ts, s.keys, s.take).mask;   // barriers inside order misc[8]
+    } else {
+#pragma unroll
+        for (int j = 0; j < KPT; ++j)
+            if (key[j] != 0u) mask |= 1u << j;
+        __syncthreads();
+    }
+#pragma unroll
+    for (int j = 0; j < KPT; ++j) {
+        if ((mask >> j) & 1u) {
+            const int slot = (int)atomicAdd(&s.ts.misc[8], 1u);
+            s.tmp_key[slot] = key[j];
+            s.tmp_idx[slot] = tid + j * stride;
         }
-        s.win_key[rank] = key;
-        s.win_idx[rank] = idx;
     }
     __syncthreads();
+    order_winners(K, s);
     return K;
 }
 

@@ -58,14 +58,17 @@ def test_canon_dot_order_is_the_documented_tree():
     x[64], y[64] = 1.0, 1.0
     x[96], y[96] = 1.0, 1.0
     assert oracle.canon_dot(_bf(x), _bf(y)) == np.float32(1.0)
-    # inside a chunk the sum runs left to right: (2^24 + 1) + 1 = 2^24, then - 2^24 = 0
+    # inside a chunk the even and the odd elements form two left-to-right chains:
+    # even: ((2^24 + 1) + 1) - 2^24 = 0 (both +1 are rounded away), odd: 1; total 1.
+    # One chain over all eight elements would give 0, the exact value is 3.
     x[:] = 0
     y[:] = 0
     x[0], y[0] = 4096.0, 4096.0
     x[1], y[1] = 1.0, 1.0
     x[2], y[2] = 1.0, 1.0
-    x[3], y[3] = 4096.0, -4096.0
-    assert oracle.canon_dot(_bf(x), _bf(y)) == np.float32(0.0)
+    x[4], y[4] = 1.0, 1.0
+    x[6], y[6] = 4096.0, -4096.0
+    assert oracle.canon_dot(_bf(x), _bf(y)) == np.float32(1.0)
     # the same four products spread so that the tree pairs them (c, c+8): (2^24 - 2^24) + (1 + 1)
     x[:] = 0
     y[:] = 0
