@@ -37,6 +37,8 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, c = lane & 15, gi = lane >> 4;
     const int n_groups = geo.batch * geo.n_kv_heads;
+    pdl_wait();
+    pdl_launch_dependents();
 
     // ---- which heads of which groups are listed? ----
     if (fallback_count) {
@@ -315,9 +317,10 @@ cudaError_t launch_dense(const Geometry& g, const void* q, const void* k_cache, 
         if (per_sm < 1) per_sm = 1;                                                                              \
         long long blocks = (long long)num_sms() * per_sm;                                                        \
         if (blocks > n_items) blocks = n_items;                                                                  \
-        dense_split_kernel<GG><<<(unsigned)blocks, kDenseThreads, mask_bytes, stream>>>(                         \
-            g, qq, kk, vv, block_table, seq_lens, fallback_list, fallback_count, epsilon, partials, counters,   \
-            out, diag, pps, ns);                                                                                 \
+        e = launch_pdl(dense_split_kernel<GG>, dim3((unsigned)blocks), dim3(kDenseThreads), mask_bytes, stream, \
+                       g, qq, kk, vv, block_table, seq_lens, fallback_list, fallback_count, epsilon, partials,   \
+                       counters, out, diag, pps, ns);                                                            \
+        if (e != cudaSuccess) return e;                                                                          \
     }
     switch (g.group) {
         case 1: VSA_DENSE_LAUNCH(1); break;

@@ -16,15 +16,40 @@ namespace {
 
 constexpr int kScanThreads = 256;
 constexpr int kScanWarps = kScanThreads / 32;
-constexpr int kBlockPages = 32;   // pages whose block-table entries one warp holds in a register
+constexpr int kBlockPages = 32;      // pages per block-table block (one coalesced 128-byte load per warp)
+constexpr int kMaxBlocksPerWarp = 16;
+
+template <int G>
+struct ScanCfg {
+    static constexpr int ROWS = G == 1 ? 8 : 16 / G;      // rows per half-warp per round
+    static constexpr int VALS = ROWS * G;                 // (row, head) partials per lane per round (8 or 16)
+    static constexpr int ROUND_PAGES = 2 * ROWS;          // pages (rows of one KV head) per warp per round
+    static constexpr int ROUNDS = kBlockPages / ROUND_PAGES;
+    // rounds kept in flight per warp: about 8 KB of rows
+    static constexpr int STAGES = (8192 / (ROUND_PAGES * kRowBytes) < 2 ? 2 : 8192 / (ROUND_PAGES * kRowBytes)) + 1;
+    static constexpr int RING_BYTES = STAGES * ROUND_PAGES * kRowBytes;
+    static constexpr int WARP_BYTES = RING_BYTES + kMaxBlocksPerWarp * kBlockPages * 4;
+};
+
+__device__ __forceinline__ void cp_async_16(uint32_t smem_addr, const void* gptr)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr), "l"(gptr) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait()
+{
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
 
 // Warp w of the grid row of sequence b handles KV head (w % n_kv) and the 32-page blocks
 // [slice * blocks_per_warp, (slice + 1) * blocks_per_warp), slice = w / n_kv, so the warps of a
 // thread block read the summaries of all KV heads of the same pages (2 KB contiguous per page).
-// A half-warp reads one 256-byte row per load instruction; the G query heads of the row's group
-// share each unpacked element; 16 (row, head) partials are reduced at once.  The loads of the next
-// round are issued before the current round is reduced (two register buffers), and the block-table
-// entries of the block after next are fetched while the current block is processed.
+// Every lane streams its own 16-byte column of the rows through a private ring in shared memory
+// with cp.async (several rounds in flight, no registers held by loads in flight, and no
+// cross-thread synchronisation: a lane only ever reads back what it copied itself).  A half-warp
+// covers one 256-byte row per copy instruction; the G query heads of the row's group share each
+// unpacked element; 16 (row, head) partials are reduced at once.
 template <int G>
 __global__ void __launch_bounds__(kScanThreads, 2)
 route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* __restrict__ summaries,
@@ -32,11 +57,11 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
                   float* __restrict__ scores, int blocks_per_warp, int32_t* zero_word, int32_t* zero_words,
                   int zero_count)
 {
-    constexpr int ROWS = G == 1 ? 8 : 16 / G;      // rows per half-warp per round
-    constexpr int VALS = ROWS * G;                 // (row, head) partials per lane per round (8 or 16)
-    constexpr int ROUND_PAGES = 2 * ROWS;          // pages per warp per round
-    constexpr int ROUNDS = kBlockPages / ROUND_PAGES;   // rounds per 32-page block (even)
-    static_assert(ROUNDS % 2 == 0, "the round loop is unrolled by two");
+    using Cfg = ScanCfg<G>;
+    constexpr int ROWS = Cfg::ROWS, VALS = Cfg::VALS, ROUND_PAGES = Cfg::ROUND_PAGES, STAGES = Cfg::STAGES;
+    extern __shared__ __align__(16) uint8_t scan_smem[];
+    pdl_wait();                 // the score scratch may still be read by the previous step's kernels
+    pdl_launch_dependents();
 
     // housekeeping for the kernels that follow in a step: clear the fallback counter and the
     // per-group tickets of the dense pass
@@ -48,27 +73,34 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
     }
 
     const int b = blockIdx.y;
-    const int lane = threadIdx.x & 31, c = lane & 15, gi = lane >> 4;
-    const int w = blockIdx.x * kScanWarps + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, c = lane & 15, gi = lane >> 4;
+    const int w = blockIdx.x * kScanWarps + warp;
     const int g = w % geo.n_kv_heads;
     const int slice = w / geo.n_kv_heads;
     const int T = seq_lens[b];
     if (T <= 0 || T > geo.max_pages * kPageSize) return;
     const int nb = (T + kPageSize - 1) / kPageSize;
-    const int first_block = slice * blocks_per_warp;
-    if (first_block * kBlockPages >= nb) return;
-    const int n_blocks = min(blocks_per_warp, (nb - first_block * kBlockPages + kBlockPages - 1) / kBlockPages);
+    const int first_page = slice * blocks_per_warp * kBlockPages;
+    if (first_page >= nb) return;
+    const int n_pages = min(blocks_per_warp * kBlockPages, nb - first_page);
+    const int n_blocks = (n_pages + kBlockPages - 1) / kBlockPages;
+    const int n_rounds = (n_pages + ROUND_PAGES - 1) / ROUND_PAGES;
 
-    const int32_t* bt = block_table + (long long)b * geo.max_pages;
-    auto load_bt = [&](int blk) -> int {   // physical page of this lane's page in block `blk`, -1 if none
-        const int l = blk * kBlockPages + lane;
-        if (blk >= first_block + n_blocks || l >= nb) return -1;
-        const int p = bt[l];
-        return (p >= 0 && p < geo.pool_pages) ? p : -1;
-    };
-    int phys_even = load_bt(first_block);       // blocks first_block + 0, 2, 4, ...
-    int phys_odd = load_bt(first_block + 1);    // blocks first_block + 1, 3, 5, ...
+    uint8_t* my_smem = scan_smem + warp * Cfg::WARP_BYTES;
+    int32_t* phys_tab = (int32_t*)(my_smem + Cfg::RING_BYTES);   // [n_blocks * 32], -1 = no valid page
+    const uint32_t ring = (uint32_t)__cvta_generic_to_shared(my_smem);
 
+    // block-table entries of the whole page range of this warp (independent coalesced loads)
+    const int32_t* bt = block_table + (long long)b * geo.max_pages + first_page;
+    for (int k = 0; k < n_blocks; ++k) {
+        const int i = k * kBlockPages + lane;
+        int p = -1;
+        if (i < n_pages) {
+            p = bt[i];
+            if (p < 0 || p >= geo.pool_pages) p = -1;
+        }
+        phys_tab[i] = p;
+    }
     float qf[G][8];
 #pragma unroll
     for (int hh = 0; hh < G; ++hh) {
@@ -76,27 +108,41 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
             q + ((long long)b * geo.n_q_heads + g * G + hh) * kHeadDim + c * 8);
         unpack8(v, qf[hh]);
     }
+    __syncwarp();
+
     const uint16_t* srow = summaries + (long long)g * kHeadDim + c * 8;
     const long long page_elems = (long long)geo.n_kv_heads * kHeadDim;
+    const uint32_t lane_off = (uint32_t)(gi * ROWS * kRowBytes + c * 16);
     // after the reduction this lane owns (row own_r, head own_h) of its half-warp's ROWS rows
     const int own_r = VALS == 16 ? c / G : (c & 7) / G, own_h = c % G;
-    float* out_lane = scores + ((long long)b * geo.n_q_heads + g * G + own_h) * geo.max_pages + gi * ROWS + own_r;
+    const bool owns = VALS == 16 || c < 8;
+    float* out_lane = scores + ((long long)b * geo.n_q_heads + g * G + own_h) * geo.max_pages + first_page +
+                      gi * ROWS + own_r;
 
-    // rows of round `rnd` (0 .. ROUNDS-1) of a block whose block-table entries sit in `phys_reg`;
     // rows without a valid page read row 0 of the pool instead (their result is never stored)
-    auto issue = [&](uint4 (&buf)[ROWS], int phys_reg, int rnd) {
+    auto issue = [&](int R) {
+        const uint32_t dst = ring + (uint32_t)((R % STAGES) * ROUND_PAGES * kRowBytes) + lane_off;
+        const int* tab = phys_tab + R * ROUND_PAGES + gi * ROWS;
 #pragma unroll
-        for (int r = 0; r < ROWS; ++r) {
-            const int phys = __shfl_sync(kFullMask, phys_reg, rnd * ROUND_PAGES + gi * ROWS + r);
-            buf[r] = ld_nc_16B(srow + max(phys, 0) * page_elems);
-        }
+        for (int r = 0; r < ROWS; ++r) cp_async_16(dst + r * kRowBytes, srow + max(tab[r], 0) * page_elems);
     };
-    auto reduce_store = [&](const uint4 (&buf)[ROWS], int phys_reg, int blk, int rnd) {
+
+#pragma unroll
+    for (int s = 0; s < STAGES - 1; ++s) {
+        if (s < n_rounds) issue(s);
+        cp_async_commit();
+    }
+    for (int R = 0; R < n_rounds; ++R) {
+        if (R + STAGES - 1 < n_rounds) issue(R + STAGES - 1);
+        cp_async_commit();
+        cp_async_wait<STAGES - 1>();   // this lane's copies of round R have landed
+        const uint8_t* src = my_smem + (R % STAGES) * ROUND_PAGES * kRowBytes + lane_off;
         float vals[16];
 #pragma unroll
         for (int r = 0; r < ROWS; ++r) {
+            const uint4 v = *reinterpret_cast<const uint4*>(src + r * kRowBytes);
             float kf[8];
-            unpack8(buf[r], kf);
+            unpack8(v, kf);
 #pragma unroll
             for (int hh = 0; hh < G; ++hh) vals[r * G + hh] = chunk_partial(qf[hh], kf);
         }
@@ -105,35 +151,8 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
             for (int i = VALS; i < 16; ++i) vals[i] = 0.0f;
         }
         const float s = reduce_scatter16(vals, c);
-        const int pl = rnd * ROUND_PAGES + gi * ROWS + own_r;
-        const int phys = __shfl_sync(kFullMask, phys_reg, pl);
-        const int l = blk * kBlockPages + pl;
-        if (l < nb && (VALS == 16 || c < 8)) out_lane[blk * kBlockPages + rnd * ROUND_PAGES] = phys >= 0 ? s : -INFINITY;
-    };
-
-    uint4 buf_a[ROWS], buf_b[ROWS];
-    issue(buf_a, phys_even, 0);
-    for (int k = 0; k < n_blocks; ++k) {
-        const int blk = first_block + k;
-        const bool even = (k & 1) == 0;
-        const int phys_cur = even ? phys_even : phys_odd;
-        const int phys_nxt = even ? phys_odd : phys_even;
-#pragma unroll
-        for (int rnd = 0; rnd < ROUNDS; rnd += 2) {
-            issue(buf_b, phys_cur, rnd + 1);
-            reduce_store(buf_a, phys_cur, blk, rnd);
-            if (rnd + 2 < ROUNDS)
-                issue(buf_a, phys_cur, rnd + 2);
-            else if (k + 1 < n_blocks)
-                issue(buf_a, phys_nxt, 0);
-            reduce_store(buf_b, phys_cur, blk, rnd + 1);
-        }
-        // this block's register is free: fetch the entries of the block after next into it
-        const int refill = load_bt(blk + 2);
-        if (even)
-            phys_even = refill;
-        else
-            phys_odd = refill;
+        const int pl = R * ROUND_PAGES + gi * ROWS + own_r;
+        if (owns && pl < n_pages) out_lane[R * ROUND_PAGES] = phys_tab[pl] >= 0 ? s : -INFINITY;
     }
 }
 
@@ -146,6 +165,8 @@ __global__ void route_select_kernel(Geometry geo, const float* __restrict__ scor
                                     int32_t* __restrict__ routed_pages, float* __restrict__ routed_scores)
 {
     extern __shared__ uint32_t smem[];
+    pdl_wait();
+    pdl_launch_dependents();
     const PageSelectSmem s = carve_page_select(smem, geo.max_pages, P);
     const int h = blockIdx.x, b = blockIdx.y;
     const long long unit = (long long)b * geo.n_q_heads + h;
@@ -168,12 +189,35 @@ size_t select_smem_bytes(const Geometry& g, int P) { return (size_t)select_pages
 int scan_blocks_per_warp(const Geometry& g)
 {
     // 32-page blocks per warp: about one resident wave of warps (2 thread blocks of 8 warps per SM
-    // on 148 SMs) when the problem is large enough, never more than 16 blocks per warp
+    // on 148 SMs) when the problem is large enough, never more than kMaxBlocksPerWarp
     const long long blocks = (long long)g.batch * g.n_kv_heads * ((g.max_pages + kBlockPages - 1) / kBlockPages);
     long long k = (blocks + 2367) / 2368;
     if (k < 1) k = 1;
-    if (k > 16) k = 16;
+    if (k > kMaxBlocksPerWarp) k = kMaxBlocksPerWarp;
     return (int)k;
+}
+
+template <int G>
+cudaError_t launch_scan_g(const Geometry& g, const uint16_t* q, const uint16_t* summaries, const int32_t* block_table,
+                          const int32_t* seq_lens, float* scores, int32_t* zero_word, int32_t* zero_words,
+                          int zero_count, cudaStream_t stream)
+{
+    const int bpw = scan_blocks_per_warp(g);
+    const int slices = ((g.max_pages + kBlockPages - 1) / kBlockPages + bpw - 1) / bpw;
+    const int warps = slices * g.n_kv_heads;
+    const dim3 grid((unsigned)((warps + kScanWarps - 1) / kScanWarps), (unsigned)g.batch);
+    const size_t smem = (size_t)kScanWarps * ScanCfg<G>::WARP_BYTES;
+    static int attr_device = -1;   // per template instance: the device whose function attribute is set
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (attr_device != dev) {
+        e = cudaFuncSetAttribute(route_scan_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        attr_device = dev;
+    }
+    return launch_pdl(route_scan_kernel<G>, grid, dim3(kScanThreads), smem, stream, g, q, summaries, block_table,
+                      seq_lens, scores, bpw, zero_word, zero_words, zero_count);
 }
 
 }  // namespace
@@ -188,24 +232,15 @@ cudaError_t launch_route_scan(const Geometry& g, const void* q, const void* summ
                               int zero_count, cudaStream_t stream)
 {
     float* scores = (float*)ws;
-    const int bpw = scan_blocks_per_warp(g);
-    const int slices = ((g.max_pages + kBlockPages - 1) / kBlockPages + bpw - 1) / bpw;
-    const int warps = slices * g.n_kv_heads;
-    dim3 grid((unsigned)((warps + kScanWarps - 1) / kScanWarps), (unsigned)g.batch);
     const uint16_t* qq = (const uint16_t*)q;
     const uint16_t* ss = (const uint16_t*)summaries;
-#define VSA_SCAN_LAUNCH(GG)                                                                                      \
-    route_scan_kernel<GG><<<grid, kScanThreads, 0, stream>>>(g, qq, ss, block_table, seq_lens, scores, bpw,      \
-                                                             zero_word, zero_words, zero_count)
     switch (g.group) {
-        case 1: VSA_SCAN_LAUNCH(1); break;
-        case 2: VSA_SCAN_LAUNCH(2); break;
-        case 4: VSA_SCAN_LAUNCH(4); break;
-        case 8: VSA_SCAN_LAUNCH(8); break;
+        case 1: return launch_scan_g<1>(g, qq, ss, block_table, seq_lens, scores, zero_word, zero_words, zero_count, stream);
+        case 2: return launch_scan_g<2>(g, qq, ss, block_table, seq_lens, scores, zero_word, zero_words, zero_count, stream);
+        case 4: return launch_scan_g<4>(g, qq, ss, block_table, seq_lens, scores, zero_word, zero_words, zero_count, stream);
+        case 8: return launch_scan_g<8>(g, qq, ss, block_table, seq_lens, scores, zero_word, zero_words, zero_count, stream);
         default: return cudaErrorInvalidValue;
     }
-#undef VSA_SCAN_LAUNCH
-    return cudaGetLastError();
 }
 
 cudaError_t launch_route_select(const Geometry& g, const void* ws, const int32_t* seq_lens, int P,
@@ -220,8 +255,9 @@ cudaError_t launch_route_select(const Geometry& g, const void* ws, const int32_t
                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);        \
             if (e != cudaSuccess) return e;                                                                      \
         }                                                                                                        \
-        route_select_kernel<KPT><<<grid, THREADS, smem, stream>>>(g, (const float*)ws, seq_lens, P, routed_pages, \
-                                                                 routed_scores);                                \
+        cudaError_t e2 = launch_pdl(route_select_kernel<KPT>, grid, dim3(THREADS), smem, stream, g,            \
+                                    (const float*)ws, seq_lens, P, routed_pages, routed_scores);               \
+        if (e2 != cudaSuccess) return e2;                                                                       \
     }
     if (g.max_pages <= 2048) VSA_SELECT_LAUNCH(8, 256)
     else if (g.max_pages <= 4096) VSA_SELECT_LAUNCH(16, 256)

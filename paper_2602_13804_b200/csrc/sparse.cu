@@ -87,6 +87,8 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, c = lane & 15, gi = lane >> 4;
     const long long unit = blockIdx.x;
     const int b = (int)(unit / geo.n_q_heads), h = (int)(unit % geo.n_q_heads), g = h / geo.group;
+    pdl_wait();
+    pdl_launch_dependents();
     const int T = seq_lens[b];
     if (T <= 0 || T > geo.max_pages * kPageSize) {
         write_failed_unit(out, diag, unit, VSA_UNIT_BAD_LENGTH);
@@ -370,10 +372,9 @@ cudaError_t launch_one(const Geometry& g, size_t smem, const uint16_t* q, const 
         if (e != cudaSuccess) return e;
     }
     const unsigned units = (unsigned)(g.batch * g.n_q_heads);
-    sparse_decode_kernel<PAGE_KPT, TOK_KPT><<<units, kSparseThreads, smem, stream>>>(
-        g, q, k, v, block_table, seq_lens, routed_pages, page_scores, P, K_c, epsilon, gap_threshold, out, diag,
-        fallback_list, fallback_count);
-    return cudaGetLastError();
+    return launch_pdl(sparse_decode_kernel<PAGE_KPT, TOK_KPT>, dim3(units), dim3(kSparseThreads), smem, stream, g, q,
+                      k, v, block_table, seq_lens, routed_pages, page_scores, P, K_c, epsilon, gap_threshold, out,
+                      diag, fallback_list, fallback_count);
 }
 
 template <int PAGE_KPT>

@@ -27,6 +27,15 @@ constexpr int kPageSize = 16;   // tokens per page
 constexpr int kRowBytes = kHeadDim * 2;
 constexpr unsigned kFullMask = 0xffffffffu;
 
+// ---- programmatic dependent launch ----------------------------------------------------------
+// Every kernel of the step is launched with programmatic stream serialization: it may be
+// scheduled while its predecessor in the stream is still running.  pdl_wait() blocks until the
+// predecessor grid has completed and its memory is visible (a no-op for ordinary launches), so
+// it precedes the first access to anything another kernel writes or reads;
+// pdl_launch_dependents() lets the successor start being scheduled.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- bf16 ------------------------------------------------------------------------------
 // A 16-byte vector holds 8 consecutive bf16 values, element 0 in the low half of .x
 __device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8])
