@@ -61,6 +61,7 @@ extern "C" {
 #define VSA_ERR_WORKSPACE_TOO_SMALL (-3)
 #define VSA_ERR_MISALIGNED (-4)        /* a pointer or stride is not 16-byte aligned                  */
 #define VSA_ERR_CUDA (-5)              /* a launch or copy was rejected by the CUDA runtime           */
+#define VSA_ERR_STATIC_SCRATCH_EXCEEDED (-6) /* shape too large for the built-in scratch array       */
 
 typedef struct {
     int32_t batch, n_q_heads, n_kv_heads, head_dim, page_size;
@@ -190,6 +191,30 @@ int vsa_decode_step_host(const vsa_shape_t* shape, const void* q_host, void* q_d
                          float gap_threshold, float* out_host, float* out_dev, vsa_diag_t* diag_host,
                          vsa_diag_t* diag_dev, int32_t* routed_pages, int32_t* fallback_list,
                          int32_t* fallback_count, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Page routing without a caller-provided workspace (no counterpart in the paper: this is a
+ * deployment convenience of the library).  Same inputs, outputs and results as vsa_route_pages,
+ * but the page-score scratch lives in a fixed array inside the library's device image, so the
+ * call needs no device memory from the caller and performs no allocation of any kind.  It is
+ * meant for callers that cannot obtain device memory at call time: an attention backend inside a
+ * serving engine whose KV-cache pool already owns all free HBM (a later cudaMalloc would fail
+ * or stall the device), or code in a decode loop where allocation calls are forbidden.
+ *   Limit: batch * n_q_heads * max_pages_per_seq <= VSA_STATIC_ROUTE_SCORES (one fp32 score per
+ *   unit and logical page; the array occupies 4 MiB on every GPU that loads the library, until
+ *   the process exits).  Larger shapes are rejected with VSA_ERR_STATIC_SCRATCH_EXCEEDED before
+ *   anything is launched.
+ *   The first call on each device looks up the array's device address (with that device
+ *   current); make that first call outside any stream capture.
+ *   All calls share the one array, which keeps the scores of the last call; nothing in it has to
+ *   be cleared, because the selection only reads scores that the scan of the same call wrote.
+ *   Two calls that overlap on the GPU (different streams, or host threads) race on it: serialise
+ *   them, or use vsa_route_pages with separate workspaces.
+ */
+#define VSA_STATIC_ROUTE_SCORES (1 << 20)
+int vsa_route_pages_static(const vsa_shape_t* shape, const void* q, const void* summaries,
+                           const int32_t* block_table, const int32_t* seq_lens, int32_t P,
+                           int32_t* routed_pages, float* routed_scores, void* stream);
 
 /* Scratch bytes needed by one call kind for this shape (0 if the shape is invalid). */
 size_t vsa_workspace_bytes(const vsa_shape_t* shape, int32_t P, int32_t K_c, int which_call);

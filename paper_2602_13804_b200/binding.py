@@ -64,6 +64,8 @@ def lib() -> C.CDLL:
         _lib.vsa_workspace_bytes.argtypes = [shp, i32, i32, C.c_int]
         _lib.vsa_build_page_summaries.argtypes = [shp, vp, vp, vp, vp, vp, vp]
         _lib.vsa_route_pages.argtypes = [shp, vp, vp, vp, vp, i32, vp, vp, vp, sz, vp]
+        _lib.vsa_route_pages_static.argtypes = [shp, vp, vp, vp, vp, i32, vp, vp, vp]
+        _lib.vsa_route_pages_static.restype = C.c_int
         _lib.vsa_sparse_decode.argtypes = [shp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, vp, vp, vp, vp, vp, sz, vp]
         _lib.vsa_dense_decode_fallback.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, f32, vp, vp, vp, sz, vp]
         _lib.vsa_decode_step.argtypes = [shp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -130,6 +132,23 @@ def vsa_route_pages(shape, q, summaries, block_table, seq_lens, P, routed_pages,
                                  _ptr(routed_pages), _ptr(routed_scores), _ptr(ws),
                                  0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
            "vsa_route_pages")
+
+
+VSA_STATIC_ROUTE_SCORES = 1 << 20
+
+
+def vsa_route_pages_static(shape, q, summaries, block_table, seq_lens, P, routed_pages, routed_scores,
+                           stream=None) -> None:
+    """vsa_route_pages for callers that have no device memory to lend (a backend inside an engine whose
+    pool owns all of HBM, a loop where allocation is banned): the score scratch is a fixed 4 MiB array
+    inside the library, so no workspace is passed and nothing is allocated.  Shapes with
+    batch * n_q_heads * max_pages_per_seq > VSA_STATIC_ROUTE_SCORES raise VsaError (-6).  Calls share the
+    array: do not let two of them overlap on the GPU.  Make the first call on a device outside stream
+    capture (it looks up the array's address)."""
+    _check(lib().vsa_route_pages_static(C.byref(shape), _ptr(q), _ptr(summaries), _ptr(block_table),
+                                        _ptr(seq_lens), P, _ptr(routed_pages), _ptr(routed_scores),
+                                        _stream(stream)),
+           "vsa_route_pages_static")
 
 
 def vsa_sparse_decode(shape, q, k_cache, v_cache, block_table, seq_lens, routed_pages, P, K_c, epsilon,

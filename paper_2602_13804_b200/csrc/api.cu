@@ -82,6 +82,8 @@ const char* vsa_strerror(int code)
         case VSA_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
         case VSA_ERR_MISALIGNED: return "pointer or stride not 16-byte aligned";
         case VSA_ERR_CUDA: return "CUDA runtime error";
+        case VSA_ERR_STATIC_SCRATCH_EXCEEDED:
+            return "shape exceeds the built-in scratch array (batch * n_q_heads * max_pages_per_seq > 2^20)";
         default: return "unknown error code";
     }
 }
@@ -278,3 +280,58 @@ int vsa_decode_step_host(const vsa_shape_t* shape, const void* q_host, void* q_d
 }
 
 }  // extern "C"
+
+// ---- routing for callers that cannot allocate ------------------------------------------------------
+// The page-score scratch of vsa_route_pages_static: part of the library's device image, so every GPU
+// that loads the library holds these 4 MiB until the process exits.  In host code the symbol's name
+// is only a handle - it is not a device address and must never be handed to a kernel; the device
+// address is looked up once per device with cudaGetSymbolAddress and cached below.
+static __device__ __align__(256) float vsa_static_route_scratch[VSA_STATIC_ROUTE_SCORES];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+float* g_static_scratch_addr[kMaxDevices];   // per device ordinal; nullptr = not looked up yet
+
+// Device address of the scratch array on the current device.  The first call on a device performs
+// the lookup (it may initialise the device's copy of the module, so it belongs outside stream
+// capture); later calls only read the cached pointer.  Concurrent first calls store the same value.
+int static_scratch_address(float** out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return VSA_ERR_CUDA;
+    float* p = g_static_scratch_addr[dev];
+    if (!p) {
+        void* sym = nullptr;
+        if (cudaGetSymbolAddress(&sym, vsa_static_route_scratch) != cudaSuccess || !sym) return VSA_ERR_CUDA;
+        p = static_cast<float*>(sym);
+        g_static_scratch_addr[dev] = p;
+    }
+    *out = p;
+    return VSA_OK;
+}
+
+}  // namespace
+
+extern "C" int vsa_route_pages_static(const vsa_shape_t* shape, const void* q, const void* summaries,
+                                      const int32_t* block_table, const int32_t* seq_lens, int32_t P,
+                                      int32_t* routed_pages, float* routed_scores, void* stream)
+{
+    Geometry g;
+    int rc = make_geometry(shape, &g);
+    if (rc) return rc;
+    if ((rc = check_routing_sizes(g, P, 0, false))) return rc;
+    if (!q || !summaries || !block_table || !seq_lens || !routed_pages) return VSA_ERR_INVALID_ARGUMENT;
+    if (!aligned16(q) || !aligned16(summaries)) return VSA_ERR_MISALIGNED;
+    // one fp32 score per (unit, logical page) must fit the fixed array
+    if ((unsigned long long)g.batch * g.n_q_heads * g.max_pages > (unsigned long long)VSA_STATIC_ROUTE_SCORES)
+        return VSA_ERR_STATIC_SCRATCH_EXCEEDED;
+    float* scratch = nullptr;
+    if ((rc = static_scratch_address(&scratch))) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    // nothing in the array needs clearing: the selection reads scores [0, n_b) of every unit, all of
+    // which the scan below writes first; whatever an earlier call left beyond n_b is never read
+    cudaError_t e = vsa::launch_route_scan(g, q, summaries, block_table, seq_lens, scratch, nullptr, nullptr, 0, st);
+    if (e != cudaSuccess) return VSA_ERR_CUDA;
+    return cuda_rc(vsa::launch_route_select(g, scratch, seq_lens, P, routed_pages, routed_scores, st));
+}

@@ -41,7 +41,7 @@ def test_struct_layouts_match_the_header():
 
 
 def test_strerror_covers_all_codes(lib):
-    texts = {c: B.vsa_strerror(c) for c in (0, -1, -2, -3, -4, -5, -99)}
+    texts = {c: B.vsa_strerror(c) for c in (0, -1, -2, -3, -4, -5, -6, -99)}
     assert texts[0] == "ok" and "unknown" in texts[-99]
     assert len(set(texts.values())) == len(texts)
 
