@@ -114,6 +114,22 @@ class ClockSampler:
                 "power_w_max": max(float(r[2]) for r in rows), "reasons": reasons, "samples": len(rows)}
 
 
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """Time of the slowest rank: every rank decodes its own sequences, the job is done when all are."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def us_per_token_per_layer(ms_per_step: float, world: int, batch_per_rank: int, layers: int) -> float:
+    """Whole-job figure: one step decodes world * batch tokens through `layers` layers."""
+    return ms_per_step * 1e3 / (world * batch_per_rank * layers)
+
+
 def host_bits(t):
     import numpy as np
     import torch
@@ -283,11 +299,7 @@ def run_ours(args):
         e1.record(stream)
         barrier()
         t_wall1 = time.time()
-        ms_total = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms_total], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_total = float(t.item())
+        ms_total = max_over_ranks(e0.elapsed_time(e1), world, dev)
         ms_per_step = ms_total / args.steps
         # keep the GPU loaded a little longer if the region was too short to sample clocks
         if t_wall1 - t_wall0 < 0.5:
@@ -350,15 +362,10 @@ def run_ours(args):
                 step_e2e()
             e1.record(stream)
             barrier()
-            ms_e2e = e0.elapsed_time(e1)
-            if world > 1:
-                t = torch.tensor([ms_e2e], device=dev)
-                dist.all_reduce(t, op=dist.ReduceOp.MAX)
-                ms_e2e = float(t.item())
-            ms_e2e /= args.steps
+            ms_e2e = max_over_ranks(e0.elapsed_time(e1), world, dev) / args.steps
             h2d = L * units * 128 * 2
             d2h = L * units * (128 * 4 + B.DIAG_BYTES)
-            e2e = {"value": ms_e2e * 1e3 / (world * shape.batch * L), "unit": UNIT, "ms_per_step": ms_e2e,
+            e2e = {"value": us_per_token_per_layer(ms_e2e, world, shape.batch, L), "unit": UNIT, "ms_per_step": ms_e2e,
                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                    "api": "vsa_decode_step_host per layer, plain stream launches, one stream sync per step"}
 
@@ -397,7 +404,7 @@ def run_ours(args):
                         "sample": f"layer 0 of {L}, all {shape.batch} sequences, {reps} repetitions of one "
                                   f"oracle decode step (summaries prebuilt)"}
 
-    value = ms_per_step * 1e3 / (world * shape.batch * L)
+    value = us_per_token_per_layer(ms_per_step, world, shape.batch, L)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
