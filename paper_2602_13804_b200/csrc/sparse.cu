@@ -15,15 +15,13 @@ namespace vsa {
 
 namespace {
 
-constexpr int kSparseThreads = 256;
-constexpr int kSparseWarps = kSparseThreads / 32;
-constexpr int kGroups = 2 * kSparseWarps;   // half-warps per block
+constexpr int kMaxSparseWarps = 16;
 
 // token-phase shared memory, in 4-byte words, after the two page arrays
 __host__ __device__ constexpr int token_phase_words(int P, int K_c)
 {
     return P * kPageSize /*keys*/ + (P * kPageSize + 3) / 4 /*take*/ + K_c /*sel*/ + 256 + 16 + 72 + kTopkList +
-           kSparseWarps * kHeadDim + kSparseWarps + 4;
+           kMaxSparseWarps * kHeadDim + kMaxSparseWarps + 4;
 }
 
 struct TokenSmem {
@@ -47,7 +45,7 @@ __device__ __forceinline__ TokenSmem carve_tokens(uint32_t* base, int P, int K_c
     s.ts.wred = s.ts.misc + 16;
     s.ts.list = (int32_t*)(s.ts.wred + 72);
     s.red = (float*)(s.ts.list + kTopkList);
-    s.zred = s.red + kSparseWarps * kHeadDim;
+    s.zred = s.red + kMaxSparseWarps * kHeadDim;
     return s;
 }
 
@@ -64,14 +62,16 @@ __device__ __forceinline__ void write_failed_unit(float* out, vsa_diag_t* diag, 
     }
 }
 
+// THREADS: 256 (two blocks per SM; the throughput shape) or 512 (one block per SM; used when there
+//   are no more units than SMs, so that one unit gets twice the loads in flight and half the passes).
 // PAGE_KPT ==  0: routed_pages is an input.
 // PAGE_KPT == -1: fused with routing; page scores staged in shared memory (any block-table width).
 // PAGE_KPT  >  0: fused with routing; each thread keeps PAGE_KPT page scores in registers.
 //   In both fused forms the unit's top-P pages are selected here from page_scores[unit][0..n_b) and
 //   written to routed_pages (best first, -1 padded).
-// TOK_KPT: token scores per thread, P * 16 <= TOK_KPT * 256.
-template <int PAGE_KPT, int TOK_KPT>
-__global__ void __launch_bounds__(kSparseThreads, 2)
+// TOK_KPT: token scores per thread, P * 16 <= TOK_KPT * THREADS.
+template <int THREADS, int PAGE_KPT, int TOK_KPT>
+__global__ void __launch_bounds__(THREADS, 512 / THREADS)
 sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* __restrict__ k_cache,
                      const uint16_t* __restrict__ v_cache, const int32_t* __restrict__ block_table,
                      const int32_t* __restrict__ seq_lens, int32_t* __restrict__ routed_pages,
@@ -79,6 +79,8 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                      float* __restrict__ out, vsa_diag_t* __restrict__ diag, int32_t* __restrict__ fallback_list,
                      int32_t* __restrict__ fallback_count)
 {
+    constexpr int WARPS = THREADS / 32, GROUPS = 2 * WARPS;
+    static_assert(TOK_KPT * WARPS <= 64 && 3 * WARPS <= 72, "wred capacity");
     extern __shared__ uint32_t smem_raw[];
     int32_t* page_l = (int32_t*)smem_raw;   // [P] routed logical pages, ascending, invalid entries last
     int32_t* page_phys = page_l + P;        // [P]
@@ -93,7 +95,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     if (T <= 0 || T > geo.max_pages * kPageSize) {
         write_failed_unit(out, diag, unit, VSA_UNIT_BAD_LENGTH);
         if (PAGE_KPT != 0)
-            for (int t = tid; t < P; t += kSparseThreads) routed_pages[unit * P + t] = -1;
+            for (int t = tid; t < P; t += THREADS) routed_pages[unit * P + t] = -1;
         return;
     }
     const int nb = (T + kPageSize - 1) / kPageSize;
@@ -109,7 +111,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
             np = select_top_pages_reg<PAGE_KPT>(page_scores + unit * geo.max_pages, nb, P, ps);
         else
             np = select_top_pages(page_scores + unit * geo.max_pages, nb, P, ps);
-        for (int t = tid; t < P; t += kSparseThreads) {
+        for (int t = tid; t < P; t += THREADS) {
             routed_pages[unit * P + t] = t < np ? ps.win_idx[t] : -1;
             int l = INT_MAX, phys = -1;
             if (t < np) {
@@ -125,12 +127,12 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         }
     } else {
         int32_t* raw = (int32_t*)region;   // staging; dead before the token phase reuses the region
-        for (int t = tid; t < P; t += kSparseThreads) {
+        for (int t = tid; t < P; t += THREADS) {
             const int l = routed_pages[unit * P + t];
             raw[t] = (l >= 0 && l < nb) ? l : INT_MAX;
         }
         __syncthreads();
-        for (int t = tid; t < P; t += kSparseThreads) {
+        for (int t = tid; t < P; t += THREADS) {
             const int l = raw[t];
             int rank = 0;
 #pragma unroll 8
@@ -146,7 +148,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
             page_l[rank] = l;
             page_phys[rank] = phys;
         }
-        // (P <= 128 < blockDim.x: thread t < P owns slot t in the count)
+        // (P <= 128 < THREADS: thread t < P owns slot t in the count)
         np = __syncthreads_count(tid < P && raw[tid < P ? tid : 0] != INT_MAX);
     }
     VSA_PROBE(1);
@@ -157,7 +159,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     const TokenSmem sm = carve_tokens(region, P, K_c);
 #pragma unroll
     for (int j = 0; j < TOK_KPT; ++j)
-        if (tid + j * kSparseThreads < N) sm.keys[tid + j * kSparseThreads] = 0u;
+        if (tid + j * THREADS < N) sm.keys[tid + j * THREADS] = 0u;
     __syncthreads();
 
     VSA_PROBE(2);
@@ -167,7 +169,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         const uint4 v = *reinterpret_cast<const uint4*>(q + unit * kHeadDim + c * 8);
         unpack8(v, qf);
     }
-    for (int pp = warp; pp * 2 < np; pp += kSparseWarps) {
+    for (int pp = warp; pp * 2 < np; pp += WARPS) {
         const int slot = pp * 2 + gi;
         const bool active = slot < np;
         uint4 rows[kPageSize];
@@ -199,7 +201,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     uint32_t a1 = 0u, a2 = 0u;   // best and second-best key (multiset order statistics)
 #pragma unroll
     for (int j = 0; j < TOK_KPT; ++j) {
-        const int i = tid + j * kSparseThreads;
+        const int i = tid + j * THREADS;
         key[j] = i < N ? sm.keys[i] : 0u;
         present += key[j] != 0u;
         if (key[j] > a1) {
@@ -227,7 +229,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     uint32_t key1 = 0u, key2 = 0u;
     int n_valid = 0;
 #pragma unroll
-    for (int w = 0; w < kSparseWarps; ++w) {
+    for (int w = 0; w < WARPS; ++w) {
         const uint32_t b1 = sm.ts.wred[3 * w], b2 = sm.ts.wred[3 * w + 1];
         const uint32_t n1 = max(key1, b1), n2 = max(min(key1, b1), max(key2, b2));
         key1 = n1;
@@ -247,7 +249,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         mask = r.mask;
 #pragma unroll
         for (int j = 0; j < TOK_KPT; ++j)
-            if (tid + j * kSparseThreads == r.kth_idx) mask &= ~(1u << j);
+            if (tid + j * THREADS == r.kth_idx) mask &= ~(1u << j);
     } else {
 #pragma unroll
         for (int j = 0; j < TOK_KPT; ++j)
@@ -262,20 +264,21 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         for (int j = 0; j < TOK_KPT; ++j) {
             const unsigned bal = __ballot_sync(kFullMask, (mask >> j) & 1u);
             before[j] = __popc(bal & ((1u << lane) - 1u));
-            if (lane == 0) sm.ts.wred[j * kSparseWarps + warp] = (uint32_t)__popc(bal);
+            if (lane == 0) sm.ts.wred[j * WARPS + warp] = (uint32_t)__popc(bal);
         }
         __syncthreads();
         int base = 0;
 #pragma unroll
         for (int j = 0; j < TOK_KPT; ++j) {
-            // elements of row j (indices j * 256 + tid) come after all of rows < j
+            // elements of row j (indices j * THREADS + tid) come after all of rows < j
             int mine = base;
-            for (int w = 0; w < kSparseWarps; ++w) {
-                const int cw = (int)sm.ts.wred[j * kSparseWarps + w];
+#pragma unroll
+            for (int w = 0; w < WARPS; ++w) {
+                const int cw = (int)sm.ts.wred[j * WARPS + w];
                 if (w < warp) mine += cw;
                 base += cw;
             }
-            if ((mask >> j) & 1u) sm.sel[mine + before[j]] = tid + j * kSparseThreads;
+            if ((mask >> j) & 1u) sm.sel[mine + before[j]] = tid + j * THREADS;
         }
     }
     __syncthreads();
@@ -289,12 +292,12 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     for (int e = 0; e < 8; ++e) acc[e] = 0.0f;
     const int gidx = warp * 2 + gi;
     constexpr int UNR = 8;
-    for (int j0 = gidx; j0 < ns; j0 += kGroups * UNR) {
+    for (int j0 = gidx; j0 < ns; j0 += GROUPS * UNR) {
         uint4 rows[UNR];
         float w[UNR];
 #pragma unroll
         for (int u = 0; u < UNR; ++u) {
-            const int j = j0 + u * kGroups;
+            const int j = j0 + u * GROUPS;
             rows[u] = make_uint4(0u, 0u, 0u, 0u);
             w[u] = 0.0f;
             if (j < ns) {
@@ -326,11 +329,11 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     __syncthreads();
     float Z = 0.0f;
 #pragma unroll
-    for (int w = 0; w < kSparseWarps; ++w) Z += sm.zred[w];
+    for (int w = 0; w < WARPS; ++w) Z += sm.zred[w];
     if (tid < kHeadDim) {
         float a = 0.0f;
 #pragma unroll
-        for (int w = 0; w < kSparseWarps; ++w) a += sm.red[w * kHeadDim + tid];
+        for (int w = 0; w < WARPS; ++w) a += sm.red[w * kHeadDim + tid];
         out[unit * kHeadDim + tid] = ns > 0 ? a / Z : 0.0f;
     }
 
@@ -360,35 +363,69 @@ size_t sparse_smem_bytes(const Geometry& g, int P, int K_c, bool fused)
     return (size_t)(2 * P + words) * 4 + 16;
 }
 
-template <int PAGE_KPT, int TOK_KPT>
-cudaError_t launch_one(const Geometry& g, size_t smem, const uint16_t* q, const uint16_t* k, const uint16_t* v,
-                       const int32_t* block_table, const int32_t* seq_lens, int32_t* routed_pages,
-                       const float* page_scores, int P, int K_c, float epsilon, float gap_threshold, float* out,
-                       vsa_diag_t* diag, int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream)
+struct SparseArgs {
+    Geometry g;
+    size_t smem;
+    const uint16_t *q, *k, *v;
+    const int32_t *block_table, *seq_lens;
+    int32_t* routed_pages;
+    const float* page_scores;
+    int P, K_c;
+    float epsilon, gap_threshold;
+    float* out;
+    vsa_diag_t* diag;
+    int32_t *fallback_list, *fallback_count;
+    cudaStream_t stream;
+};
+
+template <int THREADS, int PAGE_KPT, int TOK_KPT>
+cudaError_t launch_one(const SparseArgs& a)
 {
-    if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(sparse_decode_kernel<PAGE_KPT, TOK_KPT>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (a.smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(sparse_decode_kernel<THREADS, PAGE_KPT, TOK_KPT>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)a.smem);
         if (e != cudaSuccess) return e;
     }
-    const unsigned units = (unsigned)(g.batch * g.n_q_heads);
-    return launch_pdl(sparse_decode_kernel<PAGE_KPT, TOK_KPT>, dim3(units), dim3(kSparseThreads), smem, stream, g, q,
-                      k, v, block_table, seq_lens, routed_pages, page_scores, P, K_c, epsilon, gap_threshold, out,
-                      diag, fallback_list, fallback_count);
+    const unsigned units = (unsigned)(a.g.batch * a.g.n_q_heads);
+    return launch_pdl(sparse_decode_kernel<THREADS, PAGE_KPT, TOK_KPT>, dim3(units), dim3(THREADS), a.smem, a.stream,
+                      a.g, a.q, a.k, a.v, a.block_table, a.seq_lens, a.routed_pages, a.page_scores, a.P, a.K_c,
+                      a.epsilon, a.gap_threshold, a.out, a.diag, a.fallback_list, a.fallback_count);
 }
 
-template <int PAGE_KPT>
-cudaError_t launch_tok(const Geometry& g, size_t smem, const uint16_t* q, const uint16_t* k, const uint16_t* v,
-                       const int32_t* block_table, const int32_t* seq_lens, int32_t* routed_pages,
-                       const float* page_scores, int P, int K_c, float epsilon, float gap_threshold, float* out,
-                       vsa_diag_t* diag, int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream)
+template <int THREADS, int PAGE_KPT>
+cudaError_t launch_tok(const SparseArgs& a)
 {
-    const int N = P * kPageSize;
-#define VSA_ARGS g, smem, q, k, v, block_table, seq_lens, routed_pages, page_scores, P, K_c, epsilon, gap_threshold, \
-                 out, diag, fallback_list, fallback_count, stream
-    if (N <= 2 * kSparseThreads) return launch_one<PAGE_KPT, 2>(VSA_ARGS);
-    if (N <= 4 * kSparseThreads) return launch_one<PAGE_KPT, 4>(VSA_ARGS);
-    return launch_one<PAGE_KPT, 8>(VSA_ARGS);
+    const int N = a.P * kPageSize;
+    if (N <= 2 * THREADS) return launch_one<THREADS, PAGE_KPT, 2>(a);
+    if (N <= 4 * THREADS) return launch_one<THREADS, PAGE_KPT, 4>(a);
+    if constexpr (THREADS == 256)
+        return launch_one<THREADS, PAGE_KPT, 8>(a);
+    else
+        return cudaErrorInvalidValue;   // 128 pages * 16 tokens = 4 * 512: never reached
+}
+
+template <int THREADS>
+cudaError_t launch_threads(const SparseArgs& a)
+{
+    if (!a.page_scores) return launch_tok<THREADS, 0>(a);
+    if (a.g.max_pages <= 8 * THREADS) return launch_tok<THREADS, 8>(a);
+    if (a.g.max_pages <= 16 * THREADS) return launch_tok<THREADS, 16>(a);
+    if (a.g.max_pages <= 32 * THREADS) return launch_tok<THREADS, 32>(a);
+    return launch_tok<THREADS, -1>(a);
+}
+
+int g_sm_count = 0;
+int sm_count()
+{
+    if (g_sm_count == 0) {
+        int dev = 0, n = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+            g_sm_count = n;
+        else
+            return 148;
+    }
+    return g_sm_count;
 }
 
 }  // namespace
@@ -405,18 +442,28 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
                           const float* page_scores, int P, int K_c, float epsilon, float gap_threshold, float* out,
                           vsa_diag_t* diag, int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream)
 {
-    const size_t smem = sparse_smem_bytes(g, P, K_c, page_scores != nullptr);
-    const uint16_t *qq = (const uint16_t*)q, *k = (const uint16_t*)k_cache, *v = (const uint16_t*)v_cache;
-    const uint16_t* q_ = qq;
-#undef VSA_ARGS
-#define VSA_ARGS g, smem, q_, k, v, block_table, seq_lens, routed_pages, page_scores, P, K_c, epsilon, gap_threshold, \
-                 out, diag, fallback_list, fallback_count, stream
-    if (!page_scores) return launch_tok<0>(VSA_ARGS);
-    if (g.max_pages <= 8 * kSparseThreads) return launch_tok<8>(VSA_ARGS);
-    if (g.max_pages <= 16 * kSparseThreads) return launch_tok<16>(VSA_ARGS);
-    if (g.max_pages <= 32 * kSparseThreads) return launch_tok<32>(VSA_ARGS);
-    return launch_tok<-1>(VSA_ARGS);
-#undef VSA_ARGS
+    SparseArgs a;
+    a.g = g;
+    a.smem = sparse_smem_bytes(g, P, K_c, page_scores != nullptr);
+    a.q = (const uint16_t*)q;
+    a.k = (const uint16_t*)k_cache;
+    a.v = (const uint16_t*)v_cache;
+    a.block_table = block_table;
+    a.seq_lens = seq_lens;
+    a.routed_pages = routed_pages;
+    a.page_scores = page_scores;
+    a.P = P;
+    a.K_c = K_c;
+    a.epsilon = epsilon;
+    a.gap_threshold = gap_threshold;
+    a.out = out;
+    a.diag = diag;
+    a.fallback_list = fallback_list;
+    a.fallback_count = fallback_count;
+    a.stream = stream;
+    // no more units than SMs: one larger block per unit (latency shape); otherwise two blocks per SM
+    if ((long long)g.batch * g.n_q_heads <= sm_count()) return launch_threads<512>(a);
+    return launch_threads<256>(a);
 }
 
 }  // namespace vsa

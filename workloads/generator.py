@@ -170,14 +170,19 @@ def make_workload(spec: WorkloadSpec, seed: Optional[int] = None, device="cpu",
     """Draw one cache + query batch.
 
     Host-side structure (lengths, block tables, needle positions) always comes
-    from a CPU generator seeded with ``seed``; the large tensors are drawn on
-    ``device`` with a generator of that device seeded with ``seed + 1``.
+    from a CPU generator seeded with ``seed`` (default: ``seed_for(config, sub)``);
+    the large tensors are drawn on ``device`` with a generator of that device
+    seeded with ``seed + 1 + rep``, so ``rep`` selects one of several caches with
+    identical structure and different contents (the layers of one model).
     """
+    # `rep` (the layer-cache index) changes the contents only: all layer caches of one workload share
+    # the sequence lengths, block tables and needle positions, as the layers of one model do
     if seed is None:
-        seed = seed_for(spec.config, sub, rep)
+        seed = seed_for(spec.config, sub, 0)
     device = torch.device(device)
     hgen = torch.Generator(device="cpu").manual_seed(seed)
-    dgen = torch.Generator(device=device).manual_seed(seed + 1)
+    dgen = torch.Generator(device=device).manual_seed(seed + 1 + int(rep))
+    seed = seed + int(rep)
 
     B, Hq, Hkv, d, bs = spec.batch, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, spec.page_size
     assert Hq % Hkv == 0
