@@ -1,9 +1,19 @@
 // Dense fallback (paper Sec. 10.3, "fallback-to-dense"): plain softmax attention over every token of
-// the flagged units, as a split-K pass over the paged cache.  A work item is one (sequence, KV head,
-// token range): K and V are read once for all query heads of the group, every half-warp keeps an
-// online-softmax state over its own pages, and the partial (max, sum, acc) triples are merged by the
-// last block that finishes an item of a (sequence, KV head).  The grid is persistent: a fixed number
-// of blocks walk the item list, so a step without any flagged unit costs one nearly empty launch.
+// the flagged units, as a split-K pass over the paged cache.
+//
+// This is the one place of the step where the arithmetic is a real dense contraction - the G query
+// heads of a GQA group against the same K and V tiles - and where only the output (not a discrete
+// decision) depends on it, so it runs on the tensor cores: per 16-token page and warp,
+//   S[heads x 16]  = Q[heads x 128] . K_page^T      (16 mma.m16n8k16, bf16 in, fp32 accumulate)
+//   O[heads x 128] += P[heads x 16] . V_page        (16 mma.m16n8k16)
+// with the heads padded to the 16-row MMA tile and an online softmax in between.  K and V tiles
+// stream through a per-warp cp.async ring (three pages deep, XOR-swizzled for ldmatrix).
+//
+// Work decomposition: an item is (sequence, KV head, range of pages); K and V are read once for all
+// listed heads of the group.  The number of pages per item is chosen ON THE DEVICE from how much
+// was flagged, so that one flagged head of a 128k-token sequence is spread over the whole chip
+// while a full dense pass uses long items.  A persistent grid (one block per SM) walks the items;
+// the block that finishes the last item of a (sequence, KV head) combines its partials.
 #include <math.h>
 
 #include "vsa_device.cuh"
@@ -15,28 +25,78 @@ namespace {
 
 constexpr int kDenseThreads = 256;
 constexpr int kDenseWarps = kDenseThreads / 32;
-constexpr int kDenseGroups = 2 * kDenseWarps;
+constexpr int kStages = 3;                         // pages in flight per warp
+constexpr int kTileBytes = kPageSize * kRowBytes;  // 4 KB: K (or V) rows of one page and KV head
+constexpr int kStageBytes = 2 * kTileBytes;        // K tile + V tile
+constexpr int kRingBytes = kDenseWarps * kStages * kStageBytes;   // 192 KB per block
+constexpr int kPartialFloats = 2 + kHeadDim;       // per (item, head): max (log2 domain), sum, acc[128]
+constexpr int kMaxGroups = 4096;                   // batch * n_kv_heads the bookkeeping arrays can hold
+constexpr int kItemsPerBlockTarget = 2;
+constexpr int kMinPagesPerItem = 2 * kDenseWarps;  // at least two pages per warp: one would expose the DRAM latency
 
-// partial record per (unit, split): [0] = running max (log2 domain), [1] = sum, [2..130) = acc
-constexpr int kPartialFloats = 2 + kHeadDim;
+__device__ __forceinline__ void cp_async_16_zfill(uint32_t smem_addr, const void* gptr, bool valid)
+{
+    const int n = valid ? 16 : 0;   // src-size 0: the 16 destination bytes are zero-filled
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_addr), "l"(gptr), "r"(n) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait()
+{
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+// D (16x8, fp32) += A (16x16, bf16, row) * B (16x8, bf16, col); rows 8..15 of A are zero here
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1)
+{
+    const uint32_t zero = 0u;
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+                 "{%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(zero), "r"(a2), "r"(zero), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+struct DenseSmem {
+    uint8_t* ring;         // [warps][stages][K tile | V tile]; reused for the cross-warp merge
+    int32_t* item_base;    // [n_groups + 1] first item of every group (exclusive scan)
+    uint8_t* group_mask;   // [n_groups] listed heads of the group
+    int32_t* misc;         // [16]
+};
 
 template <int G>
-__global__ void __launch_bounds__(kDenseThreads)
+__global__ void __launch_bounds__(kDenseThreads, 1)
 dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* __restrict__ k_cache,
                    const uint16_t* __restrict__ v_cache, const int32_t* __restrict__ block_table,
                    const int32_t* __restrict__ seq_lens, const int32_t* __restrict__ fallback_list,
                    const int32_t* __restrict__ fallback_count, float epsilon, float* __restrict__ partials,
                    int32_t* __restrict__ counters, float* __restrict__ out, vsa_diag_t* __restrict__ diag,
-                   int pages_per_split, int n_splits)
+                   int max_items)
 {
-    constexpr int ROWS = 16 / G;   // token rows per half-warp per step
-    __shared__ float sm_m[kDenseWarps][G], sm_l[kDenseWarps][G];
-    __shared__ float sm_acc[kDenseWarps][G][kHeadDim];
-    __shared__ int sm_last;
-    extern __shared__ uint8_t sm_group_mask[];   // [batch * n_kv_heads] heads of each group that are listed
-
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, c = lane & 15, gi = lane >> 4;
+    extern __shared__ __align__(128) uint8_t dense_smem[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n_groups = geo.batch * geo.n_kv_heads;
+    DenseSmem sm;
+    sm.ring = dense_smem;
+    sm.item_base = (int32_t*)(dense_smem + kRingBytes);
+    sm.misc = sm.item_base + n_groups + 1;
+    sm.group_mask = (uint8_t*)(sm.misc + 16);
     pdl_wait();
     pdl_launch_dependents();
 
@@ -44,147 +104,242 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
     if (fallback_count) {
         const int count = *fallback_count;
         if (count <= 0) return;
-        for (int i = tid; i < n_groups; i += kDenseThreads) sm_group_mask[i] = 0;
+        for (int i = tid; i < n_groups; i += kDenseThreads) sm.group_mask[i] = 0;
         __syncthreads();
         for (int i = tid; i < count; i += kDenseThreads) {
             const int u = fallback_list[i];
             const int ub = u / geo.n_q_heads, uh = u % geo.n_q_heads;
-            // byte-wide OR through the aligned 32-bit word that holds the group's byte
             const int grp = ub * geo.n_kv_heads + uh / G;
-            atomicOr(reinterpret_cast<unsigned int*>(sm_group_mask) + (grp >> 2), (1u << (uh % G)) << (8 * (grp & 3)));
+            // byte-wide OR through the aligned 32-bit word that holds the group's byte
+            atomicOr(reinterpret_cast<unsigned int*>(sm.group_mask) + (grp >> 2), (1u << (uh % G)) << (8 * (grp & 3)));
         }
     } else {
-        for (int i = tid; i < n_groups; i += kDenseThreads) sm_group_mask[i] = (uint8_t)((1u << G) - 1u);
+        for (int i = tid; i < n_groups; i += kDenseThreads) sm.group_mask[i] = (uint8_t)((1u << G) - 1u);
     }
+    if (tid < 16) sm.misc[tid] = 0;
     __syncthreads();
 
+    // ---- pages per item from the amount of flagged work, then the item table ----
+    auto pages_of = [&](int grp) -> int {
+        if (!sm.group_mask[grp]) return 0;
+        const int T = seq_lens[grp / geo.n_kv_heads];
+        if (T <= 0 || T > geo.max_pages * kPageSize) return 0;
+        return (T + kPageSize - 1) / kPageSize;
+    };
+    {
+        int pages = 0, groups = 0;
+        for (int i = tid; i < n_groups; i += kDenseThreads) {
+            const int p = pages_of(i);
+            pages += p;
+            groups += p > 0;
+        }
+#pragma unroll
+        for (int off = 16; off; off >>= 1) {
+            pages += __shfl_xor_sync(kFullMask, pages, off);
+            groups += __shfl_xor_sync(kFullMask, groups, off);
+        }
+        if (lane == 0) {
+            atomicAdd(&sm.misc[0], pages);
+            atomicAdd(&sm.misc[1], groups);
+        }
+    }
+    __syncthreads();
+    const int total_pages = sm.misc[0], flagged_groups = sm.misc[1];
+    if (total_pages == 0) return;
+    int ppi;   // pages per item, a multiple of the warp count
+    {
+        const long long target = (long long)gridDim.x * kItemsPerBlockTarget;
+        long long want = (total_pages + target - 1) / target;
+        const long long room = max_items - flagged_groups;   // every group may add one ragged item
+        const long long need = (total_pages + room - 1) / room;
+        if (want < need) want = need;
+        ppi = (int)((want + kDenseWarps - 1) / kDenseWarps) * kDenseWarps;
+        if (ppi < kMinPagesPerItem) ppi = kMinPagesPerItem;
+    }
+    {
+        // exclusive scan of items per group: contiguous ranges per thread, then across threads
+        const int per = (n_groups + kDenseThreads - 1) / kDenseThreads;
+        const int lo = tid * per, hi = min(n_groups, lo + per);
+        int mine = 0;
+        for (int i = lo; i < hi; ++i) mine += (pages_of(i) + ppi - 1) / ppi;
+        int incl = mine;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int o = __shfl_up_sync(kFullMask, incl, off);
+            if (lane >= off) incl += o;
+        }
+        if (lane == 31) sm.misc[4 + warp] = incl;
+        __syncthreads();
+        int base = incl - mine;
+        for (int w = 0; w < warp; ++w) base += sm.misc[4 + w];
+        for (int i = lo; i < hi; ++i) {
+            sm.item_base[i] = base;
+            base += (pages_of(i) + ppi - 1) / ppi;
+        }
+        if (tid == kDenseThreads - 1) sm.item_base[n_groups] = base;
+    }
+    __syncthreads();
+    const int n_items = sm.item_base[n_groups];
+
     const float scale = 1.4426950408889634f / epsilon;   // scores are kept in the log2 domain
-    const long long n_items = (long long)n_groups * n_splits;
-    for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
-        const int grp = (int)(item / n_splits), split = (int)(item % n_splits);
-        const uint32_t mask = sm_group_mask[grp];
-        if (mask == 0u) continue;
+    const int head = lane >> 2;                          // MMA row of this lane = query head in the group
+    const int quad = lane & 3;
+    uint8_t* my_ring = sm.ring + warp * kStages * kStageBytes;
+    const uint32_t ring_addr = (uint32_t)__cvta_generic_to_shared(my_ring);
+    // copy mapping: lane covers 16-byte chunk (lane & 15) of rows (lane >> 4) + 2 i, i = 0..7
+    const int cp_chunk = lane & 15, cp_row0 = lane >> 4;
+
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+        // group of this item: last g with item_base[g] <= item
+        int glo = 0, ghi = n_groups;
+        while (ghi - glo > 1) {
+            const int mid = (glo + ghi) >> 1;
+            if (sm.item_base[mid] <= item) glo = mid; else ghi = mid;
+        }
+        const int grp = glo;
+        const uint32_t mask = sm.group_mask[grp];
         const int b = grp / geo.n_kv_heads, g = grp % geo.n_kv_heads;
         const int T = seq_lens[b];
-        if (T <= 0 || T > geo.max_pages * kPageSize) continue;
         const int nb = (T + kPageSize - 1) / kPageSize;
-        const int first_page = split * pages_per_split;
-        if (first_page >= nb) continue;
-        const int end_page = min(nb, first_page + pages_per_split);
-        const int active_splits = (nb + pages_per_split - 1) / pages_per_split;
-
-        float qf[G][8];
-#pragma unroll
-        for (int hh = 0; hh < G; ++hh) {
-            const uint4 v = *reinterpret_cast<const uint4*>(
-                q + ((long long)b * geo.n_q_heads + g * G + hh) * kHeadDim + c * 8);
-            unpack8(v, qf[hh]);
-        }
-        float m[G], l[G], acc[G][8];
-#pragma unroll
-        for (int hh = 0; hh < G; ++hh) {
-            m[hh] = -INFINITY;
-            l[hh] = 0.0f;
-#pragma unroll
-            for (int e = 0; e < 8; ++e) acc[hh][e] = 0.0f;
-        }
-
+        const int chunk = item - sm.item_base[grp];
+        const int items_of_group = sm.item_base[grp + 1] - sm.item_base[grp];
+        // the group's pages are split evenly over its items (whole multiples of the warp count)
+        const int even = ((nb + items_of_group - 1) / items_of_group + kDenseWarps - 1) / kDenseWarps * kDenseWarps;
+        const int first_page = min(nb, chunk * even);
+        const int end_page = min(nb, first_page + even);
         const int32_t* bt = block_table + (long long)b * geo.max_pages;
-        // both half-warps of a warp run the same number of iterations (shuffles need all 32 lanes)
-        for (int pl0 = first_page + warp * 2; pl0 < end_page; pl0 += kDenseGroups) {
-            const int pl = pl0 + gi;
-            bool page_ok = pl < end_page;
-            long long phys = 0;
-            if (page_ok) {
-                phys = bt[pl];
-                page_ok = phys >= 0 && phys < geo.pool_pages;
-                if (!page_ok) phys = 0;
-            }
-            const uint16_t* kp = k_cache + phys * geo.page_stride + (long long)g * geo.head_stride + c * 8;
-            const uint16_t* vp = v_cache + phys * geo.page_stride + (long long)g * geo.head_stride + c * 8;
-#pragma unroll 1
-            for (int step = 0; step < G; ++step) {
-                uint4 kr[ROWS], vr[ROWS];
+
+        // Q fragments of the group: bf16 pairs straight from memory, rows >= G are zero
+        uint32_t qa0[8], qa2[8];
+        {
+            const uint16_t* qrow = q + ((long long)b * geo.n_q_heads + g * G + (head < G ? head : 0)) * kHeadDim;
 #pragma unroll
-                for (int r = 0; r < ROWS; ++r) {
-                    const int t = step * ROWS + r;
-                    const bool ok = page_ok && pl * kPageSize + t < T;
-                    kr[r] = make_uint4(0u, 0u, 0u, 0u);
-                    vr[r] = make_uint4(0u, 0u, 0u, 0u);
-                    if (ok) {
-                        kr[r] = ld_nc_16B(kp + (long long)t * geo.token_stride);
-                        vr[r] = ld_nc_16B(vp + (long long)t * geo.token_stride);
-                    }
-                }
-                float vals[16];
-#pragma unroll
-                for (int r = 0; r < ROWS; ++r) {
-                    float kf[8];
-                    unpack8(kr[r], kf);
-#pragma unroll
-                    for (int hh = 0; hh < G; ++hh) vals[r * G + hh] = chunk_partial(qf[hh], kf);
-                }
-                const float s_own = reduce_scatter16(vals, c);   // lane c: (row c / G, head c % G)
-                const bool own_ok = page_ok && pl * kPageSize + step * ROWS + c / G < T;
-                const float t_own = own_ok ? s_own * scale : -INFINITY;
-                float sv[16];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) sv[i] = __shfl_sync(kFullMask, t_own, (lane & 16) | i);
-                float vf[ROWS][8];
-#pragma unroll
-                for (int r = 0; r < ROWS; ++r) unpack8(vr[r], vf[r]);
-#pragma unroll
-                for (int hh = 0; hh < G; ++hh) {
-                    float mx = sv[hh];
-#pragma unroll
-                    for (int r = 1; r < ROWS; ++r) mx = fmaxf(mx, sv[r * G + hh]);
-                    const float m_new = fmaxf(m[hh], mx);
-                    if (m_new == -INFINITY) continue;   // nothing valid seen yet
-                    const float corr = exp2f(m[hh] - m_new);
-                    m[hh] = m_new;
-                    float p[ROWS], psum = 0.0f;
-#pragma unroll
-                    for (int r = 0; r < ROWS; ++r) {
-                        p[r] = exp2f(sv[r * G + hh] - m_new);
-                        psum += p[r];
-                    }
-                    l[hh] = fmaf(l[hh], corr, psum);
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        float a = acc[hh][e] * corr;
-#pragma unroll
-                        for (int r = 0; r < ROWS; ++r) a = fmaf(p[r], vf[r][e], a);
-                        acc[hh][e] = a;
-                    }
-                }
+            for (int ks = 0; ks < 8; ++ks) {
+                const uint32_t v0 = *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + quad * 2);
+                const uint32_t v2 = *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8 + quad * 2);
+                qa0[ks] = head < G ? v0 : 0u;
+                qa2[ks] = head < G ? v2 : 0u;
             }
         }
+        float m_run = -INFINITY, l_run = 0.0f;   // per lane: head `head`, partial over this lane's columns
+        float o[16][4];
+#pragma unroll
+        for (int n = 0; n < 16; ++n)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) o[n][i] = 0.0f;
 
-        // ---- merge the two half-warps of each warp, then the warps, into one partial per head ----
+        // pages of this warp: first_page + warp, + 8, ...
+        const int my_first = first_page + warp;
+        const int my_count = my_first < end_page ? (end_page - my_first + kDenseWarps - 1) / kDenseWarps : 0;
+        auto issue = [&](int k) {   // k-th page of this warp into stage k % kStages
+            const int pl = my_first + k * kDenseWarps;
+            long long phys = bt[pl];
+            const bool page_ok = phys >= 0 && phys < geo.pool_pages;
+            if (!page_ok) phys = 0;
+            const int valid_rows = page_ok ? min(kPageSize, T - pl * kPageSize) : 0;
+            const uint16_t* kp = k_cache + phys * geo.page_stride + (long long)g * geo.head_stride + cp_chunk * 8;
+            const uint16_t* vp = v_cache + phys * geo.page_stride + (long long)g * geo.head_stride + cp_chunk * 8;
+            const uint32_t dst = ring_addr + (uint32_t)((k % kStages) * kStageBytes);
 #pragma unroll
-        for (int hh = 0; hh < G; ++hh) {
-            const float m2 = __shfl_xor_sync(kFullMask, m[hh], 16);
-            const float l2 = __shfl_xor_sync(kFullMask, l[hh], 16);
-            const float M = fmaxf(m[hh], m2);
-            const float f1 = M == -INFINITY ? 0.0f : exp2f(m[hh] - M);
-            const float f2 = M == -INFINITY ? 0.0f : exp2f(m2 - M);
-            // lower half-warp first, so that both halves compute the same bits
-            const float la = gi == 0 ? l[hh] * f1 : l2 * f2;
-            const float lb = gi == 0 ? l2 * f2 : l[hh] * f1;
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                const float a2 = __shfl_xor_sync(kFullMask, acc[hh][e], 16);
-                const float xa = gi == 0 ? acc[hh][e] * f1 : a2 * f2;
-                const float xb = gi == 0 ? a2 * f2 : acc[hh][e] * f1;
-                acc[hh][e] = xa + xb;
+            for (int i = 0; i < 8; ++i) {
+                const int r = cp_row0 + 2 * i;
+                const uint32_t off = (uint32_t)(r * kRowBytes + ((cp_chunk ^ (r & 7)) << 4));
+                const bool ok = r < valid_rows;
+                cp_async_16_zfill(dst + off, kp + (long long)r * geo.token_stride, ok);
+                cp_async_16_zfill(dst + kTileBytes + off, vp + (long long)r * geo.token_stride, ok);
             }
-            if (gi == 0) {
+        };
 #pragma unroll
-                for (int e = 0; e < 8; ++e) sm_acc[warp][hh][c * 8 + e] = acc[hh][e];
-                if (c == 0) {
-                    sm_m[warp][hh] = M;
-                    sm_l[warp][hh] = la + lb;
+        for (int s = 0; s < kStages - 1; ++s) {
+            if (s < my_count) issue(s);
+            cp_async_commit();
+        }
+        for (int k = 0; k < my_count; ++k) {
+            if (k + kStages - 1 < my_count) issue(k + kStages - 1);
+            cp_async_commit();
+            cp_async_wait<kStages - 1>();
+            __syncwarp();
+            const int pl = my_first + k * kDenseWarps;
+            const int valid = min(kPageSize, T - pl * kPageSize);   // > 0
+            {
+                const long long phys = bt[pl];   // a page outside the pool contributes nothing
+                if (phys < 0 || phys >= geo.pool_pages) {
+                    __syncwarp();
+                    continue;
                 }
+            }
+            const uint32_t kbase = ring_addr + (uint32_t)((k % kStages) * kStageBytes);
+            const uint32_t vbase = kbase + kTileBytes;
+
+            // S = Q K^T for the 16 tokens of the page (two 8-token column tiles)
+            float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+            {
+                const int mi = lane >> 3, tok = (mi >> 1) * 8 + (lane & 7);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const int ch = 2 * ks + (mi & 1);
+                    uint32_t r[4];
+                    ldmatrix_x4(r, kbase + (uint32_t)(tok * kRowBytes + ((ch ^ (tok & 7)) << 4)));
+                    mma_bf16(s0, qa0[ks], qa2[ks], r[0], r[1]);
+                    mma_bf16(s1, qa0[ks], qa2[ks], r[2], r[3]);
+                }
+            }
+            // this lane: head `head`, tokens 2 quad, 2 quad + 1 (tile 0) and 8 + the same (tile 1)
+            float t[4];
+            t[0] = (2 * quad < valid) ? s0[0] * scale : -INFINITY;
+            t[1] = (2 * quad + 1 < valid) ? s0[1] * scale : -INFINITY;
+            t[2] = (8 + 2 * quad < valid) ? s1[0] * scale : -INFINITY;
+            t[3] = (8 + 2 * quad + 1 < valid) ? s1[1] * scale : -INFINITY;
+            float pm = fmaxf(fmaxf(t[0], t[1]), fmaxf(t[2], t[3]));
+            pm = fmaxf(pm, __shfl_xor_sync(kFullMask, pm, 1));
+            pm = fmaxf(pm, __shfl_xor_sync(kFullMask, pm, 2));
+            const float m_new = fmaxf(m_run, pm);       // finite: token 0 of a page is always valid
+            const float corr = exp2f(m_run - m_new);    // 0 on the first page
+            float p[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) p[i] = exp2f(t[i] - m_new);
+            l_run = fmaf(l_run, corr, (p[0] + p[1]) + (p[2] + p[3]));
+            if (__any_sync(kFullMask, m_new > m_run)) {
+#pragma unroll
+                for (int n = 0; n < 16; ++n) {
+                    o[n][0] *= corr;
+                    o[n][1] *= corr;
+                }
+            }
+            m_run = m_new;
+            const uint32_t pa0 = pack_bf16x2(p[0], p[1]), pa2 = pack_bf16x2(p[2], p[3]);
+
+            // O += P V
+            {
+                const int mi = lane >> 3, tok = (mi & 1) * 8 + (lane & 7);
+#pragma unroll
+                for (int dp = 0; dp < 8; ++dp) {
+                    const int ch = 2 * dp + (mi >> 1);
+                    uint32_t r[4];
+                    ldmatrix_x4_trans(r, vbase + (uint32_t)(tok * kRowBytes + ((ch ^ (tok & 7)) << 4)));
+                    mma_bf16(o[2 * dp], pa0, pa2, r[0], r[1]);
+                    mma_bf16(o[2 * dp + 1], pa0, pa2, r[2], r[3]);
+                }
+            }
+            __syncwarp();   // the stage is overwritten by a later issue
+        }
+        cp_async_wait<0>();
+
+        // ---- merge: quad lanes share a head (sum l), then the warps, into one partial per head ----
+        l_run += __shfl_xor_sync(kFullMask, l_run, 1);
+        l_run += __shfl_xor_sync(kFullMask, l_run, 2);
+        __syncthreads();   // every warp is done with its ring: reuse it for the merge
+        float* mg = reinterpret_cast<float*>(sm.ring);   // [warps][G][2 + 128]
+        if (head < G) {
+            float* rec = mg + (warp * G + head) * kPartialFloats;
+            if (quad == 0) {
+                rec[0] = m_run;
+                rec[1] = l_run;
+            }
+#pragma unroll
+            for (int n = 0; n < 16; ++n) {
+                rec[2 + n * 8 + quad * 2] = o[n][0];
+                rec[2 + n * 8 + quad * 2 + 1] = o[n][1];
             }
         }
         __syncthreads();
@@ -193,53 +348,57 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
             if (!((mask >> hh) & 1u)) continue;
             float M = -INFINITY;
 #pragma unroll
-            for (int w = 0; w < kDenseWarps; ++w) M = fmaxf(M, sm_m[w][hh]);
+            for (int w = 0; w < kDenseWarps; ++w) M = fmaxf(M, mg[(w * G + hh) * kPartialFloats]);
             float a = 0.0f, L = 0.0f;
 #pragma unroll
             for (int w = 0; w < kDenseWarps; ++w) {
-                const float f = sm_m[w][hh] == -INFINITY ? 0.0f : exp2f(sm_m[w][hh] - M);
-                a = fmaf(sm_acc[w][hh][e], f, a);
-                L = fmaf(sm_l[w][hh], f, L);
+                const float* rec = mg + (w * G + hh) * kPartialFloats;
+                const float f = rec[0] == -INFINITY ? 0.0f : exp2f(rec[0] - M);
+                a = fmaf(rec[2 + e], f, a);
+                L = fmaf(rec[1], f, L);
             }
-            const long long unit = (long long)b * geo.n_q_heads + g * G + hh;
-            float* rec = partials + (unit * n_splits + split) * kPartialFloats;
-            rec[2 + e] = a;
+            float* dst = partials + ((long long)item * G + hh) * kPartialFloats;
+            dst[2 + e] = a;
             if (e == 0) {
-                rec[0] = M;
-                rec[1] = L;
+                dst[0] = M;
+                dst[1] = L;
             }
         }
 
-        // ---- the block that finishes the last split of this (sequence, KV head) combines them ----
+        // ---- the block that finishes the last item of this (sequence, KV head) combines them ----
         __threadfence();
         __syncthreads();
-        if (tid == 0) {
-            const int ticket = atomicAdd(&counters[grp], 1);
-            sm_last = ticket == active_splits - 1;
-        }
+        if (tid == 0) sm.misc[12] = atomicAdd(&counters[grp], 1) == items_of_group - 1;
         __syncthreads();
-        if (sm_last) {
+        if (sm.misc[12]) {
             __threadfence();
+            const float* gp = partials + (long long)sm.item_base[grp] * G * kPartialFloats;
             for (int idx = tid; idx < G * kHeadDim; idx += kDenseThreads) {
                 const int hh = idx / kHeadDim, e = idx % kHeadDim;
                 if (!((mask >> hh) & 1u)) continue;
-                const long long unit = (long long)b * geo.n_q_heads + g * G + hh;
-                const float* rec0 = partials + unit * n_splits * kPartialFloats;
-                float M = -INFINITY;
-                for (int s = 0; s < active_splits; ++s) M = fmaxf(M, __ldcg(rec0 + s * kPartialFloats));
-                float a = 0.0f, L = 0.0f;
-                for (int s = 0; s < active_splits; ++s) {
-                    const float* rec = rec0 + s * kPartialFloats;
-                    const float ms = __ldcg(rec);
-                    const float f = ms == -INFINITY ? 0.0f : exp2f(ms - M);
-                    a = fmaf(__ldcg(rec + 2 + e), f, a);
-                    L = fmaf(__ldcg(rec + 1), f, L);
+                // one pass in item order, rescaling when a later item raises the maximum
+                float M = -INFINITY, a = 0.0f, L = 0.0f;
+#pragma unroll 4
+                for (int s = 0; s < items_of_group; ++s) {
+                    const float* rec = gp + ((long long)s * G + hh) * kPartialFloats;
+                    const float ms = __ldcg(rec), ls = __ldcg(rec + 1), as = __ldcg(rec + 2 + e);
+                    if (ms == -INFINITY) continue;
+                    if (ms > M) {
+                        const float r = exp2f(M - ms);   // 0 for the first contributing item
+                        a *= r;
+                        L *= r;
+                        M = ms;
+                    }
+                    const float f = exp2f(ms - M);
+                    a = fmaf(as, f, a);
+                    L = fmaf(ls, f, L);
                 }
-                out[unit * kHeadDim + e] = a / L;
+                const long long unit = (long long)b * geo.n_q_heads + g * G + hh;
+                out[unit * kHeadDim + e] = L > 0.0f ? a / L : 0.0f;
                 if (e == 0 && diag) diag[unit].lse = (M + log2f(L)) * 0.6931471805599453f;
             }
         }
-        __syncthreads();   // sm_* are reused by the next item
+        __syncthreads();   // the ring (merge buffer) and misc are reused by the next item
     }
 }
 
@@ -258,23 +417,16 @@ int num_sms()
     return g_num_sms;
 }
 
+// room for the items the kernel may create: one ragged item per group plus the balancing target
+int dense_max_items(const Geometry& g) { return g.batch * g.n_kv_heads + 2048; }
+
+size_t dense_smem_bytes(const Geometry& g)
+{
+    const size_t n_groups = (size_t)g.batch * g.n_kv_heads;
+    return kRingBytes + (n_groups + 1) * 4 + 16 * 4 + (n_groups + 15) / 16 * 16;
+}
+
 }  // namespace
-
-int dense_pages_per_split(const Geometry& g)
-{
-    // aim for a few thousand items when every unit is listed; a split is a multiple of 16 pages
-    const long long total_pages = (long long)g.batch * g.n_kv_heads * g.max_pages;
-    long long pps = (total_pages / 2048 + 15) / 16 * 16;
-    if (pps < 16) pps = 16;
-    if (pps > 256) pps = 256;
-    return (int)pps;
-}
-
-static int dense_n_splits(const Geometry& g)
-{
-    const int pps = dense_pages_per_split(g);
-    return (g.max_pages + pps - 1) / pps;
-}
 
 static size_t dense_counter_bytes(const Geometry& g)
 {
@@ -287,8 +439,29 @@ int dense_ticket_count(const Geometry& g) { return g.batch * g.n_kv_heads; }
 
 size_t dense_workspace_bytes(const Geometry& g)
 {
-    return dense_counter_bytes(g) +
-           (size_t)g.batch * g.n_q_heads * dense_n_splits(g) * kPartialFloats * sizeof(float);
+    return dense_counter_bytes(g) + (size_t)dense_max_items(g) * g.group * kPartialFloats * sizeof(float);
+}
+
+template <int G>
+static cudaError_t launch_dense_g(const Geometry& g, const uint16_t* q, const uint16_t* k, const uint16_t* v,
+                                  const int32_t* block_table, const int32_t* seq_lens, const int32_t* fallback_list,
+                                  const int32_t* fallback_count, float epsilon, float* partials, int32_t* counters,
+                                  float* out, vsa_diag_t* diag, cudaStream_t stream)
+{
+    const size_t smem = dense_smem_bytes(g);
+    static int attr_device = -1;   // per template instance: the device whose function attribute is set
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (attr_device != dev) {
+        e = cudaFuncSetAttribute(dense_split_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_device = dev;
+    }
+    // persistent grid: one block per SM (the ring fills the shared memory)
+    return launch_pdl(dense_split_kernel<G>, dim3((unsigned)num_sms()), dim3(kDenseThreads), smem, stream, g, q, k, v,
+                      block_table, seq_lens, fallback_list, fallback_count, epsilon, partials, counters, out, diag,
+                      dense_max_items(g));
 }
 
 cudaError_t launch_dense(const Geometry& g, const void* q, const void* k_cache, const void* v_cache,
@@ -298,39 +471,18 @@ cudaError_t launch_dense(const Geometry& g, const void* q, const void* k_cache, 
 {
     int32_t* counters = (int32_t*)ws;
     float* partials = (float*)((char*)ws + dense_counter_bytes(g));
-    cudaError_t e = cudaSuccess;
     if (!tickets_cleared) {
-        e = cudaMemsetAsync(counters, 0, dense_counter_bytes(g), stream);
+        cudaError_t e = cudaMemsetAsync(counters, 0, dense_counter_bytes(g), stream);
         if (e != cudaSuccess) return e;
     }
-    const int pps = dense_pages_per_split(g), ns = dense_n_splits(g);
-    const long long n_items = (long long)g.batch * g.n_kv_heads * ns;
-    const size_t mask_bytes = ((size_t)g.batch * g.n_kv_heads + 15) / 16 * 16;
     const uint16_t *qq = (const uint16_t*)q, *kk = (const uint16_t*)k_cache, *vv = (const uint16_t*)v_cache;
-    // persistent grid: exactly as many blocks as can be resident at once
-#define VSA_DENSE_LAUNCH(GG)                                                                                     \
-    {                                                                                                            \
-        int per_sm = 0;                                                                                          \
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dense_split_kernel<GG>, kDenseThreads,        \
-                                                          mask_bytes);                                           \
-        if (e != cudaSuccess) return e;                                                                          \
-        if (per_sm < 1) per_sm = 1;                                                                              \
-        long long blocks = (long long)num_sms() * per_sm;                                                        \
-        if (blocks > n_items) blocks = n_items;                                                                  \
-        e = launch_pdl(dense_split_kernel<GG>, dim3((unsigned)blocks), dim3(kDenseThreads), mask_bytes, stream, \
-                       g, qq, kk, vv, block_table, seq_lens, fallback_list, fallback_count, epsilon, partials,   \
-                       counters, out, diag, pps, ns);                                                            \
-        if (e != cudaSuccess) return e;                                                                          \
-    }
     switch (g.group) {
-        case 1: VSA_DENSE_LAUNCH(1); break;
-        case 2: VSA_DENSE_LAUNCH(2); break;
-        case 4: VSA_DENSE_LAUNCH(4); break;
-        case 8: VSA_DENSE_LAUNCH(8); break;
+        case 1: return launch_dense_g<1>(g, qq, kk, vv, block_table, seq_lens, fallback_list, fallback_count, epsilon, partials, counters, out, diag, stream);
+        case 2: return launch_dense_g<2>(g, qq, kk, vv, block_table, seq_lens, fallback_list, fallback_count, epsilon, partials, counters, out, diag, stream);
+        case 4: return launch_dense_g<4>(g, qq, kk, vv, block_table, seq_lens, fallback_list, fallback_count, epsilon, partials, counters, out, diag, stream);
+        case 8: return launch_dense_g<8>(g, qq, kk, vv, block_table, seq_lens, fallback_list, fallback_count, epsilon, partials, counters, out, diag, stream);
         default: return cudaErrorInvalidValue;
     }
-#undef VSA_DENSE_LAUNCH
-    return cudaGetLastError();
 }
 
 }  // namespace vsa

@@ -59,7 +59,6 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
                           vsa_diag_t* diag, int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream);
 
 // ---- dense split-K pass -------------------------------------------------------------------------
-int dense_pages_per_split(const Geometry& g);
 size_t dense_workspace_bytes(const Geometry& g);
 cudaError_t launch_dense(const Geometry& g, const void* q, const void* k_cache, const void* v_cache,
                          const int32_t* block_table, const int32_t* seq_lens, const int32_t* fallback_list,
