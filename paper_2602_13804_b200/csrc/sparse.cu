@@ -80,7 +80,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                      int32_t* __restrict__ fallback_count)
 {
     constexpr int WARPS = THREADS / 32, GROUPS = 2 * WARPS;
-    static_assert(TOK_KPT * WARPS <= 64 && 3 * WARPS <= 72, "wred capacity");
+    static_assert(TOK_KPT * WARPS <= 64 && 4 * WARPS <= 72, "wred capacity");
     extern __shared__ uint32_t smem_raw[];
     int32_t* page_l = (int32_t*)smem_raw;   // [P] routed logical pages, ascending, invalid entries last
     int32_t* page_phys = page_l + P;        // [P]
@@ -136,7 +136,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
             const int l = raw[t];
             int rank = 0;
 #pragma unroll 8
-            for (int j = 0; j < P; ++j) rank += (raw[j] < l) || (raw[j] == l && j < t);
+            for (int j = 0; j < P; ++j) rank += (int)((raw[j] < l) | ((raw[j] == l) & (j < t)));
             int phys = -1;
             if (l != INT_MAX) {
                 phys = bt[l];
@@ -199,11 +199,13 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     uint32_t key[TOK_KPT];
     int present = 0;
     uint32_t a1 = 0u, a2 = 0u;   // best and second-best key (multiset order statistics)
+    uint32_t amin = 0xffffffffu;  // smallest present key
 #pragma unroll
     for (int j = 0; j < TOK_KPT; ++j) {
         const int i = tid + j * THREADS;
         key[j] = i < N ? sm.keys[i] : 0u;
         present += key[j] != 0u;
+        if (key[j] != 0u) amin = min(amin, key[j]);
         if (key[j] > a1) {
             a2 = a1;
             a1 = key[j];
@@ -211,40 +213,47 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
             a2 = key[j];
         }
     }
-    // number of valid scored tokens, and the two best keys, block-wide
+    // number of valid scored tokens, the two best keys and the smallest key, block-wide
 #pragma unroll
     for (int off = 16; off; off >>= 1) {
         present += __shfl_xor_sync(kFullMask, present, off);
+        amin = min(amin, __shfl_xor_sync(kFullMask, amin, off));
         const uint32_t b1 = __shfl_xor_sync(kFullMask, a1, off), b2 = __shfl_xor_sync(kFullMask, a2, off);
         const uint32_t n1 = max(a1, b1), n2 = max(min(a1, b1), max(a2, b2));
         a1 = n1;
         a2 = n2;
     }
     if (lane == 0) {
-        sm.ts.wred[3 * warp] = a1;
-        sm.ts.wred[3 * warp + 1] = a2;
-        sm.ts.wred[3 * warp + 2] = (uint32_t)present;
+        sm.ts.wred[4 * warp] = a1;
+        sm.ts.wred[4 * warp + 1] = a2;
+        sm.ts.wred[4 * warp + 2] = (uint32_t)present;
+        sm.ts.wred[4 * warp + 3] = amin;
     }
+    // the selection below starts from a cleared histogram and list counter
+    for (int i = tid; i < 256; i += THREADS) sm.ts.hist[i] = 0u;
+    if (tid == 0) sm.ts.misc[4] = 0u;
     __syncthreads();
-    uint32_t key1 = 0u, key2 = 0u;
+    uint32_t key1 = 0u, key2 = 0u, kmin = 0xffffffffu;
     int n_valid = 0;
 #pragma unroll
     for (int w = 0; w < WARPS; ++w) {
-        const uint32_t b1 = sm.ts.wred[3 * w], b2 = sm.ts.wred[3 * w + 1];
+        const uint32_t b1 = sm.ts.wred[4 * w], b2 = sm.ts.wred[4 * w + 1];
         const uint32_t n1 = max(key1, b1), n2 = max(min(key1, b1), max(key2, b2));
         key1 = n1;
         key2 = n2;
-        n_valid += (int)sm.ts.wred[3 * w + 2];
+        n_valid += (int)sm.ts.wred[4 * w + 2];
+        kmin = min(kmin, sm.ts.wred[4 * w + 3]);
     }
     const int ns = min(K_c, n_valid);
-    __syncthreads();   // wred is reused by the selection
 
     VSA_PROBE(4);
     // ---- exact top-(ns+1): its last element is the best rejected token, the rest are the candidates ----
     uint32_t out_key = 0u, mask = 0u;
     const bool has_rejected = n_valid > ns;
     if (has_rejected) {
-        const TopkRegResult r = block_topk_reg<TOK_KPT>(key, N, ns + 1, sm.ts, sm.keys, sm.take);
+        // token scores are finite, so the smallest and largest keys are the range of the finite scores
+        const TopkRegResult r = block_topk_reg<TOK_KPT, true>(key, N, ns + 1, sm.ts, sm.keys, sm.take,
+                                                             key_to_float(kmin), key_to_float(key1));
         out_key = r.kth_key;
         mask = r.mask;
 #pragma unroll
@@ -254,6 +263,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
 #pragma unroll
         for (int j = 0; j < TOK_KPT; ++j)
             if (key[j] != 0u) mask |= 1u << j;
+        __syncthreads();   // wred is rewritten by the compaction
     }
 
     VSA_PROBE(5);
@@ -291,7 +301,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[e] = 0.0f;
     const int gidx = warp * 2 + gi;
-    constexpr int UNR = 8;
+    constexpr int UNR = THREADS == 256 ? 16 : 8;   // K_c = 256: every half-warp's rows in one batch
     for (int j0 = gidx; j0 < ns; j0 += GROUPS * UNR) {
         uint4 rows[UNR];
         float w[UNR];

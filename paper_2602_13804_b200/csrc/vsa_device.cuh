@@ -16,8 +16,13 @@ static __device__ long long vsa_probe_buf[64];
     do {                                                                               \
         if (blockIdx.x == VSA_PROBE_BLOCK && blockIdx.y == 0 && threadIdx.x == 0) vsa_probe_buf[i] = clock64(); \
     } while (0)
+#define VSA_PROBE_VAL(i, v)                                                            \
+    do {                                                                               \
+        if (blockIdx.x == VSA_PROBE_BLOCK && blockIdx.y == 0 && threadIdx.x == 0) vsa_probe_buf[i] = (long long)(v); \
+    } while (0)
 #else
 #define VSA_PROBE(i)
+#define VSA_PROBE_VAL(i, v)
 #endif
 
 namespace vsa {
@@ -388,7 +393,7 @@ __device__ __forceinline__ TopkResult block_topk_mark(const uint32_t* keys, int 
             for (int j = 0; j < m; ++j) {
                 const int ij = s.list[j];
                 const uint32_t kj = keys[ij];
-                rank += (kj > key) || (kj == key && ij < idx);
+                rank += (int)((kj > key) | ((kj == key) & (ij < idx)));
             }
             if (rank < need) take[idx] = 1;
             if (rank == need - 1) {
@@ -426,9 +431,13 @@ struct TopkRegResult {
     int kth_idx;
 };
 
-template <int KPT>
+// HAVE_RANGE: the caller already knows the smallest finite and the largest score of the block
+// (lo_in, hi_in) and has zeroed hist[0..256) and misc[4] before its last barrier, which saves the
+// range reduction and one barrier here.
+template <int KPT, bool HAVE_RANGE = false>
 __device__ __forceinline__ TopkRegResult block_topk_reg(const uint32_t (&key)[KPT], int n, int K,
-                                                        const TopkScratch& s, uint32_t* spill, uint8_t* spill_take)
+                                                        const TopkScratch& s, uint32_t* spill, uint8_t* spill_take,
+                                                        float lo_in = 0.0f, float hi_in = 0.0f)
 {
     static_assert(KPT <= 32, "one mask bit per owned element");
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
@@ -438,28 +447,33 @@ __device__ __forceinline__ TopkRegResult block_topk_reg(const uint32_t (&key)[KP
 #pragma unroll
     for (int j = 0; j < KPT; ++j) {
         f[j] = key_to_float(key[j]);
-        if (key[j] != 0u) {
+        if (!HAVE_RANGE && key[j] != 0u) {
             if (f[j] > -INFINITY) lo = fminf(lo, f[j]);
             hi = fmaxf(hi, f[j]);
         }
     }
+    if constexpr (HAVE_RANGE) {
+        lo = lo_in;
+        hi = hi_in;
+    } else {
 #pragma unroll
-    for (int off = 16; off; off >>= 1) {
-        lo = fminf(lo, __shfl_xor_sync(kFullMask, lo, off));
-        hi = fmaxf(hi, __shfl_xor_sync(kFullMask, hi, off));
-    }
-    if (lane == 0) {
-        s.wred[2 * warp] = __float_as_uint(lo);
-        s.wred[2 * warp + 1] = __float_as_uint(hi);
-    }
-    for (int i = tid; i < 256; i += stride) s.hist[i] = 0u;
-    if (tid == 0) s.misc[4] = 0u;   // list length
-    __syncthreads();
-    lo = INFINITY;
-    hi = -INFINITY;
-    for (int w = 0; w < nwarps; ++w) {
-        lo = fminf(lo, __uint_as_float(s.wred[2 * w]));
-        hi = fmaxf(hi, __uint_as_float(s.wred[2 * w + 1]));
+        for (int off = 16; off; off >>= 1) {
+            lo = fminf(lo, __shfl_xor_sync(kFullMask, lo, off));
+            hi = fmaxf(hi, __shfl_xor_sync(kFullMask, hi, off));
+        }
+        if (lane == 0) {
+            s.wred[2 * warp] = __float_as_uint(lo);
+            s.wred[2 * warp + 1] = __float_as_uint(hi);
+        }
+        for (int i = tid; i < 256; i += stride) s.hist[i] = 0u;
+        if (tid == 0) s.misc[4] = 0u;   // list length
+        __syncthreads();
+        lo = INFINITY;
+        hi = -INFINITY;
+        for (int w = 0; w < nwarps; ++w) {
+            lo = fminf(lo, __uint_as_float(s.wred[2 * w]));
+            hi = fmaxf(hi, __uint_as_float(s.wred[2 * w + 1]));
+        }
     }
     const float scale = 256.0f / (hi - lo);
     const bool fast = hi > lo && isfinite(scale) && isfinite(hi - lo);
@@ -472,7 +486,8 @@ __device__ __forceinline__ TopkRegResult block_topk_reg(const uint32_t (&key)[KP
             if (key[j] != 0u) atomicAdd(&s.hist[bucket[j]], 1u);
         }
         __syncthreads();
-        if (tid < 32) {
+        {
+            // every warp scans the histogram for itself (same data, same answer): no second barrier
             uint32_t c[8], mine = 0;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
@@ -486,23 +501,29 @@ __device__ __forceinline__ TopkRegResult block_topk_reg(const uint32_t (&key)[KP
                 if (lane + off < 32) incl += o;
             }
             uint32_t above = incl - mine;
+            int my_cut = -1, my_above = 0, my_count = 0;
             if (above < (uint32_t)K && (uint32_t)K <= incl) {
 #pragma unroll
                 for (int j = 7; j >= 0; --j) {
                     if (above < (uint32_t)K && (uint32_t)K <= above + c[j]) {
-                        s.misc[0] = (uint32_t)(lane * 8 + j);
-                        s.misc[1] = above;
-                        s.misc[2] = c[j];
+                        my_cut = lane * 8 + j;
+                        my_above = (int)above;
+                        my_count = (int)c[j];
                     }
                     above += c[j];
                 }
             }
+            const unsigned found = __ballot_sync(kFullMask, my_cut >= 0);
+            const int src = __ffs(found) - 1;   // exactly one lane owns the cut bucket
+            my_cut = __shfl_sync(kFullMask, my_cut, src);
+            my_above = __shfl_sync(kFullMask, my_above, src);
+            my_count = __shfl_sync(kFullMask, my_count, src);
+            if (my_count <= kTopkList) {
+                cut = my_cut;
+                need = K - my_above;
+            }
         }
-        __syncthreads();
-        if ((int)s.misc[2] <= kTopkList) {
-            cut = (int)s.misc[0];
-            need = K - (int)s.misc[1];
-        }
+        __syncthreads();   // all warps have read the histogram: its words are reused for the cut bucket's keys
     }
     TopkRegResult out;
     out.mask = 0u;
@@ -528,9 +549,11 @@ __device__ __forceinline__ TopkRegResult block_topk_reg(const uint32_t (&key)[KP
             const int idx = s.list[t];
             const uint32_t kt = s.hist[t];
             int rank = 0;
+#pragma unroll 8
             for (int u = 0; u < m; ++u) {
                 const uint32_t ku = s.hist[u];
-                rank += (ku > kt) || (ku == kt && s.list[u] < idx);
+                const int iu = s.list[u];
+                rank += (int)((ku > kt) | ((ku == kt) & (iu < idx)));
             }
             spill_take[idx] = rank < need ? 1 : 0;   // read back by the element's owner below
             if (rank == need - 1) {

@@ -54,7 +54,7 @@ __device__ __forceinline__ void order_winners(int K, const PageSelectSmem& s)
         for (int j = 0; j < K; ++j) {
             const uint32_t kj = s.tmp_key[j];
             const int ij = s.tmp_idx[j];
-            rank += (kj > key) || (kj == key && ij < idx);
+            rank += (int)((kj > key) | ((kj == key) & (ij < idx)));
             rank_asc += ij < idx;
         }
         s.win_key[rank] = key;
@@ -111,6 +111,73 @@ __device__ __forceinline__ int select_top_pages_reg(const float* __restrict__ sc
     if (tid == 0) s.ts.misc[8] = 0u;
     uint32_t mask = 0u;
     if (n > P) {
+        // Filter first: take each thread's best score; in every warp find the r-th largest of these
+        // (r = ceil(K / warps)); the smallest such value over the warps, theta, has at least K scores
+        // at or above it, so the top K are among the scores >= theta - typically only a few more than
+        // K of them - which are then ranked exactly against each other.
+        const int lane = tid & 31, warp = tid >> 5, nwarps = stride >> 5;
+        // only warps whose 32 threads all own a score take part (short sequences fill fewer warps)
+        const int nw_full = min(nwarps, n >> 5);
+        const int r = nw_full > 0 ? (K + nw_full - 1) / nw_full : 33;
+        VSA_PROBE(20);
+        uint32_t tmax = 0u;
+#pragma unroll
+        for (int j = 0; j < KPT; ++j) tmax = max(tmax, key[j]);
+        uint32_t v = tmax, thr = 0u;
+        for (int i = 0; i < r && r <= 32; ++i) {
+            thr = __reduce_max_sync(kFullMask, v);
+            const unsigned holders = __ballot_sync(kFullMask, v == thr);
+            if (lane == __ffs(holders) - 1) v = 0u;   // remove one holder of the maximum
+        }
+        if (lane == 0) s.ts.wred[warp] = thr;
+        if (tid == 0) s.ts.misc[4] = 0u;
+        __syncthreads();
+        uint32_t theta = 0xffffffffu;
+        for (int w = 0; w < nw_full; ++w) theta = min(theta, s.ts.wred[w]);
+        if (r > 32) theta = 0u;   // too few scores to filter: every score is a candidate
+#pragma unroll
+        for (int j = 0; j < KPT; ++j) {
+            if (key[j] != 0u && key[j] >= theta) {
+                const int slot = (int)atomicAdd(&s.ts.misc[4], 1u);
+                if (slot < kTopkList) {
+                    s.ts.list[slot] = tid + j * stride;
+                    s.ts.hist[slot] = key[j];
+                }
+            }
+        }
+        __syncthreads();
+        const int m = (int)s.ts.misc[4];
+        VSA_PROBE(21);
+        VSA_PROBE_VAL(40, m);
+        if (m <= kTopkList) {
+            for (int t = tid; t < m; t += stride) {
+                const int idx = s.ts.list[t];
+                const uint32_t kt = s.ts.hist[t];
+                int rank = 0;
+#pragma unroll 8
+                for (int u = 0; u < m; ++u) {
+                    const uint32_t ku = s.ts.hist[u];
+                    const int iu = s.ts.list[u];
+                    rank += (int)((ku > kt) | ((ku == kt) & (iu < idx)));
+                }
+                if (rank < K) {   // ranks are distinct: the K winners land best first
+                    s.win_key[rank] = kt;
+                    s.win_idx[rank] = idx;
+                }
+            }
+            __syncthreads();
+            for (int t = tid; t < K; t += stride) {
+                const int idx = s.win_idx[t];
+                int rank_asc = 0;
+#pragma unroll 8
+                for (int u = 0; u < K; ++u) rank_asc += s.win_idx[u] < idx;
+                s.asc_idx[rank_asc] = idx;
+            }
+            __syncthreads();
+            return K;
+        }
+        // crowded (many equal scores): the general selection decides
+        __syncthreads();
         mask = block_topk_reg<KPT>(key, n, K, s.ts, s.keys, s.take).mask;   // barriers inside order misc[8]
     } else {
 #pragma unroll
