@@ -303,21 +303,22 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     const int gidx = warp * 2 + gi;
     constexpr int UNR = THREADS == 256 ? 16 : 8;   // K_c = 256: every half-warp's rows in one batch
     for (int j0 = gidx; j0 < ns; j0 += GROUPS * UNR) {
-        uint4 rows[UNR];
+        // addresses and weights first (shared-memory lookups only), then all value rows at once;
+        // slots past the candidate count re-read the last candidate with weight 0
+        const uint16_t* ptr[UNR];
         float w[UNR];
 #pragma unroll
         for (int u = 0; u < UNR; ++u) {
             const int j = j0 + u * GROUPS;
-            rows[u] = make_uint4(0u, 0u, 0u, 0u);
-            w[u] = 0.0f;
-            if (j < ns) {
-                const int i = sm.sel[j];
-                const int slot = i >> 4, t = i & 15;
-                rows[u] = ld_nc_16B(v_cache + (long long)page_phys[slot] * geo.page_stride +
-                                    (long long)g * geo.head_stride + (long long)t * geo.token_stride + c * 8);
-                w[u] = exp2f((key_to_float(sm.keys[i]) - s1) * scale);
-            }
+            const int i = sm.sel[min(j, ns - 1)];
+            const int slot = i >> 4, t = i & 15;
+            ptr[u] = v_cache + (long long)page_phys[slot] * geo.page_stride + (long long)g * geo.head_stride +
+                     (long long)t * geo.token_stride + c * 8;
+            w[u] = j < ns ? exp2f((key_to_float(sm.keys[i]) - s1) * scale) : 0.0f;
         }
+        uint4 rows[UNR];
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) rows[u] = ld_nc_16B(ptr[u]);
 #pragma unroll
         for (int u = 0; u < UNR; ++u) {
             float vf[8];
