@@ -25,8 +25,9 @@ struct ScanCfg {
     static constexpr int VALS = ROWS * G;                 // (row, head) partials per lane per round (8 or 16)
     static constexpr int ROUND_PAGES = 2 * ROWS;          // pages (rows of one KV head) per warp per round
     static constexpr int ROUNDS = kBlockPages / ROUND_PAGES;
-    // rounds kept in flight per warp: about 8 KB of rows
-    static constexpr int STAGES = (8192 / (ROUND_PAGES * kRowBytes) < 2 ? 2 : 8192 / (ROUND_PAGES * kRowBytes)) + 1;
+    // ring slots per warp: a power of two (cheap slot index), about 8 KB of rows
+    static constexpr int STAGES = 8192 / (ROUND_PAGES * kRowBytes) < 2 ? 2 : 8192 / (ROUND_PAGES * kRowBytes);
+    static_assert((STAGES & (STAGES - 1)) == 0, "slot index is R & (STAGES - 1)");
     static constexpr int RING_BYTES = STAGES * ROUND_PAGES * kRowBytes;
     static constexpr int WARP_BYTES = RING_BYTES + kMaxBlocksPerWarp * kBlockPages * 4;
 };
@@ -121,7 +122,7 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
 
     // rows without a valid page read row 0 of the pool instead (their result is never stored)
     auto issue = [&](int R) {
-        const uint32_t dst = ring + (uint32_t)((R % STAGES) * ROUND_PAGES * kRowBytes) + lane_off;
+        const uint32_t dst = ring + (uint32_t)((R & (STAGES - 1)) * ROUND_PAGES * kRowBytes) + lane_off;
         const int* tab = phys_tab + R * ROUND_PAGES + gi * ROWS;
 #pragma unroll
         for (int r = 0; r < ROWS; ++r) cp_async_16(dst + r * kRowBytes, srow + max(tab[r], 0) * page_elems);
@@ -136,7 +137,7 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
         if (R + STAGES - 1 < n_rounds) issue(R + STAGES - 1);
         cp_async_commit();
         cp_async_wait<STAGES - 1>();   // this lane's copies of round R have landed
-        const uint8_t* src = my_smem + (R % STAGES) * ROUND_PAGES * kRowBytes + lane_off;
+        const uint8_t* src = my_smem + (R & (STAGES - 1)) * ROUND_PAGES * kRowBytes + lane_off;
         float vals[16];
 #pragma unroll
         for (int r = 0; r < ROWS; ++r) {
