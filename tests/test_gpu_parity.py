@@ -171,6 +171,29 @@ def test_host_buffer_step_matches_device_step():
     check_out(out_host.numpy(), st.out, "host step")
 
 
+def test_largest_routing_sizes():
+    # P = 128, K_c = 2048: eight token scores per thread, four page-list entries per lane
+    w = make_workload(spec(batch=3, n_q_heads=8, n_kv_heads=2, seq_lens=(40000, 5000, 2100), P=128, K_c=2048,
+                           needles=40), seed=212)
+    compare(w, run_gpu(w), dense_sample=8)
+    # more units than SMs with the same sizes: the 256-thread shape
+    w = make_workload(spec(batch=20, n_q_heads=8, n_kv_heads=1, seq_lens=(3000,) * 20, P=128, K_c=1500,
+                           needles=10), seed=213)
+    compare(w, run_gpu(w), dense_sample=8)
+
+
+def test_block_table_wider_than_the_register_select():
+    # 9000 pages per sequence: beyond 32 scores per thread at 256 threads, within it at 512;
+    # batch 40 x 4 heads = 160 units > SMs forces the 256-thread kernel and its shared-memory select
+    w = make_workload(spec(batch=40, n_q_heads=4, n_kv_heads=4, seq_lens=(144000,) + (600,) * 39, P=16, K_c=100,
+                           needles=5), seed=214)
+    compare(w, run_gpu(w), dense_sample=4)
+    # few units: 512 threads, 18 scores per thread rounded up to the 32-wide register select
+    w = make_workload(spec(batch=1, n_q_heads=4, n_kv_heads=2, seq_lens=(144000,), P=16, K_c=100, needles=5),
+                      seed=215)
+    compare(w, run_gpu(w), dense_sample=2)
+
+
 # ---------------------------------------------------------------- the named configurations
 
 def test_config0_full():
