@@ -230,9 +230,13 @@ def run_ours(args):
     distinct = max(1, min(L, int(0.8 * free // per_layer) + 1))
     layers = [w0] + [make_workload(spec, device=dev, rep=i, sub=rank) for i in range(1, distinct)]
     shape = B.shape_of(w0.q, w0.k_cache, w0.block_table)
-    for w in layers:   # one shape struct serves every layer: their caches must share the structure
+    # A paged KV cache has ONE block table and one length vector per sequence, used by every layer
+    # (the layers' K/V pools are separate tensors indexed by the same page numbers): all layers get
+    # layer 0's tensors.  The generator gives every layer the same structure, which is checked.
+    for w in layers:
         assert w.pool_pages == w0.pool_pages and torch.equal(w.block_table, w0.block_table) and \
             torch.equal(w.seq_lens, w0.seq_lens)
+        w.block_table, w.seq_lens = w0.block_table, w0.seq_lens
     units = shape.batch * shape.n_q_heads
     P, K_c, eps, tau = spec.P, spec.K_c, w0.epsilon, w0.gap_threshold
 

@@ -32,6 +32,7 @@ int make_geometry(const vsa_shape_t* s, Geometry* g)
     if (s->num_pool_pages > 0x7fffffffLL) return VSA_ERR_UNSUPPORTED_SHAPE;
     if ((long long)s->batch * s->n_q_heads > 0x3fffffffLL) return VSA_ERR_UNSUPPORTED_SHAPE;
     if ((long long)s->batch * s->n_kv_heads > 4096) return VSA_ERR_UNSUPPORTED_SHAPE;
+    if (s->num_pool_pages * s->n_kv_heads >= (1LL << 27)) return VSA_ERR_UNSUPPORTED_SHAPE;
     g->batch = s->batch;
     g->n_q_heads = s->n_q_heads;
     g->n_kv_heads = s->n_kv_heads;

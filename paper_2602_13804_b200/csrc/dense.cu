@@ -97,12 +97,15 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
     sm.item_base = (int32_t*)(dense_smem + kRingBytes);
     sm.misc = sm.item_base + n_groups + 1;
     sm.group_mask = (uint8_t*)(sm.misc + 16);
+    VSA_PROBE_T0(53);
     pdl_wait();
     pdl_launch_dependents();
+    VSA_PROBE_T0(54);
 
     // ---- which heads of which groups are listed? ----
     if (fallback_count) {
         const int count = *fallback_count;
+        VSA_PROBE_TMAX(55);
         if (count <= 0) return;
         for (int i = tid; i < n_groups; i += kDenseThreads) sm.group_mask[i] = 0;
         __syncthreads();
@@ -486,3 +489,10 @@ cudaError_t launch_dense(const Geometry& g, const void* q, const void* k_cache, 
 }
 
 }  // namespace vsa
+
+#ifdef VSA_ENABLE_PROBES
+extern "C" int vsa_probe_read_dense(long long* host64)
+{
+    return (int)cudaMemcpyFromSymbol(host64, vsa_probe_buf, sizeof(long long) * 64);
+}
+#endif

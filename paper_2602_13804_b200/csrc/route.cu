@@ -50,7 +50,9 @@ __device__ __forceinline__ void cp_async_wait()
 // with cp.async (several rounds in flight, no registers held by loads in flight, and no
 // cross-thread synchronisation: a lane only ever reads back what it copied itself).  A half-warp
 // covers one 256-byte row per copy instruction; the G query heads of the row's group share each
-// unpacked element; 16 (row, head) partials are reduced at once.
+// unpacked element; 16 (row, head) partials are reduced at once.  For G >= 2 lane c takes the
+// rows and the heads of a round in the order (r ^ c / G, h ^ c % G), which is what lets the
+// reduction run without per-lane selects (reduce_scatter16_xor).
 template <int G>
 __global__ void __launch_bounds__(kScanThreads, 2)
 route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* __restrict__ summaries,
@@ -60,9 +62,14 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
 {
     using Cfg = ScanCfg<G>;
     constexpr int ROWS = Cfg::ROWS, VALS = Cfg::VALS, ROUND_PAGES = Cfg::ROUND_PAGES, STAGES = Cfg::STAGES;
+    constexpr bool XOR_MAP = VALS == 16;
+    constexpr int kFirstBlocks = 4;   // block-table blocks fetched before the sequence length is known
     extern __shared__ __align__(16) uint8_t scan_smem[];
+    VSA_PROBE_T0(47);
     pdl_wait();                 // the score scratch may still be read by the previous step's kernels
     pdl_launch_dependents();
+    VSA_PROBE_T0(48);
+    VSA_PROBE(9);
 
     // housekeeping for the kernels that follow in a step: clear the fallback counter and the
     // per-group tickets of the dense pass
@@ -78,42 +85,59 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
     const int w = blockIdx.x * kScanWarps + warp;
     const int g = w % geo.n_kv_heads;
     const int slice = w / geo.n_kv_heads;
+    const int first_page = slice * blocks_per_warp * kBlockPages;
+    if (first_page >= geo.max_pages) return;
+    const int kr = XOR_MAP ? c / G : 0, kh = XOR_MAP ? c % G : 0;
+
+    // Three groups of loads that do not depend on one another go out back to back: the sequence
+    // length, the query rows, and the block-table entries of the first blocks of this warp's range
+    // (every index below max_pages is inside the table's row, whatever the sequence length is).
     const int T = seq_lens[b];
+    uint4 qraw[G];
+#pragma unroll
+    for (int hh = 0; hh < G; ++hh)
+        qraw[hh] = *reinterpret_cast<const uint4*>(
+            q + ((long long)b * geo.n_q_heads + g * G + (hh ^ kh)) * kHeadDim + c * 8);
+    const int32_t* bt = block_table + (long long)b * geo.max_pages + first_page;
+    const int span = min(blocks_per_warp * kBlockPages, geo.max_pages - first_page);
+    int first_entries[kFirstBlocks];
+#pragma unroll
+    for (int k = 0; k < kFirstBlocks; ++k) {
+        const int i = k * kBlockPages + lane;
+        first_entries[k] = i < span ? bt[i] : -1;
+    }
+
     if (T <= 0 || T > geo.max_pages * kPageSize) return;
     const int nb = (T + kPageSize - 1) / kPageSize;
-    const int first_page = slice * blocks_per_warp * kBlockPages;
     if (first_page >= nb) return;
     const int n_pages = min(blocks_per_warp * kBlockPages, nb - first_page);
     const int n_blocks = (n_pages + kBlockPages - 1) / kBlockPages;
     const int n_rounds = (n_pages + ROUND_PAGES - 1) / ROUND_PAGES;
 
     uint8_t* my_smem = scan_smem + warp * Cfg::WARP_BYTES;
-    int32_t* phys_tab = (int32_t*)(my_smem + Cfg::RING_BYTES);   // [n_blocks * 32], -1 = no valid page
+    // [n_blocks * 32] offset of the page's summary row in 16-byte units, -1 = no valid page
+    int32_t* off_tab = (int32_t*)(my_smem + Cfg::RING_BYTES);
     const uint32_t ring = (uint32_t)__cvta_generic_to_shared(my_smem);
-
-    // block-table entries of the whole page range of this warp (independent coalesced loads)
-    const int32_t* bt = block_table + (long long)b * geo.max_pages + first_page;
-    for (int k = 0; k < n_blocks; ++k) {
+    const int page_units = geo.n_kv_heads * (kRowBytes / 16);
+    auto encode = [&](int p, int i) { return (i < n_pages && p >= 0 && p < geo.pool_pages) ? p * page_units : -1; };
+#pragma unroll
+    for (int k = 0; k < kFirstBlocks; ++k)
+        if (k < n_blocks) off_tab[k * kBlockPages + lane] = encode(first_entries[k], k * kBlockPages + lane);
+    for (int k = kFirstBlocks; k < n_blocks; ++k) {
         const int i = k * kBlockPages + lane;
-        int p = -1;
-        if (i < n_pages) {
-            p = bt[i];
-            if (p < 0 || p >= geo.pool_pages) p = -1;
-        }
-        phys_tab[i] = p;
+        off_tab[i] = encode(i < n_pages ? bt[i] : -1, i);
     }
+    VSA_PROBE(10);
     float qf[G][8];
 #pragma unroll
-    for (int hh = 0; hh < G; ++hh) {
-        const uint4 v = *reinterpret_cast<const uint4*>(
-            q + ((long long)b * geo.n_q_heads + g * G + hh) * kHeadDim + c * 8);
-        unpack8(v, qf[hh]);
-    }
+    for (int hh = 0; hh < G; ++hh) unpack8(qraw[hh], qf[hh]);
     __syncwarp();
 
-    const uint16_t* srow = summaries + (long long)g * kHeadDim + c * 8;
-    const long long page_elems = (long long)geo.n_kv_heads * kHeadDim;
+    const uint8_t* srow = reinterpret_cast<const uint8_t*>(summaries) + (long long)g * kRowBytes + c * 16;
     const uint32_t lane_off = (uint32_t)(gi * ROWS * kRowBytes + c * 16);
+    int tab_row[ROWS];   // the table entry of this lane's r-th row of a round
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) tab_row[r] = gi * ROWS + (r ^ kr);
     // after the reduction this lane owns (row own_r, head own_h) of its half-warp's ROWS rows
     const int own_r = VALS == 16 ? c / G : (c & 7) / G, own_h = c % G;
     const bool owns = VALS == 16 || c < 8;
@@ -123,11 +147,13 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
     // rows without a valid page read row 0 of the pool instead (their result is never stored)
     auto issue = [&](int R) {
         const uint32_t dst = ring + (uint32_t)((R & (STAGES - 1)) * ROUND_PAGES * kRowBytes) + lane_off;
-        const int* tab = phys_tab + R * ROUND_PAGES + gi * ROWS;
+        const int* tab = off_tab + R * ROUND_PAGES;
 #pragma unroll
-        for (int r = 0; r < ROWS; ++r) cp_async_16(dst + r * kRowBytes, srow + max(tab[r], 0) * page_elems);
+        for (int r = 0; r < ROWS; ++r)
+            cp_async_16(dst + r * kRowBytes, srow + (long long)max(tab[tab_row[r]], 0) * 16);
     };
 
+    VSA_PROBE(11);
 #pragma unroll
     for (int s = 0; s < STAGES - 1; ++s) {
         if (s < n_rounds) issue(s);
@@ -137,6 +163,8 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
         if (R + STAGES - 1 < n_rounds) issue(R + STAGES - 1);
         cp_async_commit();
         cp_async_wait<STAGES - 1>();   // this lane's copies of round R have landed
+        if (R == 0) VSA_PROBE(12);
+        if (R == 1) VSA_PROBE(13);
         const uint8_t* src = my_smem + (R & (STAGES - 1)) * ROUND_PAGES * kRowBytes + lane_off;
         float vals[16];
 #pragma unroll
@@ -147,14 +175,19 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
 #pragma unroll
             for (int hh = 0; hh < G; ++hh) vals[r * G + hh] = chunk_partial(qf[hh], kf);
         }
-        if (VALS < 16) {
+        float s;
+        if constexpr (XOR_MAP) {
+            s = reduce_scatter16_xor(vals);
+        } else {
 #pragma unroll
             for (int i = VALS; i < 16; ++i) vals[i] = 0.0f;
+            s = reduce_scatter16(vals, c);
         }
-        const float s = reduce_scatter16(vals, c);
         const int pl = R * ROUND_PAGES + gi * ROWS + own_r;
-        if (owns && pl < n_pages) out_lane[R * ROUND_PAGES] = phys_tab[pl] >= 0 ? s : -INFINITY;
+        if (owns && pl < n_pages) out_lane[R * ROUND_PAGES] = off_tab[pl] >= 0 ? s : -INFINITY;
     }
+    VSA_PROBE(14);
+    VSA_PROBE_TMAX(49);
 }
 
 // Exact top-P of one unit's page scores, order (score descending, page ascending).
@@ -184,6 +217,17 @@ __global__ void route_select_kernel(Geometry geo, const float* __restrict__ scor
         if (routed_scores) routed_scores[unit * P + t] = t < K ? key_to_float(s.win_key[t]) : -INFINITY;
     }
 }
+
+#ifdef VSA_ENABLE_PROBES
+}  // namespace
+}  // namespace vsa
+extern "C" int vsa_probe_read_route(long long* host64)
+{
+    return (int)cudaMemcpyFromSymbol(host64, vsa_probe_buf, sizeof(long long) * 64);
+}
+namespace vsa {
+namespace {
+#endif
 
 size_t select_smem_bytes(const Geometry& g, int P) { return (size_t)select_pages_words(g.max_pages, P) * 4; }
 

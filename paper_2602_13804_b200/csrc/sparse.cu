@@ -20,14 +20,23 @@ constexpr int kMaxSparseWarps = 16;
 // token-phase shared memory, in 4-byte words, after the two page arrays
 __host__ __device__ constexpr int token_phase_words(int P, int K_c)
 {
-    return P * kPageSize /*keys*/ + (P * kPageSize + 3) / 4 /*take*/ + K_c /*sel*/ + 256 + 16 + 72 + kTopkList +
-           kMaxSparseWarps * kHeadDim + kMaxSparseWarps + 4;
+    return P * kPageSize /*keys*/ + (P * kPageSize + 3) / 4 /*take*/ + 2 * K_c + 2 /*voff*/ + K_c /*wgt*/ + 256 + 16 +
+           72 + kTopkList + kMaxSparseWarps * kHeadDim + kMaxSparseWarps + 4;
+}
+
+// first word of the block-table copy: after the two page arrays and the larger of the two phases
+__host__ __device__ inline int bt_stage_offset_words(int max_pages, int P, int K_c, bool fused)
+{
+    int words = token_phase_words(P, K_c);
+    if (fused && select_pages_words(max_pages, P) > words) words = select_pages_words(max_pages, P);
+    return 2 * P + words;
 }
 
 struct TokenSmem {
     uint32_t* keys;   // [P * 16] token score keys, array index = 16 * slot + token (position order)
     uint8_t* take;    // [P * 16] scratch of the selection's slow path
-    int32_t* sel;     // [K_c] array indices of the candidates, ascending
+    long long* voff;  // [K_c] element offset of each candidate's value row, candidates in position order
+    float* wgt;       // [K_c] unnormalised softmax weight of each candidate
     TopkScratch ts;
     float* red;       // [warps][128]
     float* zred;      // [warps]
@@ -39,8 +48,11 @@ __device__ __forceinline__ TokenSmem carve_tokens(uint32_t* base, int P, int K_c
     const int N = P * kPageSize;
     s.keys = base;
     s.take = (uint8_t*)(s.keys + N);
-    s.sel = (int32_t*)(s.keys + N + (N + 3) / 4);
-    s.ts.hist = (uint32_t*)(s.sel + K_c);
+    uint32_t* after_take = s.keys + N + (N + 3) / 4;
+    after_take += ((uintptr_t)after_take & 4u) ? 1 : 0;   // 8-byte alignment of the offsets
+    s.voff = (long long*)after_take;
+    s.wgt = (float*)(s.voff + K_c);
+    s.ts.hist = (uint32_t*)(s.wgt + K_c);
     s.ts.misc = s.ts.hist + 256;
     s.ts.wred = s.ts.misc + 16;
     s.ts.list = (int32_t*)(s.ts.wred + 72);
@@ -89,17 +101,39 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, c = lane & 15, gi = lane >> 4;
     const long long unit = blockIdx.x;
     const int b = (int)(unit / geo.n_q_heads), h = (int)(unit % geo.n_q_heads), g = h / geo.group;
+    VSA_PROBE_T0(50);
     pdl_wait();
     pdl_launch_dependents();
+    VSA_PROBE_T0(51);
+    // Loads that depend on nothing computed here go out back to back: the sequence length, this
+    // unit's page scores (every index below max_pages is inside the unit's scratch row, whatever
+    // the sequence length is), the query row, and a copy of the block-table row for the page
+    // lookups that follow the selection.
+    const int32_t* bt = block_table + (long long)b * geo.max_pages;
     const int T = seq_lens[b];
+    float praw[PAGE_KPT > 0 ? PAGE_KPT : 1];
+    if constexpr (PAGE_KPT > 0) {
+#pragma unroll
+        for (int j = 0; j < PAGE_KPT; ++j) {
+            const int i = tid + j * THREADS;
+            praw[j] = i < geo.max_pages ? ld_cg_f32(page_scores + unit * geo.max_pages + i) : 0.0f;
+        }
+    }
+    const uint4 qraw = ld_nc_16B(q + unit * kHeadDim + c * 8);
+    int32_t* bt_s = (int32_t*)(smem_raw + bt_stage_offset_words(geo.max_pages, P, K_c, PAGE_KPT > 0));
+    if constexpr (PAGE_KPT > 0) {
+        const uint32_t dst = (uint32_t)__cvta_generic_to_shared(bt_s);
+        for (int i = tid; i < geo.max_pages; i += THREADS) cp_async_4(dst + 4u * (uint32_t)i, bt + i);
+        cp_async_commit_group();
+    }
     if (T <= 0 || T > geo.max_pages * kPageSize) {
+        cp_async_wait_all();
         write_failed_unit(out, diag, unit, VSA_UNIT_BAD_LENGTH);
         if (PAGE_KPT != 0)
             for (int t = tid; t < P; t += THREADS) routed_pages[unit * P + t] = -1;
         return;
     }
     const int nb = (T + kPageSize - 1) / kPageSize;
-    const int32_t* bt = block_table + (long long)b * geo.max_pages;
     VSA_PROBE(0);
 
     // ---- routed pages -> page_l[] sorted by logical page, so that array order = position order ----
@@ -107,16 +141,21 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     int bad = 0;
     if constexpr (PAGE_KPT != 0) {
         const PageSelectSmem ps = carve_page_select(region, geo.max_pages, P);
-        if constexpr (PAGE_KPT > 0)
-            np = select_top_pages_reg<PAGE_KPT>(page_scores + unit * geo.max_pages, nb, P, ps);
-        else
+        if constexpr (PAGE_KPT > 0) {
+            uint32_t pkey[PAGE_KPT];
+#pragma unroll
+            for (int j = 0; j < PAGE_KPT; ++j) pkey[j] = tid + j * THREADS < nb ? float_to_key(praw[j]) : 0u;
+            cp_async_wait_all();   // this thread's part of the block-table copy; the selection's barriers publish it
+            np = select_top_pages_keys<PAGE_KPT>(pkey, nb, P, ps);
+        } else {
             np = select_top_pages(page_scores + unit * geo.max_pages, nb, P, ps);
+        }
         for (int t = tid; t < P; t += THREADS) {
             routed_pages[unit * P + t] = t < np ? ps.win_idx[t] : -1;
             int l = INT_MAX, phys = -1;
             if (t < np) {
                 l = ps.asc_idx[t];
-                phys = bt[l];
+                phys = PAGE_KPT > 0 ? bt_s[l] : bt[l];
                 if (phys < 0 || phys >= geo.pool_pages) {
                     phys = -1;
                     bad = 1;
@@ -165,10 +204,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     VSA_PROBE(2);
     // ---- token routing: score all 16 tokens of a page per half-warp ----
     float qf[8];
-    {
-        const uint4 v = *reinterpret_cast<const uint4*>(q + unit * kHeadDim + c * 8);
-        unpack8(v, qf);
-    }
+    unpack8(qraw, qf);
     for (int pp = warp; pp * 2 < np; pp += WARPS) {
         const int slot = pp * 2 + gi;
         const bool active = slot < np;
@@ -267,7 +303,10 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     }
 
     VSA_PROBE(5);
-    // ---- ordered compaction of the candidates: sel[] ascending in array (= position) order ----
+    // ---- ordered compaction of the candidates (position order); the thread that holds a candidate's
+    //      key writes the address of its value row and its softmax weight ----
+    const float s1 = ns > 0 ? key_to_float(key1) : -INFINITY;
+    const float scale = 1.4426950408889634f / epsilon;   // log2(e) / epsilon
     {
         int before[TOK_KPT];
 #pragma unroll
@@ -288,43 +327,40 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                 if (w < warp) mine += cw;
                 base += cw;
             }
-            if ((mask >> j) & 1u) sm.sel[mine + before[j]] = tid + j * THREADS;
+            if ((mask >> j) & 1u) {
+                const int i = tid + j * THREADS, pos = mine + before[j];
+                sm.voff[pos] = (long long)page_phys[i >> 4] * geo.page_stride + (long long)(i & 15) * geo.token_stride;
+                sm.wgt[pos] = exp2f((key_to_float(key[j]) - s1) * scale);
+            }
         }
     }
     __syncthreads();
 
     VSA_PROBE(6);
-    // ---- softmax weights and value gather ----
-    const float s1 = ns > 0 ? key_to_float(key1) : -INFINITY;
-    const float scale = 1.4426950408889634f / epsilon;   // log2(e) / epsilon
+    // ---- value gather ----
     float acc[8], z = 0.0f;
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[e] = 0.0f;
     const int gidx = warp * 2 + gi;
+    const uint16_t* vbase = v_cache + (long long)g * geo.head_stride + c * 8;
     constexpr int UNR = THREADS == 256 ? 16 : 8;   // K_c = 256: every half-warp's rows in one batch
     for (int j0 = gidx; j0 < ns; j0 += GROUPS * UNR) {
-        // addresses and weights first (shared-memory lookups only), then all value rows at once;
-        // slots past the candidate count re-read the last candidate with weight 0
-        const uint16_t* ptr[UNR];
+        // all value rows of the batch at once; slots past the candidate count re-read the last
+        // candidate with weight 0
+        uint4 rows[UNR];
         float w[UNR];
 #pragma unroll
         for (int u = 0; u < UNR; ++u) {
-            const int j = j0 + u * GROUPS;
-            const int i = sm.sel[min(j, ns - 1)];
-            const int slot = i >> 4, t = i & 15;
-            ptr[u] = v_cache + (long long)page_phys[slot] * geo.page_stride + (long long)g * geo.head_stride +
-                     (long long)t * geo.token_stride + c * 8;
-            w[u] = j < ns ? exp2f((key_to_float(sm.keys[i]) - s1) * scale) : 0.0f;
+            const int j = j0 + u * GROUPS, jc = min(j, ns - 1);
+            rows[u] = ld_nc_16B(vbase + sm.voff[jc]);
+            w[u] = j < ns ? sm.wgt[jc] : 0.0f;
         }
-        uint4 rows[UNR];
-#pragma unroll
-        for (int u = 0; u < UNR; ++u) rows[u] = ld_nc_16B(ptr[u]);
 #pragma unroll
         for (int u = 0; u < UNR; ++u) {
             float vf[8];
             unpack8(rows[u], vf);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] = fmaf(w[u], vf[e], acc[e]);
+            for (int e = 0; e < 8; e += 2) fma2(acc[e], acc[e + 1], w[u], w[u], vf[e], vf[e + 1]);
             z += w[u];
         }
     }
@@ -365,13 +401,15 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         diag[unit] = d;
         if (d.fallback) fallback_list[atomicAdd(fallback_count, 1)] = (int32_t)unit;
     }
+    VSA_PROBE_TMAX(52);
 }
 
-size_t sparse_smem_bytes(const Geometry& g, int P, int K_c, bool fused)
+size_t sparse_smem_bytes(const Geometry& g, int P, int K_c, bool fused, int threads)
 {
-    int words = token_phase_words(P, K_c);
-    if (fused && select_pages_words(g.max_pages, P) > words) words = select_pages_words(g.max_pages, P);
-    return (size_t)(2 * P + words) * 4 + 16;
+    size_t words = (size_t)bt_stage_offset_words(g.max_pages, P, K_c, fused);
+    // the register variants of the fused kernel (PAGE_KPT > 0) keep a copy of the block-table row
+    if (fused && g.max_pages <= 32 * threads) words += (size_t)g.max_pages;
+    return words * 4 + 16;
 }
 
 struct SparseArgs {
@@ -455,7 +493,9 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
 {
     SparseArgs a;
     a.g = g;
-    a.smem = sparse_smem_bytes(g, P, K_c, page_scores != nullptr);
+    // no more units than SMs: one larger block per unit (latency shape); otherwise two blocks per SM
+    const int threads = (long long)g.batch * g.n_q_heads <= sm_count() ? 512 : 256;
+    a.smem = sparse_smem_bytes(g, P, K_c, page_scores != nullptr, threads);
     a.q = (const uint16_t*)q;
     a.k = (const uint16_t*)k_cache;
     a.v = (const uint16_t*)v_cache;
@@ -472,9 +512,7 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
     a.fallback_list = fallback_list;
     a.fallback_count = fallback_count;
     a.stream = stream;
-    // no more units than SMs: one larger block per unit (latency shape); otherwise two blocks per SM
-    if ((long long)g.batch * g.n_q_heads <= sm_count()) return launch_threads<512>(a);
-    return launch_threads<256>(a);
+    return threads == 512 ? launch_threads<512>(a) : launch_threads<256>(a);
 }
 
 }  // namespace vsa

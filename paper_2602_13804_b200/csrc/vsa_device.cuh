@@ -20,9 +20,27 @@ static __device__ long long vsa_probe_buf[64];
     do {                                                                               \
         if (blockIdx.x == VSA_PROBE_BLOCK && blockIdx.y == 0 && threadIdx.x == 0) vsa_probe_buf[i] = (long long)(v); \
     } while (0)
+// wall-clock (globaltimer, ns) timeline of a step: block 0's time at a point, and the latest time
+// any block passed a point
+__device__ __forceinline__ long long vsa_probe_ns()
+{
+    long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+#define VSA_PROBE_T0(i)                                                                \
+    do {                                                                               \
+        if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) vsa_probe_buf[i] = vsa_probe_ns(); \
+    } while (0)
+#define VSA_PROBE_TMAX(i)                                                              \
+    do {                                                                               \
+        if (threadIdx.x == 0) atomicMax((unsigned long long*)&vsa_probe_buf[i], (unsigned long long)vsa_probe_ns()); \
+    } while (0)
 #else
 #define VSA_PROBE(i)
 #define VSA_PROBE_VAL(i, v)
+#define VSA_PROBE_T0(i)
+#define VSA_PROBE_TMAX(i)
 #endif
 
 namespace vsa {
@@ -73,6 +91,23 @@ __device__ __forceinline__ uint4 ld_nc_16B(const void* p)
     return v;
 }
 
+// global load that the compiler keeps where it is written (used to issue independent loads
+// ahead of the first branch that needs any of them)
+__device__ __forceinline__ float ld_cg_f32(const float* p)
+{
+    float v;
+    asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p));
+    return v;
+}
+
+// 4-byte asynchronous copies into shared memory (sources with no 16-byte alignment guarantee)
+__device__ __forceinline__ void cp_async_4(uint32_t smem_addr, const void* gptr)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_addr), "l"(gptr) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit_group() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
 // ---- the fixed-order dot product ---------------------------------------------------------
 // A row of 128 elements is spread over 16 lanes, lane c holding elements 8c .. 8c+7.
 // chunk_partial() sums the lane's 8 products as two interleaved chains,
@@ -104,6 +139,21 @@ __device__ __forceinline__ float chunk_partial(const float (&x)[8], const float 
     fma2(even, odd, x[4], x[5], y[4], y[5]);
     fma2(even, odd, x[6], x[7], y[6], y[7]);
     return even + odd;
+}
+
+// The same tree without any per-lane selection: on entry slot i of lane c holds this lane's partial
+// of value (i ^ c) - the caller arranges that through which data each lane loads - so that at
+// every level the slot a lane sends and the slot it adds into are fixed.  On return lane c holds
+// the complete sum of value c.  Per value the additions are again p[c] += p[c+off], off = 8, 4, 2, 1.
+__device__ __forceinline__ float reduce_scatter16_xor(float (&v)[16])
+{
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] += __shfl_xor_sync(kFullMask, v[i + 8], 8);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) v[i] += __shfl_xor_sync(kFullMask, v[i + 4], 4);
+#pragma unroll
+    for (int i = 0; i < 2; ++i) v[i] += __shfl_xor_sync(kFullMask, v[i + 2], 2);
+    return v[0] + __shfl_xor_sync(kFullMask, v[1], 1);
 }
 
 // Halving tree over the 16 lanes of a half-warp for 16 independent values at once

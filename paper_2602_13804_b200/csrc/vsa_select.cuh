@@ -95,19 +95,14 @@ __device__ __forceinline__ int select_top_pages(const float* __restrict__ sc, in
     return K;
 }
 
-// The same with each thread holding its KPT scores in registers (n <= KPT * blockDim.x).
+// The same with each thread holding its KPT scores in registers (n <= KPT * blockDim.x):
+// key[j] is the key of score tid + j * blockDim.x, 0 for indices at or beyond n.
 template <int KPT>
-__device__ __forceinline__ int select_top_pages_reg(const float* __restrict__ sc, int n, int P,
-                                                    const PageSelectSmem& s)
+__device__ __forceinline__ int select_top_pages_keys(const uint32_t (&key)[KPT], int n, int P,
+                                                     const PageSelectSmem& s)
 {
     const int K = min(P, n);
     const int tid = threadIdx.x, stride = blockDim.x;
-    uint32_t key[KPT];
-#pragma unroll
-    for (int j = 0; j < KPT; ++j) {
-        const int i = tid + j * stride;
-        key[j] = i < n ? float_to_key(__ldcg(sc + i)) : 0u;
-    }
     if (tid == 0) s.ts.misc[8] = 0u;
     uint32_t mask = 0u;
     if (n > P) {
@@ -196,6 +191,20 @@ __device__ __forceinline__ int select_top_pages_reg(const float* __restrict__ sc
     __syncthreads();
     order_winners(K, s);
     return K;
+}
+
+// The register variant fed from the scores in global memory.
+template <int KPT>
+__device__ __forceinline__ int select_top_pages_reg(const float* __restrict__ sc, int n, int P,
+                                                    const PageSelectSmem& s)
+{
+    uint32_t key[KPT];
+#pragma unroll
+    for (int j = 0; j < KPT; ++j) {
+        const int i = threadIdx.x + j * blockDim.x;
+        key[j] = i < n ? float_to_key(__ldcg(sc + i)) : 0u;
+    }
+    return select_top_pages_keys<KPT>(key, n, P, s);
 }
 
 }  // namespace vsa
