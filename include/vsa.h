@@ -17,6 +17,12 @@
  *     any of them.  All buffers are owned by the caller.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls
  *     only enqueue work on that stream and return; they never synchronise.
+ *   - Kernels are launched with programmatic stream serialisation: a kernel may become
+ *     resident while its predecessor on the stream is still running and then reads
+ *     `block_table`, `seq_lens` and (second kernel of a step onwards) `q` before it waits for
+ *     that predecessor.  Consequently the KERNEL that immediately precedes a call on the
+ *     stream must not be the one that writes `block_table` or `seq_lens` (copies, and
+ *     anything enqueued earlier than that kernel, are complete and visible first).
  *   - Return value: 0 on success, a negative VSA_ERR_* code otherwise.  Errors are detected
  *     on the host before anything is launched, so a failed call leaves all buffers untouched.
  *   - Data-dependent anomalies (a block-table entry outside the pool, a sequence longer

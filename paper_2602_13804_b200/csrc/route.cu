@@ -66,6 +66,32 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
     constexpr int kFirstBlocks = 4;   // block-table blocks fetched before the sequence length is known
     extern __shared__ __align__(16) uint8_t scan_smem[];
     VSA_PROBE_T0(47);
+    const int b = blockIdx.y;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, c = lane & 15, gi = lane >> 4;
+    const int w = blockIdx.x * kScanWarps + warp;
+    const int g = w % geo.n_kv_heads;
+    const int slice = w / geo.n_kv_heads;
+    const int first_page = slice * blocks_per_warp * kBlockPages;
+    const bool has_range = first_page < geo.max_pages;
+    const int kr = XOR_MAP ? c / G : 0, kh = XOR_MAP ? c % G : 0;
+
+    // The sequence length and the block-table entries of the first blocks of this warp's range are
+    // fetched before the wait on the preceding kernel (they are scheduler state, not the product of a
+    // kernel that signals early completion) so that their latency overlaps that kernel's tail.
+    // Every index below max_pages is inside the table's row, whatever the sequence length is.
+    const int32_t* bt = block_table + (long long)b * geo.max_pages + first_page;
+    const int span = min(blocks_per_warp * kBlockPages, geo.max_pages - first_page);
+    int T = 0;
+    int first_entries[kFirstBlocks];
+    if (has_range) {
+        T = ld_ca_s32(seq_lens + b);
+#pragma unroll
+        for (int k = 0; k < kFirstBlocks; ++k) {
+            const int i = k * kBlockPages + lane;
+            first_entries[k] = i < span ? ld_ca_s32(bt + i) : -1;
+        }
+    }
+
     pdl_wait();                 // the score scratch may still be read by the previous step's kernels
     pdl_launch_dependents();
     VSA_PROBE_T0(48);
@@ -79,33 +105,12 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
             for (int i = blockIdx.x * kScanThreads + threadIdx.x; i < zero_count; i += gridDim.x * kScanThreads)
                 zero_words[i] = 0;
     }
+    if (!has_range) return;
 
-    const int b = blockIdx.y;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, c = lane & 15, gi = lane >> 4;
-    const int w = blockIdx.x * kScanWarps + warp;
-    const int g = w % geo.n_kv_heads;
-    const int slice = w / geo.n_kv_heads;
-    const int first_page = slice * blocks_per_warp * kBlockPages;
-    if (first_page >= geo.max_pages) return;
-    const int kr = XOR_MAP ? c / G : 0, kh = XOR_MAP ? c % G : 0;
-
-    // Three groups of loads that do not depend on one another go out back to back: the sequence
-    // length, the query rows, and the block-table entries of the first blocks of this warp's range
-    // (every index below max_pages is inside the table's row, whatever the sequence length is).
-    const int T = seq_lens[b];
     uint4 qraw[G];
 #pragma unroll
     for (int hh = 0; hh < G; ++hh)
-        qraw[hh] = *reinterpret_cast<const uint4*>(
-            q + ((long long)b * geo.n_q_heads + g * G + (hh ^ kh)) * kHeadDim + c * 8);
-    const int32_t* bt = block_table + (long long)b * geo.max_pages + first_page;
-    const int span = min(blocks_per_warp * kBlockPages, geo.max_pages - first_page);
-    int first_entries[kFirstBlocks];
-#pragma unroll
-    for (int k = 0; k < kFirstBlocks; ++k) {
-        const int i = k * kBlockPages + lane;
-        first_entries[k] = i < span ? bt[i] : -1;
-    }
+        qraw[hh] = ld_nc_16B(q + ((long long)b * geo.n_q_heads + g * G + (hh ^ kh)) * kHeadDim + c * 8);
 
     if (T <= 0 || T > geo.max_pages * kPageSize) return;
     const int nb = (T + kPageSize - 1) / kPageSize;

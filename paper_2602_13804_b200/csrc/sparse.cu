@@ -102,15 +102,23 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     const long long unit = blockIdx.x;
     const int b = (int)(unit / geo.n_q_heads), h = (int)(unit % geo.n_q_heads), g = h / geo.group;
     VSA_PROBE_T0(50);
+    // Loads that depend on nothing computed in this step go out before the wait on the preceding
+    // kernel: the sequence length, the query row (the routing kernel that precedes this one in a step
+    // has read it already) and a copy of the block-table row for the page lookups that follow the
+    // selection.  The page scores, which that kernel writes, are fetched right after the wait; every
+    // index below max_pages is inside the unit's scratch row, whatever the sequence length is.
+    const int32_t* bt = block_table + (long long)b * geo.max_pages;
+    const int T = ld_ca_s32(seq_lens + b);
+    const uint4 qraw = ld_nc_16B(q + unit * kHeadDim + c * 8);
+    int32_t* bt_s = (int32_t*)(smem_raw + bt_stage_offset_words(geo.max_pages, P, K_c, PAGE_KPT > 0));
+    if constexpr (PAGE_KPT > 0) {
+        const uint32_t dst = (uint32_t)__cvta_generic_to_shared(bt_s);
+        for (int i = tid; i < geo.max_pages; i += THREADS) cp_async_4(dst + 4u * (uint32_t)i, bt + i);
+        cp_async_commit_group();
+    }
     pdl_wait();
     pdl_launch_dependents();
     VSA_PROBE_T0(51);
-    // Loads that depend on nothing computed here go out back to back: the sequence length, this
-    // unit's page scores (every index below max_pages is inside the unit's scratch row, whatever
-    // the sequence length is), the query row, and a copy of the block-table row for the page
-    // lookups that follow the selection.
-    const int32_t* bt = block_table + (long long)b * geo.max_pages;
-    const int T = seq_lens[b];
     float praw[PAGE_KPT > 0 ? PAGE_KPT : 1];
     if constexpr (PAGE_KPT > 0) {
 #pragma unroll
@@ -118,13 +126,6 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
             const int i = tid + j * THREADS;
             praw[j] = i < geo.max_pages ? ld_cg_f32(page_scores + unit * geo.max_pages + i) : 0.0f;
         }
-    }
-    const uint4 qraw = ld_nc_16B(q + unit * kHeadDim + c * 8);
-    int32_t* bt_s = (int32_t*)(smem_raw + bt_stage_offset_words(geo.max_pages, P, K_c, PAGE_KPT > 0));
-    if constexpr (PAGE_KPT > 0) {
-        const uint32_t dst = (uint32_t)__cvta_generic_to_shared(bt_s);
-        for (int i = tid; i < geo.max_pages; i += THREADS) cp_async_4(dst + 4u * (uint32_t)i, bt + i);
-        cp_async_commit_group();
     }
     if (T <= 0 || T > geo.max_pages * kPageSize) {
         cp_async_wait_all();
@@ -249,15 +250,18 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
             a2 = key[j];
         }
     }
-    // number of valid scored tokens, the two best keys and the smallest key, block-wide
-#pragma unroll
-    for (int off = 16; off; off >>= 1) {
-        present += __shfl_xor_sync(kFullMask, present, off);
-        amin = min(amin, __shfl_xor_sync(kFullMask, amin, off));
-        const uint32_t b1 = __shfl_xor_sync(kFullMask, a1, off), b2 = __shfl_xor_sync(kFullMask, a2, off);
-        const uint32_t n1 = max(a1, b1), n2 = max(min(a1, b1), max(a2, b2));
-        a1 = n1;
-        a2 = n2;
+    // number of valid scored tokens, the two best keys and the smallest key: per warp with the
+    // single-instruction warp reductions, then across the warps through shared memory.  Each warp
+    // also publishes its best key: the smallest of those (hi_r) and the largest of the warps' smallest
+    // keys (lo_r) bracket the bulk of the scores and serve as the histogram range of the selection.
+    {
+        present = __reduce_add_sync(kFullMask, present);
+        amin = __reduce_min_sync(kFullMask, amin);
+        const uint32_t wmax = __reduce_max_sync(kFullMask, a1);
+        const int holder = __ffs(__ballot_sync(kFullMask, a1 == wmax)) - 1;
+        const uint32_t wsecond = __reduce_max_sync(kFullMask, lane == holder ? a2 : a1);
+        a1 = wmax;
+        a2 = wsecond;
     }
     if (lane == 0) {
         sm.ts.wred[4 * warp] = a1;
@@ -269,16 +273,18 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     for (int i = tid; i < 256; i += THREADS) sm.ts.hist[i] = 0u;
     if (tid == 0) sm.ts.misc[4] = 0u;
     __syncthreads();
-    uint32_t key1 = 0u, key2 = 0u, kmin = 0xffffffffu;
+    uint32_t key1 = 0u, key2 = 0u, kmin = 0xffffffffu, hi_r = 0xffffffffu, lo_r = 0u;
     int n_valid = 0;
 #pragma unroll
     for (int w = 0; w < WARPS; ++w) {
-        const uint32_t b1 = sm.ts.wred[4 * w], b2 = sm.ts.wred[4 * w + 1];
+        const uint32_t b1 = sm.ts.wred[4 * w], b2 = sm.ts.wred[4 * w + 1], bmin = sm.ts.wred[4 * w + 3];
         const uint32_t n1 = max(key1, b1), n2 = max(min(key1, b1), max(key2, b2));
         key1 = n1;
         key2 = n2;
         n_valid += (int)sm.ts.wred[4 * w + 2];
-        kmin = min(kmin, sm.ts.wred[4 * w + 3]);
+        kmin = min(kmin, bmin);
+        if (b1 != 0u) hi_r = min(hi_r, b1);                 // warps without a valid token do not count
+        if (bmin != 0xffffffffu) lo_r = max(lo_r, bmin);
     }
     const int ns = min(K_c, n_valid);
 
@@ -288,7 +294,9 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     const bool has_rejected = n_valid > ns;
     if (has_rejected) {
         // token scores are finite, so the smallest and largest keys are the range of the finite scores
+        // (when the bracket is empty or inverted the selection falls back to the full range itself)
         const TopkRegResult r = block_topk_reg<TOK_KPT, true>(key, N, ns + 1, sm.ts, sm.keys, sm.take,
+                                                             key_to_float(lo_r), key_to_float(hi_r),
                                                              key_to_float(kmin), key_to_float(key1));
         out_key = r.kth_key;
         mask = r.mask;

@@ -100,6 +100,13 @@ __device__ __forceinline__ float ld_cg_f32(const float* p)
     return v;
 }
 
+__device__ __forceinline__ int ld_ca_s32(const int32_t* p)
+{
+    int v;
+    asm volatile("ld.global.ca.s32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+
 // 4-byte asynchronous copies into shared memory (sources with no 16-byte alignment guarantee)
 __device__ __forceinline__ void cp_async_4(uint32_t smem_addr, const void* gptr)
 {
@@ -468,6 +475,25 @@ __device__ __forceinline__ TopkResult block_topk_mark(const uint32_t* keys, int 
     return out;
 }
 
+// Block-wide list append without one atomic per entry: every thread of a (converged) warp passes
+// the number of entries it wants to add and gets the first of its consecutive slots; the warp
+// takes its range with a single atomic on `counter`.
+__device__ __forceinline__ int warp_append_slots(int cnt, uint32_t* counter)
+{
+    const int lane = threadIdx.x & 31;
+    int incl = cnt;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int o = __shfl_up_sync(kFullMask, incl, off);
+        if (lane >= off) incl += o;
+    }
+    const int total = __shfl_sync(kFullMask, incl, 31);
+    int base = 0;
+    if (lane == 31 && total > 0) base = (int)atomicAdd(counter, (uint32_t)total);
+    base = __shfl_sync(kFullMask, base, 31);
+    return base + incl - cnt;
+}
+
 // ---- the same selection with the keys held in registers -------------------------------------------
 // Thread t owns elements t, t + blockDim, ..., t + (KPT-1) * blockDim (key[j] = 0 where the element is
 // absent or past n).  On return bit j of the result's `mask` is set iff element t + j * blockDim is
@@ -481,13 +507,16 @@ struct TopkRegResult {
     int kth_idx;
 };
 
-// HAVE_RANGE: the caller already knows the smallest finite and the largest score of the block
-// (lo_in, hi_in) and has zeroed hist[0..256) and misc[4] before its last barrier, which saves the
-// range reduction and one barrier here.
+// HAVE_RANGE: the caller supplies the histogram range and has zeroed hist[0..256) and misc[4] before
+// its last barrier, which saves the range reduction and one barrier here.  (lo_in, hi_in) may be any
+// bracket of the bulk of the scores - scores outside it fall into the first or the last bucket, which
+// keeps the buckets fine where the cut is when a few outliers stretch the full range - and
+// (lo_full, hi_full), the smallest finite and the largest score, is used when that bracket is empty.
 template <int KPT, bool HAVE_RANGE = false>
 __device__ __forceinline__ TopkRegResult block_topk_reg(const uint32_t (&key)[KPT], int n, int K,
                                                         const TopkScratch& s, uint32_t* spill, uint8_t* spill_take,
-                                                        float lo_in = 0.0f, float hi_in = 0.0f)
+                                                        float lo_in = 0.0f, float hi_in = 0.0f, float lo_full = 0.0f,
+                                                        float hi_full = 0.0f)
 {
     static_assert(KPT <= 32, "one mask bit per owned element");
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
@@ -503,8 +532,9 @@ __device__ __forceinline__ TopkRegResult block_topk_reg(const uint32_t (&key)[KP
         }
     }
     if constexpr (HAVE_RANGE) {
-        lo = lo_in;
-        hi = hi_in;
+        const bool bracket = hi_in > lo_in;
+        lo = bracket ? lo_in : lo_full;
+        hi = bracket ? hi_in : hi_full;
     } else {
 #pragma unroll
         for (int off = 16; off; off >>= 1) {
@@ -525,6 +555,7 @@ __device__ __forceinline__ TopkRegResult block_topk_reg(const uint32_t (&key)[KP
             hi = fmaxf(hi, __uint_as_float(s.wred[2 * w + 1]));
         }
     }
+    if (HAVE_RANGE) VSA_PROBE(22);
     const float scale = 256.0f / (hi - lo);
     const bool fast = hi > lo && isfinite(scale) && isfinite(hi - lo);
     int cut = -1, need = K;
@@ -532,12 +563,14 @@ __device__ __forceinline__ TopkRegResult block_topk_reg(const uint32_t (&key)[KP
     if (fast) {
 #pragma unroll
         for (int j = 0; j < KPT; ++j) {
-            bucket[j] = f[j] > -INFINITY ? min(255, (int)((f[j] - lo) * scale)) : 0;
+            bucket[j] = f[j] > -INFINITY ? (int)fminf(fmaxf((f[j] - lo) * scale, 0.0f), 255.0f) : 0;
             if (key[j] != 0u) atomicAdd(&s.hist[bucket[j]], 1u);
         }
+        if (HAVE_RANGE) VSA_PROBE(23);
         __syncthreads();
-        {
-            // every warp scans the histogram for itself (same data, same answer): no second barrier
+        if (HAVE_RANGE) VSA_PROBE(24);
+        if (warp == 0) {
+            // one warp scans the histogram and publishes the cut through the barrier that follows
             uint32_t c[8], mine = 0;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
@@ -568,12 +601,17 @@ __device__ __forceinline__ TopkRegResult block_topk_reg(const uint32_t (&key)[KP
             my_cut = __shfl_sync(kFullMask, my_cut, src);
             my_above = __shfl_sync(kFullMask, my_above, src);
             my_count = __shfl_sync(kFullMask, my_count, src);
-            if (my_count <= kTopkList) {
-                cut = my_cut;
-                need = K - my_above;
+            if (lane == 0) {
+                s.misc[9] = my_count <= kTopkList ? (uint32_t)my_cut : 0xffffffffu;
+                s.misc[10] = (uint32_t)(K - my_above);
             }
         }
-        __syncthreads();   // all warps have read the histogram: its words are reused for the cut bucket's keys
+        if (HAVE_RANGE) VSA_PROBE(25);
+        __syncthreads();   // the histogram has been read: its words are reused for the cut bucket's keys
+        if (s.misc[9] != 0xffffffffu) {
+            cut = (int)s.misc[9];
+            need = (int)s.misc[10];
+        }
     }
     TopkRegResult out;
     out.mask = 0u;
@@ -584,17 +622,25 @@ __device__ __forceinline__ TopkRegResult block_topk_reg(const uint32_t (&key)[KP
         for (int j = 0; j < KPT; ++j) {
             if (key[j] != 0u) {
                 if (bucket[j] > cut) out.mask |= 1u << j;
-                if (bucket[j] == cut) {
-                    // the histogram is dead (warp 0 read it before the last barrier): reuse it for the keys
-                    const int slot = (int)atomicAdd(&s.misc[4], 1u);
+                if (bucket[j] == cut) in_cut |= 1u << j;
+            }
+        }
+        {
+            // the histogram is dead (read before the last barrier): its words take the listed keys
+            int slot = warp_append_slots(__popc(in_cut), &s.misc[4]);
+#pragma unroll
+            for (int j = 0; j < KPT; ++j) {
+                if ((in_cut >> j) & 1u) {
                     s.list[slot] = tid + j * stride;
                     s.hist[slot] = key[j];
-                    in_cut |= 1u << j;
+                    ++slot;
                 }
             }
         }
+        if (HAVE_RANGE) VSA_PROBE(26);
         __syncthreads();
         const int m = (int)s.misc[4];
+        if (HAVE_RANGE) VSA_PROBE_VAL(41, m);
         for (int t = tid; t < m; t += stride) {
             const int idx = s.list[t];
             const uint32_t kt = s.hist[t];
@@ -611,10 +657,12 @@ __device__ __forceinline__ TopkRegResult block_topk_reg(const uint32_t (&key)[KP
                 s.misc[6] = (uint32_t)idx;
             }
         }
+        if (HAVE_RANGE) VSA_PROBE(27);
         __syncthreads();
 #pragma unroll
         for (int j = 0; j < KPT; ++j)
             if (((in_cut >> j) & 1u) && spill_take[tid + j * stride]) out.mask |= 1u << j;
+        if (HAVE_RANGE) VSA_PROBE(28);
     } else {
         __syncthreads();
 #pragma unroll

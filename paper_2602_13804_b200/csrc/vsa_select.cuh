@@ -130,13 +130,20 @@ __device__ __forceinline__ int select_top_pages_keys(const uint32_t (&key)[KPT],
         uint32_t theta = 0xffffffffu;
         for (int w = 0; w < nw_full; ++w) theta = min(theta, s.ts.wred[w]);
         if (r > 32) theta = 0u;   // too few scores to filter: every score is a candidate
+        {
+            uint32_t keep = 0u;
 #pragma unroll
-        for (int j = 0; j < KPT; ++j) {
-            if (key[j] != 0u && key[j] >= theta) {
-                const int slot = (int)atomicAdd(&s.ts.misc[4], 1u);
-                if (slot < kTopkList) {
-                    s.ts.list[slot] = tid + j * stride;
-                    s.ts.hist[slot] = key[j];
+            for (int j = 0; j < KPT; ++j)
+                if (key[j] != 0u && key[j] >= theta) keep |= 1u << j;
+            int slot = warp_append_slots(__popc(keep), &s.ts.misc[4]);
+#pragma unroll
+            for (int j = 0; j < KPT; ++j) {
+                if ((keep >> j) & 1u) {
+                    if (slot < kTopkList) {
+                        s.ts.list[slot] = tid + j * stride;
+                        s.ts.hist[slot] = key[j];
+                    }
+                    ++slot;
                 }
             }
         }
