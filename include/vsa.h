@@ -187,11 +187,17 @@ int vsa_decode_step_timed(const vsa_shape_t* shape, const void* q, const void* s
  * (bf16 [batch][n_q_heads][head_dim]) to q_dev, runs vsa_decode_step, and copies the results
  * back into out_host (fp32 [batch][n_q_heads][head_dim]) and diag_host ([batch][n_q_heads],
  * may be NULL).  The KV cache, summaries, block table and lengths stay device-resident: they
- * are the decode state, not per-step inputs.  Copies are asynchronous on `stream`; the host
- * buffers must stay valid until the stream has been synchronised by the caller.
- *   q_host, out_host, diag_host: host (pinned for real asynchrony).
+ * are the decode state, not per-step inputs.  Everything is asynchronous on `stream`; the host
+ * buffers must stay valid, and hold the results, once the stream has been synchronised by the
+ * caller.
+ *   q_host, out_host, diag_host: host.  q is brought into q_dev on the stream (by a kernel
+ *   that reads it across the bus when it is page-locked, by a copy otherwise).  A page-locked
+ *   (cudaHostAlloc / cudaHostRegister) out_host or diag_host is written IN PLACE by the kernels,
+ *   with no copy and without touching its staging buffer; a pageable one is staged through
+ *   out_dev / diag_dev with a copy on the stream.
  *   q_dev, out_dev, diag_dev, routed_pages, fallback_list, fallback_count, ws: device staging
- *   and scratch buffers of the sizes given for vsa_decode_step.
+ *   and scratch buffers of the sizes given for vsa_decode_step; the contents of the three staging
+ *   buffers after the call are unspecified.
  */
 int vsa_decode_step_host(const vsa_shape_t* shape, const void* q_host, void* q_dev, const void* summaries,
                          const void* k_cache, const void* v_cache, const int32_t* block_table,

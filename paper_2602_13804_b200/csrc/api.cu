@@ -16,6 +16,31 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// device-side address of a page-locked (pinned or registered) host buffer, NULL for anything else
+const void* mapped_device_pointer(const void* host)
+{
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, host) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return nullptr;
+    }
+    if (attr.type != cudaMemoryTypeHost || !attr.devicePointer) return nullptr;
+    return attr.devicePointer;
+}
+
+// Brings the step's queries from page-locked host memory into the device staging buffer with plain
+// 16-byte loads across the bus: one short kernel in the stream's launch chain instead of a copy
+// operation, which would serialise fully against the kernels before and after it.
+__global__ void fetch_rows_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, int n16)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (i < n16) v = vsa::ld_nc_16B(src + i);   // host memory is stable: fetched before the wait
+    vsa::pdl_wait();                            // the previous step's kernels may still read dst
+    vsa::pdl_launch_dependents();
+    if (i < n16) dst[i] = v;
+}
+
 // shape checks shared by every entry point; fills the kernel-side geometry
 int make_geometry(const vsa_shape_t* s, Geometry* g)
 {
@@ -265,16 +290,31 @@ int vsa_decode_step_host(const vsa_shape_t* shape, const void* q_host, void* q_d
     if (ws_bytes < step_route_part(g) + vsa::dense_workspace_bytes(g)) return VSA_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t st = (cudaStream_t)stream;
     const size_t units = (size_t)g.batch * g.n_q_heads;
-    if (cudaMemcpyAsync(q_dev, q_host, units * vsa::kHeadDim * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    // Page-locked result buffers are written in place by the kernels (posted stores across the bus,
+    // overlapped with the rest of the step); pageable ones go through the device staging buffers
+    // with a copy on the stream.  q is always staged (every warp of the routing scan re-reads it, which
+    // only the device's caches serve well): by a fetch kernel when page-locked, by a copy otherwise.
+    float* out_direct = (float*)mapped_device_pointer(out_host);
+    vsa_diag_t* diag_direct = diag_host ? (vsa_diag_t*)mapped_device_pointer(diag_host) : nullptr;
+    const void* q_mapped = mapped_device_pointer(q_host);
+    if (q_mapped && aligned16(q_mapped)) {
+        const int n16 = (int)(units * vsa::kHeadDim * 2 / 16);
+        if (vsa::launch_pdl(fetch_rows_kernel, dim3((unsigned)((n16 + 255) / 256)), dim3(256), 0, st,
+                            (const uint4*)q_mapped, (uint4*)q_dev, n16) != cudaSuccess)
+            return VSA_ERR_CUDA;
+    } else if (cudaMemcpyAsync(q_dev, q_host, units * vsa::kHeadDim * 2, cudaMemcpyHostToDevice, st) !=
+               cudaSuccess) {
         return VSA_ERR_CUDA;
-    rc = vsa_decode_step(shape, q_dev, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon,
-                         gap_threshold, out_dev, diag_dev, routed_pages, fallback_list, fallback_count, ws,
+    }
+    rc = vsa_decode_step(shape, q_dev, summaries, k_cache, v_cache, block_table, seq_lens, P,
+                         K_c, epsilon, gap_threshold, out_direct ? out_direct : out_dev,
+                         diag_direct ? diag_direct : diag_dev, routed_pages, fallback_list, fallback_count, ws,
                          ws_bytes, stream);
     if (rc) return rc;
-    if (cudaMemcpyAsync(out_host, out_dev, units * vsa::kHeadDim * sizeof(float), cudaMemcpyDeviceToHost, st) !=
-        cudaSuccess)
+    if (!out_direct && cudaMemcpyAsync(out_host, out_dev, units * vsa::kHeadDim * sizeof(float),
+                                       cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return VSA_ERR_CUDA;
-    if (diag_host &&
+    if (diag_host && !diag_direct &&
         cudaMemcpyAsync(diag_host, diag_dev, units * sizeof(vsa_diag_t), cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return VSA_ERR_CUDA;
     return VSA_OK;

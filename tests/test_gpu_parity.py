@@ -166,6 +166,16 @@ def test_host_buffer_step_matches_device_step():
     torch.cuda.synchronize()
     assert torch.equal(out_host, out_dev.cpu())
     assert torch.equal(dec.diag_host, dec.diag.cpu())
+    # pageable host buffers take the staged-copy route; page-locked ones above are used in place
+    diag_ref = dec.diag.cpu().clone()
+    out_pg = torch.full(out_host.shape, float("nan"), dtype=torch.float32)
+    diag_pg = torch.zeros_like(dec.diag_host, pin_memory=False)
+    assert not out_pg.is_pinned() and not w.q.is_pinned()
+    B.vsa_decode_step_host(shape, w.q, dec.q_dev, summ, wd.k_cache, wd.v_cache, wd.block_table, wd.seq_lens, 6, 48,
+                           w.epsilon, w.gap_threshold, out_pg, dec.out, diag_pg, dec.diag, dec.routed_pages,
+                           dec.fallback_list, dec.fallback_count, dec.ws)
+    torch.cuda.synchronize()
+    assert torch.equal(out_pg, out_dev.cpu()) and torch.equal(diag_pg, diag_ref)
     q, K, V, bt, sl = host_arrays(w)
     st = oracle.decode_step(geometry(w), q, K, V, bt, sl, 6, 48, w.epsilon, w.gap_threshold)
     check_out(out_host.numpy(), st.out, "host step")
