@@ -43,6 +43,9 @@ def parse_args():
     ap.add_argument("--dense-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--solver-iters", type=int, default=None,
+                    help="time the step whose candidate weights come from this many entropic mirror-descent "
+                         "iterations (vsa_decode_step_entropic) instead of the closed form")
     return ap.parse_args()
 
 
@@ -260,11 +263,16 @@ def run_ours(args):
     ws = B.alloc_workspace(shape, P, K_c, B.VSA_WS_STEP, dev)
     ws_dense = B.alloc_workspace(shape, P, K_c, B.VSA_WS_DENSE, dev)
 
+    solve = B.alloc_solve(units, dev) if args.solver_iters is not None else None
+
     def layer_call(i):
         w, s = layers[i % distinct], summaries[i % distinct]
         if args.dense_baseline:
             B.vsa_dense_decode_fallback(shape, w.q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, None, None,
                                         eps, out, diag, ws_dense)
+        elif solve is not None:
+            B.vsa_decode_step_entropic(shape, w.q, s, w.k_cache, w.v_cache, w.block_table, w.seq_lens, P, K_c, eps,
+                                       tau, args.solver_iters, out, diag, solve, routed, flist, fcount, ws)
         else:
             B.vsa_decode_step(shape, w.q, s, w.k_cache, w.v_cache, w.block_table, w.seq_lens, P, K_c, eps, tau,
                               out, diag, routed, flist, fcount, ws)
@@ -345,9 +353,33 @@ def run_ours(args):
             per_kernel = dict(zip(["route_scan", "route_select", "sparse_decode", "dense_fallback"],
                                   (acc / (n_rep * L) * 1e3).tolist()))    # us per launch
 
+        # ---- with --solver-iters: the closed-form step timed the same way, for the cost of the iterations ----
+        closed_form_us_per_layer = None
+        if solve is not None:
+            def step_closed():
+                for i in range(L):
+                    w, s = layers[i % distinct], summaries[i % distinct]
+                    B.vsa_decode_step(shape, w.q, s, w.k_cache, w.v_cache, w.block_table, w.seq_lens, P, K_c, eps, tau,
+                                      out, diag, routed, flist, fcount, ws)
+            step_c = step_closed
+            if use_graph:
+                graph_c = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph_c, stream=stream):
+                    step_closed()
+                step_c = graph_c.replay
+            for _ in range(3):
+                step_c()
+            barrier()
+            e0.record(stream)
+            for _ in range(args.steps):
+                step_c()
+            e1.record(stream)
+            barrier()
+            closed_form_us_per_layer = max_over_ranks(e0.elapsed_time(e1), world, dev) / args.steps * 1e3 / L
+
         # ---- end to end: q from pinned host memory, out + diag back to the host, every layer ----
         e2e = None
-        if not args.dense_baseline:
+        if not args.dense_baseline and solve is None:
             q_host = [w.q.cpu().pin_memory() for w in layers]
             q_dev = torch.empty_like(w0.q)
             out_host = torch.empty(out.shape, dtype=torch.float32).pin_memory()
@@ -421,12 +453,20 @@ def run_ours(args):
         overhead = per_kernel["route_select"]
         roof = {"kernel": dom, "bytes_per_launch": alg[dom], "us_per_launch": per_kernel[dom] - overhead,
                 "us_event_interval": per_kernel[dom], "us_event_pair_overhead": overhead}
+        if solve is not None:
+            # the events bracket the closed-form kernels; the iterations' cost is the difference of the
+            # two graph-replayed steps and belongs to the sparse kernel
+            extra = ms_per_step * 1e3 / L - closed_form_us_per_layer
+            roof = {"kernel": "sparse_decode", "bytes_per_launch": alg["sparse_decode"],
+                    "us_per_launch": per_kernel["sparse_decode"] - overhead + extra,
+                    "us_event_interval": per_kernel["sparse_decode"], "us_event_pair_overhead": overhead,
+                    "us_solver_iterations": extra}
     achieved = roof["bytes_per_launch"] / (roof["us_per_launch"] * 1e-6) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": ncu_traffic(roof["kernel"], spec.name), "kernel": roof["kernel"],
                 "bytes_per_launch": roof["bytes_per_launch"], "us_per_launch": roof["us_per_launch"],
                 "peak_kind": f"of {peak_kind}", "frac_of_8TBps": achieved / 8000.0}
-    for k in ("us_event_interval", "us_event_pair_overhead"):
+    for k in ("us_event_interval", "us_event_pair_overhead", "us_solver_iterations"):
         if k in roof:
             roofline[k] = roof[k]
 
@@ -449,9 +489,12 @@ def run_ours(args):
                    "l2": f"inputs larger than L2: {distinct} distinct layer caches, "
                          f"{(scan_bytes + sparse_bytes) * distinct / 1e6:.0f} MB touched per pass over them",
                    "launch": "cuda graph replay of the whole step" if use_graph else "plain stream launches",
-                   "path": "dense split-K baseline" if args.dense_baseline else "route -> sparse -> dense fallback"},
+                   "path": "dense split-K baseline" if args.dense_baseline else
+                           ("route -> sparse -> dense fallback" if solve is None else
+                            f"route -> sparse with {args.solver_iters} entropic mirror-descent iterations -> dense fallback")},
         "latency_us_per_layer": ms_per_step * 1e3 / L,
-        "per_kernel_us": per_kernel, "fallback_fraction_last_layer": fb_count / units,
+        "per_kernel_us": per_kernel, "closed_form_latency_us_per_layer": closed_form_us_per_layer,
+        "fallback_fraction_last_layer": fb_count / units,
         "summary_build_ms_per_layer": summary_ms_per_layer,
         "gpu_launches": args.steps * L * kernels_per_layer, "clocks": clocks, "e2e": e2e, "roofline": roofline,
         "cpu_baseline": cpu_baseline,

@@ -143,6 +143,39 @@ int vsa_sparse_decode(const vsa_shape_t* shape, const void* q, const void* k_cac
                       size_t ws_bytes, void* stream);
 
 /*
+ * The same pass with the weights of step 3 obtained by an iterative solve (Sec. 7 step 3
+ * "convex sparse solve ... small iterations and certificates"; Sec. 5.3 and App. E name entropic
+ * mirror descent and the Frank-Wolfe gap; App. F sweeps 2, 4 and 6 iterations).  On the candidate
+ * set S of the unit, with k_i its key rows, the problem is Eq. (5.1) restricted to S,
+ *     minimise over the simplex  1/2 |sum_i a_i k_i - q|^2 + epsilon * sum_i a_i log a_i,
+ * started from the closed form a = softmax(<q, k_i> / epsilon) that vsa_sparse_decode uses and
+ * advanced by `solver_iters` entropic mirror-descent steps
+ *     g = K_S (K_S^T a) - K_S q,   log a <- (log a - eta * g) / (1 + eta * epsilon) + const,
+ * eta = 1 / max_i |k_i|^2 (the paper fixes neither start nor step; with this eta the objective
+ * never increases).  out = sum_i a_i V_i with the final weights.  solve[b][h] receives the
+ * certificate and the objective at the final weights.  Candidates, diag (lse is that of the
+ * closed-form weights) and the fallback list are exactly those of vsa_sparse_decode; units that
+ * fall back are later overwritten by plain dense softmax attention, as there.
+ *   solver_iters in [0, 64]; 0 returns the closed-form weights together with their certificate.
+ *   K_c <= VSA_SOLVER_MAX_CANDIDATES (the candidate keys are held on chip across iterations).
+ *   solve: device vsa_solve_t [batch][n_q_heads].  Everything else as for vsa_sparse_decode.
+ */
+#define VSA_SOLVER_MAX_CANDIDATES 256
+#define VSA_SOLVER_MAX_ITERS 64
+typedef struct {
+    float fw_gap;    /* App. E: <grad f(a), a> - min_j grad f(a)_j >= f(a) - min f,  f = 1/2 |K_S^T a - q|^2 */
+    float objective; /* 1/2 |K_S^T a - q|^2 + epsilon * sum_i a_i log a_i                                   */
+    float residual2; /* |K_S^T a - q|^2                                                                      */
+    float step;      /* eta                                                                                  */
+} vsa_solve_t;
+
+int vsa_sparse_decode_entropic(const vsa_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,
+                               const int32_t* block_table, const int32_t* seq_lens, const int32_t* routed_pages,
+                               int32_t P, int32_t K_c, float epsilon, float gap_threshold, int32_t solver_iters,
+                               float* out, vsa_diag_t* diag, vsa_solve_t* solve, int32_t* fallback_list,
+                               int32_t* fallback_count, void* stream);
+
+/*
  * Dense fallback (Sec. 10.3 "fallback-to-dense"): for every unit in fallback_list[0 ..
  * *fallback_count) recompute out[b][h][:] = softmax(<q, k_t> / epsilon over all T_b tokens) V
  * with a split-K pass (K and V of a KV head are read once for all listed heads of its
@@ -167,6 +200,16 @@ int vsa_decode_step(const vsa_shape_t* shape, const void* q, const void* summari
                     int32_t K_c, float epsilon, float gap_threshold, float* out, vsa_diag_t* diag,
                     int32_t* routed_pages, int32_t* fallback_list, int32_t* fallback_count, void* ws,
                     size_t ws_bytes, void* stream);
+
+/*
+ * vsa_decode_step with the iterative solve of vsa_sparse_decode_entropic in place of the closed-form
+ * weights: vsa_route_pages -> vsa_sparse_decode_entropic -> vsa_dense_decode_fallback.
+ */
+int vsa_decode_step_entropic(const vsa_shape_t* shape, const void* q, const void* summaries, const void* k_cache,
+                             const void* v_cache, const int32_t* block_table, const int32_t* seq_lens, int32_t P,
+                             int32_t K_c, float epsilon, float gap_threshold, int32_t solver_iters, float* out,
+                             vsa_diag_t* diag, vsa_solve_t* solve, int32_t* routed_pages, int32_t* fallback_list,
+                             int32_t* fallback_count, void* ws, size_t ws_bytes, void* stream);
 
 /*
  * vsa_decode_step with CUDA events recorded on `stream` between its kernels, for per-kernel

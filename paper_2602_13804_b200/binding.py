@@ -73,9 +73,13 @@ def lib() -> C.CDLL:
                                                vp, C.POINTER(C.c_void_p)]
         _lib.vsa_decode_step_host.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32,
                                               vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        _lib.vsa_sparse_decode_entropic.argtypes = [shp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, i32, vp, vp, vp,
+                                                    vp, vp, vp]
+        _lib.vsa_decode_step_entropic.argtypes = [shp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, i32, vp, vp, vp,
+                                                  vp, vp, vp, vp, sz, vp]
         for name in ("vsa_build_page_summaries", "vsa_route_pages", "vsa_sparse_decode",
                      "vsa_dense_decode_fallback", "vsa_decode_step", "vsa_decode_step_timed",
-                     "vsa_decode_step_host"):
+                     "vsa_decode_step_host", "vsa_sparse_decode_entropic", "vsa_decode_step_entropic"):
             getattr(_lib, name).restype = C.c_int
     return _lib
 
@@ -178,6 +182,27 @@ def vsa_decode_step(shape, q, summaries, k_cache, v_cache, block_table, seq_lens
            "vsa_decode_step")
 
 
+def vsa_sparse_decode_entropic(shape, q, k_cache, v_cache, block_table, seq_lens, routed_pages, P, K_c, epsilon,
+                               gap_threshold, solver_iters, out, diag, solve, fallback_list, fallback_count,
+                               stream=None) -> None:
+    _check(lib().vsa_sparse_decode_entropic(C.byref(shape), _ptr(q), _ptr(k_cache), _ptr(v_cache),
+                                            _ptr(block_table), _ptr(seq_lens), _ptr(routed_pages), P, K_c, epsilon,
+                                            gap_threshold, solver_iters, _ptr(out), _ptr(diag), _ptr(solve),
+                                            _ptr(fallback_list), _ptr(fallback_count), _stream(stream)),
+           "vsa_sparse_decode_entropic")
+
+
+def vsa_decode_step_entropic(shape, q, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon,
+                             gap_threshold, solver_iters, out, diag, solve, routed_pages, fallback_list,
+                             fallback_count, ws, stream=None) -> None:
+    _check(lib().vsa_decode_step_entropic(C.byref(shape), _ptr(q), _ptr(summaries), _ptr(k_cache), _ptr(v_cache),
+                                          _ptr(block_table), _ptr(seq_lens), P, K_c, epsilon, gap_threshold,
+                                          solver_iters, _ptr(out), _ptr(diag), _ptr(solve), _ptr(routed_pages),
+                                          _ptr(fallback_list), _ptr(fallback_count), _ptr(ws),
+                                          0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
+           "vsa_decode_step_entropic")
+
+
 def vsa_decode_step_timed(shape, q, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon,
                           gap_threshold, out, diag, routed_pages, fallback_list, fallback_count, ws, events,
                           stream=None) -> None:
@@ -210,6 +235,15 @@ def vsa_decode_step_host(shape, q_host, q_dev, summaries, k_cache, v_cache, bloc
 def alloc_diag(units: int, device) -> torch.Tensor:
     """Device buffer for `units` vsa_diag_t records, viewed as int32 [units, 8]."""
     return torch.zeros((units, DIAG_BYTES // 4), dtype=torch.int32, device=device)
+
+
+SOLVE_FIELDS = ("fw_gap", "objective", "residual2", "step")
+VSA_SOLVER_MAX_CANDIDATES = 256
+
+
+def alloc_solve(units: int, device) -> torch.Tensor:
+    """Device buffer for `units` vsa_solve_t records: float32 [units, 4], columns = SOLVE_FIELDS."""
+    return torch.zeros((units, len(SOLVE_FIELDS)), dtype=torch.float32, device=device)
 
 
 def diag_to_dict(diag: torch.Tensor) -> dict:

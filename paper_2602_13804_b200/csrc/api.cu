@@ -84,6 +84,13 @@ int check_routing_sizes(const Geometry& g, int P, int K_c, bool need_kc)
     return VSA_OK;
 }
 
+int check_solver_sizes(int K_c, int solver_iters)
+{
+    if (solver_iters < 0 || solver_iters > VSA_SOLVER_MAX_ITERS) return VSA_ERR_INVALID_ARGUMENT;
+    if (K_c > VSA_SOLVER_MAX_CANDIDATES) return VSA_ERR_UNSUPPORTED_SHAPE;
+    return VSA_OK;
+}
+
 int check_epsilon(float epsilon)
 {
     if (!(epsilon > 0.0f) || isinf(epsilon)) return VSA_ERR_INVALID_ARGUMENT;
@@ -182,6 +189,30 @@ int vsa_sparse_decode(const vsa_shape_t* shape, const void* q, const void* k_cac
                                       P, K_c, epsilon, gap_threshold, out, diag, fallback_list, fallback_count, st));
 }
 
+int vsa_sparse_decode_entropic(const vsa_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,
+                               const int32_t* block_table, const int32_t* seq_lens, const int32_t* routed_pages,
+                               int32_t P, int32_t K_c, float epsilon, float gap_threshold, int32_t solver_iters,
+                               float* out, vsa_diag_t* diag, vsa_solve_t* solve, int32_t* fallback_list,
+                               int32_t* fallback_count, void* stream)
+{
+    Geometry g;
+    int rc = make_geometry(shape, &g);
+    if (rc) return rc;
+    if ((rc = check_routing_sizes(g, P, K_c, true))) return rc;
+    if ((rc = check_solver_sizes(K_c, solver_iters))) return rc;
+    if ((rc = check_epsilon(epsilon))) return rc;
+    if (isnan(gap_threshold)) return VSA_ERR_INVALID_ARGUMENT;
+    if (!q || !k_cache || !v_cache || !block_table || !seq_lens || !routed_pages || !out || !diag || !solve ||
+        !fallback_list || !fallback_count)
+        return VSA_ERR_INVALID_ARGUMENT;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache)) return VSA_ERR_MISALIGNED;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemsetAsync(fallback_count, 0, sizeof(int32_t), st) != cudaSuccess) return VSA_ERR_CUDA;
+    return cuda_rc(vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, (int32_t*)routed_pages, nullptr,
+                                      P, K_c, epsilon, gap_threshold, out, diag, fallback_list, fallback_count, st,
+                                      solver_iters, solve));
+}
+
 int vsa_dense_decode_fallback(const vsa_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,
                               const int32_t* block_table, const int32_t* seq_lens, const int32_t* fallback_list,
                               const int32_t* fallback_count, float epsilon, float* out, vsa_diag_t* diag,
@@ -203,12 +234,14 @@ static int decode_step_impl(const vsa_shape_t* shape, const void* q, const void*
                             const void* v_cache, const int32_t* block_table, const int32_t* seq_lens, int32_t P,
                             int32_t K_c, float epsilon, float gap_threshold, float* out, vsa_diag_t* diag,
                             int32_t* routed_pages, int32_t* fallback_list, int32_t* fallback_count, void* ws,
-                            size_t ws_bytes, void* stream, void* const* events)
+                            size_t ws_bytes, void* stream, void* const* events, int solver_iters = 0,
+                            vsa_solve_t* solve = nullptr)
 {
     Geometry g;
     int rc = make_geometry(shape, &g);
     if (rc) return rc;
     if ((rc = check_routing_sizes(g, P, K_c, true))) return rc;
+    if (solve && (rc = check_solver_sizes(K_c, solver_iters))) return rc;
     if ((rc = check_epsilon(epsilon))) return rc;
     if (isnan(gap_threshold)) return VSA_ERR_INVALID_ARGUMENT;
     if (!q || !summaries || !k_cache || !v_cache || !block_table || !seq_lens || !out || !diag ||
@@ -234,7 +267,7 @@ static int decode_step_impl(const vsa_shape_t* shape, const void* q, const void*
     // the top-P selection runs inside the fused kernel, on the scores the scan left in ws
     if (ev[2] && cudaEventRecord(ev[2], st) != cudaSuccess) return VSA_ERR_CUDA;
     e = vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, routed_pages, (const float*)ws, P, K_c,
-                           epsilon, gap_threshold, out, diag, fallback_list, fallback_count, st);
+                           epsilon, gap_threshold, out, diag, fallback_list, fallback_count, st, solver_iters, solve);
     if (e != cudaSuccess) return VSA_ERR_CUDA;
     if (ev[3] && cudaEventRecord(ev[3], st) != cudaSuccess) return VSA_ERR_CUDA;
     e = vsa::launch_dense(g, q, k_cache, v_cache, block_table, seq_lens, fallback_list, fallback_count, epsilon,
@@ -253,6 +286,18 @@ int vsa_decode_step(const vsa_shape_t* shape, const void* q, const void* summari
     return decode_step_impl(shape, q, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon,
                             gap_threshold, out, diag, routed_pages, fallback_list, fallback_count, ws, ws_bytes,
                             stream, nullptr);
+}
+
+int vsa_decode_step_entropic(const vsa_shape_t* shape, const void* q, const void* summaries, const void* k_cache,
+                             const void* v_cache, const int32_t* block_table, const int32_t* seq_lens, int32_t P,
+                             int32_t K_c, float epsilon, float gap_threshold, int32_t solver_iters, float* out,
+                             vsa_diag_t* diag, vsa_solve_t* solve, int32_t* routed_pages, int32_t* fallback_list,
+                             int32_t* fallback_count, void* ws, size_t ws_bytes, void* stream)
+{
+    if (!solve) return VSA_ERR_INVALID_ARGUMENT;
+    return decode_step_impl(shape, q, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon,
+                            gap_threshold, out, diag, routed_pages, fallback_list, fallback_count, ws, ws_bytes,
+                            stream, nullptr, solver_iters, solve);
 }
 
 int vsa_decode_step_timed(const vsa_shape_t* shape, const void* q, const void* summaries, const void* k_cache,

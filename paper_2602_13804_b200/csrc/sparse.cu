@@ -20,8 +20,8 @@ constexpr int kMaxSparseWarps = 16;
 // token-phase shared memory, in 4-byte words, after the two page arrays
 __host__ __device__ constexpr int token_phase_words(int P, int K_c)
 {
-    return P * kPageSize /*keys*/ + (P * kPageSize + 3) / 4 /*take*/ + 2 * K_c + 2 /*voff*/ + K_c /*wgt*/ + 256 + 16 +
-           72 + kTopkList + kMaxSparseWarps * kHeadDim + kMaxSparseWarps + 4;
+    return P * kPageSize /*keys*/ + (P * kPageSize + 3) / 4 /*take*/ + 2 * K_c + 2 /*voff*/ + K_c /*wgt*/ +
+           K_c /*score*/ + 256 + 16 + 72 + kTopkList + kMaxSparseWarps * kHeadDim + kMaxSparseWarps + 4;
 }
 
 // first word of the block-table copy: after the two page arrays and the larger of the two phases
@@ -32,11 +32,24 @@ __host__ __device__ inline int bt_stage_offset_words(int max_pages, int P, int K
     return 2 * P + words;
 }
 
+// rows of the candidate key tile of the iterative solve: K_c rounded up to whole half-warps of
+// sixteen, plus sixteen rows of zeros for the half-warps that own no candidate
+__host__ __device__ constexpr int solve_tile_rows(int K_c) { return ((K_c + 15) & ~15) + 16; }
+
+// first word of that tile ([rows][128] bf16, 16-byte aligned): after the block-table copy when there
+// is one
+__host__ __device__ inline int solve_tile_offset_words(int max_pages, int P, int K_c, bool fused, bool staged)
+{
+    const int w = bt_stage_offset_words(max_pages, P, K_c, fused) + (staged ? max_pages : 0);
+    return (w + 3) & ~3;
+}
+
 struct TokenSmem {
     uint32_t* keys;   // [P * 16] token score keys, array index = 16 * slot + token (position order)
     uint8_t* take;    // [P * 16] scratch of the selection's slow path
     long long* voff;  // [K_c] element offset of each candidate's value row, candidates in position order
     float* wgt;       // [K_c] unnormalised softmax weight of each candidate
+    float* score;     // [K_c] score of each candidate (read by the iterative solve only)
     TopkScratch ts;
     float* red;       // [warps][128]
     float* zred;      // [warps]
@@ -52,7 +65,8 @@ __device__ __forceinline__ TokenSmem carve_tokens(uint32_t* base, int P, int K_c
     after_take += ((uintptr_t)after_take & 4u) ? 1 : 0;   // 8-byte alignment of the offsets
     s.voff = (long long*)after_take;
     s.wgt = (float*)(s.voff + K_c);
-    s.ts.hist = (uint32_t*)(s.wgt + K_c);
+    s.score = s.wgt + K_c;
+    s.ts.hist = (uint32_t*)(s.score + K_c);
     s.ts.misc = s.ts.hist + 256;
     s.ts.wred = s.ts.misc + 16;
     s.ts.list = (int32_t*)(s.ts.wred + 72);
@@ -82,16 +96,19 @@ __device__ __forceinline__ void write_failed_unit(float* out, vsa_diag_t* diag, 
 //   In both fused forms the unit's top-P pages are selected here from page_scores[unit][0..n_b) and
 //   written to routed_pages (best first, -1 padded).
 // TOK_KPT: token scores per thread, P * 16 <= TOK_KPT * THREADS.
-template <int THREADS, int PAGE_KPT, int TOK_KPT>
+// SOLVE: the weights on the candidates come from `solver_iters` entropic mirror-descent iterations
+//   (256 threads only: every lane owns one candidate, every half-warp sixteen candidate rows).
+template <int THREADS, int PAGE_KPT, int TOK_KPT, bool SOLVE = false>
 __global__ void __launch_bounds__(THREADS, 512 / THREADS)
 sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* __restrict__ k_cache,
                      const uint16_t* __restrict__ v_cache, const int32_t* __restrict__ block_table,
                      const int32_t* __restrict__ seq_lens, int32_t* __restrict__ routed_pages,
                      const float* __restrict__ page_scores, int P, int K_c, float epsilon, float gap_threshold,
                      float* __restrict__ out, vsa_diag_t* __restrict__ diag, int32_t* __restrict__ fallback_list,
-                     int32_t* __restrict__ fallback_count)
+                     int32_t* __restrict__ fallback_count, int solver_iters, vsa_solve_t* __restrict__ solve)
 {
     constexpr int WARPS = THREADS / 32, GROUPS = 2 * WARPS;
+    static_assert(!SOLVE || THREADS == 256, "the solve maps one candidate to each of 256 lanes");
     static_assert(TOK_KPT * WARPS <= 64 && 4 * WARPS <= 72, "wred capacity");
     extern __shared__ uint32_t smem_raw[];
     int32_t* page_l = (int32_t*)smem_raw;   // [P] routed logical pages, ascending, invalid entries last
@@ -130,6 +147,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     if (T <= 0 || T > geo.max_pages * kPageSize) {
         cp_async_wait_all();
         write_failed_unit(out, diag, unit, VSA_UNIT_BAD_LENGTH);
+        if (SOLVE && tid == 0) solve[unit] = vsa_solve_t{0.0f, 0.0f, 0.0f, 0.0f};
         if (PAGE_KPT != 0)
             for (int t = tid; t < P; t += THREADS) routed_pages[unit * P + t] = -1;
         return;
@@ -194,6 +212,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     VSA_PROBE(1);
     if (__syncthreads_or(bad)) {
         write_failed_unit(out, diag, unit, VSA_UNIT_BAD_PAGE);
+        if (SOLVE && tid == 0) solve[unit] = vsa_solve_t{0.0f, 0.0f, 0.0f, 0.0f};
         return;
     }
     const TokenSmem sm = carve_tokens(region, P, K_c);
@@ -339,12 +358,172 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                 const int i = tid + j * THREADS, pos = mine + before[j];
                 sm.voff[pos] = (long long)page_phys[i >> 4] * geo.page_stride + (long long)(i & 15) * geo.token_stride;
                 sm.wgt[pos] = exp2f((key_to_float(key[j]) - s1) * scale);
+                if constexpr (SOLVE) sm.score[pos] = key_to_float(key[j]);
             }
         }
     }
     __syncthreads();
 
     VSA_PROBE(6);
+    float lse_closed = 0.0f;   // log-sum-exp of the closed-form weights (SOLVE only)
+    if constexpr (SOLVE) {
+        if (ns > 0) {
+            // ---- iterative entropic solve on the candidates (Eq. (5.1) restricted to S) ----
+            // Lane (half-warp hw, column c) owns candidate j = 16 * hw + c: its score, log-weight and
+            // gradient entry live in registers.  Half-warp hw keeps the key rows of its sixteen
+            // candidates in shared memory, lane c reading column c of each.
+            const int hw = warp * 2 + gi, j_own = hw * 16 + c;
+            const bool have = j_own < ns;
+            uint8_t* ktile = (uint8_t*)(smem_raw + solve_tile_offset_words(geo.max_pages, P, K_c, PAGE_KPT != 0,
+                                                                           PAGE_KPT > 0));
+            // a half-warp without candidates works on the block of sixteen zero rows behind the tile
+            const int my_first = hw * 16 < ns ? hw * 16 : solve_tile_rows(K_c) - 16;
+            uint8_t* my_rows = ktile + (size_t)my_first * kRowBytes + c * 16;   // row r at + r * kRowBytes
+            {
+                const uint32_t dst = (uint32_t)__cvta_generic_to_shared(my_rows);
+                const uint16_t* kbase = k_cache + (long long)g * geo.head_stride + c * 8;
+#pragma unroll
+                for (int r = 0; r < 16; ++r) {
+                    if (hw * 16 + r < ns)
+                        cp_async_16B(dst + r * kRowBytes, kbase + sm.voff[hw * 16 + r]);
+                    else
+                        *reinterpret_cast<uint4*>(my_rows + r * kRowBytes) = make_uint4(0u, 0u, 0u, 0u);
+                }
+                cp_async_commit_group();
+                cp_async_wait_all();
+                __syncwarp();
+            }
+            const float s_own = have ? sm.score[j_own] : 0.0f;
+            float* ybuf = reinterpret_cast<float*>(sm.ts.hist);   // [128] current readout in key space
+            float vals[16];
+            // step: eta = 1 / max_i |k_i|^2
+#pragma unroll
+            for (int r = 0; r < 16; ++r) {
+                float uf[8];
+                unpack8(*reinterpret_cast<const uint4*>(my_rows + r * kRowBytes), uf);
+                vals[r] = chunk_partial(uf, uf);
+            }
+            {
+                const float nrm = reduce_scatter16(vals, c);
+                const uint32_t wmax = __reduce_max_sync(kFullMask, have ? float_to_key(nrm) : 0u);
+                if (lane == 0) sm.ts.wred[warp] = wmax;
+            }
+            __syncthreads();
+            uint32_t lkey = 0u;
+#pragma unroll
+            for (int w = 0; w < WARPS; ++w) lkey = max(lkey, sm.ts.wred[w]);
+            const float Lmax = lkey != 0u ? key_to_float(lkey) : 0.0f;
+            const float eta = Lmax > 0.0f ? 1.0f / Lmax : 0.0f;
+            const float shrink = 1.0f / (1.0f + eta * epsilon);
+            float l_own = have ? s_own / epsilon : -INFINITY;
+            float m = 0.0f, Z = 1.0f, a_own = 0.0f, g_own = 0.0f;
+            float yq[8];
+            __syncthreads();   // wred is rewritten below
+            for (int it = 0;; ++it) {
+                // softmax of the log-weights: block maximum, exponentials, block sum
+                {
+                    const uint32_t wmax = __reduce_max_sync(kFullMask, float_to_key(l_own));
+                    if (lane == 0) sm.ts.wred[warp] = wmax;
+                }
+                __syncthreads();
+                {
+                    uint32_t mk = 0u;
+#pragma unroll
+                    for (int w = 0; w < WARPS; ++w) mk = max(mk, sm.ts.wred[w]);
+                    m = key_to_float(mk);
+                }
+                a_own = have ? __expf(l_own - m) : 0.0f;
+                // y = sum_i a_i k_i: this half-warp's sixteen rows, then the block
+                float ya[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) ya[e] = 0.0f;
+#pragma unroll
+                for (int r = 0; r < 16; ++r) {
+                    const float a_r = __shfl_sync(kFullMask, a_own, (lane & 16) | r);
+                    float uf[8];
+                    unpack8(*reinterpret_cast<const uint4*>(my_rows + r * kRowBytes), uf);
+#pragma unroll
+                    for (int e = 0; e < 8; e += 2) fma2(ya[e], ya[e + 1], a_r, a_r, uf[e], uf[e + 1]);
+                }
+                float zw = a_own;
+#pragma unroll
+                for (int off = 16; off; off >>= 1) zw += __shfl_xor_sync(kFullMask, zw, off);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) ya[e] += __shfl_xor_sync(kFullMask, ya[e], 16);
+                if (gi == 0) {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) sm.red[warp * kHeadDim + c * 8 + e] = ya[e];
+                    if (c == 0) sm.zred[warp] = zw;
+                }
+                __syncthreads();
+                Z = 0.0f;
+#pragma unroll
+                for (int w = 0; w < WARPS; ++w) Z += sm.zred[w];
+                if (tid < kHeadDim) {
+                    float y = 0.0f;
+#pragma unroll
+                    for (int w = 0; w < WARPS; ++w) y += sm.red[w * kHeadDim + tid];
+                    ybuf[tid] = y / Z;
+                }
+                __syncthreads();
+#pragma unroll
+                for (int e = 0; e < 8; ++e) yq[e] = ybuf[c * 8 + e];
+                // gradient of the quadratic part: g_i = <k_i, y> - <k_i, q>
+#pragma unroll
+                for (int r = 0; r < 16; ++r) {
+                    float uf[8];
+                    unpack8(*reinterpret_cast<const uint4*>(my_rows + r * kRowBytes), uf);
+                    vals[r] = chunk_partial(yq, uf);
+                }
+                g_own = reduce_scatter16(vals, c) - s_own;
+                if (it == 0) lse_closed = m + logf(Z);
+                if (it >= solver_iters) break;
+                l_own = have ? ((l_own - m) - eta * g_own) * shrink : -INFINITY;
+            }
+            // certificate and objective at the final weights a_i = a_own / Z
+            {
+                const float alpha = a_own / Z;
+                float sum_ag = have ? alpha * g_own : 0.0f;
+                float ent = (have && alpha > 0.0f) ? alpha * ((l_own - m) - logf(Z)) : 0.0f;
+                float r2 = 0.0f;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) r2 += (yq[e] - qf[e]) * (yq[e] - qf[e]);
+#pragma unroll
+                for (int off = 8; off; off >>= 1) r2 += __shfl_xor_sync(kFullMask, r2, off);
+#pragma unroll
+                for (int off = 16; off; off >>= 1) {
+                    sum_ag += __shfl_xor_sync(kFullMask, sum_ag, off);
+                    ent += __shfl_xor_sync(kFullMask, ent, off);
+                }
+                // (-g) as a key: the largest key is the smallest gradient entry
+                const uint32_t wmin = __reduce_max_sync(kFullMask, have ? float_to_key(-g_own) : 0u);
+                if (lane == 0) {
+                    sm.ts.wred[8 + warp] = wmin;
+                    sm.ts.wred[16 + warp] = __float_as_uint(sum_ag);
+                    sm.ts.wred[24 + warp] = __float_as_uint(ent);
+                }
+                if (have) sm.wgt[j_own] = a_own;
+                __syncthreads();
+                if (tid == 0) {
+                    uint32_t gk = 0u;
+                    float sag = 0.0f, en = 0.0f;
+                    for (int w = 0; w < WARPS; ++w) {
+                        gk = max(gk, sm.ts.wred[8 + w]);
+                        sag += __uint_as_float(sm.ts.wred[16 + w]);
+                        en += __uint_as_float(sm.ts.wred[24 + w]);
+                    }
+                    vsa_solve_t sv;
+                    sv.fw_gap = sag + key_to_float(gk);   // <g, a> - min_j g_j
+                    sv.objective = 0.5f * r2 + epsilon * en;
+                    sv.residual2 = r2;
+                    sv.step = eta;
+                    solve[unit] = sv;
+                }
+            }
+        } else if (tid == 0) {
+            solve[unit] = vsa_solve_t{0.0f, 0.0f, 0.0f, 0.0f};
+        }
+    }
     // ---- value gather ----
     float acc[8], z = 0.0f;
 #pragma unroll
@@ -401,7 +580,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         d.delta = delta;
         d.delta12 = ns > 0 ? s1 - s2 : INFINITY;
         d.s_max = s1;
-        d.lse = ns > 0 ? s1 / epsilon + logf(Z) : -INFINITY;
+        d.lse = ns > 0 ? (SOLVE ? lse_closed : s1 / epsilon + logf(Z)) : -INFINITY;
         d.leak_bound = fminf(1.0f, (float)(T - ns) * expf(-delta / epsilon));
         d.n_candidates = ns;
         d.fallback = (delta < gap_threshold && ns < T) ? 1 : 0;
@@ -412,11 +591,15 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     VSA_PROBE_TMAX(52);
 }
 
-size_t sparse_smem_bytes(const Geometry& g, int P, int K_c, bool fused, int threads)
+size_t sparse_smem_bytes(const Geometry& g, int P, int K_c, bool fused, int threads, bool solve)
 {
-    size_t words = (size_t)bt_stage_offset_words(g.max_pages, P, K_c, fused);
     // the register variants of the fused kernel (PAGE_KPT > 0) keep a copy of the block-table row
-    if (fused && g.max_pages <= 32 * threads) words += (size_t)g.max_pages;
+    const bool staged = fused && g.max_pages <= 32 * threads;
+    if (solve)
+        return (size_t)solve_tile_offset_words(g.max_pages, P, K_c, fused, staged) * 4 +
+               (size_t)solve_tile_rows(K_c) * kRowBytes + 16;
+    size_t words = (size_t)bt_stage_offset_words(g.max_pages, P, K_c, fused);
+    if (staged) words += (size_t)g.max_pages;
     return words * 4 + 16;
 }
 
@@ -432,21 +615,33 @@ struct SparseArgs {
     float* out;
     vsa_diag_t* diag;
     int32_t *fallback_list, *fallback_count;
+    int solver_iters;
+    vsa_solve_t* solve;   // non-null: the iterative-solve variant of the kernel
     cudaStream_t stream;
 };
 
-template <int THREADS, int PAGE_KPT, int TOK_KPT>
-cudaError_t launch_one(const SparseArgs& a)
+template <int THREADS, int PAGE_KPT, int TOK_KPT, bool SOLVE>
+cudaError_t launch_variant(const SparseArgs& a)
 {
     if (a.smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(sparse_decode_kernel<THREADS, PAGE_KPT, TOK_KPT>,
+        cudaError_t e = cudaFuncSetAttribute(sparse_decode_kernel<THREADS, PAGE_KPT, TOK_KPT, SOLVE>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)a.smem);
         if (e != cudaSuccess) return e;
     }
     const unsigned units = (unsigned)(a.g.batch * a.g.n_q_heads);
-    return launch_pdl(sparse_decode_kernel<THREADS, PAGE_KPT, TOK_KPT>, dim3(units), dim3(THREADS), a.smem, a.stream,
-                      a.g, a.q, a.k, a.v, a.block_table, a.seq_lens, a.routed_pages, a.page_scores, a.P, a.K_c,
-                      a.epsilon, a.gap_threshold, a.out, a.diag, a.fallback_list, a.fallback_count);
+    return launch_pdl(sparse_decode_kernel<THREADS, PAGE_KPT, TOK_KPT, SOLVE>, dim3(units), dim3(THREADS), a.smem,
+                      a.stream, a.g, a.q, a.k, a.v, a.block_table, a.seq_lens, a.routed_pages, a.page_scores, a.P,
+                      a.K_c, a.epsilon, a.gap_threshold, a.out, a.diag, a.fallback_list, a.fallback_count,
+                      a.solver_iters, a.solve);
+}
+
+template <int THREADS, int PAGE_KPT, int TOK_KPT>
+cudaError_t launch_one(const SparseArgs& a)
+{
+    if constexpr (THREADS == 256) {
+        if (a.solve) return launch_variant<THREADS, PAGE_KPT, TOK_KPT, true>(a);
+    }
+    return launch_variant<THREADS, PAGE_KPT, TOK_KPT, false>(a);
 }
 
 template <int THREADS, int PAGE_KPT>
@@ -497,13 +692,17 @@ extern "C" int vsa_probe_read(long long* host64)
 cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache, const void* v_cache,
                           const int32_t* block_table, const int32_t* seq_lens, int32_t* routed_pages,
                           const float* page_scores, int P, int K_c, float epsilon, float gap_threshold, float* out,
-                          vsa_diag_t* diag, int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream)
+                          vsa_diag_t* diag, int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream,
+                          int solver_iters, vsa_solve_t* solve)
 {
     SparseArgs a;
     a.g = g;
-    // no more units than SMs: one larger block per unit (latency shape); otherwise two blocks per SM
-    const int threads = (long long)g.batch * g.n_q_heads <= sm_count() ? 512 : 256;
-    a.smem = sparse_smem_bytes(g, P, K_c, page_scores != nullptr, threads);
+    // no more units than SMs: one larger block per unit (latency shape); otherwise two blocks per SM.
+    // The iterative solve exists in the 256-thread shape only.
+    const int threads = (!solve && (long long)g.batch * g.n_q_heads <= sm_count()) ? 512 : 256;
+    a.smem = sparse_smem_bytes(g, P, K_c, page_scores != nullptr, threads, solve != nullptr);
+    a.solver_iters = solver_iters;
+    a.solve = solve;
     a.q = (const uint16_t*)q;
     a.k = (const uint16_t*)k_cache;
     a.v = (const uint16_t*)v_cache;

@@ -52,11 +52,13 @@ cudaError_t launch_route_select(const Geometry& g, const void* ws, const int32_t
 
 // ---- fused sparse pass ------------------------------------------------------------------------
 // page_scores == nullptr: routed_pages is read; otherwise the top-P selection runs inside the kernel on
-// page_scores (the scan's output) and routed_pages is written.
+// page_scores (the scan's output) and routed_pages is written.  solve != nullptr: the weights on the
+// candidates come from solver_iters entropic mirror-descent iterations (K_c <= 256).
 cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache, const void* v_cache,
                           const int32_t* block_table, const int32_t* seq_lens, int32_t* routed_pages,
                           const float* page_scores, int P, int K_c, float epsilon, float gap_threshold, float* out,
-                          vsa_diag_t* diag, int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream);
+                          vsa_diag_t* diag, int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream,
+                          int solver_iters = 0, vsa_solve_t* solve = nullptr);
 
 // ---- dense split-K pass -------------------------------------------------------------------------
 size_t dense_workspace_bytes(const Geometry& g);

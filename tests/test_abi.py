@@ -108,6 +108,27 @@ def test_sparse_argument_validation(lib):
     assert _sparse(lib, ok, q=ODD) == -4
 
 
+def test_entropic_argument_validation(lib):
+    ok = B.make_shape(2, 8, 2, 64, 256)
+    s = C.byref(ok)
+
+    def call(P=32, K_c=16, iters=4, solve=FAKE, eps=1.0):
+        return lib.vsa_sparse_decode_entropic(s, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, P, K_c, eps, 0.0, iters, FAKE, FAKE,
+                                              solve, FAKE, FAKE, None)
+
+    assert call(K_c=257) == -2             # more candidates than the on-chip tile holds
+    assert call(iters=-1) == -1 and call(iters=65) == -1
+    assert call(solve=None) == -1
+    assert call(eps=0.0) == -1
+    assert call(P=4, K_c=65) == -2
+    step = lib.vsa_decode_step_entropic
+    assert step(s, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, 32, 257, 1.0, 0.0, 2, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE,
+                1 << 40, None) == -2
+    assert step(s, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, 32, 16, 1.0, 0.0, 2, FAKE, FAKE, None, FAKE, FAKE, FAKE, FAKE,
+                1 << 40, None) == -1
+    assert C.sizeof(C.c_float) * len(B.SOLVE_FIELDS) == 16
+
+
 def test_dense_and_step_argument_validation(lib):
     ok = B.make_shape(2, 8, 2, 64, 256)
     s = C.byref(ok)
