@@ -394,7 +394,6 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                 __syncwarp();
             }
             const float s_own = have ? sm.score[j_own] : 0.0f;
-            float* ybuf = reinterpret_cast<float*>(sm.ts.hist);   // [128] current readout in key space
             float vals[16];
             // step: eta = 1 / max_i |k_i|^2
 #pragma unroll
@@ -419,55 +418,67 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
             float m = 0.0f, Z = 1.0f, a_own = 0.0f, g_own = 0.0f;
             float yq[8];
             __syncthreads();   // wred is rewritten below
+            // One block barrier per pass: every warp exponentiates against its own maximum and publishes
+            // (partial readout, partial sum, maximum); after the barrier every lane rebuilds the block-wide
+            // readout for its own eight columns.  The buffers alternate between passes.
             for (int it = 0;; ++it) {
-                // softmax of the log-weights: block maximum, exponentials, block sum
-                {
-                    const uint32_t wmax = __reduce_max_sync(kFullMask, float_to_key(l_own));
-                    if (lane == 0) sm.ts.wred[warp] = wmax;
-                }
-                __syncthreads();
-                {
-                    uint32_t mk = 0u;
-#pragma unroll
-                    for (int w = 0; w < WARPS; ++w) mk = max(mk, sm.ts.wred[w]);
-                    m = key_to_float(mk);
-                }
-                a_own = have ? __expf(l_own - m) : 0.0f;
-                // y = sum_i a_i k_i: this half-warp's sixteen rows, then the block
+                const float mw = key_to_float(__reduce_max_sync(kFullMask, float_to_key(l_own)));
+                const float e_own = have ? __expf(l_own - mw) : 0.0f;
+                // sum_i e_i k_i over this half-warp's sixteen rows, then over the warp
                 float ya[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) ya[e] = 0.0f;
 #pragma unroll
                 for (int r = 0; r < 16; ++r) {
-                    const float a_r = __shfl_sync(kFullMask, a_own, (lane & 16) | r);
+                    const float e_r = __shfl_sync(kFullMask, e_own, (lane & 16) | r);
                     float uf[8];
                     unpack8(*reinterpret_cast<const uint4*>(my_rows + r * kRowBytes), uf);
 #pragma unroll
-                    for (int e = 0; e < 8; e += 2) fma2(ya[e], ya[e + 1], a_r, a_r, uf[e], uf[e + 1]);
+                    for (int e = 0; e < 8; e += 2) fma2(ya[e], ya[e + 1], e_r, e_r, uf[e], uf[e + 1]);
                 }
-                float zw = a_own;
+                float zw = e_own;
 #pragma unroll
                 for (int off = 16; off; off >>= 1) zw += __shfl_xor_sync(kFullMask, zw, off);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) ya[e] += __shfl_xor_sync(kFullMask, ya[e], 16);
+                float* redb = sm.red + (it & 1) * (WARPS * kHeadDim);
+                uint32_t* statb = sm.ts.wred + (it & 1) * 16;   // [0..8) partial sums, [8..16) maxima
                 if (gi == 0) {
+                    // layout [warp][element pair][column]: the sixteen lanes of a half-warp touch 128
+                    // consecutive bytes (the area is 8-byte aligned, not more)
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) sm.red[warp * kHeadDim + c * 8 + e] = ya[e];
-                    if (c == 0) sm.zred[warp] = zw;
+                    for (int e = 0; e < 8; e += 2)
+                        *reinterpret_cast<float2*>(redb + ((warp * 4 + e / 2) * 16 + c) * 2) = make_float2(ya[e], ya[e + 1]);
+                    if (c == 0) {
+                        statb[warp] = __float_as_uint(zw);
+                        statb[8 + warp] = __float_as_uint(mw);
+                    }
                 }
                 __syncthreads();
+                m = -INFINITY;
+#pragma unroll
+                for (int w = 0; w < WARPS; ++w) m = fmaxf(m, __uint_as_float(statb[8 + w]));
                 Z = 0.0f;
 #pragma unroll
-                for (int w = 0; w < WARPS; ++w) Z += sm.zred[w];
-                if (tid < kHeadDim) {
-                    float y = 0.0f;
+                for (int e = 0; e < 8; ++e) yq[e] = 0.0f;
 #pragma unroll
-                    for (int w = 0; w < WARPS; ++w) y += sm.red[w * kHeadDim + tid];
-                    ybuf[tid] = y / Z;
+                for (int w = 0; w < WARPS; ++w) {
+                    const float mwv = __uint_as_float(statb[8 + w]);
+                    const float f = mwv > -INFINITY ? __expf(mwv - m) : 0.0f;
+                    Z = fmaf(__uint_as_float(statb[w]), f, Z);
+#pragma unroll
+                    for (int e = 0; e < 8; e += 2) {
+                        const float2 p = *reinterpret_cast<const float2*>(redb + ((w * 4 + e / 2) * 16 + c) * 2);
+                        yq[e] = fmaf(f, p.x, yq[e]);
+                        yq[e + 1] = fmaf(f, p.y, yq[e + 1]);
+                    }
                 }
-                __syncthreads();
+                {
+                    const float rz = 1.0f / Z;
 #pragma unroll
-                for (int e = 0; e < 8; ++e) yq[e] = ybuf[c * 8 + e];
+                    for (int e = 0; e < 8; ++e) yq[e] *= rz;
+                }
+                a_own = have ? e_own * __expf(mw - m) : 0.0f;   // exp(l_own - m)
                 // gradient of the quadratic part: g_i = <k_i, y> - <k_i, q>
 #pragma unroll
                 for (int r = 0; r < 16; ++r) {
@@ -498,9 +509,9 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                 // (-g) as a key: the largest key is the smallest gradient entry
                 const uint32_t wmin = __reduce_max_sync(kFullMask, have ? float_to_key(-g_own) : 0u);
                 if (lane == 0) {
-                    sm.ts.wred[8 + warp] = wmin;
-                    sm.ts.wred[16 + warp] = __float_as_uint(sum_ag);
-                    sm.ts.wred[24 + warp] = __float_as_uint(ent);
+                    sm.ts.wred[32 + warp] = wmin;
+                    sm.ts.wred[40 + warp] = __float_as_uint(sum_ag);
+                    sm.ts.wred[48 + warp] = __float_as_uint(ent);
                 }
                 if (have) sm.wgt[j_own] = a_own;
                 __syncthreads();
@@ -508,9 +519,9 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                     uint32_t gk = 0u;
                     float sag = 0.0f, en = 0.0f;
                     for (int w = 0; w < WARPS; ++w) {
-                        gk = max(gk, sm.ts.wred[8 + w]);
-                        sag += __uint_as_float(sm.ts.wred[16 + w]);
-                        en += __uint_as_float(sm.ts.wred[24 + w]);
+                        gk = max(gk, sm.ts.wred[32 + w]);
+                        sag += __uint_as_float(sm.ts.wred[40 + w]);
+                        en += __uint_as_float(sm.ts.wred[48 + w]);
                     }
                     vsa_solve_t sv;
                     sv.fw_gap = sag + key_to_float(gk);   // <g, a> - min_j g_j
