@@ -43,6 +43,8 @@ def parse_args():
     ap.add_argument("--dense-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--P", type=int, default=None, help="override the workload's routed pages per unit")
+    ap.add_argument("--Kc", type=int, default=None, help="override the workload's candidate count per unit")
     ap.add_argument("--solver-iters", type=int, default=None,
                     help="time the step whose candidate weights come from this many entropic mirror-descent "
                          "iterations (vsa_decode_step_entropic) instead of the closed form")
@@ -225,6 +227,11 @@ def run_ours(args):
     B.lib()
 
     spec = workload_spec(args.workload, args.layers)
+    if args.P is not None or args.Kc is not None:      # the (P, K_c) ablation grid of the paper's Table 3
+        from dataclasses import replace
+        P_new = args.P if args.P is not None else spec.P
+        K_new = args.Kc if args.Kc is not None else spec.K_c
+        spec = replace(spec, P=P_new, K_c=K_new, name=f"{spec.name}_P{P_new}_Kc{K_new}")
     L = spec.layers
     # one distinct KV cache per layer, sized against free memory (never more than 80% of it)
     w0 = make_workload(spec, device=dev, rep=0, sub=rank)
