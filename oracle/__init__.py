@@ -171,6 +171,7 @@ class SparseResult:
     fallback: np.ndarray      # int32 [B, Hq]
     cand_pos: np.ndarray      # int32 [B, Hq, K_c] token positions, -1 padded, selection order
     cand_weight: np.ndarray   # fp64 [B, Hq, K_c] normalised weights
+    best_rejected: np.ndarray = None   # fp32 [B, Hq] best scored token outside S, -inf if none
 
 
 def sparse(geo: Geometry, q, k_cache, v_cache, block_table, seq_lens, routed_pages, K_c: int,
@@ -183,12 +184,55 @@ def sparse(geo: Geometry, q, k_cache, v_cache, block_table, seq_lens, routed_pag
         out=np.zeros((B, H, d)), delta=np.zeros((B, H), np.float32), delta12=np.zeros((B, H), np.float32),
         s_max=np.zeros((B, H), np.float32), lse=np.zeros((B, H)), leak_bound=np.zeros((B, H)),
         n_candidates=np.zeros((B, H), np.int32), fallback=np.zeros((B, H), np.int32),
-        cand_pos=np.full((B, H, K_c), -1, np.int32), cand_weight=np.zeros((B, H, K_c)))
+        cand_pos=np.full((B, H, K_c), -1, np.int32), cand_weight=np.zeros((B, H, K_c)),
+        best_rejected=np.zeros((B, H), np.float32))
     s = geo.c()
     rc = lib().orc_sparse(C.byref(s), _p(qb), _p(k), _p(v), _p(bt), _p(sl), _p(rp), C.c_int(P), C.c_int(K_c),
                           C.c_float(epsilon), C.c_float(gap_threshold), _p(r.out), _p(r.delta), _p(r.delta12),
                           _p(r.s_max), _p(r.lse), _p(r.leak_bound), _p(r.n_candidates), _p(r.fallback),
-                          _p(r.cand_pos), _p(r.cand_weight))
+                          _p(r.cand_pos), _p(r.cand_weight), _p(r.best_rejected))
+    assert rc == 0, rc
+    return r
+
+
+def build_radii(geo: Geometry, k_cache, summaries, block_table, seq_lens, first_page=None, radii=None) -> np.ndarray:
+    """fp32 [pool, Hkv]: the slack-inflated radius of every owned page around its stored summary."""
+    k, sm = _u16(k_cache), _u16(summaries)
+    bt, sl = _i32(block_table), _i32(seq_lens)
+    if radii is None:
+        radii = np.zeros((geo.num_pool_pages, geo.n_kv_heads), np.float32)
+    fp = None if first_page is None else _i32(first_page)
+    s = geo.c()
+    rc = lib().orc_build_radii(C.byref(s), _p(k), _p(sm), _p(bt), _p(sl), _p(fp), _p(radii))
+    assert rc == 0, rc
+    return radii
+
+
+@dataclass
+class CertResult:
+    ub_unrouted: np.ndarray   # fp32 [B, Hq]
+    delta_cert: np.ndarray    # fp32 [B, Hq]
+    certified: np.ndarray     # int32 [B, Hq]
+    leak_cert: np.ndarray     # fp64 [B, Hq]
+
+
+def certify(geo: Geometry, q, radii, block_table, seq_lens, route: "RouteResult", sp: SparseResult,
+            epsilon: float, gap_threshold: float) -> CertResult:
+    """Certified gap of every unit from the page scores of `route` (made with want_all_scores=True)
+    and the closed-form pass `sp`."""
+    assert route.all_scores is not None
+    qb, bt, sl = _u16(q), _i32(block_table), _i32(seq_lens)
+    B, H = geo.batch, geo.n_q_heads
+    rp = _i32(route.pages)
+    r = CertResult(np.zeros((B, H), np.float32), np.zeros((B, H), np.float32), np.zeros((B, H), np.int32),
+                   np.zeros((B, H)))
+    rad = np.ascontiguousarray(radii, dtype=np.float32)
+    alls = np.ascontiguousarray(route.all_scores, dtype=np.float32)
+    s = geo.c()
+    rc = lib().orc_certify(C.byref(s), _p(qb), _p(rad), _p(bt), _p(sl), _p(alls), _p(rp), C.c_int(rp.shape[-1]),
+                           _p(np.ascontiguousarray(sp.s_max)), _p(np.ascontiguousarray(sp.best_rejected)),
+                           _p(np.ascontiguousarray(sp.n_candidates)), C.c_float(epsilon), C.c_float(gap_threshold),
+                           _p(r.ub_unrouted), _p(r.delta_cert), _p(r.certified), _p(r.leak_cert))
     assert rc == 0, rc
     return r
 

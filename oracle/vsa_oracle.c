@@ -17,6 +17,9 @@
  *                        Diagnostics: Def. 1 (face gap) evaluated with r -> q and
  *                        I -> candidate set; Sec. 8 gap statistic s(1) - s(2); Cor. 1
  *                        leakage bound with c = 1; Sec. 10.3 fallback-to-dense policy.
+ *   orc_build_radii,     a certificate for the routing (App. E "screening"; construction not in the
+ *   orc_certify          paper): per-page ball around the summary, upper bound on every un-scored
+ *                        token, certified gap and leakage bound.
  *   orc_dense            the plain definition: softmax(<q,k_t>/epsilon) over every token.
  * (The theory objects on tiny dictionaries - Euclidean projection, exact gap, the full
  *  entropic minimiser of Eq. (5.1) - live in theory.py next to this file.)
@@ -213,7 +216,7 @@ int orc_sparse(const orc_shape *s, const uint16_t *q, const uint16_t *K, const u
                const int32_t *seq_lens, const int32_t *routed_pages, int P, int K_c, float epsilon,
                float gap_threshold, double *out, float *delta, float *delta12, float *s_max, double *lse,
                double *leak_bound, int32_t *n_candidates, int32_t *fallback, int32_t *cand_pos,
-               double *cand_weight)
+               double *cand_weight, float *best_rejected)
 {
     if (!shape_ok(s) || P < 1 || K_c < 1 || !(epsilon > 0.0f)) return -1;
     const int G = s->n_q_heads / s->n_kv_heads;
@@ -276,6 +279,7 @@ int orc_sparse(const orc_shape *s, const uint16_t *q, const uint16_t *K, const u
         float d = nv > ns ? s1 - c[ns].s : INFINITY; /* best rejected scored token */
         float d12 = ns > 0 ? s1 - s2 : INFINITY;
         s_max[u] = s1;
+        if (best_rejected) best_rejected[u] = nv > ns ? c[ns].s : -INFINITY;
         delta[u] = d;
         delta12[u] = d12;
         n_candidates[u] = ns;
@@ -284,6 +288,108 @@ int orc_sparse(const orc_shape *s, const uint16_t *q, const uint16_t *K, const u
         fallback[u] = (d < gap_threshold && ns < T) ? 1 : 0;
         free(s64);
         free(c);
+    }
+    return 0;
+}
+
+/* ---- certified routing: an upper bound on every score that was never computed ----------
+ * (App. E "screening": a certificate that the candidate set holds the active face.  The paper
+ * gives no construction; this is the library's: a ball around each page summary.)
+ * For a page with stored summary mu (bf16) every valid key row k satisfies |k - mu| <= r, so for any
+ * query  <q, k> <= <q, mu> + |q| r.  The stored radius already carries the slack that covers all
+ * fp32 rounding on either side of that inequality:
+ *     rhat = r * 1.001 + 2^-12 * |mu|,   r = sqrt(max_t |k_t - mu|^2),
+ * with the squared norms summed in the canonical order (products fused into the additions, the
+ * first product of a chain rounded on its own - what a packed multiply followed by packed fused
+ * multiply-adds computes).  Every operation below is a single correctly rounded fp32 operation,
+ * so that a GPU can reproduce the numbers bit for bit. */
+static float canon_sumsq(const float *d)
+{
+    float p[16];
+    for (int c = 0; c < 16; ++c) {
+        float part[2];
+        for (int par = 0; par < 2; ++par) {
+            float acc = d[8 * c + par] * d[8 * c + par];
+            for (int e = 2 + par; e < 8; e += 2) acc = fmaf(d[8 * c + e], d[8 * c + e], acc);
+            part[par] = acc;
+        }
+        p[c] = part[0] + part[1];
+    }
+    for (int off = 8; off >= 1; off >>= 1)
+        for (int c = 0; c < off; ++c) p[c] = p[c] + p[c + off];
+    return p[0];
+}
+
+int orc_build_radii(const orc_shape *s, const uint16_t *K, const uint16_t *summaries, const int32_t *bt,
+                    const int32_t *seq_lens, const int32_t *first_page, float *radii)
+{
+    if (!shape_ok(s)) return -1;
+    for (int b = 0; b < s->batch; ++b) {
+        int T = seq_lens[b];
+        int nb = n_pages_of(s, T);
+        int l0 = first_page ? first_page[b] : 0;
+        for (int l = l0; l < nb; ++l) {
+            int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
+            int n = T - l * s->page_size;
+            if (n > s->page_size) n = s->page_size;
+            for (int g = 0; g < s->n_kv_heads; ++g) {
+                float mu[ORC_D], diff[ORC_D];
+                for (int e = 0; e < ORC_D; ++e) mu[e] = orc_bf16_to_f32(summaries[(p * s->n_kv_heads + g) * ORC_D + e]);
+                float d2max = 0.0f;
+                for (int t = 0; t < n; ++t) {
+                    const uint16_t *row = kv_row(s, K, p, g, t);
+                    for (int e = 0; e < ORC_D; ++e) diff[e] = orc_bf16_to_f32(row[e]) - mu[e];
+                    float d2 = canon_sumsq(diff);
+                    if (d2 > d2max) d2max = d2;
+                }
+                float r = sqrtf(d2max), mun = sqrtf(canon_sumsq(mu));
+                float t1 = r * 1.001f, t2 = mun * 0x1p-12f;
+                radii[p * s->n_kv_heads + g] = t1 + t2;
+            }
+        }
+    }
+    return 0;
+}
+
+/* Per unit, from the page scores of orc_route (all_scores), its routed pages, and s(1) / the best
+ * rejected scored token of orc_sparse:
+ *   ub_unrouted = max over valid un-routed pages of  c_l + qn * rhat_l,  qn = sqrt(|q|^2) * (1 + 2^-20)
+ *                 (-INF when every page is routed),
+ *   delta_cert  = s(1) - max(best rejected scored token, ub_unrouted)   (+INF when nothing is outside S):
+ *                 no token outside S scores above s(1) - delta_cert,
+ *   certified   = delta_cert >= gap_threshold,
+ *   leak_cert   = min(1, (T - |S|) exp(-delta_cert / eps))  (Cor. 1 with the certified gap). */
+int orc_certify(const orc_shape *s, const uint16_t *q, const float *radii, const int32_t *bt,
+                const int32_t *seq_lens, const float *all_scores, const int32_t *routed_pages, int P,
+                const float *s_max, const float *best_rejected, const int32_t *n_candidates, float epsilon,
+                float gap_threshold, float *ub_unrouted, float *delta_cert, int32_t *certified, double *leak_cert)
+{
+    if (!shape_ok(s) || P < 1) return -1;
+    const int G = s->n_q_heads / s->n_kv_heads;
+    const int units = s->batch * s->n_q_heads;
+    for (int u = 0; u < units; ++u) {
+        int b = u / s->n_q_heads, h = u % s->n_q_heads, g = h / G;
+        int T = seq_lens[b], nb = n_pages_of(s, T);
+        float qf[ORC_D];
+        for (int e = 0; e < ORC_D; ++e) qf[e] = orc_bf16_to_f32(q[(int64_t)u * ORC_D + e]);
+        float qn = sqrtf(canon_sumsq(qf)) * 1.00000095367431640625f;
+        float ub = -INFINITY;
+        for (int l = 0; l < nb; ++l) {
+            int routed = 0;
+            for (int i = 0; i < P; ++i) routed |= routed_pages[(int64_t)u * P + i] == l;
+            if (routed) continue;
+            int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
+            float t = qn * radii[p * s->n_kv_heads + g];
+            float v = all_scores[(int64_t)u * s->max_pages_per_seq + l] + t;
+            if (v > ub) ub = v;
+        }
+        float m = best_rejected[u] > ub ? best_rejected[u] : ub;
+        float d = m == -INFINITY ? INFINITY : s_max[u] - m;
+        ub_unrouted[u] = ub;
+        delta_cert[u] = d;
+        certified[u] = d >= gap_threshold ? 1 : 0;
+        double lb = (double)(T - n_candidates[u]) * exp(-(double)d / (double)epsilon);
+        leak_cert[u] = lb < 1.0 ? lb : 1.0;
     }
     return 0;
 }
