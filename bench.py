@@ -45,6 +45,9 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--P", type=int, default=None, help="override the workload's routed pages per unit")
     ap.add_argument("--Kc", type=int, default=None, help="override the workload's candidate count per unit")
+    ap.add_argument("--certified", action="store_true",
+                    help="time vsa_decode_step_certified (routing certificate computed, certified gap decides the "
+                         "fallback) instead of vsa_decode_step")
     ap.add_argument("--solver-iters", type=int, default=None,
                     help="time the step whose candidate weights come from this many entropic mirror-descent "
                          "iterations (vsa_decode_step_entropic) instead of the closed form")
@@ -271,12 +274,24 @@ def run_ours(args):
     ws_dense = B.alloc_workspace(shape, P, K_c, B.VSA_WS_DENSE, dev)
 
     solve = B.alloc_solve(units, dev) if args.solver_iters is not None else None
+    cert = radii = None
+    if args.certified:
+        cert = B.alloc_cert(units, dev)
+        ws = B.alloc_workspace(shape, P, K_c, B.VSA_WS_STEP_CERTIFIED, dev)
+        radii = []
+        for w, s_ in zip(layers, summaries):      # cache maintenance, like the summaries
+            r = torch.zeros((shape.num_pool_pages, shape.n_kv_heads), dtype=torch.float32, device=dev)
+            B.vsa_build_page_radii(shape, w.k_cache, s_, w.block_table, w.seq_lens, None, r)
+            radii.append(r)
 
     def layer_call(i):
         w, s = layers[i % distinct], summaries[i % distinct]
         if args.dense_baseline:
             B.vsa_dense_decode_fallback(shape, w.q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, None, None,
                                         eps, out, diag, ws_dense)
+        elif cert is not None:
+            B.vsa_decode_step_certified(shape, w.q, s, radii[i % distinct], w.k_cache, w.v_cache, w.block_table,
+                                        w.seq_lens, P, K_c, eps, tau, out, diag, cert, routed, flist, fcount, ws)
         elif solve is not None:
             B.vsa_decode_step_entropic(shape, w.q, s, w.k_cache, w.v_cache, w.block_table, w.seq_lens, P, K_c, eps,
                                        tau, args.solver_iters, out, diag, solve, routed, flist, fcount, ws)
@@ -362,7 +377,7 @@ def run_ours(args):
 
         # ---- with --solver-iters: the closed-form step timed the same way, for the cost of the iterations ----
         closed_form_us_per_layer = None
-        if solve is not None:
+        if solve is not None or cert is not None:
             def step_closed():
                 for i in range(L):
                     w, s = layers[i % distinct], summaries[i % distinct]
@@ -386,7 +401,7 @@ def run_ours(args):
 
         # ---- end to end: q from pinned host memory, out + diag back to the host, every layer ----
         e2e = None
-        if not args.dense_baseline and solve is None:
+        if not args.dense_baseline and solve is None and cert is None:
             q_host = [w.q.cpu().pin_memory() for w in layers]
             q_dev = torch.empty_like(w0.q)
             out_host = torch.empty(out.shape, dtype=torch.float32).pin_memory()
@@ -460,9 +475,9 @@ def run_ours(args):
         overhead = per_kernel["route_select"]
         roof = {"kernel": dom, "bytes_per_launch": alg[dom], "us_per_launch": per_kernel[dom] - overhead,
                 "us_event_interval": per_kernel[dom], "us_event_pair_overhead": overhead}
-        if solve is not None:
-            # the events bracket the closed-form kernels; the iterations' cost is the difference of the
-            # two graph-replayed steps and belongs to the sparse kernel
+        if solve is not None or cert is not None:
+            # the events bracket the plain step's kernels; the cost of the iterations (of the certificate)
+            # is the difference of the two graph-replayed steps and is booked on the sparse kernel
             extra = ms_per_step * 1e3 / L - closed_form_us_per_layer
             roof = {"kernel": "sparse_decode", "bytes_per_launch": alg["sparse_decode"],
                     "us_per_launch": per_kernel["sparse_decode"] - overhead + extra,
@@ -497,7 +512,8 @@ def run_ours(args):
                          f"{(scan_bytes + sparse_bytes) * distinct / 1e6:.0f} MB touched per pass over them",
                    "launch": "cuda graph replay of the whole step" if use_graph else "plain stream launches",
                    "path": "dense split-K baseline" if args.dense_baseline else
-                           ("route -> sparse -> dense fallback" if solve is None else
+                           ("route -> sparse with routing certificate -> dense fallback" if cert is not None else
+                            "route -> sparse -> dense fallback" if solve is None else
                             f"route -> sparse with {args.solver_iters} entropic mirror-descent iterations -> dense fallback")},
         "latency_us_per_layer": ms_per_step * 1e3 / L,
         "per_kernel_us": per_kernel, "closed_form_latency_us_per_layer": closed_form_us_per_layer,

@@ -98,6 +98,7 @@ typedef struct {
 #define VSA_WS_SPARSE 2
 #define VSA_WS_DENSE 3
 #define VSA_WS_STEP 4
+#define VSA_WS_STEP_CERTIFIED 5
 
 /*
  * Page summaries (Sec. 7 step 1: "coarse page summaries k_page"; the paper leaves them
@@ -210,6 +211,48 @@ int vsa_decode_step_entropic(const vsa_shape_t* shape, const void* q, const void
                              int32_t K_c, float epsilon, float gap_threshold, int32_t solver_iters, float* out,
                              vsa_diag_t* diag, vsa_solve_t* solve, int32_t* routed_pages, int32_t* fallback_list,
                              int32_t* fallback_count, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Routing certificate (App. E asks for "certificates" that the screened candidate set is the right
+ * one and for a fallback when they fail; it gives no construction - this one is the library's).
+ * Every page carries the radius of a ball around its stored summary mu that holds all its valid key
+ * rows, so no token of the page can score above  <q, mu> + |q| * radius.  The largest such bound
+ * over the pages that were NOT routed, together with the best rejected token of the routed pages,
+ * bounds every score outside the candidate set S:
+ *     delta_cert = s(1) - max(best rejected scored token, ub_unrouted)   (+INF if nothing is outside S),
+ * a true lower bound on the gap between s(1) and anything outside S, where diag.delta only sees the
+ * routed pages.  Cor. 1 with it gives leak_bound_cert >= the dense softmax mass outside S.
+ *
+ * vsa_build_page_radii: radii[page][kv_head] (device fp32 [num_pool_pages][n_kv_heads]) for the pages
+ * each sequence owns from first_page[b] on (NULL = all), from k_cache and the summaries already
+ * built for them: 1.001 * max_t |k_t - mu| + 2^-12 * |mu| in fp32 (the slack covers every rounding
+ * in the bound and in the scores it is compared with).  Cache maintenance, like the summaries.
+ *
+ * vsa_decode_step_certified: vsa_decode_step with the certificate computed in the same pass; the
+ * fallback decision becomes  !(delta_cert >= gap_threshold) && |S| < T  (the certified gap instead
+ * of diag.delta; diag.fallback and the fallback list follow it), everything else is unchanged.
+ *   cert: device vsa_cert_t [batch][n_q_heads].
+ *   ws: device scratch of vsa_workspace_bytes(shape, P, K_c, VSA_WS_STEP_CERTIFIED) bytes.
+ *   Shapes: max_pages_per_seq <= 8192 (16384 when batch * n_q_heads does not exceed the SM count),
+ *   VSA_ERR_UNSUPPORTED_SHAPE beyond.
+ */
+typedef struct {
+    float delta_cert;      /* certified gap, see above                                          */
+    float ub_unrouted;     /* best upper bound over the un-routed pages, -INF if all are routed */
+    float leak_bound_cert; /* min(1, (T - |S|) exp(-delta_cert / epsilon))                      */
+    int32_t certified;     /* delta_cert >= gap_threshold                                       */
+} vsa_cert_t;
+
+int vsa_build_page_radii(const vsa_shape_t* shape, const void* k_cache, const void* summaries,
+                         const int32_t* block_table, const int32_t* seq_lens, const int32_t* first_page,
+                         float* radii, void* stream);
+
+int vsa_decode_step_certified(const vsa_shape_t* shape, const void* q, const void* summaries, const float* radii,
+                              const void* k_cache, const void* v_cache, const int32_t* block_table,
+                              const int32_t* seq_lens, int32_t P, int32_t K_c, float epsilon, float gap_threshold,
+                              float* out, vsa_diag_t* diag, vsa_cert_t* cert, int32_t* routed_pages,
+                              int32_t* fallback_list, int32_t* fallback_count, void* ws, size_t ws_bytes,
+                              void* stream);
 
 /*
  * vsa_decode_step with CUDA events recorded on `stream` between its kernels, for per-kernel

@@ -16,7 +16,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libvsa.so")
 
-VSA_WS_ROUTE, VSA_WS_SPARSE, VSA_WS_DENSE, VSA_WS_STEP = 1, 2, 3, 4
+VSA_WS_ROUTE, VSA_WS_SPARSE, VSA_WS_DENSE, VSA_WS_STEP, VSA_WS_STEP_CERTIFIED = 1, 2, 3, 4, 5
 DIAG_BYTES = 32
 DIAG_FIELDS = ("delta", "delta12", "s_max", "lse", "leak_bound", "n_candidates", "fallback", "status")
 
@@ -77,6 +77,11 @@ def lib() -> C.CDLL:
                                                     vp, vp, vp]
         _lib.vsa_decode_step_entropic.argtypes = [shp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, i32, vp, vp, vp,
                                                   vp, vp, vp, vp, sz, vp]
+        _lib.vsa_build_page_radii.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp]
+        _lib.vsa_decode_step_certified.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, vp, vp, vp, vp,
+                                                   vp, vp, vp, sz, vp]
+        _lib.vsa_build_page_radii.restype = C.c_int
+        _lib.vsa_decode_step_certified.restype = C.c_int
         for name in ("vsa_build_page_summaries", "vsa_route_pages", "vsa_sparse_decode",
                      "vsa_dense_decode_fallback", "vsa_decode_step", "vsa_decode_step_timed",
                      "vsa_decode_step_host", "vsa_sparse_decode_entropic", "vsa_decode_step_entropic"):
@@ -203,6 +208,23 @@ def vsa_decode_step_entropic(shape, q, summaries, k_cache, v_cache, block_table,
            "vsa_decode_step_entropic")
 
 
+def vsa_build_page_radii(shape, k_cache, summaries, block_table, seq_lens, first_page, radii, stream=None) -> None:
+    _check(lib().vsa_build_page_radii(C.byref(shape), _ptr(k_cache), _ptr(summaries), _ptr(block_table),
+                                      _ptr(seq_lens), _ptr(first_page), _ptr(radii), _stream(stream)),
+           "vsa_build_page_radii")
+
+
+def vsa_decode_step_certified(shape, q, summaries, radii, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon,
+                              gap_threshold, out, diag, cert, routed_pages, fallback_list, fallback_count, ws,
+                              stream=None) -> None:
+    _check(lib().vsa_decode_step_certified(C.byref(shape), _ptr(q), _ptr(summaries), _ptr(radii), _ptr(k_cache),
+                                           _ptr(v_cache), _ptr(block_table), _ptr(seq_lens), P, K_c, epsilon,
+                                           gap_threshold, _ptr(out), _ptr(diag), _ptr(cert), _ptr(routed_pages),
+                                           _ptr(fallback_list), _ptr(fallback_count), _ptr(ws),
+                                           0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
+           "vsa_decode_step_certified")
+
+
 def vsa_decode_step_timed(shape, q, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon,
                           gap_threshold, out, diag, routed_pages, fallback_list, fallback_count, ws, events,
                           stream=None) -> None:
@@ -235,6 +257,21 @@ def vsa_decode_step_host(shape, q_host, q_dev, summaries, k_cache, v_cache, bloc
 def alloc_diag(units: int, device) -> torch.Tensor:
     """Device buffer for `units` vsa_diag_t records, viewed as int32 [units, 8]."""
     return torch.zeros((units, DIAG_BYTES // 4), dtype=torch.int32, device=device)
+
+
+CERT_FIELDS = ("delta_cert", "ub_unrouted", "leak_bound_cert", "certified")
+
+
+def alloc_cert(units: int, device) -> torch.Tensor:
+    """Device buffer for `units` vsa_cert_t records, viewed as int32 [units, 4] (see cert_to_dict)."""
+    return torch.zeros((units, 4), dtype=torch.int32, device=device)
+
+
+def cert_to_dict(cert: torch.Tensor) -> dict:
+    c = cert.detach().cpu()
+    out = {name: c[:, i].contiguous().view(torch.float32).clone() for i, name in enumerate(CERT_FIELDS[:3])}
+    out["certified"] = c[:, 3].clone()
+    return out
 
 
 SOLVE_FIELDS = ("fw_gap", "objective", "residual2", "step")

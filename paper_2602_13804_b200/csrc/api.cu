@@ -100,6 +100,10 @@ int check_epsilon(float epsilon)
 // step workspace = [ route scores | dense scratch ], each part 256-byte aligned
 size_t step_route_part(const Geometry& g) { return align_up(vsa::route_workspace_bytes(g), 256); }
 
+// certified step: [ route scores | dense scratch | page radii in logical order, fp32 [batch][n_kv_heads][max_pages] ]
+size_t step_rad_offset(const Geometry& g) { return step_route_part(g) + align_up(vsa::dense_workspace_bytes(g), 256); }
+size_t step_rad_bytes(const Geometry& g) { return (size_t)g.batch * g.n_kv_heads * g.max_pages * sizeof(float); }
+
 int cuda_rc(cudaError_t e) { return e == cudaSuccess ? VSA_OK : VSA_ERR_CUDA; }
 
 }  // namespace
@@ -132,6 +136,7 @@ size_t vsa_workspace_bytes(const vsa_shape_t* shape, int32_t P, int32_t K_c, int
         case VSA_WS_SPARSE: return 0;
         case VSA_WS_DENSE: return vsa::dense_workspace_bytes(g);
         case VSA_WS_STEP: return step_route_part(g) + vsa::dense_workspace_bytes(g);
+        case VSA_WS_STEP_CERTIFIED: return step_rad_offset(g) + step_rad_bytes(g);
         default: return 0;
     }
 }
@@ -146,6 +151,19 @@ int vsa_build_page_summaries(const vsa_shape_t* shape, const void* k_cache, cons
     if (!aligned16(k_cache) || !aligned16(summaries)) return VSA_ERR_MISALIGNED;
     return cuda_rc(vsa::launch_build_summaries(g, k_cache, block_table, seq_lens, first_page, summaries,
                                                (cudaStream_t)stream));
+}
+
+int vsa_build_page_radii(const vsa_shape_t* shape, const void* k_cache, const void* summaries,
+                         const int32_t* block_table, const int32_t* seq_lens, const int32_t* first_page,
+                         float* radii, void* stream)
+{
+    Geometry g;
+    int rc = make_geometry(shape, &g);
+    if (rc) return rc;
+    if (!k_cache || !summaries || !block_table || !seq_lens || !radii) return VSA_ERR_INVALID_ARGUMENT;
+    if (!aligned16(k_cache) || !aligned16(summaries)) return VSA_ERR_MISALIGNED;
+    return cuda_rc(vsa::launch_build_radii(g, k_cache, summaries, block_table, seq_lens, first_page, radii,
+                                           (cudaStream_t)stream));
 }
 
 int vsa_route_pages(const vsa_shape_t* shape, const void* q, const void* summaries, const int32_t* block_table,
@@ -235,7 +253,7 @@ static int decode_step_impl(const vsa_shape_t* shape, const void* q, const void*
                             int32_t K_c, float epsilon, float gap_threshold, float* out, vsa_diag_t* diag,
                             int32_t* routed_pages, int32_t* fallback_list, int32_t* fallback_count, void* ws,
                             size_t ws_bytes, void* stream, void* const* events, int solver_iters = 0,
-                            vsa_solve_t* solve = nullptr)
+                            vsa_solve_t* solve = nullptr, const float* radii = nullptr, vsa_cert_t* cert = nullptr)
 {
     Geometry g;
     int rc = make_geometry(shape, &g);
@@ -250,6 +268,14 @@ static int decode_step_impl(const vsa_shape_t* shape, const void* q, const void*
     if (!aligned16(q) || !aligned16(summaries) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(ws))
         return VSA_ERR_MISALIGNED;
     if (ws_bytes < step_route_part(g) + vsa::dense_workspace_bytes(g)) return VSA_ERR_WORKSPACE_TOO_SMALL;
+    float* rad_logical = nullptr;
+    if (cert) {
+        if (!radii) return VSA_ERR_INVALID_ARGUMENT;
+        if (g.max_pages > vsa::sparse_register_select_max_pages((long long)g.batch * g.n_q_heads))
+            return VSA_ERR_UNSUPPORTED_SHAPE;
+        if (ws_bytes < step_rad_offset(g) + step_rad_bytes(g)) return VSA_ERR_WORKSPACE_TOO_SMALL;
+        rad_logical = (float*)((char*)ws + step_rad_offset(g));
+    }
     cudaStream_t st = (cudaStream_t)stream;
     cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
     if (events)
@@ -261,13 +287,15 @@ static int decode_step_impl(const vsa_shape_t* shape, const void* q, const void*
     if (ev[0] && cudaEventRecord(ev[0], st) != cudaSuccess) return VSA_ERR_CUDA;
     // the scan kernel clears fallback_count and the dense pass's tickets: the step enqueues no memset
     cudaError_t e = vsa::launch_route_scan(g, q, summaries, block_table, seq_lens, ws, fallback_count,
-                                           vsa::dense_tickets(ws_dense), vsa::dense_ticket_count(g), st);
+                                           vsa::dense_tickets(ws_dense), vsa::dense_ticket_count(g), st,
+                                           cert ? radii : nullptr, rad_logical);
     if (e != cudaSuccess) return VSA_ERR_CUDA;
     if (ev[1] && cudaEventRecord(ev[1], st) != cudaSuccess) return VSA_ERR_CUDA;
     // the top-P selection runs inside the fused kernel, on the scores the scan left in ws
     if (ev[2] && cudaEventRecord(ev[2], st) != cudaSuccess) return VSA_ERR_CUDA;
     e = vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, routed_pages, (const float*)ws, P, K_c,
-                           epsilon, gap_threshold, out, diag, fallback_list, fallback_count, st, solver_iters, solve);
+                           epsilon, gap_threshold, out, diag, fallback_list, fallback_count, st, solver_iters, solve,
+                           rad_logical, cert);
     if (e != cudaSuccess) return VSA_ERR_CUDA;
     if (ev[3] && cudaEventRecord(ev[3], st) != cudaSuccess) return VSA_ERR_CUDA;
     e = vsa::launch_dense(g, q, k_cache, v_cache, block_table, seq_lens, fallback_list, fallback_count, epsilon,
@@ -298,6 +326,19 @@ int vsa_decode_step_entropic(const vsa_shape_t* shape, const void* q, const void
     return decode_step_impl(shape, q, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon,
                             gap_threshold, out, diag, routed_pages, fallback_list, fallback_count, ws, ws_bytes,
                             stream, nullptr, solver_iters, solve);
+}
+
+int vsa_decode_step_certified(const vsa_shape_t* shape, const void* q, const void* summaries, const float* radii,
+                              const void* k_cache, const void* v_cache, const int32_t* block_table,
+                              const int32_t* seq_lens, int32_t P, int32_t K_c, float epsilon, float gap_threshold,
+                              float* out, vsa_diag_t* diag, vsa_cert_t* cert, int32_t* routed_pages,
+                              int32_t* fallback_list, int32_t* fallback_count, void* ws, size_t ws_bytes,
+                              void* stream)
+{
+    if (!cert || !radii) return VSA_ERR_INVALID_ARGUMENT;
+    return decode_step_impl(shape, q, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon,
+                            gap_threshold, out, diag, routed_pages, fallback_list, fallback_count, ws, ws_bytes,
+                            stream, nullptr, 0, nullptr, radii, cert);
 }
 
 int vsa_decode_step_timed(const vsa_shape_t* shape, const void* q, const void* summaries, const void* k_cache,

@@ -29,7 +29,9 @@ struct ScanCfg {
     static constexpr int STAGES = 8192 / (ROUND_PAGES * kRowBytes) < 2 ? 2 : 8192 / (ROUND_PAGES * kRowBytes);
     static_assert((STAGES & (STAGES - 1)) == 0, "slot index is R & (STAGES - 1)");
     static constexpr int RING_BYTES = STAGES * ROUND_PAGES * kRowBytes;
-    static constexpr int WARP_BYTES = RING_BYTES + kMaxBlocksPerWarp * kBlockPages * 4;
+    static constexpr int TAB_BYTES = kMaxBlocksPerWarp * kBlockPages * 4;
+    static constexpr int RAD_BYTES = STAGES * ROUND_PAGES * 4;   // page radii of the rounds in flight (CERT)
+    static constexpr int WARP_BYTES = RING_BYTES + TAB_BYTES + RAD_BYTES;
 };
 
 __device__ __forceinline__ void cp_async_16(uint32_t smem_addr, const void* gptr)
@@ -53,12 +55,14 @@ __device__ __forceinline__ void cp_async_wait()
 // unpacked element; 16 (row, head) partials are reduced at once.  For G >= 2 lane c takes the
 // rows and the heads of a round in the order (r ^ c / G, h ^ c % G), which is what lets the
 // reduction run without per-lane selects (reduce_scatter16_xor).
-template <int G>
+// CERT: the radius of every page (radii[page][kv head], see radii_kernel) is copied into logical page
+// order, rad_logical[b][kv head][page], for the certificate that the fused kernel computes.
+template <int G, bool CERT>
 __global__ void __launch_bounds__(kScanThreads, 2)
 route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* __restrict__ summaries,
                   const int32_t* __restrict__ block_table, const int32_t* __restrict__ seq_lens,
                   float* __restrict__ scores, int blocks_per_warp, int32_t* zero_word, int32_t* zero_words,
-                  int zero_count)
+                  int zero_count, const float* __restrict__ radii, float* __restrict__ rad_logical)
 {
     using Cfg = ScanCfg<G>;
     constexpr int ROWS = Cfg::ROWS, VALS = Cfg::VALS, ROUND_PAGES = Cfg::ROUND_PAGES, STAGES = Cfg::STAGES;
@@ -148,6 +152,13 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
     const bool owns = VALS == 16 || c < 8;
     float* out_lane = scores + ((long long)b * geo.n_q_heads + g * G + own_h) * geo.max_pages + first_page +
                       gi * ROWS + own_r;
+    // CERT: the lane that owns (row, head 0) also moves the row's radius
+    const bool rad_lane = CERT && owns && own_h == 0;
+    float* rad_ring = (float*)(my_smem + Cfg::RING_BYTES + Cfg::TAB_BYTES);
+    const uint32_t rad_ring_s = (uint32_t)__cvta_generic_to_shared(rad_ring);
+    float* rad_out = nullptr;
+    if constexpr (CERT)
+        rad_out = rad_logical + ((long long)b * geo.n_kv_heads + g) * geo.max_pages + first_page + gi * ROWS + own_r;
 
     // rows without a valid page read row 0 of the pool instead (their result is never stored)
     auto issue = [&](int R) {
@@ -156,6 +167,14 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
 #pragma unroll
         for (int r = 0; r < ROWS; ++r)
             cp_async_16(dst + r * kRowBytes, srow + (long long)max(tab[tab_row[r]], 0) * 16);
+        if constexpr (CERT) {
+            if (rad_lane) {
+                // off / 16 = page * n_kv_heads: the row of this page in radii[][n_kv_heads]
+                const int off = max(tab[gi * ROWS + own_r], 0);
+                cp_async_4(rad_ring_s + 4u * (uint32_t)((R & (STAGES - 1)) * ROUND_PAGES + gi * ROWS + own_r),
+                           radii + (off >> 4) + g);
+            }
+        }
     };
 
     VSA_PROBE(11);
@@ -190,6 +209,11 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
         }
         const int pl = R * ROUND_PAGES + gi * ROWS + own_r;
         if (owns && pl < n_pages) out_lane[R * ROUND_PAGES] = off_tab[pl] >= 0 ? s : -INFINITY;
+        if constexpr (CERT) {
+            if (rad_lane && pl < n_pages)
+                rad_out[R * ROUND_PAGES] =
+                    off_tab[pl] >= 0 ? rad_ring[(R & (STAGES - 1)) * ROUND_PAGES + gi * ROWS + own_r] : 0.0f;
+        }
     }
     VSA_PROBE(14);
     VSA_PROBE_TMAX(49);
@@ -247,10 +271,10 @@ int scan_blocks_per_warp(const Geometry& g)
     return (int)k;
 }
 
-template <int G>
+template <int G, bool CERT>
 cudaError_t launch_scan_g(const Geometry& g, const uint16_t* q, const uint16_t* summaries, const int32_t* block_table,
                           const int32_t* seq_lens, float* scores, int32_t* zero_word, int32_t* zero_words,
-                          int zero_count, cudaStream_t stream)
+                          int zero_count, const float* radii, float* rad_logical, cudaStream_t stream)
 {
     const int bpw = scan_blocks_per_warp(g);
     const int slices = ((g.max_pages + kBlockPages - 1) / kBlockPages + bpw - 1) / bpw;
@@ -262,12 +286,12 @@ cudaError_t launch_scan_g(const Geometry& g, const uint16_t* q, const uint16_t* 
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (attr_device != dev) {
-        e = cudaFuncSetAttribute(route_scan_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        e = cudaFuncSetAttribute(route_scan_kernel<G, CERT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         attr_device = dev;
     }
-    return launch_pdl(route_scan_kernel<G>, grid, dim3(kScanThreads), smem, stream, g, q, summaries, block_table,
-                      seq_lens, scores, bpw, zero_word, zero_words, zero_count);
+    return launch_pdl(route_scan_kernel<G, CERT>, grid, dim3(kScanThreads), smem, stream, g, q, summaries,
+                      block_table, seq_lens, scores, bpw, zero_word, zero_words, zero_count, radii, rad_logical);
 }
 
 }  // namespace
@@ -279,18 +303,25 @@ size_t route_workspace_bytes(const Geometry& g)
 
 cudaError_t launch_route_scan(const Geometry& g, const void* q, const void* summaries, const int32_t* block_table,
                               const int32_t* seq_lens, void* ws, int32_t* zero_word, int32_t* zero_words,
-                              int zero_count, cudaStream_t stream)
+                              int zero_count, cudaStream_t stream, const float* radii, float* rad_logical)
 {
     float* scores = (float*)ws;
     const uint16_t* qq = (const uint16_t*)q;
     const uint16_t* ss = (const uint16_t*)summaries;
+#define VSA_SCAN_CASE(G)                                                                                       \
+    case G:                                                                                                    \
+        return radii ? launch_scan_g<G, true>(g, qq, ss, block_table, seq_lens, scores, zero_word, zero_words, \
+                                              zero_count, radii, rad_logical, stream)                          \
+                     : launch_scan_g<G, false>(g, qq, ss, block_table, seq_lens, scores, zero_word, zero_words, \
+                                               zero_count, nullptr, nullptr, stream);
     switch (g.group) {
-        case 1: return launch_scan_g<1>(g, qq, ss, block_table, seq_lens, scores, zero_word, zero_words, zero_count, stream);
-        case 2: return launch_scan_g<2>(g, qq, ss, block_table, seq_lens, scores, zero_word, zero_words, zero_count, stream);
-        case 4: return launch_scan_g<4>(g, qq, ss, block_table, seq_lens, scores, zero_word, zero_words, zero_count, stream);
-        case 8: return launch_scan_g<8>(g, qq, ss, block_table, seq_lens, scores, zero_word, zero_words, zero_count, stream);
+        VSA_SCAN_CASE(1)
+        VSA_SCAN_CASE(2)
+        VSA_SCAN_CASE(4)
+        VSA_SCAN_CASE(8)
         default: return cudaErrorInvalidValue;
     }
+#undef VSA_SCAN_CASE
 }
 
 cudaError_t launch_route_select(const Geometry& g, const void* ws, const int32_t* seq_lens, int P,

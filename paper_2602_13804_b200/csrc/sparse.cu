@@ -98,17 +98,22 @@ __device__ __forceinline__ void write_failed_unit(float* out, vsa_diag_t* diag, 
 // TOK_KPT: token scores per thread, P * 16 <= TOK_KPT * THREADS.
 // SOLVE: the weights on the candidates come from `solver_iters` entropic mirror-descent iterations
 //   (256 threads only: every lane owns one candidate, every half-warp sixteen candidate rows).
-template <int THREADS, int PAGE_KPT, int TOK_KPT, bool SOLVE = false>
+// CERT (fused register variants only): the certified gap of the unit - an upper bound on every score
+//   of the pages that were not routed, from the pages' radii (rad_logical, written by the scan) -
+//   is computed, reported in cert[] and used for the fallback decision in place of the proxy gap.
+template <int THREADS, int PAGE_KPT, int TOK_KPT, bool SOLVE = false, bool CERT = false>
 __global__ void __launch_bounds__(THREADS, 512 / THREADS)
 sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* __restrict__ k_cache,
                      const uint16_t* __restrict__ v_cache, const int32_t* __restrict__ block_table,
                      const int32_t* __restrict__ seq_lens, int32_t* __restrict__ routed_pages,
                      const float* __restrict__ page_scores, int P, int K_c, float epsilon, float gap_threshold,
                      float* __restrict__ out, vsa_diag_t* __restrict__ diag, int32_t* __restrict__ fallback_list,
-                     int32_t* __restrict__ fallback_count, int solver_iters, vsa_solve_t* __restrict__ solve)
+                     int32_t* __restrict__ fallback_count, int solver_iters, vsa_solve_t* __restrict__ solve,
+                     const float* __restrict__ rad_logical, vsa_cert_t* __restrict__ cert)
 {
     constexpr int WARPS = THREADS / 32, GROUPS = 2 * WARPS;
     static_assert(!SOLVE || THREADS == 256, "the solve maps one candidate to each of 256 lanes");
+    static_assert(!CERT || PAGE_KPT > 0, "the certificate needs every page score of the unit in registers");
     static_assert(TOK_KPT * WARPS <= 64 && 4 * WARPS <= 72, "wred capacity");
     extern __shared__ uint32_t smem_raw[];
     int32_t* page_l = (int32_t*)smem_raw;   // [P] routed logical pages, ascending, invalid entries last
@@ -144,10 +149,21 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
             praw[j] = i < geo.max_pages ? ld_cg_f32(page_scores + unit * geo.max_pages + i) : 0.0f;
         }
     }
+    float prad[CERT ? PAGE_KPT : 1];
+    if constexpr (CERT) {
+#pragma unroll
+        for (int j = 0; j < PAGE_KPT; ++j) {
+            const int i = tid + j * THREADS;
+            prad[j] = i < geo.max_pages
+                          ? ld_cg_f32(rad_logical + ((long long)b * geo.n_kv_heads + g) * geo.max_pages + i)
+                          : 0.0f;
+        }
+    }
     if (T <= 0 || T > geo.max_pages * kPageSize) {
         cp_async_wait_all();
         write_failed_unit(out, diag, unit, VSA_UNIT_BAD_LENGTH);
         if (SOLVE && tid == 0) solve[unit] = vsa_solve_t{0.0f, 0.0f, 0.0f, 0.0f};
+        if (CERT && tid == 0) cert[unit] = vsa_cert_t{0.0f, 0.0f, 0.0f, 0};
         if (PAGE_KPT != 0)
             for (int t = tid; t < P; t += THREADS) routed_pages[unit * P + t] = -1;
         return;
@@ -166,6 +182,29 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
             for (int j = 0; j < PAGE_KPT; ++j) pkey[j] = tid + j * THREADS < nb ? float_to_key(praw[j]) : 0u;
             cp_async_wait_all();   // this thread's part of the block-table copy; the selection's barriers publish it
             np = select_top_pages_keys<PAGE_KPT>(pkey, nb, P, ps);
+            if constexpr (CERT) {
+                // |q| (rounded up a little), every lane of a half-warp computing the same value
+                float qe[8];
+                unpack8(qraw, qe);
+                float q2 = chunk_partial(qe, qe);
+#pragma unroll
+                for (int off = 8; off; off >>= 1) q2 = q2 + __shfl_xor_sync(kFullMask, q2, off);
+                const float qn = __fmul_rn(__fsqrt_rn(q2), 1.00000095367431640625f);
+                // a page is un-routed iff it is ordered after the last winner (score descending, index
+                // ascending); its tokens score at most  c + |q| * radius
+                const uint32_t k_last = ps.win_key[np - 1];
+                const int i_last = ps.win_idx[np - 1];
+                uint32_t ub_key = 0u;
+#pragma unroll
+                for (int j = 0; j < PAGE_KPT; ++j) {
+                    const int i = tid + j * THREADS;
+                    const bool unrouted = pkey[j] != 0u && ((pkey[j] < k_last) | ((pkey[j] == k_last) & (i > i_last)));
+                    if (unrouted)
+                        ub_key = max(ub_key, float_to_key(__fadd_rn(key_to_float(pkey[j]), __fmul_rn(qn, prad[j]))));
+                }
+                ub_key = __reduce_max_sync(kFullMask, ub_key);
+                if (lane == 0) ps.ts.wred[warp] = ub_key;   // published by the barrier below, read right after it
+            }
         } else {
             np = select_top_pages(page_scores + unit * geo.max_pages, nb, P, ps);
         }
@@ -210,9 +249,18 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         np = __syncthreads_count(tid < P && raw[tid < P ? tid : 0] != INT_MAX);
     }
     VSA_PROBE(1);
-    if (__syncthreads_or(bad)) {
+    const int any_bad = __syncthreads_or(bad);
+    uint32_t ub_unrouted_key = 0u;   // CERT: key of the best upper bound over the un-routed pages, 0 = none
+    if constexpr (CERT) {
+        const PageSelectSmem ps = carve_page_select(region, geo.max_pages, P);
+#pragma unroll
+        for (int w = 0; w < WARPS; ++w) ub_unrouted_key = max(ub_unrouted_key, ps.ts.wred[w]);
+        __syncthreads();   // the selection scratch is rewritten by the token phase
+    }
+    if (any_bad) {
         write_failed_unit(out, diag, unit, VSA_UNIT_BAD_PAGE);
         if (SOLVE && tid == 0) solve[unit] = vsa_solve_t{0.0f, 0.0f, 0.0f, 0.0f};
+        if (CERT && tid == 0) cert[unit] = vsa_cert_t{0.0f, 0.0f, 0.0f, 0};
         return;
     }
     const TokenSmem sm = carve_tokens(region, P, K_c);
@@ -595,6 +643,18 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         d.leak_bound = fminf(1.0f, (float)(T - ns) * expf(-delta / epsilon));
         d.n_candidates = ns;
         d.fallback = (delta < gap_threshold && ns < T) ? 1 : 0;
+        if constexpr (CERT) {
+            const float ub = ub_unrouted_key != 0u ? key_to_float(ub_unrouted_key) : -INFINITY;
+            const float rej = has_rejected ? key_to_float(out_key) : -INFINITY;
+            const float m = fmaxf(rej, ub);
+            vsa_cert_t ce;
+            ce.ub_unrouted = ub;
+            ce.delta_cert = m == -INFINITY ? INFINITY : s1 - m;
+            ce.certified = ce.delta_cert >= gap_threshold ? 1 : 0;
+            ce.leak_bound_cert = fminf(1.0f, (float)(T - ns) * expf(-ce.delta_cert / epsilon));
+            cert[unit] = ce;
+            d.fallback = (!ce.certified && ns < T) ? 1 : 0;   // the certified gap decides
+        }
         d.status = 0;
         diag[unit] = d;
         if (d.fallback) fallback_list[atomicAdd(fallback_count, 1)] = (int32_t)unit;
@@ -628,31 +688,38 @@ struct SparseArgs {
     int32_t *fallback_list, *fallback_count;
     int solver_iters;
     vsa_solve_t* solve;   // non-null: the iterative-solve variant of the kernel
+    const float* rad_logical;
+    vsa_cert_t* cert;     // non-null: the certificate variant (fused register variants only)
     cudaStream_t stream;
 };
 
-template <int THREADS, int PAGE_KPT, int TOK_KPT, bool SOLVE>
+template <int THREADS, int PAGE_KPT, int TOK_KPT, bool SOLVE, bool CERT>
 cudaError_t launch_variant(const SparseArgs& a)
 {
     if (a.smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(sparse_decode_kernel<THREADS, PAGE_KPT, TOK_KPT, SOLVE>,
+        cudaError_t e = cudaFuncSetAttribute(sparse_decode_kernel<THREADS, PAGE_KPT, TOK_KPT, SOLVE, CERT>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)a.smem);
         if (e != cudaSuccess) return e;
     }
     const unsigned units = (unsigned)(a.g.batch * a.g.n_q_heads);
-    return launch_pdl(sparse_decode_kernel<THREADS, PAGE_KPT, TOK_KPT, SOLVE>, dim3(units), dim3(THREADS), a.smem,
-                      a.stream, a.g, a.q, a.k, a.v, a.block_table, a.seq_lens, a.routed_pages, a.page_scores, a.P,
-                      a.K_c, a.epsilon, a.gap_threshold, a.out, a.diag, a.fallback_list, a.fallback_count,
-                      a.solver_iters, a.solve);
+    return launch_pdl(sparse_decode_kernel<THREADS, PAGE_KPT, TOK_KPT, SOLVE, CERT>, dim3(units), dim3(THREADS),
+                      a.smem, a.stream, a.g, a.q, a.k, a.v, a.block_table, a.seq_lens, a.routed_pages, a.page_scores,
+                      a.P, a.K_c, a.epsilon, a.gap_threshold, a.out, a.diag, a.fallback_list, a.fallback_count,
+                      a.solver_iters, a.solve, a.rad_logical, a.cert);
 }
 
 template <int THREADS, int PAGE_KPT, int TOK_KPT>
 cudaError_t launch_one(const SparseArgs& a)
 {
     if constexpr (THREADS == 256) {
-        if (a.solve) return launch_variant<THREADS, PAGE_KPT, TOK_KPT, true>(a);
+        if (a.solve) return launch_variant<THREADS, PAGE_KPT, TOK_KPT, true, false>(a);
     }
-    return launch_variant<THREADS, PAGE_KPT, TOK_KPT, false>(a);
+    if constexpr (PAGE_KPT > 0) {
+        if (a.cert) return launch_variant<THREADS, PAGE_KPT, TOK_KPT, false, true>(a);
+    } else {
+        if (a.cert) return cudaErrorInvalidValue;   // (refused by the entry point before any launch)
+    }
+    return launch_variant<THREADS, PAGE_KPT, TOK_KPT, false, false>(a);
 }
 
 template <int THREADS, int PAGE_KPT>
@@ -700,11 +767,13 @@ extern "C" int vsa_probe_read(long long* host64)
 }
 #endif
 
+int sparse_register_select_max_pages(long long units) { return 32 * (units <= sm_count() ? 512 : 256); }
+
 cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache, const void* v_cache,
                           const int32_t* block_table, const int32_t* seq_lens, int32_t* routed_pages,
                           const float* page_scores, int P, int K_c, float epsilon, float gap_threshold, float* out,
                           vsa_diag_t* diag, int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream,
-                          int solver_iters, vsa_solve_t* solve)
+                          int solver_iters, vsa_solve_t* solve, const float* rad_logical, vsa_cert_t* cert)
 {
     SparseArgs a;
     a.g = g;
@@ -714,6 +783,8 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
     a.smem = sparse_smem_bytes(g, P, K_c, page_scores != nullptr, threads, solve != nullptr);
     a.solver_iters = solver_iters;
     a.solve = solve;
+    a.rad_logical = rad_logical;
+    a.cert = cert;
     a.q = (const uint16_t*)q;
     a.k = (const uint16_t*)k_cache;
     a.v = (const uint16_t*)v_cache;

@@ -57,6 +57,71 @@ __global__ void __launch_bounds__(256) summaries_kernel(Geometry geo, const uint
     *reinterpret_cast<uint4*>(summaries + (p * geo.n_kv_heads + g) * kHeadDim + c * 8) = o;
 }
 
+// Radius of each page around its stored summary (the ball bound of the routing certificate):
+//   rhat = 1.001 * sqrt(max_t |k_t - mu|^2) + 2^-12 * |mu|,
+// squared norms summed in the library's canonical order, every operation a single rounded fp32
+// operation so that the CPU oracle reproduces the value bit for bit.  Same thread mapping as the
+// summaries kernel; the 16 threads of a (page, head) form a half-warp and only talk to each other.
+__global__ void __launch_bounds__(256) radii_kernel(Geometry geo, const uint16_t* __restrict__ k_cache,
+                                                    const uint16_t* __restrict__ summaries,
+                                                    const int32_t* __restrict__ block_table,
+                                                    const int32_t* __restrict__ seq_lens,
+                                                    const int32_t* __restrict__ first_page,
+                                                    float* __restrict__ radii)
+{
+    const int b = blockIdx.y;
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const int c = (int)(idx & 15);
+    const int g = (int)((idx >> 4) % geo.n_kv_heads);
+    const long long l = (idx >> 4) / geo.n_kv_heads;
+    const int T = seq_lens[b];
+    if (T <= 0 || T > geo.max_pages * kPageSize) return;
+    const int nb = (T + kPageSize - 1) / kPageSize;
+    const int l0 = first_page ? first_page[b] : 0;
+    if (l < l0 || l >= nb) return;
+    const long long p = block_table[(long long)b * geo.max_pages + l];
+    if (p < 0 || p >= geo.pool_pages) return;
+    const int n = min(kPageSize, T - (int)l * kPageSize);
+    const unsigned hmask = 0xffffu << (threadIdx.x & 16);   // this half-warp (the other may have returned)
+
+    float mu[8];
+    unpack8(*reinterpret_cast<const uint4*>(summaries + (p * geo.n_kv_heads + g) * kHeadDim + c * 8), mu);
+    const uint16_t* src = k_cache + p * geo.page_stride + (long long)g * geo.head_stride + c * 8;
+    uint4 rows[kPageSize];
+#pragma unroll
+    for (int t = 0; t < kPageSize; ++t)
+        rows[t] = t < n ? ld_nc_16B(src + (long long)t * geo.token_stride) : make_uint4(0u, 0u, 0u, 0u);
+    float vals[16];
+#pragma unroll
+    for (int t = 0; t < kPageSize; ++t) {
+        float f[8], d[8];
+        unpack8(rows[t], f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) d[e] = __fsub_rn(f[e], mu[e]);
+        vals[t] = t < n ? chunk_partial(d, d) : 0.0f;
+    }
+    float d2 = reduce_scatter16(vals, c, hmask);   // lane t: |k_t - mu|^2, 0 for absent rows
+#pragma unroll
+    for (int off = 8; off; off >>= 1) d2 = fmaxf(d2, __shfl_xor_sync(hmask, d2, off));
+    float m2 = chunk_partial(mu, mu);
+#pragma unroll
+    for (int off = 8; off; off >>= 1) m2 = m2 + __shfl_xor_sync(hmask, m2, off);
+    if (c == 0)
+        radii[p * geo.n_kv_heads + g] =
+            __fadd_rn(__fmul_rn(__fsqrt_rn(d2), 1.001f), __fmul_rn(__fsqrt_rn(m2), 0x1p-12f));
+}
+
+cudaError_t launch_build_radii(const Geometry& g, const void* k_cache, const void* summaries,
+                               const int32_t* block_table, const int32_t* seq_lens, const int32_t* first_page,
+                               float* radii, cudaStream_t stream)
+{
+    const long long threads = (long long)g.max_pages * g.n_kv_heads * 16;
+    dim3 grid((unsigned)((threads + 255) / 256), (unsigned)g.batch);
+    radii_kernel<<<grid, 256, 0, stream>>>(g, (const uint16_t*)k_cache, (const uint16_t*)summaries, block_table,
+                                           seq_lens, first_page, radii);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_build_summaries(const Geometry& g, const void* k_cache, const int32_t* block_table,
                                    const int32_t* seq_lens, const int32_t* first_page, void* summaries,
                                    cudaStream_t stream)

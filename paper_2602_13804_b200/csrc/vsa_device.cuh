@@ -171,8 +171,9 @@ __device__ __forceinline__ float reduce_scatter16_xor(float (&v)[16])
 // ("reduce-scatter"): on entry v[i] is this lane's partial of value i, on return lane c
 // (0..15 within its half-warp) holds the complete sum of value c.  For each value the
 // additions are exactly p[c] += p[c+off] for off = 8, 4, 2, 1 (addition is commutative, so
-// which lane of a pair performs it does not change a bit).  15 shuffles for 16 values.
-__device__ __forceinline__ float reduce_scatter16(float (&v)[16], int c)
+// which lane of a pair performs it does not change a bit).  15 shuffles for 16 values.  `mask` names
+// the lanes that take part (the whole warp, or one half-warp when the other may have exited).
+__device__ __forceinline__ float reduce_scatter16(float (&v)[16], int c, unsigned mask = kFullMask)
 {
     {
         const bool hi = c & 8;
@@ -180,7 +181,7 @@ __device__ __forceinline__ float reduce_scatter16(float (&v)[16], int c)
         for (int i = 0; i < 8; ++i) {
             const float send = hi ? v[i] : v[i + 8];
             const float keep = hi ? v[i + 8] : v[i];
-            v[i] = keep + __shfl_xor_sync(kFullMask, send, 8);
+            v[i] = keep + __shfl_xor_sync(mask, send, 8);
         }
     }
     {
@@ -189,7 +190,7 @@ __device__ __forceinline__ float reduce_scatter16(float (&v)[16], int c)
         for (int i = 0; i < 4; ++i) {
             const float send = hi ? v[i] : v[i + 4];
             const float keep = hi ? v[i + 4] : v[i];
-            v[i] = keep + __shfl_xor_sync(kFullMask, send, 4);
+            v[i] = keep + __shfl_xor_sync(mask, send, 4);
         }
     }
     {
@@ -198,14 +199,14 @@ __device__ __forceinline__ float reduce_scatter16(float (&v)[16], int c)
         for (int i = 0; i < 2; ++i) {
             const float send = hi ? v[i] : v[i + 2];
             const float keep = hi ? v[i + 2] : v[i];
-            v[i] = keep + __shfl_xor_sync(kFullMask, send, 2);
+            v[i] = keep + __shfl_xor_sync(mask, send, 2);
         }
     }
     {
         const bool hi = c & 1;
         const float send = hi ? v[0] : v[1];
         const float keep = hi ? v[1] : v[0];
-        v[0] = keep + __shfl_xor_sync(kFullMask, send, 1);
+        v[0] = keep + __shfl_xor_sync(mask, send, 1);
     }
     return v[0];
 }

@@ -41,24 +41,35 @@ cudaError_t launch_build_summaries(const Geometry& g, const void* k_cache, const
                                    const int32_t* seq_lens, const int32_t* first_page, void* summaries,
                                    cudaStream_t stream);
 
+cudaError_t launch_build_radii(const Geometry& g, const void* k_cache, const void* summaries,
+                               const int32_t* block_table, const int32_t* seq_lens, const int32_t* first_page,
+                               float* radii, cudaStream_t stream);
+
 // ---- page routing ---------------------------------------------------------------------------
 size_t route_workspace_bytes(const Geometry& g);
 // zero_word (one int) and zero_words[0..zero_count) are cleared by the scan kernel when not null
+// radii != nullptr: the pages' radii are also copied into logical page order, rad_logical[b][kv head][page]
 cudaError_t launch_route_scan(const Geometry& g, const void* q, const void* summaries, const int32_t* block_table,
                               const int32_t* seq_lens, void* ws, int32_t* zero_word, int32_t* zero_words,
-                              int zero_count, cudaStream_t stream);
+                              int zero_count, cudaStream_t stream, const float* radii = nullptr,
+                              float* rad_logical = nullptr);
 cudaError_t launch_route_select(const Geometry& g, const void* ws, const int32_t* seq_lens, int P,
                                 int32_t* routed_pages, float* routed_scores, cudaStream_t stream);
 
 // ---- fused sparse pass ------------------------------------------------------------------------
 // page_scores == nullptr: routed_pages is read; otherwise the top-P selection runs inside the kernel on
 // page_scores (the scan's output) and routed_pages is written.  solve != nullptr: the weights on the
-// candidates come from solver_iters entropic mirror-descent iterations (K_c <= 256).
+// candidates come from solver_iters entropic mirror-descent iterations (K_c <= 256).  cert != nullptr
+// (with page_scores and rad_logical): the certified gap is computed and decides the fallback.
 cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache, const void* v_cache,
                           const int32_t* block_table, const int32_t* seq_lens, int32_t* routed_pages,
                           const float* page_scores, int P, int K_c, float epsilon, float gap_threshold, float* out,
                           vsa_diag_t* diag, int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream,
-                          int solver_iters = 0, vsa_solve_t* solve = nullptr);
+                          int solver_iters = 0, vsa_solve_t* solve = nullptr, const float* rad_logical = nullptr,
+                          vsa_cert_t* cert = nullptr);
+// widest block table for which the fused kernel keeps every page score of a unit in registers (the
+// certificate variant exists for those shapes only); `units` = batch * n_q_heads
+int sparse_register_select_max_pages(long long units);
 
 // ---- dense split-K pass -------------------------------------------------------------------------
 size_t dense_workspace_bytes(const Geometry& g);

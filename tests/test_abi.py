@@ -129,6 +129,29 @@ def test_entropic_argument_validation(lib):
     assert C.sizeof(C.c_float) * len(B.SOLVE_FIELDS) == 16
 
 
+def test_certificate_argument_validation(lib):
+    ok = B.make_shape(2, 8, 2, 64, 256)
+    s = C.byref(ok)
+    r = lib.vsa_build_page_radii
+    assert r(s, None, FAKE, FAKE, FAKE, None, FAKE, None) == -1
+    assert r(s, FAKE, FAKE, FAKE, FAKE, None, None, None) == -1
+    assert r(s, ODD, FAKE, FAKE, FAKE, None, FAKE, None) == -4
+    step = lib.vsa_decode_step_certified
+
+    def call(shape=ok, radii=FAKE, cert=FAKE, ws_bytes=1 << 40, P=4, K_c=16):
+        return step(C.byref(shape), FAKE, FAKE, radii, FAKE, FAKE, FAKE, FAKE, P, K_c, 1.0, 0.0, FAKE, FAKE, cert, FAKE,
+                    FAKE, FAKE, FAKE, ws_bytes, None)
+
+    assert call(radii=None) == -1 and call(cert=None) == -1
+    plain = B.vsa_workspace_bytes(ok, 4, 16, B.VSA_WS_STEP)
+    need = B.vsa_workspace_bytes(ok, 4, 16, B.VSA_WS_STEP_CERTIFIED)
+    assert need >= plain + 2 * 2 * 64 * 4            # + one fp32 radius per (sequence, kv head, logical page)
+    assert call(ws_bytes=plain) == -3
+    wide = B.make_shape(40, 8, 2, 9000, 1 << 16)     # 320 units > SMs: 256 threads hold at most 8192 page scores
+    assert call(shape=wide) == -2
+    assert C.sizeof(C.c_int32) * len(B.CERT_FIELDS) == 16
+
+
 def test_dense_and_step_argument_validation(lib):
     ok = B.make_shape(2, 8, 2, 64, 256)
     s = C.byref(ok)

@@ -1,0 +1,137 @@
+"""GPU parity of the routing certificate (vsa_build_page_radii / vsa_decode_step_certified) against the
+oracle on the same seeded bytes.  Radii, the bound over the un-routed pages, the certified gap and the
+certified flag - which decides the fallback - are single-rounded fp32 arithmetic in a fixed order and
+must match bit for bit; leak_bound_cert is an fp32 exponential compared with a relative tolerance."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2602_13804_b200 import binding as B
+from gpu_runner import check_out
+from util import geometry, host_arrays
+from workloads import WorkloadSpec, make_workload
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def spec(**kw):
+    base = dict(name="t", config=9, batch=3, n_q_heads=8, n_kv_heads=2, P=4, K_c=40,
+                seq_lens=(700, 333, 90), needles=3, needle_positions="uniform")
+    base.update(kw)
+    return WorkloadSpec(**base)
+
+
+def run_certified(w):
+    wd = w.to(DEV)
+    shape = B.shape_of(wd.q, wd.k_cache, wd.block_table)
+    units = shape.batch * shape.n_q_heads
+    P, K_c = w.spec.P, w.spec.K_c
+    summ = torch.zeros((shape.num_pool_pages, shape.n_kv_heads, 128), dtype=torch.bfloat16, device=DEV)
+    B.vsa_build_page_summaries(shape, wd.k_cache, wd.block_table, wd.seq_lens, None, summ)
+    radii = torch.full((shape.num_pool_pages, shape.n_kv_heads), -1.0, dtype=torch.float32, device=DEV)
+    B.vsa_build_page_radii(shape, wd.k_cache, summ, wd.block_table, wd.seq_lens, None, radii)
+    out = torch.full((shape.batch, shape.n_q_heads, 128), float("nan"), dtype=torch.float32, device=DEV)
+    diag, cert = B.alloc_diag(units, DEV), B.alloc_cert(units, DEV)
+    flist = torch.full((units,), -1, dtype=torch.int32, device=DEV)
+    fcount = torch.full((1,), 99, dtype=torch.int32, device=DEV)
+    routed = torch.full((shape.batch, shape.n_q_heads, P), -7, dtype=torch.int32, device=DEV)
+    ws = B.alloc_workspace(shape, P, K_c, B.VSA_WS_STEP_CERTIFIED, DEV)
+    B.vsa_decode_step_certified(shape, wd.q, summ, radii, wd.k_cache, wd.v_cache, wd.block_table, wd.seq_lens, P, K_c,
+                                w.epsilon, w.gap_threshold, out, diag, cert, routed, flist, fcount, ws)
+    torch.cuda.synchronize()
+    n = int(fcount.item())
+    return dict(out=out.cpu().numpy(), diag={k: v.numpy() for k, v in B.diag_to_dict(diag).items()},
+                cert={k: v.numpy() for k, v in B.cert_to_dict(cert).items()}, radii=radii.cpu().numpy(),
+                routed=routed.cpu().numpy(), fallback=np.sort(flist[:n].cpu().numpy()))
+
+
+def compare_certified(w, g):
+    q, K, V, bt, sl = host_arrays(w)
+    geo = geometry(w)
+    Bn, H = geo.batch, geo.n_q_heads
+    summ = oracle.build_summaries(geo, K, bt, sl)
+    rad = oracle.build_radii(geo, K, summ, bt, sl)
+    owned = np.concatenate([bt[b, : (int(sl[b]) + 15) // 16] for b in range(Bn)])
+    assert np.array_equal(g["radii"][owned].view(np.uint32), rad[owned].view(np.uint32)), "radii differ"
+    untouched = np.ones(geo.num_pool_pages, bool)
+    untouched[owned] = False
+    assert np.all(g["radii"][untouched] == -1.0)
+    rt = oracle.route(geo, q, summ, bt, sl, w.spec.P, want_all_scores=True)
+    assert np.array_equal(g["routed"], rt.pages)
+    sp = oracle.sparse(geo, q, K, V, bt, sl, rt.pages, w.spec.K_c, w.epsilon, w.gap_threshold)
+    ce = oracle.certify(geo, q, rad, bt, sl, rt, sp, w.epsilon, w.gap_threshold)
+    c = g["cert"]
+    assert np.array_equal(c["ub_unrouted"].reshape(Bn, H).view(np.uint32), ce.ub_unrouted.view(np.uint32)), "bounds differ"
+    assert np.array_equal(c["delta_cert"].reshape(Bn, H).view(np.uint32), ce.delta_cert.view(np.uint32)), "gaps differ"
+    assert np.array_equal(c["certified"].reshape(Bn, H), ce.certified)
+    lb = c["leak_bound_cert"].reshape(Bn, H).astype(np.float64)
+    assert np.all(np.abs(lb - ce.leak_cert) <= 1e-3 * ce.leak_cert + 1e-37)
+    # the certified gap decides the fallback; the other diagnostics are those of the plain step
+    want_fb = ((ce.certified == 0) & (sp.n_candidates < sl[:, None])).astype(np.int32)
+    d = g["diag"]
+    assert np.array_equal(d["fallback"].reshape(Bn, H), want_fb)
+    assert np.array_equal(g["fallback"], np.nonzero(want_fb.reshape(-1))[0])
+    for name, want in (("delta", sp.delta), ("delta12", sp.delta12), ("s_max", sp.s_max)):
+        assert np.array_equal(d[name].reshape(Bn, H), want), name
+    assert np.array_equal(d["n_candidates"].reshape(Bn, H), sp.n_candidates)
+    # outputs: sparse rows where certified, dense rows where the unit fell back
+    flat = want_fb.reshape(-1).astype(bool)
+    out = g["out"].reshape(Bn * H, -1)
+    if (~flat).any():
+        check_out(out[~flat], sp.out.reshape(Bn * H, -1)[~flat], "certified rows")
+    if flat.any():
+        dn = oracle.dense(geo, q, K, V, bt, sl, w.epsilon, unit_mask=want_fb)
+        check_out(out[flat], dn.out.reshape(Bn * H, -1)[flat], "fallback rows")
+    return ce, sp, want_fb
+
+
+@pytest.mark.parametrize("hq,hkv", [(8, 2), (8, 1), (4, 4), (4, 2)])
+def test_certified_step_matches_the_oracle(hq, hkv):
+    w = make_workload(spec(n_q_heads=hq, n_kv_heads=hkv), seed=400 + hq + hkv)
+    ce, sp, fb = compare_certified(w, run_certified(w))
+    assert np.all(ce.delta_cert <= sp.delta)
+
+
+def test_certificate_passes_for_planted_heads_and_fails_for_flat_ones():
+    # strong needles: the best score clears every ball bound; needle-free heads cannot be certified
+    w = make_workload(spec(seq_lens=(2000, 1500, 900), P=8, K_c=64, needles=4), seed=410)
+    ce, sp, fb = compare_certified(w, run_certified(w))
+    assert ce.certified.any()
+    w0 = make_workload(spec(seq_lens=(2000, 1500, 900), P=8, K_c=64, needles=0), seed=411)
+    ce0, sp0, fb0 = compare_certified(w0, run_certified(w0))
+    assert not ce0.certified.any() and fb0.all()
+
+
+def test_everything_routed_and_ragged_tails():
+    # P covers every page of the short sequences: no un-routed page, the certified gap is the proxy gap
+    w = make_workload(spec(seq_lens=(60, 17, 1), P=4, K_c=20), seed=412)
+    g = run_certified(w)
+    ce, sp, fb = compare_certified(w, g)
+    assert np.all(np.isneginf(ce.ub_unrouted)) and np.array_equal(ce.delta_cert, sp.delta)
+
+
+def test_incremental_radius_update_of_the_last_page():
+    w = make_workload(spec(needles=0), seed=413).to(DEV)
+    shape = B.shape_of(w.q, w.k_cache, w.block_table)
+    summ = torch.zeros((shape.num_pool_pages, 2, 128), dtype=torch.bfloat16, device=DEV)
+    B.vsa_build_page_summaries(shape, w.k_cache, w.block_table, w.seq_lens, None, summ)
+    full = torch.zeros((shape.num_pool_pages, 2), dtype=torch.float32, device=DEV)
+    B.vsa_build_page_radii(shape, w.k_cache, summ, w.block_table, w.seq_lens, None, full)
+    part = torch.zeros_like(full)
+    first = torch.tensor([(700 - 1) // 16, (333 - 1) // 16, (90 - 1) // 16], dtype=torch.int32, device=DEV)
+    B.vsa_build_page_radii(shape, w.k_cache, summ, w.block_table, w.seq_lens, first, part)
+    torch.cuda.synchronize()
+    for b in range(3):
+        last = int(w.block_table[b, int(first[b])])
+        assert torch.equal(part[last], full[last]) and not part[int(w.block_table[b, 0])].any()
+
+
+def test_wide_block_table_and_many_units():
+    # 2500 pages per sequence with 160 units: the 256-thread kernel with 16 page scores per thread
+    w = make_workload(spec(batch=20, n_q_heads=8, n_kv_heads=2, seq_lens=(40000,) + (900,) * 19, P=16, K_c=128,
+                           needles=6), seed=414)
+    compare_certified(w, run_certified(w))
