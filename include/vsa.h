@@ -247,6 +247,21 @@ int vsa_build_page_radii(const vsa_shape_t* shape, const void* k_cache, const vo
                          const int32_t* block_table, const int32_t* seq_lens, const int32_t* first_page,
                          float* radii, void* stream);
 
+/*
+ * Cache maintenance between two decode steps, in one kernel (the paper assumes a paged cache "as in
+ * vLLM" and has no counterpart for this call): append one token per sequence and bring the page
+ * it lands in up to date.  seq_lens are the lengths AFTER the append: sequence b's new token sits at
+ * position seq_lens[b] - 1, i.e. in page block_table[b][(seq_lens[b] - 1) / page_size], which must
+ * already be allocated.  Writes the token's key and value rows, then that page's summary and, when
+ * radii != NULL, its radius - the same values vsa_build_page_summaries / vsa_build_page_radii would
+ * produce for the page.  Sequences with an invalid length or page are skipped.
+ *   k_new, v_new: device bf16 [batch][n_kv_heads][head_dim].  k_cache, v_cache, summaries, radii: device,
+ *   updated in place.
+ */
+int vsa_append_kv(const vsa_shape_t* shape, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                  const int32_t* block_table, const int32_t* seq_lens, void* summaries, float* radii,
+                  void* stream);
+
 int vsa_decode_step_certified(const vsa_shape_t* shape, const void* q, const void* summaries, const float* radii,
                               const void* k_cache, const void* v_cache, const int32_t* block_table,
                               const int32_t* seq_lens, int32_t P, int32_t K_c, float epsilon, float gap_threshold,

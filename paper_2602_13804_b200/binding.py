@@ -80,6 +80,8 @@ def lib() -> C.CDLL:
         _lib.vsa_build_page_radii.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp]
         _lib.vsa_decode_step_certified.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, vp, vp, vp, vp,
                                                    vp, vp, vp, sz, vp]
+        _lib.vsa_append_kv.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        _lib.vsa_append_kv.restype = C.c_int
         _lib.vsa_build_page_radii.restype = C.c_int
         _lib.vsa_decode_step_certified.restype = C.c_int
         for name in ("vsa_build_page_summaries", "vsa_route_pages", "vsa_sparse_decode",
@@ -212,6 +214,13 @@ def vsa_build_page_radii(shape, k_cache, summaries, block_table, seq_lens, first
     _check(lib().vsa_build_page_radii(C.byref(shape), _ptr(k_cache), _ptr(summaries), _ptr(block_table),
                                       _ptr(seq_lens), _ptr(first_page), _ptr(radii), _stream(stream)),
            "vsa_build_page_radii")
+
+
+def vsa_append_kv(shape, k_new, v_new, k_cache, v_cache, block_table, seq_lens, summaries, radii=None,
+                  stream=None) -> None:
+    _check(lib().vsa_append_kv(C.byref(shape), _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache),
+                               _ptr(block_table), _ptr(seq_lens), _ptr(summaries), _ptr(radii), _stream(stream)),
+           "vsa_append_kv")
 
 
 def vsa_decode_step_certified(shape, q, summaries, radii, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon,

@@ -166,6 +166,20 @@ int vsa_build_page_radii(const vsa_shape_t* shape, const void* k_cache, const vo
                                            (cudaStream_t)stream));
 }
 
+int vsa_append_kv(const vsa_shape_t* shape, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                  const int32_t* block_table, const int32_t* seq_lens, void* summaries, float* radii, void* stream)
+{
+    Geometry g;
+    int rc = make_geometry(shape, &g);
+    if (rc) return rc;
+    if (!k_new || !v_new || !k_cache || !v_cache || !block_table || !seq_lens || !summaries)
+        return VSA_ERR_INVALID_ARGUMENT;
+    if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(summaries))
+        return VSA_ERR_MISALIGNED;
+    return cuda_rc(vsa::launch_append(g, k_new, v_new, k_cache, v_cache, block_table, seq_lens, summaries, radii,
+                                      (cudaStream_t)stream));
+}
+
 int vsa_route_pages(const vsa_shape_t* shape, const void* q, const void* summaries, const int32_t* block_table,
                     const int32_t* seq_lens, int32_t P, int32_t* routed_pages, float* routed_scores, void* ws,
                     size_t ws_bytes, void* stream)

@@ -30,7 +30,6 @@ constexpr int kTileBytes = kPageSize * kRowBytes;  // 4 KB: K (or V) rows of one
 constexpr int kStageBytes = 2 * kTileBytes;        // K tile + V tile
 constexpr int kRingBytes = kDenseWarps * kStages * kStageBytes;   // 192 KB per block
 constexpr int kPartialFloats = 2 + kHeadDim;       // per (item, head): max (log2 domain), sum, acc[128]
-constexpr int kMaxGroups = 4096;                   // batch * n_kv_heads the bookkeeping arrays can hold
 constexpr int kItemsPerBlockTarget = 2;
 constexpr int kMinPagesPerItem = 2 * kDenseWarps;  // at least two pages per warp: one would expose the DRAM latency
 

@@ -5,6 +5,59 @@
 
 namespace vsa {
 
+// Mean of the first n rows (this thread's 8 columns of each): fp32 sum in ascending token order, IEEE
+// division by n, round-to-nearest-even to bf16, packed.
+__device__ __forceinline__ uint4 mean_of_rows(const uint4 (&rows)[kPageSize], int n)
+{
+    float acc[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] = 0.0f;
+#pragma unroll
+    for (int t = 0; t < kPageSize; ++t) {
+        if (t < n) {
+            float f[8];
+            unpack8(rows[t], f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = acc[e] + f[e];
+        }
+    }
+    const float fn = (float)n;
+    uint32_t h[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) h[e] = bf16_bits_rne(__fdiv_rn(acc[e], fn));
+    uint4 o;
+    o.x = h[0] | (h[1] << 16);
+    o.y = h[2] | (h[3] << 16);
+    o.z = h[4] | (h[5] << 16);
+    o.w = h[6] | (h[7] << 16);
+    return o;
+}
+
+// Radius of the first n rows around mu (see radii_kernel), computed by the 16 lanes of a half-warp
+// (lane c = columns 8c .. 8c+7, `hmask` = the half-warp's lanes); every lane returns the value.
+__device__ __forceinline__ float radius_of_rows(const uint4 (&rows)[kPageSize], int n, const uint4& mu_bits, int c,
+                                                unsigned hmask)
+{
+    float mu[8];
+    unpack8(mu_bits, mu);
+    float vals[16];
+#pragma unroll
+    for (int t = 0; t < kPageSize; ++t) {
+        float f[8], d[8];
+        unpack8(rows[t], f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) d[e] = __fsub_rn(f[e], mu[e]);
+        vals[t] = t < n ? chunk_partial(d, d) : 0.0f;
+    }
+    float d2 = reduce_scatter16(vals, c, hmask);   // lane t: |k_t - mu|^2, 0 for absent rows
+#pragma unroll
+    for (int off = 8; off; off >>= 1) d2 = fmaxf(d2, __shfl_xor_sync(hmask, d2, off));
+    float m2 = chunk_partial(mu, mu);
+#pragma unroll
+    for (int off = 8; off; off >>= 1) m2 = m2 + __shfl_xor_sync(hmask, m2, off);
+    return __fadd_rn(__fmul_rn(__fsqrt_rn(d2), 1.001f), __fmul_rn(__fsqrt_rn(m2), 0x1p-12f));
+}
+
 // One thread per (logical page, kv head, 16-byte slice of the head dimension): the 16 threads of a
 // (page, head) read one contiguous 256-byte key row per iteration.  fp32 sum in ascending token
 // order, IEEE division by the number of valid rows, round-to-nearest-even to bf16.
@@ -33,28 +86,7 @@ __global__ void __launch_bounds__(256) summaries_kernel(Geometry geo, const uint
 #pragma unroll
     for (int t = 0; t < kPageSize; ++t)
         if (t < n) rows[t] = ld_nc_16B(src + (long long)t * geo.token_stride);
-    float acc[8];
-#pragma unroll
-    for (int e = 0; e < 8; ++e) acc[e] = 0.0f;
-#pragma unroll
-    for (int t = 0; t < kPageSize; ++t) {
-        if (t < n) {
-            float f[8];
-            unpack8(rows[t], f);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] = acc[e] + f[e];
-        }
-    }
-    const float fn = (float)n;
-    uint32_t h[8];
-#pragma unroll
-    for (int e = 0; e < 8; ++e) h[e] = bf16_bits_rne(__fdiv_rn(acc[e], fn));
-    uint4 o;
-    o.x = h[0] | (h[1] << 16);
-    o.y = h[2] | (h[3] << 16);
-    o.z = h[4] | (h[5] << 16);
-    o.w = h[6] | (h[7] << 16);
-    *reinterpret_cast<uint4*>(summaries + (p * geo.n_kv_heads + g) * kHeadDim + c * 8) = o;
+    *reinterpret_cast<uint4*>(summaries + (p * geo.n_kv_heads + g) * kHeadDim + c * 8) = mean_of_rows(rows, n);
 }
 
 // Radius of each page around its stored summary (the ball bound of the routing certificate):
@@ -84,31 +116,65 @@ __global__ void __launch_bounds__(256) radii_kernel(Geometry geo, const uint16_t
     const int n = min(kPageSize, T - (int)l * kPageSize);
     const unsigned hmask = 0xffffu << (threadIdx.x & 16);   // this half-warp (the other may have returned)
 
-    float mu[8];
-    unpack8(*reinterpret_cast<const uint4*>(summaries + (p * geo.n_kv_heads + g) * kHeadDim + c * 8), mu);
+    const uint4 mu_bits = *reinterpret_cast<const uint4*>(summaries + (p * geo.n_kv_heads + g) * kHeadDim + c * 8);
     const uint16_t* src = k_cache + p * geo.page_stride + (long long)g * geo.head_stride + c * 8;
     uint4 rows[kPageSize];
 #pragma unroll
     for (int t = 0; t < kPageSize; ++t)
         rows[t] = t < n ? ld_nc_16B(src + (long long)t * geo.token_stride) : make_uint4(0u, 0u, 0u, 0u);
-    float vals[16];
+    const float rhat = radius_of_rows(rows, n, mu_bits, c, hmask);
+    if (c == 0) radii[p * geo.n_kv_heads + g] = rhat;
+}
+
+// Appends one token per sequence to the paged cache and brings the page it lands in up to date: its
+// key and value rows, the page's summary and (when asked for) its radius.  A half-warp per
+// (sequence, kv head); seq_lens are the lengths AFTER the append.
+__global__ void __launch_bounds__(256) append_kernel(Geometry geo, const uint16_t* __restrict__ k_new,
+                                                     const uint16_t* __restrict__ v_new, uint16_t* __restrict__ k_cache,
+                                                     uint16_t* __restrict__ v_cache,
+                                                     const int32_t* __restrict__ block_table,
+                                                     const int32_t* __restrict__ seq_lens,
+                                                     uint16_t* __restrict__ summaries, float* __restrict__ radii)
+{
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const int c = (int)(idx & 15);
+    const long long pair = idx >> 4;
+    if (pair >= (long long)geo.batch * geo.n_kv_heads) return;
+    const int b = (int)(pair / geo.n_kv_heads), g = (int)(pair % geo.n_kv_heads);
+    const int T = seq_lens[b];
+    if (T <= 0 || T > geo.max_pages * kPageSize) return;
+    const int l = (T - 1) / kPageSize, n = (T - 1) % kPageSize + 1;   // page of the new token, rows it holds now
+    const long long p = block_table[(long long)b * geo.max_pages + l];
+    if (p < 0 || p >= geo.pool_pages) return;
+    const unsigned hmask = 0xffffu << (threadIdx.x & 16);
+
+    const long long row0 = p * geo.page_stride + (long long)g * geo.head_stride + c * 8;
+    const uint4 kn = *reinterpret_cast<const uint4*>(k_new + pair * kHeadDim + c * 8);
+    const uint4 vn = *reinterpret_cast<const uint4*>(v_new + pair * kHeadDim + c * 8);
+    *reinterpret_cast<uint4*>(k_cache + row0 + (long long)(n - 1) * geo.token_stride) = kn;
+    *reinterpret_cast<uint4*>(v_cache + row0 + (long long)(n - 1) * geo.token_stride) = vn;
+    uint4 rows[kPageSize];
 #pragma unroll
-    for (int t = 0; t < kPageSize; ++t) {
-        float f[8], d[8];
-        unpack8(rows[t], f);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) d[e] = __fsub_rn(f[e], mu[e]);
-        vals[t] = t < n ? chunk_partial(d, d) : 0.0f;
+    for (int t = 0; t < kPageSize; ++t)
+        rows[t] = t < n - 1 ? *reinterpret_cast<const uint4*>(k_cache + row0 + (long long)t * geo.token_stride)
+                            : (t == n - 1 ? kn : make_uint4(0u, 0u, 0u, 0u));
+    const uint4 mu_bits = mean_of_rows(rows, n);
+    *reinterpret_cast<uint4*>(summaries + (p * geo.n_kv_heads + g) * kHeadDim + c * 8) = mu_bits;
+    if (radii) {
+        const float rhat = radius_of_rows(rows, n, mu_bits, c, hmask);
+        if (c == 0) radii[p * geo.n_kv_heads + g] = rhat;
     }
-    float d2 = reduce_scatter16(vals, c, hmask);   // lane t: |k_t - mu|^2, 0 for absent rows
-#pragma unroll
-    for (int off = 8; off; off >>= 1) d2 = fmaxf(d2, __shfl_xor_sync(hmask, d2, off));
-    float m2 = chunk_partial(mu, mu);
-#pragma unroll
-    for (int off = 8; off; off >>= 1) m2 = m2 + __shfl_xor_sync(hmask, m2, off);
-    if (c == 0)
-        radii[p * geo.n_kv_heads + g] =
-            __fadd_rn(__fmul_rn(__fsqrt_rn(d2), 1.001f), __fmul_rn(__fsqrt_rn(m2), 0x1p-12f));
+}
+
+cudaError_t launch_append(const Geometry& g, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                          const int32_t* block_table, const int32_t* seq_lens, void* summaries, float* radii,
+                          cudaStream_t stream)
+{
+    const long long threads = (long long)g.batch * g.n_kv_heads * 16;
+    append_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(
+        g, (const uint16_t*)k_new, (const uint16_t*)v_new, (uint16_t*)k_cache, (uint16_t*)v_cache, block_table,
+        seq_lens, (uint16_t*)summaries, radii);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_build_radii(const Geometry& g, const void* k_cache, const void* summaries,

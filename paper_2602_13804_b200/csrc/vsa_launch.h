@@ -45,6 +45,10 @@ cudaError_t launch_build_radii(const Geometry& g, const void* k_cache, const voi
                                const int32_t* block_table, const int32_t* seq_lens, const int32_t* first_page,
                                float* radii, cudaStream_t stream);
 
+cudaError_t launch_append(const Geometry& g, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                          const int32_t* block_table, const int32_t* seq_lens, void* summaries, float* radii,
+                          cudaStream_t stream);
+
 // ---- page routing ---------------------------------------------------------------------------
 size_t route_workspace_bytes(const Geometry& g);
 // zero_word (one int) and zero_words[0..zero_count) are cleared by the scan kernel when not null

@@ -152,6 +152,15 @@ def test_certificate_argument_validation(lib):
     assert C.sizeof(C.c_int32) * len(B.CERT_FIELDS) == 16
 
 
+def test_append_argument_validation(lib):
+    ok = B.make_shape(2, 8, 2, 64, 256)
+    a = lib.vsa_append_kv
+    assert a(C.byref(ok), None, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, None, None) == -1
+    assert a(C.byref(ok), FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, None, None, None) == -1
+    assert a(C.byref(ok), ODD, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, None, None) == -4
+    assert a(None, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, None, None) == -1
+
+
 def test_dense_and_step_argument_validation(lib):
     ok = B.make_shape(2, 8, 2, 64, 256)
     s = C.byref(ok)

@@ -135,3 +135,47 @@ def test_wide_block_table_and_many_units():
     w = make_workload(spec(batch=20, n_q_heads=8, n_kv_heads=2, seq_lens=(40000,) + (900,) * 19, P=16, K_c=128,
                            needles=6), seed=414)
     compare_certified(w, run_certified(w))
+
+
+def test_append_keeps_cache_summaries_and_radii_in_step_with_a_full_rebuild():
+    """Three appended tokens per sequence (the first one opens a new page for sequence 0): rows,
+    summaries and radii must equal what the oracle builds from scratch on the grown cache."""
+    w = make_workload(spec(seq_lens=(160, 333, 15), needles=0), seed=415)
+    # room for the growth: the generator sizes block-table rows for the initial lengths
+    wd = w.to(DEV)
+    shape = B.shape_of(wd.q, wd.k_cache, wd.block_table)
+    summ = torch.zeros((shape.num_pool_pages, shape.n_kv_heads, 128), dtype=torch.bfloat16, device=DEV)
+    radii = torch.zeros((shape.num_pool_pages, shape.n_kv_heads), dtype=torch.float32, device=DEV)
+    B.vsa_build_page_summaries(shape, wd.k_cache, wd.block_table, wd.seq_lens, None, summ)
+    B.vsa_build_page_radii(shape, wd.k_cache, summ, wd.block_table, wd.seq_lens, None, radii)
+    q, K, V, bt, sl = host_arrays(w)
+    K, V, sl = K.copy(), V.copy(), sl.copy()
+    geo = geometry(w)
+    gen = torch.Generator().manual_seed(9)
+    lens = wd.seq_lens.clone()
+    bt = bt.copy()
+    free = sorted(set(range(geo.num_pool_pages)) - set(int(x) for x in bt.reshape(-1) if x >= 0))
+    for step in range(3):
+        for b in range(3):          # the scheduler's part: a fresh page when the new token opens one
+            if int(sl[b]) % 16 == 0:
+                bt[b, int(sl[b]) // 16] = free.pop()
+        wd.block_table = torch.from_numpy(bt).to(DEV)
+        k_new = torch.randn((3, 2, 128), generator=gen).to(torch.bfloat16)
+        v_new = torch.randn((3, 2, 128), generator=gen).to(torch.bfloat16)
+        lens = lens + 1
+        B.vsa_append_kv(shape, k_new.to(DEV), v_new.to(DEV), wd.k_cache, wd.v_cache, wd.block_table, lens, summ, radii)
+        kb = k_new.view(torch.int16).numpy().view(np.uint16)
+        vb = v_new.view(torch.int16).numpy().view(np.uint16)
+        for b in range(3):
+            pos = int(sl[b])
+            K[bt[b, pos // 16], :, pos % 16] = kb[b]
+            V[bt[b, pos // 16], :, pos % 16] = vb[b]
+        sl = sl + 1
+    torch.cuda.synchronize()
+    from util import bits
+    assert np.array_equal(bits(wd.k_cache), K) and np.array_equal(bits(wd.v_cache), V)
+    o_sum = oracle.build_summaries(geo, K, bt, sl)
+    o_rad = oracle.build_radii(geo, K, o_sum, bt, sl)
+    owned = np.concatenate([bt[b, : (int(sl[b]) + 15) // 16] for b in range(3)])
+    assert np.array_equal(bits(summ)[owned], o_sum[owned])
+    assert np.array_equal(radii.cpu().numpy()[owned].view(np.uint32), o_rad[owned].view(np.uint32))
