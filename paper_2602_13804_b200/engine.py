@@ -58,3 +58,38 @@ class SparsePagedDecoder:
                                self.diag_host, self.diag, self.routed_pages, self.fallback_list,
                                self.fallback_count, self.ws)
         return self.out_host
+
+    # ---- variants of the step ---------------------------------------------------------------------
+
+    def step_entropic(self, q, summaries, k_cache, v_cache, block_table, seq_lens, solver_iters: int) -> torch.Tensor:
+        """The step with the candidate weights taken from `solver_iters` entropic mirror-descent
+        iterations; the per-unit certificate and objective land in self.solve ([units, 4] float32)."""
+        if not hasattr(self, "solve"):
+            self.solve = B.alloc_solve(self.units, self.device)
+        B.vsa_decode_step_entropic(self.shape, q, summaries, k_cache, v_cache, block_table, seq_lens, self.P,
+                                   self.K_c, self.epsilon, self.gap_threshold, int(solver_iters), self.out,
+                                   self.diag, self.solve, self.routed_pages, self.fallback_list,
+                                   self.fallback_count, self.ws)
+        return self.out
+
+    def build_radii(self, k_cache, summaries, block_table, seq_lens, first_page=None, radii=None) -> torch.Tensor:
+        if radii is None:
+            radii = torch.zeros((self.shape.num_pool_pages, self.shape.n_kv_heads), dtype=torch.float32,
+                                device=self.device)
+        B.vsa_build_page_radii(self.shape, k_cache, summaries, block_table, seq_lens, first_page, radii)
+        return radii
+
+    def step_certified(self, q, summaries, radii, k_cache, v_cache, block_table, seq_lens) -> torch.Tensor:
+        """The step with the routing certificate: the certified gap (self.cert, [units, 4] int32 view of
+        vsa_cert_t, see binding.cert_to_dict) decides which units fall back to the dense pass."""
+        if not hasattr(self, "cert"):
+            self.cert = B.alloc_cert(self.units, self.device)
+            self.ws_cert = B.alloc_workspace(self.shape, self.P, self.K_c, B.VSA_WS_STEP_CERTIFIED, self.device)
+        B.vsa_decode_step_certified(self.shape, q, summaries, radii, k_cache, v_cache, block_table, seq_lens, self.P,
+                                    self.K_c, self.epsilon, self.gap_threshold, self.out, self.diag, self.cert,
+                                    self.routed_pages, self.fallback_list, self.fallback_count, self.ws_cert)
+        return self.out
+
+    def append(self, k_new, v_new, k_cache, v_cache, block_table, seq_lens_after, summaries, radii=None) -> None:
+        """Append one token per sequence (lengths AFTER the append) and refresh its page's summary / radius."""
+        B.vsa_append_kv(self.shape, k_new, v_new, k_cache, v_cache, block_table, seq_lens_after, summaries, radii)
