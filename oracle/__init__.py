@@ -238,6 +238,28 @@ def certify(geo: Geometry, q, radii, block_table, seq_lens, route: "RouteResult"
 
 
 @dataclass
+class FrankWolfeResult:
+    alpha: np.ndarray       # fp32 [B, Hq, K_c] weights in the order of cand_pos
+    fw_gap: np.ndarray      # fp32 [B, Hq]
+    objective: np.ndarray   # fp32 [B, Hq]  1/2 |K_S^T a - q|^2
+    residual2: np.ndarray
+    step: np.ndarray        # last gamma
+
+
+def frank_wolfe(geo: Geometry, q, k_cache, block_table, cand_pos, iters: int) -> FrankWolfeResult:
+    qb, k, bt = _u16(q), _u16(k_cache), _i32(block_table)
+    cp = _i32(cand_pos)
+    B, H, K_c = geo.batch, geo.n_q_heads, cp.shape[-1]
+    r = FrankWolfeResult(np.zeros((B, H, K_c), np.float32), np.zeros((B, H), np.float32), np.zeros((B, H), np.float32),
+                         np.zeros((B, H), np.float32), np.zeros((B, H), np.float32))
+    s = geo.c()
+    rc = lib().orc_frank_wolfe(C.byref(s), _p(qb), _p(k), _p(bt), _p(cp), C.c_int(K_c), C.c_int(iters), _p(r.alpha),
+                               _p(r.fw_gap), _p(r.objective), _p(r.residual2), _p(r.step))
+    assert rc == 0, rc
+    return r
+
+
+@dataclass
 class DenseResult:
     out: np.ndarray                    # fp64 [B, Hq, d] (rows of unmasked units only)
     lse: np.ndarray                    # fp64 [B, Hq]

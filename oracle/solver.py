@@ -120,3 +120,35 @@ def sparse_entropic(geo, q, k_cache, v_cache, block_table, seq_lens, routed_page
             res.objective[b, h], res.residual2[b, h] = sol.objective, sol.residual2
             res.fw_gap[b, h], res.step[b, h] = sol.fw_gap, sol.step
     return res
+
+
+@dataclass
+class SparseFrankWolfeResult:
+    out: np.ndarray          # fp64 [B, Hq, d]  sum_i alpha_i v_i
+    fw: object               # oracle.FrankWolfeResult (weights in the candidates' selection order)
+    base: object             # the closed-form pass (candidates, gap diagnostics, fallback flags)
+
+
+def sparse_frank_wolfe(geo, q, k_cache, v_cache, block_table, seq_lens, routed_pages, K_c: int, epsilon: float,
+                       gap_threshold: float, iters: int) -> SparseFrankWolfeResult:
+    """Sec. 7 steps 2-4 with step 3 done by `iters` Frank-Wolfe iterations on the unregularised problem
+    (App. E).  The weights come from the C oracle's mirrored-fp32 Frank-Wolfe (the vertex choices are
+    integers); the values are read out with them in fp64.  Native cache layout only."""
+    import oracle
+
+    base = oracle.sparse(geo, q, k_cache, v_cache, block_table, seq_lens, routed_pages, K_c, epsilon, gap_threshold)
+    fw = oracle.frank_wolfe(geo, q, k_cache, block_table, base.cand_pos, iters)
+    B, H, d, G = geo.batch, geo.n_q_heads, geo.head_dim, geo.n_q_heads // geo.n_kv_heads
+    ps = geo.page_size
+    Vf = oracle.bf16_to_f32(np.asarray(v_cache)).astype(np.float64)
+    bt = np.asarray(block_table)
+    out = np.zeros((B, H, d))
+    for b in range(B):
+        for h in range(H):
+            n = int(base.n_candidates[b, h])
+            if n == 0:
+                continue
+            pos = base.cand_pos[b, h, :n]
+            rows_v = Vf[bt[b, pos // ps], h // G, pos % ps]
+            out[b, h] = fw.alpha[b, h, :n].astype(np.float64) @ rows_v
+    return SparseFrankWolfeResult(out=out, fw=fw, base=base)

@@ -20,6 +20,8 @@
  *   orc_build_radii,     a certificate for the routing (App. E "screening"; construction not in the
  *   orc_certify          paper): per-page ball around the summary, upper bound on every un-scored
  *                        token, certified gap and leakage bound.
+ *   orc_frank_wolfe      App. E: Frank-Wolfe with exact line search on the candidate simplex and its
+ *                        duality gap, in mirrored fp32 (the vertex choices are integers).
  *   orc_dense            the plain definition: softmax(<q,k_t>/epsilon) over every token.
  * (The theory objects on tiny dictionaries - Euclidean projection, exact gap, the full
  *  entropic minimiser of Eq. (5.1) - live in theory.py next to this file.)
@@ -390,6 +392,100 @@ int orc_certify(const orc_shape *s, const uint16_t *q, const float *radii, const
         certified[u] = d >= gap_threshold ? 1 : 0;
         double lb = (double)(T - n_candidates[u]) * exp(-(double)d / (double)epsilon);
         leak_cert[u] = lb < 1.0 ? lb : 1.0;
+    }
+    return 0;
+}
+
+/* ---- Frank-Wolfe on the candidate set (App. E) ------------------------------------------------
+ * minimise over the simplex of S   f(a) = 1/2 |sum_i a_i k_i - q|^2   by Frank-Wolfe with exact line
+ * search, started at the best-scoring candidate:
+ *     g_i = <k_i, y> - <k_i, q>,  j = argmin_i g_i,  d = k_j - y,
+ *     gamma = clamp(<q - y, d> / |d|^2, 0, 1),  y <- y + gamma d,  a <- (1 - gamma) a + gamma e_j,
+ * and the certificate  g_t = <grad f, a> - min_j grad f_j = <y, y - q> - min_i g_i  >= f(a) - min f.
+ * The vertex choices are integers decided by floating point, so all of it is fp32 in one fixed order
+ * (canonical dot products, every operation a single rounded one, ties to the lower token position),
+ * which a GPU reproduces bit for bit.  The paper fixes neither start, step rule nor tie-break.
+ * cand_pos: the candidates' token positions (any order, -1 padded, K_c wide); alpha comes back in
+ * the same order. */
+static float canon_dot32(const float *a, const float *b)
+{
+    float p[16];
+    for (int c = 0; c < 16; ++c) {
+        float part[2];
+        for (int par = 0; par < 2; ++par) {
+            float acc = a[8 * c + par] * b[8 * c + par];
+            for (int e = 2 + par; e < 8; e += 2) acc = fmaf(a[8 * c + e], b[8 * c + e], acc);
+            part[par] = acc;
+        }
+        p[c] = part[0] + part[1];
+    }
+    for (int off = 8; off >= 1; off >>= 1)
+        for (int c = 0; c < off; ++c) p[c] = p[c] + p[c + off];
+    return p[0];
+}
+
+int orc_frank_wolfe(const orc_shape *s, const uint16_t *q, const uint16_t *K, const int32_t *bt,
+                    const int32_t *cand_pos, int K_c, int iters, float *alpha, float *fw_gap, float *objective,
+                    float *residual2, float *step)
+{
+    if (!shape_ok(s) || K_c < 1 || iters < 0) return -1;
+    const int G = s->n_q_heads / s->n_kv_heads;
+    const int units = s->batch * s->n_q_heads;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int u = 0; u < units; ++u) {
+        int b = u / s->n_q_heads, h = u % s->n_q_heads, g = h / G;
+        const int32_t *cp = cand_pos + (int64_t)u * K_c;
+        float *al = alpha + (int64_t)u * K_c;
+        int n = 0;
+        while (n < K_c && cp[n] >= 0) ++n;
+        for (int i = 0; i < K_c; ++i) al[i] = 0.0f;
+        fw_gap[u] = objective[u] = residual2[u] = step[u] = 0.0f;
+        if (n == 0) continue;
+        float *rows = (float *)malloc(sizeof(float) * (size_t)n * ORC_D);
+        float *sc = (float *)malloc(sizeof(float) * (size_t)n);
+        float *gr = (float *)malloc(sizeof(float) * (size_t)n);
+        float qf[ORC_D], y[ORC_D], d[ORC_D], r[ORC_D];
+        for (int e = 0; e < ORC_D; ++e) qf[e] = orc_bf16_to_f32(q[(int64_t)u * ORC_D + e]);
+        for (int i = 0; i < n; ++i) {
+            int l = cp[i] / s->page_size, t = cp[i] % s->page_size;
+            const uint16_t *row = kv_row(s, K, bt[(int64_t)b * s->max_pages_per_seq + l], g, t);
+            for (int e = 0; e < ORC_D; ++e) rows[(size_t)i * ORC_D + e] = orc_bf16_to_f32(row[e]);
+            sc[i] = orc_canon_dot(q + (int64_t)u * ORC_D, row);
+        }
+        /* start: best score, lower position on ties */
+        int j = 0;
+        for (int i = 1; i < n; ++i)
+            if (sc[i] > sc[j] || (sc[i] == sc[j] && cp[i] < cp[j])) j = i;
+        al[j] = 1.0f;
+        for (int e = 0; e < ORC_D; ++e) y[e] = rows[(size_t)j * ORC_D + e];
+        float gamma = 0.0f, gmin = 0.0f;
+        for (int it = 0;; ++it) {
+            for (int i = 0; i < n; ++i) gr[i] = canon_dot32(y, rows + (size_t)i * ORC_D) - sc[i];
+            j = 0;
+            for (int i = 1; i < n; ++i)
+                if (gr[i] < gr[j] || (gr[i] == gr[j] && cp[i] < cp[j])) j = i;
+            gmin = gr[j];
+            if (it >= iters) break;
+            for (int e = 0; e < ORC_D; ++e) {
+                d[e] = rows[(size_t)j * ORC_D + e] - y[e];
+                r[e] = qf[e] - y[e];
+            }
+            float num = canon_dot32(r, d), den = canon_dot32(d, d);
+            gamma = den > 0.0f ? num / den : 0.0f;
+            gamma = gamma < 0.0f ? 0.0f : (gamma > 1.0f ? 1.0f : gamma);
+            for (int e = 0; e < ORC_D; ++e) y[e] = fmaf(gamma, d[e], y[e]);
+            for (int i = 0; i < n; ++i) al[i] = fmaf(-gamma, al[i], al[i]);
+            al[j] = al[j] + gamma;
+        }
+        for (int e = 0; e < ORC_D; ++e) r[e] = y[e] - qf[e];
+        float r2 = canon_dot32(r, r);
+        fw_gap[u] = canon_dot32(y, r) - gmin;
+        residual2[u] = r2;
+        objective[u] = 0.5f * r2;
+        step[u] = gamma;
+        free(rows);
+        free(sc);
+        free(gr);
     }
     return 0;
 }
