@@ -48,6 +48,8 @@ def parse_args():
     ap.add_argument("--certified", action="store_true",
                     help="time vsa_decode_step_certified (routing certificate computed, certified gap decides the "
                          "fallback) instead of vsa_decode_step")
+    ap.add_argument("--solver", default="eg", choices=["eg", "fw"],
+                    help="with --solver-iters: entropic mirror descent (eg) or Frank-Wolfe with exact line search (fw)")
     ap.add_argument("--solver-iters", type=int, default=None,
                     help="time the step whose candidate weights come from this many entropic mirror-descent "
                          "iterations (vsa_decode_step_entropic) instead of the closed form")
@@ -292,6 +294,9 @@ def run_ours(args):
         elif cert is not None:
             B.vsa_decode_step_certified(shape, w.q, s, radii[i % distinct], w.k_cache, w.v_cache, w.block_table,
                                         w.seq_lens, P, K_c, eps, tau, out, diag, cert, routed, flist, fcount, ws)
+        elif solve is not None and args.solver == "fw":
+            B.vsa_decode_step_frank_wolfe(shape, w.q, s, w.k_cache, w.v_cache, w.block_table, w.seq_lens, P, K_c, eps,
+                                          tau, args.solver_iters, out, diag, solve, routed, flist, fcount, ws)
         elif solve is not None:
             B.vsa_decode_step_entropic(shape, w.q, s, w.k_cache, w.v_cache, w.block_table, w.seq_lens, P, K_c, eps,
                                        tau, args.solver_iters, out, diag, solve, routed, flist, fcount, ws)
@@ -514,7 +519,9 @@ def run_ours(args):
                    "path": "dense split-K baseline" if args.dense_baseline else
                            ("route -> sparse with routing certificate -> dense fallback" if cert is not None else
                             "route -> sparse -> dense fallback" if solve is None else
-                            f"route -> sparse with {args.solver_iters} entropic mirror-descent iterations -> dense fallback")},
+                            f"route -> sparse with {args.solver_iters} " +
+                            ("Frank-Wolfe" if args.solver == "fw" else "entropic mirror-descent") +
+                            " iterations -> dense fallback")},
         "latency_us_per_layer": ms_per_step * 1e3 / L,
         "per_kernel_us": per_kernel, "closed_form_latency_us_per_layer": closed_form_us_per_layer,
         "fallback_fraction_last_layer": fb_count / units,

@@ -177,6 +177,27 @@ int vsa_sparse_decode_entropic(const vsa_shape_t* shape, const void* q, const vo
                                int32_t* fallback_count, void* stream);
 
 /*
+ * The same pass with step 3 done by Frank-Wolfe (App. E; "Frank-Wolfe with small iterations and
+ * certificates", Sec. 7 step 3) on the unregularised problem over the candidate simplex,
+ *     minimise  f(a) = 1/2 |sum_i a_i k_i - q|^2 :
+ * start at the best-scoring candidate, then `solver_iters` times
+ *     g_i = <k_i, y> - <k_i, q>,  j = argmin_i g_i (ties: lower token position),  d = k_j - y,
+ *     gamma = clamp(<q - y, d> / |d|^2, 0, 1),  y <- y + gamma d,  a <- (1 - gamma) a + gamma e_j.
+ * At most solver_iters + 1 candidates carry weight.  out = sum_i a_i V_i.  solve[b][h]: fw_gap =
+ * <y, y - q> - min_i g_i at the final point, objective = f(a), residual2 = |y - q|^2, step = the last
+ * gamma.  The vertex choices are integers decided by floating point: every operation behind them is a
+ * single rounded fp32 operation in the library's canonical summation order (start, step rule and
+ * tie-break are the library's; the paper fixes none).  epsilon only enters diag (closed-form lse,
+ * leakage bound) here.  Candidates, diag, fallback list and all limits as for
+ * vsa_sparse_decode_entropic.
+ */
+int vsa_sparse_decode_frank_wolfe(const vsa_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,
+                                  const int32_t* block_table, const int32_t* seq_lens, const int32_t* routed_pages,
+                                  int32_t P, int32_t K_c, float epsilon, float gap_threshold, int32_t solver_iters,
+                                  float* out, vsa_diag_t* diag, vsa_solve_t* solve, int32_t* fallback_list,
+                                  int32_t* fallback_count, void* stream);
+
+/*
  * Dense fallback (Sec. 10.3 "fallback-to-dense"): for every unit in fallback_list[0 ..
  * *fallback_count) recompute out[b][h][:] = softmax(<q, k_t> / epsilon over all T_b tokens) V
  * with a split-K pass (K and V of a KV head are read once for all listed heads of its
@@ -211,6 +232,13 @@ int vsa_decode_step_entropic(const vsa_shape_t* shape, const void* q, const void
                              int32_t K_c, float epsilon, float gap_threshold, int32_t solver_iters, float* out,
                              vsa_diag_t* diag, vsa_solve_t* solve, int32_t* routed_pages, int32_t* fallback_list,
                              int32_t* fallback_count, void* ws, size_t ws_bytes, void* stream);
+
+/* vsa_route_pages -> vsa_sparse_decode_frank_wolfe -> vsa_dense_decode_fallback. */
+int vsa_decode_step_frank_wolfe(const vsa_shape_t* shape, const void* q, const void* summaries, const void* k_cache,
+                                const void* v_cache, const int32_t* block_table, const int32_t* seq_lens, int32_t P,
+                                int32_t K_c, float epsilon, float gap_threshold, int32_t solver_iters, float* out,
+                                vsa_diag_t* diag, vsa_solve_t* solve, int32_t* routed_pages, int32_t* fallback_list,
+                                int32_t* fallback_count, void* ws, size_t ws_bytes, void* stream);
 
 /*
  * Routing certificate (App. E asks for "certificates" that the screened candidate set is the right

@@ -75,6 +75,12 @@ def lib() -> C.CDLL:
                                               vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         _lib.vsa_sparse_decode_entropic.argtypes = [shp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, i32, vp, vp, vp,
                                                     vp, vp, vp]
+        _lib.vsa_sparse_decode_frank_wolfe.argtypes = [shp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, i32, vp, vp,
+                                                       vp, vp, vp, vp]
+        _lib.vsa_decode_step_frank_wolfe.argtypes = [shp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, i32, vp, vp, vp,
+                                                     vp, vp, vp, vp, sz, vp]
+        _lib.vsa_sparse_decode_frank_wolfe.restype = C.c_int
+        _lib.vsa_decode_step_frank_wolfe.restype = C.c_int
         _lib.vsa_decode_step_entropic.argtypes = [shp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, i32, vp, vp, vp,
                                                   vp, vp, vp, vp, sz, vp]
         _lib.vsa_build_page_radii.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp]
@@ -197,6 +203,28 @@ def vsa_sparse_decode_entropic(shape, q, k_cache, v_cache, block_table, seq_lens
                                             gap_threshold, solver_iters, _ptr(out), _ptr(diag), _ptr(solve),
                                             _ptr(fallback_list), _ptr(fallback_count), _stream(stream)),
            "vsa_sparse_decode_entropic")
+
+
+def vsa_sparse_decode_frank_wolfe(shape, q, k_cache, v_cache, block_table, seq_lens, routed_pages, P, K_c, epsilon,
+                                  gap_threshold, solver_iters, out, diag, solve, fallback_list, fallback_count,
+                                  stream=None) -> None:
+    _check(lib().vsa_sparse_decode_frank_wolfe(C.byref(shape), _ptr(q), _ptr(k_cache), _ptr(v_cache),
+                                               _ptr(block_table), _ptr(seq_lens), _ptr(routed_pages), P, K_c,
+                                               epsilon, gap_threshold, solver_iters, _ptr(out), _ptr(diag),
+                                               _ptr(solve), _ptr(fallback_list), _ptr(fallback_count),
+                                               _stream(stream)),
+           "vsa_sparse_decode_frank_wolfe")
+
+
+def vsa_decode_step_frank_wolfe(shape, q, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon,
+                                gap_threshold, solver_iters, out, diag, solve, routed_pages, fallback_list,
+                                fallback_count, ws, stream=None) -> None:
+    _check(lib().vsa_decode_step_frank_wolfe(C.byref(shape), _ptr(q), _ptr(summaries), _ptr(k_cache), _ptr(v_cache),
+                                             _ptr(block_table), _ptr(seq_lens), P, K_c, epsilon, gap_threshold,
+                                             solver_iters, _ptr(out), _ptr(diag), _ptr(solve), _ptr(routed_pages),
+                                             _ptr(fallback_list), _ptr(fallback_count), _ptr(ws),
+                                             0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
+           "vsa_decode_step_frank_wolfe")
 
 
 def vsa_decode_step_entropic(shape, q, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon,

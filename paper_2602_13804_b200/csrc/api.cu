@@ -221,11 +221,11 @@ int vsa_sparse_decode(const vsa_shape_t* shape, const void* q, const void* k_cac
                                       P, K_c, epsilon, gap_threshold, out, diag, fallback_list, fallback_count, st));
 }
 
-int vsa_sparse_decode_entropic(const vsa_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,
-                               const int32_t* block_table, const int32_t* seq_lens, const int32_t* routed_pages,
-                               int32_t P, int32_t K_c, float epsilon, float gap_threshold, int32_t solver_iters,
-                               float* out, vsa_diag_t* diag, vsa_solve_t* solve, int32_t* fallback_list,
-                               int32_t* fallback_count, void* stream)
+static int sparse_solver_impl(int solver_kind, const vsa_shape_t* shape, const void* q, const void* k_cache,
+                              const void* v_cache, const int32_t* block_table, const int32_t* seq_lens,
+                              const int32_t* routed_pages, int32_t P, int32_t K_c, float epsilon, float gap_threshold,
+                              int32_t solver_iters, float* out, vsa_diag_t* diag, vsa_solve_t* solve,
+                              int32_t* fallback_list, int32_t* fallback_count, void* stream)
 {
     Geometry g;
     int rc = make_geometry(shape, &g);
@@ -242,7 +242,27 @@ int vsa_sparse_decode_entropic(const vsa_shape_t* shape, const void* q, const vo
     if (cudaMemsetAsync(fallback_count, 0, sizeof(int32_t), st) != cudaSuccess) return VSA_ERR_CUDA;
     return cuda_rc(vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, (int32_t*)routed_pages, nullptr,
                                       P, K_c, epsilon, gap_threshold, out, diag, fallback_list, fallback_count, st,
-                                      solver_iters, solve));
+                                      solver_iters, solve, nullptr, nullptr, solver_kind));
+}
+
+int vsa_sparse_decode_entropic(const vsa_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,
+                               const int32_t* block_table, const int32_t* seq_lens, const int32_t* routed_pages,
+                               int32_t P, int32_t K_c, float epsilon, float gap_threshold, int32_t solver_iters,
+                               float* out, vsa_diag_t* diag, vsa_solve_t* solve, int32_t* fallback_list,
+                               int32_t* fallback_count, void* stream)
+{
+    return sparse_solver_impl(1, shape, q, k_cache, v_cache, block_table, seq_lens, routed_pages, P, K_c, epsilon,
+                              gap_threshold, solver_iters, out, diag, solve, fallback_list, fallback_count, stream);
+}
+
+int vsa_sparse_decode_frank_wolfe(const vsa_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,
+                                  const int32_t* block_table, const int32_t* seq_lens, const int32_t* routed_pages,
+                                  int32_t P, int32_t K_c, float epsilon, float gap_threshold, int32_t solver_iters,
+                                  float* out, vsa_diag_t* diag, vsa_solve_t* solve, int32_t* fallback_list,
+                                  int32_t* fallback_count, void* stream)
+{
+    return sparse_solver_impl(2, shape, q, k_cache, v_cache, block_table, seq_lens, routed_pages, P, K_c, epsilon,
+                              gap_threshold, solver_iters, out, diag, solve, fallback_list, fallback_count, stream);
 }
 
 int vsa_dense_decode_fallback(const vsa_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,
@@ -267,7 +287,8 @@ static int decode_step_impl(const vsa_shape_t* shape, const void* q, const void*
                             int32_t K_c, float epsilon, float gap_threshold, float* out, vsa_diag_t* diag,
                             int32_t* routed_pages, int32_t* fallback_list, int32_t* fallback_count, void* ws,
                             size_t ws_bytes, void* stream, void* const* events, int solver_iters = 0,
-                            vsa_solve_t* solve = nullptr, const float* radii = nullptr, vsa_cert_t* cert = nullptr)
+                            vsa_solve_t* solve = nullptr, const float* radii = nullptr, vsa_cert_t* cert = nullptr,
+                            int solver_kind = 1)
 {
     Geometry g;
     int rc = make_geometry(shape, &g);
@@ -309,7 +330,7 @@ static int decode_step_impl(const vsa_shape_t* shape, const void* q, const void*
     if (ev[2] && cudaEventRecord(ev[2], st) != cudaSuccess) return VSA_ERR_CUDA;
     e = vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, routed_pages, (const float*)ws, P, K_c,
                            epsilon, gap_threshold, out, diag, fallback_list, fallback_count, st, solver_iters, solve,
-                           rad_logical, cert);
+                           rad_logical, cert, solver_kind);
     if (e != cudaSuccess) return VSA_ERR_CUDA;
     if (ev[3] && cudaEventRecord(ev[3], st) != cudaSuccess) return VSA_ERR_CUDA;
     e = vsa::launch_dense(g, q, k_cache, v_cache, block_table, seq_lens, fallback_list, fallback_count, epsilon,
@@ -340,6 +361,18 @@ int vsa_decode_step_entropic(const vsa_shape_t* shape, const void* q, const void
     return decode_step_impl(shape, q, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon,
                             gap_threshold, out, diag, routed_pages, fallback_list, fallback_count, ws, ws_bytes,
                             stream, nullptr, solver_iters, solve);
+}
+
+int vsa_decode_step_frank_wolfe(const vsa_shape_t* shape, const void* q, const void* summaries, const void* k_cache,
+                                const void* v_cache, const int32_t* block_table, const int32_t* seq_lens, int32_t P,
+                                int32_t K_c, float epsilon, float gap_threshold, int32_t solver_iters, float* out,
+                                vsa_diag_t* diag, vsa_solve_t* solve, int32_t* routed_pages, int32_t* fallback_list,
+                                int32_t* fallback_count, void* ws, size_t ws_bytes, void* stream)
+{
+    if (!solve) return VSA_ERR_INVALID_ARGUMENT;
+    return decode_step_impl(shape, q, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon,
+                            gap_threshold, out, diag, routed_pages, fallback_list, fallback_count, ws, ws_bytes,
+                            stream, nullptr, solver_iters, solve, nullptr, nullptr, 2);
 }
 
 int vsa_decode_step_certified(const vsa_shape_t* shape, const void* q, const void* summaries, const float* radii,

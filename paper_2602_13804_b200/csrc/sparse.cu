@@ -96,12 +96,13 @@ __device__ __forceinline__ void write_failed_unit(float* out, vsa_diag_t* diag, 
 //   In both fused forms the unit's top-P pages are selected here from page_scores[unit][0..n_b) and
 //   written to routed_pages (best first, -1 padded).
 // TOK_KPT: token scores per thread, P * 16 <= TOK_KPT * THREADS.
-// SOLVE: the weights on the candidates come from `solver_iters` entropic mirror-descent iterations
-//   (256 threads only: every lane owns one candidate, every half-warp sixteen candidate rows).
+// SOLVE 1: the weights on the candidates come from `solver_iters` entropic mirror-descent iterations;
+// SOLVE 2: from `solver_iters` Frank-Wolfe iterations with exact line search on the unregularised
+//   problem (256 threads only: every lane owns one candidate, every half-warp sixteen candidate rows).
 // CERT (fused register variants only): the certified gap of the unit - an upper bound on every score
 //   of the pages that were not routed, from the pages' radii (rad_logical, written by the scan) -
 //   is computed, reported in cert[] and used for the fallback decision in place of the proxy gap.
-template <int THREADS, int PAGE_KPT, int TOK_KPT, bool SOLVE = false, bool CERT = false>
+template <int THREADS, int PAGE_KPT, int TOK_KPT, int SOLVE = 0, bool CERT = false>
 __global__ void __launch_bounds__(THREADS, 512 / THREADS)
 sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* __restrict__ k_cache,
                      const uint16_t* __restrict__ v_cache, const int32_t* __restrict__ block_table,
@@ -112,7 +113,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                      const float* __restrict__ rad_logical, vsa_cert_t* __restrict__ cert)
 {
     constexpr int WARPS = THREADS / 32, GROUPS = 2 * WARPS;
-    static_assert(!SOLVE || THREADS == 256, "the solve maps one candidate to each of 256 lanes");
+    static_assert(SOLVE == 0 || THREADS == 256, "the solve maps one candidate to each of 256 lanes");
     static_assert(!CERT || PAGE_KPT > 0, "the certificate needs every page score of the unit in registers");
     static_assert(TOK_KPT * WARPS <= 64 && 4 * WARPS <= 72, "wred capacity");
     extern __shared__ uint32_t smem_raw[];
@@ -406,7 +407,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                 const int i = tid + j * THREADS, pos = mine + before[j];
                 sm.voff[pos] = (long long)page_phys[i >> 4] * geo.page_stride + (long long)(i & 15) * geo.token_stride;
                 sm.wgt[pos] = exp2f((key_to_float(key[j]) - s1) * scale);
-                if constexpr (SOLVE) sm.score[pos] = key_to_float(key[j]);
+                if constexpr (SOLVE != 0) sm.score[pos] = key_to_float(key[j]);
             }
         }
     }
@@ -414,7 +415,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
 
     VSA_PROBE(6);
     float lse_closed = 0.0f;   // log-sum-exp of the closed-form weights (SOLVE only)
-    if constexpr (SOLVE) {
+    if constexpr (SOLVE != 0) {
         if (ns > 0) {
             // ---- iterative entropic solve on the candidates (Eq. (5.1) restricted to S) ----
             // Lane (half-warp hw, column c) owns candidate j = 16 * hw + c: its score, log-weight and
@@ -443,6 +444,103 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
             }
             const float s_own = have ? sm.score[j_own] : 0.0f;
             float vals[16];
+            if constexpr (SOLVE == 2) {
+                // ---- Frank-Wolfe with exact line search on f(a) = 1/2 |sum a_i k_i - q|^2 (App. E) ----
+                // Vertex choices are integers, so everything that feeds them is single-rounded fp32 in the
+                // canonical order (mirrored by the oracle): the readout y = sum a_i k_i is kept incrementally
+                // (lane c holds elements 8c .. 8c+7, every half-warp the same copy), g_i = <k_i, y> - s_i by
+                // the fixed-order dot, argmin with ties to the lower position, gamma by an IEEE division.
+                __syncthreads();   // rows staged by other half-warps are read below
+                // block-wide best (largest key, then smallest candidate index); `slot` alternates so that a
+                // fast warp cannot overwrite statistics that a slow one still reads
+                auto arg_best = [&](uint32_t key, int slot, uint32_t& best_key, int& best_j) {
+                    const uint32_t wk = __reduce_max_sync(kFullMask, key);
+                    const int wj = __reduce_min_sync(kFullMask, (key == wk && key != 0u) ? j_own : INT_MAX);
+                    if (lane == 0) {
+                        sm.ts.wred[slot * 16 + warp] = wk;
+                        sm.ts.wred[slot * 16 + 8 + warp] = (uint32_t)wj;
+                    }
+                    __syncthreads();
+                    best_key = 0u;
+                    best_j = INT_MAX;
+#pragma unroll
+                    for (int w = 0; w < WARPS; ++w) {
+                        const uint32_t k = sm.ts.wred[slot * 16 + w];
+                        const int j = (int)sm.ts.wred[slot * 16 + 8 + w];
+                        if (k > best_key || (k == best_key && j < best_j)) {
+                            best_key = k;
+                            best_j = j;
+                        }
+                    }
+                };
+                // closed-form log-sum-exp for diag (the weights written at the compaction), and the start
+                {
+                    float w0 = have ? sm.wgt[j_own] : 0.0f;
+#pragma unroll
+                    for (int off = 16; off; off >>= 1) w0 += __shfl_xor_sync(kFullMask, w0, off);
+                    if (lane == 0) sm.ts.wred[56 + warp] = __float_as_uint(w0);
+                }
+                uint32_t bk;
+                int jb;
+                arg_best(have ? float_to_key(s_own) : 0u, 0, bk, jb);
+                {
+                    float z0 = 0.0f;
+#pragma unroll
+                    for (int w = 0; w < WARPS; ++w) z0 += __uint_as_float(sm.ts.wred[56 + w]);
+                    lse_closed = s1 / epsilon + logf(z0);
+                }
+                float yv[8];
+                unpack8(*reinterpret_cast<const uint4*>(ktile + (size_t)jb * kRowBytes + c * 16), yv);
+                float a_own = (have && j_own == jb) ? 1.0f : 0.0f;
+                float gamma = 0.0f, gmin = 0.0f;
+                auto tree16 = [&](float p) {   // canonical halving tree over the half-warp, result in every lane
+#pragma unroll
+                    for (int off = 8; off; off >>= 1) p = p + __shfl_xor_sync(kFullMask, p, off);
+                    return p;
+                };
+                for (int it = 0;; ++it) {
+#pragma unroll
+                    for (int r = 0; r < 16; ++r) {
+                        float uf[8];
+                        unpack8(*reinterpret_cast<const uint4*>(my_rows + r * kRowBytes), uf);
+                        vals[r] = chunk_partial(yv, uf);
+                    }
+                    const float g_own = reduce_scatter16(vals, c) - s_own;
+                    arg_best(have ? float_to_key(-g_own) : 0u, 1 + (it & 1), bk, jb);
+                    gmin = -key_to_float(bk);
+                    if (it >= solver_iters) break;
+                    float uj[8], dv[8], rv[8];
+                    unpack8(*reinterpret_cast<const uint4*>(ktile + (size_t)jb * kRowBytes + c * 16), uj);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        dv[e] = __fsub_rn(uj[e], yv[e]);
+                        rv[e] = __fsub_rn(qf[e], yv[e]);
+                    }
+                    const float num = tree16(chunk_partial(rv, dv)), den = tree16(chunk_partial(dv, dv));
+                    gamma = den > 0.0f ? __fdiv_rn(num, den) : 0.0f;
+                    gamma = gamma < 0.0f ? 0.0f : (gamma > 1.0f ? 1.0f : gamma);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) yv[e] = __fmaf_rn(gamma, dv[e], yv[e]);
+                    a_own = __fmaf_rn(-gamma, a_own, a_own);
+                    if (have && j_own == jb) a_own = __fadd_rn(a_own, gamma);
+                }
+                {
+                    float rv[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) rv[e] = __fsub_rn(yv[e], qf[e]);
+                    const float r2 = tree16(chunk_partial(rv, rv)), yr = tree16(chunk_partial(yv, rv));
+                    if (tid == 0) {
+                        vsa_solve_t sv;
+                        sv.fw_gap = __fsub_rn(yr, gmin);
+                        sv.objective = __fmul_rn(0.5f, r2);
+                        sv.residual2 = r2;
+                        sv.step = gamma;
+                        solve[unit] = sv;
+                    }
+                }
+                if (have) sm.wgt[j_own] = a_own;
+                __syncthreads();
+            } else {
             // step: eta = 1 / max_i |k_i|^2
 #pragma unroll
             for (int r = 0; r < 16; ++r) {
@@ -579,6 +677,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                     solve[unit] = sv;
                 }
             }
+            }   // SOLVE == 1
         } else if (tid == 0) {
             solve[unit] = vsa_solve_t{0.0f, 0.0f, 0.0f, 0.0f};
         }
@@ -686,14 +785,14 @@ struct SparseArgs {
     float* out;
     vsa_diag_t* diag;
     int32_t *fallback_list, *fallback_count;
-    int solver_iters;
-    vsa_solve_t* solve;   // non-null: the iterative-solve variant of the kernel
+    int solver_iters, solver_kind;   // kind 1: entropic mirror descent, 2: Frank-Wolfe
+    vsa_solve_t* solve;   // non-null: an iterative-solve variant of the kernel
     const float* rad_logical;
     vsa_cert_t* cert;     // non-null: the certificate variant (fused register variants only)
     cudaStream_t stream;
 };
 
-template <int THREADS, int PAGE_KPT, int TOK_KPT, bool SOLVE, bool CERT>
+template <int THREADS, int PAGE_KPT, int TOK_KPT, int SOLVE, bool CERT>
 cudaError_t launch_variant(const SparseArgs& a)
 {
     if (a.smem > 48 * 1024) {
@@ -712,14 +811,15 @@ template <int THREADS, int PAGE_KPT, int TOK_KPT>
 cudaError_t launch_one(const SparseArgs& a)
 {
     if constexpr (THREADS == 256) {
-        if (a.solve) return launch_variant<THREADS, PAGE_KPT, TOK_KPT, true, false>(a);
+        if (a.solve && a.solver_kind == 2) return launch_variant<THREADS, PAGE_KPT, TOK_KPT, 2, false>(a);
+        if (a.solve) return launch_variant<THREADS, PAGE_KPT, TOK_KPT, 1, false>(a);
     }
     if constexpr (PAGE_KPT > 0) {
-        if (a.cert) return launch_variant<THREADS, PAGE_KPT, TOK_KPT, false, true>(a);
+        if (a.cert) return launch_variant<THREADS, PAGE_KPT, TOK_KPT, 0, true>(a);
     } else {
         if (a.cert) return cudaErrorInvalidValue;   // (refused by the entry point before any launch)
     }
-    return launch_variant<THREADS, PAGE_KPT, TOK_KPT, false, false>(a);
+    return launch_variant<THREADS, PAGE_KPT, TOK_KPT, 0, false>(a);
 }
 
 template <int THREADS, int PAGE_KPT>
@@ -773,7 +873,8 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
                           const int32_t* block_table, const int32_t* seq_lens, int32_t* routed_pages,
                           const float* page_scores, int P, int K_c, float epsilon, float gap_threshold, float* out,
                           vsa_diag_t* diag, int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream,
-                          int solver_iters, vsa_solve_t* solve, const float* rad_logical, vsa_cert_t* cert)
+                          int solver_iters, vsa_solve_t* solve, const float* rad_logical, vsa_cert_t* cert,
+                          int solver_kind)
 {
     SparseArgs a;
     a.g = g;
@@ -782,6 +883,7 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
     const int threads = (!solve && (long long)g.batch * g.n_q_heads <= sm_count()) ? 512 : 256;
     a.smem = sparse_smem_bytes(g, P, K_c, page_scores != nullptr, threads, solve != nullptr);
     a.solver_iters = solver_iters;
+    a.solver_kind = solver_kind;
     a.solve = solve;
     a.rad_logical = rad_logical;
     a.cert = cert;

@@ -121,6 +121,13 @@ def test_entropic_argument_validation(lib):
     assert call(solve=None) == -1
     assert call(eps=0.0) == -1
     assert call(P=4, K_c=65) == -2
+    fw = lib.vsa_sparse_decode_frank_wolfe
+    assert fw(s, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, 32, 257, 1.0, 0.0, 2, FAKE, FAKE, FAKE, FAKE, FAKE, None) == -2
+    assert fw(s, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, 32, 16, 1.0, 0.0, 65, FAKE, FAKE, FAKE, FAKE, FAKE, None) == -1
+    assert fw(s, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, 32, 16, 1.0, 0.0, 2, FAKE, FAKE, None, FAKE, FAKE, None) == -1
+    fws = lib.vsa_decode_step_frank_wolfe
+    assert fws(s, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, 32, 16, 1.0, 0.0, 2, FAKE, FAKE, None, FAKE, FAKE, FAKE, FAKE,
+               1 << 40, None) == -1
     step = lib.vsa_decode_step_entropic
     assert step(s, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, 32, 257, 1.0, 0.0, 2, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE,
                 1 << 40, None) == -2

@@ -156,3 +156,92 @@ def test_entropic_objective_does_not_increase_with_iterations():
         if prev is not None:
             assert np.all(obj <= prev + 1e-3 + 1e-5 * np.abs(prev))
         prev = obj
+
+
+# ------------------------------------------------------------------------------------- Frank-Wolfe
+
+def run_fw(w, iters, fused=False):
+    wd = w.to(DEV)
+    shape = B.shape_of(wd.q, wd.k_cache, wd.block_table)
+    units = shape.batch * shape.n_q_heads
+    P, K_c = w.spec.P, w.spec.K_c
+    summ = torch.zeros((shape.num_pool_pages, shape.n_kv_heads, 128), dtype=torch.bfloat16, device=DEV)
+    B.vsa_build_page_summaries(shape, wd.k_cache, wd.block_table, wd.seq_lens, None, summ)
+    out = torch.full((shape.batch, shape.n_q_heads, 128), float("nan"), dtype=torch.float32, device=DEV)
+    diag, sol = B.alloc_diag(units, DEV), B.alloc_solve(units, DEV)
+    sol.fill_(float("nan"))
+    flist = torch.full((units,), -1, dtype=torch.int32, device=DEV)
+    fcount = torch.full((1,), 99, dtype=torch.int32, device=DEV)
+    routed = torch.full((shape.batch, shape.n_q_heads, P), -7, dtype=torch.int32, device=DEV)
+    if fused:
+        ws = B.alloc_workspace(shape, P, K_c, B.VSA_WS_STEP, DEV)
+        B.vsa_decode_step_frank_wolfe(shape, wd.q, summ, wd.k_cache, wd.v_cache, wd.block_table, wd.seq_lens, P, K_c,
+                                      w.epsilon, w.gap_threshold, iters, out, diag, sol, routed, flist, fcount, ws)
+    else:
+        ws = B.alloc_workspace(shape, P, K_c, B.VSA_WS_ROUTE, DEV)
+        B.vsa_route_pages(shape, wd.q, summ, wd.block_table, wd.seq_lens, P, routed, None, ws)
+        B.vsa_sparse_decode_frank_wolfe(shape, wd.q, wd.k_cache, wd.v_cache, wd.block_table, wd.seq_lens, routed, P,
+                                        K_c, w.epsilon, w.gap_threshold, iters, out, diag, sol, flist, fcount)
+    torch.cuda.synchronize()
+    n = int(fcount.item())
+    return dict(out=out.cpu().numpy(), diag={k: v.numpy() for k, v in B.diag_to_dict(diag).items()},
+                solve=sol.cpu().numpy(), routed=routed.cpu().numpy(), fallback=np.sort(flist[:n].cpu().numpy()))
+
+
+def compare_fw(w, g, iters):
+    """The vertex choices are integers: the solve record (every field a product of the mirrored fp32
+    arithmetic) must match the oracle bit for bit; `out` is an fp32 gather compared with a tolerance."""
+    q, K, V, bt, sl = host_arrays(w)
+    geo = geometry(w)
+    summ = oracle.build_summaries(geo, K, bt, sl)
+    rt = oracle.route(geo, q, summ, bt, sl, w.spec.P)
+    o = solver.sparse_frank_wolfe(geo, q, K, V, bt, sl, rt.pages, w.spec.K_c, w.epsilon, w.gap_threshold, iters)
+    Bn, H = o.out.shape[:2]
+    assert np.array_equal(g["routed"], rt.pages)
+    got = g["solve"].reshape(Bn, H, 4)
+    for i, (name, want) in enumerate((("fw_gap", o.fw.fw_gap), ("objective", o.fw.objective),
+                                      ("residual2", o.fw.residual2), ("step", o.fw.step))):
+        assert np.array_equal(got[:, :, i].view(np.uint32), want.view(np.uint32)), f"{name} differs"
+    check_out(g["out"], o.out, f"frank-wolfe out, {iters} iterations")
+    d, base = g["diag"], o.base
+    for name, want in (("delta", base.delta), ("delta12", base.delta12), ("s_max", base.s_max)):
+        assert np.array_equal(d[name].reshape(Bn, H), want), name
+    assert np.array_equal(d["n_candidates"].reshape(Bn, H), base.n_candidates)
+    assert np.array_equal(d["fallback"].reshape(Bn, H), base.fallback)
+    fin = np.isfinite(base.lse)
+    assert np.all(np.abs(d["lse"].reshape(Bn, H)[fin] - base.lse[fin]) <= lse_tol(w.epsilon) + 2e-6 * np.abs(base.lse[fin]))
+    return o
+
+
+@pytest.mark.parametrize("iters", [0, 1, 3, 6])
+def test_frank_wolfe_pass_matches_the_oracle(iters):
+    w = make_workload(spec(), seed=320 + iters)
+    o = compare_fw(w, run_fw(w, iters), iters)
+    assert np.all(np.count_nonzero(o.fw.alpha, axis=-1) <= iters + 1)
+
+
+def test_frank_wolfe_needle_free_heads_and_the_fused_step():
+    # flat heads: many near-equal gradient entries, the case where an unmirrored argmin would drift
+    w = make_workload(spec(needles=0, seq_lens=(500, 260, 33)), seed=330)
+    w.gap_threshold = -math.inf
+    compare_fw(w, run_fw(w, 6), 6)
+    compare_fw(w, run_fw(w, 6, fused=True), 6)
+
+
+def test_frank_wolfe_full_tile_and_single_candidate():
+    w = make_workload(spec(batch=2, seq_lens=(9000, 1), P=32, K_c=256, needles=6), seed=331)
+    w.gap_threshold = -math.inf
+    g = run_fw(w, 6, fused=True)
+    o = compare_fw(w, g, 6)
+    assert o.base.n_candidates[0].min() == 256 and o.base.n_candidates[1].max() == 1
+    assert np.all(g["solve"].reshape(2, 8, 4)[1, :, 3] == 0.0)      # one candidate: no step to take
+
+
+def test_frank_wolfe_duplicate_keys_tie_to_the_lower_position():
+    w = make_workload(spec(batch=1, n_q_heads=4, n_kv_heads=2, seq_lens=(64,), P=4, K_c=64, needles=0), seed=332)
+    k = w.k_cache.clone()
+    p0, p1 = int(w.block_table[0, 0]), int(w.block_table[0, 2])
+    k[p1] = k[p0]                                  # tokens 32..47 repeat tokens 0..15, both kv heads
+    w.k_cache = k
+    w.gap_threshold = -math.inf
+    compare_fw(w, run_fw(w, 5), 5)
