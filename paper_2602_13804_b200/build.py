@@ -15,7 +15,7 @@ SOURCES = ["api.cu", "summaries.cu", "route.cu", "sparse.cu", "dense.cu"]
 HEADERS = ["vsa_device.cuh", "vsa_select.cuh", "vsa_launch.h", os.path.join("..", "..", "include", "vsa.h")]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "-Xcompiler", "-fPIC", "-shared", "-cudart", "static",
+    "-Xcompiler", "-fPIC", "-shared", "-cudart", "static", "--threads", "0",
 ]
 
 

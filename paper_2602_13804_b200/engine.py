@@ -93,3 +93,14 @@ class SparsePagedDecoder:
     def append(self, k_new, v_new, k_cache, v_cache, block_table, seq_lens_after, summaries, radii=None) -> None:
         """Append one token per sequence (lengths AFTER the append) and refresh its page's summary / radius."""
         B.vsa_append_kv(self.shape, k_new, v_new, k_cache, v_cache, block_table, seq_lens_after, summaries, radii)
+
+    def step_frank_wolfe(self, q, summaries, k_cache, v_cache, block_table, seq_lens, solver_iters: int) -> torch.Tensor:
+        """The step with the candidate weights taken from `solver_iters` Frank-Wolfe iterations (exact line
+        search, unregularised problem); certificate and objective land in self.solve."""
+        if not hasattr(self, "solve"):
+            self.solve = B.alloc_solve(self.units, self.device)
+        B.vsa_decode_step_frank_wolfe(self.shape, q, summaries, k_cache, v_cache, block_table, seq_lens, self.P,
+                                      self.K_c, self.epsilon, self.gap_threshold, int(solver_iters), self.out,
+                                      self.diag, self.solve, self.routed_pages, self.fallback_list,
+                                      self.fallback_count, self.ws)
+        return self.out
