@@ -30,7 +30,9 @@ constexpr int kTileBytes = kPageSize * kRowBytes;  // 4 KB: K (or V) rows of one
 constexpr int kStageBytes = 2 * kTileBytes;        // K tile + V tile
 constexpr int kRingBytes = kDenseWarps * kStages * kStageBytes;   // 192 KB per block
 constexpr int kPartialFloats = 2 + kHeadDim;       // per (item, head): max (log2 domain), sum, acc[128]
-constexpr int kItemsPerBlockTarget = 2;
+constexpr int kPagesPerItemGoal = 128;             // pages per item and block from which a second round pays
+constexpr int kMaxRounds = 2;
+constexpr int kMaxRoundsRagged = 8;
 constexpr int kMinPagesPerItem = 2 * kDenseWarps;  // at least two pages per warp: one would expose the DRAM latency
 
 __device__ __forceinline__ void cp_async_16_zfill(uint32_t smem_addr, const void* gptr, bool valid)
@@ -129,30 +131,46 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
         return (T + kPageSize - 1) / kPageSize;
     };
     {
-        int pages = 0, groups = 0;
+        int pages = 0, groups = 0, longest = 0;
         for (int i = tid; i < n_groups; i += kDenseThreads) {
             const int p = pages_of(i);
             pages += p;
             groups += p > 0;
+            longest = max(longest, p);
         }
 #pragma unroll
         for (int off = 16; off; off >>= 1) {
             pages += __shfl_xor_sync(kFullMask, pages, off);
             groups += __shfl_xor_sync(kFullMask, groups, off);
+            longest = max(longest, __shfl_xor_sync(kFullMask, longest, off));
         }
         if (lane == 0) {
             atomicAdd(&sm.misc[0], pages);
             atomicAdd(&sm.misc[1], groups);
+            atomicMax(&sm.misc[2], longest);
         }
     }
     __syncthreads();
-    const int total_pages = sm.misc[0], flagged_groups = sm.misc[1];
+    const int total_pages = sm.misc[0], flagged_groups = sm.misc[1], longest_group = sm.misc[2];
     if (total_pages == 0) return;
     int ppi;   // pages per item, a multiple of the warp count
     {
-        const long long target = (long long)gridDim.x * kItemsPerBlockTarget;
-        long long want = (total_pages + target - 1) / target;
-        const long long room = max_items - flagged_groups;   // every group may add one ragged item
+        // Whole rounds: at most `rounds` items per block - one when the work is small (an item costs a few
+        // microseconds of fixed overhead: query fragments, pipeline fill, merge, ticket), two when items
+        // stay long.  Every group may add one ragged item, so sizing for (target - groups) full items
+        // keeps the count within the target and no block starts a round the others do not have.
+        long long rounds = total_pages / ((long long)gridDim.x * kPagesPerItemGoal);
+        rounds = rounds < 1 ? 1 : (rounds > kMaxRounds ? kMaxRounds : rounds);   // 1 or 2
+        // many flagged groups of uneven length (the longest more than twice the mean): about four items
+        // per group, so that short and long groups mix over the blocks
+        if ((long long)longest_group * flagged_groups > 2LL * total_pages) {
+            const long long by_groups = (4LL * flagged_groups + gridDim.x - 1) / gridDim.x;
+            if (rounds < by_groups) rounds = by_groups < kMaxRoundsRagged ? by_groups : kMaxRoundsRagged;
+        }
+        const long long target = (long long)gridDim.x * rounds;
+        long long want = target > 2LL * flagged_groups ? (total_pages + (target - flagged_groups) - 1) / (target - flagged_groups)
+                                                       : (total_pages + target - 1) / target;
+        const long long room = max_items - flagged_groups;
         const long long need = (total_pages + room - 1) / room;
         if (want < need) want = need;
         ppi = (int)((want + kDenseWarps - 1) / kDenseWarps) * kDenseWarps;
@@ -375,28 +393,33 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
         if (sm.misc[12]) {
             __threadfence();
             const float* gp = partials + (long long)sm.item_base[grp] * G * kPartialFloats;
+            // Stage every item's (max, sum) of every head in shared memory first: the weighted sums below
+            // then consist of independent loads only (a running maximum would make each load wait for the
+            // previous item's, which costs a memory round trip per item).
+            float* ms_s = reinterpret_cast<float*>(sm.ring);          // [items][G]
+            float* ls_s = ms_s + (size_t)items_of_group * G;           // [items][G]
+            for (int i = tid; i < items_of_group * G; i += kDenseThreads) {
+                const float* rec = gp + (long long)i * kPartialFloats;
+                ms_s[i] = __ldcg(rec);
+                ls_s[i] = __ldcg(rec + 1);
+            }
+            __syncthreads();
             for (int idx = tid; idx < G * kHeadDim; idx += kDenseThreads) {
                 const int hh = idx / kHeadDim, e = idx % kHeadDim;
                 if (!((mask >> hh) & 1u)) continue;
-                // one pass in item order, rescaling when a later item raises the maximum
-                float M = -INFINITY, a = 0.0f, L = 0.0f;
-#pragma unroll 4
-                for (int s = 0; s < items_of_group; ++s) {
-                    const float* rec = gp + ((long long)s * G + hh) * kPartialFloats;
-                    const float ms = __ldcg(rec), ls = __ldcg(rec + 1), as = __ldcg(rec + 2 + e);
-                    if (ms == -INFINITY) continue;
-                    if (ms > M) {
-                        const float r = exp2f(M - ms);   // 0 for the first contributing item
-                        a *= r;
-                        L *= r;
-                        M = ms;
-                    }
-                    const float f = exp2f(ms - M);
-                    a = fmaf(as, f, a);
-                    L = fmaf(ls, f, L);
+                float M = -INFINITY;
+                for (int it = 0; it < items_of_group; ++it) M = fmaxf(M, ms_s[it * G + hh]);
+                // one pass in item order
+                float acc = 0.0f, L = 0.0f;
+#pragma unroll 8
+                for (int it = 0; it < items_of_group; ++it) {
+                    const float ms = ms_s[it * G + hh];
+                    const float f = ms == -INFINITY ? 0.0f : exp2f(ms - M);
+                    acc = fmaf(__ldcg(gp + ((long long)it * G + hh) * kPartialFloats + 2 + e), f, acc);
+                    L = fmaf(ls_s[it * G + hh], f, L);
                 }
                 const long long unit = (long long)b * geo.n_q_heads + g * G + hh;
-                out[unit * kHeadDim + e] = L > 0.0f ? a / L : 0.0f;
+                out[unit * kHeadDim + e] = L > 0.0f ? acc / L : 0.0f;
                 if (e == 0 && diag) diag[unit].lse = (M + log2f(L)) * 0.6931471805599453f;
             }
         }
