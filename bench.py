@@ -335,14 +335,19 @@ def run_ours(args):
         time.sleep(0.25)
         t_wall0 = time.time()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
         e0.record(stream)
-        for _ in range(args.steps):
+        for k in range(args.steps):
             step()
+            marks[k].record(stream)       # per-step spread only; the figure of merit is e0 -> e1
         e1.record(stream)
         barrier()
         t_wall1 = time.time()
         ms_total = max_over_ranks(e0.elapsed_time(e1), world, dev)
         ms_per_step = ms_total / args.steps
+        per_step = np.array([a.elapsed_time(b) for a, b in zip([e0] + marks[:-1], marks)])
+        step_spread = {"median_ms": float(np.median(per_step)), "p10_ms": float(np.percentile(per_step, 10)),
+                       "p90_ms": float(np.percentile(per_step, 90))}
         # keep the GPU loaded a little longer if the region was too short to sample clocks
         if t_wall1 - t_wall0 < 0.5:
             t_end = time.time() + 0.6
@@ -503,6 +508,16 @@ def run_ours(args):
         cpu_baseline = {"value": sec * 1e6 / shape.batch, "unit": UNIT, "cores": cores, "kind": "oracle",
                         "sample": f"layer 0 of {L}, all {shape.batch} sequences, {reps} repetitions of one "
                                   f"oracle decode step (summaries prebuilt)"}
+        # the same oracle step on one thread, and the oracle's dense definition on all threads, a few
+        # repetitions each (context for the figure above, same unit)
+        import oracle
+        oracle.set_num_threads(1)
+        sec1, reps1, _ = oracle_layer_time(w0, reps_budget_s=4.0)
+        oracle.set_num_threads(cores)
+        secd, repsd, _ = oracle_layer_time(w0, reps_budget_s=4.0, dense=True)
+        cpu_baseline["single_thread_value"] = sec1 * 1e6 / shape.batch
+        cpu_baseline["dense_definition_value"] = secd * 1e6 / shape.batch
+        cpu_baseline["extra_samples"] = f"{reps1} single-thread repetitions, {repsd} dense repetitions of the same layer"
 
     value = us_per_token_per_layer(ms_per_step, world, shape.batch, L)
     line = {
@@ -523,6 +538,7 @@ def run_ours(args):
                             ("Frank-Wolfe" if args.solver == "fw" else "entropic mirror-descent") +
                             " iterations -> dense fallback")},
         "latency_us_per_layer": ms_per_step * 1e3 / L,
+        "step_spread": step_spread,
         "per_kernel_us": per_kernel, "closed_form_latency_us_per_layer": closed_form_us_per_layer,
         "fallback_fraction_last_layer": fb_count / units,
         "summary_build_ms_per_layer": summary_ms_per_layer,

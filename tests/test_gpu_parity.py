@@ -35,6 +35,14 @@ def test_small_ragged(hq, hkv, needles):
     assert 0.0 <= stats["fallback_fraction"] <= 1.0
 
 
+@pytest.mark.parametrize("mode", ["per_qhead_round_robin", "unit_literal"])
+def test_other_needle_layouts(mode):
+    # needles aligned to one head of a group at a time (the heads of a group then route to different
+    # pages: no page sharing), and the literal unit-vector needle that iid keys out-score
+    w = make_workload(spec(seq_lens=(2500, 900), needles=8, P=6, K_c=64, needle_mode=mode), seed=220)
+    compare(w, run_gpu(w))
+
+
 def test_several_tiles_and_ragged_tail():
     # 5 sequences with lengths around page and 32-page-block boundaries, several scan blocks
     lens = (16 * 32 * 3 + 5, 16 * 32, 16 * 33 + 15, 1, 16)
