@@ -48,6 +48,9 @@ def parse_args():
     ap.add_argument("--certified", action="store_true",
                     help="time vsa_decode_step_certified (routing certificate computed, certified gap decides the "
                          "fallback) instead of vsa_decode_step")
+    ap.add_argument("--expand", type=int, default=None,
+                    help="with --certified: retry the refused units with this many routed pages before the dense "
+                         "pass (vsa_decode_step_certified_expand)")
     ap.add_argument("--solver", default="eg", choices=["eg", "fw"],
                     help="with --solver-iters: entropic mirror descent (eg) or Frank-Wolfe with exact line search (fw)")
     ap.add_argument("--solver-iters", type=int, default=None,
@@ -279,7 +282,10 @@ def run_ours(args):
     cert = radii = None
     if args.certified:
         cert = B.alloc_cert(units, dev)
-        ws = B.alloc_workspace(shape, P, K_c, B.VSA_WS_STEP_CERTIFIED, dev)
+        ws = B.alloc_workspace(shape, args.expand or P, K_c,
+                               B.VSA_WS_STEP_EXPAND if args.expand else B.VSA_WS_STEP_CERTIFIED, dev)
+        if args.expand:
+            routed = torch.empty((shape.batch, shape.n_q_heads, args.expand), dtype=torch.int32, device=dev)
         radii = []
         for w, s_ in zip(layers, summaries):      # cache maintenance, like the summaries
             r = torch.zeros((shape.num_pool_pages, shape.n_kv_heads), dtype=torch.float32, device=dev)
@@ -291,6 +297,10 @@ def run_ours(args):
         if args.dense_baseline:
             B.vsa_dense_decode_fallback(shape, w.q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, None, None,
                                         eps, out, diag, ws_dense)
+        elif cert is not None and args.expand:
+            B.vsa_decode_step_certified_expand(shape, w.q, s, radii[i % distinct], w.k_cache, w.v_cache, w.block_table,
+                                               w.seq_lens, P, args.expand, K_c, eps, tau, out, diag, cert, routed,
+                                               flist, fcount, ws)
         elif cert is not None:
             B.vsa_decode_step_certified(shape, w.q, s, radii[i % distinct], w.k_cache, w.v_cache, w.block_table,
                                         w.seq_lens, P, K_c, eps, tau, out, diag, cert, routed, flist, fcount, ws)
@@ -532,7 +542,9 @@ def run_ours(args):
                          f"{(scan_bytes + sparse_bytes) * distinct / 1e6:.0f} MB touched per pass over them",
                    "launch": "cuda graph replay of the whole step" if use_graph else "plain stream launches",
                    "path": "dense split-K baseline" if args.dense_baseline else
-                           ("route -> sparse with routing certificate -> dense fallback" if cert is not None else
+                           ((f"route -> sparse with routing certificate -> retry of the refused units with "
+                             f"{args.expand} pages -> dense fallback") if cert is not None and args.expand else
+                            "route -> sparse with routing certificate -> dense fallback" if cert is not None else
                             "route -> sparse -> dense fallback" if solve is None else
                             f"route -> sparse with {args.solver_iters} " +
                             ("Frank-Wolfe" if args.solver == "fw" else "entropic mirror-descent") +

@@ -99,6 +99,7 @@ typedef struct {
 #define VSA_WS_DENSE 3
 #define VSA_WS_STEP 4
 #define VSA_WS_STEP_CERTIFIED 5
+#define VSA_WS_STEP_EXPAND 6
 
 /*
  * Page summaries (Sec. 7 step 1: "coarse page summaries k_page"; the paper leaves them
@@ -296,6 +297,25 @@ int vsa_decode_step_certified(const vsa_shape_t* shape, const void* q, const voi
                               float* out, vsa_diag_t* diag, vsa_cert_t* cert, int32_t* routed_pages,
                               int32_t* fallback_list, int32_t* fallback_count, void* ws, size_t ws_bytes,
                               void* stream);
+
+/*
+ * The certified step with one round of "paged expansion" (App. E: when the certificate fails, enlarge
+ * S until it passes) before anything falls back to the dense pass: every unit is first processed
+ * with P routed pages; the units whose certificate fails are processed again with P_expand > P
+ * pages (same K_c) from the page scores of the same scan; what still fails goes to the dense pass.
+ * out, diag and cert of a unit are those of its last sparse pass (dense rows for the final fallback
+ * list).  routed_pages: device int32 [batch][n_q_heads][P_expand]; a unit's row holds the pages of its
+ * last pass, -1 padded (so a row with more than P entries marks a unit that was retried).
+ *   ws: device scratch of vsa_workspace_bytes(shape, P_expand, K_c, VSA_WS_STEP_EXPAND) bytes.
+ *   P < P_expand <= 128; K_c <= P * page_size; shapes as for vsa_decode_step_certified.
+ */
+int vsa_decode_step_certified_expand(const vsa_shape_t* shape, const void* q, const void* summaries,
+                                     const float* radii, const void* k_cache, const void* v_cache,
+                                     const int32_t* block_table, const int32_t* seq_lens, int32_t P,
+                                     int32_t P_expand, int32_t K_c, float epsilon, float gap_threshold, float* out,
+                                     vsa_diag_t* diag, vsa_cert_t* cert, int32_t* routed_pages,
+                                     int32_t* fallback_list, int32_t* fallback_count, void* ws, size_t ws_bytes,
+                                     void* stream);
 
 /*
  * vsa_decode_step with CUDA events recorded on `stream` between its kernels, for per-kernel

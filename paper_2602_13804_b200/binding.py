@@ -16,7 +16,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libvsa.so")
 
-VSA_WS_ROUTE, VSA_WS_SPARSE, VSA_WS_DENSE, VSA_WS_STEP, VSA_WS_STEP_CERTIFIED = 1, 2, 3, 4, 5
+VSA_WS_ROUTE, VSA_WS_SPARSE, VSA_WS_DENSE, VSA_WS_STEP, VSA_WS_STEP_CERTIFIED, VSA_WS_STEP_EXPAND = 1, 2, 3, 4, 5, 6
 DIAG_BYTES = 32
 DIAG_FIELDS = ("delta", "delta12", "s_max", "lse", "leak_bound", "n_candidates", "fallback", "status")
 
@@ -88,6 +88,9 @@ def lib() -> C.CDLL:
                                                    vp, vp, vp, sz, vp]
         _lib.vsa_append_kv.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         _lib.vsa_append_kv.restype = C.c_int
+        _lib.vsa_decode_step_certified_expand.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, f32, f32, vp,
+                                                          vp, vp, vp, vp, vp, vp, sz, vp]
+        _lib.vsa_decode_step_certified_expand.restype = C.c_int
         _lib.vsa_build_page_radii.restype = C.c_int
         _lib.vsa_decode_step_certified.restype = C.c_int
         for name in ("vsa_build_page_summaries", "vsa_route_pages", "vsa_sparse_decode",
@@ -260,6 +263,19 @@ def vsa_decode_step_certified(shape, q, summaries, radii, k_cache, v_cache, bloc
                                            _ptr(fallback_list), _ptr(fallback_count), _ptr(ws),
                                            0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
            "vsa_decode_step_certified")
+
+
+def vsa_decode_step_certified_expand(shape, q, summaries, radii, k_cache, v_cache, block_table, seq_lens, P, P_expand,
+                                     K_c, epsilon, gap_threshold, out, diag, cert, routed_pages, fallback_list,
+                                     fallback_count, ws, stream=None) -> None:
+    _check(lib().vsa_decode_step_certified_expand(C.byref(shape), _ptr(q), _ptr(summaries), _ptr(radii),
+                                                  _ptr(k_cache), _ptr(v_cache), _ptr(block_table), _ptr(seq_lens),
+                                                  P, P_expand, K_c, epsilon, gap_threshold, _ptr(out), _ptr(diag),
+                                                  _ptr(cert), _ptr(routed_pages), _ptr(fallback_list),
+                                                  _ptr(fallback_count), _ptr(ws),
+                                                  0 if ws is None else ws.numel() * ws.element_size(),
+                                                  _stream(stream)),
+           "vsa_decode_step_certified_expand")
 
 
 def vsa_decode_step_timed(shape, q, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon,

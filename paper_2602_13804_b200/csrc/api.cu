@@ -104,6 +104,10 @@ size_t step_route_part(const Geometry& g) { return align_up(vsa::route_workspace
 size_t step_rad_offset(const Geometry& g) { return step_route_part(g) + align_up(vsa::dense_workspace_bytes(g), 256); }
 size_t step_rad_bytes(const Geometry& g) { return (size_t)g.batch * g.n_kv_heads * g.max_pages * sizeof(float); }
 
+// expanding step: the certified layout followed by the retry list (one int per unit) and its count
+size_t step_retry_offset(const Geometry& g) { return align_up(step_rad_offset(g) + step_rad_bytes(g), 256); }
+size_t step_retry_bytes(const Geometry& g) { return ((size_t)g.batch * g.n_q_heads + 4) * sizeof(int32_t); }
+
 int cuda_rc(cudaError_t e) { return e == cudaSuccess ? VSA_OK : VSA_ERR_CUDA; }
 
 }  // namespace
@@ -137,6 +141,7 @@ size_t vsa_workspace_bytes(const vsa_shape_t* shape, int32_t P, int32_t K_c, int
         case VSA_WS_DENSE: return vsa::dense_workspace_bytes(g);
         case VSA_WS_STEP: return step_route_part(g) + vsa::dense_workspace_bytes(g);
         case VSA_WS_STEP_CERTIFIED: return step_rad_offset(g) + step_rad_bytes(g);
+        case VSA_WS_STEP_EXPAND: return step_retry_offset(g) + step_retry_bytes(g);
         default: return 0;
     }
 }
@@ -386,6 +391,56 @@ int vsa_decode_step_certified(const vsa_shape_t* shape, const void* q, const voi
     return decode_step_impl(shape, q, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon,
                             gap_threshold, out, diag, routed_pages, fallback_list, fallback_count, ws, ws_bytes,
                             stream, nullptr, 0, nullptr, radii, cert);
+}
+
+int vsa_decode_step_certified_expand(const vsa_shape_t* shape, const void* q, const void* summaries,
+                                     const float* radii, const void* k_cache, const void* v_cache,
+                                     const int32_t* block_table, const int32_t* seq_lens, int32_t P,
+                                     int32_t P_expand, int32_t K_c, float epsilon, float gap_threshold, float* out,
+                                     vsa_diag_t* diag, vsa_cert_t* cert, int32_t* routed_pages,
+                                     int32_t* fallback_list, int32_t* fallback_count, void* ws, size_t ws_bytes,
+                                     void* stream)
+{
+    Geometry g;
+    int rc = make_geometry(shape, &g);
+    if (rc) return rc;
+    if ((rc = check_routing_sizes(g, P, K_c, true))) return rc;
+    if ((rc = check_routing_sizes(g, P_expand, K_c, true))) return rc;
+    if (P_expand <= P) return VSA_ERR_INVALID_ARGUMENT;
+    if ((rc = check_epsilon(epsilon))) return rc;
+    if (isnan(gap_threshold)) return VSA_ERR_INVALID_ARGUMENT;
+    if (!q || !summaries || !radii || !k_cache || !v_cache || !block_table || !seq_lens || !out || !diag || !cert ||
+        !routed_pages || !fallback_list || !fallback_count || !ws)
+        return VSA_ERR_INVALID_ARGUMENT;
+    if (!aligned16(q) || !aligned16(summaries) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(ws))
+        return VSA_ERR_MISALIGNED;
+    if (g.max_pages > vsa::sparse_register_select_max_pages((long long)g.batch * g.n_q_heads))
+        return VSA_ERR_UNSUPPORTED_SHAPE;
+    if (ws_bytes < step_retry_offset(g) + step_retry_bytes(g)) return VSA_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = (cudaStream_t)stream;
+    void* ws_dense = (char*)ws + step_route_part(g);
+    float* rad_logical = (float*)((char*)ws + step_rad_offset(g));
+    int32_t* retry_list = (int32_t*)((char*)ws + step_retry_offset(g));
+    int32_t* retry_count = retry_list + (size_t)g.batch * g.n_q_heads;
+    if (cudaMemsetAsync(retry_count, 0, sizeof(int32_t), st) != cudaSuccess) return VSA_ERR_CUDA;
+    // the scan clears the final fallback counter and the dense tickets
+    cudaError_t e = vsa::launch_route_scan(g, q, summaries, block_table, seq_lens, ws, fallback_count,
+                                           vsa::dense_tickets(ws_dense), vsa::dense_ticket_count(g), st, radii,
+                                           rad_logical);
+    if (e != cudaSuccess) return VSA_ERR_CUDA;
+    // first pass over every unit with P pages: the units it cannot certify go to the retry list
+    e = vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, routed_pages, (const float*)ws, P, K_c,
+                           epsilon, gap_threshold, out, diag, retry_list, retry_count, st, 0, nullptr, rad_logical,
+                           cert, 1, nullptr, nullptr, P_expand);
+    if (e != cudaSuccess) return VSA_ERR_CUDA;
+    // second pass over the listed units only, with P_expand pages: what still fails goes to the dense pass
+    e = vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, routed_pages, (const float*)ws, P_expand,
+                           K_c, epsilon, gap_threshold, out, diag, fallback_list, fallback_count, st, 0, nullptr,
+                           rad_logical, cert, 1, retry_list, retry_count, P_expand);
+    if (e != cudaSuccess) return VSA_ERR_CUDA;
+    e = vsa::launch_dense(g, q, k_cache, v_cache, block_table, seq_lens, fallback_list, fallback_count, epsilon,
+                          out, diag, ws_dense, st, /*tickets_cleared=*/true);
+    return cuda_rc(e);
 }
 
 int vsa_decode_step_timed(const vsa_shape_t* shape, const void* q, const void* summaries, const void* k_cache,

@@ -110,7 +110,9 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                      const float* __restrict__ page_scores, int P, int K_c, float epsilon, float gap_threshold,
                      float* __restrict__ out, vsa_diag_t* __restrict__ diag, int32_t* __restrict__ fallback_list,
                      int32_t* __restrict__ fallback_count, int solver_iters, vsa_solve_t* __restrict__ solve,
-                     const float* __restrict__ rad_logical, vsa_cert_t* __restrict__ cert)
+                     const float* __restrict__ rad_logical, vsa_cert_t* __restrict__ cert,
+                     const int32_t* __restrict__ unit_list, const int32_t* __restrict__ unit_count,
+                     int routed_stride)
 {
     constexpr int WARPS = THREADS / 32, GROUPS = 2 * WARPS;
     static_assert(SOLVE == 0 || THREADS == 256, "the solve maps one candidate to each of 256 lanes");
@@ -122,7 +124,18 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     uint32_t* region = smem_raw + 2 * P;    // page-selection scratch first, token-phase arrays afterwards
     const int N = P * kPageSize;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, c = lane & 15, gi = lane >> 4;
-    const long long unit = blockIdx.x;
+    // unit_list != nullptr: block i handles unit_list[i] for i < *unit_count (a retry pass over the units
+    // an earlier pass of the same step listed); the list is that pass's product, so it is read after
+    // the wait
+    long long unit = blockIdx.x;
+    if (unit_list) {
+        pdl_wait();
+        if ((int)blockIdx.x >= __ldcg(unit_count)) {
+            pdl_launch_dependents();
+            return;
+        }
+        unit = __ldcg(unit_list + blockIdx.x);
+    }
     const int b = (int)(unit / geo.n_q_heads), h = (int)(unit % geo.n_q_heads), g = h / geo.group;
     VSA_PROBE_T0(50);
     // Loads that depend on nothing computed in this step go out before the wait on the preceding
@@ -166,7 +179,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         if (SOLVE && tid == 0) solve[unit] = vsa_solve_t{0.0f, 0.0f, 0.0f, 0.0f};
         if (CERT && tid == 0) cert[unit] = vsa_cert_t{0.0f, 0.0f, 0.0f, 0};
         if (PAGE_KPT != 0)
-            for (int t = tid; t < P; t += THREADS) routed_pages[unit * P + t] = -1;
+            for (int t = tid; t < routed_stride; t += THREADS) routed_pages[unit * routed_stride + t] = -1;
         return;
     }
     const int nb = (T + kPageSize - 1) / kPageSize;
@@ -209,8 +222,9 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         } else {
             np = select_top_pages(page_scores + unit * geo.max_pages, nb, P, ps);
         }
+        for (int t = P + tid; t < routed_stride; t += THREADS) routed_pages[unit * routed_stride + t] = -1;
         for (int t = tid; t < P; t += THREADS) {
-            routed_pages[unit * P + t] = t < np ? ps.win_idx[t] : -1;
+            routed_pages[unit * routed_stride + t] = t < np ? ps.win_idx[t] : -1;
             int l = INT_MAX, phys = -1;
             if (t < np) {
                 l = ps.asc_idx[t];
@@ -226,7 +240,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     } else {
         int32_t* raw = (int32_t*)region;   // staging; dead before the token phase reuses the region
         for (int t = tid; t < P; t += THREADS) {
-            const int l = routed_pages[unit * P + t];
+            const int l = routed_pages[unit * routed_stride + t];
             raw[t] = (l >= 0 && l < nb) ? l : INT_MAX;
         }
         __syncthreads();
@@ -789,6 +803,8 @@ struct SparseArgs {
     vsa_solve_t* solve;   // non-null: an iterative-solve variant of the kernel
     const float* rad_logical;
     vsa_cert_t* cert;     // non-null: the certificate variant (fused register variants only)
+    const int32_t *unit_list, *unit_count;   // non-null: only the listed units (blocks beyond the count exit)
+    int routed_stride;                       // row stride of routed_pages (>= P)
     cudaStream_t stream;
 };
 
@@ -804,7 +820,7 @@ cudaError_t launch_variant(const SparseArgs& a)
     return launch_pdl(sparse_decode_kernel<THREADS, PAGE_KPT, TOK_KPT, SOLVE, CERT>, dim3(units), dim3(THREADS),
                       a.smem, a.stream, a.g, a.q, a.k, a.v, a.block_table, a.seq_lens, a.routed_pages, a.page_scores,
                       a.P, a.K_c, a.epsilon, a.gap_threshold, a.out, a.diag, a.fallback_list, a.fallback_count,
-                      a.solver_iters, a.solve, a.rad_logical, a.cert);
+                      a.solver_iters, a.solve, a.rad_logical, a.cert, a.unit_list, a.unit_count, a.routed_stride);
 }
 
 template <int THREADS, int PAGE_KPT, int TOK_KPT>
@@ -874,7 +890,7 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
                           const float* page_scores, int P, int K_c, float epsilon, float gap_threshold, float* out,
                           vsa_diag_t* diag, int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream,
                           int solver_iters, vsa_solve_t* solve, const float* rad_logical, vsa_cert_t* cert,
-                          int solver_kind)
+                          int solver_kind, const int32_t* unit_list, const int32_t* unit_count, int routed_stride)
 {
     SparseArgs a;
     a.g = g;
@@ -887,6 +903,9 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
     a.solve = solve;
     a.rad_logical = rad_logical;
     a.cert = cert;
+    a.unit_list = unit_list;
+    a.unit_count = unit_count;
+    a.routed_stride = routed_stride > 0 ? routed_stride : P;
     a.q = (const uint16_t*)q;
     a.k = (const uint16_t*)k_cache;
     a.v = (const uint16_t*)v_cache;

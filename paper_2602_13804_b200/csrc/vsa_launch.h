@@ -66,12 +66,15 @@ cudaError_t launch_route_select(const Geometry& g, const void* ws, const int32_t
 // candidates come from solver_iters iterations of entropic mirror descent (solver_kind 1) or of
 // Frank-Wolfe with exact line search (solver_kind 2), K_c <= 256.  cert != nullptr
 // (with page_scores and rad_logical): the certified gap is computed and decides the fallback.
+// unit_list / unit_count (device): only the listed units are processed; routed_stride: row stride of
+// routed_pages when it is wider than P (0 = P), the tail of a row is filled with -1.
 cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache, const void* v_cache,
                           const int32_t* block_table, const int32_t* seq_lens, int32_t* routed_pages,
                           const float* page_scores, int P, int K_c, float epsilon, float gap_threshold, float* out,
                           vsa_diag_t* diag, int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream,
                           int solver_iters = 0, vsa_solve_t* solve = nullptr, const float* rad_logical = nullptr,
-                          vsa_cert_t* cert = nullptr, int solver_kind = 1);
+                          vsa_cert_t* cert = nullptr, int solver_kind = 1, const int32_t* unit_list = nullptr,
+                          const int32_t* unit_count = nullptr, int routed_stride = 0);
 // widest block table for which the fused kernel keeps every page score of a unit in registers (the
 // certificate variant exists for those shapes only); `units` = batch * n_q_heads
 int sparse_register_select_max_pages(long long units);

@@ -104,3 +104,21 @@ class SparsePagedDecoder:
                                       self.diag, self.solve, self.routed_pages, self.fallback_list,
                                       self.fallback_count, self.ws)
         return self.out
+
+    def step_certified_expand(self, q, summaries, radii, k_cache, v_cache, block_table, seq_lens,
+                              P_expand: int) -> torch.Tensor:
+        """The certified step with one expansion round: refused units are retried with `P_expand` pages
+        before the dense pass.  self.routed_pages_expand ([batch, heads, P_expand]) holds each unit's
+        pages of its last pass."""
+        if not hasattr(self, "cert"):
+            self.cert = B.alloc_cert(self.units, self.device)
+        if getattr(self, "_expand_P", None) != int(P_expand):
+            self._expand_P = int(P_expand)
+            self.ws_expand = B.alloc_workspace(self.shape, self._expand_P, self.K_c, B.VSA_WS_STEP_EXPAND, self.device)
+            self.routed_pages_expand = torch.empty((self.shape.batch, self.shape.n_q_heads, self._expand_P),
+                                                   dtype=torch.int32, device=self.device)
+        B.vsa_decode_step_certified_expand(self.shape, q, summaries, radii, k_cache, v_cache, block_table, seq_lens,
+                                           self.P, self._expand_P, self.K_c, self.epsilon, self.gap_threshold,
+                                           self.out, self.diag, self.cert, self.routed_pages_expand,
+                                           self.fallback_list, self.fallback_count, self.ws_expand)
+        return self.out

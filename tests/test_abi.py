@@ -156,6 +156,17 @@ def test_certificate_argument_validation(lib):
     assert call(ws_bytes=plain) == -3
     wide = B.make_shape(40, 8, 2, 9000, 1 << 16)     # 320 units > SMs: 256 threads hold at most 8192 page scores
     assert call(shape=wide) == -2
+    exp = lib.vsa_decode_step_certified_expand
+
+    def call_e(P=4, P2=8, K_c=16, ws_bytes=1 << 40, cert=FAKE):
+        return exp(s, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, P, P2, K_c, 1.0, 0.0, FAKE, FAKE, cert, FAKE, FAKE, FAKE,
+                   FAKE, ws_bytes, None)
+
+    assert call_e(P2=4) == -1 and call_e(P2=3) == -1      # the expansion must add pages
+    assert call_e(P2=129) == -2
+    assert call_e(cert=None) == -1
+    assert call_e(ws_bytes=B.vsa_workspace_bytes(ok, 4, 16, B.VSA_WS_STEP_CERTIFIED)) == -3
+    assert B.vsa_workspace_bytes(ok, 8, 16, B.VSA_WS_STEP_EXPAND) >= need + 16 * 4
     assert C.sizeof(C.c_int32) * len(B.CERT_FIELDS) == 16
 
 

@@ -179,3 +179,74 @@ def test_append_keeps_cache_summaries_and_radii_in_step_with_a_full_rebuild():
     owned = np.concatenate([bt[b, : (int(sl[b]) + 15) // 16] for b in range(3)])
     assert np.array_equal(bits(summ)[owned], o_sum[owned])
     assert np.array_equal(radii.cpu().numpy()[owned].view(np.uint32), o_rad[owned].view(np.uint32))
+
+
+def test_expansion_retries_the_refused_units_with_more_pages_before_the_dense_pass():
+    """Two to twenty needles per (sequence, kv head) against six routed pages: units with few needles
+    certify in the first pass, the others miss needle pages and are refused; with P_expand = 24 every
+    needle page is routed and all but one of them pass; that one goes to the dense pass.  The composite
+    expectation is assembled from the oracle's parts."""
+    P, P2, K_c = 6, 24, 64
+    w = make_workload(spec(batch=6, seq_lens=(3000, 2000, 700, 1500, 2600, 900), P=P, K_c=K_c, needles=(2, 20)),
+                      seed=421)
+    wd = w.to(DEV)
+    shape = B.shape_of(wd.q, wd.k_cache, wd.block_table)
+    units = shape.batch * shape.n_q_heads
+    summ = torch.zeros((shape.num_pool_pages, shape.n_kv_heads, 128), dtype=torch.bfloat16, device=DEV)
+    B.vsa_build_page_summaries(shape, wd.k_cache, wd.block_table, wd.seq_lens, None, summ)
+    radii = torch.zeros((shape.num_pool_pages, shape.n_kv_heads), dtype=torch.float32, device=DEV)
+    B.vsa_build_page_radii(shape, wd.k_cache, summ, wd.block_table, wd.seq_lens, None, radii)
+    out = torch.full((shape.batch, shape.n_q_heads, 128), float("nan"), dtype=torch.float32, device=DEV)
+    diag, cert = B.alloc_diag(units, DEV), B.alloc_cert(units, DEV)
+    flist = torch.full((units,), -1, dtype=torch.int32, device=DEV)
+    fcount = torch.full((1,), 99, dtype=torch.int32, device=DEV)
+    routed = torch.full((shape.batch, shape.n_q_heads, P2), -7, dtype=torch.int32, device=DEV)
+    ws = B.alloc_workspace(shape, P2, K_c, B.VSA_WS_STEP_EXPAND, DEV)
+    for _ in range(2):      # twice: the retry list and its counter are reset by the call itself
+        B.vsa_decode_step_certified_expand(shape, wd.q, summ, radii, wd.k_cache, wd.v_cache, wd.block_table,
+                                           wd.seq_lens, P, P2, K_c, w.epsilon, w.gap_threshold, out, diag, cert,
+                                           routed, flist, fcount, ws)
+    torch.cuda.synchronize()
+
+    q, K, V, bt, sl = host_arrays(w)
+    geo = geometry(w)
+    Bn, H = geo.batch, geo.n_q_heads
+    o_sum = oracle.build_summaries(geo, K, bt, sl)
+    o_rad = oracle.build_radii(geo, K, o_sum, bt, sl)
+
+    def one_pass(p):
+        rt = oracle.route(geo, q, o_sum, bt, sl, p, want_all_scores=True)
+        sp = oracle.sparse(geo, q, K, V, bt, sl, rt.pages, K_c, w.epsilon, w.gap_threshold)
+        ce = oracle.certify(geo, q, o_rad, bt, sl, rt, sp, w.epsilon, w.gap_threshold)
+        refused = (ce.certified == 0) & (sp.n_candidates < sl[:, None])
+        return rt, sp, ce, refused
+
+    rt1, sp1, ce1, ref1 = one_pass(P)
+    rt2, sp2, ce2, ref2 = one_pass(P2)
+    assert ref1.any() and not ref1.all(), "the workload should refuse some units with P pages and keep others"
+    final_fb = ref1 & ref2
+    assert (ref1 & ~ref2).any(), "the expansion should rescue some units"
+    assert final_fb.any(), "and leave at least one to the dense pass"
+    # routed pages: first pass rows padded with -1, retried rows from the second pass
+    want_routed = np.full((Bn, H, P2), -1, np.int32)
+    want_routed[:, :, :P] = rt1.pages
+    want_routed[ref1] = rt2.pages[ref1]
+    assert np.array_equal(routed.cpu().numpy(), want_routed)
+    c = {k: v.numpy().reshape(Bn, H) for k, v in B.cert_to_dict(cert).items()}
+    d = {k: v.numpy().reshape(Bn, H) for k, v in B.diag_to_dict(diag).items()}
+    for name, a1, a2 in (("delta_cert", ce1.delta_cert, ce2.delta_cert), ("ub_unrouted", ce1.ub_unrouted, ce2.ub_unrouted)):
+        want = np.where(ref1, a2, a1)
+        assert np.array_equal(c[name].view(np.uint32), want.view(np.uint32)), name
+    assert np.array_equal(c["certified"], np.where(ref1, ce2.certified, ce1.certified))
+    assert np.array_equal(d["n_candidates"], np.where(ref1, sp2.n_candidates, sp1.n_candidates))
+    assert np.array_equal(d["delta"], np.where(ref1, sp2.delta, sp1.delta))
+    assert np.array_equal(d["fallback"], final_fb.astype(np.int32))
+    n = int(fcount.item())
+    assert np.array_equal(np.sort(flist[:n].cpu().numpy()), np.nonzero(final_fb.reshape(-1))[0])
+    got = out.cpu().numpy().reshape(Bn * H, -1)
+    first, second, dense_rows = (~ref1).reshape(-1), (ref1 & ~ref2).reshape(-1), final_fb.reshape(-1)
+    check_out(got[first], sp1.out.reshape(Bn * H, -1)[first], "units certified by the first pass")
+    check_out(got[second], sp2.out.reshape(Bn * H, -1)[second], "units certified after the expansion")
+    if dense_rows.any():
+        dn = oracle.dense(geo, q, K, V, bt, sl, w.epsilon, unit_mask=final_fb.astype(np.int32))
+        check_out(got[dense_rows], dn.out.reshape(Bn * H, -1)[dense_rows], "units that fell back")
