@@ -1,0 +1,19 @@
+// Fused sparse pass, closed-form weights: the kernel variants without iterative solve or certificate.
+#include "sparse_kernel.cuh"
+
+namespace vsa {
+
+cudaError_t launch_sparse_plain(const SparseArgs& a, int threads)
+{
+    return threads == 512 ? launch_threads<512, 0, false>(a) : launch_threads<256, 0, false>(a);
+}
+
+}  // namespace vsa
+
+#ifdef VSA_ENABLE_PROBES
+// development aid: the phase probes of this translation unit's kernels
+extern "C" int vsa_probe_read(long long* host64)
+{
+    return (int)cudaMemcpyFromSymbol(host64, vsa_probe_buf, sizeof(long long) * 64);
+}
+#endif
