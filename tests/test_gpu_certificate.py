@@ -250,3 +250,42 @@ def test_expansion_retries_the_refused_units_with_more_pages_before_the_dense_pa
     if dense_rows.any():
         dn = oracle.dense(geo, q, K, V, bt, sl, w.epsilon, unit_mask=final_fb.astype(np.int32))
         check_out(got[dense_rows], dn.out.reshape(Bn * H, -1)[dense_rows], "units that fell back")
+
+
+def test_certified_step_with_bad_inputs_sets_status_without_trapping():
+    w = make_workload(spec(seq_lens=(300, 177, 90), needles=0), seed=430)
+    wd = w.to(DEV)
+    shape = B.shape_of(wd.q, wd.k_cache, wd.block_table)
+    units = shape.batch * shape.n_q_heads
+    summ = torch.zeros((shape.num_pool_pages, shape.n_kv_heads, 128), dtype=torch.bfloat16, device=DEV)
+    B.vsa_build_page_summaries(shape, wd.k_cache, wd.block_table, wd.seq_lens, None, summ)
+    radii = torch.zeros((shape.num_pool_pages, shape.n_kv_heads), dtype=torch.float32, device=DEV)
+    B.vsa_build_page_radii(shape, wd.k_cache, summ, wd.block_table, wd.seq_lens, None, radii)
+    sl = wd.seq_lens.clone()
+    sl[1] = shape.max_pages_per_seq * 16 + 5          # longer than its block-table row
+    sl[2] = 0                                         # empty
+    out = torch.full((shape.batch, shape.n_q_heads, 128), float("nan"), dtype=torch.float32, device=DEV)
+    diag, cert = B.alloc_diag(units, DEV), B.alloc_cert(units, DEV)
+    cert.fill_(-1)
+    flist = torch.full((units,), -1, dtype=torch.int32, device=DEV)
+    fcount = torch.full((1,), 99, dtype=torch.int32, device=DEV)
+    routed = torch.full((shape.batch, shape.n_q_heads, 4), -7, dtype=torch.int32, device=DEV)
+    ws = B.alloc_workspace(shape, 4, 40, B.VSA_WS_STEP_CERTIFIED, DEV)
+    B.vsa_decode_step_certified(shape, wd.q, summ, radii, wd.k_cache, wd.v_cache, wd.block_table, sl, 4, 40,
+                                w.epsilon, -math.inf, out, diag, cert, routed, flist, fcount, ws)
+    # the append skips the same sequences
+    k_new = torch.ones((3, 2, 128), dtype=torch.bfloat16, device=DEV)
+    before = wd.k_cache.clone()
+    B.vsa_append_kv(shape, k_new, k_new, wd.k_cache, wd.v_cache, wd.block_table, sl, summ, radii)
+    torch.cuda.synchronize()
+    d = B.diag_to_dict(diag)
+    st = d["status"].view(3, 8)
+    assert st[0].eq(0).all() and st[1].eq(2).all() and st[2].eq(2).all()
+    o = out.cpu().numpy()
+    assert np.isfinite(o[0]).all() and not o[1:].any()
+    c = B.cert_to_dict(cert)
+    assert c["certified"].view(3, 8)[1:].eq(0).all() and c["delta_cert"].view(3, 8)[1:].eq(0).all()
+    assert int(fcount.item()) == 0
+    assert np.all(routed.cpu().numpy()[1:] == -1)
+    changed = (wd.k_cache != before).flatten(1).any(1).nonzero().flatten().tolist()
+    assert changed == [int(wd.block_table[0, (300 - 1) // 16])]      # only sequence 0's last page was written

@@ -245,3 +245,17 @@ def test_frank_wolfe_duplicate_keys_tie_to_the_lower_position():
     w.k_cache = k
     w.gap_threshold = -math.inf
     compare_fw(w, run_fw(w, 5), 5)
+
+
+@pytest.mark.parametrize("kind", ["eg", "fw"])
+def test_solvers_with_a_single_candidate_per_unit(kind):
+    # K_c = 1: the candidate set is the best token alone; weight 1, zero gap, no step
+    w = make_workload(spec(K_c=1, P=2, seq_lens=(200, 90, 40)), seed=340)
+    w.gap_threshold = -math.inf
+    g = run_entropic(w, 3) if kind == "eg" else run_fw(w, 3)
+    if kind == "eg":
+        compare_entropic(w, g, 3)
+    else:
+        compare_fw(w, g, 3)
+    sol = np.asarray(g["solve"], dtype=np.float64).reshape(24, 4)
+    assert np.all(np.abs(sol[:, 0]) < 1e-3)
