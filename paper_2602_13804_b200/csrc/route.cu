@@ -6,6 +6,8 @@
 //   route_select_kernel  one block per (sequence, query head): exact top-P selection.
 #include <math.h>
 
+#include <algorithm>
+
 #include "vsa_device.cuh"
 #include "vsa_launch.h"
 #include "vsa_select.cuh"
@@ -17,14 +19,17 @@ namespace {
 constexpr int kScanThreads = 256;
 constexpr int kScanWarps = kScanThreads / 32;
 constexpr int kBlockPages = 32;      // pages per block-table block (one coalesced 128-byte load per warp)
-constexpr int kMaxBlocksPerWarp = 16;
+// Blocks of 32 pages one warp takes at most.  More per warp would amortise its start-up further, but
+// the launch then has fewer, longer warps and a ragged batch (whose short sequences leave most of a
+// grid sized for the longest one idle) ends on a long tail: 4 measured best from batch 16, T = 128k
+// (87.7 against 93.6 us per layer with 16) to a 64-sequence log-uniform batch (455 against 482 us).
+constexpr int kMaxBlocksPerWarp = 4;
 
 template <int G>
 struct ScanCfg {
     static constexpr int ROWS = G == 1 ? 8 : 16 / G;      // rows per half-warp per round
     static constexpr int VALS = ROWS * G;                 // (row, head) partials per lane per round (8 or 16)
     static constexpr int ROUND_PAGES = 2 * ROWS;          // pages (rows of one KV head) per warp per round
-    static constexpr int ROUNDS = kBlockPages / ROUND_PAGES;
     // ring slots per warp: a power of two (cheap slot index), about 8 KB of rows
     static constexpr int STAGES = 8192 / (ROUND_PAGES * kRowBytes) < 2 ? 2 : 8192 / (ROUND_PAGES * kRowBytes);
     static_assert((STAGES & (STAGES - 1)) == 0, "slot index is R & (STAGES - 1)");
@@ -67,7 +72,8 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
     using Cfg = ScanCfg<G>;
     constexpr int ROWS = Cfg::ROWS, VALS = Cfg::VALS, ROUND_PAGES = Cfg::ROUND_PAGES, STAGES = Cfg::STAGES;
     constexpr bool XOR_MAP = VALS == 16;
-    constexpr int kFirstBlocks = 4;   // block-table blocks fetched before the sequence length is known
+    // block-table blocks fetched before the sequence length is known: the warp's whole range
+    constexpr int kFirstBlocks = kMaxBlocksPerWarp;
     extern __shared__ __align__(16) uint8_t scan_smem[];
     VSA_PROBE_T0(47);
     const int b = blockIdx.y;
@@ -132,10 +138,6 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
 #pragma unroll
     for (int k = 0; k < kFirstBlocks; ++k)
         if (k < n_blocks) off_tab[k * kBlockPages + lane] = encode(first_entries[k], k * kBlockPages + lane);
-    for (int k = kFirstBlocks; k < n_blocks; ++k) {
-        const int i = k * kBlockPages + lane;
-        off_tab[i] = encode(i < n_pages ? bt[i] : -1, i);
-    }
     VSA_PROBE(10);
     float qf[G][8];
 #pragma unroll
@@ -263,7 +265,7 @@ size_t select_smem_bytes(const Geometry& g, int P) { return (size_t)select_pages
 int scan_blocks_per_warp(const Geometry& g)
 {
     // 32-page blocks per warp: about one resident wave of warps (2 thread blocks of 8 warps per SM
-    // on 148 SMs) when the problem is large enough, never more than kMaxBlocksPerWarp
+    // on 148 SMs) while that takes no more than kMaxBlocksPerWarp
     const long long blocks = (long long)g.batch * g.n_kv_heads * ((g.max_pages + kBlockPages - 1) / kBlockPages);
     long long k = (blocks + 2367) / 2368;
     if (k < 1) k = 1;
@@ -280,7 +282,10 @@ cudaError_t launch_scan_g(const Geometry& g, const uint16_t* q, const uint16_t* 
     const int slices = ((g.max_pages + kBlockPages - 1) / kBlockPages + bpw - 1) / bpw;
     const int warps = slices * g.n_kv_heads;
     const dim3 grid((unsigned)((warps + kScanWarps - 1) / kScanWarps), (unsigned)g.batch);
-    const size_t smem = (size_t)kScanWarps * ScanCfg<G>::WARP_BYTES;
+    // The request is padded to 81 KB so that exactly two blocks are resident per SM: with a third one
+    // fewer blocks of the kernel that follows fit beside the scan's to start early, and the step gets
+    // slower although the scan does not (measured: 30.0 against 24.8 us per layer at batch 8, T = 32k).
+    const size_t smem = std::max((size_t)kScanWarps * ScanCfg<G>::WARP_BYTES, (size_t)81 * 1024);
     static int attr_device = -1;   // per template instance: the device whose function attribute is set
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
