@@ -49,7 +49,16 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
     a.g = g;
     // no more units than SMs: one larger block per unit (latency shape); otherwise two blocks per SM.
     // The iterative solve exists in the 256-thread shape only.
-    const int threads = (!solve && (long long)g.batch * g.n_q_heads <= sm_count()) ? 512 : 256;
+    // More units than two blocks per SM hold: 128 threads, four blocks per SM.  A unit is a chain of
+    // dependent phases, so twice as many units in flight per SM gain more than each loses by having half
+    // the threads (measured 1.26x per unit): 512 units take one wave instead of two (25 against 30 us per
+    // layer at batch 16, T = 4k), 2048 units 80 against 101 us (batch 64, T = 8k).  Closed-form variants
+    // only; fused ones with the page scores in registers (32 per thread at most).
+    const long long units = (long long)g.batch * g.n_q_heads;
+    int threads = (!solve && units <= sm_count()) ? 512 : 256;
+    if (!solve && !cert && !unit_list && units > 2 * sm_count() &&
+        P <= 64 && g.max_pages <= 32 * 128)
+        threads = 128;
     a.smem = sparse_smem_bytes(g, P, K_c, page_scores != nullptr, threads, solve != nullptr);
     a.solver_iters = solver_iters;
     a.solver_kind = solver_kind;

@@ -93,8 +93,10 @@ __device__ __forceinline__ void write_failed_unit(float* out, vsa_diag_t* diag, 
     }
 }
 
-// THREADS: 256 (two blocks per SM; the throughput shape) or 512 (one block per SM; used when there
-//   are no more units than SMs, so that one unit gets twice the loads in flight and half the passes).
+// THREADS: 256 (two blocks per SM; the throughput shape), 512 (one block per SM; used when there
+//   are no more units than SMs, so that one unit gets twice the loads in flight and half the passes)
+//   or 128 (four blocks per SM; used when there are more units than two blocks per SM hold: more
+//   units in flight, fewer waves).
 // PAGE_KPT ==  0: routed_pages is an input.
 // PAGE_KPT == -1: fused with routing; page scores staged in shared memory (any block-table width).
 // PAGE_KPT  >  0: fused with routing; each thread keeps PAGE_KPT page scores in registers.
@@ -707,7 +709,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     for (int e = 0; e < 8; ++e) acc[e] = 0.0f;
     const int gidx = warp * 2 + gi;
     const uint16_t* vbase = v_cache + (long long)g * geo.head_stride + c * 8;
-    constexpr int UNR = THREADS == 256 ? 16 : 8;   // K_c = 256: every half-warp's rows in one batch
+    constexpr int UNR = THREADS == 512 ? 8 : 16;   // 256 threads, K_c = 256: every half-warp's rows in one batch
     for (int j0 = gidx; j0 < ns; j0 += GROUPS * UNR) {
         // all value rows of the batch at once; slots past the candidate count re-read the last
         // candidate with weight 0
@@ -829,8 +831,8 @@ cudaError_t launch_tok(const SparseArgs& a)
     const int N = a.P * kPageSize;
     if (N <= 2 * THREADS) return launch_variant<THREADS, PAGE_KPT, 2, SOLVE, CERT>(a);
     if (N <= 4 * THREADS) return launch_variant<THREADS, PAGE_KPT, 4, SOLVE, CERT>(a);
-    if constexpr (THREADS == 256)
-        return launch_variant<THREADS, PAGE_KPT, 8, SOLVE, CERT>(a);
+    if constexpr (THREADS <= 256)
+        return N <= 8 * THREADS ? launch_variant<THREADS, PAGE_KPT, 8, SOLVE, CERT>(a) : cudaErrorInvalidValue;
     else
         return cudaErrorInvalidValue;   // 128 pages * 16 tokens = 4 * 512: never reached
 }
@@ -849,6 +851,17 @@ cudaError_t launch_threads(const SparseArgs& a)
         return launch_tok<THREADS, -1, SOLVE, CERT>(a);
     else
         return cudaErrorInvalidValue;   // (refused by the entry point before any launch)
+}
+
+// the 128-thread shape: routed pages given or selected from scores held in registers, P <= 64 and
+// max_pages <= 4096 (the caller checks)
+inline cudaError_t launch_threads_128(const SparseArgs& a)
+{
+    if (!a.page_scores) return launch_tok<128, 0, 0, false>(a);
+    if (a.g.max_pages <= 8 * 128) return launch_tok<128, 8, 0, false>(a);
+    if (a.g.max_pages <= 16 * 128) return launch_tok<128, 16, 0, false>(a);
+    if (a.g.max_pages <= 32 * 128) return launch_tok<128, 32, 0, false>(a);
+    return cudaErrorInvalidValue;
 }
 
 }  // namespace

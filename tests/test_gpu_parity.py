@@ -200,6 +200,16 @@ def test_largest_routing_sizes():
     compare(w, run_gpu(w), dense_sample=8)
 
 
+def test_more_units_than_resident_blocks():
+    # 640 and 320 units: beyond two 256-thread blocks per SM the kernel takes its 128-thread shape, here
+    # with eight token scores per thread (P = 64) and with two (P = 8); ragged lengths, several waves
+    lens = tuple(200 + 37 * i for i in range(80))
+    w = make_workload(spec(batch=80, n_q_heads=8, n_kv_heads=2, seq_lens=lens, P=64, K_c=300, needles=4), seed=216)
+    compare(w, run_gpu(w), dense_sample=8)
+    w = make_workload(spec(batch=40, n_q_heads=8, n_kv_heads=1, seq_lens=lens[:40], P=8, K_c=40, needles=2), seed=217)
+    compare(w, run_gpu(w), dense_sample=8)
+
+
 def test_block_table_wider_than_the_register_select():
     # 9000 pages per sequence: beyond 32 scores per thread at 256 threads, within it at 512;
     # batch 40 x 4 heads = 160 units > SMs forces the 256-thread kernel and its shared-memory select
