@@ -148,8 +148,8 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     // Loads that depend on nothing computed in this step go out before the wait on the preceding
     // kernel: the sequence length, the query row (the routing kernel that precedes this one in a step
     // has read it already) and a copy of the block-table row for the page lookups that follow the
-    // selection.  The page scores, which that kernel writes, are fetched right after the wait; every
-    // index below max_pages is inside the unit's scratch row, whatever the sequence length is.
+    // selection.  The page scores, which that kernel writes, are fetched right after the wait (the
+    // sequence length, asked for before it, has arrived by then).
     const int32_t* bt = block_table + (long long)b * geo.max_pages;
     const int T = ld_ca_s32(seq_lens + b);
     const uint4 qraw = ld_nc_16B(q + unit * kHeadDim + c * 8);
@@ -162,12 +162,15 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     pdl_wait();
     pdl_launch_dependents();
     VSA_PROBE_T0(51);
+    // Only the scores of the sequence's own pages are fetched: the rest of the scratch row was not
+    // written in this step (in a ragged batch it is most of the row, and it would come from DRAM).
+    const int nb_fetch = (T > 0 && T <= geo.max_pages * kPageSize) ? (T + kPageSize - 1) / kPageSize : 0;
     float praw[PAGE_KPT > 0 ? PAGE_KPT : 1];
     if constexpr (PAGE_KPT > 0) {
 #pragma unroll
         for (int j = 0; j < PAGE_KPT; ++j) {
             const int i = tid + j * THREADS;
-            praw[j] = i < geo.max_pages ? ld_cg_f32(page_scores + unit * geo.max_pages + i) : 0.0f;
+            praw[j] = i < nb_fetch ? ld_cg_f32(page_scores + unit * geo.max_pages + i) : 0.0f;
         }
     }
     float prad[CERT ? PAGE_KPT : 1];
@@ -175,7 +178,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
 #pragma unroll
         for (int j = 0; j < PAGE_KPT; ++j) {
             const int i = tid + j * THREADS;
-            prad[j] = i < geo.max_pages
+            prad[j] = i < nb_fetch
                           ? ld_cg_f32(rad_logical + ((long long)b * geo.n_kv_heads + g) * geo.max_pages + i)
                           : 0.0f;
         }
