@@ -53,10 +53,10 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
     // dependent phases, so twice as many units in flight per SM gain more than each loses by having half
     // the threads (measured 1.26x per unit): 512 units take one wave instead of two (25 against 30 us per
     // layer at batch 16, T = 4k), 2048 units 80 against 101 us (batch 64, T = 8k).  Closed-form variants
-    // only; fused ones with the page scores in registers (32 per thread at most).
+    // (with or without the certificate) only; fused ones with the page scores in registers (32 per thread at most).
     const long long units = (long long)g.batch * g.n_q_heads;
     int threads = (!solve && units <= sm_count()) ? 512 : 256;
-    if (!solve && !cert && !unit_list && units > 2 * sm_count() &&
+    if (!solve && !unit_list && units > 2 * sm_count() &&
         P <= 64 && g.max_pages <= 32 * 128)
         threads = 128;
     a.smem = sparse_smem_bytes(g, P, K_c, page_scores != nullptr, threads, solve != nullptr);

@@ -137,6 +137,16 @@ def test_wide_block_table_and_many_units():
     compare_certified(w, run_certified(w))
 
 
+def test_more_units_than_resident_blocks_take_the_128_thread_shape():
+    # 320 units, ragged; then 2500 pages per sequence (32 page scores and radii per thread at 128 threads)
+    lens = tuple(150 + 41 * i for i in range(40))
+    w = make_workload(spec(batch=40, n_q_heads=8, n_kv_heads=2, seq_lens=lens, P=8, K_c=64, needles=3), seed=415)
+    compare_certified(w, run_certified(w))
+    w = make_workload(spec(batch=40, n_q_heads=8, n_kv_heads=4, seq_lens=(40000,) + (700,) * 39, P=16, K_c=128,
+                           needles=6), seed=416)
+    compare_certified(w, run_certified(w))
+
+
 def test_append_keeps_cache_summaries_and_radii_in_step_with_a_full_rebuild():
     """Three appended tokens per sequence (the first one opens a new page for sequence 0): rows,
     summaries and radii must equal what the oracle builds from scratch on the grown cache."""
