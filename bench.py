@@ -381,6 +381,13 @@ def run_ours(args):
             acc = np.zeros(4)
             for _ in range(2):
                 step()
+            # the timed entry point's own first call (with --solver-iters / --certified its kernels have not
+            # run yet: module load and function attributes would otherwise land between the events)
+            for i in range(L):
+                w, s = layers[i % distinct], summaries[i % distinct]
+                B.vsa_decode_step_timed(shape, w.q, s, w.k_cache, w.v_cache, w.block_table, w.seq_lens, P, K_c,
+                                        eps, tau, out, diag, routed, flist, fcount, ws, evs[i])
+            stream.synchronize()
             for _ in range(n_rep):
                 # hold the GPU for ~3 ms so that the host enqueues the whole step ahead of it:
                 # the events then bracket kernels that run back to back, not launch gaps
