@@ -56,8 +56,14 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
     // (with or without the certificate) only; fused ones with the page scores in registers (32 per thread at most).
     const long long units = (long long)g.batch * g.n_q_heads;
     int threads = (!solve && units <= sm_count()) ? 512 : 256;
-    if (!solve && !unit_list && units > 2 * sm_count() &&
-        P <= 64 && g.max_pages <= 32 * 128)
+    // Tables wider than 32 scores per thread: the 128-thread shape selects from shared memory, which loses
+    // to the 256-thread register selection when every sequence is long (99 against 88 us per layer at
+    // batch 16, T = 128k) and wins when most are short (410 against 445 us on the ragged config 4).  The
+    // lengths are not known here; what is known is the pool: when batch * max_pages exceeds it, the
+    // sequences cannot all be long.
+    const bool narrow = g.max_pages <= 32 * 128;
+    const bool cannot_all_be_long = (long long)g.batch * g.max_pages > (long long)g.pool_pages;
+    if (!solve && !unit_list && units > 2 * sm_count() && P <= 64 && (narrow || (!cert && cannot_all_be_long)))
         threads = 128;
     a.smem = sparse_smem_bytes(g, P, K_c, page_scores != nullptr, threads, solve != nullptr);
     a.solver_iters = solver_iters;

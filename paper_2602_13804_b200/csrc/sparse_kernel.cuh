@@ -856,15 +856,15 @@ cudaError_t launch_threads(const SparseArgs& a)
         return cudaErrorInvalidValue;   // (refused by the entry point before any launch)
 }
 
-// the 128-thread shape: routed pages given or selected from scores held in registers, P <= 64 and
-// max_pages <= 4096 (the caller checks)
+// the 128-thread shape (P <= 64, the caller checks): routed pages given, or selected from scores held
+// in registers (max_pages <= 4096) or staged in shared memory (wider tables)
 inline cudaError_t launch_threads_128(const SparseArgs& a)
 {
     if (!a.page_scores) return launch_tok<128, 0, 0, false>(a);
     if (a.g.max_pages <= 8 * 128) return launch_tok<128, 8, 0, false>(a);
     if (a.g.max_pages <= 16 * 128) return launch_tok<128, 16, 0, false>(a);
     if (a.g.max_pages <= 32 * 128) return launch_tok<128, 32, 0, false>(a);
-    return cudaErrorInvalidValue;
+    return launch_tok<128, -1, 0, false>(a);   // wider tables: selection staged in shared memory
 }
 
 }  // namespace

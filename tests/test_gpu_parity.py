@@ -208,6 +208,12 @@ def test_more_units_than_resident_blocks():
     compare(w, run_gpu(w), dense_sample=8)
     w = make_workload(spec(batch=40, n_q_heads=8, n_kv_heads=1, seq_lens=lens[:40], P=8, K_c=40, needles=2), seed=217)
     compare(w, run_gpu(w), dense_sample=8)
+    # one long sequence among many short ones, table wider than 32 page scores per thread: the pool cannot
+    # hold 80 sequences of that length, so the 128-thread shape with the selection in shared memory runs
+    w = make_workload(spec(batch=80, n_q_heads=4, n_kv_heads=2, seq_lens=(70000,) + (600,) * 79, P=16, K_c=100,
+                           needles=5), seed=218)
+    assert w.block_table.shape[0] * w.block_table.shape[1] > w.k_cache.shape[0]
+    compare(w, run_gpu(w), dense_sample=4)
 
 
 def test_block_table_wider_than_the_register_select():
