@@ -78,7 +78,7 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
     VSA_PROBE_T0(47);
     const int b = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, c = lane & 15, gi = lane >> 4;
-    const int w = blockIdx.x * kScanWarps + warp;
+    const int w = blockIdx.x * (blockDim.x >> 5) + warp;
     const int g = w % geo.n_kv_heads;
     const int slice = w / geo.n_kv_heads;
     const int first_page = slice * blocks_per_warp * kBlockPages;
@@ -112,7 +112,7 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
     if (blockIdx.y == 0) {
         if (zero_word && blockIdx.x == 0 && threadIdx.x == 0) *zero_word = 0;
         if (zero_words)
-            for (int i = blockIdx.x * kScanThreads + threadIdx.x; i < zero_count; i += gridDim.x * kScanThreads)
+            for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < zero_count; i += gridDim.x * blockDim.x)
                 zero_words[i] = 0;
     }
     if (!has_range) return;
@@ -273,6 +273,22 @@ int scan_blocks_per_warp(const Geometry& g)
     return (int)k;
 }
 
+// Warps per thread block (8 at most).  When the whole launch is resident at once (two blocks per SM
+// on 148 SMs) the busiest SM sets the time, so smaller blocks that spread the warps over more SMs
+// win: the 64 warps of one 4k-token sequence run as 64 blocks of one warp instead of 8 blocks of 8
+// (0.6 us per layer at batch 1); 2048 warps as 296 blocks of 7 instead of 256 of 8.
+int scan_warps_per_block(int warps_per_seq, int batch)
+{
+    int best = kScanWarps, best_load = 1 << 30;
+    for (int wpb = kScanWarps; wpb >= 1; --wpb) {
+        const long long blocks = (long long)batch * ((warps_per_seq + wpb - 1) / wpb);
+        if (blocks > 2 * 148) continue;
+        const int load = blocks <= 148 ? wpb : 2 * wpb;   // warps on the busiest SM
+        if (load < best_load) best = wpb, best_load = load;
+    }
+    return best;
+}
+
 template <int G, bool CERT>
 cudaError_t launch_scan_g(const Geometry& g, const uint16_t* q, const uint16_t* summaries, const int32_t* block_table,
                           const int32_t* seq_lens, float* scores, int32_t* zero_word, int32_t* zero_words,
@@ -281,7 +297,8 @@ cudaError_t launch_scan_g(const Geometry& g, const uint16_t* q, const uint16_t* 
     const int bpw = scan_blocks_per_warp(g);
     const int slices = ((g.max_pages + kBlockPages - 1) / kBlockPages + bpw - 1) / bpw;
     const int warps = slices * g.n_kv_heads;
-    const dim3 grid((unsigned)((warps + kScanWarps - 1) / kScanWarps), (unsigned)g.batch);
+    const int wpb = scan_warps_per_block(warps, g.batch);
+    const dim3 grid((unsigned)((warps + wpb - 1) / wpb), (unsigned)g.batch);
     // The request is padded to 81 KB so that exactly two blocks are resident per SM: with a third one
     // fewer blocks of the kernel that follows fit beside the scan's to start early, and the step gets
     // slower although the scan does not (measured: 30.0 against 24.8 us per layer at batch 8, T = 32k).
@@ -295,7 +312,7 @@ cudaError_t launch_scan_g(const Geometry& g, const uint16_t* q, const uint16_t* 
         if (e != cudaSuccess) return e;
         attr_device = dev;
     }
-    return launch_pdl(route_scan_kernel<G, CERT>, grid, dim3(kScanThreads), smem, stream, g, q, summaries,
+    return launch_pdl(route_scan_kernel<G, CERT>, grid, dim3(wpb * 32), smem, stream, g, q, summaries,
                       block_table, seq_lens, scores, bpw, zero_word, zero_words, zero_count, radii, rad_logical);
 }
 
