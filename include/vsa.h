@@ -92,6 +92,7 @@ typedef struct {
 
 #define VSA_UNIT_BAD_PAGE 1   /* a needed block-table entry is outside [0, num_pool_pages) */
 #define VSA_UNIT_BAD_LENGTH 2 /* seq_len <= 0 or > max_pages_per_seq * page_size           */
+#define VSA_UNIT_COPY_TIMEOUT 3 /* a tile copy did not complete within the kernel's poll limit */
 
 /* which_call values of vsa_workspace_bytes */
 #define VSA_WS_ROUTE 1
@@ -322,8 +323,11 @@ int vsa_decode_step_certified_expand(const vsa_shape_t* shape, const void* q, co
  * timing of exactly the launch sequence the step uses (a measurement aid for the latency
  * breakdown the paper asks for in Sec. 10.4; results are identical to vsa_decode_step).
  *   events: host array of 5 cudaEvent_t created by the caller with timing enabled:
- *   [0] before the page-score scan, [1] after it, [2] after the top-P selection,
+ *   [0] before the page-score scan, [1] after it, [2] recorded right after [1],
  *   [3] after the fused sparse pass, [4] after the dense fallback pass.
+ * The top-P selection runs inside the fused sparse kernel, so the interval [1] -> [2] brackets no
+ * kernel: it reads what a pair of event records costs on the stream, which every other interval
+ * also contains.
  */
 int vsa_decode_step_timed(const vsa_shape_t* shape, const void* q, const void* summaries, const void* k_cache,
                           const void* v_cache, const int32_t* block_table, const int32_t* seq_lens, int32_t P,

@@ -243,6 +243,7 @@ static int sparse_solver_impl(int solver_kind, const vsa_shape_t* shape, const v
         !fallback_list || !fallback_count)
         return VSA_ERR_INVALID_ARGUMENT;
     if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache)) return VSA_ERR_MISALIGNED;
+    if (!vsa::sparse_shared_memory_fits(g, P, K_c, false, true, false)) return VSA_ERR_UNSUPPORTED_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaMemsetAsync(fallback_count, 0, sizeof(int32_t), st) != cudaSuccess) return VSA_ERR_CUDA;
     return cuda_rc(vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, (int32_t*)routed_pages, nullptr,
@@ -308,6 +309,8 @@ static int decode_step_impl(const vsa_shape_t* shape, const void* q, const void*
     if (!aligned16(q) || !aligned16(summaries) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(ws))
         return VSA_ERR_MISALIGNED;
     if (ws_bytes < step_route_part(g) + vsa::dense_workspace_bytes(g)) return VSA_ERR_WORKSPACE_TOO_SMALL;
+    if (!vsa::sparse_shared_memory_fits(g, P, K_c, true, solve != nullptr, cert != nullptr))
+        return VSA_ERR_UNSUPPORTED_SHAPE;
     float* rad_logical = nullptr;
     if (cert) {
         if (!radii) return VSA_ERR_INVALID_ARGUMENT;

@@ -98,15 +98,12 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
     sm.item_base = (int32_t*)(dense_smem + kRingBytes);
     sm.misc = sm.item_base + n_groups + 1;
     sm.group_mask = (uint8_t*)(sm.misc + 16);
-    VSA_PROBE_T0(53);
     pdl_wait();
     pdl_launch_dependents();
-    VSA_PROBE_T0(54);
 
     // ---- which heads of which groups are listed? ----
     if (fallback_count) {
         const int count = *fallback_count;
-        VSA_PROBE_TMAX(55);
         if (count <= 0) return;
         for (int i = tid; i < n_groups; i += kDenseThreads) sm.group_mask[i] = 0;
         __syncthreads();
@@ -282,8 +279,9 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
             const int pl = my_first + k * kDenseWarps;
             const int valid = min(kPageSize, T - pl * kPageSize);   // > 0
             {
-                const long long phys = bt[pl];   // a page outside the pool contributes nothing
+                const long long phys = bt[pl];   // a page outside the pool: the group's listed heads fail
                 if (phys < 0 || phys >= geo.pool_pages) {
+                    if (lane == 0) sm.misc[13] = 1;   // (cleared at the end of the previous item)
                     __syncwarp();
                     continue;
                 }
@@ -381,7 +379,7 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
             dst[2 + e] = a;
             if (e == 0) {
                 dst[0] = M;
-                dst[1] = L;
+                dst[1] = sm.misc[13] ? -1.0f : L;   // sums are never negative: -1 marks a page outside the pool
             }
         }
 
@@ -408,7 +406,21 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
                 const int hh = idx / kHeadDim, e = idx % kHeadDim;
                 if (!((mask >> hh) & 1u)) continue;
                 float M = -INFINITY;
-                for (int it = 0; it < items_of_group; ++it) M = fmaxf(M, ms_s[it * G + hh]);
+                bool bad_page = false;
+                for (int it = 0; it < items_of_group; ++it) {
+                    M = fmaxf(M, ms_s[it * G + hh]);
+                    bad_page |= ls_s[it * G + hh] < 0.0f;
+                }
+                const long long unit = (long long)b * geo.n_q_heads + g * G + hh;
+                if (bad_page) {
+                    // a block-table entry of the sequence is outside the pool: no dense result exists
+                    out[unit * kHeadDim + e] = 0.0f;
+                    if (e == 0 && diag) {
+                        diag[unit].lse = 0.0f;
+                        diag[unit].status = VSA_UNIT_BAD_PAGE;
+                    }
+                    continue;
+                }
                 // one pass in item order
                 float acc = 0.0f, L = 0.0f;
 #pragma unroll 8
@@ -418,29 +430,16 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
                     acc = fmaf(__ldcg(gp + ((long long)it * G + hh) * kPartialFloats + 2 + e), f, acc);
                     L = fmaf(ls_s[it * G + hh], f, L);
                 }
-                const long long unit = (long long)b * geo.n_q_heads + g * G + hh;
                 out[unit * kHeadDim + e] = L > 0.0f ? acc / L : 0.0f;
                 if (e == 0 && diag) diag[unit].lse = (M + log2f(L)) * 0.6931471805599453f;
             }
         }
+        if (tid == 0) sm.misc[13] = 0;
         __syncthreads();   // the ring (merge buffer) and misc are reused by the next item
     }
 }
 
-int g_num_sms = 0;
-
-int num_sms()
-{
-    if (g_num_sms == 0) {
-        int dev = 0, n = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
-            g_num_sms = n;
-        else
-            return 148;
-    }
-    return g_num_sms;
-}
+int num_sms() { return device_sm_count(); }
 
 // room for the items the kernel may create: one ragged item per group plus the balancing target
 int dense_max_items(const Geometry& g) { return g.batch * g.n_kv_heads + 2048; }
@@ -474,15 +473,9 @@ static cudaError_t launch_dense_g(const Geometry& g, const uint16_t* q, const ui
                                   float* out, vsa_diag_t* diag, cudaStream_t stream)
 {
     const size_t smem = dense_smem_bytes(g);
-    static int attr_device = -1;   // per template instance: the device whose function attribute is set
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
+    static bool attr_done[kMaxDevices] = {};   // per template instance
+    const cudaError_t e = allow_large_dynamic_smem(dense_split_kernel<G>, attr_done);
     if (e != cudaSuccess) return e;
-    if (attr_device != dev) {
-        e = cudaFuncSetAttribute(dense_split_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e != cudaSuccess) return e;
-        attr_device = dev;
-    }
     // persistent grid: one block per SM (the ring fills the shared memory)
     return launch_pdl(dense_split_kernel<G>, dim3((unsigned)num_sms()), dim3(kDenseThreads), smem, stream, g, q, k, v,
                       block_table, seq_lens, fallback_list, fallback_count, epsilon, partials, counters, out, diag,
@@ -511,10 +504,3 @@ cudaError_t launch_dense(const Geometry& g, const void* q, const void* k_cache, 
 }
 
 }  // namespace vsa
-
-#ifdef VSA_ENABLE_PROBES
-extern "C" int vsa_probe_read_dense(long long* host64)
-{
-    return (int)cudaMemcpyFromSymbol(host64, vsa_probe_buf, sizeof(long long) * 64);
-}
-#endif

@@ -75,7 +75,6 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
     // block-table blocks fetched before the sequence length is known: the warp's whole range
     constexpr int kFirstBlocks = kMaxBlocksPerWarp;
     extern __shared__ __align__(16) uint8_t scan_smem[];
-    VSA_PROBE_T0(47);
     const int b = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, c = lane & 15, gi = lane >> 4;
     const int w = blockIdx.x * (blockDim.x >> 5) + warp;
@@ -104,8 +103,6 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
 
     pdl_wait();                 // the score scratch may still be read by the previous step's kernels
     pdl_launch_dependents();
-    VSA_PROBE_T0(48);
-    VSA_PROBE(9);
 
     // housekeeping for the kernels that follow in a step: clear the fallback counter and the
     // per-group tickets of the dense pass
@@ -138,7 +135,6 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
 #pragma unroll
     for (int k = 0; k < kFirstBlocks; ++k)
         if (k < n_blocks) off_tab[k * kBlockPages + lane] = encode(first_entries[k], k * kBlockPages + lane);
-    VSA_PROBE(10);
     float qf[G][8];
 #pragma unroll
     for (int hh = 0; hh < G; ++hh) unpack8(qraw[hh], qf[hh]);
@@ -179,7 +175,6 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
         }
     };
 
-    VSA_PROBE(11);
 #pragma unroll
     for (int s = 0; s < STAGES - 1; ++s) {
         if (s < n_rounds) issue(s);
@@ -189,8 +184,6 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
         if (R + STAGES - 1 < n_rounds) issue(R + STAGES - 1);
         cp_async_commit();
         cp_async_wait<STAGES - 1>();   // this lane's copies of round R have landed
-        if (R == 0) VSA_PROBE(12);
-        if (R == 1) VSA_PROBE(13);
         const uint8_t* src = my_smem + (R & (STAGES - 1)) * ROUND_PAGES * kRowBytes + lane_off;
         float vals[16];
 #pragma unroll
@@ -217,8 +210,6 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
                     off_tab[pl] >= 0 ? rad_ring[(R & (STAGES - 1)) * ROUND_PAGES + gi * ROWS + own_r] : 0.0f;
         }
     }
-    VSA_PROBE(14);
-    VSA_PROBE_TMAX(49);
 }
 
 // Exact top-P of one unit's page scores, order (score descending, page ascending).
@@ -249,41 +240,33 @@ __global__ void route_select_kernel(Geometry geo, const float* __restrict__ scor
     }
 }
 
-#ifdef VSA_ENABLE_PROBES
-}  // namespace
-}  // namespace vsa
-extern "C" int vsa_probe_read_route(long long* host64)
-{
-    return (int)cudaMemcpyFromSymbol(host64, vsa_probe_buf, sizeof(long long) * 64);
-}
-namespace vsa {
-namespace {
-#endif
 
 size_t select_smem_bytes(const Geometry& g, int P) { return (size_t)select_pages_words(g.max_pages, P) * 4; }
 
 int scan_blocks_per_warp(const Geometry& g)
 {
-    // 32-page blocks per warp: about one resident wave of warps (2 thread blocks of 8 warps per SM
-    // on 148 SMs) while that takes no more than kMaxBlocksPerWarp
+    // 32-page blocks per warp: about one resident wave of warps (2 thread blocks of 8 warps per SM)
+    // while that takes no more than kMaxBlocksPerWarp
     const long long blocks = (long long)g.batch * g.n_kv_heads * ((g.max_pages + kBlockPages - 1) / kBlockPages);
-    long long k = (blocks + 2367) / 2368;
+    const long long resident_warps = 2LL * kScanWarps * device_sm_count();
+    long long k = (blocks + resident_warps - 1) / resident_warps;
     if (k < 1) k = 1;
     if (k > kMaxBlocksPerWarp) k = kMaxBlocksPerWarp;
     return (int)k;
 }
 
-// Warps per thread block (8 at most).  When the whole launch is resident at once (two blocks per SM
-// on 148 SMs) the busiest SM sets the time, so smaller blocks that spread the warps over more SMs
+// Warps per thread block (8 at most).  When the whole launch is resident at once (two blocks per SM)
+// the busiest SM sets the time, so smaller blocks that spread the warps over more SMs
 // win: the 64 warps of one 4k-token sequence run as 64 blocks of one warp instead of 8 blocks of 8
 // (0.6 us per layer at batch 1); 2048 warps as 296 blocks of 7 instead of 256 of 8.
 int scan_warps_per_block(int warps_per_seq, int batch)
 {
+    const int sms = device_sm_count();
     int best = kScanWarps, best_load = 1 << 30;
     for (int wpb = kScanWarps; wpb >= 1; --wpb) {
         const long long blocks = (long long)batch * ((warps_per_seq + wpb - 1) / wpb);
-        if (blocks > 2 * 148) continue;
-        const int load = blocks <= 148 ? wpb : 2 * wpb;   // warps on the busiest SM
+        if (blocks > 2 * sms) continue;
+        const int load = blocks <= sms ? wpb : 2 * wpb;   // warps on the busiest SM
         if (load < best_load) best = wpb, best_load = load;
     }
     return best;
@@ -303,15 +286,9 @@ cudaError_t launch_scan_g(const Geometry& g, const uint16_t* q, const uint16_t* 
     // fewer blocks of the kernel that follows fit beside the scan's to start early, and the step gets
     // slower although the scan does not (measured: 30.0 against 24.8 us per layer at batch 8, T = 32k).
     const size_t smem = std::max((size_t)kScanWarps * ScanCfg<G>::WARP_BYTES, (size_t)81 * 1024);
-    static int attr_device = -1;   // per template instance: the device whose function attribute is set
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
+    static bool attr_done[kMaxDevices] = {};   // per template instance
+    const cudaError_t e = allow_large_dynamic_smem(route_scan_kernel<G, CERT>, attr_done);
     if (e != cudaSuccess) return e;
-    if (attr_device != dev) {
-        e = cudaFuncSetAttribute(route_scan_kernel<G, CERT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        attr_device = dev;
-    }
     return launch_pdl(route_scan_kernel<G, CERT>, grid, dim3(wpb * 32), smem, stream, g, q, summaries,
                       block_table, seq_lens, scores, bpw, zero_word, zero_words, zero_count, radii, rad_logical);
 }
@@ -353,9 +330,9 @@ cudaError_t launch_route_select(const Geometry& g, const void* ws, const int32_t
     const dim3 grid((unsigned)g.n_q_heads, (unsigned)g.batch);
 #define VSA_SELECT_LAUNCH(KPT, THREADS)                                                                          \
     {                                                                                                            \
+        static bool attr_done[kMaxDevices] = {};                                                                 \
         if (smem > 48 * 1024) {                                                                                  \
-            cudaError_t e = cudaFuncSetAttribute(route_select_kernel<KPT>,                                       \
-                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);        \
+            const cudaError_t e = allow_large_dynamic_smem(route_select_kernel<KPT>, attr_done);                 \
             if (e != cudaSuccess) return e;                                                                      \
         }                                                                                                        \
         cudaError_t e2 = launch_pdl(route_select_kernel<KPT>, grid, dim3(THREADS), smem, stream, g,            \

@@ -6,6 +6,7 @@
 
 namespace vsa {
 
+
 namespace {
 
 size_t sparse_smem_bytes(const Geometry& g, int P, int K_c, bool fused, int threads, bool solve)
@@ -20,21 +21,32 @@ size_t sparse_smem_bytes(const Geometry& g, int P, int K_c, bool fused, int thre
     return words * 4 + 16;
 }
 
-int g_sm_count = 0;
-int sm_count()
+int sm_count() { return device_sm_count(); }
+
+// thread-block size of the per-unit kernel for a launch
+int sparse_block_threads(const Geometry& g, int P, bool solve, bool cert, bool listed)
 {
-    if (g_sm_count == 0) {
-        int dev = 0, n = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
-            g_sm_count = n;
-        else
-            return 148;
-    }
-    return g_sm_count;
+    const long long units = (long long)g.batch * g.n_q_heads;
+    int threads = (!solve && units <= sm_count()) ? 512 : 256;
+    // Tables wider than 32 scores per thread: the 128-thread shape selects from shared memory, which loses
+    // to the 256-thread register selection when every sequence is long (99 against 88 us per layer at
+    // batch 16, T = 128k) and wins when most are short (410 against 445 us on the ragged config 4).  The
+    // lengths are not known here; what is known is the pool: when batch * max_pages exceeds it, the
+    // sequences cannot all be long.
+    const bool narrow = g.max_pages <= 32 * 128;
+    const bool cannot_all_be_long = (long long)g.batch * g.max_pages > (long long)g.pool_pages;
+    if (!solve && !listed && units > 2 * sm_count() && P <= 64 && (narrow || (!cert && cannot_all_be_long)))
+        threads = 128;
+    return threads;
 }
 
 }  // namespace
+
+bool sparse_shared_memory_fits(const Geometry& g, int P, int K_c, bool fused, bool solve, bool cert)
+{
+    const int threads = sparse_block_threads(g, P, solve, cert, false);
+    return sparse_smem_bytes(g, P, K_c, fused, threads, solve) <= (size_t)227 * 1024;
+}
 
 int sparse_register_select_max_pages(long long units) { return 32 * (units <= sm_count() ? 512 : 256); }
 
@@ -54,17 +66,7 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
     // the threads (measured 1.26x per unit): 512 units take one wave instead of two (25 against 30 us per
     // layer at batch 16, T = 4k), 2048 units 80 against 101 us (batch 64, T = 8k).  Closed-form variants
     // (with or without the certificate) only; fused ones with the page scores in registers (32 per thread at most).
-    const long long units = (long long)g.batch * g.n_q_heads;
-    int threads = (!solve && units <= sm_count()) ? 512 : 256;
-    // Tables wider than 32 scores per thread: the 128-thread shape selects from shared memory, which loses
-    // to the 256-thread register selection when every sequence is long (99 against 88 us per layer at
-    // batch 16, T = 128k) and wins when most are short (410 against 445 us on the ragged config 4).  The
-    // lengths are not known here; what is known is the pool: when batch * max_pages exceeds it, the
-    // sequences cannot all be long.
-    const bool narrow = g.max_pages <= 32 * 128;
-    const bool cannot_all_be_long = (long long)g.batch * g.max_pages > (long long)g.pool_pages;
-    if (!solve && !unit_list && units > 2 * sm_count() && P <= 64 && (narrow || (!cert && cannot_all_be_long)))
-        threads = 128;
+    const int threads = sparse_block_threads(g, P, solve != nullptr, cert != nullptr, unit_list != nullptr);
     a.smem = sparse_smem_bytes(g, P, K_c, page_scores != nullptr, threads, solve != nullptr);
     a.solver_iters = solver_iters;
     a.solver_kind = solver_kind;

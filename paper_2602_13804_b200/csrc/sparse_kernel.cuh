@@ -144,7 +144,6 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         unit = __ldcg(unit_list + blockIdx.x);
     }
     const int b = (int)(unit / geo.n_q_heads), h = (int)(unit % geo.n_q_heads), g = h / geo.group;
-    VSA_PROBE_T0(50);
     // Loads that depend on nothing computed in this step go out before the wait on the preceding
     // kernel: the sequence length, the query row (the routing kernel that precedes this one in a step
     // has read it already) and a copy of the block-table row for the page lookups that follow the
@@ -161,7 +160,6 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     }
     pdl_wait();
     pdl_launch_dependents();
-    VSA_PROBE_T0(51);
     // Only the scores of the sequence's own pages are fetched: the rest of the scratch row was not
     // written in this step (in a ragged batch it is most of the row, and it would come from DRAM).
     const int nb_fetch = (T > 0 && T <= geo.max_pages * kPageSize) ? (T + kPageSize - 1) / kPageSize : 0;
@@ -193,7 +191,6 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         return;
     }
     const int nb = (T + kPageSize - 1) / kPageSize;
-    VSA_PROBE(0);
 
     // ---- routed pages -> page_l[] sorted by logical page, so that array order = position order ----
     int np;
@@ -273,7 +270,6 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         // (P <= 128 < THREADS: thread t < P owns slot t in the count)
         np = __syncthreads_count(tid < P && raw[tid < P ? tid : 0] != INT_MAX);
     }
-    VSA_PROBE(1);
     const int any_bad = __syncthreads_or(bad);
     uint32_t ub_unrouted_key = 0u;   // CERT: key of the best upper bound over the un-routed pages, 0 = none
     if constexpr (CERT) {
@@ -294,7 +290,6 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         if (tid + j * THREADS < N) sm.keys[tid + j * THREADS] = 0u;
     __syncthreads();
 
-    VSA_PROBE(2);
     // ---- token routing: score all 16 tokens of a page per half-warp ----
     float qf[8];
     unpack8(qraw, qf);
@@ -323,7 +318,6 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     }
     __syncthreads();
 
-    VSA_PROBE(3);
     // ---- every thread takes its TOK_KPT token keys into registers ----
     uint32_t key[TOK_KPT];
     int present = 0;
@@ -380,7 +374,6 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     }
     const int ns = min(K_c, n_valid);
 
-    VSA_PROBE(4);
     // ---- exact top-(ns+1): its last element is the best rejected token, the rest are the candidates ----
     uint32_t out_key = 0u, mask = 0u;
     const bool has_rejected = n_valid > ns;
@@ -402,7 +395,6 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         __syncthreads();   // wred is rewritten by the compaction
     }
 
-    VSA_PROBE(5);
     // ---- ordered compaction of the candidates (position order); the thread that holds a candidate's
     //      key writes the address of its value row and its softmax weight ----
     const float s1 = ns > 0 ? key_to_float(key1) : -INFINITY;
@@ -437,7 +429,6 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     }
     __syncthreads();
 
-    VSA_PROBE(6);
     float lse_closed = 0.0f;   // log-sum-exp of the closed-form weights (SOLVE only)
     if constexpr (SOLVE != 0) {
         if (ns > 0) {
@@ -733,7 +724,6 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
             z += w[u];
         }
     }
-    VSA_PROBE(7);
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[e] += __shfl_xor_sync(kFullMask, acc[e], 16);
     z += __shfl_xor_sync(kFullMask, z, 16);
@@ -753,7 +743,6 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         out[unit * kHeadDim + tid] = ns > 0 ? a / Z : 0.0f;
     }
 
-    VSA_PROBE(8);
     // ---- diagnostics and fallback flag ----
     if (tid == 0) {
         const float s2 = ns > 1 ? key_to_float(key2) : -INFINITY;
@@ -782,7 +771,6 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         diag[unit] = d;
         if (d.fallback) fallback_list[atomicAdd(fallback_count, 1)] = (int32_t)unit;
     }
-    VSA_PROBE_TMAX(52);
 }
 
 }  // namespace
@@ -815,9 +803,10 @@ namespace {
 template <int THREADS, int PAGE_KPT, int TOK_KPT, int SOLVE, bool CERT>
 cudaError_t launch_variant(const SparseArgs& a)
 {
+    static bool attr_done[kMaxDevices] = {};   // per template instance
     if (a.smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(sparse_decode_kernel<THREADS, PAGE_KPT, TOK_KPT, SOLVE, CERT>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)a.smem);
+        const cudaError_t e =
+            allow_large_dynamic_smem(sparse_decode_kernel<THREADS, PAGE_KPT, TOK_KPT, SOLVE, CERT>, attr_done);
         if (e != cudaSuccess) return e;
     }
     const unsigned units = (unsigned)(a.g.batch * a.g.n_q_heads);

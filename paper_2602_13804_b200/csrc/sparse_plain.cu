@@ -10,11 +10,3 @@ cudaError_t launch_sparse_plain(const SparseArgs& a, int threads)
 }
 
 }  // namespace vsa
-
-#ifdef VSA_ENABLE_PROBES
-// development aid: the phase probes of this translation unit's kernels
-extern "C" int vsa_probe_read(long long* host64)
-{
-    return (int)cudaMemcpyFromSymbol(host64, vsa_probe_buf, sizeof(long long) * 64);
-}
-#endif

@@ -5,44 +5,6 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-// Phase-timing probes for development builds (-DVSA_ENABLE_PROBES): one thread of one block records
-// clock64() at marked points.  They compile to nothing otherwise.
-#ifdef VSA_ENABLE_PROBES
-#ifndef VSA_PROBE_BLOCK
-#define VSA_PROBE_BLOCK 0
-#endif
-static __device__ long long vsa_probe_buf[64];
-#define VSA_PROBE(i)                                                                   \
-    do {                                                                               \
-        if (blockIdx.x == VSA_PROBE_BLOCK && blockIdx.y == 0 && threadIdx.x == 0) vsa_probe_buf[i] = clock64(); \
-    } while (0)
-#define VSA_PROBE_VAL(i, v)                                                            \
-    do {                                                                               \
-        if (blockIdx.x == VSA_PROBE_BLOCK && blockIdx.y == 0 && threadIdx.x == 0) vsa_probe_buf[i] = (long long)(v); \
-    } while (0)
-// wall-clock (globaltimer, ns) timeline of a step: block 0's time at a point, and the latest time
-// any block passed a point
-__device__ __forceinline__ long long vsa_probe_ns()
-{
-    long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-#define VSA_PROBE_T0(i)                                                                \
-    do {                                                                               \
-        if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) vsa_probe_buf[i] = vsa_probe_ns(); \
-    } while (0)
-#define VSA_PROBE_TMAX(i)                                                              \
-    do {                                                                               \
-        if (threadIdx.x == 0) atomicMax((unsigned long long*)&vsa_probe_buf[i], (unsigned long long)vsa_probe_ns()); \
-    } while (0)
-#else
-#define VSA_PROBE(i)
-#define VSA_PROBE_VAL(i, v)
-#define VSA_PROBE_T0(i)
-#define VSA_PROBE_TMAX(i)
-#endif
-
 namespace vsa {
 
 constexpr int kHeadDim = 128;   // elements per head
@@ -560,7 +522,6 @@ __device__ __forceinline__ TopkRegResult block_topk_reg(const uint32_t (&key)[KP
             hi = fmaxf(hi, __uint_as_float(s.wred[2 * w + 1]));
         }
     }
-    if (HAVE_RANGE) VSA_PROBE(22);
     const float scale = 256.0f / (hi - lo);
     const bool fast = hi > lo && isfinite(scale) && isfinite(hi - lo);
     int cut = -1, need = K;
@@ -571,9 +532,7 @@ __device__ __forceinline__ TopkRegResult block_topk_reg(const uint32_t (&key)[KP
             bucket[j] = f[j] > -INFINITY ? (int)fminf(fmaxf((f[j] - lo) * scale, 0.0f), 255.0f) : 0;
             if (key[j] != 0u) atomicAdd(&s.hist[bucket[j]], 1u);
         }
-        if (HAVE_RANGE) VSA_PROBE(23);
         __syncthreads();
-        if (HAVE_RANGE) VSA_PROBE(24);
         if (warp == 0) {
             // one warp scans the histogram and publishes the cut through the barrier that follows
             uint32_t c[8], mine = 0;
@@ -611,7 +570,6 @@ __device__ __forceinline__ TopkRegResult block_topk_reg(const uint32_t (&key)[KP
                 s.misc[10] = (uint32_t)(K - my_above);
             }
         }
-        if (HAVE_RANGE) VSA_PROBE(25);
         __syncthreads();   // the histogram has been read: its words are reused for the cut bucket's keys
         if (s.misc[9] != 0xffffffffu) {
             cut = (int)s.misc[9];
@@ -642,10 +600,8 @@ __device__ __forceinline__ TopkRegResult block_topk_reg(const uint32_t (&key)[KP
                 }
             }
         }
-        if (HAVE_RANGE) VSA_PROBE(26);
         __syncthreads();
         const int m = (int)s.misc[4];
-        if (HAVE_RANGE) VSA_PROBE_VAL(41, m);
         for (int t = tid; t < m; t += stride) {
             const int idx = s.list[t];
             const uint32_t kt = s.hist[t];
@@ -662,12 +618,10 @@ __device__ __forceinline__ TopkRegResult block_topk_reg(const uint32_t (&key)[KP
                 s.misc[6] = (uint32_t)idx;
             }
         }
-        if (HAVE_RANGE) VSA_PROBE(27);
         __syncthreads();
 #pragma unroll
         for (int j = 0; j < KPT; ++j)
             if (((in_cut >> j) & 1u) && spill_take[tid + j * stride]) out.mask |= 1u << j;
-        if (HAVE_RANGE) VSA_PROBE(28);
     } else {
         __syncthreads();
 #pragma unroll

@@ -4,7 +4,6 @@
 #include <cuda_runtime.h>
 #include <stddef.h>
 #include <stdint.h>
-#include <stdlib.h>
 
 #include "../../include/vsa.h"
 
@@ -25,9 +24,46 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    static const bool disabled = getenv("VSA_NO_PDL") != nullptr;   // debugging aid: ordinary launches
-    cfg.numAttrs = disabled ? 0 : 1;
+    cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// ---- per-device facts, looked up once per device ordinal ---------------------------------------------
+constexpr int kMaxDevices = 64;
+
+// ordinal of the current device when it can index the per-device tables below, else -1
+inline int device_slot()
+{
+    int d = -1;
+    if (cudaGetDevice(&d) != cudaSuccess) return -1;
+    return (d >= 0 && d < kMaxDevices) ? d : -1;
+}
+
+// number of SMs of the current device (148 on a B200); 1 if the query fails
+inline int device_sm_count()
+{
+    static int cached[kMaxDevices] = {};
+    const int d = device_slot();
+    if (d >= 0 && cached[d] > 0) return cached[d];
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+        return 1;
+    if (d >= 0) cached[d] = n;
+    return n;
+}
+
+// Lets `kernel` request up to the device's opt-in maximum of dynamic shared memory (227 KB).  The attribute
+// belongs to the (kernel, device) pair and is set on the first launch on each device: `done` is the
+// caller's table for this kernel (a function-local static, one entry per device ordinal).
+template <typename... KArgs>
+inline cudaError_t allow_large_dynamic_smem(void (*kernel)(KArgs...), bool (&done)[kMaxDevices])
+{
+    const int d = device_slot();
+    if (d >= 0 && done[d]) return cudaSuccess;
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e == cudaSuccess && d >= 0) done[d] = true;
+    return e;
 }
 
 struct Geometry {
@@ -75,6 +111,9 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
                           int solver_iters = 0, vsa_solve_t* solve = nullptr, const float* rad_logical = nullptr,
                           vsa_cert_t* cert = nullptr, int solver_kind = 1, const int32_t* unit_list = nullptr,
                           const int32_t* unit_count = nullptr, int routed_stride = 0);
+// false when the kernel variant a launch would take needs more dynamic shared memory than a thread block
+// can have (227 KB): wide block tables together with the iterative solve's key tile
+bool sparse_shared_memory_fits(const Geometry& g, int P, int K_c, bool fused, bool solve, bool cert);
 // widest block table for which the fused kernel keeps every page score of a unit in registers (the
 // certificate variant exists for those shapes only); `units` = batch * n_q_heads
 int sparse_register_select_max_pages(long long units);

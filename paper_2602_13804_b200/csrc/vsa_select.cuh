@@ -114,7 +114,6 @@ __device__ __forceinline__ int select_top_pages_keys(const uint32_t (&key)[KPT],
         // only warps whose 32 threads all own a score take part (short sequences fill fewer warps)
         const int nw_full = min(nwarps, n >> 5);
         const int r = nw_full > 0 ? (K + nw_full - 1) / nw_full : 33;
-        VSA_PROBE(20);
         uint32_t tmax = 0u;
 #pragma unroll
         for (int j = 0; j < KPT; ++j) tmax = max(tmax, key[j]);
@@ -149,8 +148,6 @@ __device__ __forceinline__ int select_top_pages_keys(const uint32_t (&key)[KPT],
         }
         __syncthreads();
         const int m = (int)s.ts.misc[4];
-        VSA_PROBE(21);
-        VSA_PROBE_VAL(40, m);
         if (m <= kTopkList) {
             for (int t = tid; t < m; t += stride) {
                 const int idx = s.ts.list[t];

@@ -84,6 +84,7 @@ class SparsePagedDecoder:
         vsa_cert_t, see binding.cert_to_dict) decides which units fall back to the dense pass."""
         if not hasattr(self, "cert"):
             self.cert = B.alloc_cert(self.units, self.device)
+        if not hasattr(self, "ws_cert"):
             self.ws_cert = B.alloc_workspace(self.shape, self.P, self.K_c, B.VSA_WS_STEP_CERTIFIED, self.device)
         B.vsa_decode_step_certified(self.shape, q, summaries, radii, k_cache, v_cache, block_table, seq_lens, self.P,
                                     self.K_c, self.epsilon, self.gap_threshold, self.out, self.diag, self.cert,

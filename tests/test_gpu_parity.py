@@ -146,6 +146,28 @@ def test_bad_block_table_entry_and_bad_length_set_status_without_trapping():
     assert 2 not in rp[0].cpu().numpy() and np.all(rp[1].cpu().numpy() == -1)
 
 
+def test_dense_pass_fails_the_units_of_a_sequence_with_an_entry_outside_the_pool():
+    """Every page of a listed sequence is needed by the dense pass: one block-table entry outside the pool
+    (bounds-checked, never dereferenced) must give status BAD_PAGE and a zero row for all heads of that
+    sequence, and leave the other sequence's result equal to the definition."""
+    w = make_workload(spec(seq_lens=(1000, 513), n_q_heads=8, n_kv_heads=2), seed=208).to(DEV)
+    shape = B.shape_of(w.q, w.k_cache, w.block_table)
+    bt = w.block_table.clone()
+    bt[0, 40] = -3
+    out = torch.full((2, 8, 128), float("nan"), dtype=torch.float32, device=DEV)
+    diag = B.alloc_diag(16, DEV)
+    ws = B.alloc_workspace(shape, 0, 0, B.VSA_WS_DENSE, DEV)
+    B.vsa_dense_decode_fallback(shape, w.q, w.k_cache, w.v_cache, bt, w.seq_lens, None, None, w.epsilon,
+                                out, diag, ws)
+    torch.cuda.synchronize()
+    d = B.diag_to_dict(diag)
+    assert d["status"].view(2, 8)[0].tolist() == [1] * 8
+    assert not out[0].cpu().numpy().any()
+    q, K, V, bt_h, sl = host_arrays(w)
+    dn = oracle.dense(geometry(w), q, K, V, bt_h, sl, w.epsilon)
+    check_out(out[1].cpu().numpy(), dn.out[1], "dense baseline, intact sequence")
+
+
 def test_incremental_summary_update_of_the_last_page():
     w = make_workload(spec(needles=0), seed=210).to(DEV)
     shape = B.shape_of(w.q, w.k_cache, w.block_table)

@@ -89,3 +89,29 @@ def test_reference_arm_runs_on_rank_zero_only():
     line = json.loads(r.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["cpu_baseline"]["kind"] == "oracle"
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["higher_is_better"] is False
+
+
+def test_gpus_flag_starts_the_ranks_itself():
+    """`bench.py --gpus N` without a torchrun environment re-launches itself as N ranks.  The launch line
+    is exercised here with the reference arm as the CPU stand-in for the ranks' work: two processes start,
+    rank 0 prints the one JSON line with n_gpus = 2, rank 1 prints nothing, and the launcher exits 0."""
+    sys.path.insert(0, ROOT)
+    import bench
+    import json
+    cmd = bench.spawn_command(["--impl", "reference", "--workload", "cfg0", "--steps", "1", "--warmup", "0",
+                               "--gpus", "2"], 2, _free_port())
+    assert "torch.distributed.run" in cmd and "--nproc-per-node=2" in cmd and "127.0.0.1" in cmd
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    r = subprocess.run(cmd, env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["impl"] == "reference" and line["n_gpus"] == 2
+
+
+def test_expand_round_count():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.vsa_expand_rounds(32, 64) == 1 and bench.vsa_expand_rounds(32, 128) == 2
+    assert bench.vsa_expand_rounds(16, 100) == 3 and bench.vsa_expand_rounds(32, 32) == 0
