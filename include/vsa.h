@@ -300,10 +300,14 @@ int vsa_decode_step_certified(const vsa_shape_t* shape, const void* q, const voi
                               void* stream);
 
 /*
- * The certified step with one round of "paged expansion" (App. E: when the certificate fails, enlarge
+ * The certified step with the "paged expansion" loop (App. E: when the certificate fails, enlarge
  * S until it passes) before anything falls back to the dense pass: every unit is first processed
- * with P routed pages; the units whose certificate fails are processed again with P_expand > P
- * pages (same K_c) from the page scores of the same scan; what still fails goes to the dense pass.
+ * with P routed pages; the units whose certificate fails are processed again with 2P pages, those
+ * that still fail with 4P, and so on while the page count stays below P_expand (the last pass uses
+ * exactly P_expand), all from the page scores of the same scan and with the same K_c; what the last
+ * pass still refuses goes to the dense pass.  The passes are enqueued back to back (ceil(log2(P_expand /
+ * P)) extra launches, each over the device-side list its predecessor wrote; an empty list costs a launch
+ * whose blocks exit), so the loop is bounded and never synchronises with the host.
  * out, diag and cert of a unit are those of its last sparse pass (dense rows for the final fallback
  * list).  routed_pages: device int32 [batch][n_q_heads][P_expand]; a unit's row holds the pages of its
  * last pass, -1 padded (so a row with more than P entries marks a unit that was retried).

@@ -159,6 +159,48 @@ def route(geo: Geometry, q, summaries, block_table, seq_lens, P: int, want_all_s
     return RouteResult(pages, scores, alls)
 
 
+SUPER = 16    # logical pages per super-page
+
+
+def n_supers(max_pages_per_seq: int) -> int:
+    return (max_pages_per_seq + SUPER - 1) // SUPER
+
+
+def build_super_summaries(geo: Geometry, summaries, block_table, seq_lens):
+    """(super_summaries uint16 [B, max_supers, Hkv, d], super_rep int32 [B, max_supers, Hkv]): per
+    super-page of 16 logical pages the page summary of largest fp32 squared norm (ties: lowest page)."""
+    sm = _u16(summaries)
+    bt, sl = _i32(block_table), _i32(seq_lens)
+    ms = n_supers(geo.max_pages_per_seq)
+    sup = np.zeros((geo.batch, ms, geo.n_kv_heads, geo.head_dim), np.uint16)
+    rep = np.full((geo.batch, ms, geo.n_kv_heads), -1, np.int32)
+    s = geo.c()
+    rc = lib().orc_build_super_summaries(C.byref(s), _p(sm), _p(bt), _p(sl), C.c_int(ms), _p(sup), _p(rep))
+    assert rc == 0, rc
+    return sup, rep
+
+
+@dataclass
+class TwoLevelRouteResult:
+    supers: np.ndarray      # int32 [B, Hq, P_super] super-pages kept, (score desc, index asc), -1 padded
+    pages: np.ndarray       # int32 [B, Hq, P]
+    scores: np.ndarray      # fp32 [B, Hq, P]
+
+
+def route_two_level(geo: Geometry, q, summaries, super_summaries, block_table, seq_lens, P_super: int,
+                    P: int) -> TwoLevelRouteResult:
+    qb, sm, sup = _u16(q), _u16(summaries), _u16(super_summaries)
+    bt, sl = _i32(block_table), _i32(seq_lens)
+    supers = np.empty((geo.batch, geo.n_q_heads, P_super), np.int32)
+    pages = np.empty((geo.batch, geo.n_q_heads, P), np.int32)
+    scores = np.empty((geo.batch, geo.n_q_heads, P), np.float32)
+    s = geo.c()
+    rc = lib().orc_route_two_level(C.byref(s), _p(qb), _p(sm), _p(sup), C.c_int(sup.shape[1]), _p(bt), _p(sl),
+                                   C.c_int(P_super), C.c_int(P), _p(supers), _p(pages), _p(scores))
+    assert rc == 0, rc
+    return TwoLevelRouteResult(supers, pages, scores)
+
+
 @dataclass
 class SparseResult:
     out: np.ndarray           # fp64 [B, Hq, d]

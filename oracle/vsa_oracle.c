@@ -22,6 +22,11 @@
  *                        token, certified gap and leakage bound.
  *   orc_frank_wolfe      App. E: Frank-Wolfe with exact line search on the candidate simplex and its
  *                        duality gap, in mirrored fp32 (the vertex choices are integers).
+ *   orc_build_super_summaries, orc_route_two_level
+ *                        an approximate pre-filter in front of the page routing (Sec. 7 step 1 says only
+ *                        "coarse page summaries"; the two-level construction is not in the paper): one
+ *                        representative summary per 16 pages, P_super super-pages kept, exact page scores
+ *                        inside them.  Parity unpinned by the paper; pinned here by its special cases.
  *   orc_dense            the plain definition: softmax(<q,k_t>/epsilon) over every token.
  * (The theory objects on tiny dictionaries - Euclidean projection, exact gap, the full
  *  entropic minimiser of Eq. (5.1) - live in theory.py next to this file.)
@@ -208,6 +213,96 @@ int orc_route(const orc_shape *s, const uint16_t *q, const uint16_t *summaries, 
             routed_pages[(int64_t)u * P + i] = i < keep ? c[i].idx : -1;
             if (routed_scores) routed_scores[(int64_t)u * P + i] = i < keep ? c[i].s : -INFINITY;
         }
+        free(c);
+    }
+    return 0;
+}
+
+/* ---- two-level routing (an approximate pre-filter in front of step 1; construction not in the paper) ---
+ * A super-page is SUPER consecutive logical pages of a sequence.  Its representative is the page summary
+ * with the largest squared norm, the norm taken as canon_dot(row, row) in fp32 (ties: the lowest page);
+ * large-norm keys are the ones that can dominate an inner product, so the best score inside a super-page
+ * is usually its representative's.  super_summaries is [B][max_supers][Hkv][d] (logical order, per
+ * sequence), super_rep [B][max_supers][Hkv] the logical page chosen (-1: super-page past the sequence). */
+enum { ORC_SUPER = 16 };
+
+int orc_build_super_summaries(const orc_shape *s, const uint16_t *summaries, const int32_t *bt,
+                              const int32_t *seq_lens, int max_supers, uint16_t *super_summaries,
+                              int32_t *super_rep)
+{
+    if (!shape_ok(s) || max_supers < 1) return -1;
+    for (int b = 0; b < s->batch; ++b) {
+        int nb = n_pages_of(s, seq_lens[b]);
+        for (int sp = 0; sp < max_supers; ++sp) {
+            for (int g = 0; g < s->n_kv_heads; ++g) {
+                int64_t o = ((int64_t)b * max_supers + sp) * s->n_kv_heads + g;
+                int best = -1;
+                float best_n = 0.0f;
+                for (int l = sp * ORC_SUPER; l < (sp + 1) * ORC_SUPER && l < nb; ++l) {
+                    int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
+                    const uint16_t *row = summaries + (p * s->n_kv_heads + g) * ORC_D;
+                    float n2 = orc_canon_dot(row, row);
+                    if (best < 0 || n2 > best_n) {
+                        best = l;
+                        best_n = n2;
+                    }
+                }
+                super_rep[o] = best;
+                if (best >= 0) {
+                    int64_t p = bt[(int64_t)b * s->max_pages_per_seq + best];
+                    memcpy(super_summaries + o * ORC_D, summaries + (p * s->n_kv_heads + g) * ORC_D,
+                           sizeof(uint16_t) * ORC_D);
+                } else {
+                    memset(super_summaries + o * ORC_D, 0, sizeof(uint16_t) * ORC_D);
+                }
+            }
+        }
+    }
+    return 0;
+}
+
+/* Per unit: score the super-pages' representatives, keep the P_super best (score descending, super-page
+ * ascending); score every page of the kept super-pages exactly as orc_route does and keep the P best of
+ * THOSE (score descending, page ascending).  super_routed is [B][Hq][P_super], -1 padded. */
+int orc_route_two_level(const orc_shape *s, const uint16_t *q, const uint16_t *summaries,
+                        const uint16_t *super_summaries, int max_supers, const int32_t *bt,
+                        const int32_t *seq_lens, int P_super, int P, int32_t *super_routed,
+                        int32_t *routed_pages, float *routed_scores)
+{
+    if (!shape_ok(s) || P < 1 || P_super < 1 || max_supers < 1) return -1;
+    const int G = s->n_q_heads / s->n_kv_heads;
+    const int units = s->batch * s->n_q_heads;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int u = 0; u < units; ++u) {
+        int b = u / s->n_q_heads, h = u % s->n_q_heads, g = h / G;
+        int nb = n_pages_of(s, seq_lens[b]);
+        int ns = (nb + ORC_SUPER - 1) / ORC_SUPER;
+        const uint16_t *qv = q + (int64_t)u * ORC_D;
+        scored *c = (scored *)malloc(sizeof(scored) * (size_t)(ns > 0 ? ns : 1));
+        for (int sp = 0; sp < ns; ++sp) {
+            c[sp].s = orc_canon_dot(qv, super_summaries + (((int64_t)b * max_supers + sp) * s->n_kv_heads + g) * ORC_D);
+            c[sp].idx = sp;
+        }
+        qsort(c, (size_t)ns, sizeof(scored), cmp_scored);
+        int keep_s = ns < P_super ? ns : P_super;
+        for (int i = 0; i < P_super; ++i) super_routed[(int64_t)u * P_super + i] = i < keep_s ? c[i].idx : -1;
+        scored *pg = (scored *)malloc(sizeof(scored) * (size_t)(keep_s * ORC_SUPER + 1));
+        int n = 0;
+        for (int i = 0; i < keep_s; ++i) {
+            for (int l = c[i].idx * ORC_SUPER; l < (c[i].idx + 1) * ORC_SUPER && l < nb; ++l) {
+                int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
+                pg[n].s = orc_canon_dot(qv, summaries + (p * s->n_kv_heads + g) * ORC_D);
+                pg[n].idx = l;
+                ++n;
+            }
+        }
+        qsort(pg, (size_t)n, sizeof(scored), cmp_scored);
+        int keep = n < P ? n : P;
+        for (int i = 0; i < P; ++i) {
+            routed_pages[(int64_t)u * P + i] = i < keep ? pg[i].idx : -1;
+            if (routed_scores) routed_scores[(int64_t)u * P + i] = i < keep ? pg[i].s : -INFINITY;
+        }
+        free(pg);
         free(c);
     }
     return 0;

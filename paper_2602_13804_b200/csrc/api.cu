@@ -104,9 +104,14 @@ size_t step_route_part(const Geometry& g) { return align_up(vsa::route_workspace
 size_t step_rad_offset(const Geometry& g) { return step_route_part(g) + align_up(vsa::dense_workspace_bytes(g), 256); }
 size_t step_rad_bytes(const Geometry& g) { return (size_t)g.batch * g.n_kv_heads * g.max_pages * sizeof(float); }
 
-// expanding step: the certified layout followed by the retry list (one int per unit) and its count
+// expanding step: the certified layout followed by the retry lists - kMaxExpandRounds counters, then one
+// list of one int per unit for every round (P doubles per round and P <= 128, so seven rounds at most)
+constexpr int kMaxExpandRounds = 8;
 size_t step_retry_offset(const Geometry& g) { return align_up(step_rad_offset(g) + step_rad_bytes(g), 256); }
-size_t step_retry_bytes(const Geometry& g) { return ((size_t)g.batch * g.n_q_heads + 4) * sizeof(int32_t); }
+size_t step_retry_bytes(const Geometry& g)
+{
+    return ((size_t)kMaxExpandRounds * ((size_t)g.batch * g.n_q_heads + 1)) * sizeof(int32_t);
+}
 
 int cuda_rc(cudaError_t e) { return e == cudaSuccess ? VSA_OK : VSA_ERR_CUDA; }
 
@@ -423,24 +428,36 @@ int vsa_decode_step_certified_expand(const vsa_shape_t* shape, const void* q, co
     cudaStream_t st = (cudaStream_t)stream;
     void* ws_dense = (char*)ws + step_route_part(g);
     float* rad_logical = (float*)((char*)ws + step_rad_offset(g));
-    int32_t* retry_list = (int32_t*)((char*)ws + step_retry_offset(g));
-    int32_t* retry_count = retry_list + (size_t)g.batch * g.n_q_heads;
-    if (cudaMemsetAsync(retry_count, 0, sizeof(int32_t), st) != cudaSuccess) return VSA_ERR_CUDA;
+    const size_t units = (size_t)g.batch * g.n_q_heads;
+    int32_t* retry_counts = (int32_t*)((char*)ws + step_retry_offset(g));   // [kMaxExpandRounds]
+    int32_t* retry_lists = retry_counts + kMaxExpandRounds;                  // [round][units]
+    if (cudaMemsetAsync(retry_counts, 0, kMaxExpandRounds * sizeof(int32_t), st) != cudaSuccess) return VSA_ERR_CUDA;
     // the scan clears the final fallback counter and the dense tickets
     cudaError_t e = vsa::launch_route_scan(g, q, summaries, block_table, seq_lens, ws, fallback_count,
                                            vsa::dense_tickets(ws_dense), vsa::dense_ticket_count(g), st, radii,
                                            rad_logical);
     if (e != cudaSuccess) return VSA_ERR_CUDA;
-    // first pass over every unit with P pages: the units it cannot certify go to the retry list
-    e = vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, routed_pages, (const float*)ws, P, K_c,
-                           epsilon, gap_threshold, out, diag, retry_list, retry_count, st, 0, nullptr, rad_logical,
-                           cert, 1, nullptr, nullptr, P_expand);
-    if (e != cudaSuccess) return VSA_ERR_CUDA;
-    // second pass over the listed units only, with P_expand pages: what still fails goes to the dense pass
-    e = vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, routed_pages, (const float*)ws, P_expand,
-                           K_c, epsilon, gap_threshold, out, diag, fallback_list, fallback_count, st, 0, nullptr,
-                           rad_logical, cert, 1, retry_list, retry_count, P_expand);
-    if (e != cudaSuccess) return VSA_ERR_CUDA;
+    // Pass 0 over every unit with P pages; then, while the page budget allows, the units the previous pass
+    // could not certify are run again with twice the pages (at most P_expand) from the same page scores.
+    // Every pass is enqueued unconditionally - a pass whose list is empty costs blocks that read the count
+    // and exit - so the loop is bounded on the host and needs no synchronisation.  What the last pass still
+    // refuses goes to the dense pass.
+    int P_round = P, round = 0;
+    const int32_t *in_list = nullptr, *in_count = nullptr;
+    for (;;) {
+        const bool last = P_round >= P_expand;
+        int32_t* out_list = last ? fallback_list : retry_lists + (size_t)round * units;
+        int32_t* out_count = last ? fallback_count : retry_counts + round;
+        e = vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, routed_pages, (const float*)ws, P_round,
+                               K_c, epsilon, gap_threshold, out, diag, out_list, out_count, st, 0, nullptr,
+                               rad_logical, cert, 1, in_list, in_count, P_expand);
+        if (e != cudaSuccess) return VSA_ERR_CUDA;
+        if (last) break;
+        in_list = out_list;
+        in_count = out_count;
+        P_round = P_round * 2 < P_expand ? P_round * 2 : P_expand;
+        if (++round >= kMaxExpandRounds) return VSA_ERR_INVALID_ARGUMENT;   // (P >= 1, P_expand <= 128: not reached)
+    }
     e = vsa::launch_dense(g, q, k_cache, v_cache, block_table, seq_lens, fallback_list, fallback_count, epsilon,
                           out, diag, ws_dense, st, /*tickets_cleared=*/true);
     return cuda_rc(e);

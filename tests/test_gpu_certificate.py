@@ -231,32 +231,58 @@ def test_expansion_retries_the_refused_units_with_more_pages_before_the_dense_pa
         refused = (ce.certified == 0) & (sp.n_candidates < sl[:, None])
         return rt, sp, ce, refused
 
-    rt1, sp1, ce1, ref1 = one_pass(P)
-    rt2, sp2, ce2, ref2 = one_pass(P2)
+    # the loop: P, 2P, ... up to P2; a unit's state is that of the last pass it took part in
+    passes, p = [], P
+    while True:
+        passes.append((p,) + one_pass(p))
+        if p >= P2:
+            break
+        p = min(2 * p, P2)
+    assert len(passes) == 3, "6 -> 12 -> 24 pages"
+    active = np.ones((Bn, H), bool)            # units that run the current pass
+    last_pass = np.zeros((Bn, H), int)
+    for k, (_, _, _, _, refused) in enumerate(passes):
+        last_pass[active] = k
+        active = active & refused
+    final_fb = active
+    ref1 = passes[0][4]
     assert ref1.any() and not ref1.all(), "the workload should refuse some units with P pages and keep others"
-    final_fb = ref1 & ref2
-    assert (ref1 & ~ref2).any(), "the expansion should rescue some units"
+    assert (ref1 & ~final_fb).any(), "the expansion should rescue some units"
     assert final_fb.any(), "and leave at least one to the dense pass"
-    # routed pages: first pass rows padded with -1, retried rows from the second pass
+    assert (last_pass == 1).any() and (last_pass == 2).any(), "both retry passes should end some unit"
+
+    def pick(field):
+        out_ = None
+        for k, (_, rt, sp, ce, _) in enumerate(passes):
+            a = field(rt, sp, ce)
+            out_ = a.copy() if out_ is None else np.where(last_pass == k, a, out_)
+        return out_
+
     want_routed = np.full((Bn, H, P2), -1, np.int32)
-    want_routed[:, :, :P] = rt1.pages
-    want_routed[ref1] = rt2.pages[ref1]
+    for k, (pk, rt, _, _, _) in enumerate(passes):
+        rows = last_pass == k
+        want_routed[rows, :pk] = rt.pages[rows]
     assert np.array_equal(routed.cpu().numpy(), want_routed)
     c = {k: v.numpy().reshape(Bn, H) for k, v in B.cert_to_dict(cert).items()}
     d = {k: v.numpy().reshape(Bn, H) for k, v in B.diag_to_dict(diag).items()}
-    for name, a1, a2 in (("delta_cert", ce1.delta_cert, ce2.delta_cert), ("ub_unrouted", ce1.ub_unrouted, ce2.ub_unrouted)):
-        want = np.where(ref1, a2, a1)
+    for name in ("delta_cert", "ub_unrouted"):
+        want = pick(lambda rt, sp, ce: getattr(ce, name))
         assert np.array_equal(c[name].view(np.uint32), want.view(np.uint32)), name
-    assert np.array_equal(c["certified"], np.where(ref1, ce2.certified, ce1.certified))
-    assert np.array_equal(d["n_candidates"], np.where(ref1, sp2.n_candidates, sp1.n_candidates))
-    assert np.array_equal(d["delta"], np.where(ref1, sp2.delta, sp1.delta))
+    assert np.array_equal(c["certified"], pick(lambda rt, sp, ce: ce.certified))
+    assert np.array_equal(d["n_candidates"], pick(lambda rt, sp, ce: sp.n_candidates))
+    assert np.array_equal(d["delta"], pick(lambda rt, sp, ce: sp.delta))
     assert np.array_equal(d["fallback"], final_fb.astype(np.int32))
+    def pick_out():
+        o = None
+        for k, (_, _, sp, _, _) in enumerate(passes):
+            o = sp.out.copy() if o is None else np.where((last_pass == k)[..., None], sp.out, o)
+        return o
+    sp_last_out = pick_out().reshape(Bn * H, -1)
     n = int(fcount.item())
     assert np.array_equal(np.sort(flist[:n].cpu().numpy()), np.nonzero(final_fb.reshape(-1))[0])
     got = out.cpu().numpy().reshape(Bn * H, -1)
-    first, second, dense_rows = (~ref1).reshape(-1), (ref1 & ~ref2).reshape(-1), final_fb.reshape(-1)
-    check_out(got[first], sp1.out.reshape(Bn * H, -1)[first], "units certified by the first pass")
-    check_out(got[second], sp2.out.reshape(Bn * H, -1)[second], "units certified after the expansion")
+    sparse_rows, dense_rows = (~final_fb).reshape(-1), final_fb.reshape(-1)
+    check_out(got[sparse_rows], sp_last_out[sparse_rows], "units certified by their last sparse pass")
     if dense_rows.any():
         dn = oracle.dense(geo, q, K, V, bt, sl, w.epsilon, unit_mask=final_fb.astype(np.int32))
         check_out(got[dense_rows], dn.out.reshape(Bn * H, -1)[dense_rows], "units that fell back")
