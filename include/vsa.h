@@ -101,6 +101,9 @@ typedef struct {
 #define VSA_WS_STEP 4
 #define VSA_WS_STEP_CERTIFIED 5
 #define VSA_WS_STEP_EXPAND 6
+#define VSA_WS_ROUTE_TWO_LEVEL 7 /* vsa_workspace_bytes: pass P_super in the P argument */
+#define VSA_WS_STEP_TWO_LEVEL 8  /* likewise                                            */
+#define VSA_SUPER_PAGES 16       /* logical pages per super-page                        */
 
 /*
  * Page summaries (Sec. 7 step 1: "coarse page summaries k_page"; the paper leaves them
@@ -321,6 +324,45 @@ int vsa_decode_step_certified_expand(const vsa_shape_t* shape, const void* q, co
                                      vsa_diag_t* diag, vsa_cert_t* cert, int32_t* routed_pages,
                                      int32_t* fallback_list, int32_t* fallback_count, void* ws, size_t ws_bytes,
                                      void* stream);
+
+/*
+ * Two-level page routing: an approximate pre-filter in front of Sec. 7 step 1 (the paper says only
+ * "coarse page summaries"; the construction is this library's).  A super-page is VSA_SUPER_PAGES
+ * consecutive LOGICAL pages of a sequence; its representative is the page summary with the largest
+ * squared norm among them (fp32 in the library's fixed summation order, ties to the lowest page).
+ * Routing scores the representatives (1/16 of the rows the full scan reads), keeps the P_super best
+ * super-pages per query head (score descending, super-page ascending), scores the pages inside them
+ * exactly - the same numbers the full scan produces - and keeps the P best of those (score
+ * descending, page ascending).  With P_super >= the number of super-pages the result equals
+ * vsa_route_pages; otherwise a page whose super-page was not kept is lost.
+ *
+ * vsa_build_super_summaries (cache maintenance, after vsa_build_page_summaries):
+ *   summaries: device bf16 [num_pool_pages][n_kv_heads][head_dim].
+ *   first_super: device int32 [batch] or NULL: first super-page of each sequence to (re)build, e.g.
+ *     (seq_len - 1) / (16 * VSA_SUPER_PAGES) after appending one token.
+ *   super_summaries: device bf16 [batch][ceil(max_pages_per_seq / 16)][n_kv_heads][head_dim], in the
+ *     sequence's logical order (zero rows past the sequence).
+ *   super_rep: device int32 [batch][ceil(max_pages_per_seq / 16)][n_kv_heads] or NULL: the logical page
+ *     chosen (-1 past the sequence).
+ * vsa_route_pages_two_level: arguments as vsa_route_pages, plus super_summaries, P_super (1..128) and
+ *   super_routed: device int32 [batch][n_q_heads][P_super] or NULL, the kept super-pages, -1 padded.
+ *   ws: vsa_workspace_bytes(shape, P_super, 0, VSA_WS_ROUTE_TWO_LEVEL) bytes.
+ * vsa_decode_step_two_level: vsa_decode_step with the two-level routing in place of the full scan;
+ *   ws: vsa_workspace_bytes(shape, P_super, K_c, VSA_WS_STEP_TWO_LEVEL) bytes.
+ */
+int vsa_build_super_summaries(const vsa_shape_t* shape, const void* summaries, const int32_t* block_table,
+                              const int32_t* seq_lens, const int32_t* first_super, void* super_summaries,
+                              int32_t* super_rep, void* stream);
+int vsa_route_pages_two_level(const vsa_shape_t* shape, const void* q, const void* summaries,
+                              const void* super_summaries, const int32_t* block_table, const int32_t* seq_lens,
+                              int32_t P_super, int32_t P, int32_t* routed_pages, float* routed_scores,
+                              int32_t* super_routed, void* ws, size_t ws_bytes, void* stream);
+int vsa_decode_step_two_level(const vsa_shape_t* shape, const void* q, const void* summaries,
+                              const void* super_summaries, const void* k_cache, const void* v_cache,
+                              const int32_t* block_table, const int32_t* seq_lens, int32_t P_super, int32_t P,
+                              int32_t K_c, float epsilon, float gap_threshold, float* out, vsa_diag_t* diag,
+                              int32_t* routed_pages, int32_t* fallback_list, int32_t* fallback_count, void* ws,
+                              size_t ws_bytes, void* stream);
 
 /*
  * vsa_decode_step with CUDA events recorded on `stream` between its kernels, for per-kernel

@@ -17,6 +17,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libvsa.so")
 
 VSA_WS_ROUTE, VSA_WS_SPARSE, VSA_WS_DENSE, VSA_WS_STEP, VSA_WS_STEP_CERTIFIED, VSA_WS_STEP_EXPAND = 1, 2, 3, 4, 5, 6
+VSA_WS_ROUTE_TWO_LEVEL, VSA_WS_STEP_TWO_LEVEL = 7, 8
+VSA_SUPER_PAGES = 16
 DIAG_BYTES = 32
 DIAG_FIELDS = ("delta", "delta12", "s_max", "lse", "leak_bound", "n_candidates", "fallback", "status")
 
@@ -64,6 +66,10 @@ def lib() -> C.CDLL:
         _lib.vsa_workspace_bytes.argtypes = [shp, i32, i32, C.c_int]
         _lib.vsa_build_page_summaries.argtypes = [shp, vp, vp, vp, vp, vp, vp]
         _lib.vsa_route_pages.argtypes = [shp, vp, vp, vp, vp, i32, vp, vp, vp, sz, vp]
+        _lib.vsa_build_super_summaries.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp]
+        _lib.vsa_route_pages_two_level.argtypes = [shp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, sz, vp]
+        _lib.vsa_decode_step_two_level.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, f32, f32,
+                                                   vp, vp, vp, vp, vp, vp, sz, vp]
         _lib.vsa_route_pages_static.argtypes = [shp, vp, vp, vp, vp, i32, vp, vp, vp]
         _lib.vsa_route_pages_static.restype = C.c_int
         _lib.vsa_sparse_decode.argtypes = [shp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, vp, vp, vp, vp, vp, sz, vp]
@@ -152,6 +158,38 @@ def vsa_route_pages(shape, q, summaries, block_table, seq_lens, P, routed_pages,
                                  _ptr(routed_pages), _ptr(routed_scores), _ptr(ws),
                                  0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
            "vsa_route_pages")
+
+
+def n_super_pages(shape: vsa_shape_t) -> int:
+    return (shape.max_pages_per_seq + VSA_SUPER_PAGES - 1) // VSA_SUPER_PAGES
+
+
+def vsa_build_super_summaries(shape, summaries, block_table, seq_lens, first_super, super_summaries,
+                              super_rep=None, stream=None) -> None:
+    _check(lib().vsa_build_super_summaries(C.byref(shape), _ptr(summaries), _ptr(block_table), _ptr(seq_lens),
+                                           _ptr(first_super), _ptr(super_summaries), _ptr(super_rep),
+                                           _stream(stream)),
+           "vsa_build_super_summaries")
+
+
+def vsa_route_pages_two_level(shape, q, summaries, super_summaries, block_table, seq_lens, P_super, P,
+                              routed_pages, routed_scores, super_routed, ws, stream=None) -> None:
+    _check(lib().vsa_route_pages_two_level(C.byref(shape), _ptr(q), _ptr(summaries), _ptr(super_summaries),
+                                           _ptr(block_table), _ptr(seq_lens), P_super, P, _ptr(routed_pages),
+                                           _ptr(routed_scores), _ptr(super_routed), _ptr(ws),
+                                           0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
+           "vsa_route_pages_two_level")
+
+
+def vsa_decode_step_two_level(shape, q, summaries, super_summaries, k_cache, v_cache, block_table, seq_lens,
+                              P_super, P, K_c, epsilon, gap_threshold, out, diag, routed_pages, fallback_list,
+                              fallback_count, ws, stream=None) -> None:
+    _check(lib().vsa_decode_step_two_level(C.byref(shape), _ptr(q), _ptr(summaries), _ptr(super_summaries),
+                                           _ptr(k_cache), _ptr(v_cache), _ptr(block_table), _ptr(seq_lens),
+                                           P_super, P, K_c, epsilon, gap_threshold, _ptr(out), _ptr(diag),
+                                           _ptr(routed_pages), _ptr(fallback_list), _ptr(fallback_count), _ptr(ws),
+                                           0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
+           "vsa_decode_step_two_level")
 
 
 VSA_STATIC_ROUTE_SCORES = 1 << 20

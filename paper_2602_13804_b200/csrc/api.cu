@@ -115,6 +115,51 @@ size_t step_retry_bytes(const Geometry& g)
 
 int cuda_rc(cudaError_t e) { return e == cudaSuccess ? VSA_OK : VSA_ERR_CUDA; }
 
+// two-level routing scratch: [ page scores | representative scores | identity table | lengths in
+// super-pages | kept super-pages per unit ], each part 256-byte aligned; the step adds the dense scratch
+struct TwoLevelWs {
+    size_t super_scores, bt_super, sl_super, super_routed, dense, total_route;
+};
+TwoLevelWs two_level_layout(const Geometry& g, int P_super)
+{
+    const Geometry gs = vsa::two_level_super_geometry(g);
+    TwoLevelWs w;
+    size_t o = step_route_part(g);
+    w.super_scores = o;
+    o += align_up(vsa::route_workspace_bytes(gs), 256);
+    w.bt_super = o;
+    o += align_up((size_t)g.batch * gs.max_pages * sizeof(int32_t), 256);
+    w.sl_super = o;
+    o += align_up((size_t)g.batch * sizeof(int32_t), 256);
+    w.super_routed = o;
+    o += align_up((size_t)g.batch * g.n_q_heads * (size_t)P_super * sizeof(int32_t), 256);
+    w.dense = o;
+    w.total_route = o;
+    return w;
+}
+
+// prep -> representative scan -> top-P_super super-pages -> exact scores inside them (into the page-score
+// scratch at the start of ws).  zero_word / tickets: cleared by the representative scan for the step.
+int two_level_scores(const Geometry& g, const void* q, const void* summaries, const void* super_summaries,
+                     const int32_t* block_table, const int32_t* seq_lens, int P_super, int32_t* super_routed_out,
+                     void* ws, int32_t* zero_word, int32_t* zero_words, int zero_count, cudaStream_t st)
+{
+    const TwoLevelWs w = two_level_layout(g, P_super);
+    const Geometry gs = vsa::two_level_super_geometry(g);
+    char* base = (char*)ws;
+    int32_t* bt_super = (int32_t*)(base + w.bt_super);
+    int32_t* sl_super = (int32_t*)(base + w.sl_super);
+    int32_t* super_routed = super_routed_out ? super_routed_out : (int32_t*)(base + w.super_routed);
+    if (vsa::launch_two_level_prep(g, seq_lens, sl_super, bt_super, st) != cudaSuccess) return VSA_ERR_CUDA;
+    if (vsa::launch_route_scan(gs, q, super_summaries, bt_super, sl_super, base + w.super_scores, zero_word,
+                               zero_words, zero_count, st) != cudaSuccess)
+        return VSA_ERR_CUDA;
+    if (vsa::launch_route_select(gs, base + w.super_scores, sl_super, P_super, super_routed, nullptr, st) !=
+        cudaSuccess)
+        return VSA_ERR_CUDA;
+    return cuda_rc(vsa::launch_inner_scan(g, q, summaries, block_table, seq_lens, super_routed, P_super, (float*)ws, st));
+}
+
 }  // namespace
 
 extern "C" {
@@ -138,7 +183,6 @@ size_t vsa_workspace_bytes(const vsa_shape_t* shape, int32_t P, int32_t K_c, int
 {
     Geometry g;
     if (make_geometry(shape, &g) != VSA_OK) return 0;
-    (void)P;
     (void)K_c;
     switch (which_call) {
         case VSA_WS_ROUTE: return vsa::route_workspace_bytes(g);
@@ -147,6 +191,9 @@ size_t vsa_workspace_bytes(const vsa_shape_t* shape, int32_t P, int32_t K_c, int
         case VSA_WS_STEP: return step_route_part(g) + vsa::dense_workspace_bytes(g);
         case VSA_WS_STEP_CERTIFIED: return step_rad_offset(g) + step_rad_bytes(g);
         case VSA_WS_STEP_EXPAND: return step_retry_offset(g) + step_retry_bytes(g);
+        // (for the two-level kinds the P argument is P_super, the number of super-pages kept per unit)
+        case VSA_WS_ROUTE_TWO_LEVEL: return P >= 1 ? two_level_layout(g, P).total_route : 0;
+        case VSA_WS_STEP_TWO_LEVEL: return P >= 1 ? two_level_layout(g, P).dense + vsa::dense_workspace_bytes(g) : 0;
         default: return 0;
     }
 }
@@ -205,6 +252,76 @@ int vsa_route_pages(const vsa_shape_t* shape, const void* q, const void* summari
                                            (cudaStream_t)stream);
     if (e != cudaSuccess) return VSA_ERR_CUDA;
     return cuda_rc(vsa::launch_route_select(g, ws, seq_lens, P, routed_pages, routed_scores, (cudaStream_t)stream));
+}
+
+int vsa_build_super_summaries(const vsa_shape_t* shape, const void* summaries, const int32_t* block_table,
+                              const int32_t* seq_lens, const int32_t* first_super, void* super_summaries,
+                              int32_t* super_rep, void* stream)
+{
+    Geometry g;
+    int rc = make_geometry(shape, &g);
+    if (rc) return rc;
+    if (!summaries || !block_table || !seq_lens || !super_summaries) return VSA_ERR_INVALID_ARGUMENT;
+    if (!aligned16(summaries) || !aligned16(super_summaries)) return VSA_ERR_MISALIGNED;
+    return cuda_rc(vsa::launch_build_super_summaries(g, summaries, block_table, seq_lens, first_super,
+                                                     super_summaries, super_rep, (cudaStream_t)stream));
+}
+
+int vsa_route_pages_two_level(const vsa_shape_t* shape, const void* q, const void* summaries,
+                              const void* super_summaries, const int32_t* block_table, const int32_t* seq_lens,
+                              int32_t P_super, int32_t P, int32_t* routed_pages, float* routed_scores,
+                              int32_t* super_routed, void* ws, size_t ws_bytes, void* stream)
+{
+    Geometry g;
+    int rc = make_geometry(shape, &g);
+    if (rc) return rc;
+    if ((rc = check_routing_sizes(g, P, 0, false))) return rc;
+    if ((rc = check_routing_sizes(g, P_super, 0, false))) return rc;
+    if (!q || !summaries || !super_summaries || !block_table || !seq_lens || !routed_pages || !ws)
+        return VSA_ERR_INVALID_ARGUMENT;
+    if (!aligned16(q) || !aligned16(summaries) || !aligned16(super_summaries) || !aligned16(ws))
+        return VSA_ERR_MISALIGNED;
+    if (ws_bytes < two_level_layout(g, P_super).total_route) return VSA_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = (cudaStream_t)stream;
+    if ((rc = two_level_scores(g, q, summaries, super_summaries, block_table, seq_lens, P_super, super_routed, ws,
+                               nullptr, nullptr, 0, st)))
+        return rc;
+    return cuda_rc(vsa::launch_route_select(g, ws, seq_lens, P, routed_pages, routed_scores, st));
+}
+
+int vsa_decode_step_two_level(const vsa_shape_t* shape, const void* q, const void* summaries,
+                              const void* super_summaries, const void* k_cache, const void* v_cache,
+                              const int32_t* block_table, const int32_t* seq_lens, int32_t P_super, int32_t P,
+                              int32_t K_c, float epsilon, float gap_threshold, float* out, vsa_diag_t* diag,
+                              int32_t* routed_pages, int32_t* fallback_list, int32_t* fallback_count, void* ws,
+                              size_t ws_bytes, void* stream)
+{
+    Geometry g;
+    int rc = make_geometry(shape, &g);
+    if (rc) return rc;
+    if ((rc = check_routing_sizes(g, P, K_c, true))) return rc;
+    if ((rc = check_routing_sizes(g, P_super, 0, false))) return rc;
+    if ((rc = check_epsilon(epsilon))) return rc;
+    if (isnan(gap_threshold)) return VSA_ERR_INVALID_ARGUMENT;
+    if (!q || !summaries || !super_summaries || !k_cache || !v_cache || !block_table || !seq_lens || !out || !diag ||
+        !routed_pages || !fallback_list || !fallback_count || !ws)
+        return VSA_ERR_INVALID_ARGUMENT;
+    if (!aligned16(q) || !aligned16(summaries) || !aligned16(super_summaries) || !aligned16(k_cache) ||
+        !aligned16(v_cache) || !aligned16(ws))
+        return VSA_ERR_MISALIGNED;
+    const TwoLevelWs w = two_level_layout(g, P_super);
+    if (ws_bytes < w.dense + vsa::dense_workspace_bytes(g)) return VSA_ERR_WORKSPACE_TOO_SMALL;
+    if (!vsa::sparse_shared_memory_fits(g, P, K_c, true, false, false)) return VSA_ERR_UNSUPPORTED_SHAPE;
+    cudaStream_t st = (cudaStream_t)stream;
+    void* ws_dense = (char*)ws + w.dense;
+    if ((rc = two_level_scores(g, q, summaries, super_summaries, block_table, seq_lens, P_super, nullptr, ws,
+                               fallback_count, vsa::dense_tickets(ws_dense), vsa::dense_ticket_count(g), st)))
+        return rc;
+    cudaError_t e = vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, routed_pages, (const float*)ws,
+                                       P, K_c, epsilon, gap_threshold, out, diag, fallback_list, fallback_count, st);
+    if (e != cudaSuccess) return VSA_ERR_CUDA;
+    return cuda_rc(vsa::launch_dense(g, q, k_cache, v_cache, block_table, seq_lens, fallback_list, fallback_count,
+                                     epsilon, out, diag, ws_dense, st, /*tickets_cleared=*/true));
 }
 
 int vsa_sparse_decode(const vsa_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,

@@ -1,0 +1,184 @@
+// Two-level page routing: an approximate pre-filter in front of the exact page scoring (paper Sec. 7
+// step 1 speaks only of "coarse page summaries"; this construction is the library's).
+//
+// A super-page is 16 consecutive logical pages of a sequence.  Its representative is the page summary
+// with the largest squared norm among its pages (fp32, the library's fixed summation order; ties go to
+// the lowest page): keys of large norm are the ones that can dominate an inner product, so the best
+// page score inside a super-page is usually its representative's.  Routing then takes three short
+// steps instead of one scan over every page: score the representatives (1/16 of the rows), keep the
+// P_super best super-pages per query head, score the pages inside those exactly.  The page scores
+// are the same numbers the full scan would produce, so whatever is routed is routed in the exact
+// order; what the pre-filter can lose is a page whose super-page was not kept.
+//
+//   super_summaries_kernel  cache maintenance: representative (and its logical page) per super-page
+//   two_level_prep_kernel   per step: lengths in super-pages, identity table for the representative scan
+//   inner_scan_kernel       per unit: -inf over the unit's score row, exact scores of the kept super-pages
+#include <math.h>
+
+#include "vsa_device.cuh"
+#include "vsa_launch.h"
+
+namespace vsa {
+
+namespace {
+
+constexpr int kSuper = 16;   // logical pages per super-page
+
+// One half-warp per (sequence, super-page, KV head): lane c holds columns 8c .. 8c+7 of each of the
+// super-page's summary rows.
+__global__ void __launch_bounds__(256)
+super_summaries_kernel(Geometry geo, const uint16_t* __restrict__ summaries, const int32_t* __restrict__ block_table,
+                       const int32_t* __restrict__ seq_lens, const int32_t* __restrict__ first_super, int max_supers,
+                       uint16_t* __restrict__ super_summaries, int32_t* __restrict__ super_rep)
+{
+    const int b = blockIdx.y;
+    const long long hw = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 4;   // (super-page, KV head)
+    const int lane = threadIdx.x & 31, c = lane & 15;
+    const unsigned hmask = 0xffffu << (lane & 16);
+    const int g = (int)(hw % geo.n_kv_heads);
+    const long long sp = hw / geo.n_kv_heads;
+    if (sp >= max_supers) return;
+    const int T = seq_lens[b];
+    const bool okT = T > 0 && T <= geo.max_pages * kPageSize;
+    const int nb = okT ? (T + kPageSize - 1) / kPageSize : 0;
+    if (first_super && sp < first_super[b]) return;
+    const long long o = ((long long)b * max_supers + sp) * geo.n_kv_heads + g;
+    int best = -1;
+    float best_n = 0.0f;
+    uint4 best_row = make_uint4(0u, 0u, 0u, 0u);
+    for (int l = (int)sp * kSuper; l < ((int)sp + 1) * kSuper && l < nb; ++l) {
+        const long long p = block_table[(long long)b * geo.max_pages + l];
+        if (p < 0 || p >= geo.pool_pages) continue;   // an entry outside the pool is no candidate
+        const uint4 row = ld_nc_16B(summaries + (p * geo.n_kv_heads + g) * kHeadDim + c * 8);
+        float f[8];
+        unpack8(row, f);
+        float n2 = chunk_partial(f, f);
+#pragma unroll
+        for (int off = 8; off; off >>= 1) n2 = n2 + __shfl_xor_sync(hmask, n2, off);
+        if (best < 0 || n2 > best_n) {
+            best = l;
+            best_n = n2;
+            best_row = row;
+        }
+    }
+    *reinterpret_cast<uint4*>(super_summaries + o * kHeadDim + c * 8) = best_row;
+    if (super_rep && c == 0) super_rep[o] = best;
+}
+
+// sl_super[b] = 16 * (super-pages of sequence b), so that the page-routing kernels, which derive a page
+// count from a token count, see one "page" per super-page; an invalid length stays invalid.
+// bt_super[b][s] = b * max_supers + s: the representatives are stored in logical order per sequence.
+__global__ void two_level_prep_kernel(Geometry geo, const int32_t* __restrict__ seq_lens, int max_supers,
+                                      int32_t* __restrict__ sl_super, int32_t* __restrict__ bt_super)
+{
+    // No early trigger for the kernel that follows: it reads these arrays before its own wait (they are
+    // "scheduler state" to it), so it may only start once this kernel has completed.
+    pdl_wait();
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < geo.batch) {
+        const int T = seq_lens[i];
+        int v;
+        if (T <= 0) v = 0;
+        else if (T > geo.max_pages * kPageSize) v = max_supers * kPageSize + 1;
+        else v = (((T + kPageSize - 1) / kPageSize + kSuper - 1) / kSuper) * kPageSize;
+        sl_super[i] = v;
+    }
+    if (i < geo.batch * max_supers) bt_super[i] = i;
+}
+
+// One block per (sequence, query head): the unit's score row [0, n_b) is set to -inf, then every page
+// of the unit's kept super-pages gets its exact score (one super-page = 16 summary rows = one
+// 16-value reduction per half-warp, lane c ending with the score of page 16 s + c).
+__global__ void __launch_bounds__(256)
+inner_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* __restrict__ summaries,
+                  const int32_t* __restrict__ block_table, const int32_t* __restrict__ seq_lens,
+                  const int32_t* __restrict__ super_routed, int P_super, float* __restrict__ scores)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, c = lane & 15, gi = lane >> 4;
+    const unsigned hmask = 0xffffu << (lane & 16);
+    const long long unit = blockIdx.x;
+    const int b = (int)(unit / geo.n_q_heads), h = (int)(unit % geo.n_q_heads), g = h / geo.group;
+    const int T = ld_ca_s32(seq_lens + b);
+    const uint4 qraw = ld_nc_16B(q + unit * kHeadDim + c * 8);
+    pdl_wait();
+    pdl_launch_dependents();
+    if (T <= 0 || T > geo.max_pages * kPageSize) return;
+    const int nb = (T + kPageSize - 1) / kPageSize;
+    float* row = scores + unit * geo.max_pages;
+    for (int i = tid; i < nb; i += blockDim.x) row[i] = -INFINITY;
+    __syncthreads();
+    float qf[8];
+    unpack8(qraw, qf);
+    const int32_t* bt = block_table + (long long)b * geo.max_pages;
+    for (int j = warp * 2 + gi; j < P_super; j += 16) {
+        const int sp = super_routed[unit * P_super + j];
+        if (sp < 0) continue;   // (the same for the sixteen lanes of the half-warp)
+        const int l = sp * kSuper + c;
+        long long phys = -1;
+        if (l < nb) {
+            phys = bt[l];
+            if (phys < 0 || phys >= geo.pool_pages) phys = -1;
+        }
+        uint4 rows[kSuper];
+#pragma unroll
+        for (int r = 0; r < kSuper; ++r) {
+            const long long pr = __shfl_sync(hmask, phys, (lane & 16) | r);
+            rows[r] = pr >= 0 ? ld_nc_16B(summaries + (pr * geo.n_kv_heads + g) * kHeadDim + c * 8)
+                              : make_uint4(0u, 0u, 0u, 0u);
+        }
+        float vals[16];
+#pragma unroll
+        for (int r = 0; r < kSuper; ++r) {
+            float kf[8];
+            unpack8(rows[r], kf);
+            vals[r] = chunk_partial(qf, kf);
+        }
+        const float s = reduce_scatter16(vals, c, hmask);
+        if (l < nb && phys >= 0) row[l] = s;
+    }
+}
+
+}  // namespace
+
+int two_level_max_supers(const Geometry& g) { return (g.max_pages + kSuper - 1) / kSuper; }
+
+// geometry of the representative scan: one "page" per super-page, representatives in logical order
+Geometry two_level_super_geometry(const Geometry& g)
+{
+    Geometry s = g;
+    s.max_pages = two_level_max_supers(g);
+    s.pool_pages = (long long)g.batch * s.max_pages;
+    return s;
+}
+
+cudaError_t launch_build_super_summaries(const Geometry& g, const void* summaries, const int32_t* block_table,
+                                         const int32_t* seq_lens, const int32_t* first_super, void* super_summaries,
+                                         int32_t* super_rep, cudaStream_t stream)
+{
+    const int ms = two_level_max_supers(g);
+    const long long halfwarps = (long long)ms * g.n_kv_heads;
+    const dim3 grid((unsigned)((halfwarps * 16 + 255) / 256), (unsigned)g.batch);
+    super_summaries_kernel<<<grid, 256, 0, stream>>>(g, (const uint16_t*)summaries, block_table, seq_lens,
+                                                     first_super, ms, (uint16_t*)super_summaries, super_rep);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_two_level_prep(const Geometry& g, const int32_t* seq_lens, int32_t* sl_super, int32_t* bt_super,
+                                  cudaStream_t stream)
+{
+    const int ms = two_level_max_supers(g);
+    const int n = g.batch * ms;
+    return launch_pdl(two_level_prep_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, stream, g, seq_lens, ms,
+                      sl_super, bt_super);
+}
+
+cudaError_t launch_inner_scan(const Geometry& g, const void* q, const void* summaries, const int32_t* block_table,
+                              const int32_t* seq_lens, const int32_t* super_routed, int P_super, float* scores,
+                              cudaStream_t stream)
+{
+    return launch_pdl(inner_scan_kernel, dim3((unsigned)(g.batch * g.n_q_heads)), dim3(256), 0, stream, g,
+                      (const uint16_t*)q, (const uint16_t*)summaries, block_table, seq_lens, super_routed, P_super,
+                      scores);
+}
+
+}  // namespace vsa

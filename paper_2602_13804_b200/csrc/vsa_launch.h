@@ -96,6 +96,18 @@ cudaError_t launch_route_scan(const Geometry& g, const void* q, const void* summ
 cudaError_t launch_route_select(const Geometry& g, const void* ws, const int32_t* seq_lens, int P,
                                 int32_t* routed_pages, float* routed_scores, cudaStream_t stream);
 
+// ---- two-level routing (two_level.cu) -----------------------------------------------------------
+int two_level_max_supers(const Geometry& g);
+Geometry two_level_super_geometry(const Geometry& g);
+cudaError_t launch_build_super_summaries(const Geometry& g, const void* summaries, const int32_t* block_table,
+                                         const int32_t* seq_lens, const int32_t* first_super, void* super_summaries,
+                                         int32_t* super_rep, cudaStream_t stream);
+cudaError_t launch_two_level_prep(const Geometry& g, const int32_t* seq_lens, int32_t* sl_super, int32_t* bt_super,
+                                  cudaStream_t stream);
+cudaError_t launch_inner_scan(const Geometry& g, const void* q, const void* summaries, const int32_t* block_table,
+                              const int32_t* seq_lens, const int32_t* super_routed, int P_super, float* scores,
+                              cudaStream_t stream);
+
 // ---- fused sparse pass ------------------------------------------------------------------------
 // page_scores == nullptr: routed_pages is read; otherwise the top-P selection runs inside the kernel on
 // page_scores (the scan's output) and routed_pages is written.  solve != nullptr: the weights on the

@@ -91,6 +91,27 @@ class SparsePagedDecoder:
                                     self.routed_pages, self.fallback_list, self.fallback_count, self.ws_cert)
         return self.out
 
+    def build_super_summaries(self, summaries, block_table, seq_lens, first_super=None) -> torch.Tensor:
+        """Representative summary per 16 logical pages (cache maintenance for step_two_level)."""
+        if not hasattr(self, "super_summaries"):
+            self.super_summaries = torch.zeros((self.shape.batch, B.n_super_pages(self.shape), self.shape.n_kv_heads,
+                                                self.shape.head_dim), dtype=torch.bfloat16, device=self.device)
+        B.vsa_build_super_summaries(self.shape, summaries, block_table, seq_lens, first_super, self.super_summaries)
+        return self.super_summaries
+
+    def step_two_level(self, q, summaries, super_summaries, k_cache, v_cache, block_table, seq_lens,
+                       P_super: int) -> torch.Tensor:
+        """The step with two-level routing: only the pages of the P_super best super-pages are scored."""
+        if getattr(self, "_P_super", None) != int(P_super):
+            self._P_super = int(P_super)
+            self.ws_two_level = B.alloc_workspace(self.shape, self._P_super, self.K_c, B.VSA_WS_STEP_TWO_LEVEL,
+                                                  self.device)
+        B.vsa_decode_step_two_level(self.shape, q, summaries, super_summaries, k_cache, v_cache, block_table,
+                                    seq_lens, self._P_super, self.P, self.K_c, self.epsilon, self.gap_threshold,
+                                    self.out, self.diag, self.routed_pages, self.fallback_list,
+                                    self.fallback_count, self.ws_two_level)
+        return self.out
+
     def append(self, k_new, v_new, k_cache, v_cache, block_table, seq_lens_after, summaries, radii=None) -> None:
         """Append one token per sequence (lengths AFTER the append) and refresh its page's summary / radius."""
         B.vsa_append_kv(self.shape, k_new, v_new, k_cache, v_cache, block_table, seq_lens_after, summaries, radii)
