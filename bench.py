@@ -64,6 +64,9 @@ def parse_args(argv=None):
     ap.add_argument("--expand", type=int, default=None,
                     help="with --certified: retry the refused units with up to this many routed pages before the "
                          "dense pass (vsa_decode_step_certified_expand)")
+    ap.add_argument("--two-level", type=int, default=None, metavar="P_SUPER",
+                    help="time vsa_decode_step_two_level: only the pages of the P_SUPER best super-pages (16 pages "
+                         "each, scored through one representative summary) are scored per unit")
     ap.add_argument("--solver", default="eg", choices=["eg", "fw"],
                     help="with --solver-iters: entropic mirror descent (eg) or Frank-Wolfe with exact line search (fw)")
     ap.add_argument("--solver-iters", type=int, default=None,
@@ -332,7 +335,9 @@ class Harness:
         self.fcount = torch.zeros(1, dtype=torch.int32, device=dev)
         self.ws = B.alloc_workspace(shape, P, K_c, B.VSA_WS_STEP, dev)
         self.ws_dense = B.alloc_workspace(shape, P, K_c, B.VSA_WS_DENSE, dev)
+        self.ws_plain = self.ws
         self.solve = self.cert = self.radii = None
+        self.routed_plain = self.routed
         a = args
         if a is not None and a.solver_iters is not None:
             self.solve = B.alloc_solve(units, dev)
@@ -347,6 +352,15 @@ class Harness:
                 r = torch.zeros((shape.num_pool_pages, shape.n_kv_heads), dtype=torch.float32, device=dev)
                 B.vsa_build_page_radii(shape, w.k_cache, s_, w.block_table, w.seq_lens, None, r)
                 self.radii.append(r)
+        self.supers = None
+        if a is not None and getattr(a, "two_level", None):
+            self.ws = B.alloc_workspace(shape, a.two_level, K_c, B.VSA_WS_STEP_TWO_LEVEL, dev)
+            self.supers = []
+            for w, s_ in zip(self.layers, self.summaries):      # cache maintenance, like the summaries
+                sp = torch.zeros((shape.batch, B.n_super_pages(shape), shape.n_kv_heads, shape.head_dim),
+                                 dtype=torch.bfloat16, device=dev)
+                B.vsa_build_super_summaries(shape, s_, w.block_table, w.seq_lens, None, sp)
+                self.supers.append(sp)
         self.stream = torch.cuda.Stream(device=dev)
         self.graph = None
 
@@ -360,6 +374,10 @@ class Harness:
         if a is not None and a.dense_baseline and not plain:
             B.vsa_dense_decode_fallback(shape, w.q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, None, None,
                                         eps, out, diag, self.ws_dense)
+        elif self.supers is not None and not plain:
+            B.vsa_decode_step_two_level(shape, w.q, s, self.supers[k], w.k_cache, w.v_cache, w.block_table,
+                                        w.seq_lens, a.two_level, P, K_c, eps, tau, out, diag, routed, flist, fcount,
+                                        ws)
         elif self.cert is not None and a.expand and not plain:
             B.vsa_decode_step_certified_expand(shape, w.q, s, self.radii[k], w.k_cache, w.v_cache, w.block_table,
                                                w.seq_lens, P, a.expand, K_c, eps, tau, out, diag, self.cert, routed,
@@ -375,7 +393,8 @@ class Harness:
                                        tau, a.solver_iters, out, diag, self.solve, routed, flist, fcount, ws)
         else:
             B.vsa_decode_step(shape, w.q, s, w.k_cache, w.v_cache, w.block_table, w.seq_lens, P, K_c, eps, tau,
-                              out, diag, routed, flist, fcount, ws)
+                              out, diag, routed if routed.shape[-1] == P else self.routed_plain, flist, fcount,
+                              self.ws_plain)
 
     def step_plain(self, plain=False):
         for i in range(self.L):
@@ -513,6 +532,31 @@ def measure_point(spec, dev, steps, want_kernels=True, use_graph=True, oracle_se
     return point
 
 
+def two_level_point(spec, dev, P_super, steps):
+    """The step with two-level routing against the plain step on the same caches, and the fraction of the
+    exact routing's pages that the pre-filter keeps (both page lists come from the GPU, last layer)."""
+    import numpy as np
+    a = parse_args(["--two-level", str(P_super)])
+    h = Harness(spec, dev, args=a)
+    res = {}
+    lists = {}
+    for name, plain in (("two_level", False), ("full_scan", True)):
+        step = h.capture(True, plain=plain)
+        with h.torch.cuda.stream(h.stream):
+            for _ in range(3):
+                step()
+        res[name] = h.time_steps(step, steps) / steps * 1e3 / h.L
+        lists[name] = h.routed.cpu().numpy().reshape(h.units, -1)
+    hit = tot = 0
+    for u in range(h.units):
+        e = set(int(x) for x in lists["full_scan"][u] if x >= 0)
+        hit += len(e & set(int(x) for x in lists["two_level"][u]))
+        tot += len(e)
+    h.release()
+    return {"workload": spec.name, "P_super": P_super, "us_per_layer": res["two_level"],
+            "us_per_layer_full_scan": res["full_scan"], "page_recall_vs_exact_routing": hit / max(tot, 1)}
+
+
 def sweep(dev, steps_small=200):
     """The context sweep at batch 1 (flatness), one fallback-regime point and one large scan point."""
     from dataclasses import replace
@@ -530,6 +574,11 @@ def sweep(dev, steps_small=200):
     # the scan where its traffic dominates: batch 16, T = 128k, two layer caches
     spec16 = config_spec(2, batch=16, T=131072, layers=2, name="cfg2_b16_t131072_2layers")
     out["scan_large"] = measure_point(spec16, dev, 40)
+    # two-level routing at batch 16: growth of the step from 4k to 128k against the full scan's
+    tl = [two_level_point(config_spec(2, batch=16, T=4096, layers=16, name="cfg2_b16_t4096"), dev, 32, 100),
+          two_level_point(spec16, dev, 32, 40)]
+    out["two_level_b16"] = {"points": tl, "growth_4k_to_128k": tl[1]["us_per_layer"] / tl[0]["us_per_layer"],
+                            "growth_4k_to_128k_full_scan": tl[1]["us_per_layer_full_scan"] / tl[0]["us_per_layer_full_scan"]}
     return out
 
 
@@ -633,6 +682,8 @@ def run_ours(args):
     kernels_per_layer = 1 if args.dense_baseline else 3   # scan, sparse (top-P selection fused in), dense
     if cert is not None and args.expand:
         kernels_per_layer = 3 + vsa_expand_rounds(P, args.expand)
+    if args.two_level:
+        kernels_per_layer = 6     # prep, representative scan, super-page selection, inner scan, sparse, dense
     use_graph = not args.no_graph
     step = h.capture(use_graph)
 
@@ -688,7 +739,7 @@ def run_ours(args):
 
         # ---- with --solver-iters / --certified: the closed-form step timed the same way ----
         closed_form_us_per_layer = None
-        if solve is not None or cert is not None:
+        if solve is not None or cert is not None or args.two_level:
             step_c = h.capture(use_graph, plain=True)
             for _ in range(3):
                 step_c()
@@ -697,7 +748,7 @@ def run_ours(args):
 
         # ---- end to end: q from pinned host memory, out + diag back to the host, every layer ----
         e2e = None
-        if not args.dense_baseline and solve is None and cert is None:
+        if not args.dense_baseline and solve is None and cert is None and not args.two_level:
             q_host = [w.q.cpu().pin_memory() for w in layers]
             q_dev = torch.empty_like(w0.q)
             out_host = torch.empty(out.shape, dtype=torch.float32).pin_memory()
@@ -790,7 +841,7 @@ def run_ours(args):
     else:
         kern = kernel_fracs(alg, per_kernel, step_us, peak)
         dom = max(("route_scan", "sparse_decode", "dense_fallback"), key=lambda k: per_kernel[k])
-        if solve is not None or cert is not None:
+        if solve is not None or cert is not None or args.two_level:
             # the events bracket the plain step's kernels; the cost of the iterations (of the certificate)
             # is the difference of the two graph-replayed steps and is booked on the sparse kernel
             extra = step_us - closed_form_us_per_layer
@@ -818,7 +869,7 @@ def run_ours(args):
 
     sweep_obj = None
     default_run = (args.workload == "cfg1" and not args.dense_baseline and solve is None and cert is None
-                   and args.P is None and args.Kc is None and args.layers is None)
+                   and args.P is None and args.Kc is None and args.layers is None and not args.two_level)
     if default_run and world == 1 and not args.no_sweep:
         h.release()
         del layers, summaries, w0, last, h
@@ -839,7 +890,9 @@ def run_ours(args):
                          f" MB touched per pass over them",
                    "launch": "cuda graph replay of the whole step" if use_graph else "plain stream launches",
                    "path": "dense split-K baseline" if args.dense_baseline else
-                           ((f"route -> sparse with routing certificate -> retries of the refused units with up to "
+                           (f"two-level route ({args.two_level} super-pages per unit) -> sparse -> dense fallback"
+                            if args.two_level else
+                            (f"route -> sparse with routing certificate -> retries of the refused units with up to "
                              f"{args.expand} pages -> dense fallback") if cert is not None and args.expand else
                             "route -> sparse with routing certificate -> dense fallback" if cert is not None else
                             "route -> sparse -> dense fallback" if solve is None else
