@@ -29,10 +29,13 @@
  *     than its block-table row, a non-positive length) never trap: the unit's
  *     diag.status becomes non-zero and its output row is zero-filled.
  *   - Inputs are assumed finite (no NaN/Inf in q, K, V).
- *   - v1 shapes: head_dim = 128, page_size = 16, n_q_heads / n_kv_heads in {1, 2, 4, 8},
+ *   - v1 shapes: head_dim = 128, page_size = 16, n_q_heads / n_kv_heads in {1, 2, 4, 8, 16, 32}
+ *     (multi-head, grouped-query and multi-query attention; groups of 16 and 32 query heads
+ *     are processed as two and four sub-groups of 8 that read the same KV head),
  *     1 <= P <= 128, 1 <= K_c <= P * page_size, max_pages_per_seq <= 32768,
- *     batch * n_kv_heads <= 4096, num_pool_pages * n_kv_heads < 2^27 (the summary pool is
- *     addressed in 16-byte units by a 32-bit offset).
+ *     batch * n_kv_heads <= 4096 (batch * n_q_heads / 8 <= 4096 for groups above 8),
+ *     num_pool_pages * n_kv_heads < 2^27 (the summary pool is addressed in 16-byte units by a
+ *     32-bit offset).
  *
  * Native layouts (row-major, last dimension contiguous)
  *   q            bf16 [batch][n_q_heads][head_dim]

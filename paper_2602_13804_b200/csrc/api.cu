@@ -52,16 +52,20 @@ int make_geometry(const vsa_shape_t* s, Geometry* g)
     if (s->kv_page_stride < 0 || s->kv_head_stride < 0 || s->kv_token_stride < 0) return VSA_ERR_INVALID_ARGUMENT;
     const int group = s->n_q_heads / s->n_kv_heads;
     if (s->head_dim != vsa::kHeadDim || s->page_size != vsa::kPageSize) return VSA_ERR_UNSUPPORTED_SHAPE;
-    if (group != 1 && group != 2 && group != 4 && group != 8) return VSA_ERR_UNSUPPORTED_SHAPE;
+    if (group != 1 && group != 2 && group != 4 && group != 8 && group != 16 && group != 32)
+        return VSA_ERR_UNSUPPORTED_SHAPE;
     if (s->max_pages_per_seq > kMaxPagesPerSeq) return VSA_ERR_UNSUPPORTED_SHAPE;
     if (s->num_pool_pages > 0x7fffffffLL) return VSA_ERR_UNSUPPORTED_SHAPE;
     if ((long long)s->batch * s->n_q_heads > 0x3fffffffLL) return VSA_ERR_UNSUPPORTED_SHAPE;
-    if ((long long)s->batch * s->n_kv_heads > 4096) return VSA_ERR_UNSUPPORTED_SHAPE;
+    // (sequence, KV head) pairs the dense pass tracks; groups above 8 count as n_q_heads / 8 heads there
+    if ((long long)s->batch * (group > 8 ? s->n_q_heads / 8 : s->n_kv_heads) > 4096) return VSA_ERR_UNSUPPORTED_SHAPE;
     if (s->num_pool_pages * s->n_kv_heads >= (1LL << 27)) return VSA_ERR_UNSUPPORTED_SHAPE;
     g->batch = s->batch;
     g->n_q_heads = s->n_q_heads;
     g->n_kv_heads = s->n_kv_heads;
     g->group = group;
+    g->kv_div = 1;
+    g->kv_heads_stored = s->n_kv_heads;
     g->max_pages = s->max_pages_per_seq;
     g->pool_pages = s->num_pool_pages;
     g->token_stride = s->kv_token_stride ? s->kv_token_stride : s->head_dim;

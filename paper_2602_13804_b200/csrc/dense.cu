@@ -254,8 +254,9 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
             const bool page_ok = phys >= 0 && phys < geo.pool_pages;
             if (!page_ok) phys = 0;
             const int valid_rows = page_ok ? min(kPageSize, T - pl * kPageSize) : 0;
-            const uint16_t* kp = k_cache + phys * geo.page_stride + (long long)g * geo.head_stride + cp_chunk * 8;
-            const uint16_t* vp = v_cache + phys * geo.page_stride + (long long)g * geo.head_stride + cp_chunk * 8;
+            const long long head_off = (long long)(g / geo.kv_div) * geo.head_stride + cp_chunk * 8;
+            const uint16_t* kp = k_cache + phys * geo.page_stride + head_off;
+            const uint16_t* vp = v_cache + phys * geo.page_stride + head_off;
             const uint32_t dst = ring_addr + (uint32_t)((k % kStages) * kStageBytes);
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
@@ -452,17 +453,23 @@ size_t dense_smem_bytes(const Geometry& g)
 
 }  // namespace
 
-static size_t dense_counter_bytes(const Geometry& g)
+static size_t dense_counter_bytes(const Geometry& g_in)
 {
+    const Geometry g = with_virtual_kv_heads(g_in);
     return (((size_t)g.batch * g.n_kv_heads * sizeof(int32_t)) + 255) / 256 * 256;
 }
 
 int32_t* dense_tickets(void* ws_dense) { return (int32_t*)ws_dense; }
 
-int dense_ticket_count(const Geometry& g) { return g.batch * g.n_kv_heads; }
-
-size_t dense_workspace_bytes(const Geometry& g)
+int dense_ticket_count(const Geometry& g_in)
 {
+    const Geometry g = with_virtual_kv_heads(g_in);
+    return g.batch * g.n_kv_heads;
+}
+
+size_t dense_workspace_bytes(const Geometry& g_in)
+{
+    const Geometry g = with_virtual_kv_heads(g_in);
     return dense_counter_bytes(g) + (size_t)dense_max_items(g) * g.group * kPartialFloats * sizeof(float);
 }
 
@@ -482,11 +489,12 @@ static cudaError_t launch_dense_g(const Geometry& g, const uint16_t* q, const ui
                       dense_max_items(g));
 }
 
-cudaError_t launch_dense(const Geometry& g, const void* q, const void* k_cache, const void* v_cache,
+cudaError_t launch_dense(const Geometry& g_in, const void* q, const void* k_cache, const void* v_cache,
                          const int32_t* block_table, const int32_t* seq_lens, const int32_t* fallback_list,
                          const int32_t* fallback_count, float epsilon, float* out, vsa_diag_t* diag, void* ws,
                          cudaStream_t stream, bool tickets_cleared)
 {
+    const Geometry g = with_virtual_kv_heads(g_in);
     int32_t* counters = (int32_t*)ws;
     float* partials = (float*)((char*)ws + dense_counter_bytes(g));
     if (!tickets_cleared) {

@@ -130,7 +130,7 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
     // [n_blocks * 32] offset of the page's summary row in 16-byte units, -1 = no valid page
     int32_t* off_tab = (int32_t*)(my_smem + Cfg::RING_BYTES);
     const uint32_t ring = (uint32_t)__cvta_generic_to_shared(my_smem);
-    const int page_units = geo.n_kv_heads * (kRowBytes / 16);
+    const int page_units = geo.kv_heads_stored * (kRowBytes / 16);
     auto encode = [&](int p, int i) { return (i < n_pages && p >= 0 && p < geo.pool_pages) ? p * page_units : -1; };
 #pragma unroll
     for (int k = 0; k < kFirstBlocks; ++k)
@@ -140,7 +140,8 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
     for (int hh = 0; hh < G; ++hh) unpack8(qraw[hh], qf[hh]);
     __syncwarp();
 
-    const uint8_t* srow = reinterpret_cast<const uint8_t*>(summaries) + (long long)g * kRowBytes + c * 16;
+    const int g_stored = g / geo.kv_div;   // the KV head whose summaries this (possibly virtual) head reads
+    const uint8_t* srow = reinterpret_cast<const uint8_t*>(summaries) + (long long)g_stored * kRowBytes + c * 16;
     const uint32_t lane_off = (uint32_t)(gi * ROWS * kRowBytes + c * 16);
     int tab_row[ROWS];   // the table entry of this lane's r-th row of a round
 #pragma unroll
@@ -156,7 +157,8 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
     const uint32_t rad_ring_s = (uint32_t)__cvta_generic_to_shared(rad_ring);
     float* rad_out = nullptr;
     if constexpr (CERT)
-        rad_out = rad_logical + ((long long)b * geo.n_kv_heads + g) * geo.max_pages + first_page + gi * ROWS + own_r;
+        rad_out = rad_logical + ((long long)b * geo.kv_heads_stored + g / geo.kv_div) * geo.max_pages + first_page +
+                  gi * ROWS + own_r;
 
     // rows without a valid page read row 0 of the pool instead (their result is never stored)
     auto issue = [&](int R) {
@@ -170,7 +172,7 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
                 // off / 16 = page * n_kv_heads: the row of this page in radii[][n_kv_heads]
                 const int off = max(tab[gi * ROWS + own_r], 0);
                 cp_async_4(rad_ring_s + 4u * (uint32_t)((R & (STAGES - 1)) * ROUND_PAGES + gi * ROWS + own_r),
-                           radii + (off >> 4) + g);
+                           radii + (off >> 4) + g / geo.kv_div);
             }
         }
     };
@@ -300,10 +302,11 @@ size_t route_workspace_bytes(const Geometry& g)
     return (size_t)g.batch * g.n_q_heads * g.max_pages * sizeof(float);
 }
 
-cudaError_t launch_route_scan(const Geometry& g, const void* q, const void* summaries, const int32_t* block_table,
+cudaError_t launch_route_scan(const Geometry& g_in, const void* q, const void* summaries, const int32_t* block_table,
                               const int32_t* seq_lens, void* ws, int32_t* zero_word, int32_t* zero_words,
                               int zero_count, cudaStream_t stream, const float* radii, float* rad_logical)
 {
+    const Geometry g = with_virtual_kv_heads(g_in);
     float* scores = (float*)ws;
     const uint16_t* qq = (const uint16_t*)q;
     const uint16_t* ss = (const uint16_t*)summaries;

@@ -70,7 +70,26 @@ struct Geometry {
     int batch, n_q_heads, n_kv_heads, group, max_pages;
     long long pool_pages;
     long long page_stride, head_stride, token_stride;   // elements
+    // Groups of more than 8 query heads per KV head (multi-query attention) reach the page scan and the
+    // dense pass as "virtual" KV heads of 8 query heads each: there n_kv_heads and group describe the
+    // virtual heads, virtual head g reads the cache of KV head g / kv_div, and kv_heads_stored is the
+    // number of KV heads the pools and the summaries are laid out with.  Elsewhere kv_div = 1.
+    int kv_div = 1;
+    int kv_heads_stored = 0;
 };
+
+// the geometry the page scan and the dense pass work with (see kv_div above)
+inline Geometry with_virtual_kv_heads(const Geometry& g)
+{
+    Geometry v = g;
+    v.kv_heads_stored = g.n_kv_heads;
+    if (g.group > 8) {
+        v.kv_div = g.group / 8;
+        v.group = 8;
+        v.n_kv_heads = g.n_q_heads / 8;
+    }
+    return v;
+}
 
 // ---- page summaries -----------------------------------------------------------------------
 cudaError_t launch_build_summaries(const Geometry& g, const void* k_cache, const int32_t* block_table,

@@ -43,6 +43,16 @@ def test_other_needle_layouts(mode):
     compare(w, run_gpu(w))
 
 
+@pytest.mark.parametrize("hq,hkv", [(16, 1), (32, 1), (32, 2)])
+def test_multi_query_groups_of_16_and_32(hq, hkv):
+    """Multi-query shapes (16 or 32 query heads per KV head): scan and dense pass split the group into
+    sub-groups of 8 that read the same KV head; everything must still match the oracle, the dense pass
+    included (threshold +inf sends every unit there)."""
+    w = make_workload(spec(seq_lens=(900, 333), n_q_heads=hq, n_kv_heads=hkv, needles=3), seed=230 + hq + hkv)
+    compare(w, run_gpu(w))
+    compare(w, run_gpu(w, gap_threshold=math.inf), gap_threshold=math.inf)
+
+
 def test_several_tiles_and_ragged_tail():
     # 5 sequences with lengths around page and 32-page-block boundaries, several scan blocks
     lens = (16 * 32 * 3 + 5, 16 * 32, 16 * 33 + 15, 1, 16)
