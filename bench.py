@@ -574,6 +574,8 @@ def sweep(dev, steps_small=200):
     # the scan where its traffic dominates: batch 16, T = 128k, two layer caches
     spec16 = config_spec(2, batch=16, T=131072, layers=2, name="cfg2_b16_t131072_2layers")
     out["scan_large"] = measure_point(spec16, dev, 40)
+    # a multi-query shape: config 1 with ONE KV head for the 32 query heads
+    out["mqa"] = measure_point(replace(config_spec(1), n_kv_heads=1, layers=16, name="cfg1_mqa_32q_1kv"), dev, 100)
     # two-level routing at batch 16: growth of the step from 4k to 128k against the full scan's
     tl = [two_level_point(config_spec(2, batch=16, T=4096, layers=16, name="cfg2_b16_t4096"), dev, 32, 100),
           two_level_point(spec16, dev, 32, 40)]

@@ -237,6 +237,40 @@ def sparse(geo: Geometry, q, k_cache, v_cache, block_table, seq_lens, routed_pag
     return r
 
 
+def route_group(geo: Geometry, q, summaries, block_table, seq_lens, P: int) -> RouteResult:
+    """Group-shared page routing: pages int32 [B, Hkv, P], scores fp32 [B, Hkv, P] (summed over the group)."""
+    qb, sm = _u16(q), _u16(summaries)
+    bt, sl = _i32(block_table), _i32(seq_lens)
+    pages = np.empty((geo.batch, geo.n_kv_heads, P), dtype=np.int32)
+    scores = np.empty((geo.batch, geo.n_kv_heads, P), dtype=np.float32)
+    s = geo.c()
+    rc = lib().orc_route_group(C.byref(s), _p(qb), _p(sm), _p(bt), _p(sl), C.c_int(P), _p(pages), _p(scores))
+    assert rc == 0, rc
+    return RouteResult(pages, scores, None)
+
+
+def sparse_group(geo: Geometry, q, k_cache, v_cache, block_table, seq_lens, routed_pages, K_c: int,
+                 epsilon: float, gap_threshold: float) -> SparseResult:
+    """Group-shared candidates: routed_pages [B, Hkv, P]; per-unit outputs and diagnostics; cand_pos is
+    [B, Hkv, K_c] (one candidate set per KV head).  cand_weight / best_rejected are not filled."""
+    qb, k, v = _u16(q), _u16(k_cache), _u16(v_cache)
+    bt, sl, rp = _i32(block_table), _i32(seq_lens), _i32(routed_pages)
+    B, H, d = geo.batch, geo.n_q_heads, geo.head_dim
+    P = rp.shape[-1]
+    r = SparseResult(
+        out=np.zeros((B, H, d)), delta=np.zeros((B, H), np.float32), delta12=np.zeros((B, H), np.float32),
+        s_max=np.zeros((B, H), np.float32), lse=np.zeros((B, H)), leak_bound=np.zeros((B, H)),
+        n_candidates=np.zeros((B, H), np.int32), fallback=np.zeros((B, H), np.int32),
+        cand_pos=np.full((B, geo.n_kv_heads, K_c), -1, np.int32), cand_weight=None, best_rejected=None)
+    s = geo.c()
+    rc = lib().orc_sparse_group(C.byref(s), _p(qb), _p(k), _p(v), _p(bt), _p(sl), _p(rp), C.c_int(P), C.c_int(K_c),
+                                C.c_float(epsilon), C.c_float(gap_threshold), _p(r.out), _p(r.delta), _p(r.delta12),
+                                _p(r.s_max), _p(r.lse), _p(r.leak_bound), _p(r.n_candidates), _p(r.fallback),
+                                _p(r.cand_pos))
+    assert rc == 0, rc
+    return r
+
+
 def build_radii(geo: Geometry, k_cache, summaries, block_table, seq_lens, first_page=None, radii=None) -> np.ndarray:
     """fp32 [pool, Hkv]: the slack-inflated radius of every owned page around its stored summary."""
     k, sm = _u16(k_cache), _u16(summaries)

@@ -27,6 +27,11 @@
  *                        "coarse page summaries"; the two-level construction is not in the paper): one
  *                        representative summary per 16 pages, P_super super-pages kept, exact page scores
  *                        inside them.  Parity unpinned by the paper; pinned here by its special cases.
+ *   orc_route_group, orc_sparse_group
+ *                        the same steps with the query heads of a GQA group routing as one query
+ *                        (summed scores, one page set and one candidate set per KV head); the paper
+ *                        has a single query per step, so this is a reading.  Parity unpinned by the
+ *                        paper; pinned by its reduction to orc_route / orc_sparse for groups of one.
  *   orc_dense            the plain definition: softmax(<q,k_t>/epsilon) over every token.
  * (The theory objects on tiny dictionaries - Euclidean projection, exact gap, the full
  *  entropic minimiser of Eq. (5.1) - live in theory.py next to this file.)
@@ -384,6 +389,164 @@ int orc_sparse(const orc_shape *s, const uint16_t *q, const uint16_t *K, const u
         leak_bound[u] = lb < 1.0 ? lb : 1.0;
         fallback[u] = (d < gap_threshold && ns < T) ? 1 : 0;
         free(s64);
+        free(c);
+    }
+    return 0;
+}
+
+/* ---- group-shared routing (a variant of Sec. 7 steps 1-4 for grouped-query attention; the paper treats
+ * a single query, so how the G query heads that read one KV head route is a reading of this library) ---
+ * The G heads of a (sequence, KV head) route as ONE query: a page's score is the sum over the group's
+ * heads of their page scores, a token's selection score the sum of their token scores - sums of the
+ * per-head fixed-order fp32 scores, added in ascending head order in fp32.  One page set (first min(P,
+ * n_b) of score descending, page ascending) and one candidate set (first min(K_c, #valid) of score
+ * descending, position ascending) per (sequence, KV head).  Each head then takes the softmax at
+ * temperature epsilon of ITS OWN scores over the shared candidates, and its diagnostics are Def. 1 /
+ * Sec. 8 / Cor. 1 evaluated with its own scores against the shared set S:
+ *   s_max = max_{t in S} s_t,  delta = s_max - max_{t scored, not in S} s_t  (negative when a rejected
+ *   token out-scores every kept one for this head; +inf when nothing was rejected),
+ *   delta12 = best - second best inside S,  leak_bound = min(1, (T - |S|) exp(-delta / eps)),
+ *   fallback = delta < threshold and |S| < T.
+ * routed_pages / routed_scores are [B][Hkv][P]; cand_pos is [B][Hkv][K_c]; everything else per unit. */
+static float group_sum(const float *per_head, int G)
+{
+    float acc = per_head[0];
+    for (int h = 1; h < G; ++h) acc = acc + per_head[h];
+    return acc;
+}
+
+int orc_route_group(const orc_shape *s, const uint16_t *q, const uint16_t *summaries, const int32_t *bt,
+                    const int32_t *seq_lens, int P, int32_t *routed_pages, float *routed_scores)
+{
+    if (!shape_ok(s) || P < 1) return -1;
+    const int G = s->n_q_heads / s->n_kv_heads;
+    const int groups = s->batch * s->n_kv_heads;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int gr = 0; gr < groups; ++gr) {
+        int b = gr / s->n_kv_heads, g = gr % s->n_kv_heads;
+        int nb = n_pages_of(s, seq_lens[b]);
+        scored *c = (scored *)malloc(sizeof(scored) * (size_t)(nb > 0 ? nb : 1));
+        float *ph = (float *)malloc(sizeof(float) * (size_t)G);
+        for (int l = 0; l < nb; ++l) {
+            int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
+            for (int h = 0; h < G; ++h)
+                ph[h] = orc_canon_dot(q + ((int64_t)b * s->n_q_heads + g * G + h) * ORC_D,
+                                      summaries + (p * s->n_kv_heads + g) * ORC_D);
+            c[l].s = group_sum(ph, G);
+            c[l].idx = l;
+        }
+        qsort(c, (size_t)nb, sizeof(scored), cmp_scored);
+        int keep = nb < P ? nb : P;
+        for (int i = 0; i < P; ++i) {
+            routed_pages[(int64_t)gr * P + i] = i < keep ? c[i].idx : -1;
+            if (routed_scores) routed_scores[(int64_t)gr * P + i] = i < keep ? c[i].s : -INFINITY;
+        }
+        free(ph);
+        free(c);
+    }
+    return 0;
+}
+
+/* a scored token of a group: summed score, position, and where its per-head scores are kept */
+typedef struct {
+    float s;
+    int32_t idx;
+    int32_t k;
+} gscored;
+
+static int cmp_gscored(const void *a, const void *b)
+{
+    const gscored *x = (const gscored *)a, *y = (const gscored *)b;
+    if (x->s > y->s) return -1;
+    if (x->s < y->s) return 1;
+    return (x->idx > y->idx) - (x->idx < y->idx);
+}
+
+int orc_sparse_group(const orc_shape *s, const uint16_t *q, const uint16_t *K, const uint16_t *V, const int32_t *bt,
+                     const int32_t *seq_lens, const int32_t *routed_pages, int P, int K_c, float epsilon,
+                     float gap_threshold, double *out, float *delta, float *delta12, float *s_max, double *lse,
+                     double *leak_bound, int32_t *n_candidates, int32_t *fallback, int32_t *cand_pos)
+{
+    if (!shape_ok(s) || P < 1 || K_c < 1) return -1;
+    const int G = s->n_q_heads / s->n_kv_heads;
+    const int groups = s->batch * s->n_kv_heads;
+    const double eps = (double)epsilon;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int gr = 0; gr < groups; ++gr) {
+        int b = gr / s->n_kv_heads, g = gr % s->n_kv_heads;
+        int T = seq_lens[b];
+        size_t cap = (size_t)P * (size_t)s->page_size + 1;
+        gscored *c = (gscored *)malloc(sizeof(gscored) * cap);
+        float *sh = (float *)malloc(sizeof(float) * cap * (size_t)G); /* per-head scores, [k][h] */
+        int nv = 0;
+        for (int i = 0; i < P; ++i) {
+            int l = routed_pages[(int64_t)gr * P + i];
+            if (l < 0) continue;
+            int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
+            for (int t = 0; t < s->page_size; ++t) {
+                int pos = l * s->page_size + t;
+                if (pos >= T) break;
+                for (int h = 0; h < G; ++h)
+                    sh[(size_t)nv * G + h] = orc_canon_dot(q + ((int64_t)b * s->n_q_heads + g * G + h) * ORC_D,
+                                                           kv_row(s, K, p, g, t));
+                c[nv].s = group_sum(sh + (size_t)nv * G, G);
+                c[nv].idx = pos;
+                c[nv].k = nv;
+                ++nv;
+            }
+        }
+        qsort(c, (size_t)nv, sizeof(gscored), cmp_gscored);
+        int ns = nv < K_c ? nv : K_c; /* |S|, shared by the group */
+        for (int i = 0; i < K_c; ++i) cand_pos[(int64_t)gr * K_c + i] = i < ns ? c[i].idx : -1;
+        for (int h = 0; h < G; ++h) {
+            int64_t u = (int64_t)b * s->n_q_heads + g * G + h;
+            const uint16_t *qv = q + u * ORC_D;
+            /* this head's softmax over the shared candidates, fp64 */
+            double m = -INFINITY, Z = 0.0, acc[ORC_D];
+            double *s64 = (double *)malloc(sizeof(double) * (size_t)(ns > 0 ? ns : 1));
+            for (int i = 0; i < ns; ++i) {
+                int pos = c[i].idx, l = pos / s->page_size, t = pos % s->page_size;
+                int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
+                s64[i] = dot64(qv, kv_row(s, K, p, g, t));
+                if (s64[i] > m) m = s64[i];
+            }
+            for (int e = 0; e < ORC_D; ++e) acc[e] = 0.0;
+            for (int i = 0; i < ns; ++i) {
+                int pos = c[i].idx, l = pos / s->page_size, t = pos % s->page_size;
+                int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
+                const uint16_t *vr = kv_row(s, V, p, g, t);
+                double w = exp((s64[i] - m) / eps);
+                Z += w;
+                for (int e = 0; e < ORC_D; ++e) acc[e] += w * (double)orc_bf16_to_f32(vr[e]);
+            }
+            for (int e = 0; e < ORC_D; ++e) out[u * ORC_D + e] = ns > 0 ? acc[e] / Z : 0.0;
+            lse[u] = ns > 0 ? m / eps + log(Z) : -INFINITY;
+            free(s64);
+            /* this head's own fp32 scores: best and second best inside S, best outside */
+            float s1 = -INFINITY, s2 = -INFINITY, rej = -INFINITY;
+            for (int i = 0; i < nv; ++i) {
+                float v = sh[(size_t)c[i].k * G + h];
+                if (i < ns) {
+                    if (v > s1) {
+                        s2 = s1;
+                        s1 = v;
+                    } else if (v > s2) {
+                        s2 = v;
+                    }
+                } else if (v > rej) {
+                    rej = v;
+                }
+            }
+            float d = nv > ns ? s1 - rej : INFINITY;
+            s_max[u] = s1;
+            delta[u] = d;
+            delta12[u] = ns > 0 ? s1 - s2 : INFINITY;
+            n_candidates[u] = ns;
+            double lb = (double)(T - ns) * exp(-(double)d / eps);
+            leak_bound[u] = lb < 1.0 ? lb : 1.0;
+            fallback[u] = (d < gap_threshold && ns < T) ? 1 : 0;
+        }
+        free(sh);
         free(c);
     }
     return 0;
