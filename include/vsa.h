@@ -329,6 +329,31 @@ int vsa_decode_step_certified_expand(const vsa_shape_t* shape, const void* q, co
                                      void* stream);
 
 /*
+ * The step with GROUP-SHARED routing (a variant for grouped-query attention; the paper's step has one
+ * query, so how a group of query heads routes is this library's reading): the G = n_q_heads / n_kv_heads
+ * heads that read one KV head route as ONE query.  A page's routing score is the sum over the group's
+ * heads of their page scores, a token's selection score the sum of their token scores - the per-head
+ * fixed-order fp32 scores added in ascending head order - so there is one page set (top-P, score
+ * descending, page ascending) and one candidate set (top-K_c, score descending, position ascending) per
+ * (sequence, KV head): every K and V tile is read once per group and both selections run once per group.
+ * Each head then takes the softmax at temperature epsilon of ITS OWN scores over the shared candidates;
+ * its diag is Def. 1 / Sec. 8 / Cor. 1 with its own scores against the shared set S: s_max = its best
+ * score in S, delta = s_max minus its best score among the scored tokens outside S (negative when a
+ * rejected token out-scores every kept one for this head, +inf when nothing was rejected), delta12 = best
+ * minus second best inside S, leak_bound and fallback as in vsa_sparse_decode.  Flagged units take the
+ * dense pass as in vsa_decode_step.
+ *   routed_pages: device int32 [batch][n_kv_heads][P] (one list per group), best first, -1 padded.
+ *   everything else as for vsa_decode_step; ws: VSA_WS_STEP bytes.
+ *   Needs the native cache layout (kv_token_stride = head_dim, kv_head_stride = page_size * head_dim) and
+ *   n_q_heads / n_kv_heads in {1, 2, 4, 8}; otherwise VSA_ERR_UNSUPPORTED_SHAPE.
+ */
+int vsa_decode_step_group_shared(const vsa_shape_t* shape, const void* q, const void* summaries, const void* k_cache,
+                                 const void* v_cache, const int32_t* block_table, const int32_t* seq_lens, int32_t P,
+                                 int32_t K_c, float epsilon, float gap_threshold, float* out, vsa_diag_t* diag,
+                                 int32_t* routed_pages, int32_t* fallback_list, int32_t* fallback_count, void* ws,
+                                 size_t ws_bytes, void* stream);
+
+/*
  * Two-level page routing: an approximate pre-filter in front of Sec. 7 step 1 (the paper says only
  * "coarse page summaries"; the construction is this library's).  A super-page is VSA_SUPER_PAGES
  * consecutive LOGICAL pages of a sequence; its representative is the page summary with the largest

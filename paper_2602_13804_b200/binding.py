@@ -66,6 +66,8 @@ def lib() -> C.CDLL:
         _lib.vsa_workspace_bytes.argtypes = [shp, i32, i32, C.c_int]
         _lib.vsa_build_page_summaries.argtypes = [shp, vp, vp, vp, vp, vp, vp]
         _lib.vsa_route_pages.argtypes = [shp, vp, vp, vp, vp, i32, vp, vp, vp, sz, vp]
+        _lib.vsa_decode_step_group_shared.argtypes = [shp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, vp, vp, vp, vp,
+                                                      vp, vp, sz, vp]
         _lib.vsa_build_super_summaries.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp]
         _lib.vsa_route_pages_two_level.argtypes = [shp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, sz, vp]
         _lib.vsa_decode_step_two_level.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, f32, f32,
@@ -158,6 +160,17 @@ def vsa_route_pages(shape, q, summaries, block_table, seq_lens, P, routed_pages,
                                  _ptr(routed_pages), _ptr(routed_scores), _ptr(ws),
                                  0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
            "vsa_route_pages")
+
+
+def vsa_decode_step_group_shared(shape, q, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon,
+                                 gap_threshold, out, diag, routed_pages, fallback_list, fallback_count, ws,
+                                 stream=None) -> None:
+    _check(lib().vsa_decode_step_group_shared(C.byref(shape), _ptr(q), _ptr(summaries), _ptr(k_cache), _ptr(v_cache),
+                                              _ptr(block_table), _ptr(seq_lens), P, K_c, epsilon, gap_threshold,
+                                              _ptr(out), _ptr(diag), _ptr(routed_pages), _ptr(fallback_list),
+                                              _ptr(fallback_count), _ptr(ws),
+                                              0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
+           "vsa_decode_step_group_shared")
 
 
 def n_super_pages(shape: vsa_shape_t) -> int:

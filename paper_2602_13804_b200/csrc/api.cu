@@ -485,6 +485,53 @@ int vsa_decode_step(const vsa_shape_t* shape, const void* q, const void* summari
                             stream, nullptr);
 }
 
+int vsa_decode_step_group_shared(const vsa_shape_t* shape, const void* q, const void* summaries, const void* k_cache,
+                                 const void* v_cache, const int32_t* block_table, const int32_t* seq_lens, int32_t P,
+                                 int32_t K_c, float epsilon, float gap_threshold, float* out, vsa_diag_t* diag,
+                                 int32_t* routed_pages, int32_t* fallback_list, int32_t* fallback_count, void* ws,
+                                 size_t ws_bytes, void* stream)
+{
+    Geometry g;
+    int rc = make_geometry(shape, &g);
+    if (rc) return rc;
+    if ((rc = check_routing_sizes(g, P, K_c, true))) return rc;
+    if ((rc = check_epsilon(epsilon))) return rc;
+    if (isnan(gap_threshold)) return VSA_ERR_INVALID_ARGUMENT;
+    if (!q || !summaries || !k_cache || !v_cache || !block_table || !seq_lens || !out || !diag || !routed_pages ||
+        !fallback_list || !fallback_count || !ws)
+        return VSA_ERR_INVALID_ARGUMENT;
+    if (!aligned16(q) || !aligned16(summaries) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(ws))
+        return VSA_ERR_MISALIGNED;
+    if (!vsa::sparse_shared_supported(g, P)) return VSA_ERR_UNSUPPORTED_SHAPE;
+    if (ws_bytes < step_route_part(g) + vsa::dense_workspace_bytes(g)) return VSA_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = (cudaStream_t)stream;
+    void* ws_dense = (char*)ws + step_route_part(g);
+    cudaError_t e = vsa::launch_route_scan(g, q, summaries, block_table, seq_lens, ws, fallback_count,
+                                           vsa::dense_tickets(ws_dense), vsa::dense_ticket_count(g), st);
+    if (e != cudaSuccess) return VSA_ERR_CUDA;
+    vsa::GroupSharedArgs a;
+    a.g = g;
+    a.q = (const uint16_t*)q;
+    a.k = (const uint16_t*)k_cache;
+    a.v = (const uint16_t*)v_cache;
+    a.block_table = block_table;
+    a.seq_lens = seq_lens;
+    a.routed_pages = routed_pages;
+    a.page_scores = (const float*)ws;
+    a.P = P;
+    a.K_c = K_c;
+    a.epsilon = epsilon;
+    a.gap_threshold = gap_threshold;
+    a.out = out;
+    a.diag = diag;
+    a.fallback_list = fallback_list;
+    a.fallback_count = fallback_count;
+    a.stream = st;
+    if (vsa::launch_sparse_shared(a) != cudaSuccess) return VSA_ERR_CUDA;
+    return cuda_rc(vsa::launch_dense(g, q, k_cache, v_cache, block_table, seq_lens, fallback_list, fallback_count,
+                                     epsilon, out, diag, ws_dense, st, /*tickets_cleared=*/true));
+}
+
 int vsa_decode_step_entropic(const vsa_shape_t* shape, const void* q, const void* summaries, const void* k_cache,
                              const void* v_cache, const int32_t* block_table, const int32_t* seq_lens, int32_t P,
                              int32_t K_c, float epsilon, float gap_threshold, int32_t solver_iters, float* out,

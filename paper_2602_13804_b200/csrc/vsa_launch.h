@@ -142,6 +142,26 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
                           int solver_iters = 0, vsa_solve_t* solve = nullptr, const float* rad_logical = nullptr,
                           vsa_cert_t* cert = nullptr, int solver_kind = 1, const int32_t* unit_list = nullptr,
                           const int32_t* unit_count = nullptr, int routed_stride = 0);
+// ---- group-shared sparse pass (sparse_shared.cuh) -------------------------------------------------
+// One thread block per (sequence, KV head); the group's heads share one page set and one candidate set
+// selected on summed scores.  page_scores: the scan's per-head scores; routed_pages [batch][n_kv][P] out.
+struct GroupSharedArgs {
+    Geometry g;
+    const uint16_t *q, *k, *v;
+    const int32_t *block_table, *seq_lens;
+    int32_t* routed_pages;
+    const float* page_scores;
+    int P, K_c;
+    float epsilon, gap_threshold;
+    float* out;
+    vsa_diag_t* diag;
+    int32_t *fallback_list, *fallback_count;
+    cudaStream_t stream;
+};
+// native cache layout, groups of 1, 2, 4 or 8 heads, shared memory within the limit
+bool sparse_shared_supported(const Geometry& g, int P);
+cudaError_t launch_sparse_shared(const GroupSharedArgs& a);
+
 // false when the kernel variant a launch would take needs more dynamic shared memory than a thread block
 // can have (227 KB): wide block tables together with the iterative solve's key tile
 bool sparse_shared_memory_fits(const Geometry& g, int P, int K_c, bool fused, bool solve, bool cert);
