@@ -67,6 +67,9 @@ def parse_args(argv=None):
     ap.add_argument("--two-level", type=int, default=None, metavar="P_SUPER",
                     help="time vsa_decode_step_two_level: only the pages of the P_SUPER best super-pages (16 pages "
                          "each, scored through one representative summary) are scored per unit")
+    ap.add_argument("--group-shared", action="store_true",
+                    help="time vsa_decode_step_group_shared: the heads of a GQA group route as one query (one page "
+                         "set and one candidate set per KV head)")
     ap.add_argument("--solver", default="eg", choices=["eg", "fw"],
                     help="with --solver-iters: entropic mirror descent (eg) or Frank-Wolfe with exact line search (fw)")
     ap.add_argument("--solver-iters", type=int, default=None,
@@ -352,6 +355,7 @@ class Harness:
                 r = torch.zeros((shape.num_pool_pages, shape.n_kv_heads), dtype=torch.float32, device=dev)
                 B.vsa_build_page_radii(shape, w.k_cache, s_, w.block_table, w.seq_lens, None, r)
                 self.radii.append(r)
+        self.routed_group = torch.empty((shape.batch, shape.n_kv_heads, P), dtype=torch.int32, device=dev)
         self.supers = None
         if a is not None and getattr(a, "two_level", None):
             self.ws = B.alloc_workspace(shape, a.two_level, K_c, B.VSA_WS_STEP_TWO_LEVEL, dev)
@@ -374,6 +378,9 @@ class Harness:
         if a is not None and a.dense_baseline and not plain:
             B.vsa_dense_decode_fallback(shape, w.q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, None, None,
                                         eps, out, diag, self.ws_dense)
+        elif a is not None and getattr(a, "group_shared", False) and not plain:
+            B.vsa_decode_step_group_shared(shape, w.q, s, w.k_cache, w.v_cache, w.block_table, w.seq_lens, P, K_c, eps,
+                                           tau, out, diag, self.routed_group, flist, fcount, self.ws_plain)
         elif self.supers is not None and not plain:
             B.vsa_decode_step_two_level(shape, w.q, s, self.supers[k], w.k_cache, w.v_cache, w.block_table,
                                         w.seq_lens, a.two_level, P, K_c, eps, tau, out, diag, routed, flist, fcount,
@@ -576,6 +583,23 @@ def sweep(dev, steps_small=200):
     out["scan_large"] = measure_point(spec16, dev, 40)
     # a multi-query shape: config 1 with ONE KV head for the 32 query heads
     out["mqa"] = measure_point(replace(config_spec(1), n_kv_heads=1, layers=16, name="cfg1_mqa_32q_1kv"), dev, 100)
+    # group-shared routing (one selection per KV head) on config 1 and at batch 16
+    gs = []
+    for spec_g in (replace(config_spec(1), layers=16, name="cfg1_16layers"),
+                   config_spec(2, batch=16, T=32768, layers=8, name="cfg2_b16_t32768")):
+        a = parse_args(["--group-shared"])
+        hg = Harness(spec_g, dev, args=a)
+        res = {}
+        for name, plain in (("group_shared", False), ("per_head", True)):
+            st = hg.capture(True, plain=plain)
+            with hg.torch.cuda.stream(hg.stream):
+                for _ in range(3):
+                    st()
+            res[name] = hg.time_steps(st, 50) / 50 * 1e3 / hg.L
+        hg.release()
+        gs.append({"workload": spec_g.name, "us_per_layer_group_shared": res["group_shared"],
+                   "us_per_layer_per_head_routing": res["per_head"]})
+    out["group_shared"] = gs
     # two-level routing at batch 16: growth of the step from 4k to 128k against the full scan's
     tl = [two_level_point(config_spec(2, batch=16, T=4096, layers=16, name="cfg2_b16_t4096"), dev, 32, 100),
           two_level_point(spec16, dev, 32, 40)]
@@ -741,7 +765,7 @@ def run_ours(args):
 
         # ---- with --solver-iters / --certified: the closed-form step timed the same way ----
         closed_form_us_per_layer = None
-        if solve is not None or cert is not None or args.two_level:
+        if solve is not None or cert is not None or args.two_level or args.group_shared:
             step_c = h.capture(use_graph, plain=True)
             for _ in range(3):
                 step_c()
@@ -750,7 +774,8 @@ def run_ours(args):
 
         # ---- end to end: q from pinned host memory, out + diag back to the host, every layer ----
         e2e = None
-        if not args.dense_baseline and solve is None and cert is None and not args.two_level:
+        if not args.dense_baseline and solve is None and cert is None and not args.two_level and \
+                not args.group_shared:
             q_host = [w.q.cpu().pin_memory() for w in layers]
             q_dev = torch.empty_like(w0.q)
             out_host = torch.empty(out.shape, dtype=torch.float32).pin_memory()
@@ -843,7 +868,7 @@ def run_ours(args):
     else:
         kern = kernel_fracs(alg, per_kernel, step_us, peak)
         dom = max(("route_scan", "sparse_decode", "dense_fallback"), key=lambda k: per_kernel[k])
-        if solve is not None or cert is not None or args.two_level:
+        if solve is not None or cert is not None or args.two_level or args.group_shared:
             # the events bracket the plain step's kernels; the cost of the iterations (of the certificate)
             # is the difference of the two graph-replayed steps and is booked on the sparse kernel
             extra = step_us - closed_form_us_per_layer
@@ -871,7 +896,8 @@ def run_ours(args):
 
     sweep_obj = None
     default_run = (args.workload == "cfg1" and not args.dense_baseline and solve is None and cert is None
-                   and args.P is None and args.Kc is None and args.layers is None and not args.two_level)
+                   and args.P is None and args.Kc is None and args.layers is None and not args.two_level
+                   and not args.group_shared)
     if default_run and world == 1 and not args.no_sweep:
         h.release()
         del layers, summaries, w0, last, h
@@ -892,7 +918,9 @@ def run_ours(args):
                          f" MB touched per pass over them",
                    "launch": "cuda graph replay of the whole step" if use_graph else "plain stream launches",
                    "path": "dense split-K baseline" if args.dense_baseline else
-                           (f"two-level route ({args.two_level} super-pages per unit) -> sparse -> dense fallback"
+                           ("route -> group-shared sparse (one page set and one candidate set per KV head) -> "
+                            "dense fallback" if args.group_shared else
+                            f"two-level route ({args.two_level} super-pages per unit) -> sparse -> dense fallback"
                             if args.two_level else
                             (f"route -> sparse with routing certificate -> retries of the refused units with up to "
                              f"{args.expand} pages -> dense fallback") if cert is not None and args.expand else
