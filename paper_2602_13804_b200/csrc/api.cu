@@ -122,7 +122,7 @@ int cuda_rc(cudaError_t e) { return e == cudaSuccess ? VSA_OK : VSA_ERR_CUDA; }
 // two-level routing scratch: [ page scores | representative scores | identity table | lengths in
 // super-pages | kept super-pages per unit ], each part 256-byte aligned; the step adds the dense scratch
 struct TwoLevelWs {
-    size_t super_scores, bt_super, sl_super, super_routed, dense, total_route;
+    size_t super_scores, bt_super, sl_super, super_routed, budget, dense, total_route;
 };
 TwoLevelWs two_level_layout(const Geometry& g, int P_super)
 {
@@ -137,6 +137,8 @@ TwoLevelWs two_level_layout(const Geometry& g, int P_super)
     o += align_up((size_t)g.batch * sizeof(int32_t), 256);
     w.super_routed = o;
     o += align_up((size_t)g.batch * g.n_q_heads * (size_t)P_super * sizeof(int32_t), 256);
+    w.budget = o;   // scored pages per unit
+    o += align_up((size_t)g.batch * g.n_q_heads * sizeof(int32_t), 256);
     w.dense = o;
     w.total_route = o;
     return w;
@@ -161,7 +163,8 @@ int two_level_scores(const Geometry& g, const void* q, const void* summaries, co
     if (vsa::launch_route_select(gs, base + w.super_scores, sl_super, P_super, super_routed, nullptr, st) !=
         cudaSuccess)
         return VSA_ERR_CUDA;
-    return cuda_rc(vsa::launch_inner_scan(g, q, summaries, block_table, seq_lens, super_routed, P_super, (float*)ws, st));
+    return cuda_rc(vsa::launch_inner_scan(g, q, summaries, block_table, seq_lens, super_routed, P_super, (float*)ws,
+                                          (int32_t*)(base + w.budget), st));
 }
 
 }  // namespace
@@ -290,7 +293,8 @@ int vsa_route_pages_two_level(const vsa_shape_t* shape, const void* q, const voi
     if ((rc = two_level_scores(g, q, summaries, super_summaries, block_table, seq_lens, P_super, super_routed, ws,
                                nullptr, nullptr, 0, st)))
         return rc;
-    return cuda_rc(vsa::launch_route_select(g, ws, seq_lens, P, routed_pages, routed_scores, st));
+    return cuda_rc(vsa::launch_route_select(g, ws, seq_lens, P, routed_pages, routed_scores, st,
+                                            (const int32_t*)((char*)ws + two_level_layout(g, P_super).budget)));
 }
 
 int vsa_decode_step_two_level(const vsa_shape_t* shape, const void* q, const void* summaries,
@@ -322,7 +326,9 @@ int vsa_decode_step_two_level(const vsa_shape_t* shape, const void* q, const voi
                                fallback_count, vsa::dense_tickets(ws_dense), vsa::dense_ticket_count(g), st)))
         return rc;
     cudaError_t e = vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, routed_pages, (const float*)ws,
-                                       P, K_c, epsilon, gap_threshold, out, diag, fallback_list, fallback_count, st);
+                                       P, K_c, epsilon, gap_threshold, out, diag, fallback_list, fallback_count, st, 0,
+                                       nullptr, nullptr, nullptr, 1, nullptr, nullptr, 0,
+                                       (const int32_t*)((char*)ws + w.budget));
     if (e != cudaSuccess) return VSA_ERR_CUDA;
     return cuda_rc(vsa::launch_dense(g, q, k_cache, v_cache, block_table, seq_lens, fallback_list, fallback_count,
                                      epsilon, out, diag, ws_dense, st, /*tickets_cleared=*/true));

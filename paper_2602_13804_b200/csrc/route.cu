@@ -220,7 +220,8 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
 template <int KPT>
 __global__ void route_select_kernel(Geometry geo, const float* __restrict__ scores,
                                     const int32_t* __restrict__ seq_lens, int P,
-                                    int32_t* __restrict__ routed_pages, float* __restrict__ routed_scores)
+                                    int32_t* __restrict__ routed_pages, float* __restrict__ routed_scores,
+                                    const int32_t* __restrict__ page_budget)
 {
     extern __shared__ uint32_t smem[];
     pdl_wait();
@@ -231,11 +232,12 @@ __global__ void route_select_kernel(Geometry geo, const float* __restrict__ scor
     const int T = seq_lens[b];
     const bool ok = T > 0 && T <= geo.max_pages * kPageSize;
     const int n = ok ? (T + kPageSize - 1) / kPageSize : 0;
+    const int P_sel = page_budget ? min(P, __ldcg(page_budget + unit)) : P;   // scored pages only (two-level routing)
     int K;
     if constexpr (KPT > 0)
-        K = select_top_pages_reg<KPT>(scores + unit * geo.max_pages, n, P, s);
+        K = select_top_pages_reg<KPT>(scores + unit * geo.max_pages, n, P_sel, s);
     else
-        K = select_top_pages(scores + unit * geo.max_pages, n, P, s);
+        K = select_top_pages(scores + unit * geo.max_pages, n, P_sel, s);
     for (int t = threadIdx.x; t < P; t += blockDim.x) {
         routed_pages[unit * P + t] = t < K ? s.win_idx[t] : -1;
         if (routed_scores) routed_scores[unit * P + t] = t < K ? key_to_float(s.win_key[t]) : -INFINITY;
@@ -327,7 +329,8 @@ cudaError_t launch_route_scan(const Geometry& g_in, const void* q, const void* s
 }
 
 cudaError_t launch_route_select(const Geometry& g, const void* ws, const int32_t* seq_lens, int P,
-                                int32_t* routed_pages, float* routed_scores, cudaStream_t stream)
+                                int32_t* routed_pages, float* routed_scores, cudaStream_t stream,
+                                const int32_t* page_budget)
 {
     const size_t smem = select_smem_bytes(g, P);
     const dim3 grid((unsigned)g.n_q_heads, (unsigned)g.batch);
@@ -339,7 +342,7 @@ cudaError_t launch_route_select(const Geometry& g, const void* ws, const int32_t
             if (e != cudaSuccess) return e;                                                                      \
         }                                                                                                        \
         cudaError_t e2 = launch_pdl(route_select_kernel<KPT>, grid, dim3(THREADS), smem, stream, g,            \
-                                    (const float*)ws, seq_lens, P, routed_pages, routed_scores);               \
+                                    (const float*)ws, seq_lens, P, routed_pages, routed_scores, page_budget);  \
         if (e2 != cudaSuccess) return e2;                                                                       \
     }
     if (g.max_pages <= 2048) VSA_SELECT_LAUNCH(8, 256)

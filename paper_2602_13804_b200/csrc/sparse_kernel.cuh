@@ -119,7 +119,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                      int32_t* __restrict__ fallback_count, int solver_iters, vsa_solve_t* __restrict__ solve,
                      const float* __restrict__ rad_logical, vsa_cert_t* __restrict__ cert,
                      const int32_t* __restrict__ unit_list, const int32_t* __restrict__ unit_count,
-                     int routed_stride)
+                     int routed_stride, const int32_t* __restrict__ page_budget)
 {
     constexpr int WARPS = THREADS / 32, GROUPS = 2 * WARPS;
     static_assert(SOLVE == 0 || THREADS == 256, "the solve maps one candidate to each of 256 lanes");
@@ -191,6 +191,9 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         return;
     }
     const int nb = (T + kPageSize - 1) / kPageSize;
+    // page_budget (two-level routing): only that many of the unit's pages carry a score, the rest of the
+    // row is -inf and must not be routed
+    const int P_sel = (PAGE_KPT != 0 && page_budget) ? min(P, __ldcg(page_budget + unit)) : P;
 
     // ---- routed pages -> page_l[] sorted by logical page, so that array order = position order ----
     int np;
@@ -202,7 +205,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
 #pragma unroll
             for (int j = 0; j < PAGE_KPT; ++j) pkey[j] = tid + j * THREADS < nb ? float_to_key(praw[j]) : 0u;
             cp_async_wait_all();   // this thread's part of the block-table copy; the selection's barriers publish it
-            np = select_top_pages_keys<PAGE_KPT>(pkey, nb, P, ps);
+            np = select_top_pages_keys<PAGE_KPT>(pkey, nb, P_sel, ps);
             if constexpr (CERT) {
                 // |q| (rounded up a little), every lane of a half-warp computing the same value
                 float qe[8];
@@ -227,7 +230,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                 if (lane == 0) ps.ts.wred[warp] = ub_key;   // published by the barrier below, read right after it
             }
         } else {
-            np = select_top_pages(page_scores + unit * geo.max_pages, nb, P, ps);
+            np = select_top_pages(page_scores + unit * geo.max_pages, nb, P_sel, ps);
         }
         for (int t = P + tid; t < routed_stride; t += THREADS) routed_pages[unit * routed_stride + t] = -1;
         for (int t = tid; t < P; t += THREADS) {
@@ -794,6 +797,7 @@ struct SparseArgs {
     vsa_cert_t* cert;     // non-null: the certificate variant (fused register variants only)
     const int32_t *unit_list, *unit_count;   // non-null: only the listed units (blocks beyond the count exit)
     int routed_stride;                       // row stride of routed_pages (>= P)
+    const int32_t* page_budget;              // non-null (fused forms): scored pages per unit, see the kernel
     cudaStream_t stream;
 };
 
@@ -813,7 +817,8 @@ cudaError_t launch_variant(const SparseArgs& a)
     return launch_pdl(sparse_decode_kernel<THREADS, PAGE_KPT, TOK_KPT, SOLVE, CERT>, dim3(units), dim3(THREADS),
                       a.smem, a.stream, a.g, a.q, a.k, a.v, a.block_table, a.seq_lens, a.routed_pages, a.page_scores,
                       a.P, a.K_c, a.epsilon, a.gap_threshold, a.out, a.diag, a.fallback_list, a.fallback_count,
-                      a.solver_iters, a.solve, a.rad_logical, a.cert, a.unit_list, a.unit_count, a.routed_stride);
+                      a.solver_iters, a.solve, a.rad_logical, a.cert, a.unit_list, a.unit_count, a.routed_stride,
+                      a.page_budget);
 }
 
 // token-score registers per thread from P

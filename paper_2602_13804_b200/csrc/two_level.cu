@@ -92,7 +92,8 @@ __global__ void two_level_prep_kernel(Geometry geo, const int32_t* __restrict__ 
 __global__ void __launch_bounds__(256)
 inner_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* __restrict__ summaries,
                   const int32_t* __restrict__ block_table, const int32_t* __restrict__ seq_lens,
-                  const int32_t* __restrict__ super_routed, int P_super, float* __restrict__ scores)
+                  const int32_t* __restrict__ super_routed, int P_super, float* __restrict__ scores,
+                  int32_t* __restrict__ page_budget)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, c = lane & 15, gi = lane >> 4;
     const unsigned hmask = 0xffffu << (lane & 16);
@@ -104,6 +105,15 @@ inner_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
     pdl_launch_dependents();
     if (T <= 0 || T > geo.max_pages * kPageSize) return;
     const int nb = (T + kPageSize - 1) / kPageSize;
+    if (tid == 0) {
+        // pages inside the kept super-pages: no more than these may be routed (the others hold -inf)
+        int n = 0;
+        for (int j = 0; j < P_super; ++j) {
+            const int sp = super_routed[unit * P_super + j];
+            if (sp >= 0) n += min(kSuper, nb - sp * kSuper);
+        }
+        page_budget[unit] = n;
+    }
     float* row = scores + unit * geo.max_pages;
     for (int i = tid; i < nb; i += blockDim.x) row[i] = -INFINITY;
     __syncthreads();
@@ -174,11 +184,11 @@ cudaError_t launch_two_level_prep(const Geometry& g, const int32_t* seq_lens, in
 
 cudaError_t launch_inner_scan(const Geometry& g, const void* q, const void* summaries, const int32_t* block_table,
                               const int32_t* seq_lens, const int32_t* super_routed, int P_super, float* scores,
-                              cudaStream_t stream)
+                              int32_t* page_budget, cudaStream_t stream)
 {
     return launch_pdl(inner_scan_kernel, dim3((unsigned)(g.batch * g.n_q_heads)), dim3(256), 0, stream, g,
                       (const uint16_t*)q, (const uint16_t*)summaries, block_table, seq_lens, super_routed, P_super,
-                      scores);
+                      scores, page_budget);
 }
 
 }  // namespace vsa

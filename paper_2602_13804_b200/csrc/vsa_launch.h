@@ -112,8 +112,11 @@ cudaError_t launch_route_scan(const Geometry& g, const void* q, const void* summ
                               const int32_t* seq_lens, void* ws, int32_t* zero_word, int32_t* zero_words,
                               int zero_count, cudaStream_t stream, const float* radii = nullptr,
                               float* rad_logical = nullptr);
+// page_budget (device, per unit, or nullptr): at most that many pages of a unit are routed (two-level
+// routing: the pages that were scored; the rest of the unit's score row is -inf)
 cudaError_t launch_route_select(const Geometry& g, const void* ws, const int32_t* seq_lens, int P,
-                                int32_t* routed_pages, float* routed_scores, cudaStream_t stream);
+                                int32_t* routed_pages, float* routed_scores, cudaStream_t stream,
+                                const int32_t* page_budget = nullptr);
 
 // ---- two-level routing (two_level.cu) -----------------------------------------------------------
 int two_level_max_supers(const Geometry& g);
@@ -125,7 +128,7 @@ cudaError_t launch_two_level_prep(const Geometry& g, const int32_t* seq_lens, in
                                   cudaStream_t stream);
 cudaError_t launch_inner_scan(const Geometry& g, const void* q, const void* summaries, const int32_t* block_table,
                               const int32_t* seq_lens, const int32_t* super_routed, int P_super, float* scores,
-                              cudaStream_t stream);
+                              int32_t* page_budget, cudaStream_t stream);
 
 // ---- fused sparse pass ------------------------------------------------------------------------
 // page_scores == nullptr: routed_pages is read; otherwise the top-P selection runs inside the kernel on
@@ -141,7 +144,8 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
                           vsa_diag_t* diag, int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream,
                           int solver_iters = 0, vsa_solve_t* solve = nullptr, const float* rad_logical = nullptr,
                           vsa_cert_t* cert = nullptr, int solver_kind = 1, const int32_t* unit_list = nullptr,
-                          const int32_t* unit_count = nullptr, int routed_stride = 0);
+                          const int32_t* unit_count = nullptr, int routed_stride = 0,
+                          const int32_t* page_budget = nullptr);
 // ---- group-shared sparse pass (sparse_shared.cuh) -------------------------------------------------
 // One thread block per (sequence, KV head); the group's heads share one page set and one candidate set
 // selected on summed scores.  page_scores: the scan's per-head scores; routed_pages [batch][n_kv][P] out.

@@ -88,6 +88,17 @@ def test_small_ragged(P_super):
     _compare(w, _run(w, P_super, 6, 40), P_super, 6, 40)
 
 
+def test_fewer_scored_pages_than_P_routes_only_the_scored_ones():
+    """One kept super-page holds at most 16 pages: with P = 64 the routed list is those pages and -1
+    padding, never a page that was not scored."""
+    spec = WorkloadSpec(name="tl", config=9, batch=3, n_q_heads=4, n_kv_heads=4, P=64, K_c=1,
+                        seq_lens=(900, 16, 2000), needles=1)
+    w = make_workload(spec, seed=915)
+    g = _run(w, 1, 64, 1)
+    _compare(w, g, 1, 64, 1)
+    assert (g["routed"] >= 0).sum(axis=-1).max() <= 16
+
+
 def test_every_super_page_kept_equals_the_full_scan():
     spec = WorkloadSpec(name="tl", config=9, batch=2, n_q_heads=4, n_kv_heads=2, P=6, K_c=40,
                         seq_lens=(1500, 333), needles=3)
