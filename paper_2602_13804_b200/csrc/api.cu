@@ -119,52 +119,40 @@ size_t step_retry_bytes(const Geometry& g)
 
 int cuda_rc(cudaError_t e) { return e == cudaSuccess ? VSA_OK : VSA_ERR_CUDA; }
 
-// two-level routing scratch: [ page scores | representative scores | identity table | lengths in
-// super-pages | kept super-pages per unit ], each part 256-byte aligned; the step adds the dense scratch
+// two-level routing scratch: [ page scores | representative scores | scored pages per unit ], each part
+// 256-byte aligned; the step adds the dense scratch
 struct TwoLevelWs {
-    size_t super_scores, bt_super, sl_super, super_routed, budget, dense, total_route;
+    size_t super_scores, budget, dense, total_route;
 };
-TwoLevelWs two_level_layout(const Geometry& g, int P_super)
+TwoLevelWs two_level_layout(const Geometry& g)
 {
     const Geometry gs = vsa::two_level_super_geometry(g);
     TwoLevelWs w;
     size_t o = step_route_part(g);
     w.super_scores = o;
     o += align_up(vsa::route_workspace_bytes(gs), 256);
-    w.bt_super = o;
-    o += align_up((size_t)g.batch * gs.max_pages * sizeof(int32_t), 256);
-    w.sl_super = o;
-    o += align_up((size_t)g.batch * sizeof(int32_t), 256);
-    w.super_routed = o;
-    o += align_up((size_t)g.batch * g.n_q_heads * (size_t)P_super * sizeof(int32_t), 256);
-    w.budget = o;   // scored pages per unit
+    w.budget = o;
     o += align_up((size_t)g.batch * g.n_q_heads * sizeof(int32_t), 256);
     w.dense = o;
     w.total_route = o;
     return w;
 }
 
-// prep -> representative scan -> top-P_super super-pages -> exact scores inside them (into the page-score
-// scratch at the start of ws).  zero_word / tickets: cleared by the representative scan for the step.
+// representative scan -> per unit: top-P_super super-pages and the exact scores inside them (into the
+// page-score scratch at the start of ws).  zero_word / tickets: cleared by the representative scan.
 int two_level_scores(const Geometry& g, const void* q, const void* summaries, const void* super_summaries,
                      const int32_t* block_table, const int32_t* seq_lens, int P_super, int32_t* super_routed_out,
                      void* ws, int32_t* zero_word, int32_t* zero_words, int zero_count, cudaStream_t st)
 {
-    const TwoLevelWs w = two_level_layout(g, P_super);
+    const TwoLevelWs w = two_level_layout(g);
     const Geometry gs = vsa::two_level_super_geometry(g);
     char* base = (char*)ws;
-    int32_t* bt_super = (int32_t*)(base + w.bt_super);
-    int32_t* sl_super = (int32_t*)(base + w.sl_super);
-    int32_t* super_routed = super_routed_out ? super_routed_out : (int32_t*)(base + w.super_routed);
-    if (vsa::launch_two_level_prep(g, seq_lens, sl_super, bt_super, st) != cudaSuccess) return VSA_ERR_CUDA;
-    if (vsa::launch_route_scan(gs, q, super_summaries, bt_super, sl_super, base + w.super_scores, zero_word,
+    // (the block-table argument is not read in a geometry whose pages are super-pages)
+    if (vsa::launch_route_scan(gs, q, super_summaries, block_table, seq_lens, base + w.super_scores, zero_word,
                                zero_words, zero_count, st) != cudaSuccess)
         return VSA_ERR_CUDA;
-    if (vsa::launch_route_select(gs, base + w.super_scores, sl_super, P_super, super_routed, nullptr, st) !=
-        cudaSuccess)
-        return VSA_ERR_CUDA;
-    return cuda_rc(vsa::launch_inner_scan(g, q, summaries, block_table, seq_lens, super_routed, P_super, (float*)ws,
-                                          (int32_t*)(base + w.budget), st));
+    return cuda_rc(vsa::launch_inner_scan(g, q, summaries, block_table, seq_lens, (const float*)(base + w.super_scores),
+                                          P_super, super_routed_out, (float*)ws, (int32_t*)(base + w.budget), st));
 }
 
 }  // namespace
@@ -199,8 +187,8 @@ size_t vsa_workspace_bytes(const vsa_shape_t* shape, int32_t P, int32_t K_c, int
         case VSA_WS_STEP_CERTIFIED: return step_rad_offset(g) + step_rad_bytes(g);
         case VSA_WS_STEP_EXPAND: return step_retry_offset(g) + step_retry_bytes(g);
         // (for the two-level kinds the P argument is P_super, the number of super-pages kept per unit)
-        case VSA_WS_ROUTE_TWO_LEVEL: return P >= 1 ? two_level_layout(g, P).total_route : 0;
-        case VSA_WS_STEP_TWO_LEVEL: return P >= 1 ? two_level_layout(g, P).dense + vsa::dense_workspace_bytes(g) : 0;
+        case VSA_WS_ROUTE_TWO_LEVEL: return P >= 1 ? two_level_layout(g).total_route : 0;
+        case VSA_WS_STEP_TWO_LEVEL: return P >= 1 ? two_level_layout(g).dense + vsa::dense_workspace_bytes(g) : 0;
         default: return 0;
     }
 }
@@ -288,13 +276,13 @@ int vsa_route_pages_two_level(const vsa_shape_t* shape, const void* q, const voi
         return VSA_ERR_INVALID_ARGUMENT;
     if (!aligned16(q) || !aligned16(summaries) || !aligned16(super_summaries) || !aligned16(ws))
         return VSA_ERR_MISALIGNED;
-    if (ws_bytes < two_level_layout(g, P_super).total_route) return VSA_ERR_WORKSPACE_TOO_SMALL;
+    if (ws_bytes < two_level_layout(g).total_route) return VSA_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t st = (cudaStream_t)stream;
     if ((rc = two_level_scores(g, q, summaries, super_summaries, block_table, seq_lens, P_super, super_routed, ws,
                                nullptr, nullptr, 0, st)))
         return rc;
     return cuda_rc(vsa::launch_route_select(g, ws, seq_lens, P, routed_pages, routed_scores, st,
-                                            (const int32_t*)((char*)ws + two_level_layout(g, P_super).budget)));
+                                            (const int32_t*)((char*)ws + two_level_layout(g).budget)));
 }
 
 int vsa_decode_step_two_level(const vsa_shape_t* shape, const void* q, const void* summaries,
@@ -317,7 +305,7 @@ int vsa_decode_step_two_level(const vsa_shape_t* shape, const void* q, const voi
     if (!aligned16(q) || !aligned16(summaries) || !aligned16(super_summaries) || !aligned16(k_cache) ||
         !aligned16(v_cache) || !aligned16(ws))
         return VSA_ERR_MISALIGNED;
-    const TwoLevelWs w = two_level_layout(g, P_super);
+    const TwoLevelWs w = two_level_layout(g);
     if (ws_bytes < w.dense + vsa::dense_workspace_bytes(g)) return VSA_ERR_WORKSPACE_TOO_SMALL;
     if (!vsa::sparse_shared_memory_fits(g, P, K_c, true, false, false)) return VSA_ERR_UNSUPPORTED_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;

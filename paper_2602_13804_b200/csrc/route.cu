@@ -97,7 +97,7 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
 #pragma unroll
         for (int k = 0; k < kFirstBlocks; ++k) {
             const int i = k * kBlockPages + lane;
-            first_entries[k] = i < span ? ld_ca_s32(bt + i) : -1;
+            first_entries[k] = i >= span ? -1 : geo.super_pages ? b * geo.max_pages + first_page + i : ld_ca_s32(bt + i);
         }
     }
 
@@ -119,6 +119,11 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
     for (int hh = 0; hh < G; ++hh)
         qraw[hh] = ld_nc_16B(q + ((long long)b * geo.n_q_heads + g * G + (hh ^ kh)) * kHeadDim + c * 8);
 
+    if (geo.super_pages) {
+        // the length in super-pages, expressed as a token count so that the page arithmetic below applies
+        const int ns = ((T + kPageSize - 1) / kPageSize + geo.super_pages - 1) / geo.super_pages;
+        T = (T > 0 && ns <= geo.max_pages) ? ns * kPageSize : 0;
+    }
     if (T <= 0 || T > geo.max_pages * kPageSize) return;
     const int nb = (T + kPageSize - 1) / kPageSize;
     if (first_page >= nb) return;

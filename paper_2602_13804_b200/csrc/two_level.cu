@@ -11,12 +11,14 @@
 // order; what the pre-filter can lose is a page whose super-page was not kept.
 //
 //   super_summaries_kernel  cache maintenance: representative (and its logical page) per super-page
-//   two_level_prep_kernel   per step: lengths in super-pages, identity table for the representative scan
-//   inner_scan_kernel       per unit: -inf over the unit's score row, exact scores of the kept super-pages
+//   (the page-routing scan, run on the representatives with a geometry whose pages are super-pages)
+//   inner_scan_kernel       per unit: top-P_super super-pages, -inf over the unit's score row, exact scores
+//                           of the pages inside the kept super-pages
 #include <math.h>
 
 #include "vsa_device.cuh"
 #include "vsa_launch.h"
+#include "vsa_select.cuh"
 
 namespace vsa {
 
@@ -65,36 +67,18 @@ super_summaries_kernel(Geometry geo, const uint16_t* __restrict__ summaries, con
     if (super_rep && c == 0) super_rep[o] = best;
 }
 
-// sl_super[b] = 16 * (super-pages of sequence b), so that the page-routing kernels, which derive a page
-// count from a token count, see one "page" per super-page; an invalid length stays invalid.
-// bt_super[b][s] = b * max_supers + s: the representatives are stored in logical order per sequence.
-__global__ void two_level_prep_kernel(Geometry geo, const int32_t* __restrict__ seq_lens, int max_supers,
-                                      int32_t* __restrict__ sl_super, int32_t* __restrict__ bt_super)
-{
-    // No early trigger for the kernel that follows: it reads these arrays before its own wait (they are
-    // "scheduler state" to it), so it may only start once this kernel has completed.
-    pdl_wait();
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < geo.batch) {
-        const int T = seq_lens[i];
-        int v;
-        if (T <= 0) v = 0;
-        else if (T > geo.max_pages * kPageSize) v = max_supers * kPageSize + 1;
-        else v = (((T + kPageSize - 1) / kPageSize + kSuper - 1) / kSuper) * kPageSize;
-        sl_super[i] = v;
-    }
-    if (i < geo.batch * max_supers) bt_super[i] = i;
-}
-
-// One block per (sequence, query head): the unit's score row [0, n_b) is set to -inf, then every page
-// of the unit's kept super-pages gets its exact score (one super-page = 16 summary rows = one
-// 16-value reduction per half-warp, lane c ending with the score of page 16 s + c).
-__global__ void __launch_bounds__(256)
+// One block (256 or 512 threads) per (sequence, query head): exact top-P_super of the unit's representative scores (score
+// descending, super-page ascending); the unit's score row [0, n_b) is set to -inf; then every page of the
+// kept super-pages gets its exact score (one super-page = 16 summary rows = one 16-value reduction per
+// half-warp, lane c ending with the score of page 16 s + c).  page_budget[unit] = pages scored.
+__global__ void __launch_bounds__(512)
 inner_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* __restrict__ summaries,
                   const int32_t* __restrict__ block_table, const int32_t* __restrict__ seq_lens,
-                  const int32_t* __restrict__ super_routed, int P_super, float* __restrict__ scores,
+                  const float* __restrict__ super_scores, int max_supers, int P_super,
+                  int32_t* __restrict__ super_routed_out, float* __restrict__ scores,
                   int32_t* __restrict__ page_budget)
 {
+    extern __shared__ uint32_t inner_smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, c = lane & 15, gi = lane >> 4;
     const unsigned hmask = 0xffffu << (lane & 16);
     const long long unit = blockIdx.x;
@@ -103,15 +87,20 @@ inner_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
     const uint4 qraw = ld_nc_16B(q + unit * kHeadDim + c * 8);
     pdl_wait();
     pdl_launch_dependents();
-    if (T <= 0 || T > geo.max_pages * kPageSize) return;
-    const int nb = (T + kPageSize - 1) / kPageSize;
+    if (T <= 0 || T > geo.max_pages * kPageSize) {
+        if (super_routed_out)
+            for (int t = tid; t < P_super; t += blockDim.x) super_routed_out[unit * P_super + t] = -1;
+        return;
+    }
+    const int nb = (T + kPageSize - 1) / kPageSize, ns = (nb + kSuper - 1) / kSuper;
+    const PageSelectSmem ps = carve_page_select(inner_smem, max_supers, P_super);
+    const int K = select_top_pages_reg<8>(super_scores + unit * max_supers, ns, P_super, ps);   // ends with a barrier
+    if (super_routed_out)
+        for (int t = tid; t < P_super; t += blockDim.x) super_routed_out[unit * P_super + t] = t < K ? ps.win_idx[t] : -1;
     if (tid == 0) {
         // pages inside the kept super-pages: no more than these may be routed (the others hold -inf)
         int n = 0;
-        for (int j = 0; j < P_super; ++j) {
-            const int sp = super_routed[unit * P_super + j];
-            if (sp >= 0) n += min(kSuper, nb - sp * kSuper);
-        }
+        for (int j = 0; j < K; ++j) n += min(kSuper, nb - ps.win_idx[j] * kSuper);
         page_budget[unit] = n;
     }
     float* row = scores + unit * geo.max_pages;
@@ -120,9 +109,8 @@ inner_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
     float qf[8];
     unpack8(qraw, qf);
     const int32_t* bt = block_table + (long long)b * geo.max_pages;
-    for (int j = warp * 2 + gi; j < P_super; j += 16) {
-        const int sp = super_routed[unit * P_super + j];
-        if (sp < 0) continue;   // (the same for the sixteen lanes of the half-warp)
+    for (int j = warp * 2 + gi; j < K; j += (int)(blockDim.x >> 4)) {
+        const int sp = ps.win_idx[j];
         const int l = sp * kSuper + c;
         long long phys = -1;
         if (l < nb) {
@@ -158,6 +146,7 @@ Geometry two_level_super_geometry(const Geometry& g)
     Geometry s = g;
     s.max_pages = two_level_max_supers(g);
     s.pool_pages = (long long)g.batch * s.max_pages;
+    s.super_pages = kSuper;
     return s;
 }
 
@@ -173,22 +162,18 @@ cudaError_t launch_build_super_summaries(const Geometry& g, const void* summarie
     return cudaGetLastError();
 }
 
-cudaError_t launch_two_level_prep(const Geometry& g, const int32_t* seq_lens, int32_t* sl_super, int32_t* bt_super,
-                                  cudaStream_t stream)
-{
-    const int ms = two_level_max_supers(g);
-    const int n = g.batch * ms;
-    return launch_pdl(two_level_prep_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, stream, g, seq_lens, ms,
-                      sl_super, bt_super);
-}
-
 cudaError_t launch_inner_scan(const Geometry& g, const void* q, const void* summaries, const int32_t* block_table,
-                              const int32_t* seq_lens, const int32_t* super_routed, int P_super, float* scores,
-                              int32_t* page_budget, cudaStream_t stream)
+                              const int32_t* seq_lens, const float* super_scores, int P_super,
+                              int32_t* super_routed_out, float* scores, int32_t* page_budget, cudaStream_t stream)
 {
-    return launch_pdl(inner_scan_kernel, dim3((unsigned)(g.batch * g.n_q_heads)), dim3(256), 0, stream, g,
-                      (const uint16_t*)q, (const uint16_t*)summaries, block_table, seq_lens, super_routed, P_super,
-                      scores, page_budget);
+    const int ms = two_level_max_supers(g);   // <= 2048: the selection keeps 8 scores per thread in registers
+    const size_t smem = (size_t)select_pages_words(ms, P_super) * 4;
+    // 512 threads when that lets every kept super-page have a half-warp of its own (one round of loads)
+    const long long units = (long long)g.batch * g.n_q_heads;
+    const unsigned threads = (P_super > 16 && units <= 2LL * device_sm_count()) ? 512u : 256u;
+    return launch_pdl(inner_scan_kernel, dim3((unsigned)units), dim3(threads), smem, stream, g,
+                      (const uint16_t*)q, (const uint16_t*)summaries, block_table, seq_lens, super_scores, ms, P_super,
+                      super_routed_out, scores, page_budget);
 }
 
 }  // namespace vsa

@@ -76,6 +76,10 @@ struct Geometry {
     // number of KV heads the pools and the summaries are laid out with.  Elsewhere kv_div = 1.
     int kv_div = 1;
     int kv_heads_stored = 0;
+    // Non-zero (two-level routing, the scan over the super-pages' representatives): a "page" of this
+    // geometry is a super-page of that many pages - lengths are still token counts of the sequence, and
+    // logical super-page s of sequence b is stored at row b * max_pages + s (no block table).
+    int super_pages = 0;
 };
 
 // the geometry the page scan and the dense pass work with (see kv_div above)
@@ -124,11 +128,12 @@ Geometry two_level_super_geometry(const Geometry& g);
 cudaError_t launch_build_super_summaries(const Geometry& g, const void* summaries, const int32_t* block_table,
                                          const int32_t* seq_lens, const int32_t* first_super, void* super_summaries,
                                          int32_t* super_rep, cudaStream_t stream);
-cudaError_t launch_two_level_prep(const Geometry& g, const int32_t* seq_lens, int32_t* sl_super, int32_t* bt_super,
-                                  cudaStream_t stream);
+// selects the P_super best super-pages of every unit from super_scores (the representative scan's output)
+// and writes the exact scores of the pages inside them (everything else -inf) and the number of scored
+// pages per unit; super_routed_out (nullable) receives the kept super-pages
 cudaError_t launch_inner_scan(const Geometry& g, const void* q, const void* summaries, const int32_t* block_table,
-                              const int32_t* seq_lens, const int32_t* super_routed, int P_super, float* scores,
-                              int32_t* page_budget, cudaStream_t stream);
+                              const int32_t* seq_lens, const float* super_scores, int P_super,
+                              int32_t* super_routed_out, float* scores, int32_t* page_budget, cudaStream_t stream);
 
 // ---- fused sparse pass ------------------------------------------------------------------------
 // page_scores == nullptr: routed_pages is read; otherwise the top-P selection runs inside the kernel on
