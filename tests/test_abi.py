@@ -205,3 +205,47 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "libvsa.so"))
     with pytest.raises(RuntimeError, match="no fallback"):
         B.lib()
+
+
+def test_two_level_and_group_shared_argument_validation(lib):
+    s = B.make_shape(8, 32, 8, 2048, 65536)
+    sp = C.byref(s)
+    # two-level routing: representatives, routing call, step
+    assert lib.vsa_build_super_summaries(sp, None, FAKE, FAKE, None, FAKE, None, None) == -1
+    assert lib.vsa_build_super_summaries(sp, FAKE, FAKE, FAKE, None, ODD, None, None) == -4
+    route_ws = B.vsa_workspace_bytes(s, 32, 0, B.VSA_WS_ROUTE_TWO_LEVEL)
+    assert route_ws > B.vsa_workspace_bytes(s, 32, 0, B.VSA_WS_ROUTE)
+    assert B.vsa_workspace_bytes(s, 32, 256, B.VSA_WS_STEP_TWO_LEVEL) > route_ws
+    assert B.vsa_workspace_bytes(s, 0, 0, B.VSA_WS_ROUTE_TWO_LEVEL) == 0
+
+    def two(P_super=32, P=32, sup=FAKE, ws_bytes=1 << 40):
+        return lib.vsa_route_pages_two_level(sp, FAKE, FAKE, sup, FAKE, FAKE, P_super, P, FAKE, None, None, FAKE,
+                                             ws_bytes, None)
+    assert two(sup=None) == -1 and two(P_super=0) == -1 and two(P_super=129) == -2 and two(P=0) == -1
+    assert two(sup=ODD) == -4 and two(ws_bytes=route_ws - 1) == -3
+
+    def two_step(K_c=256, eps=11.3, ws_bytes=1 << 40, P_super=32):
+        return lib.vsa_decode_step_two_level(sp, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, P_super, 32, K_c, eps, 90.0,
+                                             FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, ws_bytes, None)
+    assert two_step(K_c=0) == -1 and two_step(K_c=513) == -2 and two_step(eps=0.0) == -1
+    assert two_step(ws_bytes=1024) == -3 and two_step(P_super=0) == -1
+
+    # group-shared step: shapes and layouts it refuses on the host
+    def shared(shape, K_c=256, ws_bytes=1 << 40, q=FAKE):
+        return lib.vsa_decode_step_group_shared(C.byref(shape), q, FAKE, FAKE, FAKE, FAKE, FAKE, 32, K_c, 11.3, 90.0,
+                                                FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, ws_bytes, None)
+    assert shared(s, K_c=0) == -1 and shared(s, q=None) == -1 and shared(s, q=ODD) == -4
+    assert shared(s, ws_bytes=1024) == -3
+    assert shared(B.make_shape(8, 32, 1, 2048, 65536)) == -2          # 32 query heads per KV head
+    strided = B.make_shape(8, 32, 8, 2048, 65536)
+    strided.kv_token_stride = 256                                      # rows not contiguous: no 4 KB tiles
+    strided.kv_head_stride = 16 * 256
+    strided.kv_page_stride = 8 * 16 * 256
+    assert shared(strided) == -2
+
+
+def test_multi_query_group_sizes_are_accepted(lib):
+    for hq, hkv in ((16, 1), (32, 1), (32, 2)):
+        s = B.make_shape(4, hq, hkv, 2048, 65536)
+        assert B.vsa_workspace_bytes(s, 32, 256, B.VSA_WS_STEP) > 0
+    assert B.vsa_workspace_bytes(B.make_shape(4, 48, 1, 2048, 65536), 32, 256, B.VSA_WS_STEP) == 0   # group of 48
