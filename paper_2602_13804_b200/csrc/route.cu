@@ -240,9 +240,9 @@ __global__ void route_select_kernel(Geometry geo, const float* __restrict__ scor
     const int P_sel = page_budget ? min(P, __ldcg(page_budget + unit)) : P;   // scored pages only (two-level routing)
     int K;
     if constexpr (KPT > 0)
-        K = select_top_pages_reg<KPT>(scores + unit * geo.max_pages, n, P_sel, s);
+        K = select_top_pages_reg<KPT>(scores + unit * geo.max_pages, n, P_sel, s, page_budget != nullptr);
     else
-        K = select_top_pages(scores + unit * geo.max_pages, n, P_sel, s);
+        K = select_top_pages(scores + unit * geo.max_pages, n, P_sel, s, page_budget != nullptr);
     for (int t = threadIdx.x; t < P; t += blockDim.x) {
         routed_pages[unit * P + t] = t < K ? s.win_idx[t] : -1;
         if (routed_scores) routed_scores[unit * P + t] = t < K ? key_to_float(s.win_key[t]) : -INFINITY;

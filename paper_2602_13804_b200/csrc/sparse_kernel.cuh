@@ -203,7 +203,8 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         if constexpr (PAGE_KPT > 0) {
             uint32_t pkey[PAGE_KPT];
 #pragma unroll
-            for (int j = 0; j < PAGE_KPT; ++j) pkey[j] = tid + j * THREADS < nb ? float_to_key(praw[j]) : 0u;
+            for (int j = 0; j < PAGE_KPT; ++j)
+                pkey[j] = (tid + j * THREADS < nb && !(page_budget && praw[j] == -INFINITY)) ? float_to_key(praw[j]) : 0u;
             cp_async_wait_all();   // this thread's part of the block-table copy; the selection's barriers publish it
             np = select_top_pages_keys<PAGE_KPT>(pkey, nb, P_sel, ps);
             if constexpr (CERT) {
@@ -230,7 +231,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                 if (lane == 0) ps.ts.wred[warp] = ub_key;   // published by the barrier below, read right after it
             }
         } else {
-            np = select_top_pages(page_scores + unit * geo.max_pages, nb, P_sel, ps);
+            np = select_top_pages(page_scores + unit * geo.max_pages, nb, P_sel, ps, page_budget != nullptr);
         }
         for (int t = P + tid; t < routed_stride; t += THREADS) routed_pages[unit * routed_stride + t] = -1;
         for (int t = tid; t < P; t += THREADS) {

@@ -97,12 +97,8 @@ inner_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
     const int K = select_top_pages_reg<8>(super_scores + unit * max_supers, ns, P_super, ps);   // ends with a barrier
     if (super_routed_out)
         for (int t = tid; t < P_super; t += blockDim.x) super_routed_out[unit * P_super + t] = t < K ? ps.win_idx[t] : -1;
-    if (tid == 0) {
-        // pages inside the kept super-pages: no more than these may be routed (the others hold -inf)
-        int n = 0;
-        for (int j = 0; j < K; ++j) n += min(kSuper, nb - ps.win_idx[j] * kSuper);
-        page_budget[unit] = n;
-    }
+    int* scored = (int*)ps.ts.misc;   // pages that get a score (selection scratch, free after its last barrier)
+    if (tid == 0) *scored = 0;
     float* row = scores + unit * geo.max_pages;
     for (int i = tid; i < nb; i += blockDim.x) row[i] = -INFINITY;
     __syncthreads();
@@ -133,7 +129,12 @@ inner_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
         }
         const float s = reduce_scatter16(vals, c, hmask);
         if (l < nb && phys >= 0) row[l] = s;
+        const int n_ok = __popc(__ballot_sync(hmask, l < nb && phys >= 0));
+        if (c == 0) atomicAdd(scored, n_ok);
     }
+    __syncthreads();
+    // no more than the scored pages may be routed (every other entry of the row holds -inf)
+    if (tid == 0) page_budget[unit] = *scored;
 }
 
 }  // namespace

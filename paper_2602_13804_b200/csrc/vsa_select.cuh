@@ -66,11 +66,15 @@ __device__ __forceinline__ void order_winners(int K, const PageSelectSmem& s)
 
 // Exact top-min(P, n) of sc[0..n) under (score descending, page ascending), keys staged in shared
 // memory (any n up to the carve size).  Returns K; winners in s.win_* / s.asc_idx.
-__device__ __forceinline__ int select_top_pages(const float* __restrict__ sc, int n, int P, const PageSelectSmem& s)
+// sparse_row: scores of -inf mark pages that were never scored (two-level routing); they are treated as
+// absent, and the caller guarantees P <= the number of scored pages.
+__device__ __forceinline__ int select_top_pages(const float* __restrict__ sc, int n, int P, const PageSelectSmem& s,
+                                                bool sparse_row = false)
 {
     const int K = min(P, n);
     for (int i = threadIdx.x; i < n; i += blockDim.x) {
-        s.keys[i] = float_to_key(__ldcg(sc + i));
+        const float v = __ldcg(sc + i);
+        s.keys[i] = (sparse_row && v == -INFINITY) ? 0u : float_to_key(v);
         s.take[i] = 0;
     }
     if (threadIdx.x == 0) s.ts.misc[8] = 0u;
@@ -126,9 +130,18 @@ __device__ __forceinline__ int select_top_pages_keys(const uint32_t (&key)[KPT],
         if (lane == 0) s.ts.wred[warp] = thr;
         if (tid == 0) s.ts.misc[4] = 0u;
         __syncthreads();
+        // (a warp with fewer than r present scores publishes 0 and does not count: with a sparse row of
+        // scores only the warps that vouch for r scores each may set the threshold)
         uint32_t theta = 0xffffffffu;
-        for (int w = 0; w < nw_full; ++w) theta = min(theta, s.ts.wred[w]);
-        if (r > 32) theta = 0u;   // too few scores to filter: every score is a candidate
+        int vouching = 0;
+        for (int w = 0; w < nw_full; ++w) {
+            const uint32_t tw = s.ts.wred[w];
+            if (tw != 0u) {
+                theta = min(theta, tw);
+                ++vouching;
+            }
+        }
+        if (r > 32 || vouching * r < K) theta = 0u;   // too few scores to filter: every score is a candidate
         {
             uint32_t keep = 0u;
 #pragma unroll
@@ -200,13 +213,14 @@ __device__ __forceinline__ int select_top_pages_keys(const uint32_t (&key)[KPT],
 // The register variant fed from the scores in global memory.
 template <int KPT>
 __device__ __forceinline__ int select_top_pages_reg(const float* __restrict__ sc, int n, int P,
-                                                    const PageSelectSmem& s)
+                                                    const PageSelectSmem& s, bool sparse_row = false)
 {
     uint32_t key[KPT];
 #pragma unroll
     for (int j = 0; j < KPT; ++j) {
         const int i = threadIdx.x + j * blockDim.x;
-        key[j] = i < n ? float_to_key(__ldcg(sc + i)) : 0u;
+        const float v = i < n ? __ldcg(sc + i) : 0.0f;
+        key[j] = (i < n && !(sparse_row && v == -INFINITY)) ? float_to_key(v) : 0u;
     }
     return select_top_pages_keys<KPT>(key, n, P, s);
 }
