@@ -56,6 +56,8 @@ def parse_args(argv=None):
                     help="time the (P, K_c) grid of the paper's Table 3 at batch 8, T = 65536 and print it")
     ap.add_argument("--leak-curve", action="store_true",
                     help="leakage against the gap statistic on config-0-shaped workloads (CPU oracle only)")
+    ap.add_argument("--needle-mode", default=None, choices=["group_sum", "per_qhead_round_robin", "unit_literal"],
+                    help="override how the planted keys are aligned with the queries (workloads/generator.py)")
     ap.add_argument("--P", type=int, default=None, help="override the workload's routed pages per unit")
     ap.add_argument("--Kc", type=int, default=None, help="override the workload's candidate count per unit")
     ap.add_argument("--certified", action="store_true",
@@ -600,6 +602,20 @@ def sweep(dev, steps_small=200):
         gs.append({"workload": spec_g.name, "us_per_layer_group_shared": res["group_shared"],
                    "us_per_layer_per_head_routing": res["per_head"]})
     out["group_shared"] = gs
+    # the expansion loop where it rescues units: config 1 routed with 8 pages although 32 pages hold a planted
+    # key - the certificate refuses every unit; doubling the page budget up to 32 certifies them all
+    ex = []
+    spec_e = replace(config_spec(1), layers=8, P=8, K_c=128, name="cfg1_8layers_P8_Kc128")
+    for flags in (["--certified"], ["--certified", "--expand", "32"]):
+        he = Harness(spec_e, dev, args=parse_args(flags))
+        st = he.capture(True)
+        with he.torch.cuda.stream(he.stream):
+            for _ in range(3):
+                st()
+        us = he.time_steps(st, 20) / 20 * 1e3 / he.L
+        ex.append({"flags": " ".join(flags), "us_per_layer": us, "fallback_fraction": len(he.fallback_units()) / he.units})
+        he.release()
+    out["expansion_rescue"] = {"workload": spec_e.name, "points": ex}
     # two-level routing at batch 16: growth of the step from 4k to 128k against the full scan's
     tl = [two_level_point(config_spec(2, batch=16, T=4096, layers=16, name="cfg2_b16_t4096"), dev, 32, 100),
           two_level_point(spec16, dev, 32, 40)]
@@ -696,6 +712,9 @@ def run_ours(args):
         P_new = args.P if args.P is not None else spec.P
         K_new = args.Kc if args.Kc is not None else spec.K_c
         spec = replace(spec, P=P_new, K_c=K_new, name=f"{spec.name}_P{P_new}_Kc{K_new}")
+    if args.needle_mode:
+        from dataclasses import replace
+        spec = replace(spec, needle_mode=args.needle_mode, name=f"{spec.name}_{args.needle_mode}")
     h = Harness(spec, dev, rank=rank, args=args)
     L, distinct, shape, units = h.L, h.distinct, h.shape, h.units
     P, K_c, eps, tau = h.P, h.K_c, h.eps, h.tau
@@ -897,7 +916,7 @@ def run_ours(args):
     sweep_obj = None
     default_run = (args.workload == "cfg1" and not args.dense_baseline and solve is None and cert is None
                    and args.P is None and args.Kc is None and args.layers is None and not args.two_level
-                   and not args.group_shared)
+                   and not args.group_shared and not args.needle_mode)
     if default_run and world == 1 and not args.no_sweep:
         h.release()
         del layers, summaries, w0, last, h
