@@ -585,6 +585,9 @@ def sweep(dev, steps_small=200):
     out["scan_large"] = measure_point(spec16, dev, 40)
     # a multi-query shape: config 1 with ONE KV head for the 32 query heads
     out["mqa"] = measure_point(replace(config_spec(1), n_kv_heads=1, layers=16, name="cfg1_mqa_32q_1kv"), dev, 100)
+    # 32-token pages: config 1 with half as many pages routed (the same 512 scored tokens per unit)
+    c1 = config_spec(1)
+    out["page32"] = measure_point(replace(c1, page_size=32, P=c1.P // 2, layers=16, name="cfg1_page32_halfP"), dev, 100)
     # group-shared routing (one selection per KV head) on config 1 and at batch 16
     gs = []
     for spec_g in (replace(config_spec(1), layers=16, name="cfg1_16layers"),
@@ -929,7 +932,7 @@ def run_ours(args):
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": spec.name, "batch": shape.batch, "n_q_heads": shape.n_q_heads,
-                   "n_kv_heads": shape.n_kv_heads, "head_dim": 128, "page_size": 16,
+                   "n_kv_heads": shape.n_kv_heads, "head_dim": 128, "page_size": spec.page_size,
                    "context": int(sl.max()), "P": P, "K_c": K_c, "epsilon": eps, "gap_threshold": tau,
                    "layers_per_step": L, "distinct_layer_caches": distinct,
                    "l2": f"inputs larger than L2: {distinct} distinct layer caches, "

@@ -29,10 +29,11 @@
  *     than its block-table row, a non-positive length) never trap: the unit's
  *     diag.status becomes non-zero and its output row is zero-filled.
  *   - Inputs are assumed finite (no NaN/Inf in q, K, V).
- *   - v1 shapes: head_dim = 128, page_size = 16, n_q_heads / n_kv_heads in {1, 2, 4, 8, 16, 32}
+ *   - v1 shapes: head_dim = 128, page_size = 16 or 32, n_q_heads / n_kv_heads in {1, 2, 4, 8, 16, 32}
  *     (multi-head, grouped-query and multi-query attention; groups of 16 and 32 query heads
  *     are processed as two and four sub-groups of 8 that read the same KV head),
- *     1 <= P <= 128, 1 <= K_c <= P * page_size, max_pages_per_seq <= 32768,
+ *     1 <= P <= 128 and P * page_size <= 2048 (the tokens scored per unit), 1 <= K_c <= P * page_size,
+ *     max_pages_per_seq <= 32768,
  *     batch * n_kv_heads <= 4096 (batch * n_q_heads / 8 <= 4096 for groups above 8),
  *     num_pool_pages * n_kv_heads < 2^27 (the summary pool is addressed in 16-byte units by a
  *     32-bit offset).
@@ -45,6 +46,10 @@
  *   seq_lens     int32 [batch]                      tokens in each sequence (T_b)
  *   out          fp32 [batch][n_q_heads][head_dim]
  * Query head h reads KV head h / (n_q_heads / n_kv_heads).  A unit id is b * n_q_heads + h.
+ * With 32-token pages the summary of a page is the mean of its (up to) 32 valid key rows and a routed
+ * page contributes 32 tokens; the token-level steps see the same tokens as with 16-token pages (their
+ * results do not depend on where page boundaries fall).  vsa_decode_step_group_shared takes 16-token
+ * pages only.
  *
  * Arithmetic contract
  *   Every score that feeds a selection (page scores, token scores) is an fp32 dot product in

@@ -51,7 +51,7 @@ int make_geometry(const vsa_shape_t* s, Geometry* g)
     if (s->n_q_heads % s->n_kv_heads != 0) return VSA_ERR_INVALID_ARGUMENT;
     if (s->kv_page_stride < 0 || s->kv_head_stride < 0 || s->kv_token_stride < 0) return VSA_ERR_INVALID_ARGUMENT;
     const int group = s->n_q_heads / s->n_kv_heads;
-    if (s->head_dim != vsa::kHeadDim || s->page_size != vsa::kPageSize) return VSA_ERR_UNSUPPORTED_SHAPE;
+    if (s->head_dim != vsa::kHeadDim || (s->page_size != 16 && s->page_size != 32)) return VSA_ERR_UNSUPPORTED_SHAPE;
     if (group != 1 && group != 2 && group != 4 && group != 8 && group != 16 && group != 32)
         return VSA_ERR_UNSUPPORTED_SHAPE;
     if (s->max_pages_per_seq > kMaxPagesPerSeq) return VSA_ERR_UNSUPPORTED_SHAPE;
@@ -67,6 +67,9 @@ int make_geometry(const vsa_shape_t* s, Geometry* g)
     g->kv_div = 1;
     g->kv_heads_stored = s->n_kv_heads;
     g->max_pages = s->max_pages_per_seq;
+    g->page_size = s->page_size;
+    g->tile_shift = s->page_size == 32 ? 1 : 0;
+    g->super_pages = 0;
     g->pool_pages = s->num_pool_pages;
     g->token_stride = s->kv_token_stride ? s->kv_token_stride : s->head_dim;
     g->head_stride = s->kv_head_stride ? s->kv_head_stride : (long long)s->page_size * g->token_stride;
@@ -82,9 +85,9 @@ int check_routing_sizes(const Geometry& g, int P, int K_c, bool need_kc)
     if (P > kMaxP) return VSA_ERR_UNSUPPORTED_SHAPE;
     if (need_kc) {
         if (K_c < 1) return VSA_ERR_INVALID_ARGUMENT;
-        if (K_c > P * vsa::kPageSize) return VSA_ERR_UNSUPPORTED_SHAPE;
+        if (K_c > P * g.page_size) return VSA_ERR_UNSUPPORTED_SHAPE;
+        if (P * g.page_size > kMaxP * 16) return VSA_ERR_UNSUPPORTED_SHAPE;   // candidate tokens before the top-K_c
     }
-    (void)g;
     return VSA_OK;
 }
 

@@ -26,7 +26,8 @@ namespace {
 constexpr int kDenseThreads = 256;
 constexpr int kDenseWarps = kDenseThreads / 32;
 constexpr int kStages = 3;                         // pages in flight per warp
-constexpr int kTileBytes = kPageSize * kRowBytes;  // 4 KB: K (or V) rows of one page and KV head
+constexpr int kTileRows = 16;                      // the pass walks tiles of 16 tokens: one per 16-token page, two per 32-token page
+constexpr int kTileBytes = kTileRows * kRowBytes;  // 4 KB: K (or V) rows of one tile and KV head
 constexpr int kStageBytes = 2 * kTileBytes;        // K tile + V tile
 constexpr int kRingBytes = kDenseWarps * kStages * kStageBytes;   // 192 KB per block
 constexpr int kPartialFloats = 2 + kHeadDim;       // per (item, head): max (log2 domain), sum, acc[128]
@@ -124,8 +125,8 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
     auto pages_of = [&](int grp) -> int {
         if (!sm.group_mask[grp]) return 0;
         const int T = seq_lens[grp / geo.n_kv_heads];
-        if (T <= 0 || T > geo.max_pages * kPageSize) return 0;
-        return (T + kPageSize - 1) / kPageSize;
+        if (!geo.length_ok(T)) return 0;
+        return (T + kTileRows - 1) / kTileRows;
     };
     {
         int pages = 0, groups = 0, longest = 0;
@@ -217,7 +218,7 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
         const uint32_t mask = sm.group_mask[grp];
         const int b = grp / geo.n_kv_heads, g = grp % geo.n_kv_heads;
         const int T = seq_lens[b];
-        const int nb = (T + kPageSize - 1) / kPageSize;
+        const int nb = (T + kTileRows - 1) / kTileRows;   // tiles of the sequence
         const int chunk = item - sm.item_base[grp];
         const int items_of_group = sm.item_base[grp + 1] - sm.item_base[grp];
         // the group's pages are split evenly over its items (whole multiples of the warp count)
@@ -250,11 +251,12 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
         const int my_count = my_first < end_page ? (end_page - my_first + kDenseWarps - 1) / kDenseWarps : 0;
         auto issue = [&](int k) {   // k-th page of this warp into stage k % kStages
             const int pl = my_first + k * kDenseWarps;
-            long long phys = bt[pl];
+            long long phys = bt[pl >> geo.tile_shift];
             const bool page_ok = phys >= 0 && phys < geo.pool_pages;
             if (!page_ok) phys = 0;
-            const int valid_rows = page_ok ? min(kPageSize, T - pl * kPageSize) : 0;
-            const long long head_off = (long long)(g / geo.kv_div) * geo.head_stride + cp_chunk * 8;
+            const int valid_rows = page_ok ? min(kTileRows, T - pl * kTileRows) : 0;
+            const long long head_off = (long long)(g / geo.kv_div) * geo.head_stride + cp_chunk * 8 +
+                                       (long long)((pl & ((1 << geo.tile_shift) - 1)) * kTileRows) * geo.token_stride;
             const uint16_t* kp = k_cache + phys * geo.page_stride + head_off;
             const uint16_t* vp = v_cache + phys * geo.page_stride + head_off;
             const uint32_t dst = ring_addr + (uint32_t)((k % kStages) * kStageBytes);
@@ -278,9 +280,9 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
             cp_async_wait<kStages - 1>();
             __syncwarp();
             const int pl = my_first + k * kDenseWarps;
-            const int valid = min(kPageSize, T - pl * kPageSize);   // > 0
+            const int valid = min(kTileRows, T - pl * kTileRows);   // > 0
             {
-                const long long phys = bt[pl];   // a page outside the pool: the group's listed heads fail
+                const long long phys = bt[pl >> geo.tile_shift];   // a page outside the pool: the group's listed heads fail
                 if (phys < 0 || phys >= geo.pool_pages) {
                     if (lane == 0) sm.misc[13] = 1;   // (cleared at the end of the previous item)
                     __syncwarp();

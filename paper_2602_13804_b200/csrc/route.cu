@@ -121,11 +121,11 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
 
     if (geo.super_pages) {
         // the length in super-pages, expressed as a token count so that the page arithmetic below applies
-        const int ns = ((T + kPageSize - 1) / kPageSize + geo.super_pages - 1) / geo.super_pages;
-        T = (T > 0 && ns <= geo.max_pages) ? ns * kPageSize : 0;
+        const int ns = (geo.pages_of(T) + geo.super_pages - 1) / geo.super_pages;
+        T = (T > 0 && ns <= geo.max_pages) ? ns * geo.page_size : 0;
     }
-    if (T <= 0 || T > geo.max_pages * kPageSize) return;
-    const int nb = (T + kPageSize - 1) / kPageSize;
+    if (!geo.length_ok(T)) return;
+    const int nb = geo.pages_of(T);
     if (first_page >= nb) return;
     const int n_pages = min(blocks_per_warp * kBlockPages, nb - first_page);
     const int n_blocks = (n_pages + kBlockPages - 1) / kBlockPages;
@@ -235,8 +235,8 @@ __global__ void route_select_kernel(Geometry geo, const float* __restrict__ scor
     const int h = blockIdx.x, b = blockIdx.y;
     const long long unit = (long long)b * geo.n_q_heads + h;
     const int T = seq_lens[b];
-    const bool ok = T > 0 && T <= geo.max_pages * kPageSize;
-    const int n = ok ? (T + kPageSize - 1) / kPageSize : 0;
+    const bool ok = geo.length_ok(T);
+    const int n = ok ? geo.pages_of(T) : 0;
     const int P_sel = page_budget ? min(P, __ldcg(page_budget + unit)) : P;   // scored pages only (two-level routing)
     int K;
     if constexpr (KPT > 0)

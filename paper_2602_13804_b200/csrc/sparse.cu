@@ -13,10 +13,11 @@ size_t sparse_smem_bytes(const Geometry& g, int P, int K_c, bool fused, int thre
 {
     // the register variants of the fused kernel (PAGE_KPT > 0) keep a copy of the block-table row
     const bool staged = fused && g.max_pages <= 32 * threads;
+    const int PT = P << g.tile_shift;   // routed tiles of 16 tokens
     if (solve)
-        return (size_t)solve_tile_offset_words(g.max_pages, P, K_c, fused, staged) * 4 +
+        return (size_t)solve_tile_offset_words(g.max_pages, P, PT, K_c, fused, staged) * 4 +
                (size_t)solve_tile_rows(K_c) * kRowBytes + 16;
-    size_t words = (size_t)bt_stage_offset_words(g.max_pages, P, K_c, fused);
+    size_t words = (size_t)bt_stage_offset_words(g.max_pages, P, PT, K_c, fused);
     if (staged) words += (size_t)g.max_pages;
     return words * 4 + 16;
 }
@@ -35,7 +36,7 @@ int sparse_block_threads(const Geometry& g, int P, bool solve, bool cert, bool l
     // sequences cannot all be long.
     const bool narrow = g.max_pages <= 32 * 128;
     const bool cannot_all_be_long = (long long)g.batch * g.max_pages > (long long)g.pool_pages;
-    if (!solve && !listed && units > 2 * sm_count() && P <= 64 && (narrow || (!cert && cannot_all_be_long)))
+    if (!solve && !listed && units > 2 * sm_count() && (P << g.tile_shift) <= 64 && (narrow || (!cert && cannot_all_be_long)))
         threads = 128;
     return threads;
 }

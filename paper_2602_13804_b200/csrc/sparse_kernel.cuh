@@ -22,19 +22,19 @@ namespace {
 
 constexpr int kMaxSparseWarps = 16;
 
-// token-phase shared memory, in 4-byte words, after the two page arrays
-__host__ __device__ constexpr int token_phase_words(int P, int K_c)
+// token-phase shared memory, in 4-byte words, after the two tile arrays (PT = routed tiles of 16 tokens)
+__host__ __device__ constexpr int token_phase_words(int PT, int K_c)
 {
-    return P * kPageSize /*keys*/ + (P * kPageSize + 3) / 4 /*take*/ + 2 * K_c + 2 /*voff*/ + K_c /*wgt*/ +
+    return PT * 16 /*keys*/ + (PT * 16 + 3) / 4 /*take*/ + 2 * K_c + 2 /*voff*/ + K_c /*wgt*/ +
            K_c /*score*/ + 256 + 16 + 72 + kTopkList + kMaxSparseWarps * kHeadDim + kMaxSparseWarps + 4;
 }
 
-// first word of the block-table copy: after the two page arrays and the larger of the two phases
-__host__ __device__ inline int bt_stage_offset_words(int max_pages, int P, int K_c, bool fused)
+// first word of the block-table copy: after the two tile arrays and the larger of the two phases
+__host__ __device__ inline int bt_stage_offset_words(int max_pages, int P, int PT, int K_c, bool fused)
 {
-    int words = token_phase_words(P, K_c);
+    int words = token_phase_words(PT, K_c);
     if (fused && select_pages_words(max_pages, P) > words) words = select_pages_words(max_pages, P);
-    return 2 * P + words;
+    return 2 * PT + words;
 }
 
 // rows of the candidate key tile of the iterative solve: K_c rounded up to whole half-warps of
@@ -43,15 +43,15 @@ __host__ __device__ constexpr int solve_tile_rows(int K_c) { return ((K_c + 15) 
 
 // first word of that tile ([rows][128] bf16, 16-byte aligned): after the block-table copy when there
 // is one
-__host__ __device__ inline int solve_tile_offset_words(int max_pages, int P, int K_c, bool fused, bool staged)
+__host__ __device__ inline int solve_tile_offset_words(int max_pages, int P, int PT, int K_c, bool fused, bool staged)
 {
-    const int w = bt_stage_offset_words(max_pages, P, K_c, fused) + (staged ? max_pages : 0);
+    const int w = bt_stage_offset_words(max_pages, P, PT, K_c, fused) + (staged ? max_pages : 0);
     return (w + 3) & ~3;
 }
 
 struct TokenSmem {
-    uint32_t* keys;   // [P * 16] token score keys, array index = 16 * slot + token (position order)
-    uint8_t* take;    // [P * 16] scratch of the selection's slow path
+    uint32_t* keys;   // [PT * 16] token score keys, array index = 16 * slot + token (position order)
+    uint8_t* take;    // [PT * 16] scratch of the selection's slow path
     long long* voff;  // [K_c] element offset of each candidate's value row, candidates in position order
     float* wgt;       // [K_c] unnormalised softmax weight of each candidate
     float* score;     // [K_c] score of each candidate (read by the iterative solve only)
@@ -60,10 +60,10 @@ struct TokenSmem {
     float* zred;      // [warps]
 };
 
-__device__ __forceinline__ TokenSmem carve_tokens(uint32_t* base, int P, int K_c)
+__device__ __forceinline__ TokenSmem carve_tokens(uint32_t* base, int PT, int K_c)
 {
     TokenSmem s;
-    const int N = P * kPageSize;
+    const int N = PT * 16;
     s.keys = base;
     s.take = (uint8_t*)(s.keys + N);
     uint32_t* after_take = s.keys + N + (N + 3) / 4;
@@ -126,10 +126,13 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     static_assert(!CERT || PAGE_KPT > 0, "the certificate needs every page score of the unit in registers");
     static_assert(TOK_KPT * WARPS <= 64 && 4 * WARPS <= 72, "wred capacity");
     extern __shared__ uint32_t smem_raw[];
-    int32_t* page_l = (int32_t*)smem_raw;   // [P] routed logical pages, ascending, invalid entries last
-    int32_t* page_phys = page_l + P;        // [P]
-    uint32_t* region = smem_raw + 2 * P;    // page-selection scratch first, token-phase arrays afterwards
-    const int N = P * kPageSize;
+    // The token phases work on tiles of 16 rows: a routed page is 1 << tile_shift of them (one at 16 tokens
+    // per page, two at 32).  Tile v of the sequence holds tokens 16 v .. 16 v + 15.
+    const int tsh = geo.tile_shift, PT = P << tsh;
+    int32_t* page_l = (int32_t*)smem_raw;   // [PT] tiles of the routed pages, ascending, invalid entries last
+    int32_t* page_phys = page_l + PT;       // [PT] pool page of each tile
+    uint32_t* region = smem_raw + 2 * PT;   // page-selection scratch first, token-phase arrays afterwards
+    const int N = PT * 16;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, c = lane & 15, gi = lane >> 4;
     // unit_list != nullptr: block i handles unit_list[i] for i < *unit_count (a retry pass over the units
     // an earlier pass of the same step listed); the list is that pass's product, so it is read after
@@ -152,7 +155,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     const int32_t* bt = block_table + (long long)b * geo.max_pages;
     const int T = ld_ca_s32(seq_lens + b);
     const uint4 qraw = ld_nc_16B(q + unit * kHeadDim + c * 8);
-    int32_t* bt_s = (int32_t*)(smem_raw + bt_stage_offset_words(geo.max_pages, P, K_c, PAGE_KPT > 0));
+    int32_t* bt_s = (int32_t*)(smem_raw + bt_stage_offset_words(geo.max_pages, P, PT, K_c, PAGE_KPT > 0));
     if constexpr (PAGE_KPT > 0) {
         const uint32_t dst = (uint32_t)__cvta_generic_to_shared(bt_s);
         for (int i = tid; i < geo.max_pages; i += THREADS) cp_async_4(dst + 4u * (uint32_t)i, bt + i);
@@ -162,7 +165,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     pdl_launch_dependents();
     // Only the scores of the sequence's own pages are fetched: the rest of the scratch row was not
     // written in this step (in a ragged batch it is most of the row, and it would come from DRAM).
-    const int nb_fetch = (T > 0 && T <= geo.max_pages * kPageSize) ? (T + kPageSize - 1) / kPageSize : 0;
+    const int nb_fetch = geo.length_ok(T) ? geo.pages_of(T) : 0;
     float praw[PAGE_KPT > 0 ? PAGE_KPT : 1];
     if constexpr (PAGE_KPT > 0) {
 #pragma unroll
@@ -181,7 +184,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                           : 0.0f;
         }
     }
-    if (T <= 0 || T > geo.max_pages * kPageSize) {
+    if (!geo.length_ok(T)) {
         cp_async_wait_all();
         write_failed_unit(out, diag, unit, VSA_UNIT_BAD_LENGTH);
         if (SOLVE && tid == 0) solve[unit] = vsa_solve_t{0.0f, 0.0f, 0.0f, 0.0f};
@@ -190,7 +193,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
             for (int t = tid; t < routed_stride; t += THREADS) routed_pages[unit * routed_stride + t] = -1;
         return;
     }
-    const int nb = (T + kPageSize - 1) / kPageSize;
+    const int nb = geo.pages_of(T);
     // page_budget (two-level routing): only that many of the unit's pages carry a score, the rest of the
     // row is -inf and must not be routed
     const int P_sel = (PAGE_KPT != 0 && page_budget) ? min(P, __ldcg(page_budget + unit)) : P;
@@ -245,8 +248,10 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                     bad = 1;
                 }
             }
-            page_l[t] = l;
-            page_phys[t] = phys;
+            for (int hf = 0; hf < (1 << tsh); ++hf) {
+                page_l[(t << tsh) + hf] = l == INT_MAX ? INT_MAX : (l << tsh) + hf;
+                page_phys[(t << tsh) + hf] = phys;
+            }
         }
     } else {
         int32_t* raw = (int32_t*)region;   // staging; dead before the token phase reuses the region
@@ -268,8 +273,10 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                     bad = 1;
                 }
             }
-            page_l[rank] = l;
-            page_phys[rank] = phys;
+            for (int hf = 0; hf < (1 << tsh); ++hf) {
+                page_l[(rank << tsh) + hf] = l == INT_MAX ? INT_MAX : (l << tsh) + hf;
+                page_phys[(rank << tsh) + hf] = phys;
+            }
         }
         // (P <= 128 < THREADS: thread t < P owns slot t in the count)
         np = __syncthreads_count(tid < P && raw[tid < P ? tid : 0] != INT_MAX);
@@ -288,7 +295,8 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         if (CERT && tid == 0) cert[unit] = vsa_cert_t{0.0f, 0.0f, 0.0f, 0};
         return;
     }
-    const TokenSmem sm = carve_tokens(region, P, K_c);
+    const TokenSmem sm = carve_tokens(region, PT, K_c);
+    const int nt = np << tsh;   // tiles of the routed pages
 #pragma unroll
     for (int j = 0; j < TOK_KPT; ++j)
         if (tid + j * THREADS < N) sm.keys[tid + j * THREADS] = 0u;
@@ -297,28 +305,29 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     // ---- token routing: score all 16 tokens of a page per half-warp ----
     float qf[8];
     unpack8(qraw, qf);
-    for (int pp = warp; pp * 2 < np; pp += WARPS) {
+    for (int pp = warp; pp * 2 < nt; pp += WARPS) {
         const int slot = pp * 2 + gi;
-        const bool active = slot < np;
-        uint4 rows[kPageSize];
+        const bool active = slot < nt;
+        uint4 rows[16];
         if (active) {
             const uint16_t* src = k_cache + (long long)page_phys[slot] * geo.page_stride +
-                                  (long long)g * geo.head_stride + c * 8;
+                                  (long long)g * geo.head_stride + c * 8 +
+                                  (long long)((page_l[slot] & ((1 << tsh) - 1)) * 16) * geo.token_stride;
 #pragma unroll
-            for (int t = 0; t < kPageSize; ++t) rows[t] = ld_nc_16B(src + (long long)t * geo.token_stride);
+            for (int t = 0; t < 16; ++t) rows[t] = ld_nc_16B(src + (long long)t * geo.token_stride);
         } else {
 #pragma unroll
-            for (int t = 0; t < kPageSize; ++t) rows[t] = make_uint4(0u, 0u, 0u, 0u);
+            for (int t = 0; t < 16; ++t) rows[t] = make_uint4(0u, 0u, 0u, 0u);
         }
         float vals[16];
 #pragma unroll
-        for (int t = 0; t < kPageSize; ++t) {
+        for (int t = 0; t < 16; ++t) {
             float kf[8];
             unpack8(rows[t], kf);
             vals[t] = chunk_partial(qf, kf);
         }
         const float s = reduce_scatter16(vals, c);   // lane c: score of token c of the page
-        if (active && page_l[slot] * kPageSize + c < T) sm.keys[slot * kPageSize + c] = float_to_key(s);
+        if (active && page_l[slot] * 16 + c < T) sm.keys[slot * 16 + c] = float_to_key(s);
     }
     __syncthreads();
 
@@ -425,7 +434,8 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
             }
             if ((mask >> j) & 1u) {
                 const int i = tid + j * THREADS, pos = mine + before[j];
-                sm.voff[pos] = (long long)page_phys[i >> 4] * geo.page_stride + (long long)(i & 15) * geo.token_stride;
+                sm.voff[pos] = (long long)page_phys[i >> 4] * geo.page_stride +
+                               (long long)((page_l[i >> 4] & ((1 << tsh) - 1)) * 16 + (i & 15)) * geo.token_stride;
                 sm.wgt[pos] = exp2f((key_to_float(key[j]) - s1) * scale);
                 if constexpr (SOLVE != 0) sm.score[pos] = key_to_float(key[j]);
             }
@@ -442,7 +452,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
             // candidates in shared memory, lane c reading column c of each.
             const int hw = warp * 2 + gi, j_own = hw * 16 + c;
             const bool have = j_own < ns;
-            uint8_t* ktile = (uint8_t*)(smem_raw + solve_tile_offset_words(geo.max_pages, P, K_c, PAGE_KPT != 0,
+            uint8_t* ktile = (uint8_t*)(smem_raw + solve_tile_offset_words(geo.max_pages, P, PT, K_c, PAGE_KPT != 0,
                                                                            PAGE_KPT > 0));
             // a half-warp without candidates works on the block of sixteen zero rows behind the tile
             const int my_first = hw * 16 < ns ? hw * 16 : solve_tile_rows(K_c) - 16;
@@ -822,11 +832,11 @@ cudaError_t launch_variant(const SparseArgs& a)
                       a.page_budget);
 }
 
-// token-score registers per thread from P
+// token-score registers per thread from the number of routed tokens
 template <int THREADS, int PAGE_KPT, int SOLVE, bool CERT>
 cudaError_t launch_tok(const SparseArgs& a)
 {
-    const int N = a.P * kPageSize;
+    const int N = a.P * a.g.page_size;
     if (N <= 2 * THREADS) return launch_variant<THREADS, PAGE_KPT, 2, SOLVE, CERT>(a);
     if (N <= 4 * THREADS) return launch_variant<THREADS, PAGE_KPT, 4, SOLVE, CERT>(a);
     if constexpr (THREADS <= 256)

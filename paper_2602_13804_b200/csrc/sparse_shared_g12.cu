@@ -9,6 +9,7 @@ cudaError_t launch_sparse_shared_g8(const GroupSharedArgs& a);
 
 bool sparse_shared_supported(const Geometry& g, int P)
 {
+    if (g.page_size != kPageSize) return false;   // 16-token pages only
     if (g.token_stride != kHeadDim || g.head_stride != (long long)kPageSize * kHeadDim) return false;
     if (g.group != 1 && g.group != 2 && g.group != 4 && g.group != 8) return false;
     return (size_t)shared_layout(g.group, P).total * 4 <= (size_t)227 * 1024;

@@ -41,8 +41,8 @@ super_summaries_kernel(Geometry geo, const uint16_t* __restrict__ summaries, con
     const long long sp = hw / geo.n_kv_heads;
     if (sp >= max_supers) return;
     const int T = seq_lens[b];
-    const bool okT = T > 0 && T <= geo.max_pages * kPageSize;
-    const int nb = okT ? (T + kPageSize - 1) / kPageSize : 0;
+    const bool okT = geo.length_ok(T);
+    const int nb = okT ? geo.pages_of(T) : 0;
     if (first_super && sp < first_super[b]) return;
     const long long o = ((long long)b * max_supers + sp) * geo.n_kv_heads + g;
     int best = -1;
@@ -87,12 +87,12 @@ inner_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
     const uint4 qraw = ld_nc_16B(q + unit * kHeadDim + c * 8);
     pdl_wait();
     pdl_launch_dependents();
-    if (T <= 0 || T > geo.max_pages * kPageSize) {
+    if (!geo.length_ok(T)) {
         if (super_routed_out)
             for (int t = tid; t < P_super; t += blockDim.x) super_routed_out[unit * P_super + t] = -1;
         return;
     }
-    const int nb = (T + kPageSize - 1) / kPageSize, ns = (nb + kSuper - 1) / kSuper;
+    const int nb = geo.pages_of(T), ns = (nb + kSuper - 1) / kSuper;
     const PageSelectSmem ps = carve_page_select(inner_smem, max_supers, P_super);
     const int K = select_top_pages_reg<8>(super_scores + unit * max_supers, ns, P_super, ps);   // ends with a barrier
     if (super_routed_out)

@@ -80,6 +80,14 @@ struct Geometry {
     // geometry is a super-page of that many pages - lengths are still token counts of the sequence, and
     // logical super-page s of sequence b is stored at row b * max_pages + s (no block table).
     int super_pages = 0;
+    // Tokens per page, 16 or 32.  The token-level kernels work on tiles of 16 rows; a page holds
+    // 1 << tile_shift of them, and tile v of a sequence (tokens 16 v .. 16 v + 15) lies in logical page
+    // v >> tile_shift at row offset 16 * (v & ((1 << tile_shift) - 1)).
+    int page_size = 16;
+    int tile_shift = 0;
+    // pages a sequence of T tokens occupies / whether T is a length the block table can hold
+    __host__ __device__ int pages_of(int T) const { return (T + page_size - 1) >> (4 + tile_shift); }
+    __host__ __device__ bool length_ok(int T) const { return T > 0 && T <= max_pages * page_size; }
 };
 
 // the geometry the page scan and the dense pass work with (see kv_div above)

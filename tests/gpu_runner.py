@@ -119,7 +119,7 @@ def compare(w: Workload, g: GpuRun, P=None, K_c=None, epsilon=None, gap_threshol
     # S0: summaries, bit exact on every page a sequence owns
     o_sum = oracle.build_summaries(geo, K, bt, sl)
     g_sum = bits(g.summaries)
-    owned = np.concatenate([bt[b, : (int(sl[b]) + 15) // 16] for b in range(Bn) if sl[b] > 0])
+    owned = np.concatenate([bt[b, : -(-int(sl[b]) // geo.page_size)] for b in range(Bn) if sl[b] > 0])
     assert np.array_equal(g_sum[owned], o_sum[owned]), "page summaries differ"
 
     # S1: routed pages (ordered lists) and their scores, bit exact

@@ -77,7 +77,7 @@ def test_route_argument_validation(lib):
     assert _route(lib, ok, P=0) == -1
     assert _route(lib, ok, P=129) == -2
     assert _route(lib, B.make_shape(2, 8, 2, 64, 256, head_dim=64)) == -2
-    assert _route(lib, B.make_shape(2, 8, 2, 64, 256, page_size=32)) == -2
+    assert _route(lib, B.make_shape(2, 8, 2, 64, 256, page_size=64)) == -2
     assert _route(lib, B.make_shape(2, 6, 2, 64, 256)) == -2          # group of 3
     assert _route(lib, B.make_shape(2, 7, 2, 64, 256)) == -1          # heads do not divide
     assert _route(lib, B.make_shape(0, 8, 2, 64, 256)) == -1

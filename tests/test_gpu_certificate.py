@@ -55,7 +55,7 @@ def compare_certified(w, g):
     Bn, H = geo.batch, geo.n_q_heads
     summ = oracle.build_summaries(geo, K, bt, sl)
     rad = oracle.build_radii(geo, K, summ, bt, sl)
-    owned = np.concatenate([bt[b, : (int(sl[b]) + 15) // 16] for b in range(Bn)])
+    owned = np.concatenate([bt[b, : -(-int(sl[b]) // geo.page_size)] for b in range(Bn)])
     assert np.array_equal(g["radii"][owned].view(np.uint32), rad[owned].view(np.uint32)), "radii differ"
     untouched = np.ones(geo.num_pool_pages, bool)
     untouched[owned] = False
