@@ -620,10 +620,13 @@ def sweep(dev, steps_small=200):
         he.release()
     out["expansion_rescue"] = {"workload": spec_e.name, "points": ex}
     # two-level routing at batch 16: growth of the step from 4k to 128k against the full scan's
+    # (at 4k every super-page is kept, so the call runs the exact step) and at batch 1, T = 128k
     tl = [two_level_point(config_spec(2, batch=16, T=4096, layers=16, name="cfg2_b16_t4096"), dev, 32, 100),
           two_level_point(spec16, dev, 32, 40)]
     out["two_level_b16"] = {"points": tl, "growth_4k_to_128k": tl[1]["us_per_layer"] / tl[0]["us_per_layer"],
                             "growth_4k_to_128k_full_scan": tl[1]["us_per_layer_full_scan"] / tl[0]["us_per_layer_full_scan"]}
+    out["two_level_b1"] = [two_level_point(config_spec(2, batch=1, T=T, layers=16, name=f"cfg2_b1_t{T}"), dev, 32, 100)
+                           for T in (32768, 131072)]
     return out
 
 

@@ -310,16 +310,28 @@ int vsa_decode_step_two_level(const vsa_shape_t* shape, const void* q, const voi
         return VSA_ERR_MISALIGNED;
     const TwoLevelWs w = two_level_layout(g);
     if (ws_bytes < w.dense + vsa::dense_workspace_bytes(g)) return VSA_ERR_WORKSPACE_TOO_SMALL;
-    if (!vsa::sparse_shared_memory_fits(g, P, K_c, true, false, false)) return VSA_ERR_UNSUPPORTED_SHAPE;
+    if (!vsa::sparse_shared_memory_fits(g, P, K_c, true, false, false, P_super)) return VSA_ERR_UNSUPPORTED_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;
     void* ws_dense = (char*)ws + w.dense;
-    if ((rc = two_level_scores(g, q, summaries, super_summaries, block_table, seq_lens, P_super, nullptr, ws,
-                               fallback_count, vsa::dense_tickets(ws_dense), vsa::dense_ticket_count(g), st)))
-        return rc;
-    cudaError_t e = vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, routed_pages, (const float*)ws,
-                                       P, K_c, epsilon, gap_threshold, out, diag, fallback_list, fallback_count, st, 0,
-                                       nullptr, nullptr, nullptr, 1, nullptr, nullptr, 0,
-                                       (const int32_t*)((char*)ws + w.budget));
+    // Every super-page of every sequence would be kept: the routing is the exact one, which the full scan
+    // computes with less work per unit (same routed pages, same order)
+    if (vsa::two_level_max_supers(g) <= P_super) {
+        if (ws_bytes < step_route_part(g) + vsa::dense_workspace_bytes(g)) return VSA_ERR_WORKSPACE_TOO_SMALL;
+        return vsa_decode_step(shape, q, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon,
+                               gap_threshold, out, diag, routed_pages, fallback_list, fallback_count, ws, ws_bytes,
+                               stream);
+    }
+    // Three launches: the scan over the representatives (1/16 of the full scan's rows; it also clears the
+    // fallback counter and the dense tickets), the fused kernel whose front end keeps the P_super best
+    // super-pages of its unit, scores their pages exactly and routes the best P, and the dense pass.
+    const Geometry gs = vsa::two_level_super_geometry(g);
+    const float* super_scores = (const float*)((char*)ws + w.super_scores);
+    if (vsa::launch_route_scan(gs, q, super_summaries, block_table, seq_lens, (void*)super_scores, fallback_count,
+                               vsa::dense_tickets(ws_dense), vsa::dense_ticket_count(g), st) != cudaSuccess)
+        return VSA_ERR_CUDA;
+    cudaError_t e = vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, routed_pages, super_scores, P,
+                                       K_c, epsilon, gap_threshold, out, diag, fallback_list, fallback_count, st, 0,
+                                       nullptr, nullptr, nullptr, 1, nullptr, nullptr, 0, nullptr, summaries, P_super);
     if (e != cudaSuccess) return VSA_ERR_CUDA;
     return cuda_rc(vsa::launch_dense(g, q, k_cache, v_cache, block_table, seq_lens, fallback_list, fallback_count,
                                      epsilon, out, diag, ws_dense, st, /*tickets_cleared=*/true));

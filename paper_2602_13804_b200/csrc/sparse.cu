@@ -9,8 +9,10 @@ namespace vsa {
 
 namespace {
 
-size_t sparse_smem_bytes(const Geometry& g, int P, int K_c, bool fused, int threads, bool solve)
+size_t sparse_smem_bytes(const Geometry& g, int P, int K_c, bool fused, int threads, bool solve, int P_super = 0)
 {
+    if (P_super > 0)   // two-level front end
+        return (size_t)two_level_smem_words(g.max_pages, P, P << g.tile_shift, K_c, P_super) * 4 + 16;
     // the register variants of the fused kernel (PAGE_KPT > 0) keep a copy of the block-table row
     const bool staged = fused && g.max_pages <= 32 * threads;
     const int PT = P << g.tile_shift;   // routed tiles of 16 tokens
@@ -25,10 +27,17 @@ size_t sparse_smem_bytes(const Geometry& g, int P, int K_c, bool fused, int thre
 int sm_count() { return device_sm_count(); }
 
 // thread-block size of the per-unit kernel for a launch
-int sparse_block_threads(const Geometry& g, int P, bool solve, bool cert, bool listed)
+int sparse_block_threads(const Geometry& g, int P, bool solve, bool cert, bool listed, bool two_level = false,
+                         int P_super = 0)
 {
     const long long units = (long long)g.batch * g.n_q_heads;
     int threads = (!solve && units <= sm_count()) ? 512 : 256;
+    // two-level front end: every thread holds 8 representative scores and 8 of the 16 * P_super exact scores
+    if (two_level) {
+        const int max_supers = (g.max_pages + 15) / 16;
+        if (units > 2 * sm_count() && (P << g.tile_shift) <= 64 && max_supers <= 8 * 128 && P_super <= 64) threads = 128;
+        return threads;
+    }
     // Tables wider than 32 scores per thread: the 128-thread shape selects from shared memory, which loses
     // to the 256-thread register selection when every sequence is long (99 against 88 us per layer at
     // batch 16, T = 128k) and wins when most are short (410 against 445 us on the ragged config 4).  The
@@ -43,10 +52,10 @@ int sparse_block_threads(const Geometry& g, int P, bool solve, bool cert, bool l
 
 }  // namespace
 
-bool sparse_shared_memory_fits(const Geometry& g, int P, int K_c, bool fused, bool solve, bool cert)
+bool sparse_shared_memory_fits(const Geometry& g, int P, int K_c, bool fused, bool solve, bool cert, int P_super)
 {
-    const int threads = sparse_block_threads(g, P, solve, cert, false);
-    return sparse_smem_bytes(g, P, K_c, fused, threads, solve) <= (size_t)227 * 1024;
+    const int threads = sparse_block_threads(g, P, solve, cert, false, P_super > 0, P_super);
+    return sparse_smem_bytes(g, P, K_c, fused, threads, solve, P_super) <= (size_t)227 * 1024;
 }
 
 int sparse_register_select_max_pages(long long units) { return 32 * (units <= sm_count() ? 512 : 256); }
@@ -57,7 +66,7 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
                           vsa_diag_t* diag, int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream,
                           int solver_iters, vsa_solve_t* solve, const float* rad_logical, vsa_cert_t* cert,
                           int solver_kind, const int32_t* unit_list, const int32_t* unit_count, int routed_stride,
-                          const int32_t* page_budget)
+                          const int32_t* page_budget, const void* tl_summaries, int P_super)
 {
     SparseArgs a;
     a.g = g;
@@ -68,8 +77,12 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
     // the threads (measured 1.26x per unit): 512 units take one wave instead of two (25 against 30 us per
     // layer at batch 16, T = 4k), 2048 units 80 against 101 us (batch 64, T = 8k).  Closed-form variants
     // (with or without the certificate) only; fused ones with the page scores in registers (32 per thread at most).
-    const int threads = sparse_block_threads(g, P, solve != nullptr, cert != nullptr, unit_list != nullptr);
-    a.smem = sparse_smem_bytes(g, P, K_c, page_scores != nullptr, threads, solve != nullptr);
+    const int threads = sparse_block_threads(g, P, solve != nullptr, cert != nullptr, unit_list != nullptr,
+                                             tl_summaries != nullptr, P_super);
+    a.smem = sparse_smem_bytes(g, P, K_c, page_scores != nullptr, threads, solve != nullptr,
+                               tl_summaries ? P_super : 0);
+    a.tl_summaries = (const uint16_t*)tl_summaries;
+    a.P_super = P_super;
     a.solver_iters = solver_iters;
     a.solver_kind = solver_kind;
     a.solve = solve;
@@ -95,6 +108,7 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
     a.fallback_list = fallback_list;
     a.fallback_count = fallback_count;
     a.stream = stream;
+    if (tl_summaries) return (solve || cert || !page_scores) ? cudaErrorInvalidValue : launch_sparse_two_level(a, threads);
     if (solve) return launch_sparse_solve(a);
     if (cert) return page_scores ? launch_sparse_cert(a, threads) : cudaErrorInvalidValue;
     return launch_sparse_plain(a, threads);

@@ -37,6 +37,19 @@ __host__ __device__ inline int bt_stage_offset_words(int max_pages, int P, int P
     return 2 * PT + words;
 }
 
+// Two-level front end (PAGE_KPT == -2): [selection over the super-pages | exact keys of the pages inside the
+// kept super-pages, 16 per super-page | selection over those], all dead before the token phase
+__host__ __device__ inline int two_level_words(int max_pages, int P, int P_super)
+{
+    const int max_supers = (max_pages + 15) / 16;
+    return select_pages_words(max_supers, P_super) + 16 * P_super + select_pages_words(16 * P_super, P);
+}
+__host__ __device__ inline int two_level_smem_words(int max_pages, int P, int PT, int K_c, int P_super)
+{
+    const int a = token_phase_words(PT, K_c), b = two_level_words(max_pages, P, P_super);
+    return 2 * PT + (a > b ? a : b);
+}
+
 // rows of the candidate key tile of the iterative solve: K_c rounded up to whole half-warps of
 // sixteen, plus sixteen rows of zeros for the half-warps that own no candidate
 __host__ __device__ constexpr int solve_tile_rows(int K_c) { return ((K_c + 15) & ~15) + 16; }
@@ -99,6 +112,9 @@ __device__ __forceinline__ void write_failed_unit(float* out, vsa_diag_t* diag, 
 //   units in flight, fewer waves).
 // PAGE_KPT ==  0: routed_pages is an input.
 // PAGE_KPT == -1: fused with routing; page scores staged in shared memory (any block-table width).
+// PAGE_KPT == -2: fused with two-level routing; page_scores holds the unit's scores of the super-pages'
+//   representatives [unit][ceil(max_pages / 16)]; the P_super best super-pages are kept, the pages inside
+//   them scored exactly from tl_summaries, and the top-P of those routed.
 // PAGE_KPT  >  0: fused with routing; each thread keeps PAGE_KPT page scores in registers.
 //   In both fused forms the unit's top-P pages are selected here from page_scores[unit][0..n_b) and
 //   written to routed_pages (best first, -1 padded).
@@ -119,9 +135,11 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                      int32_t* __restrict__ fallback_count, int solver_iters, vsa_solve_t* __restrict__ solve,
                      const float* __restrict__ rad_logical, vsa_cert_t* __restrict__ cert,
                      const int32_t* __restrict__ unit_list, const int32_t* __restrict__ unit_count,
-                     int routed_stride, const int32_t* __restrict__ page_budget)
+                     int routed_stride, const int32_t* __restrict__ page_budget,
+                     const uint16_t* __restrict__ tl_summaries, int P_super)
 {
     constexpr int WARPS = THREADS / 32, GROUPS = 2 * WARPS;
+    static_assert(PAGE_KPT != -2 || (SOLVE == 0 && !CERT), "two-level front end: plain family only");
     static_assert(SOLVE == 0 || THREADS == 256, "the solve maps one candidate to each of 256 lanes");
     static_assert(!CERT || PAGE_KPT > 0, "the certificate needs every page score of the unit in registers");
     static_assert(TOK_KPT * WARPS <= 64 && 4 * WARPS <= 72, "wred capacity");
@@ -202,7 +220,10 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     int np;
     int bad = 0;
     if constexpr (PAGE_KPT != 0) {
-        const PageSelectSmem ps = carve_page_select(region, geo.max_pages, P);
+        const PageSelectSmem ps =
+            PAGE_KPT == -2 ? carve_page_select(region + select_pages_words((geo.max_pages + 15) >> 4, P_super) + 16 * P_super,
+                                               16 * P_super, P)
+                           : carve_page_select(region, geo.max_pages, P);
         if constexpr (PAGE_KPT > 0) {
             uint32_t pkey[PAGE_KPT];
 #pragma unroll
@@ -233,15 +254,75 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                 ub_key = __reduce_max_sync(kFullMask, ub_key);
                 if (lane == 0) ps.ts.wred[warp] = ub_key;   // published by the barrier below, read right after it
             }
-        } else {
+        } else if constexpr (PAGE_KPT == -1) {
             np = select_top_pages(page_scores + unit * geo.max_pages, nb, P_sel, ps, page_budget != nullptr);
         }
+        // position -> logical page of a winner (two-level: position 16 j + c is page c of the j-th kept
+        // super-page in ascending order)
+        const int32_t* asc_super = nullptr;
+        if constexpr (PAGE_KPT == -2) {
+            const int max_supers = (geo.max_pages + 15) >> 4, ns = (nb + 15) >> 4;
+            const PageSelectSmem ps1 = carve_page_select(region, max_supers, P_super);
+            uint32_t* exact = region + select_pages_words(max_supers, P_super);
+            uint32_t skey[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int i = tid + j * THREADS;
+                skey[j] = i < ns ? float_to_key(ld_cg_f32(page_scores + unit * max_supers + i)) : 0u;
+            }
+            if (tid == 0) ps1.ts.misc[12] = 0u;   // pages that get a score (a word the selection does not use)
+            const int Ks = select_top_pages_keys<8>(skey, ns, P_super, ps1);   // ends with a barrier
+            asc_super = ps1.asc_idx;
+            float qe[8];
+            unpack8(qraw, qe);
+            // one kept super-page = 16 summary rows = one 16-value reduction per half-warp; lane c ends with
+            // the exact score of page 16 s + c
+            for (int j0 = warp * 2; j0 < Ks; j0 += GROUPS) {
+                const int j = j0 + gi;
+                const bool have = j < Ks;
+                const int l = have ? asc_super[j] * 16 + c : nb;
+                long long phys = -1;
+                if (l < nb) {
+                    phys = bt[l];
+                    if (phys < 0 || phys >= geo.pool_pages) phys = -1;
+                }
+                uint4 srows[16];
+#pragma unroll
+                for (int r = 0; r < 16; ++r) {
+                    const long long pr = __shfl_sync(kFullMask, phys, (lane & 16) | r);
+                    srows[r] = pr >= 0 ? ld_nc_16B(tl_summaries + (pr * geo.n_kv_heads + g) * kHeadDim + c * 8)
+                                       : make_uint4(0u, 0u, 0u, 0u);
+                }
+                float vals[16];
+#pragma unroll
+                for (int r = 0; r < 16; ++r) {
+                    float kf[8];
+                    unpack8(srows[r], kf);
+                    vals[r] = chunk_partial(qe, kf);
+                }
+                const float sc = reduce_scatter16(vals, c);
+                const bool scored = have && phys >= 0;
+                if (have) exact[j * 16 + c] = scored ? float_to_key(sc) : 0u;
+                const int n_ok = __popc(__ballot_sync(kFullMask, scored));
+                if (lane == 0 && n_ok) atomicAdd(&ps1.ts.misc[12], (uint32_t)n_ok);
+            }
+            __syncthreads();
+            const int n2 = Ks * 16, P2 = min(P, (int)ps1.ts.misc[12]);
+            uint32_t pkey2[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int i = tid + j * THREADS;
+                pkey2[j] = i < n2 ? exact[i] : 0u;
+            }
+            np = P2 > 0 ? select_top_pages_keys<8>(pkey2, n2, P2, ps) : 0;
+        }
+        auto page_of = [&](int pos) { return PAGE_KPT == -2 ? asc_super[pos >> 4] * 16 + (pos & 15) : pos; };
         for (int t = P + tid; t < routed_stride; t += THREADS) routed_pages[unit * routed_stride + t] = -1;
         for (int t = tid; t < P; t += THREADS) {
-            routed_pages[unit * routed_stride + t] = t < np ? ps.win_idx[t] : -1;
+            routed_pages[unit * routed_stride + t] = t < np ? page_of(ps.win_idx[t]) : -1;
             int l = INT_MAX, phys = -1;
             if (t < np) {
-                l = ps.asc_idx[t];
+                l = page_of(ps.asc_idx[t]);
                 phys = PAGE_KPT > 0 ? bt_s[l] : bt[l];
                 if (phys < 0 || phys >= geo.pool_pages) {
                     phys = -1;
@@ -809,6 +890,8 @@ struct SparseArgs {
     const int32_t *unit_list, *unit_count;   // non-null: only the listed units (blocks beyond the count exit)
     int routed_stride;                       // row stride of routed_pages (>= P)
     const int32_t* page_budget;              // non-null (fused forms): scored pages per unit, see the kernel
+    const uint16_t* tl_summaries;            // non-null: two-level front end (page_scores = representative scores)
+    int P_super;
     cudaStream_t stream;
 };
 
@@ -829,7 +912,7 @@ cudaError_t launch_variant(const SparseArgs& a)
                       a.smem, a.stream, a.g, a.q, a.k, a.v, a.block_table, a.seq_lens, a.routed_pages, a.page_scores,
                       a.P, a.K_c, a.epsilon, a.gap_threshold, a.out, a.diag, a.fallback_list, a.fallback_count,
                       a.solver_iters, a.solve, a.rad_logical, a.cert, a.unit_list, a.unit_count, a.routed_stride,
-                      a.page_budget);
+                      a.page_budget, a.tl_summaries, a.P_super);
 }
 
 // token-score registers per thread from the number of routed tokens
@@ -878,5 +961,6 @@ inline cudaError_t launch_threads_128(const SparseArgs& a)
 cudaError_t launch_sparse_plain(const SparseArgs& a, int threads);   // closed-form weights
 cudaError_t launch_sparse_solve(const SparseArgs& a);                // iterative solves (256 threads)
 cudaError_t launch_sparse_cert(const SparseArgs& a, int threads);    // routing certificate
+cudaError_t launch_sparse_two_level(const SparseArgs& a, int threads);   // two-level front end
 
 }  // namespace vsa

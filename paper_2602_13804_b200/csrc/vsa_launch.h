@@ -158,7 +158,11 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
                           int solver_iters = 0, vsa_solve_t* solve = nullptr, const float* rad_logical = nullptr,
                           vsa_cert_t* cert = nullptr, int solver_kind = 1, const int32_t* unit_list = nullptr,
                           const int32_t* unit_count = nullptr, int routed_stride = 0,
-                          const int32_t* page_budget = nullptr);
+                          const int32_t* page_budget = nullptr, const void* tl_summaries = nullptr,
+                          int P_super = 0);
+// tl_summaries != nullptr: the two-level front end - page_scores then holds the scores of the super-pages'
+// representatives, fp32 [batch][n_q_heads][two_level_max_supers], and the kernel keeps the P_super best
+// super-pages, scores their pages from tl_summaries and routes the best P of those.
 // ---- group-shared sparse pass (sparse_shared.cuh) -------------------------------------------------
 // One thread block per (sequence, KV head); the group's heads share one page set and one candidate set
 // selected on summed scores.  page_scores: the scan's per-head scores; routed_pages [batch][n_kv][P] out.
@@ -181,7 +185,8 @@ cudaError_t launch_sparse_shared(const GroupSharedArgs& a);
 
 // false when the kernel variant a launch would take needs more dynamic shared memory than a thread block
 // can have (227 KB): wide block tables together with the iterative solve's key tile
-bool sparse_shared_memory_fits(const Geometry& g, int P, int K_c, bool fused, bool solve, bool cert);
+bool sparse_shared_memory_fits(const Geometry& g, int P, int K_c, bool fused, bool solve, bool cert,
+                               int P_super = 0);
 // widest block table for which the fused kernel keeps every page score of a unit in registers (the
 // certificate variant exists for those shapes only); `units` = batch * n_q_heads
 int sparse_register_select_max_pages(long long units);
