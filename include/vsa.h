@@ -380,7 +380,10 @@ int vsa_decode_step_group_shared(const vsa_shape_t* shape, const void* q, const 
  * vsa_route_pages_two_level: arguments as vsa_route_pages, plus super_summaries, P_super (1..128) and
  *   super_routed: device int32 [batch][n_q_heads][P_super] or NULL, the kept super-pages, -1 padded.
  *   ws: vsa_workspace_bytes(shape, P_super, 0, VSA_WS_ROUTE_TWO_LEVEL) bytes.
- * vsa_decode_step_two_level: vsa_decode_step with the two-level routing in place of the full scan;
+ * vsa_decode_step_two_level: vsa_decode_step with the two-level routing in place of the full scan (the
+ *   representatives are scanned by one kernel; keeping the super-pages, scoring their pages and routing
+ *   happen inside the fused kernel of the step); when ceil(max_pages_per_seq / 16) <= P_super every
+ *   super-page would be kept and the call runs vsa_decode_step itself (same results).
  *   ws: vsa_workspace_bytes(shape, P_super, K_c, VSA_WS_STEP_TWO_LEVEL) bytes.
  */
 int vsa_build_super_summaries(const vsa_shape_t* shape, const void* summaries, const int32_t* block_table,
