@@ -49,6 +49,7 @@ def lib():
     if _lib is None:
         _lib = C.CDLL(build())
         _lib.orc_canon_dot.restype = C.c_float
+        _lib.orc_canon_dot_d.restype = C.c_float
         _lib.orc_bf16_to_f32.restype = C.c_float
         _lib.orc_f32_to_bf16.restype = C.c_uint16
         _lib.orc_f32_to_bf16.argtypes = [C.c_float]
@@ -122,8 +123,8 @@ def f32_to_bf16(x) -> np.ndarray:
 
 def canon_dot(x_bits, y_bits) -> np.float32:
     x, y = _u16(x_bits), _u16(y_bits)
-    assert x.size == 128 and y.size == 128
-    return np.float32(lib().orc_canon_dot(_p(x), _p(y)))
+    assert x.size == y.size and x.size in (64, 128, 256)
+    return np.float32(lib().orc_canon_dot_d(_p(x), _p(y), C.c_int(int(x.size))))
 
 
 def build_summaries(geo: Geometry, k_cache, block_table, seq_lens, first_page=None,

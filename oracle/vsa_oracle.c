@@ -61,7 +61,7 @@ typedef struct {
     int64_t kv_page_stride, kv_head_stride, kv_token_stride; /* in elements */
 } orc_shape;
 
-enum { ORC_D = 128 };
+enum { ORC_DMAX = 256 }; /* head_dim is 64, 128 or 256 */
 
 int orc_num_threads(void)
 {
@@ -109,11 +109,23 @@ uint16_t orc_f32_to_bf16(float f)
  * Then a halving tree over the 16 partials: p[c] += p[c+off], off = 8, 4, 2, 1.
  * A product of two bf16 numbers is exact in fp32, so it does not matter whether a
  * machine fuses the multiply into the add.  (The paper fixes no order; this one is the
- * library's arithmetic contract.) */
-float orc_canon_dot(const uint16_t *x, const uint16_t *y)
+ * library's arithmetic contract.)  Other head dimensions keep the chunking: d = 256 has 32 partials and
+ * one more tree level (off = 16 first); d = 64 has 8 partials, padded with +0 to 16 for the same tree. */
+/* d = 64, 128 or 256: d / 8 chunk partials; the tree runs over max(16, d / 8) partials, the missing ones
+ * (d = 64) being +0, off = 16 (d = 256 only), 8, 4, 2, 1. */
+static float canon_tree(float *p, int nchunks)
 {
-    float p[16];
-    for (int c = 0; c < 16; ++c) {
+    int n = nchunks < 16 ? 16 : nchunks;
+    for (int c = nchunks; c < n; ++c) p[c] = 0.0f;
+    for (int off = n / 2; off >= 1; off >>= 1)
+        for (int c = 0; c < off; ++c) p[c] = p[c] + p[c + off];
+    return p[0];
+}
+
+float orc_canon_dot_d(const uint16_t *x, const uint16_t *y, int d)
+{
+    float p[ORC_DMAX / 8];
+    for (int c = 0; c < d / 8; ++c) {
         float part[2];
         for (int par = 0; par < 2; ++par) {
             float acc = orc_bf16_to_f32(x[8 * c + par]) * orc_bf16_to_f32(y[8 * c + par]);
@@ -125,21 +137,21 @@ float orc_canon_dot(const uint16_t *x, const uint16_t *y)
         }
         p[c] = part[0] + part[1];
     }
-    for (int off = 8; off >= 1; off >>= 1)
-        for (int c = 0; c < off; ++c) p[c] = p[c] + p[c + off];
-    return p[0];
+    return canon_tree(p, d / 8);
 }
 
-static double dot64(const uint16_t *x, const uint16_t *y)
+float orc_canon_dot(const uint16_t *x, const uint16_t *y) { return orc_canon_dot_d(x, y, 128); }
+
+static double dot64(const uint16_t *x, const uint16_t *y, int d)
 {
     double s = 0.0;
-    for (int e = 0; e < ORC_D; ++e) s += (double)orc_bf16_to_f32(x[e]) * (double)orc_bf16_to_f32(y[e]);
+    for (int e = 0; e < d; ++e) s += (double)orc_bf16_to_f32(x[e]) * (double)orc_bf16_to_f32(y[e]);
     return s;
 }
 
 static int shape_ok(const orc_shape *s)
 {
-    return s && s->head_dim == ORC_D && s->page_size > 0 && s->batch > 0 && s->n_kv_heads > 0 &&
+    return s && (s->head_dim == 64 || s->head_dim == 128 || s->head_dim == 256) && s->page_size > 0 && s->batch > 0 && s->n_kv_heads > 0 &&
            s->n_q_heads > 0 && s->n_q_heads % s->n_kv_heads == 0 && s->max_pages_per_seq > 0;
 }
 
@@ -165,8 +177,8 @@ int orc_build_summaries(const orc_shape *s, const uint16_t *K, const int32_t *bt
             int n = T - l * s->page_size;
             if (n > s->page_size) n = s->page_size;
             for (int g = 0; g < s->n_kv_heads; ++g) {
-                uint16_t *dst = summaries + (p * s->n_kv_heads + g) * ORC_D;
-                for (int e = 0; e < ORC_D; ++e) {
+                uint16_t *dst = summaries + (p * s->n_kv_heads + g) * s->head_dim;
+                for (int e = 0; e < s->head_dim; ++e) {
                     float acc = 0.0f;
                     for (int t = 0; t < n; ++t) acc = acc + orc_bf16_to_f32(kv_row(s, K, p, g, t)[e]);
                     dst[e] = orc_f32_to_bf16(acc / (float)n);
@@ -205,10 +217,10 @@ int orc_route(const orc_shape *s, const uint16_t *q, const uint16_t *summaries, 
         int b = u / s->n_q_heads, h = u % s->n_q_heads, g = h / G;
         int nb = n_pages_of(s, seq_lens[b]);
         scored *c = (scored *)malloc(sizeof(scored) * (size_t)(nb > 0 ? nb : 1));
-        const uint16_t *qv = q + (int64_t)u * ORC_D;
+        const uint16_t *qv = q + (int64_t)u * s->head_dim;
         for (int l = 0; l < nb; ++l) {
             int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
-            c[l].s = orc_canon_dot(qv, summaries + (p * s->n_kv_heads + g) * ORC_D);
+            c[l].s = orc_canon_dot_d(qv, summaries + (p * s->n_kv_heads + g) * s->head_dim, s->head_dim);
             c[l].idx = l;
             if (all_scores) all_scores[(int64_t)u * s->max_pages_per_seq + l] = c[l].s;
         }
@@ -245,8 +257,8 @@ int orc_build_super_summaries(const orc_shape *s, const uint16_t *summaries, con
                 float best_n = 0.0f;
                 for (int l = sp * ORC_SUPER; l < (sp + 1) * ORC_SUPER && l < nb; ++l) {
                     int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
-                    const uint16_t *row = summaries + (p * s->n_kv_heads + g) * ORC_D;
-                    float n2 = orc_canon_dot(row, row);
+                    const uint16_t *row = summaries + (p * s->n_kv_heads + g) * s->head_dim;
+                    float n2 = orc_canon_dot_d(row, row, s->head_dim);
                     if (best < 0 || n2 > best_n) {
                         best = l;
                         best_n = n2;
@@ -255,10 +267,10 @@ int orc_build_super_summaries(const orc_shape *s, const uint16_t *summaries, con
                 super_rep[o] = best;
                 if (best >= 0) {
                     int64_t p = bt[(int64_t)b * s->max_pages_per_seq + best];
-                    memcpy(super_summaries + o * ORC_D, summaries + (p * s->n_kv_heads + g) * ORC_D,
-                           sizeof(uint16_t) * ORC_D);
+                    memcpy(super_summaries + o * s->head_dim, summaries + (p * s->n_kv_heads + g) * s->head_dim,
+                           sizeof(uint16_t) * s->head_dim);
                 } else {
-                    memset(super_summaries + o * ORC_D, 0, sizeof(uint16_t) * ORC_D);
+                    memset(super_summaries + o * s->head_dim, 0, sizeof(uint16_t) * s->head_dim);
                 }
             }
         }
@@ -282,10 +294,10 @@ int orc_route_two_level(const orc_shape *s, const uint16_t *q, const uint16_t *s
         int b = u / s->n_q_heads, h = u % s->n_q_heads, g = h / G;
         int nb = n_pages_of(s, seq_lens[b]);
         int ns = (nb + ORC_SUPER - 1) / ORC_SUPER;
-        const uint16_t *qv = q + (int64_t)u * ORC_D;
+        const uint16_t *qv = q + (int64_t)u * s->head_dim;
         scored *c = (scored *)malloc(sizeof(scored) * (size_t)(ns > 0 ? ns : 1));
         for (int sp = 0; sp < ns; ++sp) {
-            c[sp].s = orc_canon_dot(qv, super_summaries + (((int64_t)b * max_supers + sp) * s->n_kv_heads + g) * ORC_D);
+            c[sp].s = orc_canon_dot_d(qv, super_summaries + (((int64_t)b * max_supers + sp) * s->n_kv_heads + g) * s->head_dim, s->head_dim);
             c[sp].idx = sp;
         }
         qsort(c, (size_t)ns, sizeof(scored), cmp_scored);
@@ -296,7 +308,7 @@ int orc_route_two_level(const orc_shape *s, const uint16_t *q, const uint16_t *s
         for (int i = 0; i < keep_s; ++i) {
             for (int l = c[i].idx * ORC_SUPER; l < (c[i].idx + 1) * ORC_SUPER && l < nb; ++l) {
                 int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
-                pg[n].s = orc_canon_dot(qv, summaries + (p * s->n_kv_heads + g) * ORC_D);
+                pg[n].s = orc_canon_dot_d(qv, summaries + (p * s->n_kv_heads + g) * s->head_dim, s->head_dim);
                 pg[n].idx = l;
                 ++n;
             }
@@ -328,7 +340,7 @@ int orc_sparse(const orc_shape *s, const uint16_t *q, const uint16_t *K, const u
     for (int u = 0; u < units; ++u) {
         int b = u / s->n_q_heads, h = u % s->n_q_heads, g = h / G;
         int T = seq_lens[b];
-        const uint16_t *qv = q + (int64_t)u * ORC_D;
+        const uint16_t *qv = q + (int64_t)u * s->head_dim;
         scored *c = (scored *)malloc(sizeof(scored) * (size_t)P * (size_t)s->page_size);
         int nv = 0;
         /* token routing: exact fp32 score of every valid token of every routed page */
@@ -339,7 +351,7 @@ int orc_sparse(const orc_shape *s, const uint16_t *q, const uint16_t *K, const u
             for (int t = 0; t < s->page_size; ++t) {
                 int pos = l * s->page_size + t;
                 if (pos >= T) break;
-                c[nv].s = orc_canon_dot(qv, kv_row(s, K, p, g, t));
+                c[nv].s = orc_canon_dot_d(qv, kv_row(s, K, p, g, t), s->head_dim);
                 c[nv].idx = pos;
                 ++nv;
             }
@@ -353,21 +365,21 @@ int orc_sparse(const orc_shape *s, const uint16_t *q, const uint16_t *K, const u
         for (int i = 0; i < ns; ++i) {
             int pos = c[i].idx, l = pos / s->page_size, t = pos % s->page_size;
             int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
-            s64[i] = dot64(qv, kv_row(s, K, p, g, t));
+            s64[i] = dot64(qv, kv_row(s, K, p, g, t), s->head_dim);
             if (s64[i] > m) m = s64[i];
         }
-        double Z = 0.0, acc[ORC_D];
-        for (int e = 0; e < ORC_D; ++e) acc[e] = 0.0;
+        double Z = 0.0, acc[ORC_DMAX];
+        for (int e = 0; e < s->head_dim; ++e) acc[e] = 0.0;
         for (int i = 0; i < ns; ++i) {
             int pos = c[i].idx, l = pos / s->page_size, t = pos % s->page_size;
             int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
             const uint16_t *vr = kv_row(s, V, p, g, t);
             double w = exp((s64[i] - m) / eps);
             Z += w;
-            for (int e = 0; e < ORC_D; ++e) acc[e] += w * (double)orc_bf16_to_f32(vr[e]);
+            for (int e = 0; e < s->head_dim; ++e) acc[e] += w * (double)orc_bf16_to_f32(vr[e]);
             if (cand_weight) cand_weight[(int64_t)u * K_c + i] = w;
         }
-        for (int e = 0; e < ORC_D; ++e) out[(int64_t)u * ORC_D + e] = ns > 0 ? acc[e] / Z : 0.0;
+        for (int e = 0; e < s->head_dim; ++e) out[(int64_t)u * s->head_dim + e] = ns > 0 ? acc[e] / Z : 0.0;
         if (cand_weight)
             for (int i = 0; i < K_c; ++i)
                 cand_weight[(int64_t)u * K_c + i] = i < ns ? cand_weight[(int64_t)u * K_c + i] / Z : 0.0;
@@ -430,8 +442,8 @@ int orc_route_group(const orc_shape *s, const uint16_t *q, const uint16_t *summa
         for (int l = 0; l < nb; ++l) {
             int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
             for (int h = 0; h < G; ++h)
-                ph[h] = orc_canon_dot(q + ((int64_t)b * s->n_q_heads + g * G + h) * ORC_D,
-                                      summaries + (p * s->n_kv_heads + g) * ORC_D);
+                ph[h] = orc_canon_dot_d(q + ((int64_t)b * s->n_q_heads + g * G + h) * s->head_dim,
+                                      summaries + (p * s->n_kv_heads + g) * s->head_dim, s->head_dim);
             c[l].s = group_sum(ph, G);
             c[l].idx = l;
         }
@@ -487,8 +499,8 @@ int orc_sparse_group(const orc_shape *s, const uint16_t *q, const uint16_t *K, c
                 int pos = l * s->page_size + t;
                 if (pos >= T) break;
                 for (int h = 0; h < G; ++h)
-                    sh[(size_t)nv * G + h] = orc_canon_dot(q + ((int64_t)b * s->n_q_heads + g * G + h) * ORC_D,
-                                                           kv_row(s, K, p, g, t));
+                    sh[(size_t)nv * G + h] = orc_canon_dot_d(q + ((int64_t)b * s->n_q_heads + g * G + h) * s->head_dim,
+                                                           kv_row(s, K, p, g, t), s->head_dim);
                 c[nv].s = group_sum(sh + (size_t)nv * G, G);
                 c[nv].idx = pos;
                 c[nv].k = nv;
@@ -500,26 +512,26 @@ int orc_sparse_group(const orc_shape *s, const uint16_t *q, const uint16_t *K, c
         for (int i = 0; i < K_c; ++i) cand_pos[(int64_t)gr * K_c + i] = i < ns ? c[i].idx : -1;
         for (int h = 0; h < G; ++h) {
             int64_t u = (int64_t)b * s->n_q_heads + g * G + h;
-            const uint16_t *qv = q + u * ORC_D;
+            const uint16_t *qv = q + u * s->head_dim;
             /* this head's softmax over the shared candidates, fp64 */
-            double m = -INFINITY, Z = 0.0, acc[ORC_D];
+            double m = -INFINITY, Z = 0.0, acc[ORC_DMAX];
             double *s64 = (double *)malloc(sizeof(double) * (size_t)(ns > 0 ? ns : 1));
             for (int i = 0; i < ns; ++i) {
                 int pos = c[i].idx, l = pos / s->page_size, t = pos % s->page_size;
                 int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
-                s64[i] = dot64(qv, kv_row(s, K, p, g, t));
+                s64[i] = dot64(qv, kv_row(s, K, p, g, t), s->head_dim);
                 if (s64[i] > m) m = s64[i];
             }
-            for (int e = 0; e < ORC_D; ++e) acc[e] = 0.0;
+            for (int e = 0; e < s->head_dim; ++e) acc[e] = 0.0;
             for (int i = 0; i < ns; ++i) {
                 int pos = c[i].idx, l = pos / s->page_size, t = pos % s->page_size;
                 int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
                 const uint16_t *vr = kv_row(s, V, p, g, t);
                 double w = exp((s64[i] - m) / eps);
                 Z += w;
-                for (int e = 0; e < ORC_D; ++e) acc[e] += w * (double)orc_bf16_to_f32(vr[e]);
+                for (int e = 0; e < s->head_dim; ++e) acc[e] += w * (double)orc_bf16_to_f32(vr[e]);
             }
-            for (int e = 0; e < ORC_D; ++e) out[u * ORC_D + e] = ns > 0 ? acc[e] / Z : 0.0;
+            for (int e = 0; e < s->head_dim; ++e) out[u * s->head_dim + e] = ns > 0 ? acc[e] / Z : 0.0;
             lse[u] = ns > 0 ? m / eps + log(Z) : -INFINITY;
             free(s64);
             /* this head's own fp32 scores: best and second best inside S, best outside */
@@ -563,10 +575,10 @@ int orc_sparse_group(const orc_shape *s, const uint16_t *q, const uint16_t *K, c
  * first product of a chain rounded on its own - what a packed multiply followed by packed fused
  * multiply-adds computes).  Every operation below is a single correctly rounded fp32 operation,
  * so that a GPU can reproduce the numbers bit for bit. */
-static float canon_sumsq(const float *d)
+static float canon_sumsq(const float *d, int dim)
 {
-    float p[16];
-    for (int c = 0; c < 16; ++c) {
+    float p[ORC_DMAX / 8];
+    for (int c = 0; c < dim / 8; ++c) {
         float part[2];
         for (int par = 0; par < 2; ++par) {
             float acc = d[8 * c + par] * d[8 * c + par];
@@ -575,9 +587,7 @@ static float canon_sumsq(const float *d)
         }
         p[c] = part[0] + part[1];
     }
-    for (int off = 8; off >= 1; off >>= 1)
-        for (int c = 0; c < off; ++c) p[c] = p[c] + p[c + off];
-    return p[0];
+    return canon_tree(p, dim / 8);
 }
 
 int orc_build_radii(const orc_shape *s, const uint16_t *K, const uint16_t *summaries, const int32_t *bt,
@@ -593,16 +603,16 @@ int orc_build_radii(const orc_shape *s, const uint16_t *K, const uint16_t *summa
             int n = T - l * s->page_size;
             if (n > s->page_size) n = s->page_size;
             for (int g = 0; g < s->n_kv_heads; ++g) {
-                float mu[ORC_D], diff[ORC_D];
-                for (int e = 0; e < ORC_D; ++e) mu[e] = orc_bf16_to_f32(summaries[(p * s->n_kv_heads + g) * ORC_D + e]);
+                float mu[ORC_DMAX], diff[ORC_DMAX];
+                for (int e = 0; e < s->head_dim; ++e) mu[e] = orc_bf16_to_f32(summaries[(p * s->n_kv_heads + g) * s->head_dim + e]);
                 float d2max = 0.0f;
                 for (int t = 0; t < n; ++t) {
                     const uint16_t *row = kv_row(s, K, p, g, t);
-                    for (int e = 0; e < ORC_D; ++e) diff[e] = orc_bf16_to_f32(row[e]) - mu[e];
-                    float d2 = canon_sumsq(diff);
+                    for (int e = 0; e < s->head_dim; ++e) diff[e] = orc_bf16_to_f32(row[e]) - mu[e];
+                    float d2 = canon_sumsq(diff, s->head_dim);
                     if (d2 > d2max) d2max = d2;
                 }
-                float r = sqrtf(d2max), mun = sqrtf(canon_sumsq(mu));
+                float r = sqrtf(d2max), mun = sqrtf(canon_sumsq(mu, s->head_dim));
                 float t1 = r * 1.001f, t2 = mun * 0x1p-12f;
                 radii[p * s->n_kv_heads + g] = t1 + t2;
             }
@@ -630,9 +640,9 @@ int orc_certify(const orc_shape *s, const uint16_t *q, const float *radii, const
     for (int u = 0; u < units; ++u) {
         int b = u / s->n_q_heads, h = u % s->n_q_heads, g = h / G;
         int T = seq_lens[b], nb = n_pages_of(s, T);
-        float qf[ORC_D];
-        for (int e = 0; e < ORC_D; ++e) qf[e] = orc_bf16_to_f32(q[(int64_t)u * ORC_D + e]);
-        float qn = sqrtf(canon_sumsq(qf)) * 1.00000095367431640625f;
+        float qf[ORC_DMAX];
+        for (int e = 0; e < s->head_dim; ++e) qf[e] = orc_bf16_to_f32(q[(int64_t)u * s->head_dim + e]);
+        float qn = sqrtf(canon_sumsq(qf, s->head_dim)) * 1.00000095367431640625f;
         float ub = -INFINITY;
         for (int l = 0; l < nb; ++l) {
             int routed = 0;
@@ -665,10 +675,10 @@ int orc_certify(const orc_shape *s, const uint16_t *q, const float *radii, const
  * which a GPU reproduces bit for bit.  The paper fixes neither start, step rule nor tie-break.
  * cand_pos: the candidates' token positions (any order, -1 padded, K_c wide); alpha comes back in
  * the same order. */
-static float canon_dot32(const float *a, const float *b)
+static float canon_dot32(const float *a, const float *b, int dim)
 {
-    float p[16];
-    for (int c = 0; c < 16; ++c) {
+    float p[ORC_DMAX / 8];
+    for (int c = 0; c < dim / 8; ++c) {
         float part[2];
         for (int par = 0; par < 2; ++par) {
             float acc = a[8 * c + par] * b[8 * c + par];
@@ -677,9 +687,7 @@ static float canon_dot32(const float *a, const float *b)
         }
         p[c] = part[0] + part[1];
     }
-    for (int off = 8; off >= 1; off >>= 1)
-        for (int c = 0; c < off; ++c) p[c] = p[c] + p[c + off];
-    return p[0];
+    return canon_tree(p, dim / 8);
 }
 
 int orc_frank_wolfe(const orc_shape *s, const uint16_t *q, const uint16_t *K, const int32_t *bt,
@@ -699,45 +707,45 @@ int orc_frank_wolfe(const orc_shape *s, const uint16_t *q, const uint16_t *K, co
         for (int i = 0; i < K_c; ++i) al[i] = 0.0f;
         fw_gap[u] = objective[u] = residual2[u] = step[u] = 0.0f;
         if (n == 0) continue;
-        float *rows = (float *)malloc(sizeof(float) * (size_t)n * ORC_D);
+        float *rows = (float *)malloc(sizeof(float) * (size_t)n * s->head_dim);
         float *sc = (float *)malloc(sizeof(float) * (size_t)n);
         float *gr = (float *)malloc(sizeof(float) * (size_t)n);
-        float qf[ORC_D], y[ORC_D], d[ORC_D], r[ORC_D];
-        for (int e = 0; e < ORC_D; ++e) qf[e] = orc_bf16_to_f32(q[(int64_t)u * ORC_D + e]);
+        float qf[ORC_DMAX], y[ORC_DMAX], d[ORC_DMAX], r[ORC_DMAX];
+        for (int e = 0; e < s->head_dim; ++e) qf[e] = orc_bf16_to_f32(q[(int64_t)u * s->head_dim + e]);
         for (int i = 0; i < n; ++i) {
             int l = cp[i] / s->page_size, t = cp[i] % s->page_size;
             const uint16_t *row = kv_row(s, K, bt[(int64_t)b * s->max_pages_per_seq + l], g, t);
-            for (int e = 0; e < ORC_D; ++e) rows[(size_t)i * ORC_D + e] = orc_bf16_to_f32(row[e]);
-            sc[i] = orc_canon_dot(q + (int64_t)u * ORC_D, row);
+            for (int e = 0; e < s->head_dim; ++e) rows[(size_t)i * s->head_dim + e] = orc_bf16_to_f32(row[e]);
+            sc[i] = orc_canon_dot_d(q + (int64_t)u * s->head_dim, row, s->head_dim);
         }
         /* start: best score, lower position on ties */
         int j = 0;
         for (int i = 1; i < n; ++i)
             if (sc[i] > sc[j] || (sc[i] == sc[j] && cp[i] < cp[j])) j = i;
         al[j] = 1.0f;
-        for (int e = 0; e < ORC_D; ++e) y[e] = rows[(size_t)j * ORC_D + e];
+        for (int e = 0; e < s->head_dim; ++e) y[e] = rows[(size_t)j * s->head_dim + e];
         float gamma = 0.0f, gmin = 0.0f;
         for (int it = 0;; ++it) {
-            for (int i = 0; i < n; ++i) gr[i] = canon_dot32(y, rows + (size_t)i * ORC_D) - sc[i];
+            for (int i = 0; i < n; ++i) gr[i] = canon_dot32(y, rows + (size_t)i * s->head_dim, s->head_dim) - sc[i];
             j = 0;
             for (int i = 1; i < n; ++i)
                 if (gr[i] < gr[j] || (gr[i] == gr[j] && cp[i] < cp[j])) j = i;
             gmin = gr[j];
             if (it >= iters) break;
-            for (int e = 0; e < ORC_D; ++e) {
-                d[e] = rows[(size_t)j * ORC_D + e] - y[e];
+            for (int e = 0; e < s->head_dim; ++e) {
+                d[e] = rows[(size_t)j * s->head_dim + e] - y[e];
                 r[e] = qf[e] - y[e];
             }
-            float num = canon_dot32(r, d), den = canon_dot32(d, d);
+            float num = canon_dot32(r, d, s->head_dim), den = canon_dot32(d, d, s->head_dim);
             gamma = den > 0.0f ? num / den : 0.0f;
             gamma = gamma < 0.0f ? 0.0f : (gamma > 1.0f ? 1.0f : gamma);
-            for (int e = 0; e < ORC_D; ++e) y[e] = fmaf(gamma, d[e], y[e]);
+            for (int e = 0; e < s->head_dim; ++e) y[e] = fmaf(gamma, d[e], y[e]);
             for (int i = 0; i < n; ++i) al[i] = fmaf(-gamma, al[i], al[i]);
             al[j] = al[j] + gamma;
         }
-        for (int e = 0; e < ORC_D; ++e) r[e] = y[e] - qf[e];
-        float r2 = canon_dot32(r, r);
-        fw_gap[u] = canon_dot32(y, r) - gmin;
+        for (int e = 0; e < s->head_dim; ++e) r[e] = y[e] - qf[e];
+        float r2 = canon_dot32(r, r, s->head_dim);
+        fw_gap[u] = canon_dot32(y, r, s->head_dim) - gmin;
         residual2[u] = r2;
         objective[u] = 0.5f * r2;
         step[u] = gamma;
@@ -766,7 +774,7 @@ int orc_dense(const orc_shape *s, const uint16_t *q, const uint16_t *K, const ui
         if (unit_mask && !unit_mask[u]) continue;
         int b = u / s->n_q_heads, h = u % s->n_q_heads, g = h / G;
         int T = seq_lens[b];
-        const uint16_t *qv = q + (int64_t)u * ORC_D;
+        const uint16_t *qv = q + (int64_t)u * s->head_dim;
         double *sc = (double *)malloc(sizeof(double) * (size_t)T);
         unsigned char *inS = (unsigned char *)calloc((size_t)T, 1);
         if (cand_pos)
@@ -778,32 +786,32 @@ int orc_dense(const orc_shape *s, const uint16_t *q, const uint16_t *K, const ui
         for (int pos = 0; pos < T; ++pos) {
             int l = pos / s->page_size, t = pos % s->page_size;
             int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
-            sc[pos] = dot64(qv, kv_row(s, K, p, g, t));
+            sc[pos] = dot64(qv, kv_row(s, K, p, g, t), s->head_dim);
             if (sc[pos] > m) m = sc[pos];
             if (!inS[pos] && sc[pos] > m_off) m_off = sc[pos];
         }
-        double Z = 0.0, Zoff = 0.0, acc[ORC_D], accoff[ORC_D];
-        for (int e = 0; e < ORC_D; ++e) acc[e] = accoff[e] = 0.0;
+        double Z = 0.0, Zoff = 0.0, acc[ORC_DMAX], accoff[ORC_DMAX];
+        for (int e = 0; e < s->head_dim; ++e) acc[e] = accoff[e] = 0.0;
         for (int pos = 0; pos < T; ++pos) {
             int l = pos / s->page_size, t = pos % s->page_size;
             int64_t p = bt[(int64_t)b * s->max_pages_per_seq + l];
             const uint16_t *vr = kv_row(s, V, p, g, t);
             double w = exp((sc[pos] - m) / eps);
             Z += w;
-            for (int e = 0; e < ORC_D; ++e) acc[e] += w * (double)orc_bf16_to_f32(vr[e]);
+            for (int e = 0; e < s->head_dim; ++e) acc[e] += w * (double)orc_bf16_to_f32(vr[e]);
             if (cand_pos && !inS[pos]) {
                 Zoff += w;
-                for (int e = 0; e < ORC_D; ++e) accoff[e] += w * (double)orc_bf16_to_f32(vr[e]);
+                for (int e = 0; e < s->head_dim; ++e) accoff[e] += w * (double)orc_bf16_to_f32(vr[e]);
             }
         }
-        for (int e = 0; e < ORC_D; ++e) out[(int64_t)u * ORC_D + e] = acc[e] / Z;
+        for (int e = 0; e < s->head_dim; ++e) out[(int64_t)u * s->head_dim + e] = acc[e] / Z;
         lse[u] = m / eps + log(Z);
         if (cand_pos) {
             if (true_leak) true_leak[u] = Zoff / Z;
             if (true_gap) true_gap[u] = m - m_off; /* +inf when nothing lies outside S */
             if (y_off)
-                for (int e = 0; e < ORC_D; ++e)
-                    y_off[(int64_t)u * ORC_D + e] = Zoff > 0.0 ? accoff[e] / Zoff : 0.0;
+                for (int e = 0; e < s->head_dim; ++e)
+                    y_off[(int64_t)u * s->head_dim + e] = Zoff > 0.0 ? accoff[e] / Zoff : 0.0;
         }
         free(inS);
         free(sc);
