@@ -588,6 +588,9 @@ def sweep(dev, steps_small=200):
     # 32-token pages: config 1 with half as many pages routed (the same 512 scored tokens per unit)
     c1 = config_spec(1)
     out["page32"] = measure_point(replace(c1, page_size=32, P=c1.P // 2, layers=16, name="cfg1_page32_halfP"), dev, 100)
+    # other head dimensions: config 1's shape at d = 64 and d = 256 (temperature sqrt(d))
+    out["head_dims"] = [measure_point(replace(c1, head_dim=d, epsilon=math.sqrt(d), layers=L, name=f"cfg1_d{d}"), dev, 100)
+                        for d, L in ((64, 16), (256, 8))]
     # group-shared routing (one selection per KV head) on config 1 and at batch 16
     gs = []
     for spec_g in (replace(config_spec(1), layers=16, name="cfg1_16layers"),

@@ -51,7 +51,8 @@ int make_geometry(const vsa_shape_t* s, Geometry* g)
     if (s->n_q_heads % s->n_kv_heads != 0) return VSA_ERR_INVALID_ARGUMENT;
     if (s->kv_page_stride < 0 || s->kv_head_stride < 0 || s->kv_token_stride < 0) return VSA_ERR_INVALID_ARGUMENT;
     const int group = s->n_q_heads / s->n_kv_heads;
-    if (s->head_dim != vsa::kHeadDim || (s->page_size != 16 && s->page_size != 32)) return VSA_ERR_UNSUPPORTED_SHAPE;
+    if ((s->head_dim != 64 && s->head_dim != 128 && s->head_dim != 256) || (s->page_size != 16 && s->page_size != 32))
+        return VSA_ERR_UNSUPPORTED_SHAPE;
     if (group != 1 && group != 2 && group != 4 && group != 8 && group != 16 && group != 32)
         return VSA_ERR_UNSUPPORTED_SHAPE;
     if (s->max_pages_per_seq > kMaxPagesPerSeq) return VSA_ERR_UNSUPPORTED_SHAPE;
@@ -59,7 +60,8 @@ int make_geometry(const vsa_shape_t* s, Geometry* g)
     if ((long long)s->batch * s->n_q_heads > 0x3fffffffLL) return VSA_ERR_UNSUPPORTED_SHAPE;
     // (sequence, KV head) pairs the dense pass tracks; groups above 8 count as n_q_heads / 8 heads there
     if ((long long)s->batch * (group > 8 ? s->n_q_heads / 8 : s->n_kv_heads) > 4096) return VSA_ERR_UNSUPPORTED_SHAPE;
-    if (s->num_pool_pages * s->n_kv_heads >= (1LL << 27)) return VSA_ERR_UNSUPPORTED_SHAPE;
+    // (the summary pool is addressed in 16-byte units by a 32-bit offset: 2^27 rows of 256 bytes)
+    if (s->num_pool_pages * s->n_kv_heads * (s->head_dim / 8) >= (1LL << 31)) return VSA_ERR_UNSUPPORTED_SHAPE;
     g->batch = s->batch;
     g->n_q_heads = s->n_q_heads;
     g->n_kv_heads = s->n_kv_heads;
@@ -68,6 +70,7 @@ int make_geometry(const vsa_shape_t* s, Geometry* g)
     g->kv_heads_stored = s->n_kv_heads;
     g->max_pages = s->max_pages_per_seq;
     g->page_size = s->page_size;
+    g->head_dim = s->head_dim;
     g->tile_shift = s->page_size == 32 ? 1 : 0;
     g->super_pages = 0;
     g->pool_pages = s->num_pool_pages;
@@ -215,6 +218,7 @@ int vsa_build_page_radii(const vsa_shape_t* shape, const void* k_cache, const vo
     Geometry g;
     int rc = make_geometry(shape, &g);
     if (rc) return rc;
+    if (g.head_dim != vsa::kHeadDim) return VSA_ERR_UNSUPPORTED_SHAPE;   // this entry point: head_dim 128 only
     if (!k_cache || !summaries || !block_table || !seq_lens || !radii) return VSA_ERR_INVALID_ARGUMENT;
     if (!aligned16(k_cache) || !aligned16(summaries)) return VSA_ERR_MISALIGNED;
     return cuda_rc(vsa::launch_build_radii(g, k_cache, summaries, block_table, seq_lens, first_page, radii,
@@ -227,6 +231,7 @@ int vsa_append_kv(const vsa_shape_t* shape, const void* k_new, const void* v_new
     Geometry g;
     int rc = make_geometry(shape, &g);
     if (rc) return rc;
+    if (g.head_dim != vsa::kHeadDim) return VSA_ERR_UNSUPPORTED_SHAPE;   // this entry point: head_dim 128 only
     if (!k_new || !v_new || !k_cache || !v_cache || !block_table || !seq_lens || !summaries)
         return VSA_ERR_INVALID_ARGUMENT;
     if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(summaries))
@@ -259,6 +264,7 @@ int vsa_build_super_summaries(const vsa_shape_t* shape, const void* summaries, c
     Geometry g;
     int rc = make_geometry(shape, &g);
     if (rc) return rc;
+    if (g.head_dim != vsa::kHeadDim) return VSA_ERR_UNSUPPORTED_SHAPE;   // this entry point: head_dim 128 only
     if (!summaries || !block_table || !seq_lens || !super_summaries) return VSA_ERR_INVALID_ARGUMENT;
     if (!aligned16(summaries) || !aligned16(super_summaries)) return VSA_ERR_MISALIGNED;
     return cuda_rc(vsa::launch_build_super_summaries(g, summaries, block_table, seq_lens, first_super,
@@ -273,6 +279,7 @@ int vsa_route_pages_two_level(const vsa_shape_t* shape, const void* q, const voi
     Geometry g;
     int rc = make_geometry(shape, &g);
     if (rc) return rc;
+    if (g.head_dim != vsa::kHeadDim) return VSA_ERR_UNSUPPORTED_SHAPE;   // this entry point: head_dim 128 only
     if ((rc = check_routing_sizes(g, P, 0, false))) return rc;
     if ((rc = check_routing_sizes(g, P_super, 0, false))) return rc;
     if (!q || !summaries || !super_summaries || !block_table || !seq_lens || !routed_pages || !ws)
@@ -298,6 +305,7 @@ int vsa_decode_step_two_level(const vsa_shape_t* shape, const void* q, const voi
     Geometry g;
     int rc = make_geometry(shape, &g);
     if (rc) return rc;
+    if (g.head_dim != vsa::kHeadDim) return VSA_ERR_UNSUPPORTED_SHAPE;   // this entry point: head_dim 128 only
     if ((rc = check_routing_sizes(g, P, K_c, true))) return rc;
     if ((rc = check_routing_sizes(g, P_super, 0, false))) return rc;
     if ((rc = check_epsilon(epsilon))) return rc;
@@ -370,6 +378,7 @@ static int sparse_solver_impl(int solver_kind, const vsa_shape_t* shape, const v
     Geometry g;
     int rc = make_geometry(shape, &g);
     if (rc) return rc;
+    if (g.head_dim != vsa::kHeadDim) return VSA_ERR_UNSUPPORTED_SHAPE;   // this entry point: head_dim 128 only
     if ((rc = check_routing_sizes(g, P, K_c, true))) return rc;
     if ((rc = check_solver_sizes(K_c, solver_iters))) return rc;
     if ((rc = check_epsilon(epsilon))) return rc;
@@ -434,6 +443,7 @@ static int decode_step_impl(const vsa_shape_t* shape, const void* q, const void*
     Geometry g;
     int rc = make_geometry(shape, &g);
     if (rc) return rc;
+    if (g.head_dim != vsa::kHeadDim && (solve || cert)) return VSA_ERR_UNSUPPORTED_SHAPE;   // closed form only
     if ((rc = check_routing_sizes(g, P, K_c, true))) return rc;
     if (solve && (rc = check_solver_sizes(K_c, solver_iters))) return rc;
     if ((rc = check_epsilon(epsilon))) return rc;
@@ -503,6 +513,7 @@ int vsa_decode_step_group_shared(const vsa_shape_t* shape, const void* q, const 
     Geometry g;
     int rc = make_geometry(shape, &g);
     if (rc) return rc;
+    if (g.head_dim != vsa::kHeadDim) return VSA_ERR_UNSUPPORTED_SHAPE;   // this entry point: head_dim 128 only
     if ((rc = check_routing_sizes(g, P, K_c, true))) return rc;
     if ((rc = check_epsilon(epsilon))) return rc;
     if (isnan(gap_threshold)) return VSA_ERR_INVALID_ARGUMENT;
@@ -589,6 +600,7 @@ int vsa_decode_step_certified_expand(const vsa_shape_t* shape, const void* q, co
     Geometry g;
     int rc = make_geometry(shape, &g);
     if (rc) return rc;
+    if (g.head_dim != vsa::kHeadDim) return VSA_ERR_UNSUPPORTED_SHAPE;   // this entry point: head_dim 128 only
     if ((rc = check_routing_sizes(g, P, K_c, true))) return rc;
     if ((rc = check_routing_sizes(g, P_expand, K_c, true))) return rc;
     if (P_expand <= P) return VSA_ERR_INVALID_ARGUMENT;
@@ -683,11 +695,11 @@ int vsa_decode_step_host(const vsa_shape_t* shape, const void* q_host, void* q_d
     vsa_diag_t* diag_direct = diag_host ? (vsa_diag_t*)mapped_device_pointer(diag_host) : nullptr;
     const void* q_mapped = mapped_device_pointer(q_host);
     if (q_mapped && aligned16(q_mapped)) {
-        const int n16 = (int)(units * vsa::kHeadDim * 2 / 16);
+        const int n16 = (int)(units * g.head_dim * 2 / 16);
         if (vsa::launch_pdl(fetch_rows_kernel, dim3((unsigned)((n16 + 255) / 256)), dim3(256), 0, st,
                             (const uint4*)q_mapped, (uint4*)q_dev, n16) != cudaSuccess)
             return VSA_ERR_CUDA;
-    } else if (cudaMemcpyAsync(q_dev, q_host, units * vsa::kHeadDim * 2, cudaMemcpyHostToDevice, st) !=
+    } else if (cudaMemcpyAsync(q_dev, q_host, units * g.head_dim * 2, cudaMemcpyHostToDevice, st) !=
                cudaSuccess) {
         return VSA_ERR_CUDA;
     }
@@ -696,7 +708,7 @@ int vsa_decode_step_host(const vsa_shape_t* shape, const void* q_host, void* q_d
                          diag_direct ? diag_direct : diag_dev, routed_pages, fallback_list, fallback_count, ws,
                          ws_bytes, stream);
     if (rc) return rc;
-    if (!out_direct && cudaMemcpyAsync(out_host, out_dev, units * vsa::kHeadDim * sizeof(float),
+    if (!out_direct && cudaMemcpyAsync(out_host, out_dev, units * g.head_dim * sizeof(float),
                                        cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return VSA_ERR_CUDA;
     if (diag_host && !diag_direct &&

@@ -23,18 +23,26 @@ namespace vsa {
 
 namespace {
 
-constexpr int kDenseThreads = 256;
-constexpr int kDenseWarps = kDenseThreads / 32;
 constexpr int kStages = 3;                         // pages in flight per warp
 constexpr int kTileRows = 16;                      // the pass walks tiles of 16 tokens: one per 16-token page, two per 32-token page
-constexpr int kTileBytes = kTileRows * kRowBytes;  // 4 KB: K (or V) rows of one tile and KV head
-constexpr int kStageBytes = 2 * kTileBytes;        // K tile + V tile
-constexpr int kRingBytes = kDenseWarps * kStages * kStageBytes;   // 192 KB per block
-constexpr int kPartialFloats = 2 + kHeadDim;       // per (item, head): max (log2 domain), sum, acc[128]
 constexpr int kPagesPerItemGoal = 128;             // pages per item and block from which a second round pays
 constexpr int kMaxRounds = 2;
 constexpr int kMaxRoundsRagged = 8;
-constexpr int kMinPagesPerItem = 2 * kDenseWarps;  // at least two pages per warp: one would expose the DRAM latency
+
+// Sizes that depend on the head dimension D (64, 128 or 256).  The ring of a block holds three stages of a
+// K tile and a V tile per warp: 192 KB with eight warps at D = 128; D = 256 runs four warps per block so
+// that the same ring fits.
+template <int D>
+struct DenseCfg {
+    static constexpr int kDenseThreads = D == 256 ? 128 : 256;
+    static constexpr int kDenseWarps = kDenseThreads / 32;
+    static constexpr int kRowBytes = 2 * D;
+    static constexpr int kTileBytes = kTileRows * kRowBytes;   // K (or V) rows of one tile and KV head (4 KB at D = 128)
+    static constexpr int kStageBytes = 2 * kTileBytes;         // K tile + V tile
+    static constexpr int kRingBytes = kDenseWarps * kStages * kStageBytes;
+    static constexpr int kPartialFloats = 2 + D;               // per (item, head): max (log2 domain), sum, acc[D]
+    static constexpr int kMinPagesPerItem = 2 * kDenseWarps;   // at least two pages per warp: one would expose the DRAM latency
+};
 
 __device__ __forceinline__ void cp_async_16_zfill(uint32_t smem_addr, const void* gptr, bool valid)
 {
@@ -82,8 +90,8 @@ struct DenseSmem {
     int32_t* misc;         // [16]
 };
 
-template <int G>
-__global__ void __launch_bounds__(kDenseThreads, 1)
+template <int G, int D = vsa::kHeadDim>
+__global__ void __launch_bounds__(DenseCfg<D>::kDenseThreads, 1)
 dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* __restrict__ k_cache,
                    const uint16_t* __restrict__ v_cache, const int32_t* __restrict__ block_table,
                    const int32_t* __restrict__ seq_lens, const int32_t* __restrict__ fallback_list,
@@ -91,6 +99,14 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
                    int32_t* __restrict__ counters, float* __restrict__ out, vsa_diag_t* __restrict__ diag,
                    int max_items)
 {
+    using Cfg = DenseCfg<D>;
+    constexpr int kDenseThreads = Cfg::kDenseThreads, kDenseWarps = Cfg::kDenseWarps, kRowBytes = Cfg::kRowBytes,
+                  kTileBytes = Cfg::kTileBytes, kStageBytes = Cfg::kStageBytes, kRingBytes = Cfg::kRingBytes,
+                  kPartialFloats = Cfg::kPartialFloats, kMinPagesPerItem = Cfg::kMinPagesPerItem, kHeadDim = D;
+    constexpr int KS = D / 16;    // 16-element steps of the Q K^T contraction = 16-column steps of P V
+    constexpr int NT = D / 8;     // 8-column output tiles
+    constexpr int CPR = D / 8;    // 16-byte chunks per row
+    constexpr int RPI = 32 / (CPR < 32 ? CPR : 32);   // rows one copy instruction of a warp covers
     extern __shared__ __align__(128) uint8_t dense_smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n_groups = geo.batch * geo.n_kv_heads;
@@ -204,8 +220,8 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
     const int quad = lane & 3;
     uint8_t* my_ring = sm.ring + warp * kStages * kStageBytes;
     const uint32_t ring_addr = (uint32_t)__cvta_generic_to_shared(my_ring);
-    // copy mapping: lane covers 16-byte chunk (lane & 15) of rows (lane >> 4) + 2 i, i = 0..7
-    const int cp_chunk = lane & 15, cp_row0 = lane >> 4;
+    // copy mapping: lane covers 16-byte chunk lane % CPR of rows lane / CPR + RPI i, i = 0 .. 16 / RPI - 1
+    const int cp_chunk = lane % CPR, cp_row0 = lane / CPR;
 
     for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
         // group of this item: last g with item_base[g] <= item
@@ -228,11 +244,11 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
         const int32_t* bt = block_table + (long long)b * geo.max_pages;
 
         // Q fragments of the group: bf16 pairs straight from memory, rows >= G are zero
-        uint32_t qa0[8], qa2[8];
+        uint32_t qa0[KS], qa2[KS];
         {
             const uint16_t* qrow = q + ((long long)b * geo.n_q_heads + g * G + (head < G ? head : 0)) * kHeadDim;
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
+            for (int ks = 0; ks < KS; ++ks) {
                 const uint32_t v0 = *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + quad * 2);
                 const uint32_t v2 = *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8 + quad * 2);
                 qa0[ks] = head < G ? v0 : 0u;
@@ -240,9 +256,9 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
             }
         }
         float m_run = -INFINITY, l_run = 0.0f;   // per lane: head `head`, partial over this lane's columns
-        float o[16][4];
+        float o[NT][4];
 #pragma unroll
-        for (int n = 0; n < 16; ++n)
+        for (int n = 0; n < NT; ++n)
 #pragma unroll
             for (int i = 0; i < 4; ++i) o[n][i] = 0.0f;
 
@@ -261,8 +277,8 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
             const uint16_t* vp = v_cache + phys * geo.page_stride + head_off;
             const uint32_t dst = ring_addr + (uint32_t)((k % kStages) * kStageBytes);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int r = cp_row0 + 2 * i;
+            for (int i = 0; i < kTileRows / RPI; ++i) {
+                const int r = cp_row0 + RPI * i;
                 const uint32_t off = (uint32_t)(r * kRowBytes + ((cp_chunk ^ (r & 7)) << 4));
                 const bool ok = r < valid_rows;
                 cp_async_16_zfill(dst + off, kp + (long long)r * geo.token_stride, ok);
@@ -297,7 +313,7 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
             {
                 const int mi = lane >> 3, tok = (mi >> 1) * 8 + (lane & 7);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
+                for (int ks = 0; ks < KS; ++ks) {
                     const int ch = 2 * ks + (mi & 1);
                     uint32_t r[4];
                     ldmatrix_x4(r, kbase + (uint32_t)(tok * kRowBytes + ((ch ^ (tok & 7)) << 4)));
@@ -322,7 +338,7 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
             l_run = fmaf(l_run, corr, (p[0] + p[1]) + (p[2] + p[3]));
             if (__any_sync(kFullMask, m_new > m_run)) {
 #pragma unroll
-                for (int n = 0; n < 16; ++n) {
+                for (int n = 0; n < NT; ++n) {
                     o[n][0] *= corr;
                     o[n][1] *= corr;
                 }
@@ -334,7 +350,7 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
             {
                 const int mi = lane >> 3, tok = (mi & 1) * 8 + (lane & 7);
 #pragma unroll
-                for (int dp = 0; dp < 8; ++dp) {
+                for (int dp = 0; dp < KS; ++dp) {
                     const int ch = 2 * dp + (mi >> 1);
                     uint32_t r[4];
                     ldmatrix_x4_trans(r, vbase + (uint32_t)(tok * kRowBytes + ((ch ^ (tok & 7)) << 4)));
@@ -358,7 +374,7 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
                 rec[1] = l_run;
             }
 #pragma unroll
-            for (int n = 0; n < 16; ++n) {
+            for (int n = 0; n < NT; ++n) {
                 rec[2 + n * 8 + quad * 2] = o[n][0];
                 rec[2 + n * 8 + quad * 2 + 1] = o[n][1];
             }
@@ -450,7 +466,9 @@ int dense_max_items(const Geometry& g) { return g.batch * g.n_kv_heads + 2048; }
 size_t dense_smem_bytes(const Geometry& g)
 {
     const size_t n_groups = (size_t)g.batch * g.n_kv_heads;
-    return kRingBytes + (n_groups + 1) * 4 + 16 * 4 + (n_groups + 15) / 16 * 16;
+    const size_t ring = g.head_dim == 64 ? DenseCfg<64>::kRingBytes
+                                         : (g.head_dim == 256 ? DenseCfg<256>::kRingBytes : DenseCfg<128>::kRingBytes);
+    return ring + (n_groups + 1) * 4 + 16 * 4 + (n_groups + 15) / 16 * 16;
 }
 
 }  // namespace
@@ -472,7 +490,23 @@ int dense_ticket_count(const Geometry& g_in)
 size_t dense_workspace_bytes(const Geometry& g_in)
 {
     const Geometry g = with_virtual_kv_heads(g_in);
-    return dense_counter_bytes(g) + (size_t)dense_max_items(g) * g.group * kPartialFloats * sizeof(float);
+    return dense_counter_bytes(g) + (size_t)dense_max_items(g) * g.group * (2 + g.head_dim) * sizeof(float);
+}
+
+template <int G, int D>
+static cudaError_t launch_dense_gd(const Geometry& g, const uint16_t* q, const uint16_t* k, const uint16_t* v,
+                                   const int32_t* block_table, const int32_t* seq_lens, const int32_t* fallback_list,
+                                   const int32_t* fallback_count, float epsilon, float* partials, int32_t* counters,
+                                   float* out, vsa_diag_t* diag, cudaStream_t stream)
+{
+    const size_t smem = dense_smem_bytes(g);
+    static bool attr_done[kMaxDevices] = {};   // per template instance
+    const cudaError_t e = allow_large_dynamic_smem(dense_split_kernel<G, D>, attr_done);
+    if (e != cudaSuccess) return e;
+    // persistent grid: one block per SM (the ring fills the shared memory)
+    return launch_pdl(dense_split_kernel<G, D>, dim3((unsigned)num_sms()), dim3(DenseCfg<D>::kDenseThreads), smem,
+                      stream, g, q, k, v, block_table, seq_lens, fallback_list, fallback_count, epsilon, partials,
+                      counters, out, diag, dense_max_items(g));
 }
 
 template <int G>
@@ -481,14 +515,14 @@ static cudaError_t launch_dense_g(const Geometry& g, const uint16_t* q, const ui
                                   const int32_t* fallback_count, float epsilon, float* partials, int32_t* counters,
                                   float* out, vsa_diag_t* diag, cudaStream_t stream)
 {
-    const size_t smem = dense_smem_bytes(g);
-    static bool attr_done[kMaxDevices] = {};   // per template instance
-    const cudaError_t e = allow_large_dynamic_smem(dense_split_kernel<G>, attr_done);
-    if (e != cudaSuccess) return e;
-    // persistent grid: one block per SM (the ring fills the shared memory)
-    return launch_pdl(dense_split_kernel<G>, dim3((unsigned)num_sms()), dim3(kDenseThreads), smem, stream, g, q, k, v,
-                      block_table, seq_lens, fallback_list, fallback_count, epsilon, partials, counters, out, diag,
-                      dense_max_items(g));
+    if (g.head_dim == 64)
+        return launch_dense_gd<G, 64>(g, q, k, v, block_table, seq_lens, fallback_list, fallback_count, epsilon,
+                                      partials, counters, out, diag, stream);
+    if (g.head_dim == 256)
+        return launch_dense_gd<G, 256>(g, q, k, v, block_table, seq_lens, fallback_list, fallback_count, epsilon,
+                                       partials, counters, out, diag, stream);
+    return launch_dense_gd<G, 128>(g, q, k, v, block_table, seq_lens, fallback_list, fallback_count, epsilon, partials,
+                                   counters, out, diag, stream);
 }
 
 cudaError_t launch_dense(const Geometry& g_in, const void* q, const void* k_cache, const void* v_cache,

@@ -25,8 +25,9 @@ constexpr int kBlockPages = 32;      // pages per block-table block (one coalesc
 // (87.7 against 93.6 us per layer with 16) to a 64-sequence log-uniform batch (455 against 482 us).
 constexpr int kMaxBlocksPerWarp = 4;
 
-template <int G>
+template <int G, int D = kHeadDim>
 struct ScanCfg {
+    static constexpr int kRowBytes = 2 * D;               // one summary row
     static constexpr int ROWS = G == 1 ? 8 : 16 / G;      // rows per half-warp per round
     static constexpr int VALS = ROWS * G;                 // (row, head) partials per lane per round (8 or 16)
     static constexpr int ROUND_PAGES = 2 * ROWS;          // pages (rows of one KV head) per warp per round
@@ -62,15 +63,18 @@ __device__ __forceinline__ void cp_async_wait()
 // reduction run without per-lane selects (reduce_scatter16_xor).
 // CERT: the radius of every page (radii[page][kv head], see radii_kernel) is copied into logical page
 // order, rad_logical[b][kv head][page], for the certificate that the fused kernel computes.
-template <int G, bool CERT>
+// D: head dimension (see sparse_kernel.cuh for how a row of 64 or 256 elements maps to the half-warp's lanes).
+template <int G, bool CERT, int D = kHeadDim>
 __global__ void __launch_bounds__(kScanThreads, 2)
 route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* __restrict__ summaries,
                   const int32_t* __restrict__ block_table, const int32_t* __restrict__ seq_lens,
                   float* __restrict__ scores, int blocks_per_warp, int32_t* zero_word, int32_t* zero_words,
                   int zero_count, const float* __restrict__ radii, float* __restrict__ rad_logical)
 {
-    using Cfg = ScanCfg<G>;
+    using Cfg = ScanCfg<G, D>;
     constexpr int ROWS = Cfg::ROWS, VALS = Cfg::VALS, ROUND_PAGES = Cfg::ROUND_PAGES, STAGES = Cfg::STAGES;
+    constexpr int kRowBytes = Cfg::kRowBytes, PIECES = D == 256 ? 2 : 1;
+    static_assert(D == 128 || ((D == 64 || D == 256) && !CERT), "certificate: head dimension 128 only");
     constexpr bool XOR_MAP = VALS == 16;
     // block-table blocks fetched before the sequence length is known: the warp's whole range
     constexpr int kFirstBlocks = kMaxBlocksPerWarp;
@@ -114,10 +118,14 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
     }
     if (!has_range) return;
 
-    uint4 qraw[G];
+    const bool lane_has = D != 64 || c < 8;   // this lane holds a piece of every row
+    uint4 qraw[G][PIECES];
 #pragma unroll
     for (int hh = 0; hh < G; ++hh)
-        qraw[hh] = ld_nc_16B(q + ((long long)b * geo.n_q_heads + g * G + (hh ^ kh)) * kHeadDim + c * 8);
+#pragma unroll
+        for (int pc = 0; pc < PIECES; ++pc)
+            qraw[hh][pc] = lane_has ? ld_nc_16B(q + ((long long)b * geo.n_q_heads + g * G + (hh ^ kh)) * D + pc * 128 + c * 8)
+                                    : make_uint4(0u, 0u, 0u, 0u);
 
     if (geo.super_pages) {
         // the length in super-pages, expressed as a token count so that the page arithmetic below applies
@@ -140,9 +148,11 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
 #pragma unroll
     for (int k = 0; k < kFirstBlocks; ++k)
         if (k < n_blocks) off_tab[k * kBlockPages + lane] = encode(first_entries[k], k * kBlockPages + lane);
-    float qf[G][8];
+    float qf[G][PIECES][8];
 #pragma unroll
-    for (int hh = 0; hh < G; ++hh) unpack8(qraw[hh], qf[hh]);
+    for (int hh = 0; hh < G; ++hh)
+#pragma unroll
+        for (int pc = 0; pc < PIECES; ++pc) unpack8(qraw[hh][pc], qf[hh][pc]);
     __syncwarp();
 
     const int g_stored = g / geo.kv_div;   // the KV head whose summaries this (possibly virtual) head reads
@@ -170,8 +180,12 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
         const uint32_t dst = ring + (uint32_t)((R & (STAGES - 1)) * ROUND_PAGES * kRowBytes) + lane_off;
         const int* tab = off_tab + R * ROUND_PAGES;
 #pragma unroll
-        for (int r = 0; r < ROWS; ++r)
-            cp_async_16(dst + r * kRowBytes, srow + (long long)max(tab[tab_row[r]], 0) * 16);
+        for (int r = 0; r < ROWS; ++r) {
+            const uint8_t* from = srow + (long long)max(tab[tab_row[r]], 0) * 16;
+#pragma unroll
+            for (int pc = 0; pc < PIECES; ++pc)
+                if (lane_has) cp_async_16(dst + r * kRowBytes + pc * 256, from + pc * 256);
+        }
         if constexpr (CERT) {
             if (rad_lane) {
                 // off / 16 = page * n_kv_heads: the row of this page in radii[][n_kv_heads]
@@ -195,11 +209,18 @@ route_scan_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* 
         float vals[16];
 #pragma unroll
         for (int r = 0; r < ROWS; ++r) {
-            const uint4 v = *reinterpret_cast<const uint4*>(src + r * kRowBytes);
-            float kf[8];
-            unpack8(v, kf);
 #pragma unroll
-            for (int hh = 0; hh < G; ++hh) vals[r * G + hh] = chunk_partial(qf[hh], kf);
+            for (int pc = 0; pc < PIECES; ++pc) {
+                const uint4 v = lane_has ? *reinterpret_cast<const uint4*>(src + r * kRowBytes + pc * 256)
+                                         : make_uint4(0u, 0u, 0u, 0u);
+                float kf[8];
+                unpack8(v, kf);
+#pragma unroll
+                for (int hh = 0; hh < G; ++hh) {
+                    const float part = chunk_partial(qf[hh][pc], kf);
+                    vals[r * G + hh] = pc == 0 ? part : vals[r * G + hh] + part;
+                }
+            }
         }
         float s;
         if constexpr (XOR_MAP) {
@@ -281,7 +302,7 @@ int scan_warps_per_block(int warps_per_seq, int batch)
     return best;
 }
 
-template <int G, bool CERT>
+template <int G, bool CERT, int D = kHeadDim>
 cudaError_t launch_scan_g(const Geometry& g, const uint16_t* q, const uint16_t* summaries, const int32_t* block_table,
                           const int32_t* seq_lens, float* scores, int32_t* zero_word, int32_t* zero_words,
                           int zero_count, const float* radii, float* rad_logical, cudaStream_t stream)
@@ -294,11 +315,11 @@ cudaError_t launch_scan_g(const Geometry& g, const uint16_t* q, const uint16_t* 
     // The request is padded to 81 KB so that exactly two blocks are resident per SM: with a third one
     // fewer blocks of the kernel that follows fit beside the scan's to start early, and the step gets
     // slower although the scan does not (measured: 30.0 against 24.8 us per layer at batch 8, T = 32k).
-    const size_t smem = std::max((size_t)kScanWarps * ScanCfg<G>::WARP_BYTES, (size_t)81 * 1024);
+    const size_t smem = std::max((size_t)kScanWarps * ScanCfg<G, D>::WARP_BYTES, (size_t)81 * 1024);
     static bool attr_done[kMaxDevices] = {};   // per template instance
-    const cudaError_t e = allow_large_dynamic_smem(route_scan_kernel<G, CERT>, attr_done);
+    const cudaError_t e = allow_large_dynamic_smem(route_scan_kernel<G, CERT, D>, attr_done);
     if (e != cudaSuccess) return e;
-    return launch_pdl(route_scan_kernel<G, CERT>, grid, dim3(wpb * 32), smem, stream, g, q, summaries,
+    return launch_pdl(route_scan_kernel<G, CERT, D>, grid, dim3(wpb * 32), smem, stream, g, q, summaries,
                       block_table, seq_lens, scores, bpw, zero_word, zero_words, zero_count, radii, rad_logical);
 }
 
@@ -319,10 +340,17 @@ cudaError_t launch_route_scan(const Geometry& g_in, const void* q, const void* s
     const uint16_t* ss = (const uint16_t*)summaries;
 #define VSA_SCAN_CASE(G)                                                                                       \
     case G:                                                                                                    \
+        if (g.head_dim == 64)                                                                                  \
+            return launch_scan_g<G, false, 64>(g, qq, ss, block_table, seq_lens, scores, zero_word, zero_words, \
+                                               zero_count, nullptr, nullptr, stream);                          \
+        if (g.head_dim == 256)                                                                                 \
+            return launch_scan_g<G, false, 256>(g, qq, ss, block_table, seq_lens, scores, zero_word, zero_words, \
+                                                zero_count, nullptr, nullptr, stream);                         \
         return radii ? launch_scan_g<G, true>(g, qq, ss, block_table, seq_lens, scores, zero_word, zero_words, \
                                               zero_count, radii, rad_logical, stream)                          \
                      : launch_scan_g<G, false>(g, qq, ss, block_table, seq_lens, scores, zero_word, zero_words, \
                                                zero_count, nullptr, nullptr, stream);
+    if (g.head_dim != kHeadDim && radii) return cudaErrorInvalidValue;   // (refused by the entry points)
     switch (g.group) {
         VSA_SCAN_CASE(1)
         VSA_SCAN_CASE(2)

@@ -19,7 +19,7 @@ size_t sparse_smem_bytes(const Geometry& g, int P, int K_c, bool fused, int thre
     if (solve)
         return (size_t)solve_tile_offset_words(g.max_pages, P, PT, K_c, fused, staged) * 4 +
                (size_t)solve_tile_rows(K_c) * kRowBytes + 16;
-    size_t words = (size_t)bt_stage_offset_words(g.max_pages, P, PT, K_c, fused);
+    size_t words = (size_t)bt_stage_offset_words(g.max_pages, P, PT, K_c, fused, g.head_dim);
     if (staged) words += (size_t)g.max_pages;
     return words * 4 + 16;
 }
@@ -108,6 +108,10 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
     a.fallback_list = fallback_list;
     a.fallback_count = fallback_count;
     a.stream = stream;
+    if (g.head_dim != kHeadDim) {
+        if (solve || cert || tl_summaries) return cudaErrorInvalidValue;   // (refused by the entry points)
+        return g.head_dim == 64 ? launch_sparse_plain_d64(a, threads) : launch_sparse_plain_d256(a, threads);
+    }
     if (tl_summaries) return (solve || cert || !page_scores) ? cudaErrorInvalidValue : launch_sparse_two_level(a, threads);
     if (solve) return launch_sparse_solve(a);
     if (cert) return page_scores ? launch_sparse_cert(a, threads) : cudaErrorInvalidValue;

@@ -23,16 +23,17 @@ namespace {
 constexpr int kMaxSparseWarps = 16;
 
 // token-phase shared memory, in 4-byte words, after the two tile arrays (PT = routed tiles of 16 tokens)
-__host__ __device__ constexpr int token_phase_words(int PT, int K_c)
+__host__ __device__ constexpr int token_phase_words(int PT, int K_c, int D = kHeadDim)
 {
     return PT * 16 /*keys*/ + (PT * 16 + 3) / 4 /*take*/ + 2 * K_c + 2 /*voff*/ + K_c /*wgt*/ +
-           K_c /*score*/ + 256 + 16 + 72 + kTopkList + kMaxSparseWarps * kHeadDim + kMaxSparseWarps + 4;
+           K_c /*score*/ + 256 + 16 + 72 + kTopkList + kMaxSparseWarps * D + kMaxSparseWarps + 4;
 }
 
 // first word of the block-table copy: after the two tile arrays and the larger of the two phases
-__host__ __device__ inline int bt_stage_offset_words(int max_pages, int P, int PT, int K_c, bool fused)
+__host__ __device__ inline int bt_stage_offset_words(int max_pages, int P, int PT, int K_c, bool fused,
+                                                     int D = kHeadDim)
 {
-    int words = token_phase_words(PT, K_c);
+    int words = token_phase_words(PT, K_c, D);
     if (fused && select_pages_words(max_pages, P) > words) words = select_pages_words(max_pages, P);
     return 2 * PT + words;
 }
@@ -69,11 +70,11 @@ struct TokenSmem {
     float* wgt;       // [K_c] unnormalised softmax weight of each candidate
     float* score;     // [K_c] score of each candidate (read by the iterative solve only)
     TopkScratch ts;
-    float* red;       // [warps][128]
+    float* red;       // [warps][D]
     float* zred;      // [warps]
 };
 
-__device__ __forceinline__ TokenSmem carve_tokens(uint32_t* base, int PT, int K_c)
+__device__ __forceinline__ TokenSmem carve_tokens(uint32_t* base, int PT, int K_c, int D = kHeadDim)
 {
     TokenSmem s;
     const int N = PT * 16;
@@ -89,13 +90,14 @@ __device__ __forceinline__ TokenSmem carve_tokens(uint32_t* base, int PT, int K_
     s.ts.wred = s.ts.misc + 16;
     s.ts.list = (int32_t*)(s.ts.wred + 72);
     s.red = (float*)(s.ts.list + kTopkList);
-    s.zred = s.red + kMaxSparseWarps * kHeadDim;
+    s.zred = s.red + kMaxSparseWarps * D;
     return s;
 }
 
-__device__ __forceinline__ void write_failed_unit(float* out, vsa_diag_t* diag, long long unit, int status)
+__device__ __forceinline__ void write_failed_unit(float* out, vsa_diag_t* diag, long long unit, int status,
+                                                  int D = kHeadDim)
 {
-    if (threadIdx.x < kHeadDim) out[unit * kHeadDim + threadIdx.x] = 0.0f;
+    for (int e = threadIdx.x; e < D; e += blockDim.x) out[unit * D + e] = 0.0f;
     if (threadIdx.x == 0) {
         vsa_diag_t d;
         d.delta = d.delta12 = d.s_max = d.lse = d.leak_bound = 0.0f;
@@ -125,7 +127,11 @@ __device__ __forceinline__ void write_failed_unit(float* out, vsa_diag_t* diag, 
 // CERT (fused register variants only): the certified gap of the unit - an upper bound on every score
 //   of the pages that were not routed, from the pages' radii (rad_logical, written by the scan) -
 //   is computed, reported in cert[] and used for the fallback decision in place of the proxy gap.
-template <int THREADS, int PAGE_KPT, int TOK_KPT, int SOLVE = 0, bool CERT = false>
+// D: head dimension.  A row is spread over the 16 lanes of a half-warp in pieces of 8 elements: lane c holds
+//   elements 8c .. 8c+7 and, at D = 256, 128 + 8c .. 128 + 8c + 7 as well (its partial is the sum of the two
+//   pieces' partials: the first level of the 32-partial tree); at D = 64 only lanes 0 .. 7 hold data, the
+//   others contribute +0.  Iterative solves, certificate and the two-level front end exist at D = 128 only.
+template <int THREADS, int PAGE_KPT, int TOK_KPT, int SOLVE = 0, bool CERT = false, int D = kHeadDim>
 __global__ void __launch_bounds__(THREADS, 512 / THREADS)
 sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* __restrict__ k_cache,
                      const uint16_t* __restrict__ v_cache, const int32_t* __restrict__ block_table,
@@ -140,6 +146,8 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
 {
     constexpr int WARPS = THREADS / 32, GROUPS = 2 * WARPS;
     static_assert(PAGE_KPT != -2 || (SOLVE == 0 && !CERT), "two-level front end: plain family only");
+    static_assert(D == 128 || ((D == 64 || D == 256) && SOLVE == 0 && !CERT && PAGE_KPT != -2), "other head dimensions: plain family");
+    constexpr int PIECES = D == 256 ? 2 : 1;
     static_assert(SOLVE == 0 || THREADS == 256, "the solve maps one candidate to each of 256 lanes");
     static_assert(!CERT || PAGE_KPT > 0, "the certificate needs every page score of the unit in registers");
     static_assert(TOK_KPT * WARPS <= 64 && 4 * WARPS <= 72, "wred capacity");
@@ -172,8 +180,10 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     // sequence length, asked for before it, has arrived by then).
     const int32_t* bt = block_table + (long long)b * geo.max_pages;
     const int T = ld_ca_s32(seq_lens + b);
-    const uint4 qraw = ld_nc_16B(q + unit * kHeadDim + c * 8);
-    int32_t* bt_s = (int32_t*)(smem_raw + bt_stage_offset_words(geo.max_pages, P, PT, K_c, PAGE_KPT > 0));
+    const bool lane_has = D != 64 || c < 8;   // this lane holds a piece of every row
+    const uint4 qraw = lane_has ? ld_nc_16B(q + unit * D + c * 8) : make_uint4(0u, 0u, 0u, 0u);
+    const uint4 qraw1 = PIECES == 2 ? ld_nc_16B(q + unit * D + 128 + c * 8) : make_uint4(0u, 0u, 0u, 0u);
+    int32_t* bt_s = (int32_t*)(smem_raw + bt_stage_offset_words(geo.max_pages, P, PT, K_c, PAGE_KPT > 0, D));
     if constexpr (PAGE_KPT > 0) {
         const uint32_t dst = (uint32_t)__cvta_generic_to_shared(bt_s);
         for (int i = tid; i < geo.max_pages; i += THREADS) cp_async_4(dst + 4u * (uint32_t)i, bt + i);
@@ -204,7 +214,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     }
     if (!geo.length_ok(T)) {
         cp_async_wait_all();
-        write_failed_unit(out, diag, unit, VSA_UNIT_BAD_LENGTH);
+        write_failed_unit(out, diag, unit, VSA_UNIT_BAD_LENGTH, D);
         if (SOLVE && tid == 0) solve[unit] = vsa_solve_t{0.0f, 0.0f, 0.0f, 0.0f};
         if (CERT && tid == 0) cert[unit] = vsa_cert_t{0.0f, 0.0f, 0.0f, 0};
         if (PAGE_KPT != 0)
@@ -371,12 +381,12 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         __syncthreads();   // the selection scratch is rewritten by the token phase
     }
     if (any_bad) {
-        write_failed_unit(out, diag, unit, VSA_UNIT_BAD_PAGE);
+        write_failed_unit(out, diag, unit, VSA_UNIT_BAD_PAGE, D);
         if (SOLVE && tid == 0) solve[unit] = vsa_solve_t{0.0f, 0.0f, 0.0f, 0.0f};
         if (CERT && tid == 0) cert[unit] = vsa_cert_t{0.0f, 0.0f, 0.0f, 0};
         return;
     }
-    const TokenSmem sm = carve_tokens(region, PT, K_c);
+    const TokenSmem sm = carve_tokens(region, PT, K_c, D);
     const int nt = np << tsh;   // tiles of the routed pages
 #pragma unroll
     for (int j = 0; j < TOK_KPT; ++j)
@@ -386,26 +396,32 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
     // ---- token routing: score all 16 tokens of a page per half-warp ----
     float qf[8];
     unpack8(qraw, qf);
+    float qf1[8];
+    unpack8(qraw1, qf1);
     for (int pp = warp; pp * 2 < nt; pp += WARPS) {
         const int slot = pp * 2 + gi;
         const bool active = slot < nt;
-        uint4 rows[16];
-        if (active) {
-            const uint16_t* src = k_cache + (long long)page_phys[slot] * geo.page_stride +
-                                  (long long)g * geo.head_stride + c * 8 +
-                                  (long long)((page_l[slot] & ((1 << tsh) - 1)) * 16) * geo.token_stride;
-#pragma unroll
-            for (int t = 0; t < 16; ++t) rows[t] = ld_nc_16B(src + (long long)t * geo.token_stride);
-        } else {
-#pragma unroll
-            for (int t = 0; t < 16; ++t) rows[t] = make_uint4(0u, 0u, 0u, 0u);
-        }
         float vals[16];
 #pragma unroll
-        for (int t = 0; t < 16; ++t) {
-            float kf[8];
-            unpack8(rows[t], kf);
-            vals[t] = chunk_partial(qf, kf);
+        for (int pc = 0; pc < PIECES; ++pc) {
+            uint4 rows[16];
+            if (active && lane_has) {
+                const uint16_t* src = k_cache + (long long)page_phys[slot] * geo.page_stride +
+                                      (long long)g * geo.head_stride + c * 8 + pc * 128 +
+                                      (long long)((page_l[slot] & ((1 << tsh) - 1)) * 16) * geo.token_stride;
+#pragma unroll
+                for (int t = 0; t < 16; ++t) rows[t] = ld_nc_16B(src + (long long)t * geo.token_stride);
+            } else {
+#pragma unroll
+                for (int t = 0; t < 16; ++t) rows[t] = make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int t = 0; t < 16; ++t) {
+                float kf[8];
+                unpack8(rows[t], kf);
+                const float part = chunk_partial(pc == 0 ? qf : qf1, kf);
+                vals[t] = pc == 0 ? part : vals[t] + part;
+            }
         }
         const float s = reduce_scatter16(vals, c);   // lane c: score of token c of the page
         if (active && page_l[slot] * 16 + c < T) sm.keys[slot * 16 + c] = float_to_key(s);
@@ -793,49 +809,60 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         }
     }
     // ---- value gather ----
-    float acc[8], z = 0.0f;
+    float acc[PIECES][8], z = 0.0f;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) acc[e] = 0.0f;
+    for (int pc = 0; pc < PIECES; ++pc)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[pc][e] = 0.0f;
     const int gidx = warp * 2 + gi;
-    const uint16_t* vbase = v_cache + (long long)g * geo.head_stride + c * 8;
     constexpr int UNR = THREADS == 512 ? 8 : 16;   // 256 threads, K_c = 256: every half-warp's rows in one batch
-    for (int j0 = gidx; j0 < ns; j0 += GROUPS * UNR) {
-        // all value rows of the batch at once; slots past the candidate count re-read the last
-        // candidate with weight 0
-        uint4 rows[UNR];
-        float w[UNR];
 #pragma unroll
-        for (int u = 0; u < UNR; ++u) {
-            const int j = j0 + u * GROUPS, jc = min(j, ns - 1);
-            rows[u] = ld_nc_16B(vbase + sm.voff[jc]);
-            w[u] = j < ns ? sm.wgt[jc] : 0.0f;
-        }
+    for (int pc = 0; pc < PIECES; ++pc) {
+        const uint16_t* vbase = v_cache + (long long)g * geo.head_stride + c * 8 + pc * 128;
+        for (int j0 = gidx; j0 < ns; j0 += GROUPS * UNR) {
+            // all value rows of the batch at once; slots past the candidate count re-read the last
+            // candidate with weight 0
+            uint4 rows[UNR];
+            float w[UNR];
 #pragma unroll
-        for (int u = 0; u < UNR; ++u) {
-            float vf[8];
-            unpack8(rows[u], vf);
+            for (int u = 0; u < UNR; ++u) {
+                const int j = j0 + u * GROUPS, jc = min(j, ns - 1);
+                rows[u] = lane_has ? ld_nc_16B(vbase + sm.voff[jc]) : make_uint4(0u, 0u, 0u, 0u);
+                w[u] = j < ns ? sm.wgt[jc] : 0.0f;
+            }
 #pragma unroll
-            for (int e = 0; e < 8; e += 2) fma2(acc[e], acc[e + 1], w[u], w[u], vf[e], vf[e + 1]);
-            z += w[u];
+            for (int u = 0; u < UNR; ++u) {
+                float vf[8];
+                unpack8(rows[u], vf);
+#pragma unroll
+                for (int e = 0; e < 8; e += 2) fma2(acc[pc][e], acc[pc][e + 1], w[u], w[u], vf[e], vf[e + 1]);
+                if (pc == 0) z += w[u];
+            }
         }
     }
 #pragma unroll
-    for (int e = 0; e < 8; ++e) acc[e] += __shfl_xor_sync(kFullMask, acc[e], 16);
+    for (int pc = 0; pc < PIECES; ++pc)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[pc][e] += __shfl_xor_sync(kFullMask, acc[pc][e], 16);
     z += __shfl_xor_sync(kFullMask, z, 16);
     if (gi == 0) {
+        if (lane_has) {
 #pragma unroll
-        for (int e = 0; e < 8; ++e) sm.red[warp * kHeadDim + c * 8 + e] = acc[e];
+            for (int pc = 0; pc < PIECES; ++pc)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) sm.red[warp * D + pc * 128 + c * 8 + e] = acc[pc][e];
+        }
         if (c == 0) sm.zred[warp] = z;
     }
     __syncthreads();
     float Z = 0.0f;
 #pragma unroll
     for (int w = 0; w < WARPS; ++w) Z += sm.zred[w];
-    if (tid < kHeadDim) {
+    for (int e = tid; e < D; e += THREADS) {
         float a = 0.0f;
 #pragma unroll
-        for (int w = 0; w < WARPS; ++w) a += sm.red[w * kHeadDim + tid];
-        out[unit * kHeadDim + tid] = ns > 0 ? a / Z : 0.0f;
+        for (int w = 0; w < WARPS; ++w) a += sm.red[w * D + e];
+        out[unit * D + e] = ns > 0 ? a / Z : 0.0f;
     }
 
     // ---- diagnostics and fallback flag ----
@@ -898,17 +925,17 @@ struct SparseArgs {
 
 namespace {
 
-template <int THREADS, int PAGE_KPT, int TOK_KPT, int SOLVE, bool CERT>
+template <int THREADS, int PAGE_KPT, int TOK_KPT, int SOLVE, bool CERT, int D = kHeadDim>
 cudaError_t launch_variant(const SparseArgs& a)
 {
     static bool attr_done[kMaxDevices] = {};   // per template instance
     if (a.smem > 48 * 1024) {
         const cudaError_t e =
-            allow_large_dynamic_smem(sparse_decode_kernel<THREADS, PAGE_KPT, TOK_KPT, SOLVE, CERT>, attr_done);
+            allow_large_dynamic_smem(sparse_decode_kernel<THREADS, PAGE_KPT, TOK_KPT, SOLVE, CERT, D>, attr_done);
         if (e != cudaSuccess) return e;
     }
     const unsigned units = (unsigned)(a.g.batch * a.g.n_q_heads);
-    return launch_pdl(sparse_decode_kernel<THREADS, PAGE_KPT, TOK_KPT, SOLVE, CERT>, dim3(units), dim3(THREADS),
+    return launch_pdl(sparse_decode_kernel<THREADS, PAGE_KPT, TOK_KPT, SOLVE, CERT, D>, dim3(units), dim3(THREADS),
                       a.smem, a.stream, a.g, a.q, a.k, a.v, a.block_table, a.seq_lens, a.routed_pages, a.page_scores,
                       a.P, a.K_c, a.epsilon, a.gap_threshold, a.out, a.diag, a.fallback_list, a.fallback_count,
                       a.solver_iters, a.solve, a.rad_logical, a.cert, a.unit_list, a.unit_count, a.routed_stride,
@@ -916,49 +943,52 @@ cudaError_t launch_variant(const SparseArgs& a)
 }
 
 // token-score registers per thread from the number of routed tokens
-template <int THREADS, int PAGE_KPT, int SOLVE, bool CERT>
+template <int THREADS, int PAGE_KPT, int SOLVE, bool CERT, int D = kHeadDim>
 cudaError_t launch_tok(const SparseArgs& a)
 {
     const int N = a.P * a.g.page_size;
-    if (N <= 2 * THREADS) return launch_variant<THREADS, PAGE_KPT, 2, SOLVE, CERT>(a);
-    if (N <= 4 * THREADS) return launch_variant<THREADS, PAGE_KPT, 4, SOLVE, CERT>(a);
+    if (N <= 2 * THREADS) return launch_variant<THREADS, PAGE_KPT, 2, SOLVE, CERT, D>(a);
+    if (N <= 4 * THREADS) return launch_variant<THREADS, PAGE_KPT, 4, SOLVE, CERT, D>(a);
     if constexpr (THREADS <= 256)
-        return N <= 8 * THREADS ? launch_variant<THREADS, PAGE_KPT, 8, SOLVE, CERT>(a) : cudaErrorInvalidValue;
+        return N <= 8 * THREADS ? launch_variant<THREADS, PAGE_KPT, 8, SOLVE, CERT, D>(a) : cudaErrorInvalidValue;
     else
         return cudaErrorInvalidValue;   // 128 pages * 16 tokens = 4 * 512: never reached
 }
 
 // page-score registers per thread from the block-table width (CERT: register variants only)
-template <int THREADS, int SOLVE, bool CERT>
+template <int THREADS, int SOLVE, bool CERT, int D = kHeadDim>
 cudaError_t launch_threads(const SparseArgs& a)
 {
     if constexpr (!CERT) {
-        if (!a.page_scores) return launch_tok<THREADS, 0, SOLVE, CERT>(a);
+        if (!a.page_scores) return launch_tok<THREADS, 0, SOLVE, CERT, D>(a);
     }
-    if (a.g.max_pages <= 8 * THREADS) return launch_tok<THREADS, 8, SOLVE, CERT>(a);
-    if (a.g.max_pages <= 16 * THREADS) return launch_tok<THREADS, 16, SOLVE, CERT>(a);
-    if (a.g.max_pages <= 32 * THREADS) return launch_tok<THREADS, 32, SOLVE, CERT>(a);
+    if (a.g.max_pages <= 8 * THREADS) return launch_tok<THREADS, 8, SOLVE, CERT, D>(a);
+    if (a.g.max_pages <= 16 * THREADS) return launch_tok<THREADS, 16, SOLVE, CERT, D>(a);
+    if (a.g.max_pages <= 32 * THREADS) return launch_tok<THREADS, 32, SOLVE, CERT, D>(a);
     if constexpr (!CERT)
-        return launch_tok<THREADS, -1, SOLVE, CERT>(a);
+        return launch_tok<THREADS, -1, SOLVE, CERT, D>(a);
     else
         return cudaErrorInvalidValue;   // (refused by the entry point before any launch)
 }
 
 // the 128-thread shape (P <= 64, the caller checks): routed pages given, or selected from scores held
 // in registers (max_pages <= 4096) or staged in shared memory (wider tables)
+template <int D = kHeadDim>
 inline cudaError_t launch_threads_128(const SparseArgs& a)
 {
-    if (!a.page_scores) return launch_tok<128, 0, 0, false>(a);
-    if (a.g.max_pages <= 8 * 128) return launch_tok<128, 8, 0, false>(a);
-    if (a.g.max_pages <= 16 * 128) return launch_tok<128, 16, 0, false>(a);
-    if (a.g.max_pages <= 32 * 128) return launch_tok<128, 32, 0, false>(a);
-    return launch_tok<128, -1, 0, false>(a);   // wider tables: selection staged in shared memory
+    if (!a.page_scores) return launch_tok<128, 0, 0, false, D>(a);
+    if (a.g.max_pages <= 8 * 128) return launch_tok<128, 8, 0, false, D>(a);
+    if (a.g.max_pages <= 16 * 128) return launch_tok<128, 16, 0, false, D>(a);
+    if (a.g.max_pages <= 32 * 128) return launch_tok<128, 32, 0, false, D>(a);
+    return launch_tok<128, -1, 0, false, D>(a);   // wider tables: selection staged in shared memory
 }
 
 }  // namespace
 
 // one family of kernel variants per translation unit
 cudaError_t launch_sparse_plain(const SparseArgs& a, int threads);   // closed-form weights
+cudaError_t launch_sparse_plain_d64(const SparseArgs& a, int threads);    // the same at head dimension 64
+cudaError_t launch_sparse_plain_d256(const SparseArgs& a, int threads);   // and 256
 cudaError_t launch_sparse_solve(const SparseArgs& a);                // iterative solves (256 threads)
 cudaError_t launch_sparse_cert(const SparseArgs& a, int threads);    // routing certificate
 cudaError_t launch_sparse_two_level(const SparseArgs& a, int threads);   // two-level front end

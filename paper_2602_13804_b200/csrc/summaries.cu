@@ -64,21 +64,22 @@ __device__ __forceinline__ float radius_of_rows(const uint4 (&rows)[PS], int n, 
     return __fadd_rn(__fmul_rn(__fsqrt_rn(d2), 1.001f), __fmul_rn(__fsqrt_rn(m2), 0x1p-12f));
 }
 
-// One thread per (logical page, kv head, 16-byte slice of the head dimension): the 16 threads of a
-// (page, head) read one contiguous 256-byte key row per iteration.  fp32 sum in ascending token
+// One thread per (logical page, kv head, 16-byte slice of the head dimension): the D / 8 threads of a
+// (page, head) read one contiguous key row per iteration.  fp32 sum in ascending token
 // order, IEEE division by the number of valid rows, round-to-nearest-even to bf16.
-template <int PS>
+template <int PS, int D>
 __global__ void __launch_bounds__(256) summaries_kernel(Geometry geo, const uint16_t* __restrict__ k_cache,
                                                         const int32_t* __restrict__ block_table,
                                                         const int32_t* __restrict__ seq_lens,
                                                         const int32_t* __restrict__ first_page,
                                                         uint16_t* __restrict__ summaries)
 {
+    constexpr int SL = D / 8;   // slices per row
     const int b = blockIdx.y;
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    const int c = (int)(idx & 15);
-    const int g = (int)((idx >> 4) % geo.n_kv_heads);
-    const long long l = (idx >> 4) / geo.n_kv_heads;
+    const int c = (int)(idx % SL);
+    const int g = (int)((idx / SL) % geo.n_kv_heads);
+    const long long l = (idx / SL) / geo.n_kv_heads;
     const int T = seq_lens[b];
     if (T <= 0 || T > geo.max_pages * PS) return;
     const int nb = (T + PS - 1) / PS;
@@ -93,7 +94,7 @@ __global__ void __launch_bounds__(256) summaries_kernel(Geometry geo, const uint
 #pragma unroll
     for (int t = 0; t < PS; ++t)
         if (t < n) rows[t] = ld_nc_16B(src + (long long)t * geo.token_stride);
-    *reinterpret_cast<uint4*>(summaries + (p * geo.n_kv_heads + g) * kHeadDim + c * 8) = mean_of_rows<PS>(rows, n);
+    *reinterpret_cast<uint4*>(summaries + (p * geo.n_kv_heads + g) * D + c * 8) = mean_of_rows<PS>(rows, n);
 }
 
 // Radius of each page around its stored summary (the ball bound of the routing certificate):
@@ -203,11 +204,13 @@ cudaError_t launch_build_summaries(const Geometry& g, const void* k_cache, const
                                    const int32_t* seq_lens, const int32_t* first_page, void* summaries,
                                    cudaStream_t stream)
 {
-    const long long threads = (long long)g.max_pages * g.n_kv_heads * 16;
+    const long long threads = (long long)g.max_pages * g.n_kv_heads * (g.head_dim / 8);
     dim3 grid((unsigned)((threads + 255) / 256), (unsigned)g.batch);
-    auto* kernel = g.page_size == 32 ? summaries_kernel<32> : summaries_kernel<16>;
+    auto* kernel = g.page_size == 32 ? summaries_kernel<32, 128> : summaries_kernel<16, 128>;
+    if (g.head_dim == 64) kernel = g.page_size == 32 ? summaries_kernel<32, 64> : summaries_kernel<16, 64>;
+    if (g.head_dim == 256) kernel = g.page_size == 32 ? summaries_kernel<32, 256> : summaries_kernel<16, 256>;
     kernel<<<grid, 256, 0, stream>>>(g, (const uint16_t*)k_cache, block_table, seq_lens, first_page,
-                                               (uint16_t*)summaries);
+                                     (uint16_t*)summaries);
     return cudaGetLastError();
 }
 

@@ -85,6 +85,8 @@ struct Geometry {
     // v >> tile_shift at row offset 16 * (v & ((1 << tile_shift) - 1)).
     int page_size = 16;
     int tile_shift = 0;
+    // Elements per head: 128, or 64 / 256 (closed-form step, routing, summaries and the dense pass only).
+    int head_dim = 128;
     // pages a sequence of T tokens occupies / whether T is a length the block table can hold
     __host__ __device__ int pages_of(int T) const { return (T + page_size - 1) >> (4 + tile_shift); }
     __host__ __device__ bool length_ok(int T) const { return T > 0 && T <= max_pages * page_size; }
