@@ -29,14 +29,17 @@
  *     than its block-table row, a non-positive length) never trap: the unit's
  *     diag.status becomes non-zero and its output row is zero-filled.
  *   - Inputs are assumed finite (no NaN/Inf in q, K, V).
- *   - v1 shapes: head_dim = 128, page_size = 16 or 32, n_q_heads / n_kv_heads in {1, 2, 4, 8, 16, 32}
+ *   - v1 shapes: head_dim = 128 (every entry point) or 64 / 256 (page summaries, routing, the closed-form
+ *     sparse pass, the dense pass and the steps built from them; the iterative solves, the certificate,
+ *     two-level and group-shared routing, vsa_build_page_radii and vsa_append_kv return
+ *     VSA_ERR_UNSUPPORTED_SHAPE), page_size = 16 or 32, n_q_heads / n_kv_heads in {1, 2, 4, 8, 16, 32}
  *     (multi-head, grouped-query and multi-query attention; groups of 16 and 32 query heads
  *     are processed as two and four sub-groups of 8 that read the same KV head),
  *     1 <= P <= 128 and P * page_size <= 2048 (the tokens scored per unit), 1 <= K_c <= P * page_size,
  *     max_pages_per_seq <= 32768,
  *     batch * n_kv_heads <= 4096 (batch * n_q_heads / 8 <= 4096 for groups above 8),
- *     num_pool_pages * n_kv_heads < 2^27 (the summary pool is addressed in 16-byte units by a
- *     32-bit offset).
+ *     num_pool_pages * n_kv_heads * head_dim < 2^34 (the summary pool is addressed in 16-byte units by a
+ *     32-bit offset: 2^27 rows at head_dim 128).
  *
  * Native layouts (row-major, last dimension contiguous)
  *   q            bf16 [batch][n_q_heads][head_dim]
@@ -56,7 +59,8 @@
  *   one fixed order: 16 chunks of 8 consecutive elements; inside a chunk the even elements'
  *   products and the odd elements' products are each summed left to right and the two sums
  *   added; then the 16 chunk sums are combined by a halving tree (p[c] += p[c+off],
- *   off = 8, 4, 2, 1).  Selections
+ *   off = 8, 4, 2, 1).  head_dim 256 has 32 chunk sums and one more level (off = 16 first); head_dim 64
+ *   has 8, padded with +0 to 16 for the same tree.  Selections
  *   order by (score descending, index ascending), -0 and +0 being equal.  Routed pages,
  *   candidate sets, Delta and the fallback flags are therefore reproducible bit for bit.
  *   Softmax weights and outputs use fp32 accumulation.
