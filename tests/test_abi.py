@@ -54,7 +54,7 @@ def test_workspace_sizes(lib):
     dense = B.vsa_workspace_bytes(s, 32, 256, B.VSA_WS_DENSE)
     assert dense > 0
     assert B.vsa_workspace_bytes(s, 32, 256, B.VSA_WS_STEP) >= route + dense
-    bad = B.make_shape(8, 32, 8, 2048, 65536, head_dim=64)
+    bad = B.make_shape(8, 32, 8, 2048, 65536, head_dim=96)
     assert B.vsa_workspace_bytes(bad, 32, 256, B.VSA_WS_STEP) == 0
     assert B.vsa_workspace_bytes(s, 32, 256, 77) == 0
 
@@ -76,7 +76,7 @@ def test_route_argument_validation(lib):
     assert _route(lib, ok, ws=None) == -1
     assert _route(lib, ok, P=0) == -1
     assert _route(lib, ok, P=129) == -2
-    assert _route(lib, B.make_shape(2, 8, 2, 64, 256, head_dim=64)) == -2
+    assert _route(lib, B.make_shape(2, 8, 2, 64, 256, head_dim=96)) == -2
     assert _route(lib, B.make_shape(2, 8, 2, 64, 256, page_size=64)) == -2
     assert _route(lib, B.make_shape(2, 6, 2, 64, 256)) == -2          # group of 3
     assert _route(lib, B.make_shape(2, 7, 2, 64, 256)) == -1          # heads do not divide
