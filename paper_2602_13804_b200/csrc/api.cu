@@ -339,7 +339,7 @@ int vsa_decode_step_two_level(const vsa_shape_t* shape, const void* q, const voi
         return VSA_ERR_CUDA;
     cudaError_t e = vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, routed_pages, super_scores, P,
                                        K_c, epsilon, gap_threshold, out, diag, fallback_list, fallback_count, st, 0,
-                                       nullptr, nullptr, nullptr, 1, nullptr, nullptr, 0, nullptr, summaries, P_super);
+                                       nullptr, nullptr, nullptr, 1, nullptr, nullptr, 0, summaries, P_super);
     if (e != cudaSuccess) return VSA_ERR_CUDA;
     return cuda_rc(vsa::launch_dense(g, q, k_cache, v_cache, block_table, seq_lens, fallback_list, fallback_count,
                                      epsilon, out, diag, ws_dense, st, /*tickets_cleared=*/true));

@@ -66,7 +66,7 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
                           vsa_diag_t* diag, int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream,
                           int solver_iters, vsa_solve_t* solve, const float* rad_logical, vsa_cert_t* cert,
                           int solver_kind, const int32_t* unit_list, const int32_t* unit_count, int routed_stride,
-                          const int32_t* page_budget, const void* tl_summaries, int P_super)
+                          const void* tl_summaries, int P_super)
 {
     SparseArgs a;
     a.g = g;
@@ -91,7 +91,6 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
     a.unit_list = unit_list;
     a.unit_count = unit_count;
     a.routed_stride = routed_stride > 0 ? routed_stride : P;
-    a.page_budget = page_budget;
     a.q = (const uint16_t*)q;
     a.k = (const uint16_t*)k_cache;
     a.v = (const uint16_t*)v_cache;

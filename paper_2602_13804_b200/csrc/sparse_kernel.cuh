@@ -141,7 +141,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                      int32_t* __restrict__ fallback_count, int solver_iters, vsa_solve_t* __restrict__ solve,
                      const float* __restrict__ rad_logical, vsa_cert_t* __restrict__ cert,
                      const int32_t* __restrict__ unit_list, const int32_t* __restrict__ unit_count,
-                     int routed_stride, const int32_t* __restrict__ page_budget,
+                     int routed_stride,
                      const uint16_t* __restrict__ tl_summaries, int P_super)
 {
     constexpr int WARPS = THREADS / 32, GROUPS = 2 * WARPS;
@@ -222,9 +222,6 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         return;
     }
     const int nb = geo.pages_of(T);
-    // page_budget (two-level routing): only that many of the unit's pages carry a score, the rest of the
-    // row is -inf and must not be routed
-    const int P_sel = (PAGE_KPT != 0 && page_budget) ? min(P, __ldcg(page_budget + unit)) : P;
 
     // ---- routed pages -> page_l[] sorted by logical page, so that array order = position order ----
     int np;
@@ -238,9 +235,9 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
             uint32_t pkey[PAGE_KPT];
 #pragma unroll
             for (int j = 0; j < PAGE_KPT; ++j)
-                pkey[j] = (tid + j * THREADS < nb && !(page_budget && praw[j] == -INFINITY)) ? float_to_key(praw[j]) : 0u;
+                pkey[j] = tid + j * THREADS < nb ? float_to_key(praw[j]) : 0u;
             cp_async_wait_all();   // this thread's part of the block-table copy; the selection's barriers publish it
-            np = select_top_pages_keys<PAGE_KPT>(pkey, nb, P_sel, ps);
+            np = select_top_pages_keys<PAGE_KPT>(pkey, nb, P, ps);
             if constexpr (CERT) {
                 // |q| (rounded up a little), every lane of a half-warp computing the same value
                 float qe[8];
@@ -265,7 +262,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                 if (lane == 0) ps.ts.wred[warp] = ub_key;   // published by the barrier below, read right after it
             }
         } else if constexpr (PAGE_KPT == -1) {
-            np = select_top_pages(page_scores + unit * geo.max_pages, nb, P_sel, ps, page_budget != nullptr);
+            np = select_top_pages(page_scores + unit * geo.max_pages, nb, P, ps);
         }
         // position -> logical page of a winner (two-level: position 16 j + c is page c of the j-th kept
         // super-page in ascending order)
@@ -916,7 +913,6 @@ struct SparseArgs {
     vsa_cert_t* cert;     // non-null: the certificate variant (fused register variants only)
     const int32_t *unit_list, *unit_count;   // non-null: only the listed units (blocks beyond the count exit)
     int routed_stride;                       // row stride of routed_pages (>= P)
-    const int32_t* page_budget;              // non-null (fused forms): scored pages per unit, see the kernel
     const uint16_t* tl_summaries;            // non-null: two-level front end (page_scores = representative scores)
     int P_super;
     cudaStream_t stream;
@@ -939,7 +935,7 @@ cudaError_t launch_variant(const SparseArgs& a)
                       a.smem, a.stream, a.g, a.q, a.k, a.v, a.block_table, a.seq_lens, a.routed_pages, a.page_scores,
                       a.P, a.K_c, a.epsilon, a.gap_threshold, a.out, a.diag, a.fallback_list, a.fallback_count,
                       a.solver_iters, a.solve, a.rad_logical, a.cert, a.unit_list, a.unit_count, a.routed_stride,
-                      a.page_budget, a.tl_summaries, a.P_super);
+                      a.tl_summaries, a.P_super);
 }
 
 // token-score registers per thread from the number of routed tokens

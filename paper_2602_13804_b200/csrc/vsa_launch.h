@@ -160,8 +160,7 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
                           int solver_iters = 0, vsa_solve_t* solve = nullptr, const float* rad_logical = nullptr,
                           vsa_cert_t* cert = nullptr, int solver_kind = 1, const int32_t* unit_list = nullptr,
                           const int32_t* unit_count = nullptr, int routed_stride = 0,
-                          const int32_t* page_budget = nullptr, const void* tl_summaries = nullptr,
-                          int P_super = 0);
+                          const void* tl_summaries = nullptr, int P_super = 0);
 // tl_summaries != nullptr: the two-level front end - page_scores then holds the scores of the super-pages'
 // representatives, fp32 [batch][n_q_heads][two_level_max_supers], and the kernel keeps the P_super best
 // super-pages, scores their pages from tl_summaries and routes the best P of those.
