@@ -469,6 +469,39 @@ int vsa_route_pages_static(const vsa_shape_t* shape, const void* q, const void* 
                            const int32_t* block_table, const int32_t* seq_lens, int32_t P,
                            int32_t* routed_pages, float* routed_scores, void* stream);
 
+/*
+ * Per-rank steps of the sequence-sharded (context-parallel) decode step.  One sequence's pages may be
+ * spread over several ranks: every rank passes a block table of the full width in which only the entries
+ * of the pages IT holds are valid (every other entry negative), and the global seq_lens.  Because page
+ * scores, token scores and the readout do not depend on where a page lives (Sec. 7), three small
+ * exchanges between the ranks reproduce the single-rank step:
+ *   1. every rank calls vsa_route_pages (pages it does not hold score -inf: drop them) and the local
+ *      top-P proposals are merged under the total order into the global routed pages;
+ *   2. vsa_cp_token_candidates scores the tokens of the globally routed pages the rank holds and returns
+ *      its best K_out = K_c + 1 of them; merged, the first K_c are the candidate set and the next one is
+ *      the best rejected token of the gap statistic;
+ *   3. vsa_cp_partial_readout forms the rank's softmax readout over its own members of the global
+ *      candidate set; the partial readouts combine with weights exp(lse_r - lse).
+ * The exchanges themselves are not part of this library's C ABI (paper_2602_13804_b200/context_parallel.py
+ * runs them over torch.distributed).  head_dim 128; page_size 16 or 32.
+ *   vsa_cp_token_candidates: q device bf16 [batch][n_q_heads][128]; routed_pages device int32
+ *     [batch][n_q_heads][P] (global logical pages, any order, -1 padded); 1 <= K_out <= P * page_size + 1;
+ *     cand_pos device int32 / cand_score device fp32 [batch][n_q_heads][K_out]: the rank's best tokens in
+ *     position order, (-1, -inf) padded.  Routed pages the rank does not hold are skipped, not an error.
+ *   vsa_cp_partial_readout: cand_pos / cand_score device [batch][n_q_heads][K_c]: the global candidate set
+ *     with its scores (-1 padded, the same on every rank); out_partial device fp32 [batch][n_q_heads][128]:
+ *     the readout over the rank's own members, normalised by their weight sum (zeros if it holds none);
+ *     lse_partial device fp32 [batch][n_q_heads]: log of their sum of exp(score / epsilon) (-inf if none).
+ * Units with an invalid length get empty lists / zero rows.  Nothing is allocated; both calls are
+ * asynchronous on `stream`.
+ */
+int vsa_cp_token_candidates(const vsa_shape_t* shape, const void* q, const void* k_cache,
+                            const int32_t* block_table, const int32_t* seq_lens, const int32_t* routed_pages,
+                            int32_t P, int32_t K_out, int32_t* cand_pos, float* cand_score, void* stream);
+int vsa_cp_partial_readout(const vsa_shape_t* shape, const void* v_cache, const int32_t* block_table,
+                           const int32_t* seq_lens, const int32_t* cand_pos, const float* cand_score,
+                           int32_t K_c, float epsilon, float* out_partial, float* lse_partial, void* stream);
+
 /* Scratch bytes needed by one call kind for this shape (0 if the shape is invalid). */
 size_t vsa_workspace_bytes(const vsa_shape_t* shape, int32_t P, int32_t K_c, int which_call);
 

@@ -68,6 +68,8 @@ def lib() -> C.CDLL:
         _lib.vsa_route_pages.argtypes = [shp, vp, vp, vp, vp, i32, vp, vp, vp, sz, vp]
         _lib.vsa_decode_step_group_shared.argtypes = [shp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, vp, vp, vp, vp,
                                                       vp, vp, sz, vp]
+        _lib.vsa_cp_token_candidates.argtypes = [shp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]
+        _lib.vsa_cp_partial_readout.argtypes = [shp, vp, vp, vp, vp, vp, i32, f32, vp, vp, vp]
         _lib.vsa_build_super_summaries.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp]
         _lib.vsa_route_pages_two_level.argtypes = [shp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, sz, vp]
         _lib.vsa_decode_step_two_level.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, f32, f32,
@@ -206,6 +208,22 @@ def vsa_decode_step_two_level(shape, q, summaries, super_summaries, k_cache, v_c
 
 
 VSA_STATIC_ROUTE_SCORES = 1 << 20
+
+
+def vsa_cp_token_candidates(shape, q, k_cache, block_table, seq_lens, routed_pages, P, K_out, cand_pos, cand_score,
+                            stream=None) -> None:
+    _check(lib().vsa_cp_token_candidates(C.byref(shape), _ptr(q), _ptr(k_cache), _ptr(block_table), _ptr(seq_lens),
+                                         _ptr(routed_pages), P, K_out, _ptr(cand_pos), _ptr(cand_score),
+                                         _stream(stream)),
+           "vsa_cp_token_candidates")
+
+
+def vsa_cp_partial_readout(shape, v_cache, block_table, seq_lens, cand_pos, cand_score, K_c, epsilon, out_partial,
+                           lse_partial, stream=None) -> None:
+    _check(lib().vsa_cp_partial_readout(C.byref(shape), _ptr(v_cache), _ptr(block_table), _ptr(seq_lens),
+                                        _ptr(cand_pos), _ptr(cand_score), K_c, epsilon, _ptr(out_partial),
+                                        _ptr(lse_partial), _stream(stream)),
+           "vsa_cp_partial_readout")
 
 
 def vsa_route_pages_static(shape, q, summaries, block_table, seq_lens, P, routed_pages, routed_scores,

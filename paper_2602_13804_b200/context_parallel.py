@@ -40,16 +40,14 @@ def _all_gather_cat(t: torch.Tensor, group=None) -> torch.Tensor:
     return torch.cat(parts, dim=-1)
 
 
-def merge_top(scores: torch.Tensor, index: torch.Tensor, k: int, group=None) -> Tuple[torch.Tensor, torch.Tensor]:
-    """Global top-k of the ranks' proposals under (score descending, index ascending).
+def merge_lists(s: torch.Tensor, i: torch.Tensor, k: int) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Top-k of concatenated proposals under (score descending, index ascending); no communication.
 
-    scores fp32 [..., n], index int32/int64 [..., n] (global page or token ids; -1 marks an unused slot,
-    whose score is ignored).  Every rank must propose at least its local top-k for the result to be the
-    top-k of the union.  Returns (scores [..., k], index [..., k]), unused slots (-inf, -1), identical on
-    every rank.
+    s fp32 [..., n], i int [..., n] (global page or token ids; -1 marks an unused slot, whose score is
+    ignored).  Returns (scores [..., k], index [..., k]), unused slots (-inf, -1).
     """
-    s = _all_gather_cat(scores.to(torch.float32), group)
-    i = _all_gather_cat(index.to(torch.int64), group)
+    s = s.to(torch.float32)
+    i = i.to(torch.int64)
     unused = i < 0
     s = s + 0.0                                   # -0 and +0 are one key
     s = torch.where(unused, torch.full_like(s, float("-inf")), s)
@@ -68,6 +66,29 @@ def merge_top(scores: torch.Tensor, index: torch.Tensor, k: int, group=None) -> 
     return torch.where(pad, torch.full_like(s2, float("-inf")), s2), torch.where(pad, torch.full_like(i2, -1), i2)
 
 
+def merge_top(scores: torch.Tensor, index: torch.Tensor, k: int, group=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Global top-k of the ranks' proposals under (score descending, index ascending).
+
+    scores fp32 [..., n], index int32/int64 [..., n] (global page or token ids; -1 marks an unused slot,
+    whose score is ignored).  Every rank must propose at least its local top-k for the result to be the
+    top-k of the union.  Returns (scores [..., k], index [..., k]), unused slots (-inf, -1), identical on
+    every rank.
+    """
+    s = _all_gather_cat(scores.to(torch.float32), group)
+    i = _all_gather_cat(index.to(torch.int64), group)
+    return merge_lists(s, i, k)
+
+
+def combine_lists(outs: torch.Tensor, lses: torch.Tensor) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Readout over the union from stacked partial readouts; no communication.
+    outs [R, ..., d], lses [R, ...] (-inf where a rank holds no token)."""
+    total = torch.logsumexp(lses, dim=0)
+    w = torch.exp(lses - total.unsqueeze(0))
+    w = torch.where(torch.isfinite(lses), w, torch.zeros_like(w))
+    O = torch.where(torch.isfinite(lses).unsqueeze(-1), outs, torch.zeros_like(outs))
+    return (w.unsqueeze(-1) * O).sum(dim=0), total
+
+
 def combine_partials(out: torch.Tensor, lse: torch.Tensor, group=None) -> Tuple[torch.Tensor, torch.Tensor]:
     """Readout over the union of the ranks' token sets from each rank's partial readout.
 
@@ -80,13 +101,7 @@ def combine_partials(out: torch.Tensor, lse: torch.Tensor, group=None) -> Tuple[
     lses = [torch.empty_like(lse) for _ in range(world)]
     dist.all_gather(outs, out.contiguous(), group=group)
     dist.all_gather(lses, lse.contiguous(), group=group)
-    L = torch.stack(lses, dim=0)
-    total = torch.logsumexp(L, dim=0)
-    w = torch.exp(L - total.unsqueeze(0))
-    w = torch.where(torch.isfinite(L), w, torch.zeros_like(w))
-    O = torch.stack(outs, dim=0)
-    O = torch.where(torch.isfinite(L).unsqueeze(-1), O, torch.zeros_like(O))
-    return (w.unsqueeze(-1) * O).sum(dim=0), total
+    return combine_lists(torch.stack(outs, dim=0), torch.stack(lses, dim=0))
 
 
 def gap_from_merged(scores: torch.Tensor, index: torch.Tensor, k_c: int) -> Tuple[torch.Tensor, torch.Tensor]:
@@ -98,3 +113,54 @@ def gap_from_merged(scores: torch.Tensor, index: torch.Tensor, k_c: int) -> Tupl
     rej = scores[..., k_c] if index.shape[-1] > k_c else torch.full_like(s1, float("-inf"))
     delta = torch.where(has_rejected, s1 - rej, torch.full_like(s1, float("inf")))
     return cand, delta
+
+
+class RankKernels:
+    """The per-rank GPU steps of the sequence-sharded decode step (one instance per rank and shape): thin
+    calls into the C ABI on this rank's shard.  `block_table` has the full width, with negative entries for
+    the pages other ranks hold; `seq_lens` are the global lengths."""
+
+    def __init__(self, shape, P: int, K_c: int, device):
+        from . import binding as B
+        self.B, self.shape, self.P, self.K_c, self.device = B, shape, P, K_c, device
+        bh = (shape.batch, shape.n_q_heads)
+        self.ws_route = B.alloc_workspace(shape, P, K_c, B.VSA_WS_ROUTE, device)
+        self.pages = torch.empty(bh + (P,), dtype=torch.int32, device=device)
+        self.page_scores = torch.empty(bh + (P,), dtype=torch.float32, device=device)
+        self.cand_pos = torch.empty(bh + (K_c + 1,), dtype=torch.int32, device=device)
+        self.cand_score = torch.empty(bh + (K_c + 1,), dtype=torch.float32, device=device)
+        self.out = torch.empty(bh + (shape.head_dim,), dtype=torch.float32, device=device)
+        self.lse = torch.empty(bh, dtype=torch.float32, device=device)
+
+    def propose_pages(self, q, summaries, block_table, seq_lens):
+        """local top-P (score, logical page); pages this rank does not hold (score -inf) are dropped"""
+        self.B.vsa_route_pages(self.shape, q, summaries, block_table, seq_lens, self.P, self.pages, self.page_scores,
+                               self.ws_route)
+        held = self.page_scores > float("-inf")
+        return self.page_scores, torch.where(held, self.pages, torch.full_like(self.pages, -1))
+
+    def propose_tokens(self, q, k_cache, block_table, seq_lens, routed_pages):
+        """local top-(K_c + 1) tokens (score, position) of the globally routed pages this rank holds"""
+        self.B.vsa_cp_token_candidates(self.shape, q, k_cache, block_table, seq_lens, routed_pages.to(torch.int32).contiguous(),
+                                       self.P, self.K_c + 1, self.cand_pos, self.cand_score)
+        return self.cand_score, self.cand_pos
+
+    def partial_readout(self, v_cache, block_table, seq_lens, cand_pos, cand_score, epsilon: float):
+        """(out, lse) over this rank's own members of the global candidate set"""
+        self.B.vsa_cp_partial_readout(self.shape, v_cache, block_table, seq_lens, cand_pos.to(torch.int32).contiguous(),
+                                      cand_score.to(torch.float32).contiguous(), self.K_c, epsilon, self.out, self.lse)
+        return self.out, self.lse
+
+
+def decode_step(rank: RankKernels, q, summaries, k_cache, v_cache, block_table, seq_lens, epsilon: float, group=None):
+    """The whole sequence-sharded step on one rank: three kernels, three exchanges.  Returns
+    (out [B, H, d], lse [B, H], delta [B, H], routed_pages [B, H, P], cand_pos [B, H, K_c]), identical on
+    every rank."""
+    ps, pi = rank.propose_pages(q, summaries, block_table, seq_lens)
+    _, routed = merge_top(ps, pi, rank.P, group)
+    ts, ti = rank.propose_tokens(q, k_cache, block_table, seq_lens, routed)
+    ms, mi = merge_top(ts, ti, rank.K_c + 1, group)
+    cand, delta = gap_from_merged(ms, mi, rank.K_c)
+    o, l = rank.partial_readout(v_cache, block_table, seq_lens, cand, ms[..., :rank.K_c], epsilon)
+    out, lse = combine_partials(o, l, group)
+    return out, lse, delta, routed, cand

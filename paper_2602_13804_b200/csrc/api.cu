@@ -773,3 +773,41 @@ extern "C" int vsa_route_pages_static(const vsa_shape_t* shape, const void* q, c
     if (e != cudaSuccess) return VSA_ERR_CUDA;
     return cuda_rc(vsa::launch_route_select(g, scratch, seq_lens, P, routed_pages, routed_scores, st));
 }
+
+extern "C" int vsa_cp_token_candidates(const vsa_shape_t* shape, const void* q, const void* k_cache,
+                                       const int32_t* block_table, const int32_t* seq_lens,
+                                       const int32_t* routed_pages, int32_t P, int32_t K_out, int32_t* cand_pos,
+                                       float* cand_score, void* stream)
+{
+    Geometry g;
+    int rc = make_geometry(shape, &g);
+    if (rc) return rc;
+    if (g.head_dim != vsa::kHeadDim) return VSA_ERR_UNSUPPORTED_SHAPE;
+    if ((rc = check_routing_sizes(g, P, 1, true))) return rc;
+    if (K_out < 1) return VSA_ERR_INVALID_ARGUMENT;
+    if (K_out > P * g.page_size + 1) return VSA_ERR_UNSUPPORTED_SHAPE;
+    if (!q || !k_cache || !block_table || !seq_lens || !routed_pages || !cand_pos || !cand_score)
+        return VSA_ERR_INVALID_ARGUMENT;
+    if (!aligned16(q) || !aligned16(k_cache)) return VSA_ERR_MISALIGNED;
+    return cuda_rc(vsa::launch_cp_token_candidates(g, q, k_cache, block_table, seq_lens, routed_pages, P, K_out,
+                                                   cand_pos, cand_score, (cudaStream_t)stream));
+}
+
+extern "C" int vsa_cp_partial_readout(const vsa_shape_t* shape, const void* v_cache, const int32_t* block_table,
+                                      const int32_t* seq_lens, const int32_t* cand_pos, const float* cand_score,
+                                      int32_t K_c, float epsilon, float* out_partial, float* lse_partial,
+                                      void* stream)
+{
+    Geometry g;
+    int rc = make_geometry(shape, &g);
+    if (rc) return rc;
+    if (g.head_dim != vsa::kHeadDim) return VSA_ERR_UNSUPPORTED_SHAPE;
+    if (K_c < 1) return VSA_ERR_INVALID_ARGUMENT;
+    if (K_c > kMaxP * 16) return VSA_ERR_UNSUPPORTED_SHAPE;
+    if ((rc = check_epsilon(epsilon))) return rc;
+    if (!v_cache || !block_table || !seq_lens || !cand_pos || !cand_score || !out_partial || !lse_partial)
+        return VSA_ERR_INVALID_ARGUMENT;
+    if (!aligned16(v_cache)) return VSA_ERR_MISALIGNED;
+    return cuda_rc(vsa::launch_cp_partial_readout(g, v_cache, block_table, seq_lens, cand_pos, cand_score, K_c,
+                                                  epsilon, out_partial, lse_partial, (cudaStream_t)stream));
+}

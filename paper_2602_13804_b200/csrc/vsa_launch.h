@@ -202,4 +202,14 @@ cudaError_t launch_dense(const Geometry& g, const void* q, const void* k_cache, 
 int32_t* dense_tickets(void* ws_dense);
 int dense_ticket_count(const Geometry& g);
 
+// ---- per-rank kernels of the context-parallel step (context_parallel.cu) ---------------------------
+cudaError_t launch_cp_token_candidates(const Geometry& g, const void* q, const void* k_cache,
+                                       const int32_t* block_table, const int32_t* seq_lens,
+                                       const int32_t* routed_pages, int P, int K_out, int32_t* cand_pos,
+                                       float* cand_score, cudaStream_t stream);
+cudaError_t launch_cp_partial_readout(const Geometry& g, const void* v_cache, const int32_t* block_table,
+                                      const int32_t* seq_lens, const int32_t* cand_pos, const float* cand_score,
+                                      int K_c, float epsilon, float* out_partial, float* lse_partial,
+                                      cudaStream_t stream);
+
 }  // namespace vsa

@@ -249,3 +249,30 @@ def test_multi_query_group_sizes_are_accepted(lib):
         s = B.make_shape(4, hq, hkv, 2048, 65536)
         assert B.vsa_workspace_bytes(s, 32, 256, B.VSA_WS_STEP) > 0
     assert B.vsa_workspace_bytes(B.make_shape(4, 48, 1, 2048, 65536), 32, 256, B.VSA_WS_STEP) == 0   # group of 48
+
+
+def test_context_parallel_and_head_dimension_argument_validation(lib):
+    s = B.make_shape(8, 32, 8, 2048, 65536)
+    sp = C.byref(s)
+
+    def cand(q=FAKE, P=32, K_out=257, pos=FAKE, shape=sp):
+        return lib.vsa_cp_token_candidates(shape, q, FAKE, FAKE, FAKE, FAKE, P, K_out, pos, FAKE, None)
+    assert cand(q=None) == -1 and cand(pos=None) == -1 and cand(K_out=0) == -1 and cand(P=0) == -1
+    assert cand(P=129) == -2 and cand(P=2, K_out=34) == -2 and cand(q=ODD) == -4
+
+    def readout(v=FAKE, K_c=256, eps=11.3, out=FAKE, shape=sp):
+        return lib.vsa_cp_partial_readout(shape, v, FAKE, FAKE, FAKE, FAKE, K_c, eps, out, FAKE, None)
+    assert readout(v=None) == -1 and readout(out=None) == -1 and readout(K_c=0) == -1 and readout(eps=0.0) == -1
+    assert readout(K_c=4096) == -2 and readout(v=ODD) == -4
+    # the sharded kernels and the variants beyond the closed-form step exist at head dimension 128 only
+    for d in (64, 256):
+        sd = B.make_shape(8, 32, 8, 2048, 65536, head_dim=d)
+        assert cand(shape=C.byref(sd)) == -2 and readout(shape=C.byref(sd)) == -2
+        assert lib.vsa_build_page_radii(C.byref(sd), FAKE, FAKE, FAKE, FAKE, None, FAKE, None) == -2
+        assert lib.vsa_append_kv(C.byref(sd), FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, None, None) == -2
+        assert lib.vsa_build_super_summaries(C.byref(sd), FAKE, FAKE, FAKE, None, FAKE, None, None) == -2
+        assert B.vsa_workspace_bytes(sd, 32, 256, B.VSA_WS_STEP) > 0
+    # 32-token pages: at most 64 routed pages (2048 scored tokens per unit)
+    s32 = B.make_shape(8, 32, 8, 2048, 65536, page_size=32)
+    assert lib.vsa_sparse_decode(C.byref(s32), FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, 65, 256, 11.3, 90.0, FAKE, FAKE, FAKE,
+                                 FAKE, None, 0, None) == -2
