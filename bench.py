@@ -921,6 +921,16 @@ def run_ours(args):
         roofline["frac_per_head_model"] = d["frac_per_head_model"]
     if "sparse_union_pages" in alg:
         roofline["union_pages"], roofline["union_rows"] = alg["sparse_union_pages"], alg["sparse_union_rows"]
+    # the second ceiling of a kernel that is not limited by bytes: warp instructions issued (one ncu capture,
+    # profiles/ncu_traffic.txt) against the SMs' issue slots, 4 schedulers per SM at the sampled SM clock
+    inst = ncu_traffic(dom + "_warp_instructions", spec.name)
+    if inst and clocks.get("sm_mhz"):
+        sms = torch.cuda.get_device_properties(dev).multi_processor_count
+        issue_peak = sms * 4 * clocks["sm_mhz"] * 1e6
+        roofline["issue_slots"] = {"warp_instructions_per_launch": inst, "peak_per_s": issue_peak,
+                                   "frac": inst / (d["us_per_launch"] * 1e-6) / issue_peak,
+                                   "note": "neither ceiling is approached: the kernel is a chain of dependent phases "
+                                           "(two exact selections, two dependent gathers) bound by latency"}
 
     sweep_obj = None
     default_run = (args.workload == "cfg1" and not args.dense_baseline and solve is None and cert is None
