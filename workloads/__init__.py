@@ -11,5 +11,6 @@ from .generator import (  # noqa: F401
     WorkloadSpec,
     config_spec,
     make_workload,
+    quantize_kv_fp8,
     seed_for,
 )

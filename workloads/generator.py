@@ -271,3 +271,33 @@ def make_workload(spec: WorkloadSpec, seed: Optional[int] = None, device="cpu",
         epsilon=eps, gap_threshold=tau,
         needle_positions=positions, needle_seq_ids=needle_seq_ids,
     )
+
+
+def quantize_kv_fp8(w: Workload):
+    """An fp8 copy of a workload's KV cache: e4m3 values with one power-of-two scale per (pool page, KV head).
+
+    For every (page, KV head) block of K (and of V) the exponent e is the smallest integer with
+    max|x| / 2^e <= 448 (the largest e4m3 value), the stored byte is round-to-nearest-even e4m3 of x / 2^e,
+    and the value it stands for is byte * 2^e.  Because the scale is a power of two, that value is exactly
+    representable in bf16, so the returned workload - whose bf16 caches hold exactly the values the fp8 cache
+    stands for - is what a reference for the fp8 path computes on.
+
+    Returns (workload with the dequantised bf16 caches, k8, v8, k_exp, v_exp): uint8 [pool, Hkv, page, d]
+    and int8 [pool, Hkv].
+    """
+    out = []
+    for x in (w.k_cache, w.v_cache):
+        xf = x.to(torch.float32)
+        amax = xf.abs().amax(dim=(2, 3))                                   # [pool, Hkv]
+        e = torch.ceil(torch.log2(torch.clamp(amax, min=1e-30) / 448.0))
+        e = torch.where(amax > 0, e, torch.zeros_like(e)).clamp(-100, 100)
+        # log2 can land one ulp low at exact powers of two: make sure the scaled block fits
+        e = torch.where(amax / torch.exp2(e) > 448.0, e + 1, e)
+        scale = torch.exp2(e)[:, :, None, None]
+        q8 = (xf / scale).to(torch.float8_e4m3fn)
+        deq = (q8.to(torch.float32) * scale).to(torch.bfloat16)
+        assert torch.equal(deq.to(torch.float32), q8.to(torch.float32) * scale)   # exact in bf16
+        out.append((q8.view(torch.uint8), e.to(torch.int8), deq))
+    (k8, ke, kd), (v8, ve, vd) = out
+    from dataclasses import replace as _replace
+    return _replace(w, k_cache=kd, v_cache=vd), k8, v8, ke, ve
