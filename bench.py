@@ -566,6 +566,52 @@ def two_level_point(spec, dev, P_super, steps):
             "us_per_layer_full_scan": res["full_scan"], "page_recall_vs_exact_routing": hit / max(tot, 1)}
 
 
+def fp8_point(spec, dev, steps):
+    """The step on an fp8 (e4m3, power-of-two scale per page and KV head) copy of the caches against the bf16
+    step on the bf16 caches that hold the same values (same routed pages, candidates and flags by construction)."""
+    from workloads import quantize_kv_fp8
+    h = Harness(spec, dev, mem_fraction=0.5)
+    torch, B, shape = h.torch, h.B, h.shape
+    k8s, v8s, kss, vss = [], [], [], []
+    for i, w in enumerate(h.layers):
+        wq, k8, v8, ke, ve = quantize_kv_fp8(w)
+        h.layers[i] = wq                        # the bf16 side runs on the dequantised values
+        k8s.append(k8); v8s.append(v8)
+        kss.append(torch.exp2(ke.float())); vss.append(torch.exp2(ve.float()))
+        B.vsa_build_page_summaries_fp8(shape, k8, kss[-1], wq.block_table, wq.seq_lens, None, h.summaries[i])
+    del w, wq
+    torch.cuda.synchronize()
+
+    def fp8_step():
+        for i in range(h.L):
+            k = i % h.distinct
+            w = h.layers[k]
+            B.vsa_decode_step_fp8(shape, w.q, h.summaries[k], k8s[k], v8s[k], kss[k], vss[k], w.block_table, w.seq_lens,
+                                  h.P, h.K_c, h.eps, h.tau, h.out, h.diag, h.routed, h.flist, h.fcount, h.ws_plain)
+    res = {}
+    with torch.cuda.stream(h.stream):
+        fp8_step()
+        h.stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=h.stream):
+            fp8_step()
+        for _ in range(3):
+            g.replay()
+    res["fp8"] = h.time_steps(g.replay, steps) / steps * 1e3 / h.L
+    fb8 = len(h.fallback_units()) / h.units
+    st = h.capture(True)
+    with torch.cuda.stream(h.stream):
+        for _ in range(3):
+            st()
+    res["bf16"] = h.time_steps(st, steps) / steps * 1e3 / h.L
+    fb16 = len(h.fallback_units()) / h.units
+    point = {"workload": spec.name, "layers": h.L, "distinct_layer_caches": h.distinct,
+             "us_per_layer_fp8": res["fp8"], "us_per_layer_bf16_same_values": res["bf16"],
+             "fallback_fraction_fp8": fb8, "fallback_fraction_bf16": fb16}
+    h.release()
+    return point
+
+
 def sweep(dev, steps_small=200):
     """The context sweep at batch 1 (flatness), one fallback-regime point and one large scan point."""
     from dataclasses import replace
@@ -591,6 +637,9 @@ def sweep(dev, steps_small=200):
     # other head dimensions: config 1's shape at d = 64 and d = 256 (temperature sqrt(d))
     out["head_dims"] = [measure_point(replace(c1, head_dim=d, epsilon=math.sqrt(d), layers=L, name=f"cfg1_d{d}"), dev, 100)
                         for d, L in ((64, 16), (256, 8))]
+    # fp8 KV cache against bf16 on the same values: config 1 (no fallback) and config 3's shape (75 % dense)
+    out["fp8"] = [fp8_point(replace(c1, layers=8, name="cfg1_8layers"), dev, 100),
+                  fp8_point(replace(config_spec(3), layers=2, name="cfg3_fallback_2layers"), dev, 20)]
     # group-shared routing (one selection per KV head) on config 1 and at batch 16
     gs = []
     for spec_g in (replace(config_spec(1), layers=16, name="cfg1_16layers"),

@@ -470,6 +470,38 @@ int vsa_route_pages_static(const vsa_shape_t* shape, const void* q, const void* 
                            int32_t* routed_pages, float* routed_scores, void* stream);
 
 /*
+ * fp8 KV cache (the paper's system sketch, Sec. 7, fixes no storage format; this is a deployment option of
+ * the library).  k_cache / v_cache hold e4m3 bytes (OCP e4m3fn, no NaN encodings expected) in the native
+ * layout [num_pool_pages][n_kv_heads][page_size][head_dim] with the shape's strides counted in BYTES (each
+ * a multiple of 16); k_scale / v_scale, device fp32 [num_pool_pages][n_kv_heads], give the value a byte
+ * stands for: value = e4m3(byte) * scale[page][kv head].  Summaries stay bf16, so routing is unchanged.
+ * Token scores are the fixed-order dot of q with the decoded bytes, multiplied by the page's key scale;
+ * the readout multiplies each candidate's weight by its page's value scale.  With POWER-OF-TWO scales every
+ * one of those multiplications is exact, and all results equal - discrete ones bit for bit - those of
+ * the bf16 entry points on a bf16 cache that holds the same values; with other scales the score carries
+ * one more rounding.  head_dim 128; page_size 16 or 32; closed-form weights only.  Otherwise the four entry
+ * points take the arguments, workspaces and error rules of the entry points they are named after.
+ */
+int vsa_build_page_summaries_fp8(const vsa_shape_t* shape, const void* k_cache, const float* k_scale,
+                                 const int32_t* block_table, const int32_t* seq_lens, const int32_t* first_page,
+                                 void* summaries, void* stream);
+int vsa_sparse_decode_fp8(const vsa_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,
+                          const float* k_scale, const float* v_scale, const int32_t* block_table,
+                          const int32_t* seq_lens, const int32_t* routed_pages, int32_t P, int32_t K_c, float epsilon,
+                          float gap_threshold, float* out, vsa_diag_t* diag, int32_t* fallback_list,
+                          int32_t* fallback_count, void* stream);
+int vsa_dense_decode_fallback_fp8(const vsa_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,
+                                  const float* k_scale, const float* v_scale, const int32_t* block_table,
+                                  const int32_t* seq_lens, const int32_t* fallback_list,
+                                  const int32_t* fallback_count, float epsilon, float* out, vsa_diag_t* diag,
+                                  void* ws, size_t ws_bytes, void* stream);
+int vsa_decode_step_fp8(const vsa_shape_t* shape, const void* q, const void* summaries, const void* k_cache,
+                        const void* v_cache, const float* k_scale, const float* v_scale, const int32_t* block_table,
+                        const int32_t* seq_lens, int32_t P, int32_t K_c, float epsilon, float gap_threshold,
+                        float* out, vsa_diag_t* diag, int32_t* routed_pages, int32_t* fallback_list,
+                        int32_t* fallback_count, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * Per-rank steps of the sequence-sharded (context-parallel) decode step.  One sequence's pages may be
  * spread over several ranks: every rank passes a block table of the full width in which only the entries
  * of the pages IT holds are valid (every other entry negative), and the global seq_lens.  Because page

@@ -76,6 +76,11 @@ def lib() -> C.CDLL:
                                                    vp, vp, vp, vp, vp, vp, sz, vp]
         _lib.vsa_route_pages_static.argtypes = [shp, vp, vp, vp, vp, i32, vp, vp, vp]
         _lib.vsa_route_pages_static.restype = C.c_int
+        _lib.vsa_build_page_summaries_fp8.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp]
+        _lib.vsa_sparse_decode_fp8.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, vp, vp, vp, vp, vp]
+        _lib.vsa_dense_decode_fallback_fp8.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, vp, vp, f32, vp, vp, vp, sz, vp]
+        _lib.vsa_decode_step_fp8.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, vp, vp, vp, vp, vp,
+                                             vp, sz, vp]
         _lib.vsa_sparse_decode.argtypes = [shp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, vp, vp, vp, vp, vp, sz, vp]
         _lib.vsa_dense_decode_fallback.argtypes = [shp, vp, vp, vp, vp, vp, vp, vp, f32, vp, vp, vp, sz, vp]
         _lib.vsa_decode_step.argtypes = [shp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -265,6 +270,43 @@ def vsa_decode_step(shape, q, summaries, k_cache, v_cache, block_table, seq_lens
                                  _ptr(diag), _ptr(routed_pages), _ptr(fallback_list), _ptr(fallback_count),
                                  _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
            "vsa_decode_step")
+
+
+# ---- fp8 (e4m3) KV cache: uint8 caches with fp32 scales [pool pages][n_kv_heads]; the shape's strides are bytes ----
+
+def vsa_build_page_summaries_fp8(shape, k_cache, k_scale, block_table, seq_lens, first_page, summaries,
+                                 stream=None) -> None:
+    _check(lib().vsa_build_page_summaries_fp8(C.byref(shape), _ptr(k_cache), _ptr(k_scale), _ptr(block_table),
+                                              _ptr(seq_lens), _ptr(first_page), _ptr(summaries), _stream(stream)),
+           "vsa_build_page_summaries_fp8")
+
+
+def vsa_sparse_decode_fp8(shape, q, k_cache, v_cache, k_scale, v_scale, block_table, seq_lens, routed_pages, P, K_c,
+                          epsilon, gap_threshold, out, diag, fallback_list, fallback_count, stream=None) -> None:
+    _check(lib().vsa_sparse_decode_fp8(C.byref(shape), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(k_scale),
+                                       _ptr(v_scale), _ptr(block_table), _ptr(seq_lens), _ptr(routed_pages), P, K_c,
+                                       epsilon, gap_threshold, _ptr(out), _ptr(diag), _ptr(fallback_list),
+                                       _ptr(fallback_count), _stream(stream)),
+           "vsa_sparse_decode_fp8")
+
+
+def vsa_dense_decode_fallback_fp8(shape, q, k_cache, v_cache, k_scale, v_scale, block_table, seq_lens, fallback_list,
+                                  fallback_count, epsilon, out, diag, ws, stream=None) -> None:
+    _check(lib().vsa_dense_decode_fallback_fp8(C.byref(shape), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(k_scale),
+                                               _ptr(v_scale), _ptr(block_table), _ptr(seq_lens), _ptr(fallback_list),
+                                               _ptr(fallback_count), epsilon, _ptr(out), _ptr(diag), _ptr(ws),
+                                               0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
+           "vsa_dense_decode_fallback_fp8")
+
+
+def vsa_decode_step_fp8(shape, q, summaries, k_cache, v_cache, k_scale, v_scale, block_table, seq_lens, P, K_c, epsilon,
+                        gap_threshold, out, diag, routed_pages, fallback_list, fallback_count, ws, stream=None) -> None:
+    _check(lib().vsa_decode_step_fp8(C.byref(shape), _ptr(q), _ptr(summaries), _ptr(k_cache), _ptr(v_cache),
+                                     _ptr(k_scale), _ptr(v_scale), _ptr(block_table), _ptr(seq_lens), P, K_c, epsilon,
+                                     gap_threshold, _ptr(out), _ptr(diag), _ptr(routed_pages), _ptr(fallback_list),
+                                     _ptr(fallback_count), _ptr(ws),
+                                     0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
+           "vsa_decode_step_fp8")
 
 
 def vsa_sparse_decode_entropic(shape, q, k_cache, v_cache, block_table, seq_lens, routed_pages, P, K_c, epsilon,

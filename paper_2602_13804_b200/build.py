@@ -11,7 +11,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libvsa.so")
-SOURCES = ["api.cu", "summaries.cu", "route.cu", "two_level.cu", "sparse.cu", "sparse_plain.cu", "sparse_plain_d64.cu", "sparse_plain_d256.cu", "sparse_solve.cu", "sparse_cert.cu", "sparse_two_level.cu", "sparse_shared_g12.cu", "sparse_shared_g4.cu", "sparse_shared_g8.cu",
+SOURCES = ["api.cu", "summaries.cu", "route.cu", "two_level.cu", "sparse.cu", "sparse_plain.cu", "sparse_plain_d64.cu", "sparse_plain_d256.cu", "sparse_plain_fp8.cu", "sparse_solve.cu", "sparse_cert.cu", "sparse_two_level.cu", "sparse_shared_g12.cu", "sparse_shared_g4.cu", "sparse_shared_g8.cu",
            "dense.cu", "context_parallel.cu"]
 HEADERS = ["vsa_device.cuh", "vsa_select.cuh", "sparse_kernel.cuh", "sparse_shared.cuh", "vsa_team.cuh", "vsa_launch.h", os.path.join("..", "..", "include", "vsa.h")]
 NVCC_FLAGS = [

@@ -82,6 +82,15 @@ int make_geometry(const vsa_shape_t* s, Geometry* g)
     return VSA_OK;
 }
 
+// an fp8 cache: head dimension 128, rows copied in 16-byte pieces (strides are in bytes there)
+int check_fp8_cache(const Geometry& g, const void* k_scale, const void* v_scale)
+{
+    if (!k_scale || !v_scale) return VSA_ERR_INVALID_ARGUMENT;
+    if (g.head_dim != vsa::kHeadDim) return VSA_ERR_UNSUPPORTED_SHAPE;
+    if ((g.token_stride % 16) || (g.head_stride % 16) || (g.page_stride % 16)) return VSA_ERR_MISALIGNED;
+    return VSA_OK;
+}
+
 int check_routing_sizes(const Geometry& g, int P, int K_c, bool need_kc)
 {
     if (P < 1) return VSA_ERR_INVALID_ARGUMENT;
@@ -209,6 +218,20 @@ int vsa_build_page_summaries(const vsa_shape_t* shape, const void* k_cache, cons
     if (!aligned16(k_cache) || !aligned16(summaries)) return VSA_ERR_MISALIGNED;
     return cuda_rc(vsa::launch_build_summaries(g, k_cache, block_table, seq_lens, first_page, summaries,
                                                (cudaStream_t)stream));
+}
+
+int vsa_build_page_summaries_fp8(const vsa_shape_t* shape, const void* k_cache, const float* k_scale,
+                                 const int32_t* block_table, const int32_t* seq_lens, const int32_t* first_page,
+                                 void* summaries, void* stream)
+{
+    Geometry g;
+    int rc = make_geometry(shape, &g);
+    if (rc) return rc;
+    if (!k_cache || !k_scale || !block_table || !seq_lens || !summaries) return VSA_ERR_INVALID_ARGUMENT;
+    if ((rc = check_fp8_cache(g, k_scale, k_scale))) return rc;
+    if (!aligned16(k_cache) || !aligned16(summaries)) return VSA_ERR_MISALIGNED;
+    return cuda_rc(vsa::launch_build_summaries_fp8(g, k_cache, k_scale, block_table, seq_lens, first_page, summaries,
+                                                   (cudaStream_t)stream));
 }
 
 int vsa_build_page_radii(const vsa_shape_t* shape, const void* k_cache, const void* summaries,
@@ -345,16 +368,16 @@ int vsa_decode_step_two_level(const vsa_shape_t* shape, const void* q, const voi
                                      epsilon, out, diag, ws_dense, st, /*tickets_cleared=*/true));
 }
 
-int vsa_sparse_decode(const vsa_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,
-                      const int32_t* block_table, const int32_t* seq_lens, const int32_t* routed_pages,
-                      int32_t P, int32_t K_c, float epsilon, float gap_threshold, float* out, vsa_diag_t* diag,
-                      int32_t* fallback_list, int32_t* fallback_count, void* ws, size_t ws_bytes, void* stream)
+static int sparse_decode_impl(const vsa_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,
+                              const float* k_scale, const float* v_scale, bool fp8, const int32_t* block_table,
+                              const int32_t* seq_lens, const int32_t* routed_pages, int32_t P, int32_t K_c,
+                              float epsilon, float gap_threshold, float* out, vsa_diag_t* diag, int32_t* fallback_list,
+                              int32_t* fallback_count, void* stream)
 {
-    (void)ws;
-    (void)ws_bytes;
     Geometry g;
     int rc = make_geometry(shape, &g);
     if (rc) return rc;
+    if (fp8 && (rc = check_fp8_cache(g, k_scale, v_scale))) return rc;
     if ((rc = check_routing_sizes(g, P, K_c, true))) return rc;
     if ((rc = check_epsilon(epsilon))) return rc;
     if (isnan(gap_threshold)) return VSA_ERR_INVALID_ARGUMENT;
@@ -366,7 +389,29 @@ int vsa_sparse_decode(const vsa_shape_t* shape, const void* q, const void* k_cac
     cudaError_t e = cudaMemsetAsync(fallback_count, 0, sizeof(int32_t), st);
     if (e != cudaSuccess) return VSA_ERR_CUDA;
     return cuda_rc(vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, (int32_t*)routed_pages, nullptr,
-                                      P, K_c, epsilon, gap_threshold, out, diag, fallback_list, fallback_count, st));
+                                      P, K_c, epsilon, gap_threshold, out, diag, fallback_list, fallback_count, st, 0,
+                                      nullptr, nullptr, nullptr, 1, nullptr, nullptr, 0, nullptr, 0, k_scale, v_scale));
+}
+
+int vsa_sparse_decode(const vsa_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,
+                      const int32_t* block_table, const int32_t* seq_lens, const int32_t* routed_pages,
+                      int32_t P, int32_t K_c, float epsilon, float gap_threshold, float* out, vsa_diag_t* diag,
+                      int32_t* fallback_list, int32_t* fallback_count, void* ws, size_t ws_bytes, void* stream)
+{
+    (void)ws;
+    (void)ws_bytes;
+    return sparse_decode_impl(shape, q, k_cache, v_cache, nullptr, nullptr, false, block_table, seq_lens, routed_pages,
+                              P, K_c, epsilon, gap_threshold, out, diag, fallback_list, fallback_count, stream);
+}
+
+int vsa_sparse_decode_fp8(const vsa_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,
+                          const float* k_scale, const float* v_scale, const int32_t* block_table,
+                          const int32_t* seq_lens, const int32_t* routed_pages, int32_t P, int32_t K_c, float epsilon,
+                          float gap_threshold, float* out, vsa_diag_t* diag, int32_t* fallback_list,
+                          int32_t* fallback_count, void* stream)
+{
+    return sparse_decode_impl(shape, q, k_cache, v_cache, k_scale, v_scale, true, block_table, seq_lens, routed_pages,
+                              P, K_c, epsilon, gap_threshold, out, diag, fallback_list, fallback_count, stream);
 }
 
 static int sparse_solver_impl(int solver_kind, const vsa_shape_t* shape, const void* q, const void* k_cache,
@@ -415,21 +460,41 @@ int vsa_sparse_decode_frank_wolfe(const vsa_shape_t* shape, const void* q, const
                               gap_threshold, solver_iters, out, diag, solve, fallback_list, fallback_count, stream);
 }
 
-int vsa_dense_decode_fallback(const vsa_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,
-                              const int32_t* block_table, const int32_t* seq_lens, const int32_t* fallback_list,
-                              const int32_t* fallback_count, float epsilon, float* out, vsa_diag_t* diag,
-                              void* ws, size_t ws_bytes, void* stream)
+static int dense_impl(const vsa_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,
+                      const float* k_scale, const float* v_scale, bool fp8, const int32_t* block_table,
+                      const int32_t* seq_lens, const int32_t* fallback_list, const int32_t* fallback_count,
+                      float epsilon, float* out, vsa_diag_t* diag, void* ws, size_t ws_bytes, void* stream)
 {
     Geometry g;
     int rc = make_geometry(shape, &g);
     if (rc) return rc;
+    if (fp8 && (rc = check_fp8_cache(g, k_scale, v_scale))) return rc;
     if ((rc = check_epsilon(epsilon))) return rc;
     if (!q || !k_cache || !v_cache || !block_table || !seq_lens || !out || !ws) return VSA_ERR_INVALID_ARGUMENT;
     if (fallback_count && !fallback_list) return VSA_ERR_INVALID_ARGUMENT;
     if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(ws)) return VSA_ERR_MISALIGNED;
     if (ws_bytes < vsa::dense_workspace_bytes(g)) return VSA_ERR_WORKSPACE_TOO_SMALL;
     return cuda_rc(vsa::launch_dense(g, q, k_cache, v_cache, block_table, seq_lens, fallback_list, fallback_count,
-                                     epsilon, out, diag, ws, (cudaStream_t)stream));
+                                     epsilon, out, diag, ws, (cudaStream_t)stream, false, k_scale, v_scale));
+}
+
+int vsa_dense_decode_fallback(const vsa_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,
+                              const int32_t* block_table, const int32_t* seq_lens, const int32_t* fallback_list,
+                              const int32_t* fallback_count, float epsilon, float* out, vsa_diag_t* diag,
+                              void* ws, size_t ws_bytes, void* stream)
+{
+    return dense_impl(shape, q, k_cache, v_cache, nullptr, nullptr, false, block_table, seq_lens, fallback_list,
+                      fallback_count, epsilon, out, diag, ws, ws_bytes, stream);
+}
+
+int vsa_dense_decode_fallback_fp8(const vsa_shape_t* shape, const void* q, const void* k_cache, const void* v_cache,
+                                  const float* k_scale, const float* v_scale, const int32_t* block_table,
+                                  const int32_t* seq_lens, const int32_t* fallback_list,
+                                  const int32_t* fallback_count, float epsilon, float* out, vsa_diag_t* diag,
+                                  void* ws, size_t ws_bytes, void* stream)
+{
+    return dense_impl(shape, q, k_cache, v_cache, k_scale, v_scale, true, block_table, seq_lens, fallback_list,
+                      fallback_count, epsilon, out, diag, ws, ws_bytes, stream);
 }
 
 static int decode_step_impl(const vsa_shape_t* shape, const void* q, const void* summaries, const void* k_cache,
@@ -438,11 +503,13 @@ static int decode_step_impl(const vsa_shape_t* shape, const void* q, const void*
                             int32_t* routed_pages, int32_t* fallback_list, int32_t* fallback_count, void* ws,
                             size_t ws_bytes, void* stream, void* const* events, int solver_iters = 0,
                             vsa_solve_t* solve = nullptr, const float* radii = nullptr, vsa_cert_t* cert = nullptr,
-                            int solver_kind = 1)
+                            int solver_kind = 1, bool fp8 = false, const float* k_scale = nullptr,
+                            const float* v_scale = nullptr)
 {
     Geometry g;
     int rc = make_geometry(shape, &g);
     if (rc) return rc;
+    if (fp8 && (rc = check_fp8_cache(g, k_scale, v_scale))) return rc;
     if (g.head_dim != vsa::kHeadDim && (solve || cert)) return VSA_ERR_UNSUPPORTED_SHAPE;   // closed form only
     if ((rc = check_routing_sizes(g, P, K_c, true))) return rc;
     if (solve && (rc = check_solver_sizes(K_c, solver_iters))) return rc;
@@ -483,11 +550,11 @@ static int decode_step_impl(const vsa_shape_t* shape, const void* q, const void*
     if (ev[2] && cudaEventRecord(ev[2], st) != cudaSuccess) return VSA_ERR_CUDA;
     e = vsa::launch_sparse(g, q, k_cache, v_cache, block_table, seq_lens, routed_pages, (const float*)ws, P, K_c,
                            epsilon, gap_threshold, out, diag, fallback_list, fallback_count, st, solver_iters, solve,
-                           rad_logical, cert, solver_kind);
+                           rad_logical, cert, solver_kind, nullptr, nullptr, 0, nullptr, 0, k_scale, v_scale);
     if (e != cudaSuccess) return VSA_ERR_CUDA;
     if (ev[3] && cudaEventRecord(ev[3], st) != cudaSuccess) return VSA_ERR_CUDA;
     e = vsa::launch_dense(g, q, k_cache, v_cache, block_table, seq_lens, fallback_list, fallback_count, epsilon,
-                          out, diag, ws_dense, st, /*tickets_cleared=*/true);
+                          out, diag, ws_dense, st, /*tickets_cleared=*/true, k_scale, v_scale);
     if (e != cudaSuccess) return VSA_ERR_CUDA;
     if (ev[4] && cudaEventRecord(ev[4], st) != cudaSuccess) return VSA_ERR_CUDA;
     return VSA_OK;
@@ -502,6 +569,17 @@ int vsa_decode_step(const vsa_shape_t* shape, const void* q, const void* summari
     return decode_step_impl(shape, q, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon,
                             gap_threshold, out, diag, routed_pages, fallback_list, fallback_count, ws, ws_bytes,
                             stream, nullptr);
+}
+
+int vsa_decode_step_fp8(const vsa_shape_t* shape, const void* q, const void* summaries, const void* k_cache,
+                        const void* v_cache, const float* k_scale, const float* v_scale, const int32_t* block_table,
+                        const int32_t* seq_lens, int32_t P, int32_t K_c, float epsilon, float gap_threshold,
+                        float* out, vsa_diag_t* diag, int32_t* routed_pages, int32_t* fallback_list,
+                        int32_t* fallback_count, void* ws, size_t ws_bytes, void* stream)
+{
+    return decode_step_impl(shape, q, summaries, k_cache, v_cache, block_table, seq_lens, P, K_c, epsilon,
+                            gap_threshold, out, diag, routed_pages, fallback_list, fallback_count, ws, ws_bytes,
+                            stream, nullptr, 0, nullptr, nullptr, nullptr, 1, true, k_scale, v_scale);
 }
 
 int vsa_decode_step_group_shared(const vsa_shape_t* shape, const void* q, const void* summaries, const void* k_cache,

@@ -32,14 +32,18 @@ constexpr int kMaxRoundsRagged = 8;
 // Sizes that depend on the head dimension D (64, 128 or 256).  The ring of a block holds three stages of a
 // K tile and a V tile per warp: 192 KB with eight warps at D = 128; D = 256 runs four warps per block so
 // that the same ring fits.
-template <int D>
+// FP8 (D = 128): a stage holds the raw e4m3 tiles (2 KB each, plus the two scales); each warp converts the
+// stage it is about to use into one bf16 working pair of tiles behind its stages.
+template <int D, bool FP8 = false>
 struct DenseCfg {
     static constexpr int kDenseThreads = D == 256 ? 128 : 256;
     static constexpr int kDenseWarps = kDenseThreads / 32;
     static constexpr int kRowBytes = 2 * D;
     static constexpr int kTileBytes = kTileRows * kRowBytes;   // K (or V) rows of one tile and KV head (4 KB at D = 128)
-    static constexpr int kStageBytes = 2 * kTileBytes;         // K tile + V tile
-    static constexpr int kRingBytes = kDenseWarps * kStages * kStageBytes;
+    static constexpr int kRawTileBytes = kTileRows * D;        // the same rows as e4m3 bytes
+    static constexpr int kStageBytes = FP8 ? 2 * kRawTileBytes + 16 : 2 * kTileBytes;   // K tile + V tile (+ scales)
+    static constexpr int kWarpBytes = kStages * kStageBytes + (FP8 ? 2 * kTileBytes : 0);
+    static constexpr int kRingBytes = kDenseWarps * kWarpBytes;
     static constexpr int kPartialFloats = 2 + D;               // per (item, head): max (log2 domain), sum, acc[D]
     static constexpr int kMinPagesPerItem = 2 * kDenseWarps;   // at least two pages per warp: one would expose the DRAM latency
 };
@@ -90,16 +94,17 @@ struct DenseSmem {
     int32_t* misc;         // [16]
 };
 
-template <int G, int D = vsa::kHeadDim>
+template <int G, int D = vsa::kHeadDim, bool FP8 = false>
 __global__ void __launch_bounds__(DenseCfg<D>::kDenseThreads, 1)
 dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* __restrict__ k_cache,
                    const uint16_t* __restrict__ v_cache, const int32_t* __restrict__ block_table,
                    const int32_t* __restrict__ seq_lens, const int32_t* __restrict__ fallback_list,
                    const int32_t* __restrict__ fallback_count, float epsilon, float* __restrict__ partials,
                    int32_t* __restrict__ counters, float* __restrict__ out, vsa_diag_t* __restrict__ diag,
-                   int max_items)
+                   int max_items, const float* __restrict__ k_scale, const float* __restrict__ v_scale)
 {
-    using Cfg = DenseCfg<D>;
+    static_assert(!FP8 || D == 128, "fp8 cache: head dimension 128");
+    using Cfg = DenseCfg<D, FP8>;
     constexpr int kDenseThreads = Cfg::kDenseThreads, kDenseWarps = Cfg::kDenseWarps, kRowBytes = Cfg::kRowBytes,
                   kTileBytes = Cfg::kTileBytes, kStageBytes = Cfg::kStageBytes, kRingBytes = Cfg::kRingBytes,
                   kPartialFloats = Cfg::kPartialFloats, kMinPagesPerItem = Cfg::kMinPagesPerItem, kHeadDim = D;
@@ -218,7 +223,7 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
     const float scale = 1.4426950408889634f / epsilon;   // scores are kept in the log2 domain
     const int head = lane >> 2;                          // MMA row of this lane = query head in the group
     const int quad = lane & 3;
-    uint8_t* my_ring = sm.ring + warp * kStages * kStageBytes;
+    uint8_t* my_ring = sm.ring + warp * Cfg::kWarpBytes;
     const uint32_t ring_addr = (uint32_t)__cvta_generic_to_shared(my_ring);
     // copy mapping: lane covers 16-byte chunk lane % CPR of rows lane / CPR + RPI i, i = 0 .. 16 / RPI - 1
     const int cp_chunk = lane % CPR, cp_row0 = lane / CPR;
@@ -273,9 +278,29 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
             const int valid_rows = page_ok ? min(kTileRows, T - pl * kTileRows) : 0;
             const long long head_off = (long long)(g / geo.kv_div) * geo.head_stride + cp_chunk * 8 +
                                        (long long)((pl & ((1 << geo.tile_shift) - 1)) * kTileRows) * geo.token_stride;
+            const uint32_t dst = ring_addr + (uint32_t)((k % kStages) * kStageBytes);
+            if constexpr (FP8) {
+                // raw rows of 128 bytes: lane covers 16-byte chunk lane % 8 of rows lane / 8 + 4 i
+                const int ch = lane & 7, r0 = lane >> 3;
+                const long long off8 = phys * geo.page_stride + (long long)(g / geo.kv_div) * geo.head_stride + ch * 16 +
+                                       (long long)((pl & ((1 << geo.tile_shift) - 1)) * kTileRows) * geo.token_stride;
+                const uint8_t* kp = reinterpret_cast<const uint8_t*>(k_cache) + off8;
+                const uint8_t* vp = reinterpret_cast<const uint8_t*>(v_cache) + off8;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int r = r0 + 4 * i;
+                    const uint32_t off = (uint32_t)(r * 128 + ch * 16);
+                    const bool ok = r < valid_rows;
+                    cp_async_16_zfill(dst + off, kp + (long long)r * geo.token_stride, ok);
+                    cp_async_16_zfill(dst + Cfg::kRawTileBytes + off, vp + (long long)r * geo.token_stride, ok);
+                }
+                if (lane < 2) {   // the tile's two scales ride the same stage
+                    const float* sp = (lane == 0 ? k_scale : v_scale) + phys * geo.kv_heads_stored + g / geo.kv_div;
+                    cp_async_4(dst + 2 * Cfg::kRawTileBytes + 4 * lane, sp);
+                }
+            } else {
             const uint16_t* kp = k_cache + phys * geo.page_stride + head_off;
             const uint16_t* vp = v_cache + phys * geo.page_stride + head_off;
-            const uint32_t dst = ring_addr + (uint32_t)((k % kStages) * kStageBytes);
 #pragma unroll
             for (int i = 0; i < kTileRows / RPI; ++i) {
                 const int r = cp_row0 + RPI * i;
@@ -283,6 +308,7 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
                 const bool ok = r < valid_rows;
                 cp_async_16_zfill(dst + off, kp + (long long)r * geo.token_stride, ok);
                 cp_async_16_zfill(dst + kTileBytes + off, vp + (long long)r * geo.token_stride, ok);
+            }
             }
         };
 #pragma unroll
@@ -305,8 +331,36 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
                     continue;
                 }
             }
-            const uint32_t kbase = ring_addr + (uint32_t)((k % kStages) * kStageBytes);
-            const uint32_t vbase = kbase + kTileBytes;
+            uint32_t kbase = ring_addr + (uint32_t)((k % kStages) * kStageBytes);
+            uint32_t vbase = kbase + kTileBytes;
+            float kscale = 1.0f, vscale = 1.0f;
+            if constexpr (FP8) {
+                // e4m3 -> bf16 (exact) into the warp's working pair of tiles, in the swizzled layout ldmatrix reads
+                const uint8_t* raw = my_ring + (k % kStages) * kStageBytes;
+                uint8_t* work = my_ring + kStages * kStageBytes;
+                kscale = *reinterpret_cast<const float*>(raw + 2 * Cfg::kRawTileBytes);
+                vscale = *reinterpret_cast<const float*>(raw + 2 * Cfg::kRawTileBytes + 4);
+                const int ch = lane & 7, r0 = lane >> 3;
+#pragma unroll
+                for (int kv = 0; kv < 2; ++kv) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int r = r0 + 4 * i;
+                        const uint4 in = *reinterpret_cast<const uint4*>(raw + kv * Cfg::kRawTileBytes + r * 128 + ch * 16);
+                        uint4 o0, o1;
+                        e4m3x4_to_bf16x2x2(in.x, o0.x, o0.y);
+                        e4m3x4_to_bf16x2x2(in.y, o0.z, o0.w);
+                        e4m3x4_to_bf16x2x2(in.z, o1.x, o1.y);
+                        e4m3x4_to_bf16x2x2(in.w, o1.z, o1.w);
+                        uint8_t* row = work + kv * kTileBytes + r * kRowBytes;
+                        *reinterpret_cast<uint4*>(row + (((2 * ch) ^ (r & 7)) << 4)) = o0;
+                        *reinterpret_cast<uint4*>(row + (((2 * ch + 1) ^ (r & 7)) << 4)) = o1;
+                    }
+                }
+                __syncwarp();
+                kbase = ring_addr + (uint32_t)(kStages * kStageBytes);
+                vbase = kbase + kTileBytes;
+            }
 
             // S = Q K^T for the 16 tokens of the page (two 8-token column tiles)
             float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
@@ -322,11 +376,12 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
                 }
             }
             // this lane: head `head`, tokens 2 quad, 2 quad + 1 (tile 0) and 8 + the same (tile 1)
+            const float tscale = FP8 ? scale * kscale : scale;   // fp8: the page's key scale folded in
             float t[4];
-            t[0] = (2 * quad < valid) ? s0[0] * scale : -INFINITY;
-            t[1] = (2 * quad + 1 < valid) ? s0[1] * scale : -INFINITY;
-            t[2] = (8 + 2 * quad < valid) ? s1[0] * scale : -INFINITY;
-            t[3] = (8 + 2 * quad + 1 < valid) ? s1[1] * scale : -INFINITY;
+            t[0] = (2 * quad < valid) ? s0[0] * tscale : -INFINITY;
+            t[1] = (2 * quad + 1 < valid) ? s0[1] * tscale : -INFINITY;
+            t[2] = (8 + 2 * quad < valid) ? s1[0] * tscale : -INFINITY;
+            t[3] = (8 + 2 * quad + 1 < valid) ? s1[1] * tscale : -INFINITY;
             float pm = fmaxf(fmaxf(t[0], t[1]), fmaxf(t[2], t[3]));
             pm = fmaxf(pm, __shfl_xor_sync(kFullMask, pm, 1));
             pm = fmaxf(pm, __shfl_xor_sync(kFullMask, pm, 2));
@@ -344,7 +399,8 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
                 }
             }
             m_run = m_new;
-            const uint32_t pa0 = pack_bf16x2(p[0], p[1]), pa2 = pack_bf16x2(p[2], p[3]);
+            // fp8: the page's value scale rides on the probabilities (the running sum keeps the unscaled ones)
+            const uint32_t pa0 = pack_bf16x2(p[0] * vscale, p[1] * vscale), pa2 = pack_bf16x2(p[2] * vscale, p[3] * vscale);
 
             // O += P V
             {
@@ -463,11 +519,12 @@ int num_sms() { return device_sm_count(); }
 // room for the items the kernel may create: one ragged item per group plus the balancing target
 int dense_max_items(const Geometry& g) { return g.batch * g.n_kv_heads + 2048; }
 
-size_t dense_smem_bytes(const Geometry& g)
+size_t dense_smem_bytes(const Geometry& g, bool fp8 = false)
 {
     const size_t n_groups = (size_t)g.batch * g.n_kv_heads;
-    const size_t ring = g.head_dim == 64 ? DenseCfg<64>::kRingBytes
-                                         : (g.head_dim == 256 ? DenseCfg<256>::kRingBytes : DenseCfg<128>::kRingBytes);
+    const size_t ring = fp8 ? DenseCfg<128, true>::kRingBytes
+                            : g.head_dim == 64 ? DenseCfg<64>::kRingBytes
+                                               : (g.head_dim == 256 ? DenseCfg<256>::kRingBytes : DenseCfg<128>::kRingBytes);
     return ring + (n_groups + 1) * 4 + 16 * 4 + (n_groups + 15) / 16 * 16;
 }
 
@@ -493,28 +550,33 @@ size_t dense_workspace_bytes(const Geometry& g_in)
     return dense_counter_bytes(g) + (size_t)dense_max_items(g) * g.group * (2 + g.head_dim) * sizeof(float);
 }
 
-template <int G, int D>
+template <int G, int D, bool FP8 = false>
 static cudaError_t launch_dense_gd(const Geometry& g, const uint16_t* q, const uint16_t* k, const uint16_t* v,
                                    const int32_t* block_table, const int32_t* seq_lens, const int32_t* fallback_list,
                                    const int32_t* fallback_count, float epsilon, float* partials, int32_t* counters,
-                                   float* out, vsa_diag_t* diag, cudaStream_t stream)
+                                   float* out, vsa_diag_t* diag, cudaStream_t stream, const float* k_scale = nullptr,
+                                   const float* v_scale = nullptr)
 {
-    const size_t smem = dense_smem_bytes(g);
+    const size_t smem = dense_smem_bytes(g, FP8);
     static bool attr_done[kMaxDevices] = {};   // per template instance
-    const cudaError_t e = allow_large_dynamic_smem(dense_split_kernel<G, D>, attr_done);
+    const cudaError_t e = allow_large_dynamic_smem(dense_split_kernel<G, D, FP8>, attr_done);
     if (e != cudaSuccess) return e;
     // persistent grid: one block per SM (the ring fills the shared memory)
-    return launch_pdl(dense_split_kernel<G, D>, dim3((unsigned)num_sms()), dim3(DenseCfg<D>::kDenseThreads), smem,
+    return launch_pdl(dense_split_kernel<G, D, FP8>, dim3((unsigned)num_sms()), dim3(DenseCfg<D>::kDenseThreads), smem,
                       stream, g, q, k, v, block_table, seq_lens, fallback_list, fallback_count, epsilon, partials,
-                      counters, out, diag, dense_max_items(g));
+                      counters, out, diag, dense_max_items(g), k_scale, v_scale);
 }
 
 template <int G>
 static cudaError_t launch_dense_g(const Geometry& g, const uint16_t* q, const uint16_t* k, const uint16_t* v,
                                   const int32_t* block_table, const int32_t* seq_lens, const int32_t* fallback_list,
                                   const int32_t* fallback_count, float epsilon, float* partials, int32_t* counters,
-                                  float* out, vsa_diag_t* diag, cudaStream_t stream)
+                                  float* out, vsa_diag_t* diag, cudaStream_t stream, const float* k_scale,
+                                  const float* v_scale)
 {
+    if (k_scale)
+        return launch_dense_gd<G, 128, true>(g, q, k, v, block_table, seq_lens, fallback_list, fallback_count, epsilon,
+                                             partials, counters, out, diag, stream, k_scale, v_scale);
     if (g.head_dim == 64)
         return launch_dense_gd<G, 64>(g, q, k, v, block_table, seq_lens, fallback_list, fallback_count, epsilon,
                                       partials, counters, out, diag, stream);
@@ -528,8 +590,9 @@ static cudaError_t launch_dense_g(const Geometry& g, const uint16_t* q, const ui
 cudaError_t launch_dense(const Geometry& g_in, const void* q, const void* k_cache, const void* v_cache,
                          const int32_t* block_table, const int32_t* seq_lens, const int32_t* fallback_list,
                          const int32_t* fallback_count, float epsilon, float* out, vsa_diag_t* diag, void* ws,
-                         cudaStream_t stream, bool tickets_cleared)
+                         cudaStream_t stream, bool tickets_cleared, const float* k_scale, const float* v_scale)
 {
+    if ((k_scale || v_scale) && (!k_scale || !v_scale || g_in.head_dim != kHeadDim)) return cudaErrorInvalidValue;
     const Geometry g = with_virtual_kv_heads(g_in);
     int32_t* counters = (int32_t*)ws;
     float* partials = (float*)((char*)ws + dense_counter_bytes(g));
@@ -539,10 +602,10 @@ cudaError_t launch_dense(const Geometry& g_in, const void* q, const void* k_cach
     }
     const uint16_t *qq = (const uint16_t*)q, *kk = (const uint16_t*)k_cache, *vv = (const uint16_t*)v_cache;
     switch (g.group) {
-        case 1: return launch_dense_g<1>(g, qq, kk, vv, block_table, seq_lens, fallback_list, fallback_count, epsilon, partials, counters, out, diag, stream);
-        case 2: return launch_dense_g<2>(g, qq, kk, vv, block_table, seq_lens, fallback_list, fallback_count, epsilon, partials, counters, out, diag, stream);
-        case 4: return launch_dense_g<4>(g, qq, kk, vv, block_table, seq_lens, fallback_list, fallback_count, epsilon, partials, counters, out, diag, stream);
-        case 8: return launch_dense_g<8>(g, qq, kk, vv, block_table, seq_lens, fallback_list, fallback_count, epsilon, partials, counters, out, diag, stream);
+        case 1: return launch_dense_g<1>(g, qq, kk, vv, block_table, seq_lens, fallback_list, fallback_count, epsilon, partials, counters, out, diag, stream, k_scale, v_scale);
+        case 2: return launch_dense_g<2>(g, qq, kk, vv, block_table, seq_lens, fallback_list, fallback_count, epsilon, partials, counters, out, diag, stream, k_scale, v_scale);
+        case 4: return launch_dense_g<4>(g, qq, kk, vv, block_table, seq_lens, fallback_list, fallback_count, epsilon, partials, counters, out, diag, stream, k_scale, v_scale);
+        case 8: return launch_dense_g<8>(g, qq, kk, vv, block_table, seq_lens, fallback_list, fallback_count, epsilon, partials, counters, out, diag, stream, k_scale, v_scale);
         default: return cudaErrorInvalidValue;
     }
 }

@@ -66,7 +66,7 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
                           vsa_diag_t* diag, int32_t* fallback_list, int32_t* fallback_count, cudaStream_t stream,
                           int solver_iters, vsa_solve_t* solve, const float* rad_logical, vsa_cert_t* cert,
                           int solver_kind, const int32_t* unit_list, const int32_t* unit_count, int routed_stride,
-                          const void* tl_summaries, int P_super)
+                          const void* tl_summaries, int P_super, const float* k_scale, const float* v_scale)
 {
     SparseArgs a;
     a.g = g;
@@ -83,6 +83,8 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
                                tl_summaries ? P_super : 0);
     a.tl_summaries = (const uint16_t*)tl_summaries;
     a.P_super = P_super;
+    a.k_scale = k_scale;
+    a.v_scale = v_scale;
     a.solver_iters = solver_iters;
     a.solver_kind = solver_kind;
     a.solve = solve;
@@ -107,6 +109,10 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
     a.fallback_list = fallback_list;
     a.fallback_count = fallback_count;
     a.stream = stream;
+    if (k_scale || v_scale) {   // fp8 cache
+        if (!k_scale || !v_scale || solve || cert || tl_summaries || g.head_dim != kHeadDim) return cudaErrorInvalidValue;
+        return launch_sparse_plain_fp8(a, threads);
+    }
     if (g.head_dim != kHeadDim) {
         if (solve || cert || tl_summaries) return cudaErrorInvalidValue;   // (refused by the entry points)
         return g.head_dim == 64 ? launch_sparse_plain_d64(a, threads) : launch_sparse_plain_d256(a, threads);

@@ -131,7 +131,11 @@ __device__ __forceinline__ void write_failed_unit(float* out, vsa_diag_t* diag, 
 //   elements 8c .. 8c+7 and, at D = 256, 128 + 8c .. 128 + 8c + 7 as well (its partial is the sum of the two
 //   pieces' partials: the first level of the 32-partial tree); at D = 64 only lanes 0 .. 7 hold data, the
 //   others contribute +0.  Iterative solves, certificate and the two-level front end exist at D = 128 only.
-template <int THREADS, int PAGE_KPT, int TOK_KPT, int SOLVE = 0, bool CERT = false, int D = kHeadDim>
+// FP8: k_cache / v_cache hold e4m3 bytes, value = byte * scale with one scale per (pool page, KV head) in
+//   k_scale / v_scale (fp32 [pool pages][n_kv_heads]); strides are in elements (= bytes).  The decoded bytes go
+//   through the same fixed-order dot and the score is multiplied by the scale afterwards; with power-of-two
+//   scales that is exact and every discrete result equals that of a bf16 cache holding the same values.  Closed-form family, D = 128.
+template <int THREADS, int PAGE_KPT, int TOK_KPT, int SOLVE = 0, bool CERT = false, int D = kHeadDim, bool FP8 = false>
 __global__ void __launch_bounds__(THREADS, 512 / THREADS)
 sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t* __restrict__ k_cache,
                      const uint16_t* __restrict__ v_cache, const int32_t* __restrict__ block_table,
@@ -142,11 +146,13 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                      const float* __restrict__ rad_logical, vsa_cert_t* __restrict__ cert,
                      const int32_t* __restrict__ unit_list, const int32_t* __restrict__ unit_count,
                      int routed_stride,
-                     const uint16_t* __restrict__ tl_summaries, int P_super)
+                     const uint16_t* __restrict__ tl_summaries, int P_super,
+                     const float* __restrict__ k_scale, const float* __restrict__ v_scale)
 {
     constexpr int WARPS = THREADS / 32, GROUPS = 2 * WARPS;
     static_assert(PAGE_KPT != -2 || (SOLVE == 0 && !CERT), "two-level front end: plain family only");
     static_assert(D == 128 || ((D == 64 || D == 256) && SOLVE == 0 && !CERT && PAGE_KPT != -2), "other head dimensions: plain family");
+    static_assert(!FP8 || (D == 128 && SOLVE == 0 && !CERT && PAGE_KPT != -2), "fp8 cache: closed-form family, D = 128");
     constexpr int PIECES = D == 256 ? 2 : 1;
     static_assert(SOLVE == 0 || THREADS == 256, "the solve maps one candidate to each of 256 lanes");
     static_assert(!CERT || PAGE_KPT > 0, "the certificate needs every page score of the unit in registers");
@@ -399,6 +405,27 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         const int slot = pp * 2 + gi;
         const bool active = slot < nt;
         float vals[16];
+        float kscale = 1.0f;
+        if constexpr (FP8) {
+            uint2 rows[16];
+            if (active) {
+                const uint8_t* src = reinterpret_cast<const uint8_t*>(k_cache) + (long long)page_phys[slot] * geo.page_stride +
+                                     (long long)g * geo.head_stride + c * 8 +
+                                     (long long)((page_l[slot] & ((1 << tsh) - 1)) * 16) * geo.token_stride;
+                kscale = __ldg(k_scale + (long long)page_phys[slot] * geo.n_kv_heads + g);
+#pragma unroll
+                for (int t = 0; t < 16; ++t) rows[t] = ld_nc_8B(src + (long long)t * geo.token_stride);
+            } else {
+#pragma unroll
+                for (int t = 0; t < 16; ++t) rows[t] = make_uint2(0u, 0u);
+            }
+#pragma unroll
+            for (int t = 0; t < 16; ++t) {
+                float kf[8];
+                unpack8_e4m3(rows[t], kf);
+                vals[t] = chunk_partial(qf, kf);
+            }
+        } else {
 #pragma unroll
         for (int pc = 0; pc < PIECES; ++pc) {
             uint4 rows[16];
@@ -420,7 +447,9 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                 vals[t] = pc == 0 ? part : vals[t] + part;
             }
         }
-        const float s = reduce_scatter16(vals, c);   // lane c: score of token c of the page
+        }
+        float s = reduce_scatter16(vals, c);   // lane c: score of token c of the page
+        if constexpr (FP8) s = __fmul_rn(s, kscale);   // exact: a power of two
         if (active && page_l[slot] * 16 + c < T) sm.keys[slot * 16 + c] = float_to_key(s);
     }
     __syncthreads();
@@ -532,6 +561,8 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                                (long long)((page_l[i >> 4] & ((1 << tsh) - 1)) * 16 + (i & 15)) * geo.token_stride;
                 sm.wgt[pos] = exp2f((key_to_float(key[j]) - s1) * scale);
                 if constexpr (SOLVE != 0) sm.score[pos] = key_to_float(key[j]);
+                // fp8: the scale of the candidate's value row (the score array is free in the closed-form family)
+                if constexpr (FP8) sm.score[pos] = __ldg(v_scale + (long long)page_phys[i >> 4] * geo.n_kv_heads + g);
             }
         }
     }
@@ -813,6 +844,28 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
         for (int e = 0; e < 8; ++e) acc[pc][e] = 0.0f;
     const int gidx = warp * 2 + gi;
     constexpr int UNR = THREADS == 512 ? 8 : 16;   // 256 threads, K_c = 256: every half-warp's rows in one batch
+    if constexpr (FP8) {
+        const uint8_t* vbase = reinterpret_cast<const uint8_t*>(v_cache) + (long long)g * geo.head_stride + c * 8;
+        for (int j0 = gidx; j0 < ns; j0 += GROUPS * UNR) {
+            uint2 rows[UNR];
+            float w[UNR], ws[UNR];
+#pragma unroll
+            for (int u = 0; u < UNR; ++u) {
+                const int j = j0 + u * GROUPS, jc = min(j, ns - 1);
+                rows[u] = ld_nc_8B(vbase + sm.voff[jc]);
+                w[u] = j < ns ? sm.wgt[jc] : 0.0f;
+                ws[u] = w[u] * sm.score[jc];   // weight times the row's power-of-two scale
+            }
+#pragma unroll
+            for (int u = 0; u < UNR; ++u) {
+                float vf[8];
+                unpack8_e4m3(rows[u], vf);
+#pragma unroll
+                for (int e = 0; e < 8; e += 2) fma2(acc[0][e], acc[0][e + 1], ws[u], ws[u], vf[e], vf[e + 1]);
+                z += w[u];
+            }
+        }
+    } else {
 #pragma unroll
     for (int pc = 0; pc < PIECES; ++pc) {
         const uint16_t* vbase = v_cache + (long long)g * geo.head_stride + c * 8 + pc * 128;
@@ -836,6 +889,7 @@ sparse_decode_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_
                 if (pc == 0) z += w[u];
             }
         }
+    }
     }
 #pragma unroll
     for (int pc = 0; pc < PIECES; ++pc)
@@ -915,68 +969,69 @@ struct SparseArgs {
     int routed_stride;                       // row stride of routed_pages (>= P)
     const uint16_t* tl_summaries;            // non-null: two-level front end (page_scores = representative scores)
     int P_super;
+    const float *k_scale, *v_scale;          // non-null: fp8 cache (one scale per pool page and KV head)
     cudaStream_t stream;
 };
 
 
 namespace {
 
-template <int THREADS, int PAGE_KPT, int TOK_KPT, int SOLVE, bool CERT, int D = kHeadDim>
+template <int THREADS, int PAGE_KPT, int TOK_KPT, int SOLVE, bool CERT, int D = kHeadDim, bool FP8 = false>
 cudaError_t launch_variant(const SparseArgs& a)
 {
     static bool attr_done[kMaxDevices] = {};   // per template instance
     if (a.smem > 48 * 1024) {
         const cudaError_t e =
-            allow_large_dynamic_smem(sparse_decode_kernel<THREADS, PAGE_KPT, TOK_KPT, SOLVE, CERT, D>, attr_done);
+            allow_large_dynamic_smem(sparse_decode_kernel<THREADS, PAGE_KPT, TOK_KPT, SOLVE, CERT, D, FP8>, attr_done);
         if (e != cudaSuccess) return e;
     }
     const unsigned units = (unsigned)(a.g.batch * a.g.n_q_heads);
-    return launch_pdl(sparse_decode_kernel<THREADS, PAGE_KPT, TOK_KPT, SOLVE, CERT, D>, dim3(units), dim3(THREADS),
+    return launch_pdl(sparse_decode_kernel<THREADS, PAGE_KPT, TOK_KPT, SOLVE, CERT, D, FP8>, dim3(units), dim3(THREADS),
                       a.smem, a.stream, a.g, a.q, a.k, a.v, a.block_table, a.seq_lens, a.routed_pages, a.page_scores,
                       a.P, a.K_c, a.epsilon, a.gap_threshold, a.out, a.diag, a.fallback_list, a.fallback_count,
                       a.solver_iters, a.solve, a.rad_logical, a.cert, a.unit_list, a.unit_count, a.routed_stride,
-                      a.tl_summaries, a.P_super);
+                      a.tl_summaries, a.P_super, a.k_scale, a.v_scale);
 }
 
 // token-score registers per thread from the number of routed tokens
-template <int THREADS, int PAGE_KPT, int SOLVE, bool CERT, int D = kHeadDim>
+template <int THREADS, int PAGE_KPT, int SOLVE, bool CERT, int D = kHeadDim, bool FP8 = false>
 cudaError_t launch_tok(const SparseArgs& a)
 {
     const int N = a.P * a.g.page_size;
-    if (N <= 2 * THREADS) return launch_variant<THREADS, PAGE_KPT, 2, SOLVE, CERT, D>(a);
-    if (N <= 4 * THREADS) return launch_variant<THREADS, PAGE_KPT, 4, SOLVE, CERT, D>(a);
+    if (N <= 2 * THREADS) return launch_variant<THREADS, PAGE_KPT, 2, SOLVE, CERT, D, FP8>(a);
+    if (N <= 4 * THREADS) return launch_variant<THREADS, PAGE_KPT, 4, SOLVE, CERT, D, FP8>(a);
     if constexpr (THREADS <= 256)
-        return N <= 8 * THREADS ? launch_variant<THREADS, PAGE_KPT, 8, SOLVE, CERT, D>(a) : cudaErrorInvalidValue;
+        return N <= 8 * THREADS ? launch_variant<THREADS, PAGE_KPT, 8, SOLVE, CERT, D, FP8>(a) : cudaErrorInvalidValue;
     else
         return cudaErrorInvalidValue;   // 128 pages * 16 tokens = 4 * 512: never reached
 }
 
 // page-score registers per thread from the block-table width (CERT: register variants only)
-template <int THREADS, int SOLVE, bool CERT, int D = kHeadDim>
+template <int THREADS, int SOLVE, bool CERT, int D = kHeadDim, bool FP8 = false>
 cudaError_t launch_threads(const SparseArgs& a)
 {
     if constexpr (!CERT) {
-        if (!a.page_scores) return launch_tok<THREADS, 0, SOLVE, CERT, D>(a);
+        if (!a.page_scores) return launch_tok<THREADS, 0, SOLVE, CERT, D, FP8>(a);
     }
-    if (a.g.max_pages <= 8 * THREADS) return launch_tok<THREADS, 8, SOLVE, CERT, D>(a);
-    if (a.g.max_pages <= 16 * THREADS) return launch_tok<THREADS, 16, SOLVE, CERT, D>(a);
-    if (a.g.max_pages <= 32 * THREADS) return launch_tok<THREADS, 32, SOLVE, CERT, D>(a);
+    if (a.g.max_pages <= 8 * THREADS) return launch_tok<THREADS, 8, SOLVE, CERT, D, FP8>(a);
+    if (a.g.max_pages <= 16 * THREADS) return launch_tok<THREADS, 16, SOLVE, CERT, D, FP8>(a);
+    if (a.g.max_pages <= 32 * THREADS) return launch_tok<THREADS, 32, SOLVE, CERT, D, FP8>(a);
     if constexpr (!CERT)
-        return launch_tok<THREADS, -1, SOLVE, CERT, D>(a);
+        return launch_tok<THREADS, -1, SOLVE, CERT, D, FP8>(a);
     else
         return cudaErrorInvalidValue;   // (refused by the entry point before any launch)
 }
 
 // the 128-thread shape (P <= 64, the caller checks): routed pages given, or selected from scores held
 // in registers (max_pages <= 4096) or staged in shared memory (wider tables)
-template <int D = kHeadDim>
+template <int D = kHeadDim, bool FP8 = false>
 inline cudaError_t launch_threads_128(const SparseArgs& a)
 {
-    if (!a.page_scores) return launch_tok<128, 0, 0, false, D>(a);
-    if (a.g.max_pages <= 8 * 128) return launch_tok<128, 8, 0, false, D>(a);
-    if (a.g.max_pages <= 16 * 128) return launch_tok<128, 16, 0, false, D>(a);
-    if (a.g.max_pages <= 32 * 128) return launch_tok<128, 32, 0, false, D>(a);
-    return launch_tok<128, -1, 0, false, D>(a);   // wider tables: selection staged in shared memory
+    if (!a.page_scores) return launch_tok<128, 0, 0, false, D, FP8>(a);
+    if (a.g.max_pages <= 8 * 128) return launch_tok<128, 8, 0, false, D, FP8>(a);
+    if (a.g.max_pages <= 16 * 128) return launch_tok<128, 16, 0, false, D, FP8>(a);
+    if (a.g.max_pages <= 32 * 128) return launch_tok<128, 32, 0, false, D, FP8>(a);
+    return launch_tok<128, -1, 0, false, D, FP8>(a);   // wider tables: selection staged in shared memory
 }
 
 }  // namespace
@@ -985,6 +1040,7 @@ inline cudaError_t launch_threads_128(const SparseArgs& a)
 cudaError_t launch_sparse_plain(const SparseArgs& a, int threads);   // closed-form weights
 cudaError_t launch_sparse_plain_d64(const SparseArgs& a, int threads);    // the same at head dimension 64
 cudaError_t launch_sparse_plain_d256(const SparseArgs& a, int threads);   // and 256
+cudaError_t launch_sparse_plain_fp8(const SparseArgs& a, int threads);    // closed-form weights on an fp8 cache
 cudaError_t launch_sparse_solve(const SparseArgs& a);                // iterative solves (256 threads)
 cudaError_t launch_sparse_cert(const SparseArgs& a, int threads);    // routing certificate
 cudaError_t launch_sparse_two_level(const SparseArgs& a, int threads);   // two-level front end

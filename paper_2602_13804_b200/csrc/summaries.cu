@@ -97,6 +97,61 @@ __global__ void __launch_bounds__(256) summaries_kernel(Geometry geo, const uint
     *reinterpret_cast<uint4*>(summaries + (p * geo.n_kv_heads + g) * D + c * 8) = mean_of_rows<PS>(rows, n);
 }
 
+// The same for an fp8 cache (e4m3 bytes, value = byte * scale with one scale per page and KV head): the
+// decoded bytes are summed in fp32 in ascending token order, multiplied by the scale, divided by the number of
+// valid rows and rounded to bf16 - with power-of-two scales bit for bit the summary of the bf16 cache that
+// holds the same values.
+// One thread per (logical page, kv head, 8-byte slice); head dimension 128.
+template <int PS>
+__global__ void __launch_bounds__(256) summaries_fp8_kernel(Geometry geo, const uint8_t* __restrict__ k_cache,
+                                                            const float* __restrict__ k_scale,
+                                                            const int32_t* __restrict__ block_table,
+                                                            const int32_t* __restrict__ seq_lens,
+                                                            const int32_t* __restrict__ first_page,
+                                                            uint16_t* __restrict__ summaries)
+{
+    const int b = blockIdx.y;
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const int c = (int)(idx & 15);
+    const int g = (int)((idx >> 4) % geo.n_kv_heads);
+    const long long l = (idx >> 4) / geo.n_kv_heads;
+    const int T = seq_lens[b];
+    if (T <= 0 || T > geo.max_pages * PS) return;
+    const int nb = (T + PS - 1) / PS;
+    const int l0 = first_page ? first_page[b] : 0;
+    if (l < l0 || l >= nb) return;
+    const long long p = block_table[(long long)b * geo.max_pages + l];
+    if (p < 0 || p >= geo.pool_pages) return;
+    const int n = min(PS, T - (int)l * PS);
+    const uint8_t* src = k_cache + p * geo.page_stride + (long long)g * geo.head_stride + c * 8;
+    uint2 rows[PS];
+#pragma unroll
+    for (int t = 0; t < PS; ++t)
+        if (t < n) rows[t] = ld_nc_8B(src + (long long)t * geo.token_stride);
+    float acc[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] = 0.0f;
+#pragma unroll
+    for (int t = 0; t < PS; ++t) {
+        if (t < n) {
+            float f[8];
+            unpack8_e4m3(rows[t], f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = acc[e] + f[e];
+        }
+    }
+    const float scale = k_scale[p * geo.n_kv_heads + g], fn = (float)n;
+    uint32_t h[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) h[e] = bf16_bits_rne(__fdiv_rn(__fmul_rn(acc[e], scale), fn));
+    uint4 o;
+    o.x = h[0] | (h[1] << 16);
+    o.y = h[2] | (h[3] << 16);
+    o.z = h[4] | (h[5] << 16);
+    o.w = h[6] | (h[7] << 16);
+    *reinterpret_cast<uint4*>(summaries + (p * geo.n_kv_heads + g) * kHeadDim + c * 8) = o;
+}
+
 // Radius of each page around its stored summary (the ball bound of the routing certificate):
 //   rhat = 1.001 * sqrt(max_t |k_t - mu|^2) + 2^-12 * |mu|,
 // squared norms summed in the library's canonical order, every operation a single rounded fp32
@@ -210,6 +265,18 @@ cudaError_t launch_build_summaries(const Geometry& g, const void* k_cache, const
     if (g.head_dim == 64) kernel = g.page_size == 32 ? summaries_kernel<32, 64> : summaries_kernel<16, 64>;
     if (g.head_dim == 256) kernel = g.page_size == 32 ? summaries_kernel<32, 256> : summaries_kernel<16, 256>;
     kernel<<<grid, 256, 0, stream>>>(g, (const uint16_t*)k_cache, block_table, seq_lens, first_page,
+                                     (uint16_t*)summaries);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_build_summaries_fp8(const Geometry& g, const void* k_cache, const float* k_scale,
+                                       const int32_t* block_table, const int32_t* seq_lens,
+                                       const int32_t* first_page, void* summaries, cudaStream_t stream)
+{
+    const long long threads = (long long)g.max_pages * g.n_kv_heads * 16;
+    dim3 grid((unsigned)((threads + 255) / 256), (unsigned)g.batch);
+    auto* kernel = g.page_size == 32 ? summaries_fp8_kernel<32> : summaries_fp8_kernel<16>;
+    kernel<<<grid, 256, 0, stream>>>(g, (const uint8_t*)k_cache, k_scale, block_table, seq_lens, first_page,
                                      (uint16_t*)summaries);
     return cudaGetLastError();
 }

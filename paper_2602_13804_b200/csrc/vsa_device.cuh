@@ -35,6 +35,45 @@ __device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8])
     f[7] = __uint_as_float(v.w & 0xffff0000u);
 }
 
+// ---- fp8 (e4m3) -----------------------------------------------------------------------------
+// An 8-byte vector holds 8 consecutive e4m3 values, element 0 in the low byte of .x.  The conversion is
+// exact (every e4m3 value is an fp16 value).  A cache stores value = byte * scale with one fp32 scale per
+// (pool page, KV head); multiplying by a power-of-two scale is exact.
+__device__ __forceinline__ void unpack8_e4m3(const uint2& v, float (&f)[8])
+{
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const unsigned short pair = (unsigned short)(((i < 2) ? v.x : v.y) >> (16 * (i & 1)));
+        unsigned int h2;
+        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(pair));
+        asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tcvt.f32.f16 %0, lo;\n\tcvt.f32.f16 %1, hi;\n\t}"
+            : "=f"(f[2 * i]), "=f"(f[2 * i + 1])
+            : "r"(h2));
+    }
+}
+
+// Four e4m3 bytes of a 32-bit word -> two packed bf16 pairs (bytes 0, 1 -> lo; bytes 2, 3 -> hi) with integer
+// operations and one packed multiply (the conversion instructions run at a fraction of that rate): the seven
+// exponent and mantissa bits of a byte, placed at the top of a bf16's exponent and mantissa fields, read as
+// 2^(e - 127) (1 + m / 8) - or, for e = 0, as the bf16 subnormal (m / 8) 2^-126 - and the product with 2^120
+// is the e4m3 value in both cases, exactly.
+__device__ __forceinline__ void e4m3x4_to_bf16x2x2(uint32_t w, uint32_t& lo, uint32_t& hi)
+{
+    const uint32_t a = __byte_perm(w, 0u, 0x4140), b = __byte_perm(w, 0u, 0x4342);   // 0x00b1'00b0, 0x00b3'00b2
+    const uint32_t xa = ((a << 8) & 0x80008000u) | ((a << 4) & 0x07f007f0u);
+    const uint32_t xb = ((b << 8) & 0x80008000u) | ((b << 4) & 0x07f007f0u);
+    const uint32_t two120 = 0x7b807b80u;   // bf16 2^120, twice
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(lo) : "r"(xa), "r"(two120));
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(hi) : "r"(xb), "r"(two120));
+}
+
+__device__ __forceinline__ uint2 ld_nc_8B(const void* p)
+{
+    uint2 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+    return v;
+}
+
 // round-to-nearest-even fp32 -> bf16 bits (finite inputs)
 __device__ __forceinline__ uint32_t bf16_bits_rne(float f)
 {

@@ -110,6 +110,10 @@ cudaError_t launch_build_summaries(const Geometry& g, const void* k_cache, const
                                    const int32_t* seq_lens, const int32_t* first_page, void* summaries,
                                    cudaStream_t stream);
 
+cudaError_t launch_build_summaries_fp8(const Geometry& g, const void* k_cache, const float* k_scale,
+                                       const int32_t* block_table, const int32_t* seq_lens,
+                                       const int32_t* first_page, void* summaries, cudaStream_t stream);
+
 cudaError_t launch_build_radii(const Geometry& g, const void* k_cache, const void* summaries,
                                const int32_t* block_table, const int32_t* seq_lens, const int32_t* first_page,
                                float* radii, cudaStream_t stream);
@@ -160,7 +164,10 @@ cudaError_t launch_sparse(const Geometry& g, const void* q, const void* k_cache,
                           int solver_iters = 0, vsa_solve_t* solve = nullptr, const float* rad_logical = nullptr,
                           vsa_cert_t* cert = nullptr, int solver_kind = 1, const int32_t* unit_list = nullptr,
                           const int32_t* unit_count = nullptr, int routed_stride = 0,
-                          const void* tl_summaries = nullptr, int P_super = 0);
+                          const void* tl_summaries = nullptr, int P_super = 0, const float* k_scale = nullptr,
+                          const float* v_scale = nullptr);
+// k_scale / v_scale != nullptr: k_cache / v_cache hold e4m3 bytes, value = byte * scale[pool page][KV head]
+// (closed-form family, head dimension 128).
 // tl_summaries != nullptr: the two-level front end - page_scores then holds the scores of the super-pages'
 // representatives, fp32 [batch][n_q_heads][two_level_max_supers], and the kernel keeps the P_super best
 // super-pages, scores their pages from tl_summaries and routes the best P of those.
@@ -197,7 +204,8 @@ size_t dense_workspace_bytes(const Geometry& g);
 cudaError_t launch_dense(const Geometry& g, const void* q, const void* k_cache, const void* v_cache,
                          const int32_t* block_table, const int32_t* seq_lens, const int32_t* fallback_list,
                          const int32_t* fallback_count, float epsilon, float* out, vsa_diag_t* diag, void* ws,
-                         cudaStream_t stream, bool tickets_cleared = false);
+                         cudaStream_t stream, bool tickets_cleared = false, const float* k_scale = nullptr,
+                         const float* v_scale = nullptr);
 // the per-(sequence, KV head) tickets at the start of the dense workspace, and how many there are
 int32_t* dense_tickets(void* ws_dense);
 int dense_ticket_count(const Geometry& g);
