@@ -69,6 +69,9 @@ def parse_args(argv=None):
     ap.add_argument("--two-level", type=int, default=None, metavar="P_SUPER",
                     help="time vsa_decode_step_two_level: only the pages of the P_SUPER best super-pages (16 pages "
                          "each, scored through one representative summary) are scored per unit")
+    ap.add_argument("--fp8", action="store_true",
+                    help="time vsa_decode_step_fp8 on an e4m3 copy of the workload's caches against vsa_decode_step on the "
+                         "bf16 caches that hold the same values, and print that comparison as one JSON line")
     ap.add_argument("--group-shared", action="store_true",
                     help="time vsa_decode_step_group_shared: the heads of a GQA group route as one query (one page "
                          "set and one candidate set per KV head)")
@@ -1061,6 +1064,12 @@ def main():
     args = parse_args()
     if args.leak_curve:
         return run_leak_curve(args)
+    if args.fp8:
+        import torch
+        dev = torch.device("cuda", 0)
+        torch.cuda.set_device(dev)
+        print(json.dumps(fp8_point(workload_spec(args.workload, args.layers), dev, args.steps)))
+        return
     if args.impl == "reference" and "WORLD_SIZE" not in os.environ:
         return run_reference(args)           # one process: the oracle runs on this host's cores
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:

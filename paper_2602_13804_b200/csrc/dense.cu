@@ -16,6 +16,8 @@
 // the block that finishes the last item of a (sequence, KV head) combines its partials.
 #include <math.h>
 
+#include <cuda_fp8.h>
+
 #include "vsa_device.cuh"
 #include "vsa_launch.h"
 
@@ -32,17 +34,18 @@ constexpr int kMaxRoundsRagged = 8;
 // Sizes that depend on the head dimension D (64, 128 or 256).  The ring of a block holds three stages of a
 // K tile and a V tile per warp: 192 KB with eight warps at D = 128; D = 256 runs four warps per block so
 // that the same ring fits.
-// FP8 (D = 128): a stage holds the raw e4m3 tiles (2 KB each, plus the two scales); each warp converts the
-// stage it is about to use into one bf16 working pair of tiles behind its stages.
+// FP8 (D = 128): the unit of work is 32 tokens (two tiles); a stage holds their e4m3 rows as they are (4 KB of
+// K, 4 KB of V, the four scales) and the tensor cores consume them directly (m16n8k32 e4m3 MMAs).
 template <int D, bool FP8 = false>
 struct DenseCfg {
     static constexpr int kDenseThreads = D == 256 ? 128 : 256;
     static constexpr int kDenseWarps = kDenseThreads / 32;
     static constexpr int kRowBytes = 2 * D;
     static constexpr int kTileBytes = kTileRows * kRowBytes;   // K (or V) rows of one tile and KV head (4 KB at D = 128)
-    static constexpr int kRawTileBytes = kTileRows * D;        // the same rows as e4m3 bytes
-    static constexpr int kStageBytes = FP8 ? 2 * kRawTileBytes + 16 : 2 * kTileBytes;   // K tile + V tile (+ scales)
-    static constexpr int kWarpBytes = kStages * kStageBytes + (FP8 ? 2 * kTileBytes : 0);
+    static constexpr int kUnitRows = FP8 ? 32 : kTileRows;     // tokens per unit of work of a warp
+    static constexpr int kRawBytes = 32 * D;                   // FP8: K (or V) rows of a unit as e4m3 bytes
+    static constexpr int kStageBytes = FP8 ? 2 * kRawBytes + 16 : 2 * kTileBytes;   // K + V (+ scales)
+    static constexpr int kWarpBytes = kStages * kStageBytes;
     static constexpr int kRingBytes = kDenseWarps * kWarpBytes;
     static constexpr int kPartialFloats = 2 + D;               // per (item, head): max (log2 domain), sum, acc[D]
     static constexpr int kMinPagesPerItem = 2 * kDenseWarps;   // at least two pages per warp: one would expose the DRAM latency
@@ -80,6 +83,35 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a2
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a0), "r"(zero), "r"(a2), "r"(zero), "r"(b0), "r"(b1));
 }
+// D (16x8, fp32) += A (16x32, e4m3, row) * B (32x8, e4m3, col).  The (at most eight) heads occupy rows 0..7 of
+// A with the high e4m3 term of each operand value and rows 8..15 with the low term (a1, a3), so that one MMA
+// forms both partial products: d[0], d[1] (row g) and d[2], d[3] (row g + 8) are added by the caller.
+__device__ __forceinline__ void mma_e4m3(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.f32.e4m3.e4m3.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+                 "{%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// 16 x 16 bytes, transposed: lane (g = lane / 4, t = lane % 4) receives rows 4t .. 4t+3 of column g (first
+// register) and of column g + 8 (second); .x2 loads a second matrix (addresses from lanes 16 .. 31) into r2, r3
+__device__ __forceinline__ void ldmatrix_x2_trans_b8(uint32_t (&r)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m16n16.x2.trans.shared.b8 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+// x = hi + lo with hi, lo e4m3 (x of up to eight significant bits inside the e4m3 range splits exactly)
+__device__ __forceinline__ void split_e4m3x2(float x0, float x1, uint32_t& hi, uint32_t& lo)
+{
+    const __nv_fp8x2_storage_t h = __nv_cvt_float2_to_fp8x2(make_float2(x0, x1), __NV_SATFINITE, __NV_E4M3);
+    const __half2_raw hr = __nv_cvt_fp8x2_to_halfraw2(h, __NV_E4M3);
+    const float2 hf = __half22float2(*reinterpret_cast<const __half2*>(&hr));
+    const __nv_fp8x2_storage_t l = __nv_cvt_float2_to_fp8x2(make_float2(x0 - hf.x, x1 - hf.y), __NV_SATFINITE, __NV_E4M3);
+    hi = h;
+    lo = l;
+}
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 {
     uint32_t r;
@@ -108,6 +140,7 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
     constexpr int kDenseThreads = Cfg::kDenseThreads, kDenseWarps = Cfg::kDenseWarps, kRowBytes = Cfg::kRowBytes,
                   kTileBytes = Cfg::kTileBytes, kStageBytes = Cfg::kStageBytes, kRingBytes = Cfg::kRingBytes,
                   kPartialFloats = Cfg::kPartialFloats, kMinPagesPerItem = Cfg::kMinPagesPerItem, kHeadDim = D;
+    constexpr int kUnit = Cfg::kUnitRows;
     constexpr int KS = D / 16;    // 16-element steps of the Q K^T contraction = 16-column steps of P V
     constexpr int NT = D / 8;     // 8-column output tiles
     constexpr int CPR = D / 8;    // 16-byte chunks per row
@@ -147,7 +180,7 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
         if (!sm.group_mask[grp]) return 0;
         const int T = seq_lens[grp / geo.n_kv_heads];
         if (!geo.length_ok(T)) return 0;
-        return (T + kTileRows - 1) / kTileRows;
+        return (T + kUnit - 1) / kUnit;
     };
     {
         int pages = 0, groups = 0, longest = 0;
@@ -239,7 +272,7 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
         const uint32_t mask = sm.group_mask[grp];
         const int b = grp / geo.n_kv_heads, g = grp % geo.n_kv_heads;
         const int T = seq_lens[b];
-        const int nb = (T + kTileRows - 1) / kTileRows;   // tiles of the sequence
+        const int nb = (T + kUnit - 1) / kUnit;   // units (tiles of 16 tokens; fp8: pairs of tiles) of the sequence
         const int chunk = item - sm.item_base[grp];
         const int items_of_group = sm.item_base[grp + 1] - sm.item_base[grp];
         // the group's pages are split evenly over its items (whole multiples of the warp count)
@@ -250,7 +283,44 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
 
         // Q fragments of the group: bf16 pairs straight from memory, rows >= G are zero
         uint32_t qa0[KS], qa2[KS];
-        {
+        float q_unscale = 1.0f;
+        if constexpr (FP8) {
+            // q as e4m3 operands: scaled by a power of two into the top of the e4m3 range, split into hi + lo
+            // (qa0 / qa2 hold, per 32-column step, {hi, lo} of columns 4 quad .. + 3 and of 16 + the same)
+            const uint16_t* qrow = q + ((long long)b * geo.n_q_heads + g * G + (head < G ? head : 0)) * kHeadDim;
+            float qv[4][8];
+            float amax = 0.0f;
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+#pragma unroll
+                for (int part = 0; part < 2; ++part) {
+                    const uint2 raw = *reinterpret_cast<const uint2*>(qrow + ks * 32 + part * 16 + quad * 4);
+                    qv[ks][part * 4 + 0] = __uint_as_float(raw.x << 16);
+                    qv[ks][part * 4 + 1] = __uint_as_float(raw.x & 0xffff0000u);
+                    qv[ks][part * 4 + 2] = __uint_as_float(raw.y << 16);
+                    qv[ks][part * 4 + 3] = __uint_as_float(raw.y & 0xffff0000u);
+                }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(qv[ks][i]));
+            }
+            amax = fmaxf(amax, __shfl_xor_sync(kFullMask, amax, 1));
+            amax = fmaxf(amax, __shfl_xor_sync(kFullMask, amax, 2));
+            const int sq = amax > 0.0f ? 7 - ilogbf(amax) : 0;   // largest |q| of the head lands in [128, 256)
+            q_unscale = ldexpf(1.0f, -sq);
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+                uint32_t h01, l01, h23, l23, h45, l45, h67, l67;
+                split_e4m3x2(ldexpf(qv[ks][0], sq), ldexpf(qv[ks][1], sq), h01, l01);
+                split_e4m3x2(ldexpf(qv[ks][2], sq), ldexpf(qv[ks][3], sq), h23, l23);
+                split_e4m3x2(ldexpf(qv[ks][4], sq), ldexpf(qv[ks][5], sq), h45, l45);
+                split_e4m3x2(ldexpf(qv[ks][6], sq), ldexpf(qv[ks][7], sq), h67, l67);
+                const bool on = head < G;
+                qa0[2 * ks] = on ? (h01 | (h23 << 16)) : 0u;       // hi: columns 4 quad .. + 3
+                qa0[2 * ks + 1] = on ? (h45 | (h67 << 16)) : 0u;   // hi: columns 16 + 4 quad .. + 3
+                qa2[2 * ks] = on ? (l01 | (l23 << 16)) : 0u;       // lo, likewise
+                qa2[2 * ks + 1] = on ? (l45 | (l67 << 16)) : 0u;
+            }
+        } else {
             const uint16_t* qrow = q + ((long long)b * geo.n_q_heads + g * G + (head < G ? head : 0)) * kHeadDim;
 #pragma unroll
             for (int ks = 0; ks < KS; ++ks) {
@@ -270,35 +340,45 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
         // pages of this warp: first_page + warp, + 8, ...
         const int my_first = first_page + warp;
         const int my_count = my_first < end_page ? (end_page - my_first + kDenseWarps - 1) / kDenseWarps : 0;
-        auto issue = [&](int k) {   // k-th page of this warp into stage k % kStages
+        auto issue = [&](int k) {   // k-th unit of this warp into stage k % kStages
             const int pl = my_first + k * kDenseWarps;
+            const uint32_t dst = ring_addr + (uint32_t)((k % kStages) * kStageBytes);
+            if constexpr (FP8) {
+                // 32 rows of 128 bytes per cache: lane covers 16-byte chunk lane % 8 of rows lane / 8 + 4 i; the two
+                // halves of the unit are tiles 2 pl and 2 pl + 1 (one page, or two pages with their own scales)
+                const int ch = lane & 7, r0 = lane >> 3;
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    const int tile = 2 * pl + hf;
+                    const int rows_here = min(kTileRows, T - tile * kTileRows);   // <= 0: the half lies past the sequence
+                    long long phys = rows_here > 0 ? bt[tile >> geo.tile_shift] : -1;
+                    const bool page_ok = phys >= 0 && phys < geo.pool_pages;
+                    if (!page_ok) phys = 0;
+                    const int valid_rows = page_ok ? rows_here : 0;
+                    const long long off8 = phys * geo.page_stride + (long long)(g / geo.kv_div) * geo.head_stride + ch * 16 +
+                                           (long long)((tile & ((1 << geo.tile_shift) - 1)) * kTileRows) * geo.token_stride;
+                    const uint8_t* kp = reinterpret_cast<const uint8_t*>(k_cache) + off8;
+                    const uint8_t* vp = reinterpret_cast<const uint8_t*>(v_cache) + off8;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int r = r0 + 4 * i, row = hf * 16 + r;
+                        const uint32_t off = (uint32_t)(row * 128 + ((ch ^ (row & 7)) << 4));
+                        const bool ok = r < valid_rows;
+                        cp_async_16_zfill(dst + off, kp + (long long)r * geo.token_stride, ok);
+                        cp_async_16_zfill(dst + Cfg::kRawBytes + off, vp + (long long)r * geo.token_stride, ok);
+                    }
+                    if (lane < 2) {   // the half's two scales ride the same stage: [k0, k1, v0, v1]
+                        const float* sp = (lane == 0 ? k_scale : v_scale) + phys * geo.kv_heads_stored + g / geo.kv_div;
+                        cp_async_4(dst + 2 * Cfg::kRawBytes + 8 * lane + 4 * hf, sp);
+                    }
+                }
+            } else {
             long long phys = bt[pl >> geo.tile_shift];
             const bool page_ok = phys >= 0 && phys < geo.pool_pages;
             if (!page_ok) phys = 0;
             const int valid_rows = page_ok ? min(kTileRows, T - pl * kTileRows) : 0;
             const long long head_off = (long long)(g / geo.kv_div) * geo.head_stride + cp_chunk * 8 +
                                        (long long)((pl & ((1 << geo.tile_shift) - 1)) * kTileRows) * geo.token_stride;
-            const uint32_t dst = ring_addr + (uint32_t)((k % kStages) * kStageBytes);
-            if constexpr (FP8) {
-                // raw rows of 128 bytes: lane covers 16-byte chunk lane % 8 of rows lane / 8 + 4 i
-                const int ch = lane & 7, r0 = lane >> 3;
-                const long long off8 = phys * geo.page_stride + (long long)(g / geo.kv_div) * geo.head_stride + ch * 16 +
-                                       (long long)((pl & ((1 << geo.tile_shift) - 1)) * kTileRows) * geo.token_stride;
-                const uint8_t* kp = reinterpret_cast<const uint8_t*>(k_cache) + off8;
-                const uint8_t* vp = reinterpret_cast<const uint8_t*>(v_cache) + off8;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int r = r0 + 4 * i;
-                    const uint32_t off = (uint32_t)(r * 128 + ch * 16);
-                    const bool ok = r < valid_rows;
-                    cp_async_16_zfill(dst + off, kp + (long long)r * geo.token_stride, ok);
-                    cp_async_16_zfill(dst + Cfg::kRawTileBytes + off, vp + (long long)r * geo.token_stride, ok);
-                }
-                if (lane < 2) {   // the tile's two scales ride the same stage
-                    const float* sp = (lane == 0 ? k_scale : v_scale) + phys * geo.kv_heads_stored + g / geo.kv_div;
-                    cp_async_4(dst + 2 * Cfg::kRawTileBytes + 4 * lane, sp);
-                }
-            } else {
             const uint16_t* kp = k_cache + phys * geo.page_stride + head_off;
             const uint16_t* vp = v_cache + phys * geo.page_stride + head_off;
 #pragma unroll
@@ -321,6 +401,108 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
             cp_async_commit();
             cp_async_wait<kStages - 1>();
             __syncwarp();
+            if constexpr (FP8) {
+            const int pl = my_first + k * kDenseWarps;
+            const int valid = min(kUnit, T - pl * kUnit);   // > 0
+            {
+                // a page outside the pool: the group's listed heads fail
+                const long long ph0 = bt[(2 * pl) >> geo.tile_shift];
+                const long long ph1 = valid > kTileRows ? bt[(2 * pl + 1) >> geo.tile_shift] : ph0;
+                if (ph0 < 0 || ph0 >= geo.pool_pages || ph1 < 0 || ph1 >= geo.pool_pages) {
+                    if (lane == 0) sm.misc[13] = 1;   // (cleared at the end of the previous item)
+                    __syncwarp();
+                    continue;
+                }
+            }
+            const uint32_t kbase = ring_addr + (uint32_t)((k % kStages) * kStageBytes);
+            const uint32_t vbase = kbase + Cfg::kRawBytes;
+            const float* scales = reinterpret_cast<const float*>(my_ring + (k % kStages) * kStageBytes + 2 * Cfg::kRawBytes);
+            const float ks0 = scales[0], ks1 = scales[1], vs0 = scales[2], vs1 = scales[3];
+
+            // S = Q K^T for the 32 tokens of the unit (four 8-token column tiles), q = hi + lo
+            float sc4[4][4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) sc4[j][i] = 0.0f;
+            {
+                // ldmatrix.x4 on byte rows: matrix mi = lane / 8 is (tokens 8 (mi / 2) .. + 7) x (16-byte chunk 2 ks + mi % 2);
+                // a lane receives 4 consecutive columns of one token: the B fragment of an m16n8k32 MMA
+                const int mi = lane >> 3, rr = lane & 7;
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    const int tok = hf * 16 + (mi >> 1) * 8 + rr;
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) {
+                        const int ch = 2 * ks + (mi & 1);
+                        uint32_t r[4];
+                        ldmatrix_x4(r, kbase + (uint32_t)(tok * 128 + ((ch ^ (tok & 7)) << 4)));
+                        mma_e4m3(sc4[2 * hf], qa0[2 * ks], qa2[2 * ks], qa0[2 * ks + 1], qa2[2 * ks + 1], r[0], r[1]);
+                        mma_e4m3(sc4[2 * hf + 1], qa0[2 * ks], qa2[2 * ks], qa0[2 * ks + 1], qa2[2 * ks + 1], r[2], r[3]);
+                    }
+                }
+            }
+            // this lane: head `head`, tokens 8 j + 2 quad, + 1 of column tile j = 0 .. 3
+            float t[8];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float ts = scale * q_unscale * (j < 2 ? ks0 : ks1);   // the page's key scale folded in
+                t[2 * j] = (8 * j + 2 * quad < valid) ? (sc4[j][0] + sc4[j][2]) * ts : -INFINITY;   // hi + lo rows
+                t[2 * j + 1] = (8 * j + 2 * quad + 1 < valid) ? (sc4[j][1] + sc4[j][3]) * ts : -INFINITY;
+            }
+            float pm = fmaxf(fmaxf(fmaxf(t[0], t[1]), fmaxf(t[2], t[3])), fmaxf(fmaxf(t[4], t[5]), fmaxf(t[6], t[7])));
+            pm = fmaxf(pm, __shfl_xor_sync(kFullMask, pm, 1));
+            pm = fmaxf(pm, __shfl_xor_sync(kFullMask, pm, 2));
+            const float m_new = fmaxf(m_run, pm);       // finite: token 0 of a unit is always valid
+            const float corr = exp2f(m_run - m_new);    // 0 on the first unit
+            float p[8], psum = 0.0f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                p[i] = exp2f(t[i] - m_new);
+                psum += p[i];
+            }
+            l_run = fmaf(l_run, corr, psum);
+            if (__any_sync(kFullMask, m_new > m_run)) {
+#pragma unroll
+                for (int n = 0; n < NT; ++n) {
+                    o[n][0] *= corr;
+                    o[n][1] *= corr;
+                }
+            }
+            m_run = m_new;
+            // P as e4m3 operands: p * (value scale of its page / the larger of the two scales) * 2^8 = hi + lo.
+            // The 8 tokens of this lane take the lane's 8 slots of the contraction index: slots 4 quad .. + 3 are
+            // tokens 2 quad, 2 quad + 1, 8 + 2 quad, 9 + 2 quad, slots 16 + 4 quad .. + 3 the same + 16; the V rows
+            // are fetched in the matching order below.
+            const float vref = fmaxf(vs0, vs1);
+            const float w0 = vref > 0.0f ? 256.0f * (vs0 / vref) : 0.0f, w1 = vref > 0.0f ? 256.0f * (vs1 / vref) : 0.0f;
+            uint32_t h01, l01, h23, l23, h45, l45, h67, l67;
+            split_e4m3x2(p[0] * w0, p[1] * w0, h01, l01);
+            split_e4m3x2(p[2] * w0, p[3] * w0, h23, l23);
+            split_e4m3x2(p[4] * w1, p[5] * w1, h45, l45);
+            split_e4m3x2(p[6] * w1, p[7] * w1, h67, l67);
+            const uint32_t ph0 = h01 | (h23 << 16), ph2 = h45 | (h67 << 16), pl0 = l01 | (l23 << 16), pl2 = l45 | (l67 << 16);
+            const float oscale = vref * (1.0f / 256.0f);
+
+            // O += P V, 16 columns at a time: one transposing byte load per 32 tokens x 16 columns
+            {
+                const int rrow = lane & 15, qd = rrow >> 2, ii = rrow & 3;
+                const int tokp = (lane >> 4) * 16 + ((ii < 2) ? 0 : 8) + 2 * qd + (ii & 1);
+                const uint32_t vrow = vbase + (uint32_t)(tokp * 128);
+#pragma unroll
+                for (int dp = 0; dp < 8; ++dp) {
+                    uint32_t r[4];
+                    ldmatrix_x2_trans_b8(r, vrow + (uint32_t)((dp ^ (tokp & 7)) << 4));
+                    float ta[4] = {0.f, 0.f, 0.f, 0.f}, tb[4] = {0.f, 0.f, 0.f, 0.f};
+                    mma_e4m3(ta, ph0, pl0, ph2, pl2, r[0], r[2]);
+                    mma_e4m3(tb, ph0, pl0, ph2, pl2, r[1], r[3]);
+                    o[2 * dp][0] = fmaf(ta[0] + ta[2], oscale, o[2 * dp][0]);
+                    o[2 * dp][1] = fmaf(ta[1] + ta[3], oscale, o[2 * dp][1]);
+                    o[2 * dp + 1][0] = fmaf(tb[0] + tb[2], oscale, o[2 * dp + 1][0]);
+                    o[2 * dp + 1][1] = fmaf(tb[1] + tb[3], oscale, o[2 * dp + 1][1]);
+                }
+            }
+            } else {
             const int pl = my_first + k * kDenseWarps;
             const int valid = min(kTileRows, T - pl * kTileRows);   // > 0
             {
@@ -331,36 +513,8 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
                     continue;
                 }
             }
-            uint32_t kbase = ring_addr + (uint32_t)((k % kStages) * kStageBytes);
-            uint32_t vbase = kbase + kTileBytes;
-            float kscale = 1.0f, vscale = 1.0f;
-            if constexpr (FP8) {
-                // e4m3 -> bf16 (exact) into the warp's working pair of tiles, in the swizzled layout ldmatrix reads
-                const uint8_t* raw = my_ring + (k % kStages) * kStageBytes;
-                uint8_t* work = my_ring + kStages * kStageBytes;
-                kscale = *reinterpret_cast<const float*>(raw + 2 * Cfg::kRawTileBytes);
-                vscale = *reinterpret_cast<const float*>(raw + 2 * Cfg::kRawTileBytes + 4);
-                const int ch = lane & 7, r0 = lane >> 3;
-#pragma unroll
-                for (int kv = 0; kv < 2; ++kv) {
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int r = r0 + 4 * i;
-                        const uint4 in = *reinterpret_cast<const uint4*>(raw + kv * Cfg::kRawTileBytes + r * 128 + ch * 16);
-                        uint4 o0, o1;
-                        e4m3x4_to_bf16x2x2(in.x, o0.x, o0.y);
-                        e4m3x4_to_bf16x2x2(in.y, o0.z, o0.w);
-                        e4m3x4_to_bf16x2x2(in.z, o1.x, o1.y);
-                        e4m3x4_to_bf16x2x2(in.w, o1.z, o1.w);
-                        uint8_t* row = work + kv * kTileBytes + r * kRowBytes;
-                        *reinterpret_cast<uint4*>(row + (((2 * ch) ^ (r & 7)) << 4)) = o0;
-                        *reinterpret_cast<uint4*>(row + (((2 * ch + 1) ^ (r & 7)) << 4)) = o1;
-                    }
-                }
-                __syncwarp();
-                kbase = ring_addr + (uint32_t)(kStages * kStageBytes);
-                vbase = kbase + kTileBytes;
-            }
+            const uint32_t kbase = ring_addr + (uint32_t)((k % kStages) * kStageBytes);
+            const uint32_t vbase = kbase + kTileBytes;
 
             // S = Q K^T for the 16 tokens of the page (two 8-token column tiles)
             float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
@@ -376,7 +530,7 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
                 }
             }
             // this lane: head `head`, tokens 2 quad, 2 quad + 1 (tile 0) and 8 + the same (tile 1)
-            const float tscale = FP8 ? scale * kscale : scale;   // fp8: the page's key scale folded in
+            const float tscale = scale;
             float t[4];
             t[0] = (2 * quad < valid) ? s0[0] * tscale : -INFINITY;
             t[1] = (2 * quad + 1 < valid) ? s0[1] * tscale : -INFINITY;
@@ -399,8 +553,7 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
                 }
             }
             m_run = m_new;
-            // fp8: the page's value scale rides on the probabilities (the running sum keeps the unscaled ones)
-            const uint32_t pa0 = pack_bf16x2(p[0] * vscale, p[1] * vscale), pa2 = pack_bf16x2(p[2] * vscale, p[3] * vscale);
+            const uint32_t pa0 = pack_bf16x2(p[0], p[1]), pa2 = pack_bf16x2(p[2], p[3]);
 
             // O += P V
             {
@@ -413,6 +566,7 @@ dense_split_kernel(Geometry geo, const uint16_t* __restrict__ q, const uint16_t*
                     mma_bf16(o[2 * dp], pa0, pa2, r[0], r[1]);
                     mma_bf16(o[2 * dp + 1], pa0, pa2, r[2], r[3]);
                 }
+            }
             }
             __syncwarp();   // the stage is overwritten by a later issue
         }
