@@ -135,3 +135,28 @@ def test_entry_points_that_exist_at_128_only_refuse(d):
         with pytest.raises(B.VsaError) as e:
             call()
         assert e.value.code == -2   # VSA_ERR_UNSUPPORTED_SHAPE
+
+
+@pytest.mark.parametrize("d", DIMS)
+def test_host_buffer_step_and_workspace_free_routing(d):
+    import oracle
+    from gpu_runner import check_out
+    from paper_2602_13804_b200 import SparsePagedDecoder
+    from util import geometry, host_arrays
+    w = make_workload(spec(d, batch=2, seq_lens=(900, 640), needles=2, P=6, K_c=48), seed=780 + d)
+    wd = w.to(DEV)
+    shape = B.shape_of(wd.q, wd.k_cache, wd.block_table)
+    dec = SparsePagedDecoder(shape, 6, 48, w.epsilon, w.gap_threshold, device=DEV, host_io=True)
+    summ = dec.build_summaries(wd.k_cache, wd.block_table, wd.seq_lens)
+    out_dev = dec.step(wd.q, summ, wd.k_cache, wd.v_cache, wd.block_table, wd.seq_lens).clone()
+    out_host = dec.step_host(w.q.pin_memory(), summ, wd.k_cache, wd.v_cache, wd.block_table, wd.seq_lens)
+    torch.cuda.synchronize()
+    assert out_host.shape[-1] == d and torch.equal(out_host, out_dev.cpu())
+    q, K, V, bt, sl = host_arrays(w)
+    st = oracle.decode_step(geometry(w), q, K, V, bt, sl, 6, 48, w.epsilon, w.gap_threshold)
+    check_out(out_host.numpy(), st.out, "host step")
+    routed = torch.full((2, 8, 6), -7, dtype=torch.int32, device=DEV)
+    scores = torch.zeros((2, 8, 6), dtype=torch.float32, device=DEV)
+    B.vsa_route_pages_static(shape, wd.q, summ, wd.block_table, wd.seq_lens, 6, routed, scores)
+    torch.cuda.synchronize()
+    assert np.array_equal(routed.cpu().numpy(), st.route.pages) and np.array_equal(scores.cpu().numpy(), st.route.scores)
