@@ -1,8 +1,8 @@
 /*
  * vsa.h - C ABI of the sparse paged decode-attention step for NVIDIA B200 (sm_100a).
  *
- * One decode step, per (sequence b, query head h) "unit", over a paged bf16 KV cache
- * (paper Sec. 7, "Paged KV and routing", steps 1-4, and Sec. 10.3 fallback policy):
+ * One decode step, per (sequence b, query head h) "unit", over a paged bf16 KV cache (an e4m3 cache
+ * through the *_fp8 entry points) (paper Sec. 7, "Paged KV and routing", steps 1-4, and Sec. 10.3 fallback policy):
  *
  *   1. page routing   score one summary vector per page, keep the P best pages
  *   2. token routing  score every token of those pages, keep the K_c best tokens
